@@ -1,0 +1,212 @@
+/*
+ * splitbrain.h - C ABI of the B200 (sm_100a) hot path of SplitBrain hybrid data/model-parallel
+ * CNN training: one synchronous SGD iteration in which the 3x3 convolution stack runs
+ * data-parallel over R logical replicas of the minibatch and every fully-connected layer is
+ * split by output column into K logical model shards whose input is the gathered activations of
+ * all replicas.
+ *
+ * General conventions
+ *  - Memory: the caller owns every byte.  The library never allocates device memory; it carves
+ *    parameters, momentum, gradients, activations, scratch and status words out of one caller
+ *    supplied device arena (size from sb_model_bytes, 256-byte aligned).  Pointers returned by
+ *    sb_tensor are borrowed views into that arena and die with it.
+ *  - "device" / "host" is stated per pointer argument.  No torch types cross this boundary.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All calls
+ *    except sb_model_bytes/create/destroy, sb_loss, sb_tensor_read/write and sb_train_step_host
+ *    only enqueue work and return immediately.
+ *  - Errors: every call returns an sb_status; nothing throws, aborts or traps.  Argument and shape
+ *    errors are detected before any launch.  sb_last_error() gives a thread-local message.
+ *  - Layouts: images and conv activations NHWC; conv weights [Cout][3][3][Cin]; FC weights
+ *    [out][in] (shard j is the contiguous row block [c_j, c_{j+1}), c_j = floor(j*out/K)); the
+ *    flatten order at the conv -> FC boundary is (h, w, c).
+ *  - Precision modes: SB_FP32 keeps everything in float.  SB_BF16 stores activations,
+ *    activation gradients and the weight copies used by the contractions in bfloat16
+ *    (round-to-nearest-even), accumulates in float, and keeps master weights, momentum, weight
+ *    gradients, logits and the loss in float.
+ *
+ * Paper references are to "SplitBrain: Hybrid Data and Model Parallel Deep Learning"
+ * (arXiv 2112.15317) by section / paragraph / listing.
+ */
+#ifndef SPLITBRAIN_H
+#define SPLITBRAIN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sb_model sb_model; /* opaque; host object owned by the library */
+
+typedef enum {
+    SB_OK = 0,
+    SB_ERR_INVALID_ARG = 1,     /* null pointer, bad enum, misaligned pointer */
+    SB_ERR_SHAPE = 2,           /* layer list / sizes that do not form a valid network */
+    SB_ERR_UNSUPPORTED = 3,
+    SB_ERR_ARENA_TOO_SMALL = 4,
+    SB_ERR_CUDA = 5,            /* a CUDA runtime/driver call failed; see sb_last_error() */
+    SB_ERR_STATE = 6,           /* call order (e.g. backward before forward) */
+    SB_ERR_TIMEOUT = 7          /* a bounded device-side wait expired (status word set by a kernel) */
+} sb_status;
+
+typedef enum {
+    SB_CONV3X3_RELU = 1, /* 3x3 cross-correlation, stride 1, zero pad 1, + bias, ReLU */
+    SB_MAXPOOL2 = 2,     /* 2x2 max, stride 2 */
+    SB_FC_RELU = 3,      /* fully connected + bias + ReLU, column-sharded K ways */
+    SB_FC = 4,           /* fully connected + bias (the logits layer) */
+    SB_SOFTMAX_XENT = 5  /* log-softmax + negative log-likelihood, mean over the batch */
+} sb_layer_kind;
+
+typedef struct {
+    int32_t kind; /* sb_layer_kind */
+    int32_t out;  /* Cout / out-features / number of classes; ignored for SB_MAXPOOL2 */
+} sb_layer;
+
+enum { SB_FP32 = 0, SB_BF16 = 1 };
+
+/* sb_config.flags */
+enum {
+    SB_FLAG_INPUT_GRAD = 1,  /* also compute the gradient w.r.t. the network input (layer 0 dgrad) */
+    SB_FLAG_FORCE_SIMT = 2   /* use the CUDA-core kernels for every layer (cross-check / debugging) */
+};
+
+typedef struct {
+    int32_t H, W, C;            /* input image geometry */
+    int32_t batch_per_replica;  /* b: images per replica; the step's batch is B = R*b */
+    int32_t R;                  /* data-parallel replicas of the conv stack (1..64) */
+    int32_t K;                  /* model shards per FC layer (1..64, K <= every FC width) */
+    int32_t precision;          /* SB_FP32 or SB_BF16 */
+    int32_t flags;
+} sb_config;
+
+/* Tensor selectors for sb_tensor. */
+enum {
+    SB_T_WEIGHT = 0,   /* master weights, float.  conv: [Cout,3,3,Cin]; FC shard: [out_j,in] */
+    SB_T_BIAS = 1,     /* float [Cout] / [out_j] */
+    SB_T_GRAD_W = 2,   /* float, same shape as the weight */
+    SB_T_GRAD_B = 3,
+    SB_T_MOM_W = 4,    /* momentum, float */
+    SB_T_MOM_B = 5,
+    SB_T_ACT = 6,      /* layer output.  conv/pool: replica `part`'s [b,H,W,C]; FC: [B,out] (part
+                          ignored); activation dtype, except the logits layer which is float */
+    SB_T_DACT = 7,     /* gradient w.r.t. the layer's pre-activation output (conv, FC) or w.r.t. its
+                          output (pool); same shape/partitioning as SB_T_ACT; activation dtype */
+    SB_T_POOL_IDX = 8, /* uint8 argmax position (dh*2+dw) per pooled element, replica `part` */
+    SB_T_ROW_LOSS = 9, /* float [B]: per-row negative log-likelihood (layer = the loss layer) */
+    SB_T_INPUT_GRAD = 10, /* gradient w.r.t. replica `part`'s input (needs SB_FLAG_INPUT_GRAD) */
+    SB_T_SHADOW_W = 11 /* bf16 copy of the weight used by the contractions (SB_BF16 only) */
+};
+enum { SB_DT_F32 = 0, SB_DT_BF16 = 1, SB_DT_U8 = 2, SB_DT_I32 = 3 };
+
+/*
+ * Size of the device arena a model needs.  [Design: the model builder supplies a sequential
+ * layer list, the batch size and the MP group size.]
+ *   layers, cfg : host pointers.  arena_bytes : host pointer, receives the size.
+ * Validation (SB_ERR_SHAPE): conv/pool layers first, then FC layers, then exactly one loss
+ * whose class count equals the last FC width; H and W even at every pool; 1 <= R,K <= 64;
+ * K <= every FC width.
+ */
+sb_status sb_model_bytes(const sb_layer* layers, int32_t n_layers, const sb_config* cfg,
+                         size_t* arena_bytes);
+
+/*
+ * Build the partitioned network [Design, Layer Partitioning / Listing 1]: conv, pool and ReLU
+ * layers are replicated over the R replicas (one parameter copy, since the replicas are kept
+ * in sync every step); every FC layer is split into K column shards of 1/K size; the modulo
+ * layer (gather of the replicas' features) and the shard layers (concatenation of the column
+ * slices) exist only as the addressing of the FC kernels.
+ *   arena : DEVICE pointer, 256-byte aligned, arena_bytes long, zero-filled by this call.
+ *   out   : host pointer, receives the model handle.
+ * All parameters start at zero: load them with sb_tensor_write (then sb_refresh_shadow).
+ * Synchronises the device once (arena clear).
+ */
+sb_status sb_model_create(const sb_layer* layers, int32_t n_layers, const sb_config* cfg,
+                          void* arena, size_t arena_bytes, sb_model** out);
+
+sb_status sb_model_destroy(sb_model* m);
+
+/*
+ * Forward pass of one training iteration [Implementation: DP through the conv layers, MP
+ * through the FC layers; Modulo Layer and Shard Layer, fprop].
+ *   x      : HOST array of R DEVICE pointers; x[r] = replica r's images [b,H,W,C] in the
+ *            activation dtype (float or bfloat16), 16-byte aligned.
+ *   labels : HOST array of R DEVICE pointers; labels[r] = int32 [b], values in [0, classes).
+ * Row g = r*b + i of every FC-side tensor belongs to replica r (the paper's owner rule
+ * "batch example index divided by B/K").  Computes the per-row and mean loss and the gradient
+ * of the loss w.r.t. the logits.  The input buffers must stay valid until sb_backward has run.
+ */
+sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* labels, void* stream);
+
+/*
+ * Backward pass [Shard Layer and Modulo Layer, bprop; DP reduce]: FC weight/bias gradients per
+ * shard; input gradients summed over the K shards and routed back to the owning replica's rows;
+ * pooling and conv backward per replica; conv weight gradients summed over the R replicas.
+ * Requires a preceding sb_forward (SB_ERR_STATE otherwise).
+ */
+sb_status sb_backward(sb_model* m, void* stream);
+
+/*
+ * SGD with momentum on every parameter [Implementation: "SGD in mini-batches"]:
+ * v <- momentum*v + g ; w <- w - lr*v ; in SB_BF16 mode also refreshes the bf16 weight copies.
+ */
+sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream);
+
+/*
+ * Mean loss of the last sb_forward.  Synchronises `stream`, copies 4 bytes to host_loss (HOST),
+ * and checks the device status word: returns SB_ERR_TIMEOUT if any kernel gave up on a bounded
+ * wait since the last call.
+ */
+sb_status sb_loss(sb_model* m, void* stream, float* host_loss);
+
+/*
+ * One whole iteration from HOST buffers (forward, backward, SGD step, loss read-back): the
+ * end-to-end call.  host_x: [B,H,W,C] in the activation dtype, rows r*b..(r+1)*b-1 = replica r;
+ * host_labels: int32 [B].  Both are copied host->device on `stream` into staging space inside
+ * the arena (pinned host memory makes the copies asynchronous).  Synchronises `stream`.
+ */
+sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels,
+                             float lr, float momentum, void* stream, float* host_loss);
+
+/*
+ * Introspection for parity tests and checkpointing: a borrowed DEVICE pointer to one tensor.
+ *   what  : SB_T_*;  layer : index into the layer list;
+ *   part  : replica r for conv-side activations, shard j for FC parameters.
+ *   dev_ptr, shape (4 entries, unused = 1), dtype (SB_DT_*) : host pointers, any may be NULL.
+ */
+sb_status sb_tensor(sb_model* m, int32_t what, int32_t layer, int32_t part, void** dev_ptr,
+                    int64_t shape[4], int32_t* dtype);
+
+/* Blocking copies between a HOST buffer (dense, the tensor's dtype) and a tensor selected as in
+ * sb_tensor.  `bytes` must equal the tensor's size. */
+sb_status sb_tensor_read(sb_model* m, int32_t what, int32_t layer, int32_t part, void* host_dst, size_t bytes);
+sb_status sb_tensor_write(sb_model* m, int32_t what, int32_t layer, int32_t part, const void* host_src, size_t bytes);
+
+/* Rebuild the bf16 weight copies from the float master weights (after sb_tensor_write). */
+sb_status sb_refresh_shadow(sb_model* m, void* stream);
+
+/*
+ * Run a sub-range of layers only, on whatever the arena buffers currently hold ("teacher
+ * forcing" for per-layer parity tests and micro-benchmarks).  sb_forward_layers runs layers
+ * first..last in order; x/labels may be NULL unless layer 0 / the loss layer is in range.
+ * sb_backward_layers runs the backward of layers last..first (last >= first) in reverse order.
+ */
+sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void* const* x,
+                            const int32_t* const* labels, void* stream);
+sb_status sb_backward_layers(sb_model* m, int32_t last, int32_t first, void* stream);
+
+/*
+ * Parameter bytes (float master copies) one worker of an MP group of size K holds: all conv
+ * parameters plus shard `shard` of every FC layer [Evaluation: parameter-memory saving].
+ */
+sb_status sb_param_bytes(const sb_model* m, int32_t shard, size_t* bytes);
+
+/* Number of kernels the last sb_forward + sb_backward + sb_sgd_step enqueued (host counter). */
+sb_status sb_launch_count(const sb_model* m, int64_t* launches);
+
+const char* sb_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPLITBRAIN_H */

@@ -1,0 +1,706 @@
+// Host side of the C ABI (include/splitbrain.h): validation, the arena carve-up, the per-layer
+// launch plan for forward / backward / update, and tensor introspection.
+//
+// Partitioning as data layout (one GPU, R logical replicas, K logical shards):
+//  * every conv-side activation buffer is [B = R*b, H, W, C]; replica r owns the image rows
+//    [r*b, (r+1)*b).  The last conv-side buffer reinterpreted as [B, H*W*C] *is* the gathered
+//    input of the first FC layer (modulo layer, forward), and the FC input gradient written in
+//    the same buffer shape *is* the scatter back to the replicas (modulo layer, backward).
+//  * an FC weight is [out, in]; shard j is the row block [c_j, c_{j+1}), c_j = floor(j*out/K),
+//    and owns the output columns with the same indices (shard layer, forward = column concat by
+//    addressing).  The FC kernels take (shard_dim, K) and never let a tile straddle two shards.
+#include "../../include/splitbrain.h"
+#include "sb_internal.h"
+#include "sb_umma.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace sb;
+
+static thread_local char g_err[512] = "";
+static sb_status fail(sb_status s, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+extern "C" const char* sb_last_error(void) { return g_err; }
+
+#define CU_TRY(expr)                                                                             \
+    do {                                                                                         \
+        cudaError_t e_ = (expr);                                                                 \
+        if (e_ != cudaSuccess) return fail(SB_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+namespace {
+
+struct Layer {
+    int kind = 0, out = 0;
+    int H = 0, W = 0, Cin = 0, Cout = 0;  // conv: input H,W,Cin -> Cout ; pool: input H,W,C=Cin=Cout
+    int in_f = 0, out_f = 0;              // fc
+    bool relu = false;
+    size_t p_w = 0, p_b = 0, n_w = 0, n_b = 0;  // element offsets/counts in the parameter regions
+    size_t out_per_img = 0;                     // elements of the layer output per image (row)
+    char* act = nullptr;                        // [B, out_per_img] activation dtype (float for the logits layer)
+    char* dact = nullptr;                       // same shape, activation dtype
+    uint8_t* idx = nullptr;                     // pool argmax
+    int wg_splits = 1;                          // conv wgrad pixel-range splits
+    int act_dt = SB_DT_F32;
+    UmmaLayer um;                               // tensor-core plan of this layer (tcgen05 path)
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct sb_model {
+    sb_config cfg{};
+    std::vector<Layer> L;
+    bool bf16 = false;
+    int B = 0, first_fc = 0, n_layers = 0;
+    size_t in_per_img = 0, esz = 4;
+    char* arena = nullptr;
+    size_t arena_bytes = 0;
+    size_t P = 0;  // padded parameter element count
+    float *Wm = nullptr, *Vm = nullptr, *Gm = nullptr;
+    __nv_bfloat16* Sm = nullptr;
+    float* ws = nullptr;
+    size_t ws_floats = 0;
+    float *row_loss = nullptr, *loss = nullptr;
+    unsigned int* counter = nullptr;
+    uint32_t* status = nullptr;
+    char* stage_x = nullptr;
+    int32_t* stage_labels = nullptr;
+    char* input_grad = nullptr;
+    PtrTab x_tab{}, label_tab{};
+    bool have_x = false, have_labels = false, have_fwd = false;
+    int64_t launches = 0, last_step_launches = 0;
+};
+
+namespace {
+
+// Walks the layer list, fills shapes, and assigns arena offsets (relative to base, which may be
+// null for a pure size computation).  Returns SB_OK and the total size.
+sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m, char* base, size_t* total)
+{
+    if (!layers || !cfg || n <= 0) return fail(SB_ERR_INVALID_ARG, "null layers/config or empty layer list");
+    if (cfg->precision != SB_FP32 && cfg->precision != SB_BF16) return fail(SB_ERR_INVALID_ARG, "precision must be SB_FP32 or SB_BF16");
+    if (cfg->R < 1 || cfg->R > MAX_PARTS || cfg->K < 1 || cfg->K > MAX_PARTS) return fail(SB_ERR_SHAPE, "R and K must be in 1..%d", MAX_PARTS);
+    if (cfg->H < 1 || cfg->W < 1 || cfg->C < 1 || cfg->batch_per_replica < 1) return fail(SB_ERR_SHAPE, "H, W, C and batch_per_replica must be positive");
+    m->cfg = *cfg;
+    m->bf16 = cfg->precision == SB_BF16;
+    m->esz = m->bf16 ? 2 : 4;
+    m->B = cfg->R * cfg->batch_per_replica;
+    m->n_layers = n;
+    m->L.assign(n, Layer());
+    m->in_per_img = (size_t)cfg->H * cfg->W * cfg->C;
+    if ((m->in_per_img * m->esz) % 16 != 0) return fail(SB_ERR_SHAPE, "one input image must be a multiple of 16 bytes");
+    int H = cfg->H, W = cfg->W, C = cfg->C;
+    long feat = -1;
+    size_t P = 0;
+    int first_fc = -1;
+    for (int i = 0; i < n; ++i) {
+        Layer& l = m->L[i];
+        l.kind = layers[i].kind;
+        l.out = layers[i].out;
+        l.act_dt = m->bf16 ? SB_DT_BF16 : SB_DT_F32;
+        switch (l.kind) {
+        case SB_CONV3X3_RELU:
+            if (feat >= 0) return fail(SB_ERR_SHAPE, "layer %d: convolution after a fully-connected layer", i);
+            if (l.out < 1) return fail(SB_ERR_SHAPE, "layer %d: Cout must be positive", i);
+            l.H = H; l.W = W; l.Cin = C; l.Cout = l.out; l.relu = true;
+            l.n_w = (size_t)l.Cout * 9 * l.Cin; l.n_b = l.Cout;
+            C = l.out;
+            l.out_per_img = (size_t)H * W * C;
+            break;
+        case SB_MAXPOOL2:
+            if (feat >= 0) return fail(SB_ERR_SHAPE, "layer %d: pooling after a fully-connected layer", i);
+            if (H % 2 || W % 2) return fail(SB_ERR_SHAPE, "layer %d: pooling needs even H and W (got %dx%d)", i, H, W);
+            if (i == 0) return fail(SB_ERR_UNSUPPORTED, "layer 0 cannot be a pooling layer");
+            l.H = H; l.W = W; l.Cin = l.Cout = C;
+            H /= 2; W /= 2;
+            l.out_per_img = (size_t)H * W * C;
+            break;
+        case SB_FC_RELU:
+        case SB_FC:
+            if (l.out < 1) return fail(SB_ERR_SHAPE, "layer %d: FC width must be positive", i);
+            if (cfg->K > l.out) return fail(SB_ERR_SHAPE, "layer %d: K=%d exceeds the FC width %d", i, cfg->K, l.out);
+            if (feat < 0) { feat = (long)H * W * C; first_fc = i; }
+            l.in_f = (int)feat; l.out_f = l.out; l.relu = l.kind == SB_FC_RELU;
+            l.n_w = (size_t)l.in_f * l.out_f; l.n_b = l.out_f;
+            feat = l.out;
+            l.out_per_img = l.out;
+            if (l.kind == SB_FC) l.act_dt = SB_DT_F32;
+            break;
+        case SB_SOFTMAX_XENT:
+            if (i != n - 1) return fail(SB_ERR_SHAPE, "the loss must be the last layer");
+            if (i == 0 || m->L[i - 1].kind != SB_FC) return fail(SB_ERR_SHAPE, "the loss must follow an SB_FC (logits) layer");
+            if (l.out != feat) return fail(SB_ERR_SHAPE, "loss classes (%d) != last FC width (%ld)", l.out, feat);
+            break;
+        default:
+            return fail(SB_ERR_INVALID_ARG, "layer %d: unknown kind %d", i, l.kind);
+        }
+        if (l.kind == SB_FC && (i + 1 >= n || layers[i + 1].kind != SB_SOFTMAX_XENT))
+            return fail(SB_ERR_SHAPE, "layer %d: SB_FC (no ReLU) is the logits layer and must be followed by the loss", i);
+        if (l.n_w) {
+            l.p_w = P; P += align_up(l.n_w, 64);
+            l.p_b = P; P += align_up(l.n_b, 64);
+        }
+    }
+    if (m->L[n - 1].kind != SB_SOFTMAX_XENT) return fail(SB_ERR_SHAPE, "the last layer must be SB_SOFTMAX_XENT");
+    m->first_fc = first_fc;
+    m->P = P;
+
+    // ---- arena carve-up -------------------------------------------------------------------
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return base ? base + o : (char*)nullptr; };
+    m->Wm = (float*)take(P * 4);
+    m->Vm = (float*)take(P * 4);
+    m->Gm = (float*)take(P * 4);
+    m->Sm = m->bf16 ? (__nv_bfloat16*)take(P * 2) : nullptr;
+    const size_t B = m->B;
+    size_t ws_floats = 1024;
+    for (int i = 0; i < n; ++i) {
+        Layer& l = m->L[i];
+        if (l.kind == SB_SOFTMAX_XENT) continue;
+        size_t e = (l.kind == SB_FC) ? 4 : m->esz;
+        l.act = take(B * l.out_per_img * e);
+        l.dact = take(B * l.out_per_img * m->esz);
+        if (l.kind == SB_MAXPOOL2) l.idx = (uint8_t*)take(B * l.out_per_img);
+        if (l.kind == SB_CONV3X3_RELU) {
+            // pixel-range splits of the weight gradient: enough blocks to fill the machine, each
+            // split a whole number of images
+            long tiles = (long)((l.Cout + 31) / 32) * ((l.Cin + 31) / 32) * 9;
+            int s = 1;
+            while (tiles * s < 148 * 4 && s * 2 <= (int)B && B % (s * 2) == 0) s *= 2;
+            l.wg_splits = s;
+            size_t need = (size_t)s * (l.n_w + l.n_b);
+            if (need > ws_floats) ws_floats = need;
+        }
+    }
+    size_t um_ws = 0;
+    sb_status us = umma_plan_scratch(m, &um_ws);
+    if (us != SB_OK) return us;
+    if (um_ws > ws_floats) ws_floats = um_ws;
+    m->ws_floats = ws_floats;
+    m->ws = (float*)take(ws_floats * 4);
+    m->row_loss = (float*)take(B * 4);
+    m->loss = (float*)take(256);
+    m->counter = (unsigned int*)take(256);
+    m->status = (uint32_t*)take(256);
+    m->stage_x = take(B * m->in_per_img * m->esz);
+    m->stage_labels = (int32_t*)take(B * 4);
+    m->input_grad = (cfg->flags & SB_FLAG_INPUT_GRAD) ? take(B * m->in_per_img * m->esz) : nullptr;
+    *total = off;
+    return SB_OK;
+}
+
+inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / K); }
+
+#define L_TRY(expr)                                                                               \
+    do {                                                                                          \
+        cudaError_t e_ = (expr);                                                                  \
+        ++m->launches;                                                                            \
+        if (e_ != cudaSuccess) return fail(SB_ERR_CUDA, "launch failed in %s: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+// Which buffer holds the input of layer i: the previous layer's output, or the caller's images.
+inline const char* layer_input(const sb_model* m, int i) { return i > 0 ? m->L[i - 1].act : nullptr; }
+
+sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
+{
+    Layer& l = m->L[i];
+    const bool bf = m->bf16;
+    const int B = m->B, b = m->cfg.batch_per_replica;
+    const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
+    switch (l.kind) {
+    case SB_CONV3X3_RELU: {
+        if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        if (l.um.fwd.enabled) {
+            sb_status s = umma_conv_fwd(m, i, st);
+            if (s != SB_OK) return s;
+            ++m->launches;
+            break;
+        }
+        ConvSimtArgs a{};
+        a.in = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
+        a.w = wts; a.bias = m->Wm + l.p_b; a.out = l.act; a.mask_ref = nullptr;
+        a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 0; a.relu = 1;
+        L_TRY(launch_conv_simt(a, bf, st));
+        break;
+    }
+    case SB_MAXPOOL2: {
+        PoolArgs a{layer_input(m, i), l.act, l.idx, B, l.H, l.W, l.Cin};
+        L_TRY(launch_pool_fwd(a, bf, st));
+        break;
+    }
+    case SB_FC_RELU:
+    case SB_FC: {
+        if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        if (l.um.fwd.enabled) {
+            sb_status s = umma_fc_fwd(m, i, st);
+            if (s != SB_OK) return s;
+            ++m->launches;
+            break;
+        }
+        GemmSimtArgs a{};
+        a.A = layer_input(m, i); a.sAm = l.in_f; a.sAk = 1;
+        a.B = wts; a.sBn = l.in_f; a.sBk = 1;
+        a.M = B; a.N = l.out_f; a.K = l.in_f;
+        a.epi = EPI_BIAS_ACT; a.ldc = l.out_f; a.bias = m->Wm + l.p_b; a.relu = l.relu;
+        if (l.kind == SB_FC) { a.C = nullptr; a.C32 = (float*)l.act; } else { a.C = l.act; a.C32 = nullptr; }
+        a.shard_dim = 1; a.shards = m->cfg.K;
+        if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 1; a.tab_b = b; }
+        L_TRY(launch_gemm_simt(a, bf, st));
+        break;
+    }
+    case SB_SOFTMAX_XENT: {
+        if (!m->have_labels) return fail(SB_ERR_STATE, "the loss layer needs label pointers");
+        Layer& fc = m->L[i - 1];
+        XentArgs a{};
+        a.logits = (const float*)fc.act; a.labels = m->label_tab; a.b_per_rep = b;
+        a.row_loss = m->row_loss; a.loss = m->loss; a.dZ = fc.dact; a.counter = m->counter;
+        a.B = B; a.C = l.out;
+        L_TRY(launch_softmax_xent(a, bf, st));
+        break;
+    }
+    }
+    return SB_OK;
+}
+
+sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
+{
+    Layer& l = m->L[i];
+    const bool bf = m->bf16;
+    const int B = m->B, b = m->cfg.batch_per_replica;
+    const bool want_in_grad = i > 0 || (m->cfg.flags & SB_FLAG_INPUT_GRAD);
+    // where the gradient w.r.t. this layer's input goes, and whether the layer below applied a ReLU
+    char* d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
+    const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
+    const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
+    switch (l.kind) {
+    case SB_SOFTMAX_XENT:
+        break;  // dZ was produced by the forward loss kernel
+    case SB_FC_RELU:
+    case SB_FC: {
+        if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        // weight gradient per shard: dW_j = dY_j^T X   (rows c_j..c_{j+1} of the [out,in] gradient)
+        if (l.um.wgrad.enabled) {
+            sb_status s = umma_fc_wgrad(m, i, st);
+            if (s != SB_OK) return s;
+            ++m->launches;
+        } else {
+            GemmSimtArgs a{};
+            a.A = l.dact; a.sAm = 1; a.sAk = l.out_f;
+            a.B = layer_input(m, i); a.sBn = 1; a.sBk = l.in_f;
+            a.M = l.out_f; a.N = l.in_f; a.K = B;
+            a.epi = EPI_F32; a.C = m->Gm + l.p_w; a.ldc = l.in_f;
+            a.shard_dim = 3; a.shards = m->cfg.K;
+            if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 2; a.tab_b = b; }
+            L_TRY(launch_gemm_simt(a, bf, st));
+        }
+        L_TRY(launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
+        if (want_in_grad) {
+            // shard-layer / modulo-layer backward: dX = sum_j dY_j W_j, rows stay with their replica
+            if (l.um.dgrad.enabled) {
+                sb_status s = umma_fc_dgrad(m, i, st);
+                if (s != SB_OK) return s;
+                ++m->launches;
+            } else {
+                GemmSimtArgs a{};
+                a.A = l.dact; a.sAm = l.out_f; a.sAk = 1;
+                a.B = wts; a.sBn = 1; a.sBk = l.in_f;
+                a.M = B; a.N = l.in_f; a.K = l.out_f;
+                a.epi = EPI_MASK; a.C = d_below; a.ldc = l.in_f;
+                a.ref = below_relu ? m->L[i - 1].act : nullptr; a.ldref = l.in_f;
+                a.shard_dim = 2; a.shards = m->cfg.K;
+                L_TRY(launch_gemm_simt(a, bf, st));
+            }
+        }
+        break;
+    }
+    case SB_MAXPOOL2: {
+        PoolBwdArgs a{l.dact, l.idx, below_relu ? l.act : nullptr, d_below, B, l.H, l.W, l.Cin};
+        L_TRY(launch_pool_bwd(a, bf, st));
+        break;
+    }
+    case SB_CONV3X3_RELU: {
+        if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
+        if (l.um.wgrad.enabled) {
+            sb_status s = umma_conv_wgrad(m, i, st);
+            if (s != SB_OK) return s;
+        } else {
+            const int S = l.wg_splits;
+            WgradSimtArgs a{};
+            a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
+            a.dy = l.dact; a.part = S > 1 ? m->ws : m->Gm + l.p_w;
+            a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
+            L_TRY(launch_wgrad_simt(a, bf, st));
+            if (S > 1) L_TRY(launch_reduce_partials(m->ws, m->Gm + l.p_w, l.n_w, S, st));
+        }
+        {
+            // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
+            const long M = (long)B * l.H * l.W;
+            int S = 1;
+            while (S * 2 <= B && B % (S * 2) == 0 && (long)S * ((l.Cout + 31) / 32) < 148 * 2) S *= 2;
+            float* part = S > 1 ? m->ws + (size_t)l.wg_splits * l.n_w : m->Gm + l.p_b;
+            if ((size_t)l.wg_splits * l.n_w + (size_t)S * l.n_b > m->ws_floats) { S = 1; part = m->Gm + l.p_b; }
+            L_TRY(launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
+            if (S > 1) L_TRY(launch_reduce_partials(part, m->Gm + l.p_b, l.n_b, S, st));
+        }
+        if (want_in_grad) {
+            if (l.um.dgrad.enabled) {
+                sb_status s = umma_conv_dgrad(m, i, st);
+                if (s != SB_OK) return s;
+                ++m->launches;
+            } else {
+                ConvSimtArgs a{};
+                a.in = l.dact; a.tab = nullptr; a.b_per_rep = b;
+                a.w = wts; a.bias = nullptr; a.out = d_below;
+                a.mask_ref = below_relu ? m->L[i - 1].act : nullptr;
+                a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 1; a.relu = 0;
+                L_TRY(launch_conv_simt(a, bf, st));
+            }
+        }
+        break;
+    }
+    }
+    return SB_OK;
+}
+
+sb_status set_inputs(sb_model* m, const void* const* x, const int32_t* const* labels)
+{
+    for (int r = 0; r < m->cfg.R; ++r) {
+        if (x) {
+            if (!x[r] || ((uintptr_t)x[r] & 15)) return fail(SB_ERR_INVALID_ARG, "x[%d] is null or not 16-byte aligned", r);
+            m->x_tab.p[r] = x[r];
+        }
+        if (labels) {
+            if (!labels[r] || ((uintptr_t)labels[r] & 3)) return fail(SB_ERR_INVALID_ARG, "labels[%d] is null or misaligned", r);
+            m->label_tab.p[r] = labels[r];
+        }
+    }
+    if (x) m->have_x = true;
+    if (labels) m->have_labels = true;
+    return SB_OK;
+}
+
+// Resolves (what, layer, part) to a device pointer, shape and dtype.
+sb_status resolve(sb_model* m, int what, int li, int part, char** ptr, int64_t shape[4], int* dtype, size_t* bytes)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (li < 0 || li >= m->n_layers) return fail(SB_ERR_INVALID_ARG, "layer %d out of range", li);
+    Layer& l = m->L[li];
+    const int b = m->cfg.batch_per_replica, R = m->cfg.R, K = m->cfg.K;
+    int64_t sh[4] = {1, 1, 1, 1};
+    char* p = nullptr;
+    int dt = SB_DT_F32;
+    const bool is_conv = l.kind == SB_CONV3X3_RELU, is_fc = l.kind == SB_FC_RELU || l.kind == SB_FC, is_pool = l.kind == SB_MAXPOOL2;
+    auto param = [&](float* region, bool weight) -> sb_status {
+        if (!is_conv && !is_fc) return fail(SB_ERR_INVALID_ARG, "layer %d has no parameters", li);
+        if (is_conv) {
+            if (part != 0) return fail(SB_ERR_INVALID_ARG, "conv parameters are replicated: part must be 0");
+            if (weight) { p = (char*)(region + l.p_w); sh[0] = l.Cout; sh[1] = 3; sh[2] = 3; sh[3] = l.Cin; }
+            else { p = (char*)(region + l.p_b); sh[0] = l.Cout; }
+        } else {
+            if (part < 0 || part >= K) return fail(SB_ERR_INVALID_ARG, "shard %d out of range", part);
+            int lo = shard_lo(part, l.out_f, K), hi = shard_lo(part + 1, l.out_f, K);
+            if (weight) { p = (char*)(region + l.p_w + (size_t)lo * l.in_f); sh[0] = hi - lo; sh[1] = l.in_f; }
+            else { p = (char*)(region + l.p_b + lo); sh[0] = hi - lo; }
+        }
+        return SB_OK;
+    };
+    sb_status s = SB_OK;
+    switch (what) {
+    case SB_T_WEIGHT: s = param(m->Wm, true); break;
+    case SB_T_BIAS: s = param(m->Wm, false); break;
+    case SB_T_GRAD_W: s = param(m->Gm, true); break;
+    case SB_T_GRAD_B: s = param(m->Gm, false); break;
+    case SB_T_MOM_W: s = param(m->Vm, true); break;
+    case SB_T_MOM_B: s = param(m->Vm, false); break;
+    case SB_T_SHADOW_W:
+        if (!m->bf16) return fail(SB_ERR_INVALID_ARG, "no bf16 weight copies in SB_FP32 mode");
+        s = param(m->Wm, true);
+        if (s == SB_OK) { p = (char*)(m->Sm + ((float*)p - m->Wm)); dt = SB_DT_BF16; }
+        break;
+    case SB_T_ACT:
+    case SB_T_DACT: {
+        if (l.kind == SB_SOFTMAX_XENT) return fail(SB_ERR_INVALID_ARG, "the loss layer has no activation tensor");
+        char* basep = what == SB_T_ACT ? l.act : l.dact;
+        dt = what == SB_T_ACT ? l.act_dt : (m->bf16 ? SB_DT_BF16 : SB_DT_F32);
+        size_t e = dt == SB_DT_BF16 ? 2 : 4;
+        if (is_fc) { p = basep; sh[0] = m->B; sh[1] = l.out_f; }
+        else {
+            if (part < 0 || part >= R) return fail(SB_ERR_INVALID_ARG, "replica %d out of range", part);
+            p = basep + (size_t)part * b * l.out_per_img * e;
+            int Ho = is_pool ? l.H / 2 : l.H, Wo = is_pool ? l.W / 2 : l.W;
+            sh[0] = b; sh[1] = Ho; sh[2] = Wo; sh[3] = l.Cout;
+        }
+        break;
+    }
+    case SB_T_POOL_IDX:
+        if (!is_pool) return fail(SB_ERR_INVALID_ARG, "layer %d is not a pooling layer", li);
+        if (part < 0 || part >= R) return fail(SB_ERR_INVALID_ARG, "replica %d out of range", part);
+        p = (char*)l.idx + (size_t)part * b * l.out_per_img;
+        sh[0] = b; sh[1] = l.H / 2; sh[2] = l.W / 2; sh[3] = l.Cout; dt = SB_DT_U8;
+        break;
+    case SB_T_ROW_LOSS:
+        p = (char*)m->row_loss; sh[0] = m->B;
+        break;
+    case SB_T_INPUT_GRAD:
+        if (!m->input_grad) return fail(SB_ERR_INVALID_ARG, "model was created without SB_FLAG_INPUT_GRAD");
+        if (part < 0 || part >= R) return fail(SB_ERR_INVALID_ARG, "replica %d out of range", part);
+        dt = m->bf16 ? SB_DT_BF16 : SB_DT_F32;
+        p = m->input_grad + (size_t)part * b * m->in_per_img * m->esz;
+        sh[0] = b; sh[1] = m->cfg.H; sh[2] = m->cfg.W; sh[3] = m->cfg.C;
+        break;
+    default:
+        return fail(SB_ERR_INVALID_ARG, "unknown tensor selector %d", what);
+    }
+    if (s != SB_OK) return s;
+    if (ptr) *ptr = p;
+    if (shape) memcpy(shape, sh, sizeof(sh));
+    if (dtype) *dtype = dt;
+    if (bytes) {
+        size_t e = dt == SB_DT_F32 || dt == SB_DT_I32 ? 4 : dt == SB_DT_BF16 ? 2 : 1;
+        *bytes = (size_t)(sh[0] * sh[1] * sh[2] * sh[3]) * e;
+    }
+    return SB_OK;
+}
+
+}  // namespace
+
+// Accessors used by the tensor-core planner (sb_umma.cu), which cannot see the struct layout.
+namespace sb {
+ModelView model_view(sb_model* m)
+{
+    ModelView v{};
+    v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
+    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; v.ws_floats = m->ws_floats; v.status = m->status;
+    v.input_grad = m->input_grad; v.x_tab = &m->x_tab;
+    return v;
+}
+LayerView layer_view(sb_model* m, int i)
+{
+    Layer& l = m->L[i];
+    LayerView v{};
+    v.kind = l.kind; v.H = l.H; v.W = l.W; v.Cin = l.Cin; v.Cout = l.Cout; v.in_f = l.in_f; v.out_f = l.out_f; v.relu = l.relu;
+    v.p_w = l.p_w; v.p_b = l.p_b; v.n_w = l.n_w; v.n_b = l.n_b;
+    v.act = l.act; v.dact = l.dact; v.um = &l.um;
+    v.in_act = i > 0 ? m->L[i - 1].act : nullptr;
+    v.d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
+    v.below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
+    return v;
+}
+int64_t* launch_counter(sb_model* m) { return &m->launches; }
+}  // namespace sb
+
+// =================================================================================================
+extern "C" {
+
+sb_status sb_model_bytes(const sb_layer* layers, int32_t n, const sb_config* cfg, size_t* arena_bytes)
+{
+    if (!arena_bytes) return fail(SB_ERR_INVALID_ARG, "arena_bytes is null");
+    sb_model tmp;
+    return plan(layers, n, cfg, &tmp, nullptr, arena_bytes);
+}
+
+sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cfg, void* arena, size_t arena_bytes, sb_model** out)
+{
+    if (!out) return fail(SB_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (!arena || ((uintptr_t)arena & 255)) return fail(SB_ERR_INVALID_ARG, "arena is null or not 256-byte aligned");
+    sb_model* m = new (std::nothrow) sb_model;
+    if (!m) return fail(SB_ERR_INVALID_ARG, "out of host memory");
+    size_t need = 0;
+    sb_status s = plan(layers, n, cfg, m, (char*)arena, &need);
+    if (s != SB_OK) { delete m; return s; }
+    if (need > arena_bytes) { delete m; return fail(SB_ERR_ARENA_TOO_SMALL, "arena has %zu bytes, model needs %zu", arena_bytes, need); }
+    m->arena = (char*)arena;
+    m->arena_bytes = need;
+    cudaError_t e = cudaMemset(arena, 0, need);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }
+    s = umma_plan_layers(m);
+    if (s != SB_OK) { delete m; return s; }
+    *out = m;
+    return SB_OK;
+}
+
+sb_status sb_model_destroy(sb_model* m)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    delete m;
+    return SB_OK;
+}
+
+sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void* const* x, const int32_t* const* labels, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (first < 0 || last >= m->n_layers || first > last) return fail(SB_ERR_INVALID_ARG, "bad layer range %d..%d", first, last);
+    if (x || labels) {
+        sb_status s = set_inputs(m, x, labels);
+        if (s != SB_OK) return s;
+    }
+    for (int i = first; i <= last; ++i) {
+        sb_status s = forward_layer(m, i, (cudaStream_t)stream);
+        if (s != SB_OK) return s;
+    }
+    return SB_OK;
+}
+
+sb_status sb_backward_layers(sb_model* m, int32_t last, int32_t first, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (first < 0 || last >= m->n_layers || first > last) return fail(SB_ERR_INVALID_ARG, "bad layer range %d..%d", last, first);
+    for (int i = last; i >= first; --i) {
+        sb_status s = backward_layer(m, i, (cudaStream_t)stream);
+        if (s != SB_OK) return s;
+    }
+    return SB_OK;
+}
+
+sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* labels, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (!x || !labels) return fail(SB_ERR_INVALID_ARG, "x or labels is null");
+    sb_status s = set_inputs(m, x, labels);
+    if (s != SB_OK) return s;
+    m->launches = 0;
+    for (int i = 0; i < m->n_layers; ++i) {
+        s = forward_layer(m, i, (cudaStream_t)stream);
+        if (s != SB_OK) return s;
+    }
+    m->have_fwd = true;
+    return SB_OK;
+}
+
+sb_status sb_backward(sb_model* m, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (!m->have_fwd) return fail(SB_ERR_STATE, "sb_backward needs a preceding sb_forward");
+    for (int i = m->n_layers - 1; i >= 0; --i) {
+        sb_status s = backward_layer(m, i, (cudaStream_t)stream);
+        if (s != SB_OK) return s;
+    }
+    return SB_OK;
+}
+
+sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    L_TRY(launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, m->P, lr, momentum, (cudaStream_t)stream));
+    m->last_step_launches = m->launches;
+    return SB_OK;
+}
+
+sb_status sb_refresh_shadow(sb_model* m, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (m->bf16) L_TRY(launch_to_bf16(m->Wm, m->Sm, m->P, (cudaStream_t)stream));
+    return SB_OK;
+}
+
+sb_status sb_loss(sb_model* m, void* stream, float* host_loss)
+{
+    if (!m || !host_loss) return fail(SB_ERR_INVALID_ARG, "null model or host_loss");
+    struct { float loss; uint32_t status; } r;
+    CU_TRY(cudaMemcpyAsync(&r.loss, m->loss, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CU_TRY(cudaMemcpyAsync(&r.status, m->status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    *host_loss = r.loss;
+    if (r.status != DEV_OK) {
+        cudaMemsetAsync(m->status, 0, 4, (cudaStream_t)stream);
+        cudaStreamSynchronize((cudaStream_t)stream);
+        return fail(SB_ERR_TIMEOUT, "a kernel gave up on a bounded wait (device status %u)", r.status);
+    }
+    return SB_OK;
+}
+
+sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum,
+                             void* stream, float* host_loss)
+{
+    if (!m || !host_x || !host_labels || !host_loss) return fail(SB_ERR_INVALID_ARG, "null argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t xb = (size_t)m->B * m->in_per_img * m->esz;
+    CU_TRY(cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st));
+    const void* xp[MAX_PARTS];
+    const int32_t* lp[MAX_PARTS];
+    const int b = m->cfg.batch_per_replica;
+    for (int r = 0; r < m->cfg.R; ++r) {
+        xp[r] = m->stage_x + (size_t)r * b * m->in_per_img * m->esz;
+        lp[r] = m->stage_labels + (size_t)r * b;
+    }
+    sb_status s = sb_forward(m, xp, lp, stream);
+    if (s != SB_OK) return s;
+    s = sb_backward(m, stream);
+    if (s != SB_OK) return s;
+    s = sb_sgd_step(m, lr, momentum, stream);
+    if (s != SB_OK) return s;
+    return sb_loss(m, stream, host_loss);
+}
+
+sb_status sb_tensor(sb_model* m, int32_t what, int32_t layer, int32_t part, void** dev_ptr, int64_t shape[4], int32_t* dtype)
+{
+    char* p = nullptr;
+    sb_status s = resolve(m, what, layer, part, &p, shape, dtype, nullptr);
+    if (s == SB_OK && dev_ptr) *dev_ptr = p;
+    return s;
+}
+
+sb_status sb_tensor_read(sb_model* m, int32_t what, int32_t layer, int32_t part, void* host_dst, size_t bytes)
+{
+    char* p = nullptr;
+    size_t nb = 0;
+    sb_status s = resolve(m, what, layer, part, &p, nullptr, nullptr, &nb);
+    if (s != SB_OK) return s;
+    if (!host_dst || bytes != nb) return fail(SB_ERR_INVALID_ARG, "host buffer is null or %zu bytes (tensor has %zu)", bytes, nb);
+    CU_TRY(cudaDeviceSynchronize());
+    CU_TRY(cudaMemcpy(host_dst, p, nb, cudaMemcpyDeviceToHost));
+    return SB_OK;
+}
+
+sb_status sb_tensor_write(sb_model* m, int32_t what, int32_t layer, int32_t part, const void* host_src, size_t bytes)
+{
+    char* p = nullptr;
+    size_t nb = 0;
+    sb_status s = resolve(m, what, layer, part, &p, nullptr, nullptr, &nb);
+    if (s != SB_OK) return s;
+    if (!host_src || bytes != nb) return fail(SB_ERR_INVALID_ARG, "host buffer is null or %zu bytes (tensor has %zu)", bytes, nb);
+    CU_TRY(cudaDeviceSynchronize());
+    CU_TRY(cudaMemcpy(p, host_src, nb, cudaMemcpyHostToDevice));
+    return SB_OK;
+}
+
+sb_status sb_param_bytes(const sb_model* m, int32_t shard, size_t* bytes)
+{
+    if (!m || !bytes) return fail(SB_ERR_INVALID_ARG, "null argument");
+    if (shard < 0 || shard >= m->cfg.K) return fail(SB_ERR_INVALID_ARG, "shard %d out of range", shard);
+    size_t n = 0;
+    for (const Layer& l : m->L) {
+        if (l.kind == SB_CONV3X3_RELU) n += l.n_w + l.n_b;
+        else if (l.kind == SB_FC_RELU || l.kind == SB_FC) {
+            size_t rows = shard_lo(shard + 1, l.out_f, m->cfg.K) - shard_lo(shard, l.out_f, m->cfg.K);
+            n += rows * l.in_f + rows;
+        }
+    }
+    *bytes = n * 4;
+    return SB_OK;
+}
+
+sb_status sb_launch_count(const sb_model* m, int64_t* launches)
+{
+    if (!m || !launches) return fail(SB_ERR_INVALID_ARG, "null argument");
+    *launches = m->last_step_launches;
+    return SB_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,111 @@
+// Internal declarations shared by the host-side planner (sb_api.cu) and the kernel files.
+// Nothing here is part of the public C ABI (see include/splitbrain.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace sb {
+
+constexpr int MAX_PARTS = 64;  // upper bound on R and K
+
+// Pointer table for per-replica caller buffers (inputs, labels): passed by value to kernels.
+struct PtrTab {
+    const void* p[MAX_PARTS];
+};
+
+// Device status word codes (written by kernels that give up on a bounded wait).
+enum : uint32_t { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3 };
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core ("SIMT") kernels: the float mode, odd channel counts, and the cross-check path.
+// All launchers return the cudaError_t of the launch.  `bf16` selects the activation dtype
+// (false: float, true: __nv_bfloat16) of every T-typed pointer.
+// ---------------------------------------------------------------------------------------------
+
+struct ConvSimtArgs {
+    const void* in;       // [B,H,W,Cred] activation dtype (ignored when tab != nullptr)
+    const PtrTab* tab;    // optional: R per-replica input pointers (host pointer to the table)
+    int b_per_rep;
+    const void* w;        // [Cout,3,3,Cin] activation dtype (float master or bf16 shadow)
+    const float* bias;    // [Cout] (forward only)
+    void* out;            // [B,H,W,Cres] activation dtype
+    const void* mask_ref; // dgrad only, optional: zero the result where mask_ref <= 0 ([B,H,W,Cres])
+    int B, H, W, Cin, Cout;
+    int dgrad;            // 0: forward (+bias, ReLU if relu) ; 1: data gradient
+    int relu;
+};
+cudaError_t launch_conv_simt(const ConvSimtArgs& a, bool bf16, cudaStream_t st);
+
+struct WgradSimtArgs {
+    const void* x;        // [B,H,W,Cin] (ignored when tab != nullptr)
+    const PtrTab* tab;
+    int b_per_rep;
+    const void* dy;       // [B,H,W,Cout]
+    float* part;          // [splits][Cout*9*Cin] partial sums (or the gradient itself if splits==1)
+    int B, H, W, Cin, Cout;
+    int splits;           // pixel-range splits; split s covers images [s*B/splits, (s+1)*B/splits)
+};
+cudaError_t launch_wgrad_simt(const WgradSimtArgs& a, bool bf16, cudaStream_t st);
+
+// part[s][n] = sum over the rows of split s of in[row][n];  rows split evenly (M % splits == 0).
+cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st);
+// out[i] = sum_{s<splits} part[s*n + i], s ascending.
+cudaError_t launch_reduce_partials(const float* part, float* out, size_t n, int splits, cudaStream_t st);
+
+struct PoolArgs {
+    const void* x;  // [B,H,W,C]
+    void* p;        // [B,H/2,W/2,C]
+    uint8_t* idx;   // [B,H/2,W/2,C]
+    int B, H, W, C;
+};
+cudaError_t launch_pool_fwd(const PoolArgs& a, bool bf16, cudaStream_t st);
+struct PoolBwdArgs {
+    const void* dp;      // [B,H/2,W/2,C] gradient w.r.t. the pooled output
+    const uint8_t* idx;
+    const void* p;       // pooled output (ReLU mask source) or nullptr for no mask
+    void* dx;            // [B,H,W,C]
+    int B, H, W, C;
+};
+cudaError_t launch_pool_bwd(const PoolBwdArgs& a, bool bf16, cudaStream_t st);
+
+struct XentArgs {
+    const float* logits;  // [B,C]
+    PtrTab labels;        // R pointers to int32 [b]
+    int b_per_rep;
+    float* row_loss;      // [B]
+    float* loss;          // [1] mean over rows
+    void* dZ;             // [B,C] activation dtype: (softmax - onehot)/B
+    unsigned int* counter; // zero-initialised word; left at zero
+    int B, C;
+};
+cudaError_t launch_softmax_xent(const XentArgs& a, bool bf16, cudaStream_t st);
+
+cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n,
+                       float lr, float mu, cudaStream_t st);
+cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cudaStream_t st);
+
+// Strided GEMM  C[m,n] = sum_k A(m,k) * B(n,k)  with A(m,k) = A[m*sAm + k*sAk], B(n,k) = B[n*sBn + k*sBk].
+enum { EPI_BIAS_ACT = 0, EPI_MASK = 1, EPI_F32 = 2 };
+struct GemmSimtArgs {
+    const void* A; long sAm, sAk;
+    const void* B; long sBn, sBk;
+    int M, N, K;
+    int epi;
+    void* C; long ldc;        // activation dtype (EPI_BIAS_ACT, EPI_MASK) or float (EPI_F32)
+    float* C32;               // EPI_BIAS_ACT: optional float copy of the result (logits), same ldc
+    const float* bias;        // EPI_BIAS_ACT: [N]
+    int relu;
+    const void* ref; long ldref;  // EPI_MASK: optional, zero where ref <= 0
+    // Model-shard partition of one GEMM dimension: 0 none, 1 = N (forward: each shard owns its
+    // output columns), 2 = K (dgrad: sum over shards), 3 = M (wgrad: each shard owns its rows).
+    int shard_dim, shards;
+    // Optional replica gather by addressing: the rows of the activation matrix live in R separate
+    // caller buffers of tab_b rows each.  tab_mode 1: A's m index is the row; 2: B's k index is.
+    const PtrTab* tab; int tab_mode, tab_b;
+};
+cudaError_t launch_gemm_simt(const GemmSimtArgs& a, bool bf16, cudaStream_t st);
+
+}  // namespace sb

@@ -1,0 +1,621 @@
+// CUDA-core kernels of the SplitBrain training step for sm_100a.
+//
+//  * bandwidth-bound steps that every mode uses: 2x2 max-pool forward/backward, softmax
+//    cross-entropy, SGD with momentum, column sums (bias gradients) and split reductions;
+//  * float-accumulating FFMA versions of the contractions (3x3 conv forward / dgrad / wgrad and
+//    a strided GEMM for the sharded FC layers).  They are the float mode, serve layers whose
+//    channel count does not fit the tensor-core tiles (e.g. the 3-channel input layer), and are
+//    the on-device cross-check of the tcgen05 kernels.
+//
+// T is the activation dtype (float or __nv_bfloat16); all sums are carried in float.
+#include "sb_internal.h"
+
+namespace sb {
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T* p, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+static inline int cdiv(long a, long b) { return (int)((a + b - 1) / b); }
+
+// =============================================================================================
+// 3x3 convolution, forward and data gradient (direct, tiled through shared memory).
+//   forward: y[n,h,w,o] = act(bias[o] + sum_{r,s,i} x[n,h+r-1,w+s-1,i] * W[o,r,s,i])
+//   dgrad  : dx[n,h,w,o] = mask * sum_{r,s,i} dy[n,h-r+1,w-s+1,i] * W[i,r,s,o]
+// Block: 8x8 output pixels x 32 output channels, 128 threads, 4 pixels x 4 channels per thread.
+// =============================================================================================
+constexpr int CV_TP = 8, CV_TC = 32, CV_CK = 16;
+
+template <typename T, bool DGRAD, bool TAB>
+__global__ void __launch_bounds__(128)
+conv3x3_simt_kernel(const T* __restrict__ in, PtrTab tab, int b_per_rep, const T* __restrict__ wt,
+                    const float* __restrict__ bias, T* __restrict__ out, const T* __restrict__ mask_ref,
+                    int H, int W, int Cred, int Cres, int Cin, int relu)
+{
+    __shared__ float s_in[CV_TP + 2][CV_TP + 2][CV_CK + 1];
+    __shared__ float s_w[9][CV_CK][CV_TC];
+    const int tiles_w = (W + CV_TP - 1) / CV_TP;
+    const int h0 = (blockIdx.x / tiles_w) * CV_TP, w0 = (blockIdx.x % tiles_w) * CV_TP;
+    const int n = blockIdx.y;
+    const int o0 = blockIdx.z * CV_TC;
+    const int tid = threadIdx.x;
+    const int cg = tid / 16, pg = tid % 16;
+    const int prow = pg / 2, pcol = (pg % 2) * 4;
+    const T* img = TAB ? (const T*)tab.p[n / b_per_rep] + (size_t)(n % b_per_rep) * H * W * Cred
+                       : in + (size_t)n * H * W * Cred;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int c0 = 0; c0 < Cred; c0 += CV_CK) {
+        for (int e = tid; e < (CV_TP + 2) * (CV_TP + 2) * CV_CK; e += 128) {
+            int c = e % CV_CK, q = e / CV_CK;
+            int ww = q % (CV_TP + 2), hh = q / (CV_TP + 2);
+            int gh = h0 + hh - 1, gw = w0 + ww - 1, gc = c0 + c;
+            float v = 0.f;
+            if (gh >= 0 && gh < H && gw >= 0 && gw < W && gc < Cred) v = ldf(img + ((size_t)gh * W + gw) * Cred + gc);
+            s_in[hh][ww][c] = v;
+        }
+        for (int e = tid; e < 9 * CV_CK * CV_TC; e += 128) {
+            int o = e % CV_TC, q = e / CV_TC;
+            int c = q % CV_CK, t = q / CV_CK;
+            int go = o0 + o, gc = c0 + c;
+            float v = 0.f;
+            if (go < Cres && gc < Cred) {
+                // weight tensor is [Cout][9][Cin]; forward: out=o, in=c ; dgrad: out index is Cin, reduce index is Cout
+                size_t wi = DGRAD ? (((size_t)gc * 9 + t) * Cin + go) : (((size_t)go * 9 + t) * Cin + gc);
+                v = ldf(wt + wi);
+            }
+            s_w[t][c][o] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+            const int r = t / 3, s = t % 3;
+            const int dr = DGRAD ? (2 - r) : r, ds = DGRAD ? (2 - s) : s;
+#pragma unroll 4
+            for (int c = 0; c < CV_CK; ++c) {
+                float xv[4], wv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xv[i] = s_in[prow + dr][pcol + i + ds][c];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) wv[j] = s_w[t][c][cg * 4 + j];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv[i], wv[j], acc[i][j]);
+            }
+        }
+        __syncthreads();
+    }
+    const int gh = h0 + prow;
+    if (gh >= H) return;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int gw = w0 + pcol + i;
+        if (gw >= W) continue;
+        size_t pix = ((size_t)n * H + gh) * W + gw;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int go = o0 + cg * 4 + j;
+            if (go >= Cres) continue;
+            float v = acc[i][j];
+            if (!DGRAD) {
+                v += bias[go];
+                if (relu && !(v > 0.f)) v = 0.f;
+            } else if (mask_ref != nullptr) {
+                if (!(ldf(mask_ref + pix * Cres + go) > 0.f)) v = 0.f;
+            }
+            stf(out + pix * Cres + go, v);
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_conv_simt_t(const ConvSimtArgs& a, cudaStream_t st)
+{
+    const int Cred = a.dgrad ? a.Cout : a.Cin, Cres = a.dgrad ? a.Cin : a.Cout;
+    dim3 grid(cdiv(a.H, CV_TP) * cdiv(a.W, CV_TP), a.B, cdiv(Cres, CV_TC));
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+    if (a.dgrad)
+        conv3x3_simt_kernel<T, true, false><<<grid, 128, 0, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
+                                                                  (T*)a.out, (const T*)a.mask_ref, a.H, a.W, Cred, Cres, a.Cin, 0);
+    else if (a.tab)
+        conv3x3_simt_kernel<T, false, true><<<grid, 128, 0, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias,
+                                                                  (T*)a.out, nullptr, a.H, a.W, Cred, Cres, a.Cin, a.relu);
+    else
+        conv3x3_simt_kernel<T, false, false><<<grid, 128, 0, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
+                                                                   (T*)a.out, nullptr, a.H, a.W, Cred, Cres, a.Cin, a.relu);
+    return cudaGetLastError();
+}
+cudaError_t launch_conv_simt(const ConvSimtArgs& a, bool bf16, cudaStream_t st)
+{
+    return bf16 ? launch_conv_simt_t<__nv_bfloat16>(a, st) : launch_conv_simt_t<float>(a, st);
+}
+
+// =============================================================================================
+// 3x3 convolution weight gradient: part[s][k,t,c] = sum over split s's pixels of
+// dy[pix,k] * x[pix shifted by tap t, c].  Block: 32 (k) x 32 (c) outputs of one tap, 256 threads.
+// =============================================================================================
+template <typename T, bool TAB>
+__global__ void __launch_bounds__(256)
+conv3x3_wgrad_simt_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ dy,
+                          float* __restrict__ part, int B, int H, int W, int Cin, int Cout, int splits)
+{
+    __shared__ float s_dy[32][33];
+    __shared__ float s_x[32][33];
+    const int k0 = blockIdx.x * 32;
+    const int ctiles = (Cin + 31) / 32;
+    const int c0 = (blockIdx.y % ctiles) * 32, t = blockIdx.y / ctiles;
+    const int r = t / 3, s = t % 3;
+    const int sp = blockIdx.z;
+    const int imgs = B / splits;
+    const long pix_begin = (long)sp * imgs * H * W, pix_end = pix_begin + (long)imgs * H * W;
+    const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
+    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    for (long p0 = pix_begin; p0 < pix_end; p0 += 32) {
+        for (int e = tid; e < 32 * 32; e += 256) {
+            int j = e % 32, pp = e / 32;
+            long pix = p0 + pp;
+            float vd = 0.f, vx = 0.f;
+            if (pix < pix_end) {
+                if (k0 + j < Cout) vd = ldf(dy + pix * Cout + k0 + j);
+                int w_ = (int)(pix % W);
+                long q = pix / W;
+                int h_ = (int)(q % H), n_ = (int)(q / H);
+                int hh = h_ + r - 1, ww = w_ + s - 1;
+                if (hh >= 0 && hh < H && ww >= 0 && ww < W && c0 + j < Cin) {
+                    const T* img = TAB ? (const T*)tab.p[n_ / b_per_rep] + (size_t)(n_ % b_per_rep) * H * W * Cin
+                                       : x + (size_t)n_ * H * W * Cin;
+                    vx = ldf(img + ((size_t)hh * W + ww) * Cin + c0 + j);
+                }
+            }
+            s_dy[pp][j] = vd;
+            s_x[pp][j] = vx;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int pp = 0; pp < 32; ++pp) {
+            float a0 = s_dy[pp][ty * 2], a1 = s_dy[pp][ty * 2 + 1];
+            float b0 = s_x[pp][tx * 2], b1 = s_x[pp][tx * 2 + 1];
+            acc[0][0] = fmaf(a0, b0, acc[0][0]);
+            acc[0][1] = fmaf(a0, b1, acc[0][1]);
+            acc[1][0] = fmaf(a1, b0, acc[1][0]);
+            acc[1][1] = fmaf(a1, b1, acc[1][1]);
+        }
+        __syncthreads();
+    }
+    float* dst = part + (size_t)sp * Cout * 9 * Cin;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            int k = k0 + ty * 2 + i, c = c0 + tx * 2 + j;
+            if (k < Cout && c < Cin) dst[((size_t)k * 9 + t) * Cin + c] = acc[i][j];
+        }
+}
+
+cudaError_t launch_wgrad_simt(const WgradSimtArgs& a, bool bf16, cudaStream_t st)
+{
+    dim3 grid(cdiv(a.Cout, 32), cdiv(a.Cin, 32) * 9, a.splits);
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+#define SB_WG(T, TABF)                                                                                         \
+    conv3x3_wgrad_simt_kernel<T, TABF><<<grid, 256, 0, st>>>((const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, \
+                                                            a.part, a.B, a.H, a.W, a.Cin, a.Cout, a.splits)
+    if (bf16) { if (a.tab) SB_WG(__nv_bfloat16, true); else SB_WG(__nv_bfloat16, false); }
+    else      { if (a.tab) SB_WG(float, true); else SB_WG(float, false); }
+#undef SB_WG
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Column sums (bias gradients) and the reduction of split partial sums.
+// =============================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+colsum_kernel(const T* __restrict__ in, float* __restrict__ part, int M, int N, int splits)
+{
+    __shared__ float s[8][33];
+    const int col = blockIdx.x * 32 + threadIdx.x % 32;
+    const int lane_row = threadIdx.x / 32;
+    const int sp = blockIdx.y;
+    const long rows = M / splits, r0 = (long)sp * rows;
+    float acc = 0.f;
+    if (col < N)
+        for (long r = lane_row; r < rows; r += 8) acc += ldf(in + (r0 + r) * N + col);
+    s[lane_row][threadIdx.x % 32] = acc;
+    __syncthreads();
+    if (lane_row == 0 && col < N) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += s[i][threadIdx.x];
+        part[(size_t)sp * N + col] = t;
+    }
+}
+cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st)
+{
+    dim3 grid(cdiv(N, 32), splits);
+    if (bf16) colsum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)in, part, M, N, splits);
+    else colsum_kernel<float><<<grid, 256, 0, st>>>((const float*)in, part, M, N, splits);
+    return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ out, size_t n, int splits)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float t = 0.f;
+        for (int s = 0; s < splits; ++s) t += part[(size_t)s * n + i];
+        out[i] = t;
+    }
+}
+cudaError_t launch_reduce_partials(const float* part, float* out, size_t n, int splits, cudaStream_t st)
+{
+    int blocks = cdiv((long)n, 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, out, n, splits);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// 2x2 max-pool, stride 2.  One thread per pooled pixel and VEC channels (16-byte accesses when the
+// channel count allows).  Ties go to the first maximum in scan order (0,0),(0,1),(1,0),(1,1).
+// =============================================================================================
+template <typename T, int VEC> struct VecT;
+template <> struct VecT<float, 4> { typedef float4 type; };
+template <> struct VecT<float, 1> { typedef float type; };
+template <> struct VecT<__nv_bfloat16, 8> { typedef uint4 type; };
+template <> struct VecT<__nv_bfloat16, 1> { typedef __nv_bfloat16 type; };
+template <int VEC> struct VecU8;
+template <> struct VecU8<8> { typedef uint2 type; };
+template <> struct VecU8<4> { typedef uint32_t type; };
+template <> struct VecU8<1> { typedef uint8_t type; };
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ p, uint8_t* __restrict__ idx, long total, int H, int W, int C)
+{
+    typedef typename VecT<T, VEC>::type V;
+    typedef typename VecU8<VEC>::type VI;
+    const int Ho = H / 2, Wo = W / 2, Cv = C / VEC;
+    for (long e = blockIdx.x * (long)blockDim.x + threadIdx.x; e < total; e += (long)gridDim.x * blockDim.x) {
+        int cv = (int)(e % Cv);
+        long q = e / Cv;
+        int wo = (int)(q % Wo);
+        q /= Wo;
+        int ho = (int)(q % Ho);
+        long n = q / Ho;
+        const T* base = x + (((size_t)n * H + 2 * ho) * W + 2 * wo) * C + (size_t)cv * VEC;
+        V v[4];
+        v[0] = *(const V*)(base);
+        v[1] = *(const V*)(base + C);
+        v[2] = *(const V*)(base + (size_t)W * C);
+        v[3] = *(const V*)(base + (size_t)W * C + C);
+        V outv;
+        VI outi;
+        T* ov = (T*)&outv;
+        uint8_t* oi = (uint8_t*)&outi;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            T bestv = ((const T*)&v[0])[k];
+            float best = ldf(&bestv);
+            int bi = 0;
+#pragma unroll
+            for (int j = 1; j < 4; ++j) {
+                T cand = ((const T*)&v[j])[k];
+                float f = ldf(&cand);
+                if (f > best) { best = f; bi = j; bestv = cand; }
+            }
+            ov[k] = bestv;
+            oi[k] = (uint8_t)bi;
+        }
+        size_t o = (size_t)e * VEC;
+        *(V*)(p + o) = outv;
+        *(VI*)(idx + o) = outi;
+    }
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+maxpool_bwd_kernel(const T* __restrict__ dp, const uint8_t* __restrict__ idx, const T* __restrict__ p,
+                   T* __restrict__ dx, long total, int H, int W, int C)
+{
+    typedef typename VecT<T, VEC>::type V;
+    typedef typename VecU8<VEC>::type VI;
+    const int Ho = H / 2, Wo = W / 2, Cv = C / VEC;
+    for (long e = blockIdx.x * (long)blockDim.x + threadIdx.x; e < total; e += (long)gridDim.x * blockDim.x) {
+        int cv = (int)(e % Cv);
+        long q = e / Cv;
+        int wo = (int)(q % Wo);
+        q /= Wo;
+        int ho = (int)(q % Ho);
+        long n = q / Ho;
+        size_t o = (size_t)e * VEC;
+        V g = *(const V*)(dp + o);
+        VI iv = *(const VI*)(idx + o);
+        const uint8_t* ii = (const uint8_t*)&iv;
+        T* gp = (T*)&g;
+        if (p != nullptr) {
+            V pv = *(const V*)(p + o);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k)
+                if (!(ldf((const T*)&pv + k) > 0.f)) stf(gp + k, 0.f);
+        }
+        T* base = dx + (((size_t)n * H + 2 * ho) * W + 2 * wo) * C + (size_t)cv * VEC;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            V ov;
+            T* op = (T*)&ov;
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) {
+                if (ii[k] == j) op[k] = gp[k]; else stf(op + k, 0.f);
+            }
+            *(V*)(base + (size_t)(j >> 1) * W * C + (size_t)(j & 1) * C) = ov;
+        }
+    }
+}
+
+static int ew_blocks(long total)
+{
+    long b = (total + 255) / 256;
+    long cap = 148L * 16;
+    return (int)(b < cap ? (b < 1 ? 1 : b) : cap);
+}
+
+cudaError_t launch_pool_fwd(const PoolArgs& a, bool bf16, cudaStream_t st)
+{
+    long pooled = (long)a.B * (a.H / 2) * (a.W / 2) * a.C;
+    if (bf16) {
+        if (a.C % 8 == 0) maxpool_fwd_kernel<__nv_bfloat16, 8><<<ew_blocks(pooled / 8), 256, 0, st>>>((const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled / 8, a.H, a.W, a.C);
+        else maxpool_fwd_kernel<__nv_bfloat16, 1><<<ew_blocks(pooled), 256, 0, st>>>((const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled, a.H, a.W, a.C);
+    } else {
+        if (a.C % 4 == 0) maxpool_fwd_kernel<float, 4><<<ew_blocks(pooled / 4), 256, 0, st>>>((const float*)a.x, (float*)a.p, a.idx, pooled / 4, a.H, a.W, a.C);
+        else maxpool_fwd_kernel<float, 1><<<ew_blocks(pooled), 256, 0, st>>>((const float*)a.x, (float*)a.p, a.idx, pooled, a.H, a.W, a.C);
+    }
+    return cudaGetLastError();
+}
+cudaError_t launch_pool_bwd(const PoolBwdArgs& a, bool bf16, cudaStream_t st)
+{
+    long pooled = (long)a.B * (a.H / 2) * (a.W / 2) * a.C;
+    if (bf16) {
+        if (a.C % 8 == 0) maxpool_bwd_kernel<__nv_bfloat16, 8><<<ew_blocks(pooled / 8), 256, 0, st>>>((const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled / 8, a.H, a.W, a.C);
+        else maxpool_bwd_kernel<__nv_bfloat16, 1><<<ew_blocks(pooled), 256, 0, st>>>((const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled, a.H, a.W, a.C);
+    } else {
+        if (a.C % 4 == 0) maxpool_bwd_kernel<float, 4><<<ew_blocks(pooled / 4), 256, 0, st>>>((const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled / 4, a.H, a.W, a.C);
+        else maxpool_bwd_kernel<float, 1><<<ew_blocks(pooled), 256, 0, st>>>((const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled, a.H, a.W, a.C);
+    }
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Softmax cross-entropy: one warp per row (shuffle max / sum), dZ = (softmax - onehot)/B.
+// The last block to finish adds the row losses in row order, so the mean is deterministic.
+// =============================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_rep, float* __restrict__ row_loss,
+                    float* __restrict__ loss, T* __restrict__ dZ, unsigned int* __restrict__ counter, int B, int C)
+{
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int g = blockIdx.x * 8 + warp;
+    if (g < B) {
+        const float* z = logits + (size_t)g * C;
+        const int y = ((const int32_t*)labels.p[g / b_per_rep])[g % b_per_rep];
+        float m = -INFINITY;
+        for (int c = lane; c < C; c += 32) m = fmaxf(m, z[c]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float s = 0.f;
+        for (int c = lane; c < C; c += 32) s += expf(z[c] - m);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float lse = m + logf(s);
+        const float invB = 1.0f / (float)B;
+        for (int c = lane; c < C; c += 32) {
+            float pr = expf(z[c] - lse);
+            stf(dZ + (size_t)g * C + c, (pr - (c == y ? 1.f : 0.f)) * invB);
+        }
+        if (lane == 0) row_loss[g] = (y >= 0 && y < C) ? lse - z[y] : 0.f;
+    }
+    __shared__ bool last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (last && warp == 0) {
+        __threadfence();
+        float t = 0.f;
+        for (int i0 = 0; i0 < B; i0 += 32) {           // fixed order: chunks of 32 rows, tree inside
+            float v = (i0 + lane < B) ? ((volatile float*)row_loss)[i0 + lane] : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            t += v;
+        }
+        if (lane == 0) { *loss = t / (float)B; *counter = 0u; }
+    }
+}
+cudaError_t launch_softmax_xent(const XentArgs& a, bool bf16, cudaStream_t st)
+{
+    int blocks = cdiv(a.B, 8);
+    if (bf16) softmax_xent_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (__nv_bfloat16*)a.dZ, a.counter, a.B, a.C);
+    else softmax_xent_kernel<float><<<blocks, 256, 0, st>>>(a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (float*)a.dZ, a.counter, a.B, a.C);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// SGD with momentum over the whole (padded, 16-byte aligned) parameter arena:
+// v <- mu*v + g ; w <- w - lr*v ; optional bf16 copy of the new w.
+// =============================================================================================
+template <bool SHADOW>
+__global__ void __launch_bounds__(256)
+sgd_kernel(float4* __restrict__ w, float4* __restrict__ v, const float4* __restrict__ g,
+           uint2* __restrict__ shadow, size_t n4, float lr, float mu)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 ww = w[i], vv = v[i], gg = __ldg(g + i);
+        vv.x = fmaf(mu, vv.x, gg.x); vv.y = fmaf(mu, vv.y, gg.y); vv.z = fmaf(mu, vv.z, gg.z); vv.w = fmaf(mu, vv.w, gg.w);
+        ww.x = fmaf(-lr, vv.x, ww.x); ww.y = fmaf(-lr, vv.y, ww.y); ww.z = fmaf(-lr, vv.z, ww.z); ww.w = fmaf(-lr, vv.w, ww.w);
+        v[i] = vv;
+        w[i] = ww;
+        if (SHADOW) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(ww.x, ww.y), hi = __floats2bfloat162_rn(ww.z, ww.w);
+            uint2 pk;
+            pk.x = *(uint32_t*)&lo;
+            pk.y = *(uint32_t*)&hi;
+            shadow[i] = pk;
+        }
+    }
+}
+cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n, float lr, float mu, cudaStream_t st)
+{
+    size_t n4 = n / 4;
+    int blocks = ew_blocks((long)n4);
+    if (shadow) sgd_kernel<true><<<blocks, 256, 0, st>>>((float4*)w, (float4*)v, (const float4*)g, (uint2*)shadow, n4, lr, mu);
+    else sgd_kernel<false><<<blocks, 256, 0, st>>>((float4*)w, (float4*)v, (const float4*)g, nullptr, n4, lr, mu);
+    return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(256)
+to_bf16_kernel(const float4* __restrict__ w, uint2* __restrict__ shadow, size_t n4)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 ww = w[i];
+        __nv_bfloat162 lo = __floats2bfloat162_rn(ww.x, ww.y), hi = __floats2bfloat162_rn(ww.z, ww.w);
+        uint2 pk;
+        pk.x = *(uint32_t*)&lo;
+        pk.y = *(uint32_t*)&hi;
+        shadow[i] = pk;
+    }
+}
+cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cudaStream_t st)
+{
+    to_bf16_kernel<<<ew_blocks((long)(n / 4)), 256, 0, st>>>((const float4*)w, (uint2*)shadow, n / 4);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Strided FFMA GEMM for the sharded FC layers:  C[m,n] = sum_k A(m,k) * B(n,k).
+// 64x64 tile, BK = 16, 256 threads, 4x4 outputs per thread.  blockIdx.z = shard for the
+// partitions that own outputs; the K-partition (dgrad) walks the shards one after another.
+// =============================================================================================
+__device__ __forceinline__ int shard_lo(int j, int total, int shards) { return (int)(((long)j * total) / shards); }
+
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const T* __restrict__ A, long sAm, long sAk, const T* __restrict__ Bm, long sBn, long sBk,
+                 int M, int N, int K, void* __restrict__ Cv, long ldc, float* __restrict__ C32,
+                 const float* __restrict__ bias, int relu, const T* __restrict__ ref, long ldref,
+                 int shard_dim, int shards, PtrTab tab, int tab_mode, int tab_b)
+{
+    __shared__ float As[16][65];
+    __shared__ float Bs[16][65];
+    int m_lo = 0, m_hi = M, n_lo = 0, n_hi = N;
+    if (shard_dim == 1) { n_lo = shard_lo(blockIdx.z, N, shards); n_hi = shard_lo(blockIdx.z + 1, N, shards); }
+    if (shard_dim == 3) { m_lo = shard_lo(blockIdx.z, M, shards); m_hi = shard_lo(blockIdx.z + 1, M, shards); }
+    const int m0 = m_lo + blockIdx.y * 64, n0 = n_lo + blockIdx.x * 64;
+    if (m0 >= m_hi || n0 >= n_hi) return;
+    const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    const int kparts = (shard_dim == 2) ? shards : 1;
+    for (int kp = 0; kp < kparts; ++kp) {
+        const int k_lo = (shard_dim == 2) ? shard_lo(kp, K, shards) : 0;
+        const int k_hi = (shard_dim == 2) ? shard_lo(kp + 1, K, shards) : K;
+        for (int k0 = k_lo; k0 < k_hi; k0 += 16) {
+            for (int e = tid; e < 64 * 16; e += 256) {
+                int mm, kk;
+                if (sAk == 1) { kk = e % 16; mm = e / 16; } else { mm = e % 64; kk = e / 64; }
+                float v = 0.f;
+                if (m0 + mm < m_hi && k0 + kk < k_hi) {
+                    const int m = m0 + mm;
+                    v = (tab_mode == 1) ? ldf((const T*)tab.p[m / tab_b] + (long)(m % tab_b) * sAm + (long)(k0 + kk) * sAk)
+                                        : ldf(A + (long)m * sAm + (long)(k0 + kk) * sAk);
+                }
+                As[kk][mm] = v;
+                int nn;
+                if (sBk == 1) { kk = e % 16; nn = e / 16; } else { nn = e % 64; kk = e / 64; }
+                v = 0.f;
+                if (n0 + nn < n_hi && k0 + kk < k_hi) {
+                    const int k = k0 + kk;
+                    v = (tab_mode == 2) ? ldf((const T*)tab.p[k / tab_b] + (long)(n0 + nn) * sBn + (long)(k % tab_b) * sBk)
+                                        : ldf(Bm + (long)(n0 + nn) * sBn + (long)k * sBk);
+                }
+                Bs[kk][nn] = v;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) {
+                float a[4], b[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
+            __syncthreads();
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int m = m0 + ty * 4 + i;
+        if (m >= m_hi) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int n = n0 + tx * 4 + j;
+            if (n >= n_hi) continue;
+            float v = acc[i][j];
+            if (EPI == EPI_BIAS_ACT) {
+                v += bias[n];
+                if (relu && !(v > 0.f)) v = 0.f;
+                if (C32) C32[(long)m * ldc + n] = v;
+                if (Cv) stf((T*)Cv + (long)m * ldc + n, v);
+            } else if (EPI == EPI_MASK) {
+                if (ref != nullptr && !(ldf(ref + (long)m * ldref + n) > 0.f)) v = 0.f;
+                stf((T*)Cv + (long)m * ldc + n, v);
+            } else {
+                ((float*)Cv)[(long)m * ldc + n] = v;
+            }
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_gemm_simt_t(const GemmSimtArgs& a, cudaStream_t st)
+{
+    int shards = a.shard_dim ? a.shards : 1;
+    int Mmax = a.M, Nmax = a.N, gz = 1;
+    if (a.shard_dim == 1) { Nmax = cdiv(a.N, shards); gz = shards; }
+    if (a.shard_dim == 3) { Mmax = cdiv(a.M, shards); gz = shards; }
+    dim3 grid(cdiv(Nmax, 64), cdiv(Mmax, 64), gz);
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+    const int tab_mode = a.tab ? a.tab_mode : 0;
+#define SB_GM(E)                                                                                                    \
+    gemm_simt_kernel<T, E><<<grid, 256, 0, st>>>((const T*)a.A, a.sAm, a.sAk, (const T*)a.B, a.sBn, a.sBk, a.M, a.N, a.K, \
+                                                 a.C, a.ldc, a.C32, a.bias, a.relu, (const T*)a.ref, a.ldref, a.shard_dim, shards, \
+                                                 tab, tab_mode, a.tab_b > 0 ? a.tab_b : 1)
+    if (a.epi == EPI_BIAS_ACT) SB_GM(EPI_BIAS_ACT);
+    else if (a.epi == EPI_MASK) SB_GM(EPI_MASK);
+    else SB_GM(EPI_F32);
+#undef SB_GM
+    return cudaGetLastError();
+}
+cudaError_t launch_gemm_simt(const GemmSimtArgs& a, bool bf16, cudaStream_t st)
+{
+    return bf16 ? launch_gemm_simt_t<__nv_bfloat16>(a, st) : launch_gemm_simt_t<float>(a, st);
+}
+
+}  // namespace sb

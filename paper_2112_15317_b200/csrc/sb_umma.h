@@ -1,0 +1,61 @@
+// Interface between the host planner (sb_api.cu) and the tcgen05 tensor-core path (sb_umma.cu).
+#pragma once
+
+#include "../../include/splitbrain.h"
+#include "sb_internal.h"
+#include <cuda.h>
+
+namespace sb {
+
+// One planned tensor-core launch: tensor maps, tile geometry and epilogue pointers.
+struct UmmaOp {
+    bool enabled = false;
+    alignas(64) CUtensorMap mapA;
+    alignas(64) CUtensorMap mapB;
+    int params[24] = {0};   // kernel geometry (see sb_umma.cu)
+};
+struct UmmaLayer {
+    UmmaOp fwd, dgrad, wgrad;
+};
+
+// Read-only views of the model for the planner in sb_umma.cu.
+struct ModelView {
+    const sb_config* cfg;
+    bool bf16;
+    int B, n_layers, first_fc;
+    float *Wm, *Gm;
+    __nv_bfloat16* Sm;
+    float* ws;
+    size_t ws_floats;
+    uint32_t* status;
+    char* input_grad;
+    const PtrTab* x_tab;
+};
+struct LayerView {
+    int kind, H, W, Cin, Cout, in_f, out_f;
+    bool relu;
+    size_t p_w, p_b, n_w, n_b;
+    char *act, *dact;
+    const char* in_act;   // previous layer's output (nullptr for layer 0)
+    char* d_below;        // where the input gradient goes
+    bool below_relu;
+    UmmaLayer* um;
+};
+ModelView model_view(sb_model* m);
+LayerView layer_view(sb_model* m, int i);
+int64_t* launch_counter(sb_model* m);
+
+// Scratch floats the tensor-core path needs (split partial sums); called during planning,
+// before the arena exists (pointers in the views are null or unset).
+sb_status umma_plan_scratch(sb_model* m, size_t* floats);
+// Encodes tensor maps and decides, per layer and pass, whether the tensor-core kernel runs.
+sb_status umma_plan_layers(sb_model* m);
+
+sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st);
+sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st);
+sb_status umma_conv_wgrad(sb_model* m, int layer, cudaStream_t st);   // counts its own launches
+sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
+sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
+sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
+
+}  // namespace sb

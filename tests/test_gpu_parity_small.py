@@ -1,0 +1,168 @@
+"""GPU parity, small sizes: the CUDA library (through the C ABI) against the CPU oracle on the same
+seeded inputs, element by element.  Tolerances are the contract's: max|err|/max|ref| <= 1e-4 in
+float mode, <= 1e-2 in bf16-operand mode; integer results (pool argmax) bit-exact."""
+import numpy as np
+import pytest
+
+import sb_inputs as si
+from sb_testutil import device_batch, frob, gpu_model, maxrel, oracle_model, outlier_fraction
+
+pytestmark = pytest.mark.gpu
+
+TOL = {False: 1e-4, True: 1e-2}
+
+
+def sb():
+    from paper_2112_15317_b200 import binding
+    return binding
+
+
+def ragged_net(classes=7):
+    # channel counts that are not multiples of the CUDA-core tiles, conv->conv, pool->conv, conv->fc paths
+    return [(si.CONV3X3_RELU, 24), (si.CONV3X3_RELU, 40), (si.MAXPOOL2, 0), (si.CONV3X3_RELU, 16), (si.MAXPOOL2, 0),
+            (si.CONV3X3_RELU, 8), (si.FC_RELU, 70), (si.FC_RELU, 33), (si.FC, classes), (si.SOFTMAX_XENT, classes)]
+
+
+WORKLOADS = {
+    "cfg0": lambda: si.config(0),
+    "ragged": lambda: si.Workload("ragged", ragged_net(), 20, 12, 4, 3, 2, 3),
+}
+
+
+def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
+    b = sb()
+    params = si.make_params(wl, bias_std=bias_std)
+    x, y = si.make_batch(wl)
+    om = oracle_model(wl, params, bf16)
+    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32)
+    xs, ys = device_batch(wl, x, y, bf16)
+    xr, yr = si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)
+    tol = TOL[bf16]
+    report = {}
+    for step in range(steps):
+        lo = om.forward(xr, yr)
+        om.backward()
+        gm.forward(xs, ys)
+        gm.backward()
+        lg = gm.loss()
+        assert abs(lg - float(lo)) <= tol * max(1.0, abs(float(lo))), (step, lg, lo)
+        nl = len(wl.layers)
+        for li, (kind, out) in enumerate(wl.layers):
+            if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
+                for r in range(wl.R):
+                    a = gm.read(b.SB_T_ACT, li, r, squeeze=False)
+                    assert maxrel(a, om.conv_out[r][li]) <= tol, ("act", step, li, r)
+                    d = gm.read(b.SB_T_DACT, li, r, squeeze=False)
+                    ref = om.d_conv[r][li]
+                    if bf16:
+                        # a rounding-order flip of a ReLU mask / pool argmax moves single elements: bound the
+                        # norm and the number of outliers instead of the single worst element
+                        assert frob(d, ref) <= tol and outlier_fraction(d, ref, tol) <= 2e-3, ("dact", step, li, r, frob(d, ref))
+                    else:
+                        assert maxrel(d, ref) <= tol, ("dact", step, li, r)
+                    if kind == si.MAXPOOL2:
+                        idx = gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)
+                        mism = float(np.mean(idx != om.pool_idx[r][li]))
+                        assert mism <= (1e-3 if bf16 else 0.0), ("pool idx", step, li, r, mism)
+            elif kind in (si.FC_RELU, si.FC):
+                a = gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0]
+                assert maxrel(a, om.fc_out[li]) <= tol, ("fc act", step, li)
+                d = gm.read(b.SB_T_DACT, li, 0, squeeze=False)[:, :, 0, 0]
+                if bf16:
+                    assert frob(d, om.d_pre[li]) <= tol, ("fc dact", step, li)
+                else:
+                    assert maxrel(d, om.d_pre[li]) <= tol, ("fc dact", step, li)
+        rl = gm.read(b.SB_T_ROW_LOSS, nl - 1, 0)
+        assert maxrel(rl, om.row_loss) <= tol
+        gg = gm.gather_params(b.SB_T_GRAD_W, b.SB_T_GRAD_B)
+        for li, (a, ref) in enumerate(zip(gg, om.full_grads())):
+            if ref is not None:
+                report[("gw", step, li)] = maxrel(a["w"].reshape(ref["w"].shape), ref["w"])
+                assert report[("gw", step, li)] <= tol, ("grad w", step, li, report[("gw", step, li)])
+                assert maxrel(a["b"], ref["b"]) <= tol, ("grad b", step, li)
+        om.sgd_step(lr, mu)
+        gm.sgd_step(lr, mu)
+        for what_w, what_b, ref_list in ((b.SB_T_WEIGHT, b.SB_T_BIAS, om.full_params()), (b.SB_T_MOM_W, b.SB_T_MOM_B, om.full_mom())):
+            got = gm.gather_params(what_w, what_b)
+            for li, (a, ref) in enumerate(zip(got, ref_list)):
+                if ref is not None:
+                    assert maxrel(a["w"].reshape(ref["w"].shape), ref["w"]) <= tol, ("param/mom w", step, li)
+                    assert maxrel(a["b"], ref["b"]) <= max(tol, 0) or np.max(np.abs(ref["b"])) == 0, ("param/mom b", step, li)
+    gm.close()
+    return report
+
+
+@pytest.mark.parametrize("name", list(WORKLOADS))
+@pytest.mark.parametrize("bf16", [False, True])
+def test_two_training_steps_match_oracle(name, bf16):
+    compare_everything(WORKLOADS[name](), bf16, steps=2, bias_std=0.2)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_cfg0_contract_one_step_zero_bias(bf16):
+    """The benchmark's first configuration exactly as stated: one step, lr 0.01, momentum 0.9, zero biases."""
+    compare_everything(si.config(0), bf16, steps=1, lr=0.01, mu=0.9, bias_std=0.0)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_partition_invariance_on_gpu(bf16):
+    """Loss, gradients and updated weights for (R,K) partitions equal the unpartitioned R=K=1 run."""
+    b = sb()
+    base = si.Workload("inv", ragged_net(), 12, 12, 4, 8, 1, 1)
+    params = si.make_params(base, bias_std=0.2)
+    x, y = si.make_batch(base)
+    results = {}
+    for R, K in [(1, 1), (2, 3), (4, 2), (8, 7)]:
+        wl = base.with_partition(R, K)
+        gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32)
+        xs, ys = device_batch(wl, x, y, bf16)
+        gm.forward(xs, ys); gm.backward(); loss = gm.loss(); gm.sgd_step(0.05, 0.9)
+        logits = gm.read(b.SB_T_ACT, len(wl.layers) - 2, 0, squeeze=False)[:, :, 0, 0]
+        results[(R, K)] = (loss, logits, gm.gather_params(b.SB_T_GRAD_W, b.SB_T_GRAD_B), gm.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS))
+        gm.close()
+    l0, z0, g0, w0 = results[(1, 1)]
+    for key, (l, z, g, w) in results.items():
+        assert np.array_equal(z, z0), key            # forward is bit-identical under re-partitioning
+        assert l == pytest.approx(l0, rel=1e-6)
+        for a, ref in zip(g, g0):
+            if ref is not None:
+                assert maxrel(a["w"], ref["w"]) <= 1e-5 and maxrel(a["b"], ref["b"]) <= 1e-5, key
+        for a, ref in zip(w, w0):
+            if ref is not None:
+                assert maxrel(a["w"], ref["w"]) <= 1e-6, key
+
+
+def test_train_step_host_matches_device_path():
+    import torch
+    b = sb()
+    wl = si.config(0)
+    params = si.make_params(wl)
+    x, y = si.make_batch(wl)
+    g1 = gpu_model(wl, params, b.SB_BF16)
+    g2 = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    hx = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    hy = torch.from_numpy(y).pin_memory()
+    for _ in range(2):
+        g1.forward(xs, ys); g1.backward(); g1.sgd_step(0.01, 0.9); l1 = g1.loss()
+        l2 = g2.train_step_host(hx, hy, 0.01, 0.9)
+        assert l1 == l2
+    for a, c in zip(g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), g2.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"])
+    assert g1.launch_count() > 10
+    g1.close(); g2.close()
+
+
+def test_state_and_argument_errors():
+    b = sb()
+    wl = si.config(0)
+    gm = gpu_model(wl, si.make_params(wl), b.SB_FP32)
+    with pytest.raises(b.SBError) as e:
+        gm.backward()
+    assert e.value.status == 6
+    with pytest.raises(b.SBError):
+        gm.read(b.SB_T_WEIGHT, 1, 0)          # pooling layer has no parameters
+    with pytest.raises(b.SBError):
+        gm.read(b.SB_T_WEIGHT, 4, 5)          # shard out of range
+    gm.close()
