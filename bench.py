@@ -1,0 +1,295 @@
+#!/usr/bin/env python
+"""Benchmark of the SplitBrain hybrid-parallel training step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1|2|3]
+
+One "step" = forward + backward + SGD-momentum update of the whole network on one batch of
+synthetic images (sb_forward, sb_backward, sb_sgd_step through the C ABI).  Prints ONE JSON line:
+training images/s (device-timed, inputs resident in HBM), the end-to-end figure through
+sb_train_step_host (pinned host buffers, H2D copies and the loss read-back inside the timed
+region), the roofline of the dominant kernel class (timed live with CUDA events by the library's
+profiling hooks), the SM clocks sampled during the timed region, and the CPU oracle timed on a
+bounded sample of the same workload.
+
+N > 1 (launched by torch.distributed.run): every rank trains its own independent copy of the
+workload on its own GPU ("replicas only": the build has no cross-GPU exchange step), the time is
+the max over ranks, the value the sum of all ranks' images.
+
+--impl reference times the CPU oracle as it stands (bounded sample per step) and prints the same
+line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import sb_inputs as si  # noqa: E402
+
+METRIC = "training images/sec (VGG-16 CIFAR shape)"
+UNIT = "images/s"
+LR, MU = 0.01, 0.9
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+def workload(cfg_id: int):
+    wl = si.config(cfg_id)
+    return wl
+
+
+def oracle_sample(wl):
+    """Bounded sample of the workload for the CPU oracle: same network, R and K, one image per replica."""
+    return wl.with_batch(1, name=wl.name + "_b1sample")
+
+
+def time_oracle(wl, steps, warmup):
+    from oracle import splitbrain_oracle as so
+    sw = oracle_sample(wl)
+    params = si.make_params(sw)
+    x, y = si.make_batch(sw)
+    m = so.from_workload(sw, real="float", bf16=True)
+    m.load_params(params)
+    xr, yr = si.split_replicas(x, sw.R), si.split_replicas(y, sw.R)
+    for _ in range(warmup):
+        m.step(xr, yr, LR, MU)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        m.step(xr, yr, LR, MU)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    omp = os.environ.get("OMP_NUM_THREADS")
+    if omp:
+        cores = min(cores, int(omp))
+    return dict(value=sw.B / dt, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{steps} step(s) of {sw.name}: batch {sw.B} (R={sw.R} x b=1, K={sw.K}), full network, fwd+bwd+sgd, {dt:.2f} s/step"), dt, sw
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[4:8]):
+                if v.strip().lower() == "active":
+                    reasons.add(nm)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as ge
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    if rank == 0:
+        ge.build()
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        dist.barrier()
+    torch.cuda.set_device(local)
+    from paper_2112_15317_b200 import binding as sb
+
+    wl = workload(args.config)
+    params = si.make_params(wl)
+    x, y = si.make_batch(wl, seed=si.SEED_DATA + rank)
+    m = sb.Model.from_workload(wl, precision=sb.SB_BF16, device=f"cuda:{local}")
+    m.load_params(params, si.shard_bounds)
+    xs = [torch.from_numpy(a).cuda().to(torch.bfloat16) for a in si.split_replicas(x, wl.R)]
+    ys = [torch.from_numpy(a).cuda() for a in si.split_replicas(y, wl.R)]
+    hx = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    hy = torch.from_numpy(y).pin_memory()
+
+    def step():
+        m.forward(xs, ys)
+        m.backward()
+        m.sgd_step(LR, MU)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    loss_w = m.loss()
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    loss_t = m.loss()
+
+    # end to end through the host-buffer entry point
+    for _ in range(max(1, min(args.warmup, 3))):
+        m.train_step_host(hx, hy, LR, MU)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        m.train_step_host(hx, hy, LR, MU)
+    torch.cuda.synchronize()
+    ms_e2e = (time.perf_counter() - t0) * 1e3
+    barrier()
+
+    # per-kernel-class timing (events around every launch), same steps again
+    m.profile_begin()
+    for _ in range(args.steps):
+        step()
+    prof = m.profile_end()
+    launches = m.launch_count()
+
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    pk = peaks()
+    ms_step = ms / args.steps
+    imgs = wl.B * world
+    value = imgs / (ms_step * 1e-3)
+    # roofline of the dominant kernel class
+    prof.sort(key=lambda r: -r["ms_total"])
+    tot_ms = sum(r["ms_total"] for r in prof) or 1.0
+    top = prof[0]
+    sec = top["ms_total"] * 1e-3
+    t_flop = top["flops"] / (pk["tf_sustained"] * 1e12)
+    t_byte = top["bytes"] / (pk["hbm_gbs"] * 1e9)
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tp):
+        traffic = json.load(open(tp)).get(f"{wl.name}:{top['name']}")
+    if t_flop >= t_byte:
+        roof = dict(bound="tensor", achieved=top["flops"] / sec / 1e12, peak=pk["tf_sustained"], unit="TFLOP/s")
+    else:
+        roof = dict(bound="hbm", achieved=top["bytes"] / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update(kernel=top["name"], launches_per_step=top["launches"] // args.steps, share_of_kernel_time=top["ms_total"] / tot_ms,
+                traffic=traffic, peak_source=pk["source"] + (" sustained bf16" if roof["bound"] == "tensor" else " copy"),
+                avg_launch_us=top["ms_total"] * 1e3 / top["launches"])
+    # whole-step roofline (the slower of all FLOPs at tensor peak and all bytes at HBM peak)
+    fl = sum(r["flops"] for r in prof) / args.steps
+    by = sum(r["bytes"] for r in prof) / args.steps
+    t_roof = max(fl / (pk["tf_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9))
+    kernels = [dict(name=r["name"], launches_per_step=r["launches"] // args.steps, ms_per_step=r["ms_total"] / args.steps,
+                    tflops=(r["flops"] / (r["ms_total"] * 1e-3) / 1e12 if r["flops"] else None),
+                    gbs=r["bytes"] / (r["ms_total"] * 1e-3) / 1e9) for r in prof]
+    cpu = None
+    if world == 1:
+        cpu, _, _ = time_oracle(wl, steps=2, warmup=0)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "network": "VGG-16 (13 conv3x3 + 3 FC), 32x32x3 inputs, 10 classes",
+                   "global_batch": imgs, "batch_per_gpu": wl.B, "R": wl.R, "K": wl.K, "b": wl.b,
+                   "precision": "bf16 operands, fp32 accumulate, fp32 master weights",
+                   "l2": "per-step working set (activations+gradients+weights, >1 GB) exceeds the 126 MB L2; no flush",
+                   "parallelism": "1 GPU: R logical replicas x K logical shards" if world == 1 else f"{world} independent replicas of the 1-GPU job"},
+        "e2e": {"value": imgs / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(hx.numel() * 2 + hy.numel() * 4), "d2h_bytes_per_step": 8},
+        "gpu_launches": int(launches * args.steps),
+        "clocks": clocks,
+        "roofline": roof,
+        "step_roofline": {"flops_per_step": fl, "bytes_per_step": by, "roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step},
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+        "loss": {"after_warmup": loss_w, "after_timed": loss_t},
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    import __graft_entry__ as ge  # noqa: F401  (builds the C oracle on demand through the oracle package)
+    wl = workload(args.config)
+    cpu, dt, sw = time_oracle(wl, steps=args.steps, warmup=args.warmup)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": cpu["sample"]},
+        "cpu_baseline": cpu,
+        "e2e": {"value": cpu["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

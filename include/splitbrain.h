@@ -201,6 +201,26 @@ sb_status sb_backward_layers(sb_model* m, int32_t last, int32_t first, void* str
  */
 sb_status sb_param_bytes(const sb_model* m, int32_t shard, size_t* bytes);
 
+/*
+ * Per-kernel timing with CUDA events on the launching stream.  sb_profile_begin switches event
+ * recording on: every kernel the library enqueues afterwards is bracketed by two events (this
+ * serialises nothing but adds launch overhead, so whole-step timings should be taken with
+ * profiling off).  sb_profile_end synchronises the stream, switches recording off and returns one
+ * entry per kernel class with its launch count, total device time, and the ALGORITHMIC work of
+ * those launches: flops = 2*M*N*K of the contractions; bytes = every operand read once and every
+ * result written once (no im2col expansion, no padding, no re-reads).
+ *   out : HOST array of max_entries entries;  n : HOST, receives the number written.
+ */
+typedef struct {
+    char name[32];      /* kernel class, e.g. "conv_fwd_umma", "sgd", "pool_bwd" */
+    int32_t launches;
+    float ms_total;
+    double flops;
+    double bytes;
+} sb_profile_entry;
+sb_status sb_profile_begin(sb_model* m, void* stream);
+sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32_t max_entries, int32_t* n);
+
 /* Number of kernels the last sb_forward + sb_backward + sb_sgd_step enqueued (host counter). */
 sb_status sb_launch_count(const sb_model* m, int64_t* launches);
 

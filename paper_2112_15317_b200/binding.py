@@ -37,6 +37,11 @@ class sb_config(ctypes.Structure):
                 ("R", c_int32), ("K", c_int32), ("precision", c_int32), ("flags", c_int32)]
 
 
+class sb_profile_entry(ctypes.Structure):
+    _fields_ = [("name", ctypes.c_char * 32), ("launches", c_int32), ("ms_total", c_float),
+                ("flops", ctypes.c_double), ("bytes", ctypes.c_double)]
+
+
 class SBError(RuntimeError):
     def __init__(self, status, msg):
         super().__init__(f"{STATUS_NAMES.get(status, status)}: {msg}")
@@ -67,6 +72,8 @@ def _load():
         "sb_backward_layers": [c_void_p, c_int32, c_int32, c_void_p],
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
         "sb_launch_count": [c_void_p, P(c_int64)],
+        "sb_profile_begin": [c_void_p, c_void_p],
+        "sb_profile_end": [c_void_p, c_void_p, P(sb_profile_entry), c_int32, P(c_int32)],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -97,6 +104,8 @@ sb_forward_layers = _lib.sb_forward_layers
 sb_backward_layers = _lib.sb_backward_layers
 sb_param_bytes = _lib.sb_param_bytes
 sb_launch_count = _lib.sb_launch_count
+sb_profile_begin = _lib.sb_profile_begin
+sb_profile_end = _lib.sb_profile_end
 
 
 def sb_last_error() -> str:
@@ -280,6 +289,17 @@ class Model:
         v = c_size_t()
         _check(sb_param_bytes(self.h, shard, byref(v)))
         return v.value
+
+    def profile_begin(self):
+        _check(sb_profile_begin(self.h, self._stream()))
+
+    def profile_end(self):
+        """Per kernel class: {'name', 'launches', 'ms_total', 'flops', 'bytes'} (algorithmic work)."""
+        arr = (sb_profile_entry * 64)()
+        n = c_int32()
+        _check(sb_profile_end(self.h, self._stream(), arr, 64, byref(n)))
+        return [dict(name=arr[i].name.decode(), launches=arr[i].launches, ms_total=arr[i].ms_total,
+                     flops=arr[i].flops, bytes=arr[i].bytes) for i in range(n.value)]
 
     def launch_count(self) -> int:
         v = c_int64()

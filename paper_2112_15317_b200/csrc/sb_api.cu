@@ -81,6 +81,25 @@ struct sb_model {
     PtrTab x_tab{}, label_tab{};
     bool have_x = false, have_labels = false, have_fwd = false;
     int64_t launches = 0, last_step_launches = 0;
+    // per-launch event recording (sb_profile_begin / sb_profile_end)
+    struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; };
+    bool profiling = false;
+    std::vector<Rec> recs;
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used = 0;
+    cudaEvent_t next_event()
+    {
+        if (ev_used == ev_pool.size()) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+            ev_pool.push_back(e);
+        }
+        return ev_pool[ev_used++];
+    }
+    ~sb_model()
+    {
+        for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
+    }
 };
 
 namespace {
@@ -203,11 +222,27 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
 
 inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / K); }
 
-#define L_TRY(expr)                                                                               \
+// Every kernel launch goes through here: counts it and, when profiling, brackets it with events.
+// `tag` names the kernel class; flops/bytes are the algorithmic work of this launch.
+#define L_TRY(tag, flops, bytes, expr)                                                            \
     do {                                                                                          \
+        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes)};              \
+        if (m->profiling) { rec_.e0 = m->next_event(); rec_.e1 = m->next_event();                 \
+                            if (rec_.e0) cudaEventRecord(rec_.e0, st); }                          \
         cudaError_t e_ = (expr);                                                                  \
         ++m->launches;                                                                            \
         if (e_ != cudaSuccess) return fail(SB_ERR_CUDA, "launch failed in %s: %s", #expr, cudaGetErrorString(e_)); \
+        if (m->profiling && rec_.e1) { cudaEventRecord(rec_.e1, st); m->recs.push_back(rec_); }   \
+    } while (0)
+// Same bracket for the tensor-core launchers, which return sb_status.
+#define U_TRY(tag, flops, bytes, expr)                                                            \
+    do {                                                                                          \
+        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes)};              \
+        if (m->profiling) { rec_.e0 = m->next_event(); rec_.e1 = m->next_event();                 \
+                            if (rec_.e0) cudaEventRecord(rec_.e0, st); }                          \
+        sb_status s_ = (expr);                                                                    \
+        if (s_ != SB_OK) return s_;                                                               \
+        if (m->profiling && rec_.e1) { cudaEventRecord(rec_.e1, st); m->recs.push_back(rec_); }   \
     } while (0)
 
 // Which buffer holds the input of layer i: the previous layer's output, or the caller's images.
@@ -218,13 +253,16 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
     Layer& l = m->L[i];
     const bool bf = m->bf16;
     const int B = m->B, b = m->cfg.batch_per_replica;
+    const double e = (double)m->esz;
     const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
     switch (l.kind) {
     case SB_CONV3X3_RELU: {
         if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        const double pix = (double)B * l.H * l.W;
+        const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
+        const double bytes = pix * l.Cin * e + (double)l.n_w * e + pix * l.Cout * e;
         if (l.um.fwd.enabled) {
-            sb_status s = umma_conv_fwd(m, i, st);
-            if (s != SB_OK) return s;
+            U_TRY("conv_fwd_umma", flops, bytes, umma_conv_fwd(m, i, st));
             ++m->launches;
             break;
         }
@@ -232,20 +270,22 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.in = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
         a.w = wts; a.bias = m->Wm + l.p_b; a.out = l.act; a.mask_ref = nullptr;
         a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 0; a.relu = 1;
-        L_TRY(launch_conv_simt(a, bf, st));
+        L_TRY("conv_fwd_simt", flops, bytes, launch_conv_simt(a, bf, st));
         break;
     }
     case SB_MAXPOOL2: {
         PoolArgs a{layer_input(m, i), l.act, l.idx, B, l.H, l.W, l.Cin};
-        L_TRY(launch_pool_fwd(a, bf, st));
+        const double pooled = (double)B * l.out_per_img;
+        L_TRY("pool_fwd", 0.0, pooled * (4 * e + e + 1), launch_pool_fwd(a, bf, st));
         break;
     }
     case SB_FC_RELU:
     case SB_FC: {
         if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        const double flops = 2.0 * B * (double)l.in_f * l.out_f;
+        const double bytes = (double)B * l.in_f * e + (double)l.n_w * e + (double)B * l.out_f * (l.kind == SB_FC ? 4.0 : e);
         if (l.um.fwd.enabled) {
-            sb_status s = umma_fc_fwd(m, i, st);
-            if (s != SB_OK) return s;
+            U_TRY("fc_fwd_umma", flops, bytes, umma_fc_fwd(m, i, st));
             ++m->launches;
             break;
         }
@@ -257,7 +297,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         if (l.kind == SB_FC) { a.C = nullptr; a.C32 = (float*)l.act; } else { a.C = l.act; a.C32 = nullptr; }
         a.shard_dim = 1; a.shards = m->cfg.K;
         if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 1; a.tab_b = b; }
-        L_TRY(launch_gemm_simt(a, bf, st));
+        L_TRY("fc_fwd_simt", flops, bytes, launch_gemm_simt(a, bf, st));
         break;
     }
     case SB_SOFTMAX_XENT: {
@@ -267,7 +307,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.logits = (const float*)fc.act; a.labels = m->label_tab; a.b_per_rep = b;
         a.row_loss = m->row_loss; a.loss = m->loss; a.dZ = fc.dact; a.counter = m->counter;
         a.B = B; a.C = l.out;
-        L_TRY(launch_softmax_xent(a, bf, st));
+        L_TRY("softmax_xent", 0.0, (double)B * l.out * (4.0 + e) + 8.0 * B, launch_softmax_xent(a, bf, st));
         break;
     }
     }
@@ -279,6 +319,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
     Layer& l = m->L[i];
     const bool bf = m->bf16;
     const int B = m->B, b = m->cfg.batch_per_replica;
+    const double e = (double)m->esz;
     const bool want_in_grad = i > 0 || (m->cfg.flags & SB_FLAG_INPUT_GRAD);
     // where the gradient w.r.t. this layer's input goes, and whether the layer below applied a ReLU
     char* d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
@@ -290,10 +331,11 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
     case SB_FC_RELU:
     case SB_FC: {
         if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        const double flops = 2.0 * B * (double)l.in_f * l.out_f;
+        const double act_bytes = (double)B * (l.in_f + l.out_f) * e;
         // weight gradient per shard: dW_j = dY_j^T X   (rows c_j..c_{j+1} of the [out,in] gradient)
         if (l.um.wgrad.enabled) {
-            sb_status s = umma_fc_wgrad(m, i, st);
-            if (s != SB_OK) return s;
+            U_TRY("fc_wgrad_umma", flops, act_bytes + (double)l.n_w * 4.0, umma_fc_wgrad(m, i, st));
             ++m->launches;
         } else {
             GemmSimtArgs a{};
@@ -303,14 +345,14 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             a.epi = EPI_F32; a.C = m->Gm + l.p_w; a.ldc = l.in_f;
             a.shard_dim = 3; a.shards = m->cfg.K;
             if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 2; a.tab_b = b; }
-            L_TRY(launch_gemm_simt(a, bf, st));
+            L_TRY("fc_wgrad_simt", flops, act_bytes + (double)l.n_w * 4.0, launch_gemm_simt(a, bf, st));
         }
-        L_TRY(launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
+        L_TRY("bias_grad", 0.0, (double)B * l.out_f * e + 4.0 * l.out_f, launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
         if (want_in_grad) {
             // shard-layer / modulo-layer backward: dX = sum_j dY_j W_j, rows stay with their replica
+            const double bytes = act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0);
             if (l.um.dgrad.enabled) {
-                sb_status s = umma_fc_dgrad(m, i, st);
-                if (s != SB_OK) return s;
+                U_TRY("fc_dgrad_umma", flops, bytes, umma_fc_dgrad(m, i, st));
                 ++m->launches;
             } else {
                 GemmSimtArgs a{};
@@ -320,18 +362,21 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
                 a.epi = EPI_MASK; a.C = d_below; a.ldc = l.in_f;
                 a.ref = below_relu ? m->L[i - 1].act : nullptr; a.ldref = l.in_f;
                 a.shard_dim = 2; a.shards = m->cfg.K;
-                L_TRY(launch_gemm_simt(a, bf, st));
+                L_TRY("fc_dgrad_simt", flops, bytes, launch_gemm_simt(a, bf, st));
             }
         }
         break;
     }
     case SB_MAXPOOL2: {
         PoolBwdArgs a{l.dact, l.idx, below_relu ? l.act : nullptr, d_below, B, l.H, l.W, l.Cin};
-        L_TRY(launch_pool_bwd(a, bf, st));
+        const double pooled = (double)B * l.out_per_img;
+        L_TRY("pool_bwd", 0.0, pooled * (e + 1 + (below_relu ? e : 0.0) + 4 * e), launch_pool_bwd(a, bf, st));
         break;
     }
     case SB_CONV3X3_RELU: {
         if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
+        const double pix = (double)B * l.H * l.W;
+        const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
         // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
         if (l.um.wgrad.enabled) {
             sb_status s = umma_conv_wgrad(m, i, st);
@@ -342,8 +387,8 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
             a.dy = l.dact; a.part = S > 1 ? m->ws : m->Gm + l.p_w;
             a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
-            L_TRY(launch_wgrad_simt(a, bf, st));
-            if (S > 1) L_TRY(launch_reduce_partials(m->ws, m->Gm + l.p_w, l.n_w, S, st));
+            L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws, m->Gm + l.p_w, l.n_w, S, st));
         }
         {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
@@ -352,13 +397,13 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             while (S * 2 <= B && B % (S * 2) == 0 && (long)S * ((l.Cout + 31) / 32) < 148 * 2) S *= 2;
             float* part = S > 1 ? m->ws + (size_t)l.wg_splits * l.n_w : m->Gm + l.p_b;
             if ((size_t)l.wg_splits * l.n_w + (size_t)S * l.n_b > m->ws_floats) { S = 1; part = m->Gm + l.p_b; }
-            L_TRY(launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
-            if (S > 1) L_TRY(launch_reduce_partials(part, m->Gm + l.p_b, l.n_b, S, st));
+            L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, m->Gm + l.p_b, l.n_b, S, st));
         }
         if (want_in_grad) {
+            const double bytes = pix * (l.Cin + l.Cout) * e + (double)l.n_w * e + (below_relu ? pix * l.Cin * e : 0.0);
             if (l.um.dgrad.enabled) {
-                sb_status s = umma_conv_dgrad(m, i, st);
-                if (s != SB_OK) return s;
+                U_TRY("conv_dgrad_umma", flops, bytes, umma_conv_dgrad(m, i, st));
                 ++m->launches;
             } else {
                 ConvSimtArgs a{};
@@ -366,7 +411,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
                 a.w = wts; a.bias = nullptr; a.out = d_below;
                 a.mask_ref = below_relu ? m->L[i - 1].act : nullptr;
                 a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 1; a.relu = 0;
-                L_TRY(launch_conv_simt(a, bf, st));
+                L_TRY("conv_dgrad_simt", flops, bytes, launch_conv_simt(a, bf, st));
             }
         }
         break;
@@ -596,7 +641,8 @@ sb_status sb_backward(sb_model* m, void* stream)
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
-    L_TRY(launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, m->P, lr, momentum, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    L_TRY("sgd", 0.0, (double)m->P * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, m->P, lr, momentum, st));
     m->last_step_launches = m->launches;
     return SB_OK;
 }
@@ -604,7 +650,8 @@ sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)
 sb_status sb_refresh_shadow(sb_model* m, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
-    if (m->bf16) L_TRY(launch_to_bf16(m->Wm, m->Sm, m->P, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (m->bf16) L_TRY("to_bf16", 0.0, (double)m->P * 6.0, launch_to_bf16(m->Wm, m->Sm, m->P, st));
     return SB_OK;
 }
 
@@ -693,6 +740,45 @@ sb_status sb_param_bytes(const sb_model* m, int32_t shard, size_t* bytes)
         }
     }
     *bytes = n * 4;
+    return SB_OK;
+}
+
+sb_status sb_profile_begin(sb_model* m, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    (void)stream;
+    m->profiling = true;
+    m->recs.clear();
+    m->ev_used = 0;
+    return SB_OK;
+}
+
+sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32_t max_entries, int32_t* n)
+{
+    if (!m || !out || !n || max_entries < 1) return fail(SB_ERR_INVALID_ARG, "null argument");
+    m->profiling = false;
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    int cnt = 0;
+    for (const sb_model::Rec& r : m->recs) {
+        float ms = 0.f;
+        CU_TRY(cudaEventElapsedTime(&ms, r.e0, r.e1));
+        int k = 0;
+        for (; k < cnt; ++k)
+            if (strncmp(out[k].name, r.tag, sizeof(out[k].name)) == 0) break;
+        if (k == cnt) {
+            if (cnt == max_entries) continue;
+            memset(&out[k], 0, sizeof(out[k]));
+            strncpy(out[k].name, r.tag, sizeof(out[k].name) - 1);
+            ++cnt;
+        }
+        out[k].launches += 1;
+        out[k].ms_total += ms;
+        out[k].flops += r.flops;
+        out[k].bytes += r.bytes;
+    }
+    m->recs.clear();
+    m->ev_used = 0;
+    *n = cnt;
     return SB_OK;
 }
 
