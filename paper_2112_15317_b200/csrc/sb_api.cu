@@ -50,7 +50,8 @@ struct Layer {
     char* act = nullptr;                        // [B, out_per_img] activation dtype (float for the logits layer)
     char* dact = nullptr;                       // same shape, activation dtype
     uint8_t* idx = nullptr;                     // pool argmax
-    int wg_splits = 1;                          // conv wgrad pixel-range splits
+    int wg_splits = 1;                          // conv wgrad pixel-range splits (CUDA-core kernel)
+    int bg_splits = 1;                          // conv bias-gradient row splits
     int act_dt = SB_DT_F32;
     UmmaLayer um;                               // tensor-core plan of this layer (tcgen05 path)
 };
@@ -199,8 +200,12 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
             int s = 1;
             while (tiles * s < 148 * 4 && s * 2 <= (int)B && B % (s * 2) == 0) s *= 2;
             l.wg_splits = s;
-            size_t need = (size_t)s * (l.n_w + l.n_b);
+            size_t need = (size_t)s * l.n_w;
             if (need > ws_floats) ws_floats = need;
+            int sb_ = 1;
+            while (sb_ * 2 <= (int)B && B % (sb_ * 2) == 0 && (long)sb_ * ((l.Cout + 31) / 32) < 148 * 2) sb_ *= 2;
+            l.bg_splits = sb_;
+            if ((size_t)sb_ * l.n_b > ws_floats) ws_floats = (size_t)sb_ * l.n_b;
         }
     }
     size_t um_ws = 0;
@@ -241,7 +246,7 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
         if (m->profiling) { rec_.e0 = m->next_event(); rec_.e1 = m->next_event();                 \
                             if (rec_.e0) cudaEventRecord(rec_.e0, st); }                          \
         sb_status s_ = (expr);                                                                    \
-        if (s_ != SB_OK) return s_;                                                               \
+        if (s_ != SB_OK) return fail(s_, "%s", umma_last_error());                                                            \
         if (m->profiling && rec_.e1) { cudaEventRecord(rec_.e1, st); m->recs.push_back(rec_); }   \
     } while (0)
 
@@ -379,8 +384,11 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
         // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
         if (l.um.wgrad.enabled) {
-            sb_status s = umma_conv_wgrad(m, i, st);
-            if (s != SB_OK) return s;
+            int S = 1;
+            float* part = nullptr;
+            U_TRY("conv_wgrad_umma", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, umma_conv_wgrad_launch(m, i, st, &S, &part));
+            ++m->launches;
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(part, m->Gm + l.p_w, l.n_w, S, st));
         } else {
             const int S = l.wg_splits;
             WgradSimtArgs a{};
@@ -393,10 +401,9 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
             const long M = (long)B * l.H * l.W;
-            int S = 1;
-            while (S * 2 <= B && B % (S * 2) == 0 && (long)S * ((l.Cout + 31) / 32) < 148 * 2) S *= 2;
-            float* part = S > 1 ? m->ws + (size_t)l.wg_splits * l.n_w : m->Gm + l.p_b;
-            if ((size_t)l.wg_splits * l.n_w + (size_t)S * l.n_b > m->ws_floats) { S = 1; part = m->Gm + l.p_b; }
+            // (stream order makes it safe to reuse the scratch the weight-gradient reduce just read)
+            const int S = l.bg_splits;
+            float* part = S > 1 ? m->ws : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
             if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, m->Gm + l.p_b, l.n_b, S, st));
         }
@@ -574,7 +581,7 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }
     s = umma_plan_layers(m);
-    if (s != SB_OK) { delete m; return s; }
+    if (s != SB_OK) { delete m; return fail(s, "tensor-core planning failed: %s", umma_last_error()); }
     *out = m;
     return SB_OK;
 }

@@ -1,12 +1,750 @@
-// tcgen05 tensor-core path (placeholder: every layer falls back to the CUDA-core kernels).
+// tcgen05 / TMEM / TMA tensor-core path for sm_100a: implicit-GEMM 3x3 convolution (forward,
+// data gradient, weight gradient) and the sharded fully-connected GEMMs, all bf16 x bf16 -> fp32.
+//
+// One kernel template, three operand arrangements ("modes"):
+//   FWD   : D[pixel, n]  = sum_{tap, c} act[pixel + tap, c] * W[n, tap, c]       A K-major,  B K-major
+//   DGRAD : D[pixel, n]  = sum_{tap, k} dy[pixel - tap, k]  * W[k, tap, n]       A K-major,  B MN-major
+//   WGRAD : D[m, n]      = sum_{pixel} dy[pixel, m] * act[pixel + tap, n]        A MN-major, B MN-major
+// A fully-connected layer is the same thing with one tap and 1x1 "images" (pixel = batch row).
+//
+// Every operand tile is a set of 128-byte rows fetched by TMA (cp.async.bulk.tensor, 4-D boxes,
+// SWIZZLE_128B; out-of-bounds coordinates read zeros, which implements the convolution padding,
+// ragged tile edges and ragged reduction tails) into a ring of shared-memory stages guarded by
+// mbarriers.  One thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) into a TMEM
+// accumulator; tcgen05.commit releases a stage back to the TMA producer; four epilogue warps read
+// the accumulator with tcgen05.ld and apply bias+ReLU / the ReLU mask / the split-sum store.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
+// warps 2..5 = epilogue (TMEM lane quadrant = warp_id % 4).
+//
+// Hang safety: every mbarrier wait is bounded (iteration cap and a wall-clock deadline); a wait
+// that gives up records a code in the model's device status word and the CTA drains and exits
+// normally (TMEM is always released), so a broken pipeline turns into SB_ERR_TIMEOUT on the
+// host instead of a stuck GPU.  No multicast is used anywhere.
 #include "sb_umma.h"
+
+#include <cstdio>
+#include <cstring>
+
 namespace sb {
-sb_status umma_plan_scratch(sb_model*, size_t* floats) { *floats = 0; return SB_OK; }
-sb_status umma_plan_layers(sb_model*) { return SB_OK; }
-sb_status umma_conv_fwd(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
-sb_status umma_conv_dgrad(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
-sb_status umma_conv_wgrad(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
-sb_status umma_fc_fwd(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
-sb_status umma_fc_dgrad(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
-sb_status umma_fc_wgrad(sb_model*, int, cudaStream_t) { return SB_ERR_UNSUPPORTED; }
+
+enum { MODE_FWD = 0, MODE_DGRAD = 1, MODE_WGRAD = 2 };
+enum { UEPI_BIAS_ACT = 0, UEPI_MASK = 1, UEPI_F32 = 2 };
+
+struct UmmaParams {
+    int mode, ntaps;
+    // pixel-box geometry of the activation-side operand(s): box = bw x bh x bn pixels
+    int bw, bh, bn;
+    int W, H, N;
+    int tiles_w, tiles_h, tiles_n;
+    // FWD / DGRAD reduction: kchunks 64-wide chunks per tap; w_cols = row length of one tap in the weight matrix
+    int kchunks, w_cols;
+    // output columns
+    int n_total;          // valid output columns (FWD: Cout, DGRAD: Cin, WGRAD: Cin)
+    int shards, tiles_per_shard;  // N-tile enumeration per model shard (FWD of a sharded FC layer); shards=1 otherwise
+    // WGRAD
+    int m_total;          // rows of the weight gradient (Cout / out-features)
+    int m_shards, m_tiles_per_shard;
+    int splits, chunks_per_split, total_chunks;
+    // epilogue
+    int epi, relu, out_f32;
+    void* out;            // FWD/DGRAD: [pixels][ldc] bf16 (or float when out_f32); WGRAD: float partial sums
+    long ldc;
+    const float* bias;
+    const __nv_bfloat16* ref;   // UEPI_MASK: same layout as out; nullptr = no mask
+    long split_stride;    // WGRAD: floats between split partial buffers
+    uint32_t* status;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after ~2 s of wall clock (or 2^28 polls) and reports failure.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t it = 0; it < (1u << 28); ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023u) == 1023u && globaltimer_ns() - t0 > 2000000000ull) break;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(const CUtensorMap* map, void* dst, uint64_t* bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, SWIZZLE_128B, 128-byte rows (64 bf16).
+//   K-major operand : rows = M/N index, 8-row groups 1024 bytes apart (stride byte offset).
+//   MN-major operand: rows = K index (8-row groups 1024 bytes apart); 64-element blocks along M/N
+//                     are `lbo_bytes` apart (leading byte offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = n.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int a_mn_major, int b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+constexpr int UMMA_THREADS = 192;
+constexpr int A_STAGE_BYTES = 16384;   // 128 rows x 128 B (K-major) or 2 boxes of 64 rows x 128 B (MN-major)
+
+template <int BN> struct Cfg {
+    static constexpr int B_STAGE_BYTES = BN * 128;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 2048 /*barriers, bias*/;
+};
+
+// ------------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------------
+template <int MODE, int BN>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaParams p)
+{
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* ctrl = smem + C::STAGES * C::STAGE_BYTES;
+    uint64_t* full = (uint64_t*)ctrl;                 // [STAGES]
+    uint64_t* empty = full + C::STAGES;               // [STAGES]
+    uint64_t* acc_full = empty + C::STAGES;           // [1]
+    uint32_t* tmem_slot = (uint32_t*)(acc_full + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* s_bias = (float*)(ctrl + 512);             // [BN]
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+    // ---- tile coordinates ---------------------------------------------------------------------
+    int tap_fixed = 0, split = 0;
+    int m_idx = blockIdx.x, n_idx = blockIdx.y;
+    int n0, n_hi;       // first output column of this tile and one past the last valid column
+    if (MODE == MODE_WGRAD) {
+        tap_fixed = blockIdx.z / p.splits;
+        split = blockIdx.z % p.splits;
+        n0 = n_idx * BN;
+        n_hi = p.n_total;
+    } else {
+        const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
+        const int lo = (int)(((long)sh * p.n_total) / p.shards), hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
+        n0 = lo + t * BN;
+        n_hi = hi;
+        if (n0 >= n_hi) return;   // uniform over the CTA, before any barrier or TMEM allocation
+    }
+    // FWD/DGRAD: the M tile is one pixel box; WGRAD: the M tile is 128 gradient rows of one shard
+    int pw0 = 0, ph0 = 0, pn0 = 0, m0 = 0, m_hi = 0;
+    if (MODE == MODE_WGRAD) {
+        const int sh = m_idx / p.m_tiles_per_shard, t = m_idx % p.m_tiles_per_shard;
+        const int lo = (int)(((long)sh * p.m_total) / p.m_shards), hi = (int)(((long)(sh + 1) * p.m_total) / p.m_shards);
+        m0 = lo + t * 128;
+        m_hi = hi;
+        if (m0 >= m_hi) return;
+    } else {
+        pw0 = (m_idx % p.tiles_w) * p.bw;
+        ph0 = ((m_idx / p.tiles_w) % p.tiles_h) * p.bh;
+        pn0 = (m_idx / (p.tiles_w * p.tiles_h)) * p.bn;
+    }
+    int k_begin = 0, k_end = 0;   // k-iterations of this CTA
+    if (MODE == MODE_WGRAD) {
+        k_begin = split * p.chunks_per_split;
+        k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
+    } else {
+        k_end = p.ntaps * p.kchunks;
+    }
+    const int n_iters = k_end - k_begin;
+
+    // ---- one-time setup -----------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapB) : "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
+        for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // =========================== TMA producer ===============================================
+        if (lane == 0) {
+            for (int it = 0; it < n_iters; ++it) {
+                const int s = it % C::STAGES;
+                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
+                if (*abort_flag) break;
+                uint8_t* sa = smem + s * C::STAGE_BYTES;
+                uint8_t* sb = sa + A_STAGE_BYTES;
+                mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES);
+                const int kit = k_begin + it;
+                if (MODE == MODE_WGRAD) {
+                    // pixel chunk kit -> box origin; A = dy (two 64-channel boxes), B = shifted activations
+                    const int cw = (kit % p.tiles_w) * p.bw, ch = ((kit / p.tiles_w) % p.tiles_h) * p.bh;
+                    const int cn = (kit / (p.tiles_w * p.tiles_h)) * p.bn;
+                    const int dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
+                    tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
+                    tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + ds, ch + dr, cn);
+                } else {
+                    const int tap = kit / p.kchunks, kc = kit % p.kchunks;
+                    int dr = 0, ds = 0;
+                    if (p.ntaps == 9) { dr = tap / 3 - 1; ds = tap % 3 - 1; }
+                    if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
+                    tma_load_4d(&mapA, sa, &full[s], kc * 64, pw0 + ds, ph0 + dr, pn0);
+                    if (MODE == MODE_FWD) {
+                        tma_load_4d(&mapB, sb, &full[s], tap * p.w_cols + kc * 64, n0, 0, 0);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer =================================================
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_WGRAD, MODE != MODE_FWD);
+            bool ok = true;
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int s = it % C::STAGES;
+                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    // K-major: 16 elements = 32 bytes along the row; MN-major: 16 k-rows = 2048 bytes
+                    const uint64_t ad = (MODE == MODE_WGRAD) ? make_desc(sa + kk * 2048, 8192) : make_desc(sa + kk * 32, 16);
+                    const uint64_t bd = (MODE == MODE_FWD) ? make_desc(sb + kk * 32, 16) : make_desc(sb + kk * 2048, 8192);
+                    umma_bf16(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(&empty[s]);      // stage reusable once these MMAs have read it
+            }
+            if (ok) umma_commit(acc_full);   // accumulator complete
+        }
+    } else {
+        // =========================== epilogue ===================================================
+        const int q = warp % 4;               // TMEM lane quadrant of this warp
+        const int row = q * 32 + lane;        // accumulator row handled by this thread
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(acc_full, 0);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) {
+            if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+        } else {
+            tc_fence_after();
+            bool row_ok;
+            size_t row_off;
+            if (MODE == MODE_WGRAD) {
+                row_ok = (m0 + row) < m_hi;
+                row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
+            } else {
+                const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
+                const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+                row_ok = w < p.W && h < p.H && n < p.N;
+                row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+            }
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(taddr + c0, v);     // warp-collective: executed by all lanes regardless of row_ok
+                tmem_ld_wait();
+                if (!row_ok || n0 + c0 >= n_hi) continue;
+                float f[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
+                const int ncol = n0 + c0;
+                const bool full16 = ncol + 16 <= n_hi;
+                if (p.epi == UEPI_BIAS_ACT) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        f[j] += s_bias[c0 + j];
+                        if (p.relu && !(f[j] > 0.f)) f[j] = 0.f;
+                    }
+                } else if (p.epi == UEPI_MASK && p.ref != nullptr) {
+                    const __nv_bfloat16* rp = p.ref + row_off + ncol;
+                    if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
+                        uint4 r0 = *(const uint4*)rp, r1 = *(const uint4*)(rp + 8);
+                        const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
+                        const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
+                            if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (ncol + j < n_hi && !(__bfloat162float(rp[j]) > 0.f)) f[j] = 0.f;
+                    }
+                }
+                if (p.epi == UEPI_F32 || p.out_f32) {
+                    float* op = (float*)p.out + row_off + ncol;
+                    if (full16 && ((p.ldc & 3) == 0) && ((ncol & 3) == 0) && ((((size_t)p.split_stride) & 3) == 0) && ((p.w_cols & 3) == 0 || MODE != MODE_WGRAD)) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (ncol + j < n_hi) op[j] = f[j];
+                    }
+                } else {
+                    __nv_bfloat16* op = (__nv_bfloat16*)p.out + row_off + ncol;
+                    if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+                            pk[j] = *(uint32_t*)&t;
+                        }
+                        ((uint4*)op)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        ((uint4*)op)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (ncol + j < n_hi) op[j] = __float2bfloat16_rn(f[j]);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that may still be in flight time to land before shared memory is released
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side: tensor maps and launch planning
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+static char g_umma_err[256] = "";
+
+static bool get_encode()
+{
+    if (g_encode) return true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        snprintf(g_umma_err, sizeof(g_umma_err), "cuTensorMapEncodeTiled is not available from the driver");
+        return false;
+    }
+    g_encode = (EncodeTiledFn)fn;
+    return true;
+}
+
+// bf16 tensor with dims d[0..3] (innermost first, elements) and byte strides s[1..3]; box b[0..3].
+static bool encode_map(CUtensorMap* map, const void* ptr, const uint64_t d[4], const uint64_t strides_bytes[3], const uint32_t box[4])
+{
+    if (!get_encode()) return false;
+    cuuint64_t gd[4] = {d[0], d[1], d[2], d[3]};
+    cuuint64_t gs[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
+    cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), gd, gs, bx, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_umma_err, sizeof(g_umma_err), "cuTensorMapEncodeTiled failed (%d): dims %llu,%llu,%llu,%llu box %u,%u,%u,%u", (int)r,
+                 (unsigned long long)d[0], (unsigned long long)d[1], (unsigned long long)d[2], (unsigned long long)d[3], box[0], box[1], box[2], box[3]);
+        return false;
+    }
+    return true;
+}
+// Activation tensor [N][H][W][C] bf16 -> 4-D map (C, W, H, N) with a (64, bw, bh, bn) box.
+static bool act_map(CUtensorMap* map, const void* ptr, int N, int H, int W, int C, int bw, int bh, int bn)
+{
+    uint64_t d[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+    uint64_t s[3] = {(uint64_t)C * 2, (uint64_t)W * C * 2, (uint64_t)H * W * C * 2};
+    uint32_t b[4] = {64, (uint32_t)bw, (uint32_t)bh, (uint32_t)bn};
+    return encode_map(map, ptr, d, s, b);
+}
+// Row-major matrix [rows][cols] bf16 -> map (cols, rows, 1, 1) with a (64, box_rows, 1, 1) box.
+static bool mat_map(CUtensorMap* map, const void* ptr, long rows, long cols, int box_rows)
+{
+    uint64_t d[4] = {(uint64_t)cols, (uint64_t)rows, 1, 1};
+    uint64_t s[3] = {(uint64_t)cols * 2, (uint64_t)rows * cols * 2, (uint64_t)rows * cols * 2};
+    uint32_t b[4] = {64, (uint32_t)box_rows, 1, 1};
+    return encode_map(map, ptr, d, s, b);
+}
+
+static int cdiv_i(long a, long b) { return (int)((a + b - 1) / b); }
+
+// Pixel box (bw, bh, bn) with bw*bh*bn = target (a power of two): least padded volume, then widest rows.
+static void choose_box(int W, int H, int N, int target, int* bw, int* bh, int* bn)
+{
+    double best = 1e300;
+    int bbw = 1, bbh = 1;
+    for (int w = 1; w <= target; w *= 2)
+        for (int h = 1; w * h <= target; h *= 2) {
+            int n = target / (w * h);
+            double vol = (double)cdiv_i(W, w) * w * cdiv_i(H, h) * h * cdiv_i(N, n) * n;
+            // prefer exact fits; among equal volumes prefer wider, then taller boxes (longer contiguous runs)
+            double score = vol * (1.0 - 1e-6 * w - 1e-8 * h);
+            if (score < best) { best = score; bbw = w; bbh = h; }
+        }
+    *bw = bbw; *bh = bbh; *bn = target / (bbw * bbh);
+}
+
+template <int MODE, int BN>
+static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<BN>::SMEM_BYTES, st>>>(op.mapA, op.mapB, p);
+    return cudaGetLastError();
+}
+
+template <int MODE>
+static cudaError_t launch_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    switch (bn) {
+    case 64: return launch_one<MODE, 64>(op, p, grid, st);
+    case 128: return launch_one<MODE, 128>(op, p, grid, st);
+    case 256: return launch_one<MODE, 256>(op, p, grid, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+// The op's full parameter block lives next to the tensor maps (host memory owned by the model).
+struct OpBlock {
+    UmmaParams p;
+    int bn;
+    dim3 grid;
+};
+static_assert(sizeof(OpBlock) <= sizeof(((UmmaOp*)nullptr)->blob), "UmmaOp::blob too small");
+static OpBlock* blk(UmmaOp& op) { return (OpBlock*)op.blob; }
+static const OpBlock* blk(const UmmaOp& op) { return (const OpBlock*)op.blob; }
+
+static sb_status launch_op(const UmmaOp& op, cudaStream_t st)
+{
+    const OpBlock* b = blk(op);
+    cudaError_t e;
+    if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, b->p, b->grid, st);
+    else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, b->p, b->grid, st);
+    else e = launch_mode<MODE_WGRAD>(b->bn, op, b->p, b->grid, st);
+    if (e != cudaSuccess) {
+        snprintf(g_umma_err, sizeof(g_umma_err), "tensor-core launch failed: %s", cudaGetErrorString(e));
+        return SB_ERR_CUDA;
+    }
+    return SB_OK;
+}
+
+const char* umma_last_error() { return g_umma_err; }
+
+static int pick_bn(int n_cols, long m_tiles)
+{
+    // widest tile that still leaves at least ~one wave of CTAs; never wider than the column count needs
+    int bn = 256;
+    while (bn > 64 && (bn / 2 >= n_cols || m_tiles * cdiv_i(n_cols, bn) < 148)) bn /= 2;
+    return bn;
+}
+
+// Conv weight-gradient split count: enough CTAs for ~2 waves, at least 4 pixel chunks per CTA.
+static int wgrad_splits(long ctas_without_split, int total_chunks)
+{
+    int s = 1;
+    while (ctas_without_split * s < 296 && total_chunks / (s * 2) >= 4) s *= 2;
+    return s;
+}
+
+static bool conv_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
+{
+    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.Cin % 64 == 0 && lv.Cout % 64 == 0;
+}
+static bool fc_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
+{
+    // TMA needs 16-byte row strides: in and out multiples of 8; the reduce dims multiples of 64 keep every box row in bounds
+    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.in_f % 64 == 0 && lv.out_f % 8 == 0;
+}
+
+sb_status umma_plan_scratch(sb_model* m, size_t* floats)
+{
+    ModelView mv = model_view(m);
+    size_t need = 0;
+    for (int i = 0; i < mv.n_layers; ++i) {
+        LayerView lv = layer_view(m, i);
+        if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
+            int bw, bh, bn;
+            choose_box(lv.W, lv.H, mv.B, 64, &bw, &bh, &bn);
+            const int total_chunks = cdiv_i(lv.W, bw) * cdiv_i(lv.H, bh) * cdiv_i(mv.B, bn);
+            const int bnt = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
+            const long ctas = (long)cdiv_i(lv.Cout, 128) * cdiv_i(lv.Cin, bnt) * 9;
+            const int S = wgrad_splits(ctas, total_chunks);
+            if (S > 1) need = need > (size_t)S * lv.n_w ? need : (size_t)S * lv.n_w;
+        }
+    }
+    *floats = need;
+    return SB_OK;
+}
+
+static sb_status fail_plan() { return SB_ERR_CUDA; }
+
+sb_status umma_plan_layers(sb_model* m)
+{
+    ModelView mv = model_view(m);
+    if (!mv.bf16 || (mv.cfg->flags & SB_FLAG_FORCE_SIMT)) return SB_OK;
+    const int B = mv.B;
+    for (int i = 0; i < mv.n_layers; ++i) {
+        LayerView lv = layer_view(m, i);
+        UmmaLayer& um = *lv.um;
+        const bool want_in_grad = i > 0;
+        if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
+            int bw, bh, bn;
+            choose_box(lv.W, lv.H, B, 128, &bw, &bh, &bn);
+            const int tw = cdiv_i(lv.W, bw), th = cdiv_i(lv.H, bh), tn = cdiv_i(B, bn);
+            const long m_tiles = (long)tw * th * tn;
+            // ---- forward ----
+            {
+                OpBlock* b = blk(um.fwd);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_FWD; p.ntaps = 9; p.bw = bw; p.bh = bh; p.bn = bn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = tw; p.tiles_h = th; p.tiles_n = tn; p.kchunks = lv.Cin / 64; p.w_cols = lv.Cin;
+                p.n_total = lv.Cout; p.shards = 1;
+                b->bn = pick_bn(lv.Cout, m_tiles);
+                p.tiles_per_shard = cdiv_i(lv.Cout, b->bn);
+                p.epi = UEPI_BIAS_ACT; p.relu = 1; p.out_f32 = 0; p.out = lv.act; p.ldc = lv.Cout; p.bias = mv.Wm + lv.p_b;
+                p.status = mv.status;
+                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
+                if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, bw, bh, bn)) return fail_plan();
+                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->bn)) return fail_plan();
+                um.fwd.enabled = true;
+            }
+            // ---- data gradient ----
+            if (want_in_grad) {
+                OpBlock* b = blk(um.dgrad);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_DGRAD; p.ntaps = 9; p.bw = bw; p.bh = bh; p.bn = bn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = tw; p.tiles_h = th; p.tiles_n = tn; p.kchunks = lv.Cout / 64; p.w_cols = lv.Cin;
+                p.n_total = lv.Cin; p.shards = 1;
+                b->bn = pick_bn(lv.Cin, m_tiles);
+                p.tiles_per_shard = cdiv_i(lv.Cin, b->bn);
+                p.epi = UEPI_MASK; p.out = lv.d_below; p.ldc = lv.Cin;
+                p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
+                p.status = mv.status;
+                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
+                if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, bw, bh, bn)) return fail_plan();
+                if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, 64)) return fail_plan();
+                um.dgrad.enabled = true;
+            }
+            // ---- weight gradient ----
+            {
+                int cw, ch, cn;
+                choose_box(lv.W, lv.H, B, 64, &cw, &ch, &cn);
+                OpBlock* b = blk(um.wgrad);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_WGRAD; p.ntaps = 9; p.bw = cw; p.bh = ch; p.bn = cn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = cdiv_i(lv.W, cw); p.tiles_h = cdiv_i(lv.H, ch); p.tiles_n = cdiv_i(B, cn);
+                p.total_chunks = p.tiles_w * p.tiles_h * p.tiles_n;
+                p.w_cols = lv.Cin; p.n_total = lv.Cin; p.shards = 1; p.tiles_per_shard = 1;
+                p.m_total = lv.Cout; p.m_shards = 1; p.m_tiles_per_shard = cdiv_i(lv.Cout, 128);
+                b->bn = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
+                const int n_tiles = cdiv_i(lv.Cin, b->bn);
+                const long ctas = (long)p.m_tiles_per_shard * n_tiles * 9;
+                p.splits = wgrad_splits(ctas, p.total_chunks);
+                p.chunks_per_split = cdiv_i(p.total_chunks, p.splits);
+                p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
+                p.split_stride = (long)lv.n_w;
+                p.out = p.splits > 1 ? (void*)mv.ws : (void*)(mv.Gm + lv.p_w);
+                p.status = mv.status;
+                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)n_tiles, (unsigned)(9 * p.splits));
+                if ((size_t)p.splits * lv.n_w > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
+                if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, cw, ch, cn)) return fail_plan();
+                if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, cw, ch, cn)) return fail_plan();
+                um.wgrad.enabled = true;
+            }
+        } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
+            const int K = mv.cfg->K;
+            const int m_tiles = cdiv_i(B, 128);
+            // ---- forward: Y[:, shard j] = X W_j^T + b_j ; N tiles enumerated per shard ----
+            {
+                OpBlock* b = blk(um.fwd);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_FWD; p.ntaps = 1; p.bw = 1; p.bh = 1; p.bn = 128; p.W = 1; p.H = 1; p.N = B;
+                p.tiles_w = 1; p.tiles_h = 1; p.tiles_n = m_tiles; p.kchunks = lv.in_f / 64; p.w_cols = lv.in_f;
+                p.n_total = lv.out_f; p.shards = K;
+                b->bn = 64;
+                const int widest = cdiv_i(lv.out_f, K);
+                p.tiles_per_shard = cdiv_i(widest, b->bn);
+                p.epi = UEPI_BIAS_ACT; p.relu = lv.relu ? 1 : 0; p.out_f32 = lv.kind == SB_FC; p.out = lv.act; p.ldc = lv.out_f;
+                p.bias = mv.Wm + lv.p_b; p.status = mv.status;
+                b->grid = dim3((unsigned)m_tiles, (unsigned)(p.tiles_per_shard * K), 1);
+                if (!act_map(&um.fwd.mapA, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
+                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->bn)) return fail_plan();
+                um.fwd.enabled = true;
+            }
+            // ---- data gradient: dX = sum_j dY_j W_j = one reduction over the concatenated width ----
+            if (want_in_grad && lv.out_f % 8 == 0) {
+                OpBlock* b = blk(um.dgrad);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_DGRAD; p.ntaps = 1; p.bw = 1; p.bh = 1; p.bn = 128; p.W = 1; p.H = 1; p.N = B;
+                p.tiles_w = 1; p.tiles_h = 1; p.tiles_n = m_tiles; p.kchunks = cdiv_i(lv.out_f, 64); p.w_cols = lv.in_f;
+                p.n_total = lv.in_f; p.shards = 1;
+                b->bn = 64;
+                p.tiles_per_shard = cdiv_i(lv.in_f, b->bn);
+                p.epi = UEPI_MASK; p.out = lv.d_below; p.ldc = lv.in_f;
+                p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
+                p.status = mv.status;
+                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
+                if (!act_map(&um.dgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 128)) return fail_plan();
+                if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, 64)) return fail_plan();
+                um.dgrad.enabled = true;
+            }
+            // ---- weight gradient: dW_j = dY_j^T X ; M tiles enumerated per shard (needs 16-byte aligned shard starts) ----
+            bool aligned = true;
+            for (int j = 0; j <= K; ++j) aligned = aligned && ((((long)j * lv.out_f) / K) % 8 == 0);
+            if (aligned) {
+                OpBlock* b = blk(um.wgrad);
+                memset(b, 0, sizeof(*b));
+                UmmaParams& p = b->p;
+                p.mode = MODE_WGRAD; p.ntaps = 1; p.bw = 1; p.bh = 1; p.bn = 64; p.W = 1; p.H = 1; p.N = B;
+                p.tiles_w = 1; p.tiles_h = 1; p.tiles_n = cdiv_i(B, 64);
+                p.total_chunks = p.tiles_n;
+                p.w_cols = lv.in_f; p.n_total = lv.in_f; p.shards = 1; p.tiles_per_shard = 1;
+                p.m_total = lv.out_f; p.m_shards = K; p.m_tiles_per_shard = cdiv_i(cdiv_i(lv.out_f, K), 128);
+                b->bn = lv.in_f >= 256 ? 256 : (lv.in_f >= 128 ? 128 : 64);
+                const int n_tiles = cdiv_i(lv.in_f, b->bn);
+                p.splits = 1; p.chunks_per_split = p.total_chunks;
+                p.epi = UEPI_F32; p.ldc = lv.in_f; p.split_stride = 0;
+                p.out = (void*)(mv.Gm + lv.p_w);
+                p.status = mv.status;
+                b->grid = dim3((unsigned)(p.m_tiles_per_shard * K), (unsigned)n_tiles, 1);
+                if (!act_map(&um.wgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 64)) return fail_plan();
+                if (!act_map(&um.wgrad.mapB, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 64)) return fail_plan();
+                um.wgrad.enabled = true;
+            }
+        }
+    }
+    return SB_OK;
+}
+
+sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st); }
+sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st); }
+sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st); }
+sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st); }
+sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->wgrad, st); }
+
+sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part)
+{
+    LayerView lv = layer_view(m, layer);
+    const OpBlock* b = blk(lv.um->wgrad);
+    *splits = b->p.splits;
+    *part = (float*)b->p.out;
+    return launch_op(lv.um->wgrad, st);
+}
+
+}  // namespace sb

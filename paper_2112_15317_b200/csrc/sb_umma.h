@@ -12,7 +12,7 @@ struct UmmaOp {
     bool enabled = false;
     alignas(64) CUtensorMap mapA;
     alignas(64) CUtensorMap mapB;
-    int params[24] = {0};   // kernel geometry (see sb_umma.cu)
+    alignas(16) unsigned char blob[512];   // kernel parameters, tile width and grid (see sb_umma.cu)
 };
 struct UmmaLayer {
     UmmaOp fwd, dgrad, wgrad;
@@ -53,9 +53,13 @@ sb_status umma_plan_layers(sb_model* m);
 
 sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st);
-sb_status umma_conv_wgrad(sb_model* m, int layer, cudaStream_t st);   // counts its own launches
+// Launches the weight-gradient kernel; *splits > 1 means it wrote split partial sums at *part
+// (to be reduced in split order by the caller), else it wrote the gradient itself.
+sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part);
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
+
+const char* umma_last_error();
 
 }  // namespace sb
