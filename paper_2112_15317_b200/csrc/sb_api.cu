@@ -15,6 +15,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -52,6 +53,8 @@ struct Layer {
     uint8_t* idx = nullptr;                     // pool argmax
     int wg_splits = 1;                          // conv wgrad pixel-range splits (CUDA-core kernel)
     int bg_splits = 1;                          // conv bias-gradient row splits
+    bool thin_input = false;                    // conv with Cin of 1/3/4: dedicated input-layer kernels
+    bool narrow = false;                        // FC with out <= 16: dedicated narrow kernels
     int act_dt = SB_DT_F32;
     UmmaLayer um;                               // tensor-core plan of this layer (tcgen05 path)
 };
@@ -84,6 +87,7 @@ struct sb_model {
     int64_t launches = 0, last_step_launches = 0;
     // per-launch event recording (sb_profile_begin / sb_profile_end)
     struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; };
+    bool debug_sync = false;   // SB_DEBUG_SYNC=1 in the environment: synchronise and check after every launch
     bool profiling = false;
     std::vector<Rec> recs;
     std::vector<cudaEvent_t> ev_pool;
@@ -193,6 +197,7 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
         l.act = take(B * l.out_per_img * e);
         l.dact = take(B * l.out_per_img * m->esz);
         if (l.kind == SB_MAXPOOL2) l.idx = (uint8_t*)take(B * l.out_per_img);
+        if (l.kind == SB_FC_RELU || l.kind == SB_FC) l.narrow = fc_narrow_supported(l.out_f, (int)B);
         if (l.kind == SB_CONV3X3_RELU) {
             // pixel-range splits of the weight gradient: enough blocks to fill the machine, each
             // split a whole number of images
@@ -206,6 +211,11 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
             while (sb_ * 2 <= (int)B && B % (sb_ * 2) == 0 && (long)sb_ * ((l.Cout + 31) / 32) < 148 * 2) sb_ *= 2;
             l.bg_splits = sb_;
             if ((size_t)sb_ * l.n_b > ws_floats) ws_floats = (size_t)sb_ * l.n_b;
+            l.thin_input = conv_in_supported(l.Cin, l.Cout);
+            if (l.thin_input) {
+                size_t nd = (size_t)conv_in_wgrad_blocks((int)B, l.H, l.W) * (l.n_w + l.n_b);
+                if (nd > ws_floats) ws_floats = nd;
+            }
         }
     }
     size_t um_ws = 0;
@@ -238,6 +248,10 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
         ++m->launches;                                                                            \
         if (e_ != cudaSuccess) return fail(SB_ERR_CUDA, "launch failed in %s: %s", #expr, cudaGetErrorString(e_)); \
         if (m->profiling && rec_.e1) { cudaEventRecord(rec_.e1, st); m->recs.push_back(rec_); }   \
+        if (m->debug_sync) {                                                                      \
+            cudaError_t d_ = cudaStreamSynchronize(st);                                           \
+            if (d_ != cudaSuccess) return fail(SB_ERR_CUDA, "kernel %s (layer call %s) failed: %s", tag, #expr, cudaGetErrorString(d_)); \
+        }                                                                                         \
     } while (0)
 // Same bracket for the tensor-core launchers, which return sb_status.
 #define U_TRY(tag, flops, bytes, expr)                                                            \
@@ -248,6 +262,10 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
         sb_status s_ = (expr);                                                                    \
         if (s_ != SB_OK) return fail(s_, "%s", umma_last_error());                                                            \
         if (m->profiling && rec_.e1) { cudaEventRecord(rec_.e1, st); m->recs.push_back(rec_); }   \
+        if (m->debug_sync) {                                                                      \
+            cudaError_t d_ = cudaStreamSynchronize(st);                                           \
+            if (d_ != cudaSuccess) return fail(SB_ERR_CUDA, "kernel %s failed: %s", tag, cudaGetErrorString(d_)); \
+        }                                                                                         \
     } while (0)
 
 // Which buffer holds the input of layer i: the previous layer's output, or the caller's images.
@@ -275,7 +293,8 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.in = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
         a.w = wts; a.bias = m->Wm + l.p_b; a.out = l.act; a.mask_ref = nullptr;
         a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 0; a.relu = 1;
-        L_TRY("conv_fwd_simt", flops, bytes, launch_conv_simt(a, bf, st));
+        if (l.thin_input) L_TRY("conv_in_fwd", flops, bytes, launch_conv_in_fwd(a, bf, st));
+        else L_TRY("conv_fwd_simt", flops, bytes, launch_conv_simt(a, bf, st));
         break;
     }
     case SB_MAXPOOL2: {
@@ -292,6 +311,14 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         if (l.um.fwd.enabled) {
             U_TRY("fc_fwd_umma", flops, bytes, umma_fc_fwd(m, i, st));
             ++m->launches;
+            break;
+        }
+        if (l.narrow) {
+            FcNarrowArgs a{};
+            a.pass = 0; a.X = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.tab_b = b; a.W = wts;
+            a.bias = m->Wm + l.p_b; a.relu = l.relu; a.B = B; a.in_f = l.in_f; a.out_f = l.out_f;
+            if (l.kind == SB_FC) a.Y32 = (float*)l.act; else a.Y = l.act;
+            L_TRY("fc_narrow_fwd", flops, bytes, launch_fc_narrow(a, bf, st));
             break;
         }
         GemmSimtArgs a{};
@@ -339,6 +366,17 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         const double flops = 2.0 * B * (double)l.in_f * l.out_f;
         const double act_bytes = (double)B * (l.in_f + l.out_f) * e;
         // weight gradient per shard: dW_j = dY_j^T X   (rows c_j..c_{j+1} of the [out,in] gradient)
+        if (l.narrow) {
+            FcNarrowArgs a{};
+            a.pass = 1; a.X = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.tab_b = b;
+            a.dY = l.dact; a.dW = m->Gm + l.p_w; a.db = m->Gm + l.p_b; a.B = B; a.in_f = l.in_f; a.out_f = l.out_f;
+            L_TRY("fc_narrow_wgrad", flops, act_bytes + (double)l.n_w * 4.0, launch_fc_narrow(a, bf, st));
+            if (want_in_grad) {
+                a.pass = 2; a.W = wts; a.ref = below_relu ? m->L[i - 1].act : nullptr; a.dX = d_below;
+                L_TRY("fc_narrow_dgrad", flops, act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0), launch_fc_narrow(a, bf, st));
+            }
+            break;
+        }
         if (l.um.wgrad.enabled) {
             U_TRY("fc_wgrad_umma", flops, act_bytes + (double)l.n_w * 4.0, umma_fc_wgrad(m, i, st));
             ++m->launches;
@@ -352,7 +390,8 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 2; a.tab_b = b; }
             L_TRY("fc_wgrad_simt", flops, act_bytes + (double)l.n_w * 4.0, launch_gemm_simt(a, bf, st));
         }
-        L_TRY("bias_grad", 0.0, (double)B * l.out_f * e + 4.0 * l.out_f, launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
+        if (!l.um.wgrad.enabled)   // the tensor-core weight-gradient kernel also produces the bias gradient
+            L_TRY("bias_grad", 0.0, (double)B * l.out_f * e + 4.0 * l.out_f, launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
         if (want_in_grad) {
             // shard-layer / modulo-layer backward: dX = sum_j dY_j W_j, rows stay with their replica
             const double bytes = act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0);
@@ -383,12 +422,24 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         const double pix = (double)B * l.H * l.W;
         const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
         // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
-        if (l.um.wgrad.enabled) {
+        if (l.thin_input) {
+            // input-layer kernel: weight and bias partial sums per block, then one ordered reduce each
+            WgradSimtArgs a{};
+            a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
+            a.dy = l.dact; a.part = m->ws; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
+            const int nb = conv_in_wgrad_blocks(B, l.H, l.W);
+            const size_t stride = l.n_w + l.n_b;
+            L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(m->ws, stride, m->Gm + l.p_w, l.n_w, nb, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(m->ws + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+        } else if (l.um.wgrad.enabled) {
             int S = 1;
             float* part = nullptr;
             U_TRY("conv_wgrad_umma", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, umma_conv_wgrad_launch(m, i, st, &S, &part));
             ++m->launches;
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(part, m->Gm + l.p_w, l.n_w, S, st));
+            // weights and bias gradient reduce together (same layout in the split buffers and in the arena)
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)(l.n_w + l.n_b) * 4.0 * (S + 1),
+                             launch_reduce_partials(part, l.n_w + l.n_b, m->Gm + l.p_w, l.n_w + l.n_b, S, st));
         } else {
             const int S = l.wg_splits;
             WgradSimtArgs a{};
@@ -396,16 +447,16 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             a.dy = l.dact; a.part = S > 1 ? m->ws : m->Gm + l.p_w;
             a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
             L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws, m->Gm + l.p_w, l.n_w, S, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
         }
-        {
+        if (!l.thin_input && !l.um.wgrad.enabled) {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
             const long M = (long)B * l.H * l.W;
             // (stream order makes it safe to reuse the scratch the weight-gradient reduce just read)
             const int S = l.bg_splits;
             float* part = S > 1 ? m->ws : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, m->Gm + l.p_b, l.n_b, S, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, l.n_b, m->Gm + l.p_b, l.n_b, S, st));
         }
         if (want_in_grad) {
             const double bytes = pix * (l.Cin + l.Cout) * e + (double)l.n_w * e + (below_relu ? pix * l.Cin * e : 0.0);
@@ -577,6 +628,8 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     if (need > arena_bytes) { delete m; return fail(SB_ERR_ARENA_TOO_SMALL, "arena has %zu bytes, model needs %zu", arena_bytes, need); }
     m->arena = (char*)arena;
     m->arena_bytes = need;
+    const char* dbg = getenv("SB_DEBUG_SYNC");
+    m->debug_sync = dbg && dbg[0] == '1';
     cudaError_t e = cudaMemset(arena, 0, need);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }

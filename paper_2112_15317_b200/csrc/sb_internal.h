@@ -50,10 +50,31 @@ struct WgradSimtArgs {
 };
 cudaError_t launch_wgrad_simt(const WgradSimtArgs& a, bool bf16, cudaStream_t st);
 
+// Input-layer convolution (Cin of 1, 3 or 4; Cout a multiple of 8): dedicated forward and weight+bias
+// gradient kernels.  The gradient kernel writes conv_in_wgrad_blocks() partial buffers of
+// Cout*9*Cin + Cout floats each (weights, then bias) into a.part, to be reduced in block order.
+bool conv_in_supported(int Cin, int Cout);
+cudaError_t launch_conv_in_fwd(const ConvSimtArgs& a, bool bf16, cudaStream_t st);
+int conv_in_wgrad_blocks(int B, int H, int W);
+cudaError_t launch_conv_in_wgrad(const WgradSimtArgs& a, bool bf16, cudaStream_t st);
+
+// Narrow FC layer (out <= 16): pass 0 forward, 1 weight+bias gradient, 2 input gradient.
+struct FcNarrowArgs {
+    int pass;
+    const void* X; const PtrTab* tab; int tab_b;   // [B,in] activations (or R per-replica buffers of tab_b rows)
+    const void* W;                                 // [out,in] activation dtype
+    const float* bias; void* Y; float* Y32; int relu;   // forward outputs (either may be null)
+    const void* dY; float* dW; float* db;          // gradient inputs/outputs
+    const void* ref; void* dX;                     // dgrad: optional ReLU mask source and output [B,in]
+    int B, in_f, out_f;
+};
+bool fc_narrow_supported(int out_f, int B);
+cudaError_t launch_fc_narrow(const FcNarrowArgs& a, bool bf16, cudaStream_t st);
+
 // part[s][n] = sum over the rows of split s of in[row][n];  rows split evenly (M % splits == 0).
 cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st);
-// out[i] = sum_{s<splits} part[s*n + i], s ascending.
-cudaError_t launch_reduce_partials(const float* part, float* out, size_t n, int splits, cudaStream_t st);
+// out[i] = sum_{s<splits} part[s*stride + i], s ascending.
+cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st);
 
 struct PoolArgs {
     const void* x;  // [B,H,W,C]

@@ -19,6 +19,23 @@ template <typename T> __device__ __forceinline__ void stf(T* p, float v);
 template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
 template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
+// store 8 consecutive values (pointer 16-byte aligned for bf16, 32-byte for float)
+__device__ __forceinline__ void store8(float* p, const float (&v)[8])
+{
+    ((float4*)p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    ((float4*)p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8])
+{
+    uint32_t pk[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        pk[j] = *(uint32_t*)&t;
+    }
+    *(uint4*)p = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+
 static inline int cdiv(long a, long b) { return (int)((a + b - 1) / b); }
 
 // =============================================================================================
@@ -248,19 +265,37 @@ cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, 
 }
 
 __global__ void __launch_bounds__(256)
-reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ out, size_t n, int splits)
+reduce_partials_kernel(const float* __restrict__ part, size_t stride, float* __restrict__ out, size_t n, int splits)
 {
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         float t = 0.f;
-        for (int s = 0; s < splits; ++s) t += part[(size_t)s * n + i];
+        for (int s = 0; s < splits; ++s) t += part[(size_t)s * stride + i];
         out[i] = t;
     }
 }
-cudaError_t launch_reduce_partials(const float* part, float* out, size_t n, int splits, cudaStream_t st)
+__global__ void __launch_bounds__(256)
+reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4* __restrict__ out, size_t n4, int splits)
 {
-    int blocks = cdiv((long)n, 256);
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, out, n, splits);
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < splits; ++s) {
+            const float4 v = __ldg(part + (size_t)s * stride4 + i);
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        out[i] = t;
+    }
+}
+cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st)
+{
+    if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0) {
+        int blocks = cdiv((long)(n / 4), 256);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        reduce_partials4_kernel<<<blocks, 256, 0, st>>>((const float4*)part, stride / 4, (float4*)out, n / 4, splits);
+    } else {
+        int blocks = cdiv((long)n, 256);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, stride, out, n, splits);
+    }
     return cudaGetLastError();
 }
 
@@ -498,6 +533,296 @@ cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cuda
 {
     to_bf16_kernel<<<ew_blocks((long)(n / 4)), 256, 0, st>>>((const float4*)w, (uint2*)shadow, n / 4);
     return cudaGetLastError();
+}
+
+// =============================================================================================
+// Input-layer convolution (Cin <= 4, e.g. RGB images): 9*Cin <= 36 products per output, far too
+// thin for tensor-core tiles and bound by the output / dy traffic.  Each thread builds the
+// 3x3xCin patch of its pixel in registers (forward) or the block stages patches in shared memory
+// (weight gradient).
+// =============================================================================================
+template <typename T, int CIN, bool TAB>
+__device__ __forceinline__ void load_patch(float (&patch)[9 * CIN], const T* __restrict__ x, const PtrTab& tab, int b_per_rep,
+                                           long pix, int H, int W)
+{
+    const int w_ = (int)(pix % W);
+    const long q = pix / W;
+    const int h_ = (int)(q % H), n_ = (int)(q / H);
+    const T* img = TAB ? (const T*)tab.p[n_ / b_per_rep] + (size_t)(n_ % b_per_rep) * H * W * CIN : x + (size_t)n_ * H * W * CIN;
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            const int hh = h_ + r - 1, ww = w_ + s - 1;
+            const bool in = hh >= 0 && hh < H && ww >= 0 && ww < W;
+#pragma unroll
+            for (int c = 0; c < CIN; ++c) patch[(r * 3 + s) * CIN + c] = in ? ldf(img + ((size_t)hh * W + ww) * CIN + c) : 0.f;
+        }
+}
+
+// Forward: 8 consecutive threads share a pixel, each produces 8 output channels (16-byte stores that
+// a warp lays down as contiguous 128-byte pixel rows).  Weights live in shared memory as [9*CIN][Cout].
+template <typename T, int CIN, bool TAB>
+__global__ void __launch_bounds__(256)
+conv_in_fwd_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ wt, const float* __restrict__ bias,
+                   T* __restrict__ y, long npix, int H, int W, int Cout, int relu)
+{
+    extern __shared__ float s_wf[];            // [9*CIN][Cout] then bias [Cout]
+    float* s_b = s_wf + 9 * CIN * Cout;
+    for (int e = threadIdx.x; e < 9 * CIN * Cout; e += 256) {
+        int k = e % Cout, j = e / Cout;
+        s_wf[e] = ldf(wt + (size_t)k * 9 * CIN + j);
+    }
+    for (int e = threadIdx.x; e < Cout; e += 256) s_b[e] = bias[e];
+    __syncthreads();
+    const int groups = Cout / 8;               // threads per pixel
+    const long t = blockIdx.x * 256L + threadIdx.x;
+    const long pix = t / groups;
+    const int kg = (int)(t % groups) * 8;
+    if (pix >= npix) return;
+    float patch[9 * CIN];
+    load_patch<T, CIN, TAB>(patch, x, tab, b_per_rep, pix, H, W);
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = s_b[kg + i];
+#pragma unroll
+    for (int j = 0; j < 9 * CIN; ++j) {
+        const float4 w0 = *(const float4*)(s_wf + j * Cout + kg), w1 = *(const float4*)(s_wf + j * Cout + kg + 4);
+        acc[0] = fmaf(patch[j], w0.x, acc[0]); acc[1] = fmaf(patch[j], w0.y, acc[1]);
+        acc[2] = fmaf(patch[j], w0.z, acc[2]); acc[3] = fmaf(patch[j], w0.w, acc[3]);
+        acc[4] = fmaf(patch[j], w1.x, acc[4]); acc[5] = fmaf(patch[j], w1.y, acc[5]);
+        acc[6] = fmaf(patch[j], w1.z, acc[6]); acc[7] = fmaf(patch[j], w1.w, acc[7]);
+    }
+    if (relu) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (!(acc[i] > 0.f)) acc[i] = 0.f;
+    }
+    store8(y + (size_t)pix * Cout + kg, acc);
+}
+
+// Weight + bias gradient: block = 64 output channels x 4 pixel lanes; per 64-pixel chunk the block stages
+// the patches in shared memory, then thread (k, q) accumulates dy[pix,k] * patch[pix,:] over its pixels.
+// part[block][k][9*CIN] and part_b[block][k] are reduced afterwards in block order.
+template <typename T, int CIN, bool TAB>
+__global__ void __launch_bounds__(256)
+conv_in_wgrad_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ dy, float* __restrict__ part,
+                     long npix, int H, int W, int Cout, long stride_floats)
+{
+    constexpr int PJ = (9 * CIN + 3) / 4 * 4;   // padded patch length (16-byte rows)
+    __shared__ __align__(16) float s_patch[64][PJ];
+    __shared__ float s_red[3][64][9 * CIN + 1];
+    const int k = threadIdx.x % 64, q = threadIdx.x / 64;
+    const int k0 = blockIdx.y * 64;
+    float acc[9 * CIN], accb = 0.f;
+#pragma unroll
+    for (int j = 0; j < 9 * CIN; ++j) acc[j] = 0.f;
+    const long nchunks = (npix + 63) / 64;
+    for (long ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
+        const long p0 = ch * 64;
+        if (threadIdx.x < 64) {
+            float patch[9 * CIN];
+            const long pix = p0 + threadIdx.x;
+            if (pix < npix) load_patch<T, CIN, TAB>(patch, x, tab, b_per_rep, pix, H, W);
+            else {
+#pragma unroll
+                for (int j = 0; j < 9 * CIN; ++j) patch[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 9 * CIN; ++j) s_patch[threadIdx.x][j] = patch[j];
+        }
+        __syncthreads();
+        if (k0 + k < Cout) {
+#pragma unroll 4
+            for (int pp = q; pp < 64; pp += 4) {
+                const long pix = p0 + pp;
+                if (pix >= npix) break;
+                const float d = ldf(dy + (size_t)pix * Cout + k0 + k);
+                accb += d;
+#pragma unroll
+                for (int j = 0; j < 9 * CIN; ++j) acc[j] = fmaf(d, s_patch[pp][j], acc[j]);
+            }
+        }
+        __syncthreads();
+    }
+    // fixed-order reduction over the 4 pixel lanes
+    if (q > 0) {
+#pragma unroll
+        for (int j = 0; j < 9 * CIN; ++j) s_red[q - 1][k][j] = acc[j];
+        s_red[q - 1][k][9 * CIN] = accb;
+    }
+    __syncthreads();
+    if (q == 0 && k0 + k < Cout) {
+        float* dst = part + (size_t)blockIdx.x * stride_floats;
+#pragma unroll
+        for (int j = 0; j < 9 * CIN; ++j) dst[(size_t)(k0 + k) * 9 * CIN + j] = acc[j] + s_red[0][k][j] + s_red[1][k][j] + s_red[2][k][j];
+        dst[(size_t)Cout * 9 * CIN + k0 + k] = accb + s_red[0][k][9 * CIN] + s_red[1][k][9 * CIN] + s_red[2][k][9 * CIN];
+    }
+}
+
+template <typename T, int CIN>
+static cudaError_t launch_conv_in_fwd_t(const ConvSimtArgs& a, cudaStream_t st)
+{
+    const long npix = (long)a.B * a.H * a.W;
+    const long threads = npix * (a.Cout / 8);
+    const int blocks = (int)((threads + 255) / 256);
+    const size_t smem = (size_t)(9 * CIN * a.Cout + a.Cout) * 4;
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+    if (a.tab) conv_in_fwd_kernel<T, CIN, true><<<blocks, 256, smem, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
+    else conv_in_fwd_kernel<T, CIN, false><<<blocks, 256, smem, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
+    return cudaGetLastError();
+}
+bool conv_in_supported(int Cin, int Cout) { return (Cin == 1 || Cin == 3 || Cin == 4) && Cout % 8 == 0 && Cout <= 256; }
+cudaError_t launch_conv_in_fwd(const ConvSimtArgs& a, bool bf16, cudaStream_t st)
+{
+#define SB_CI(T) (a.Cin == 1 ? launch_conv_in_fwd_t<T, 1>(a, st) : a.Cin == 3 ? launch_conv_in_fwd_t<T, 3>(a, st) : launch_conv_in_fwd_t<T, 4>(a, st))
+    return bf16 ? SB_CI(__nv_bfloat16) : SB_CI(float);
+#undef SB_CI
+}
+int conv_in_wgrad_blocks(int B, int H, int W)
+{
+    long chunks = ((long)B * H * W + 63) / 64;
+    return (int)(chunks < 148 * 4 ? chunks : 148 * 4);
+}
+template <typename T, int CIN>
+static cudaError_t launch_conv_in_wgrad_t(const WgradSimtArgs& a, cudaStream_t st)
+{
+    const long npix = (long)a.B * a.H * a.W;
+    dim3 grid(conv_in_wgrad_blocks(a.B, a.H, a.W), (a.Cout + 63) / 64);
+    const long stride = (long)a.Cout * 9 * CIN + a.Cout;
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+    if (a.tab) conv_in_wgrad_kernel<T, CIN, true><<<grid, 256, 0, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
+    else conv_in_wgrad_kernel<T, CIN, false><<<grid, 256, 0, st>>>((const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
+    return cudaGetLastError();
+}
+// part: [conv_in_wgrad_blocks][Cout*9*Cin + Cout] floats (weights then bias), to be reduced in block order.
+cudaError_t launch_conv_in_wgrad(const WgradSimtArgs& a, bool bf16, cudaStream_t st)
+{
+#define SB_CI(T) (a.Cin == 1 ? launch_conv_in_wgrad_t<T, 1>(a, st) : a.Cin == 3 ? launch_conv_in_wgrad_t<T, 3>(a, st) : launch_conv_in_wgrad_t<T, 4>(a, st))
+    return bf16 ? SB_CI(__nv_bfloat16) : SB_CI(float);
+#undef SB_CI
+}
+
+// =============================================================================================
+// Narrow FC layers (out <= 16, e.g. the 10-class logits layer): too narrow for any GEMM tile.
+//   forward : one block per batch row, threads split the reduction, block-wide shuffle reduce
+//   wgrad   : one thread per input column, dY staged in shared memory
+//   dgrad   : one thread per (row, input column)
+// =============================================================================================
+constexpr int NARROW_MAX = 16;
+
+template <typename T, bool TAB>
+__global__ void __launch_bounds__(256)
+fc_narrow_fwd_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ Wt, const float* __restrict__ bias,
+                     T* __restrict__ Y, float* __restrict__ Y32, int in_f, int out_f, int relu)
+{
+    __shared__ float s_red[8][NARROW_MAX];
+    const int g = blockIdx.x;
+    const T* xr = TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f;
+    float acc[NARROW_MAX];
+#pragma unroll
+    for (int j = 0; j < NARROW_MAX; ++j) acc[j] = 0.f;
+    for (int k = threadIdx.x; k < in_f; k += 256) {
+        const float xv = ldf(xr + k);
+#pragma unroll
+        for (int j = 0; j < NARROW_MAX; ++j)
+            if (j < out_f) acc[j] = fmaf(xv, ldf(Wt + (size_t)j * in_f + k), acc[j]);
+    }
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+#pragma unroll
+    for (int j = 0; j < NARROW_MAX; ++j) {
+        float v = acc[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) s_red[warp][j] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < out_f) {
+        float v = bias[threadIdx.x];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += s_red[w][threadIdx.x];
+        if (relu && !(v > 0.f)) v = 0.f;
+        if (Y32) Y32[(size_t)g * out_f + threadIdx.x] = v;
+        if (Y) stf(Y + (size_t)g * out_f + threadIdx.x, v);
+    }
+}
+
+template <typename T, bool TAB>
+__global__ void __launch_bounds__(128)
+fc_narrow_wgrad_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ dY, float* __restrict__ dW,
+                       float* __restrict__ db, int B, int in_f, int out_f)
+{
+    extern __shared__ float s_dy[];   // [B][out_f]
+    for (int e = threadIdx.x; e < B * out_f; e += 128) s_dy[e] = ldf(dY + e);
+    __syncthreads();
+    const int i = blockIdx.x * 128 + threadIdx.x;
+    if (blockIdx.x == 0 && threadIdx.x < out_f) {
+        float t = 0.f;
+        for (int g = 0; g < B; ++g) t += s_dy[g * out_f + threadIdx.x];
+        db[threadIdx.x] = t;
+    }
+    if (i >= in_f) return;
+    float acc[NARROW_MAX];
+#pragma unroll
+    for (int j = 0; j < NARROW_MAX; ++j) acc[j] = 0.f;
+    for (int g = 0; g < B; ++g) {
+        const T* xr = TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f;
+        const float xv = ldf(xr + i);
+#pragma unroll
+        for (int j = 0; j < NARROW_MAX; ++j)
+            if (j < out_f) acc[j] = fmaf(s_dy[g * out_f + j], xv, acc[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < NARROW_MAX; ++j)
+        if (j < out_f) dW[(size_t)j * in_f + i] = acc[j];
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+fc_narrow_dgrad_kernel(const T* __restrict__ dY, const T* __restrict__ Wt, const T* __restrict__ ref, T* __restrict__ dX,
+                       int in_f, int out_f)
+{
+    __shared__ float s_d[NARROW_MAX];
+    const int g = blockIdx.y;
+    if (threadIdx.x < out_f) s_d[threadIdx.x] = ldf(dY + (size_t)g * out_f + threadIdx.x);
+    __syncthreads();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= in_f) return;
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < NARROW_MAX; ++j)
+        if (j < out_f) acc = fmaf(s_d[j], ldf(Wt + (size_t)j * in_f + i), acc);
+    if (ref != nullptr && !(ldf(ref + (size_t)g * in_f + i) > 0.f)) acc = 0.f;
+    stf(dX + (size_t)g * in_f + i, acc);
+}
+
+bool fc_narrow_supported(int out_f, int B) { return out_f <= NARROW_MAX && (size_t)B * out_f * 4 <= 40 * 1024; }
+
+template <typename T>
+static cudaError_t launch_fc_narrow_t(const FcNarrowArgs& a, cudaStream_t st)
+{
+    PtrTab tab{};
+    if (a.tab) tab = *a.tab;
+    const int tb = a.tab_b > 0 ? a.tab_b : 1;
+    if (a.pass == 0) {
+        if (a.tab) fc_narrow_fwd_kernel<T, true><<<a.B, 256, 0, st>>>(nullptr, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.in_f, a.out_f, a.relu);
+        else fc_narrow_fwd_kernel<T, false><<<a.B, 256, 0, st>>>((const T*)a.X, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.in_f, a.out_f, a.relu);
+    } else if (a.pass == 1) {
+        const size_t smem = (size_t)a.B * a.out_f * 4;
+        const int blocks = (a.in_f + 127) / 128;
+        if (a.tab) fc_narrow_wgrad_kernel<T, true><<<blocks, 128, smem, st>>>(nullptr, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+        else fc_narrow_wgrad_kernel<T, false><<<blocks, 128, smem, st>>>((const T*)a.X, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+    } else {
+        dim3 grid((a.in_f + 255) / 256, a.B);
+        fc_narrow_dgrad_kernel<T><<<grid, 256, 0, st>>>((const T*)a.dY, (const T*)a.W, (const T*)a.ref, (T*)a.dX, a.in_f, a.out_f);
+    }
+    return cudaGetLastError();
+}
+cudaError_t launch_fc_narrow(const FcNarrowArgs& a, bool bf16, cudaStream_t st)
+{
+    return bf16 ? launch_fc_narrow_t<__nv_bfloat16>(a, st) : launch_fc_narrow_t<float>(a, st);
 }
 
 // =============================================================================================

@@ -53,6 +53,8 @@ struct UmmaParams {
     const float* bias;
     const __nv_bfloat16* ref;   // UEPI_MASK: same layout as out; nullptr = no mask
     long split_stride;    // WGRAD: floats between split partial buffers
+    int bias_fused;       // WGRAD: the centre-tap CTAs of the first N tile also sum dy over the pixels (the bias gradient)
+    long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
 };
 
@@ -167,12 +169,13 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, int a_mn_major, int b_m
 constexpr int UMMA_THREADS = 192;
 constexpr int A_STAGE_BYTES = 16384;   // 128 rows x 128 B (K-major) or 2 boxes of 64 rows x 128 B (MN-major)
 
-template <int BN> struct Cfg {
+constexpr int CTRL_BYTES = 2048;       // [0,512) barriers + flags, [512,1536) bias (FWD)
+template <int MODE, int BN> struct Cfg {
     static constexpr int B_STAGE_BYTES = BN * 128;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
     static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
-    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 2048 /*barriers, bias*/;
+    static constexpr int TMEM_COLS = BN;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES;
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -182,7 +185,7 @@ template <int MODE, int BN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaParams p)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<MODE, BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* ctrl = smem + C::STAGES * C::STAGE_BYTES;
@@ -232,10 +235,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         k_end = p.ntaps * p.kchunks;
     }
     const int n_iters = k_end - k_begin;
+    const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? 4 : 0);
 
     // ---- one-time setup -----------------------------------------------------------------------
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -317,7 +322,32 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         const int q = warp % 4;               // TMEM lane quadrant of this warp
         const int row = q * 32 + lane;        // accumulator row handled by this thread
         bool ok = true;
-        if (lane == 0) ok = mbar_wait(acc_full, 0);
+        if (MODE == MODE_WGRAD && do_bias) {
+            // Bias gradient: thread `row` sums dy[pixel, m0 + row] over this CTA's pixel chunks, reading the A
+            // stage (64 pixel rows of 128 bytes per 64-channel box, 16-byte chunks XOR-swizzled by row % 8)
+            // while the MMA consumes it; pixel order is fixed, so the sum is deterministic.
+            float bsum = 0.f;
+            const uint32_t box_off = (uint32_t)(row / 64) * 8192u, c = (uint32_t)(row % 64);
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int s = it % C::STAGES;
+                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                if (lane == 0) ok = mbar_wait(&full[s], ph);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                const uint8_t* sa = smem + s * C::STAGE_BYTES + box_off;
+#pragma unroll 8
+                for (uint32_t k = 0; k < 64; ++k) {
+                    const uint32_t off = k * 128u + (((c >> 3) ^ (k & 7u)) << 4) + (c & 7u) * 2u;
+                    bsum += __bfloat162float(*(const __nv_bfloat16*)(sa + off));
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[s])) : "memory");
+            }
+            if (ok && (m0 + row) < m_hi)
+                ((float*)p.out)[(size_t)split * p.split_stride + p.bias_off + m0 + row] = bsum;
+            if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+        }
+        if (lane == 0 && ok) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
@@ -496,11 +526,11 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<MODE, BN>::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<BN>::SMEM_BYTES, st>>>(op.mapA, op.mapB, p);
+    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<MODE, BN>::SMEM_BYTES, st>>>(op.mapA, op.mapB, p);
     return cudaGetLastError();
 }
 
@@ -564,7 +594,7 @@ static bool conv_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
 static bool fc_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
 {
     // TMA needs 16-byte row strides: in and out multiples of 8; the reduce dims multiples of 64 keep every box row in bounds
-    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.in_f % 64 == 0 && lv.out_f % 8 == 0;
+    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.in_f % 64 == 0 && lv.out_f % 8 == 0 && lv.out_f > 16;
 }
 
 sb_status umma_plan_scratch(sb_model* m, size_t* floats)
@@ -580,7 +610,7 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
             const int bnt = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
             const long ctas = (long)cdiv_i(lv.Cout, 128) * cdiv_i(lv.Cin, bnt) * 9;
             const int S = wgrad_splits(ctas, total_chunks);
-            if (S > 1) need = need > (size_t)S * lv.n_w ? need : (size_t)S * lv.n_w;
+            if (S > 1) need = need > (size_t)S * (lv.n_w + lv.n_b) ? need : (size_t)S * (lv.n_w + lv.n_b);
         }
     }
     *floats = need;
@@ -655,12 +685,16 @@ sb_status umma_plan_layers(sb_model* m)
                 const long ctas = (long)p.m_tiles_per_shard * n_tiles * 9;
                 p.splits = wgrad_splits(ctas, p.total_chunks);
                 p.chunks_per_split = cdiv_i(p.total_chunks, p.splits);
+                p.splits = cdiv_i(p.total_chunks, p.chunks_per_split);   // no empty trailing split
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
-                p.split_stride = (long)lv.n_w;
+                // the bias gradient rides along: in the parameter arena the bias vector directly follows the
+                // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
+                p.split_stride = (long)(lv.n_w + lv.n_b);
+                p.bias_fused = 1; p.bias_off = (long)lv.n_w;
                 p.out = p.splits > 1 ? (void*)mv.ws : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
                 b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)n_tiles, (unsigned)(9 * p.splits));
-                if ((size_t)p.splits * lv.n_w > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
+                if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, cw, ch, cn)) return fail_plan();
                 if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, cw, ch, cn)) return fail_plan();
                 um.wgrad.enabled = true;
@@ -720,6 +754,7 @@ sb_status umma_plan_layers(sb_model* m)
                 const int n_tiles = cdiv_i(lv.in_f, b->bn);
                 p.splits = 1; p.chunks_per_split = p.total_chunks;
                 p.epi = UEPI_F32; p.ldc = lv.in_f; p.split_stride = 0;
+                p.bias_fused = 1; p.bias_off = (long)lv.n_w;
                 p.out = (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
                 b->grid = dim3((unsigned)(p.m_tiles_per_shard * K), (unsigned)n_tiles, 1);

