@@ -68,7 +68,8 @@ enum { SB_FP32 = 0, SB_BF16 = 1 };
 /* sb_config.flags */
 enum {
     SB_FLAG_INPUT_GRAD = 1,  /* also compute the gradient w.r.t. the network input (layer 0 dgrad) */
-    SB_FLAG_FORCE_SIMT = 2   /* use the CUDA-core kernels for every layer (cross-check / debugging) */
+    SB_FLAG_FORCE_SIMT = 2,  /* use the CUDA-core kernels for every layer (cross-check / debugging) */
+    SB_FLAG_PROFILE_LAYERS = 4 /* sb_profile_end reports one entry per (kernel class, layer): "name#layer" */
 };
 
 typedef struct {

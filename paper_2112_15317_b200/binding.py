@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(HERE, "libsplitbrain.so")
 SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
 SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT = 1, 2, 3, 4, 5
-SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT = 1, 2
+SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS = 1, 2, 4
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
 SB_DT_F32, SB_DT_BF16, SB_DT_U8, SB_DT_I32 = 0, 1, 2, 3
@@ -295,9 +295,9 @@ class Model:
 
     def profile_end(self):
         """Per kernel class: {'name', 'launches', 'ms_total', 'flops', 'bytes'} (algorithmic work)."""
-        arr = (sb_profile_entry * 64)()
+        arr = (sb_profile_entry * 256)()
         n = c_int32()
-        _check(sb_profile_end(self.h, self._stream(), arr, 64, byref(n)))
+        _check(sb_profile_end(self.h, self._stream(), arr, 256, byref(n)))
         return [dict(name=arr[i].name.decode(), launches=arr[i].launches, ms_total=arr[i].ms_total,
                      flops=arr[i].flops, bytes=arr[i].bytes) for i in range(n.value)]
 

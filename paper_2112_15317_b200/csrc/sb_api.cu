@@ -86,7 +86,8 @@ struct sb_model {
     bool have_x = false, have_labels = false, have_fwd = false;
     int64_t launches = 0, last_step_launches = 0;
     // per-launch event recording (sb_profile_begin / sb_profile_end)
-    struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; };
+    struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; int layer; };
+    int cur_layer = -1;   // layer whose kernels are being enqueued (profiling detail)
     bool debug_sync = false;   // SB_DEBUG_SYNC=1 in the environment: synchronise and check after every launch
     bool profiling = false;
     std::vector<Rec> recs;
@@ -241,7 +242,7 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
 // `tag` names the kernel class; flops/bytes are the algorithmic work of this launch.
 #define L_TRY(tag, flops, bytes, expr)                                                            \
     do {                                                                                          \
-        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes)};              \
+        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes), m->cur_layer}; \
         if (m->profiling) { rec_.e0 = m->next_event(); rec_.e1 = m->next_event();                 \
                             if (rec_.e0) cudaEventRecord(rec_.e0, st); }                          \
         cudaError_t e_ = (expr);                                                                  \
@@ -256,7 +257,7 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
 // Same bracket for the tensor-core launchers, which return sb_status.
 #define U_TRY(tag, flops, bytes, expr)                                                            \
     do {                                                                                          \
-        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes)};              \
+        sb_model::Rec rec_{tag, nullptr, nullptr, (double)(flops), (double)(bytes), m->cur_layer}; \
         if (m->profiling) { rec_.e0 = m->next_event(); rec_.e1 = m->next_event();                 \
                             if (rec_.e0) cudaEventRecord(rec_.e0, st); }                          \
         sb_status s_ = (expr);                                                                    \
@@ -274,6 +275,7 @@ inline const char* layer_input(const sb_model* m, int i) { return i > 0 ? m->L[i
 sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
 {
     Layer& l = m->L[i];
+    m->cur_layer = i;
     const bool bf = m->bf16;
     const int B = m->B, b = m->cfg.batch_per_replica;
     const double e = (double)m->esz;
@@ -349,6 +351,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
 sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
 {
     Layer& l = m->L[i];
+    m->cur_layer = i;
     const bool bf = m->bf16;
     const int B = m->B, b = m->cfg.batch_per_replica;
     const double e = (double)m->esz;
@@ -702,6 +705,7 @@ sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     cudaStream_t st = (cudaStream_t)stream;
+    m->cur_layer = -1;
     L_TRY("sgd", 0.0, (double)m->P * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, m->P, lr, momentum, st));
     m->last_step_launches = m->launches;
     return SB_OK;
@@ -822,13 +826,16 @@ sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32
     for (const sb_model::Rec& r : m->recs) {
         float ms = 0.f;
         CU_TRY(cudaEventElapsedTime(&ms, r.e0, r.e1));
+        char name[32];
+        if ((m->cfg.flags & SB_FLAG_PROFILE_LAYERS) && r.layer >= 0) snprintf(name, sizeof(name), "%.24s#%d", r.tag, r.layer);
+        else snprintf(name, sizeof(name), "%.31s", r.tag);
         int k = 0;
         for (; k < cnt; ++k)
-            if (strncmp(out[k].name, r.tag, sizeof(out[k].name)) == 0) break;
+            if (strncmp(out[k].name, name, sizeof(out[k].name)) == 0) break;
         if (k == cnt) {
             if (cnt == max_entries) continue;
             memset(&out[k], 0, sizeof(out[k]));
-            strncpy(out[k].name, r.tag, sizeof(out[k].name) - 1);
+            strncpy(out[k].name, name, sizeof(out[k].name) - 1);
             ++cnt;
         }
         out[k].launches += 1;

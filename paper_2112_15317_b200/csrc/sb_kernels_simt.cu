@@ -285,9 +285,31 @@ reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4*
         out[i] = t;
     }
 }
+// Many splits, few elements: 32 elements per block, 8 lanes share the splits of each element and are
+// combined in lane order (fixed order -> deterministic).
+__global__ void __launch_bounds__(256)
+reduce_partials_many_kernel(const float* __restrict__ part, size_t stride, float* __restrict__ out, size_t n, int splits)
+{
+    __shared__ float s[8][33];
+    const int e = threadIdx.x % 32, lane = threadIdx.x / 32;
+    const size_t i = blockIdx.x * 32ull + e;
+    float t = 0.f;
+    if (i < n)
+        for (int sp = lane; sp < splits; sp += 8) t += part[(size_t)sp * stride + i];
+    s[lane][e] = t;
+    __syncthreads();
+    if (lane == 0 && i < n) {
+        float r = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r += s[j][e];
+        out[i] = r;
+    }
+}
 cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st)
 {
-    if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0) {
+    if (splits >= 32 && n <= (1u << 20)) {
+        reduce_partials_many_kernel<<<cdiv((long)n, 32), 256, 0, st>>>(part, stride, out, n, splits);
+    } else if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0) {
         int blocks = cdiv((long)(n / 4), 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
         reduce_partials4_kernel<<<blocks, 256, 0, st>>>((const float4*)part, stride / 4, (float4*)out, n / 4, splits);
@@ -683,7 +705,7 @@ cudaError_t launch_conv_in_fwd(const ConvSimtArgs& a, bool bf16, cudaStream_t st
 int conv_in_wgrad_blocks(int B, int H, int W)
 {
     long chunks = ((long)B * H * W + 63) / 64;
-    return (int)(chunks < 148 * 4 ? chunks : 148 * 4);
+    return (int)(chunks < 148 * 2 ? chunks : 148 * 2);
 }
 template <typename T, int CIN>
 static cudaError_t launch_conv_in_wgrad_t(const WgradSimtArgs& a, cudaStream_t st)

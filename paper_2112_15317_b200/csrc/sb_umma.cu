@@ -579,11 +579,13 @@ static int pick_bn(int n_cols, long m_tiles)
     return bn;
 }
 
-// Conv weight-gradient split count: enough CTAs for ~2 waves, at least 4 pixel chunks per CTA.
+// Conv weight-gradient split count: fill the machine once (148 CTAs), keep at least 4 pixel chunks per
+// CTA, and never write more split buffers than the pixel work justifies (each split costs a full
+// float copy of the weight gradient in traffic).
 static int wgrad_splits(long ctas_without_split, int total_chunks)
 {
     int s = 1;
-    while (ctas_without_split * s < 296 && total_chunks / (s * 2) >= 4) s *= 2;
+    while (ctas_without_split * s < 148 && total_chunks / (s * 2) >= 4) s *= 2;
     return s;
 }
 
