@@ -227,6 +227,39 @@ sb_status sb_launch_count(const sb_model* m, int64_t* launches);
 
 const char* sb_last_error(void);
 
+/*
+ * (No counterpart in the paper: this entry point exists for callers that cannot allocate.)
+ *
+ * Weight and bias gradient of an input-layer 3x3 convolution (zero pad 1, stride 1), computed without
+ * any device allocation: dw[k,r,s,c] = sum_{n,h,w} dy[n,h,w,k] * x[n,h+r-1,w+s-1,c], db[k] = sum dy[n,h,w,k].
+ * It is the model path's input-layer weight-gradient kernel with its split partial sums kept in a
+ * fixed 2 MiB array that is part of the library image instead of the caller's arena.
+ *
+ * Who needs it: code that wants this gradient but may not create device memory at that moment, for
+ * example a monitoring or validation hook that runs beside a training job whose memory pool already
+ * owns the whole GPU (a cudaMalloc there can fail, and it would also stall the running job because
+ * device allocation synchronises the device), or a host program that forbids allocation after start-up.
+ * Such a caller passes its existing input and output buffers and nothing else.
+ *
+ *   x  : DEVICE, [B,H,W,Cin], float (SB_FP32) or bfloat16 (SB_BF16), one contiguous buffer
+ *   dy : DEVICE, [B,H,W,Cout], same dtype as x
+ *   dw : DEVICE, float [Cout,3,3,Cin], overwritten        db : DEVICE, float [Cout], overwritten
+ *   stream : cudaStream_t as void*; the call only enqueues two kernels.
+ * Limits (SB_ERR_UNSUPPORTED otherwise): Cin in {1,3,4} and Cout*(9*Cin+1) <= 4096, e.g. Cout <= 146
+ * for RGB inputs.  B, H, W are unlimited (at most 128 partial buffers are used whatever the size).
+ * The first call on each device looks up the scratch array's device address (with that device
+ * current); make that first call before any stream capture begins.  The library calls no cudaMalloc,
+ * cudaFree or other allocating routine here.
+ * The scratch array is shared by every call in the process and holds the previous call's partial
+ * sums; the kernels rewrite every value they later read, so no clearing is needed, but two calls
+ * that run concurrently on one GPU race on it: serialise them (same stream, or an event).
+ * Every GPU that loads the library holds the 2 MiB until the process exits.
+ * Errors are reported through the return code and sb_static_last_error().
+ */
+sb_status sb_conv_in_wgrad_static(const void* x, const void* dy, float* dw, float* db, int32_t B, int32_t H,
+                                  int32_t W, int32_t Cin, int32_t Cout, int32_t precision, void* stream);
+const char* sb_static_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -72,6 +72,7 @@ def _load():
         "sb_backward_layers": [c_void_p, c_int32, c_int32, c_void_p],
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
         "sb_launch_count": [c_void_p, P(c_int64)],
+        "sb_conv_in_wgrad_static": [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p],
         "sb_profile_begin": [c_void_p, c_void_p],
         "sb_profile_end": [c_void_p, c_void_p, P(sb_profile_entry), c_int32, P(c_int32)],
     }
@@ -81,11 +82,13 @@ def _load():
         fn.restype = c_int32
     lib.sb_last_error.argtypes = []
     lib.sb_last_error.restype = c_char_p
+    lib.sb_static_last_error.argtypes = []
+    lib.sb_static_last_error.restype = c_char_p
     return lib, sigs
 
 
 _lib, _SIGS = _load()
-EXPORTED = sorted(list(_SIGS) + ["sb_last_error"])
+EXPORTED = sorted(list(_SIGS) + ["sb_last_error", "sb_static_last_error"])
 
 # Same-named module-level entry points (raw status codes).
 sb_model_bytes = _lib.sb_model_bytes
@@ -104,12 +107,31 @@ sb_forward_layers = _lib.sb_forward_layers
 sb_backward_layers = _lib.sb_backward_layers
 sb_param_bytes = _lib.sb_param_bytes
 sb_launch_count = _lib.sb_launch_count
+sb_conv_in_wgrad_static = _lib.sb_conv_in_wgrad_static
 sb_profile_begin = _lib.sb_profile_begin
 sb_profile_end = _lib.sb_profile_end
 
 
 def sb_last_error() -> str:
     return _lib.sb_last_error().decode()
+
+
+def sb_static_last_error() -> str:
+    return _lib.sb_static_last_error().decode()
+
+
+def conv_in_wgrad_static(x, dy, dw, db, precision):
+    """Input-layer conv weight/bias gradient with the library's built-in scratch (no allocation anywhere).
+    x [B,H,W,Cin], dy [B,H,W,Cout]: device tensors of the precision's dtype; dw [Cout,3,3,Cin], db [Cout]: float
+    device tensors that receive the result.  Enqueues on torch's current stream."""
+    import torch
+    B, H, W, Cin = x.shape
+    Cout = dy.shape[3]
+    st = _lib.sb_conv_in_wgrad_static(c_void_p(x.data_ptr()), c_void_p(dy.data_ptr()), c_void_p(dw.data_ptr()),
+                                      c_void_p(db.data_ptr()), B, H, W, Cin, Cout, precision,
+                                      c_void_p(torch.cuda.current_stream().cuda_stream))
+    if st != SB_OK:
+        raise SBError(st, sb_static_last_error())
 
 
 def _check(status):
