@@ -82,19 +82,23 @@ def time_oracle(wl, steps, warmup):
 
 
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """nvidia-smi sampled every 50 ms in the background; stop() keeps the samples taken inside [t0, t1]
+    (wall clock of the timed region) or, if the region was shorter than the sampling period, the samples
+    nearest to it."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                                        "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
-    def stop(self):
+    def stop(self, t0, t1):
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -106,20 +110,24 @@ class ClockSampler:
         self.f.flush()
         rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
         os.unlink(self.f.name)
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        samples = []
         for r in rows:
             if len(r) < 8:
                 continue
             try:
-                sm.append(float(r[1])); mx.append(float(r[2]))
+                ts = datetime.datetime.strptime(r[0].strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                samples.append((ts, float(r[1]), float(r[2]), float(r[3]), [nm for nm, v in zip(names, r[4:8]) if v.strip().lower() == "active"]))
             except ValueError:
                 continue
-            for nm, v in zip(names, r[4:8]):
-                if v.strip().lower() == "active":
-                    reasons.add(nm)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        inside = [x for x in samples if t0 <= x[0] <= t1]
+        if not inside and samples:
+            mid = 0.5 * (t0 + t1)
+            inside = sorted(samples, key=lambda x: abs(x[0] - mid))[:3]
+        if inside:
+            out.update(sm_mhz=float(np.median([x[1] for x in inside])), sm_max_mhz=float(max(x[2] for x in inside)),
+                       power_w=float(np.median([x[3] for x in inside])),
+                       reasons=sorted({nm for x in inside for nm in x[4]}), samples=len(inside), in_window=bool(t0 <= inside[0][0] <= t1))
         return out
 
 
@@ -161,19 +169,21 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(args.warmup):
         step()
     loss_w = m.loss()
-    sampler = ClockSampler(local) if rank == 0 else None
     barrier()
+    t_wall0 = time.time()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    t_wall1 = time.time()
     ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     loss_t = m.loss()
 
     # end to end through the host-buffer entry point
@@ -187,9 +197,10 @@ def run_ours(args):
     ms_e2e = (time.perf_counter() - t0) * 1e3
     barrier()
 
-    # per-kernel-class timing (events around every launch), same steps again
+    # per-kernel-class timing (events around every launch), the same steps again (at most 50 of them)
+    psteps = min(args.steps, 50)
     m.profile_begin()
-    for _ in range(args.steps):
+    for _ in range(psteps):
         step()
     prof = m.profile_end()
     launches = m.launch_count()
@@ -222,14 +233,14 @@ def run_ours(args):
     else:
         roof = dict(bound="hbm", achieved=top["bytes"] / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update(kernel=top["name"], launches_per_step=top["launches"] // args.steps, share_of_kernel_time=top["ms_total"] / tot_ms,
+    roof.update(kernel=top["name"], launches_per_step=top["launches"] // psteps, share_of_kernel_time=top["ms_total"] / tot_ms,
                 traffic=traffic, peak_source=pk["source"] + (" sustained bf16" if roof["bound"] == "tensor" else " copy"),
                 avg_launch_us=top["ms_total"] * 1e3 / top["launches"])
     # whole-step roofline (the slower of all FLOPs at tensor peak and all bytes at HBM peak)
-    fl = sum(r["flops"] for r in prof) / args.steps
-    by = sum(r["bytes"] for r in prof) / args.steps
+    fl = sum(r["flops"] for r in prof) / psteps
+    by = sum(r["bytes"] for r in prof) / psteps
     t_roof = max(fl / (pk["tf_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9))
-    kernels = [dict(name=r["name"], launches_per_step=r["launches"] // args.steps, ms_per_step=r["ms_total"] / args.steps,
+    kernels = [dict(name=r["name"], launches_per_step=r["launches"] // psteps, ms_per_step=r["ms_total"] / psteps,
                     tflops=(r["flops"] / (r["ms_total"] * 1e-3) / 1e12 if r["flops"] else None),
                     gbs=r["bytes"] / (r["ms_total"] * 1e-3) / 1e9) for r in prof]
     cpu = None
@@ -280,8 +291,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
     args = ap.parse_args()
