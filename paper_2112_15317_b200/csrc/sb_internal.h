@@ -108,8 +108,18 @@ cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow
                        float lr, float mu, cudaStream_t st);
 cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cudaStream_t st);
 
-// Strided GEMM  C[m,n] = sum_k A(m,k) * B(n,k)  with A(m,k) = A[m*sAm + k*sAk], B(n,k) = B[n*sBn + k*sBk].
 enum { EPI_BIAS_ACT = 0, EPI_MASK = 1, EPI_F32 = 2 };
+// Ordered sum of split-reduction partial sums [split][rows][N] followed by the GEMM epilogue
+// (epi = EPI_BIAS_ACT or EPI_MASK below); N must be a multiple of 4.
+struct SplitKEpiArgs {
+    const float* part; size_t split_stride; int splits;
+    long rows; int N;
+    int epi; const float* bias; int relu; const void* ref;
+    void* out; int out_f32;
+};
+cudaError_t launch_splitk_epilogue(const SplitKEpiArgs& a, cudaStream_t st);
+
+// Strided GEMM  C[m,n] = sum_k A(m,k) * B(n,k)  with A(m,k) = A[m*sAm + k*sAk], B(n,k) = B[n*sBn + k*sBk].
 struct GemmSimtArgs {
     const void* A; long sAm, sAk;
     const void* B; long sBn, sBk;

@@ -322,6 +322,64 @@ cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out,
 }
 
 // =============================================================================================
+// Split-reduction epilogue of the tensor-core GEMMs: out = epi(sum_s part[s]) with the splits added in
+// order; epi = bias + ReLU (-> bf16 or float) or the ReLU mask (-> bf16).  Four columns per thread.
+// =============================================================================================
+template <int EPI>
+__global__ void __launch_bounds__(256)
+splitk_epilogue_kernel(const float* __restrict__ part, size_t split_stride, int splits, size_t n4, int N,
+                       const float* __restrict__ bias, int relu, const __nv_bfloat16* __restrict__ ref,
+                       void* __restrict__ out, int out_f32)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t e = i * 4;
+        float4 t = __ldg((const float4*)(part + e));
+        for (int s = 1; s < splits; ++s) {
+            const float4 v = __ldg((const float4*)(part + (size_t)s * split_stride + e));
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        if (EPI == EPI_BIAS_ACT) {
+            const float4 b = *(const float4*)(bias + (e % (size_t)N));
+            t.x += b.x; t.y += b.y; t.z += b.z; t.w += b.w;
+            if (relu) {
+                if (!(t.x > 0.f)) t.x = 0.f;
+                if (!(t.y > 0.f)) t.y = 0.f;
+                if (!(t.z > 0.f)) t.z = 0.f;
+                if (!(t.w > 0.f)) t.w = 0.f;
+            }
+        } else if (ref != nullptr) {
+            const uint2 r = *(const uint2*)(ref + e);
+            const __nv_bfloat16* rb = (const __nv_bfloat16*)&r;
+            if (!(__bfloat162float(rb[0]) > 0.f)) t.x = 0.f;
+            if (!(__bfloat162float(rb[1]) > 0.f)) t.y = 0.f;
+            if (!(__bfloat162float(rb[2]) > 0.f)) t.z = 0.f;
+            if (!(__bfloat162float(rb[3]) > 0.f)) t.w = 0.f;
+        }
+        if (out_f32) {
+            *(float4*)((float*)out + e) = t;
+        } else {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+            uint2 pk;
+            pk.x = *(uint32_t*)&lo;
+            pk.y = *(uint32_t*)&hi;
+            *(uint2*)((__nv_bfloat16*)out + e) = pk;
+        }
+    }
+}
+cudaError_t launch_splitk_epilogue(const SplitKEpiArgs& a, cudaStream_t st)
+{
+    if (a.N % 4 != 0) return cudaErrorInvalidValue;
+    const size_t n4 = (size_t)a.rows * a.N / 4;
+    int blocks = cdiv((long)n4, 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (a.epi == EPI_BIAS_ACT)
+        splitk_epilogue_kernel<EPI_BIAS_ACT><<<blocks, 256, 0, st>>>(a.part, a.split_stride, a.splits, n4, a.N, a.bias, a.relu, nullptr, a.out, a.out_f32);
+    else
+        splitk_epilogue_kernel<EPI_MASK><<<blocks, 256, 0, st>>>(a.part, a.split_stride, a.splits, n4, a.N, nullptr, 0, (const __nv_bfloat16*)a.ref, a.out, 0);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
 // 2x2 max-pool, stride 2.  One thread per pooled pixel and VEC channels (16-byte accesses when the
 // channel count allows).  Ties go to the first maximum in scan order (0,0),(0,1),(1,0),(1,1).
 // =============================================================================================

@@ -45,7 +45,9 @@ struct UmmaParams {
     // WGRAD
     int m_total;          // rows of the weight gradient (Cout / out-features)
     int m_shards, m_tiles_per_shard;
-    int splits, chunks_per_split, total_chunks;
+    int splits, chunks_per_split, total_chunks;   // split of the reduction (k-iterations) over blockIdx.z
+    int stages;           // depth of the shared-memory ring (<= MAX_STAGES)
+    float* part;          // FWD/DGRAD with splits > 1: raw float partial sums [split][pixel][n_total]
     // epilogue
     int epi, relu, out_f32;
     void* out;            // FWD/DGRAD: [pixels][ldc] bf16 (or float when out_f32); WGRAD: float partial sums
@@ -170,12 +172,13 @@ constexpr int UMMA_THREADS = 192;
 constexpr int A_STAGE_BYTES = 16384;   // 128 rows x 128 B (K-major) or 2 boxes of 64 rows x 128 B (MN-major)
 
 constexpr int CTRL_BYTES = 2048;       // [0,512) barriers + flags, [512,1536) bias (FWD)
+constexpr int MAX_STAGES = 8;
 template <int MODE, int BN> struct Cfg {
     static constexpr int B_STAGE_BYTES = BN * 128;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr int MAX_STAGES_FIT = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);   // what fits in 227 KB
     static constexpr int TMEM_COLS = BN;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES;
+    static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES; }
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -188,10 +191,11 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     using C = Cfg<MODE, BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* ctrl = smem + C::STAGES * C::STAGE_BYTES;
-    uint64_t* full = (uint64_t*)ctrl;                 // [STAGES]
-    uint64_t* empty = full + C::STAGES;               // [STAGES]
-    uint64_t* acc_full = empty + C::STAGES;           // [1]
+    const int STAGES = p.stages;
+    uint8_t* ctrl = smem + STAGES * C::STAGE_BYTES;
+    uint64_t* full = (uint64_t*)ctrl;                 // [MAX_STAGES]
+    uint64_t* empty = full + MAX_STAGES;              // [MAX_STAGES]
+    uint64_t* acc_full = empty + MAX_STAGES;          // [1]
     uint32_t* tmem_slot = (uint32_t*)(acc_full + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     float* s_bias = (float*)(ctrl + 512);             // [BN]
@@ -227,20 +231,17 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         ph0 = ((m_idx / p.tiles_w) % p.tiles_h) * p.bh;
         pn0 = (m_idx / (p.tiles_w * p.tiles_h)) * p.bn;
     }
-    int k_begin = 0, k_end = 0;   // k-iterations of this CTA
-    if (MODE == MODE_WGRAD) {
-        k_begin = split * p.chunks_per_split;
-        k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
-    } else {
-        k_end = p.ntaps * p.kchunks;
-    }
+    if (MODE != MODE_WGRAD) split = blockIdx.z;
+    // k-iterations of this CTA: a contiguous range of the reduction
+    const int k_begin = split * p.chunks_per_split;
+    const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
     const int n_iters = k_end - k_begin;
     const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? 4 : 0);
 
     // ---- one-time setup -----------------------------------------------------------------------
     if (threadIdx.x == 0) {
         // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -263,8 +264,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         // =========================== TMA producer ===============================================
         if (lane == 0) {
             for (int it = 0; it < n_iters; ++it) {
-                const int s = it % C::STAGES;
-                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
                 if (*abort_flag) break;
                 uint8_t* sa = smem + s * C::STAGE_BYTES;
@@ -301,8 +302,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_WGRAD, MODE != MODE_FWD);
             bool ok = true;
             for (int it = 0; it < n_iters && ok; ++it) {
-                const int s = it % C::STAGES;
-                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
@@ -329,8 +330,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             float bsum = 0.f;
             const uint32_t box_off = (uint32_t)(row / 64) * 8192u, c = (uint32_t)(row % 64);
             for (int it = 0; it < n_iters && ok; ++it) {
-                const int s = it % C::STAGES;
-                const uint32_t ph = (uint32_t)((it / C::STAGES) & 1);
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (lane == 0) ok = mbar_wait(&full[s], ph);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
@@ -376,6 +377,19 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
                 const int ncol = n0 + c0;
                 const bool full16 = ncol + 16 <= n_hi;
+                if (MODE != MODE_WGRAD && p.splits > 1) {
+                    // split reduction: raw partial sums; bias / ReLU / mask / rounding happen in the reduce kernel
+                    float* op = p.part + (size_t)split * p.split_stride + row_off + ncol;   // ldc == n_total in these modes
+                    if (full16 && ((p.n_total & 3) == 0) && ((ncol & 3) == 0)) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (ncol + j < n_hi) op[j] = f[j];
+                    }
+                    continue;
+                }
                 if (p.epi == UEPI_BIAS_ACT) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -526,11 +540,13 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<MODE, BN>::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Cfg<MODE, BN>::smem_bytes(Cfg<MODE, BN>::MAX_STAGES_FIT));
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<MODE, BN>::SMEM_BYTES, st>>>(op.mapA, op.mapB, p);
+    if (p.stages < 1 || p.stages > Cfg<MODE, BN>::MAX_STAGES_FIT) return cudaErrorInvalidValue;
+    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<MODE, BN>::smem_bytes(p.stages), st>>>(op.mapA, op.mapB, p);
     return cudaGetLastError();
 }
 
@@ -550,18 +566,29 @@ struct OpBlock {
     UmmaParams p;
     int bn;
     dim3 grid;
+    long rows;     // output rows (pixels / batch rows) of a FWD / DGRAD op
 };
 static_assert(sizeof(OpBlock) <= sizeof(((UmmaOp*)nullptr)->blob), "UmmaOp::blob too small");
 static OpBlock* blk(UmmaOp& op) { return (OpBlock*)op.blob; }
 static const OpBlock* blk(const UmmaOp& op) { return (const OpBlock*)op.blob; }
 
-static sb_status launch_op(const UmmaOp& op, cudaStream_t st)
+static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr)
 {
     const OpBlock* b = blk(op);
     cudaError_t e;
     if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, b->p, b->grid, st);
     else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, b->p, b->grid, st);
     else e = launch_mode<MODE_WGRAD>(b->bn, op, b->p, b->grid, st);
+    if (e == cudaSuccess && b->p.mode != MODE_WGRAD && b->p.splits > 1) {
+        // ordered sum of the split partial sums + the epilogue the tensor-core kernel skipped
+        SplitKEpiArgs a{};
+        a.part = b->p.part; a.split_stride = (size_t)b->p.split_stride; a.splits = b->p.splits;
+        a.rows = b->rows; a.N = b->p.n_total;
+        a.epi = b->p.epi == UEPI_BIAS_ACT ? EPI_BIAS_ACT : EPI_MASK;
+        a.bias = b->p.bias; a.relu = b->p.relu; a.ref = b->p.ref; a.out = b->p.out; a.out_f32 = b->p.out_f32;
+        e = launch_splitk_epilogue(a, st);
+        if (launches) ++*launches;
+    }
     if (e != cudaSuccess) {
         snprintf(g_umma_err, sizeof(g_umma_err), "tensor-core launch failed: %s", cudaGetErrorString(e));
         return SB_ERR_CUDA;
@@ -571,12 +598,30 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st)
 
 const char* umma_last_error() { return g_umma_err; }
 
-static int pick_bn(int n_cols, long m_tiles)
+// Tile plan of a FWD / DGRAD GEMM: N tile, reduction split and ring depth.
+//  * N tile as wide as the column count allows (operand traffic from L2 per FLOP falls with the tile width),
+//  * if that leaves fewer CTAs than ~0.8 waves, split the reduction over blockIdx.z (float partial sums,
+//    reduced in split order by splitk_epilogue) while every CTA keeps at least 4 k-iterations,
+//  * ring depth = k-iterations per CTA, capped by what fits; for grids of several waves the ring is kept
+//    shallow enough that two CTAs share an SM, so one CTA's epilogue overlaps the other's main loop.
+struct TilePlan { int bn, splits, cps, stages; };
+static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters)
 {
-    // widest tile that still leaves at least ~one wave of CTAs; never wider than the column count needs
-    int bn = 256;
-    while (bn > 64 && (bn / 2 >= n_cols || m_tiles * cdiv_i(n_cols, bn) < 148)) bn /= 2;
-    return bn;
+    TilePlan t;
+    t.bn = n_cols_per_shard >= 256 ? 256 : (n_cols_per_shard >= 128 ? 128 : 64);
+    const long tiles = m_tiles * cdiv_i(n_cols_per_shard, t.bn) * shards;
+    int s = 1;
+    while (tiles * s < 120 && k_iters / (s * 2) >= 4) s *= 2;
+    t.cps = cdiv_i(k_iters, s);
+    t.splits = cdiv_i(k_iters, t.cps);
+    const int fit = t.bn >= 256 ? 4 : (t.bn >= 128 ? 6 : 8);
+    int st = t.cps < fit ? t.cps : fit;
+    if (tiles * t.splits >= 296) {               // >= 2 waves: prefer two resident CTAs per SM
+        const int two = t.bn >= 256 ? 2 : (t.bn >= 128 ? 3 : 4);
+        if (t.bn < 256 && st > two) st = two;
+    }
+    t.stages = st < 1 ? 1 : st;
+    return t;
 }
 
 // Conv weight-gradient split count: fill the machine once (148 CTAs), keep at least 4 pixel chunks per
@@ -599,20 +644,63 @@ static bool fc_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
     return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.in_f % 64 == 0 && lv.out_f % 8 == 0 && lv.out_f > 16;
 }
 
+// Geometry shared by the scratch sizing pass and the real planning pass.
+struct ConvGeom {
+    int bw, bh, bn, tw, th, tn;      // 128-pixel boxes (FWD / DGRAD M tiles)
+    long m_tiles;
+    TilePlan fwd, dgrad;
+    int cw, ch, cn, ctw, cth, ctn, total_chunks;   // 64-pixel boxes (WGRAD k-chunks)
+    int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps;
+};
+static ConvGeom conv_geom(const LayerView& lv, int B)
+{
+    ConvGeom g;
+    choose_box(lv.W, lv.H, B, 128, &g.bw, &g.bh, &g.bn);
+    g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
+    g.m_tiles = (long)g.tw * g.th * g.tn;
+    g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64));
+    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64));
+    choose_box(lv.W, lv.H, B, 64, &g.cw, &g.ch, &g.cn);
+    g.ctw = cdiv_i(lv.W, g.cw); g.cth = cdiv_i(lv.H, g.ch); g.ctn = cdiv_i(B, g.cn);
+    g.total_chunks = g.ctw * g.cth * g.ctn;
+    g.wg_bn = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
+    g.wg_n_tiles = cdiv_i(lv.Cin, g.wg_bn);
+    g.wg_m_tiles = cdiv_i(lv.Cout, 128);
+    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * 9, g.total_chunks);
+    g.wg_cps = cdiv_i(g.total_chunks, s);
+    g.wg_splits = cdiv_i(g.total_chunks, g.wg_cps);   // no empty trailing split
+    return g;
+}
+struct FcGeom {
+    int m_tiles;
+    TilePlan fwd, dgrad;
+};
+static FcGeom fc_geom(const LayerView& lv, int B, int K)
+{
+    FcGeom g;
+    g.m_tiles = cdiv_i(B, 128);
+    g.fwd = plan_tiles(cdiv_i(lv.out_f, K), K, g.m_tiles, lv.in_f / 64);
+    g.dgrad = plan_tiles(lv.in_f, 1, g.m_tiles, cdiv_i(lv.out_f, 64));
+    return g;
+}
+
 sb_status umma_plan_scratch(sb_model* m, size_t* floats)
 {
     ModelView mv = model_view(m);
     size_t need = 0;
+    auto upd = [&](size_t v) { if (v > need) need = v; };
     for (int i = 0; i < mv.n_layers; ++i) {
         LayerView lv = layer_view(m, i);
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            int bw, bh, bn;
-            choose_box(lv.W, lv.H, mv.B, 64, &bw, &bh, &bn);
-            const int total_chunks = cdiv_i(lv.W, bw) * cdiv_i(lv.H, bh) * cdiv_i(mv.B, bn);
-            const int bnt = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
-            const long ctas = (long)cdiv_i(lv.Cout, 128) * cdiv_i(lv.Cin, bnt) * 9;
-            const int S = wgrad_splits(ctas, total_chunks);
-            if (S > 1) need = need > (size_t)S * (lv.n_w + lv.n_b) ? need : (size_t)S * (lv.n_w + lv.n_b);
+            ConvGeom g = conv_geom(lv, mv.B);
+            const size_t pix = (size_t)mv.B * lv.H * lv.W;
+            if (g.wg_splits > 1) upd((size_t)g.wg_splits * (lv.n_w + lv.n_b));
+            if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * pix * lv.Cout);
+            if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * pix * lv.Cin);
+        } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
+            FcGeom g = fc_geom(lv, mv.B, mv.cfg->K);
+            if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * mv.B * lv.out_f);
+            if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * mv.B * lv.in_f);
         }
     }
     *floats = need;
@@ -620,6 +708,21 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
 }
 
 static sb_status fail_plan() { return SB_ERR_CUDA; }
+
+// Fills the split / ring fields of a FWD or DGRAD op from its tile plan.
+static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles, int n_tiles_total, float* ws, size_t rows)
+{
+    UmmaParams& p = b->p;
+    b->bn = t.bn;
+    p.total_chunks = k_iters;
+    p.chunks_per_split = t.cps;
+    p.splits = t.splits;
+    p.stages = t.stages;
+    p.part = t.splits > 1 ? ws : nullptr;
+    p.split_stride = (long)(rows * (size_t)p.n_total);
+    b->grid = dim3((unsigned)m_tiles, (unsigned)n_tiles_total, (unsigned)t.splits);
+    b->rows = (long)rows;
+}
 
 sb_status umma_plan_layers(sb_model* m)
 {
@@ -631,24 +734,21 @@ sb_status umma_plan_layers(sb_model* m)
         UmmaLayer& um = *lv.um;
         const bool want_in_grad = i > 0;
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            int bw, bh, bn;
-            choose_box(lv.W, lv.H, B, 128, &bw, &bh, &bn);
-            const int tw = cdiv_i(lv.W, bw), th = cdiv_i(lv.H, bh), tn = cdiv_i(B, bn);
-            const long m_tiles = (long)tw * th * tn;
+            const ConvGeom g = conv_geom(lv, B);
+            const size_t pix = (size_t)B * lv.H * lv.W;
             // ---- forward ----
             {
                 OpBlock* b = blk(um.fwd);
                 memset(b, 0, sizeof(*b));
                 UmmaParams& p = b->p;
-                p.mode = MODE_FWD; p.ntaps = 9; p.bw = bw; p.bh = bh; p.bn = bn; p.W = lv.W; p.H = lv.H; p.N = B;
-                p.tiles_w = tw; p.tiles_h = th; p.tiles_n = tn; p.kchunks = lv.Cin / 64; p.w_cols = lv.Cin;
+                p.mode = MODE_FWD; p.ntaps = 9; p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = g.tw; p.tiles_h = g.th; p.tiles_n = g.tn; p.kchunks = lv.Cin / 64; p.w_cols = lv.Cin;
                 p.n_total = lv.Cout; p.shards = 1;
-                b->bn = pick_bn(lv.Cout, m_tiles);
-                p.tiles_per_shard = cdiv_i(lv.Cout, b->bn);
+                p.tiles_per_shard = cdiv_i(lv.Cout, g.fwd.bn);
                 p.epi = UEPI_BIAS_ACT; p.relu = 1; p.out_f32 = 0; p.out = lv.act; p.ldc = lv.Cout; p.bias = mv.Wm + lv.p_b;
                 p.status = mv.status;
-                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
-                if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, bw, bh, bn)) return fail_plan();
+                apply_plan(b, g.fwd, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
+                if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->bn)) return fail_plan();
                 um.fwd.enabled = true;
             }
@@ -657,37 +757,32 @@ sb_status umma_plan_layers(sb_model* m)
                 OpBlock* b = blk(um.dgrad);
                 memset(b, 0, sizeof(*b));
                 UmmaParams& p = b->p;
-                p.mode = MODE_DGRAD; p.ntaps = 9; p.bw = bw; p.bh = bh; p.bn = bn; p.W = lv.W; p.H = lv.H; p.N = B;
-                p.tiles_w = tw; p.tiles_h = th; p.tiles_n = tn; p.kchunks = lv.Cout / 64; p.w_cols = lv.Cin;
+                p.mode = MODE_DGRAD; p.ntaps = 9; p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = g.tw; p.tiles_h = g.th; p.tiles_n = g.tn; p.kchunks = lv.Cout / 64; p.w_cols = lv.Cin;
                 p.n_total = lv.Cin; p.shards = 1;
-                b->bn = pick_bn(lv.Cin, m_tiles);
-                p.tiles_per_shard = cdiv_i(lv.Cin, b->bn);
+                p.tiles_per_shard = cdiv_i(lv.Cin, g.dgrad.bn);
                 p.epi = UEPI_MASK; p.out = lv.d_below; p.ldc = lv.Cin;
                 p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
                 p.status = mv.status;
-                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
-                if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, bw, bh, bn)) return fail_plan();
+                apply_plan(b, g.dgrad, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
+                if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, 64)) return fail_plan();
                 um.dgrad.enabled = true;
             }
             // ---- weight gradient ----
             {
-                int cw, ch, cn;
-                choose_box(lv.W, lv.H, B, 64, &cw, &ch, &cn);
                 OpBlock* b = blk(um.wgrad);
                 memset(b, 0, sizeof(*b));
                 UmmaParams& p = b->p;
-                p.mode = MODE_WGRAD; p.ntaps = 9; p.bw = cw; p.bh = ch; p.bn = cn; p.W = lv.W; p.H = lv.H; p.N = B;
-                p.tiles_w = cdiv_i(lv.W, cw); p.tiles_h = cdiv_i(lv.H, ch); p.tiles_n = cdiv_i(B, cn);
-                p.total_chunks = p.tiles_w * p.tiles_h * p.tiles_n;
+                p.mode = MODE_WGRAD; p.ntaps = 9; p.bw = g.cw; p.bh = g.ch; p.bn = g.cn; p.W = lv.W; p.H = lv.H; p.N = B;
+                p.tiles_w = g.ctw; p.tiles_h = g.cth; p.tiles_n = g.ctn;
+                p.total_chunks = g.total_chunks;
                 p.w_cols = lv.Cin; p.n_total = lv.Cin; p.shards = 1; p.tiles_per_shard = 1;
-                p.m_total = lv.Cout; p.m_shards = 1; p.m_tiles_per_shard = cdiv_i(lv.Cout, 128);
-                b->bn = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
-                const int n_tiles = cdiv_i(lv.Cin, b->bn);
-                const long ctas = (long)p.m_tiles_per_shard * n_tiles * 9;
-                p.splits = wgrad_splits(ctas, p.total_chunks);
-                p.chunks_per_split = cdiv_i(p.total_chunks, p.splits);
-                p.splits = cdiv_i(p.total_chunks, p.chunks_per_split);   // no empty trailing split
+                p.m_total = lv.Cout; p.m_shards = 1; p.m_tiles_per_shard = g.wg_m_tiles;
+                b->bn = g.wg_bn;
+                p.splits = g.wg_splits;
+                p.chunks_per_split = g.wg_cps;
+                p.stages = g.wg_cps < (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8)) ? g.wg_cps : (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8));
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
                 // the bias gradient rides along: in the parameter arena the bias vector directly follows the
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
@@ -695,15 +790,16 @@ sb_status umma_plan_layers(sb_model* m)
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
                 p.out = p.splits > 1 ? (void*)mv.ws : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
-                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)n_tiles, (unsigned)(9 * p.splits));
+                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 * p.splits));
                 if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
-                if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, cw, ch, cn)) return fail_plan();
-                if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, cw, ch, cn)) return fail_plan();
+                if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
+                if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch, g.cn)) return fail_plan();
                 um.wgrad.enabled = true;
             }
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
             const int K = mv.cfg->K;
-            const int m_tiles = cdiv_i(B, 128);
+            const FcGeom g = fc_geom(lv, B, K);
+            const int m_tiles = g.m_tiles;
             // ---- forward: Y[:, shard j] = X W_j^T + b_j ; N tiles enumerated per shard ----
             {
                 OpBlock* b = blk(um.fwd);
@@ -712,12 +808,10 @@ sb_status umma_plan_layers(sb_model* m)
                 p.mode = MODE_FWD; p.ntaps = 1; p.bw = 1; p.bh = 1; p.bn = 128; p.W = 1; p.H = 1; p.N = B;
                 p.tiles_w = 1; p.tiles_h = 1; p.tiles_n = m_tiles; p.kchunks = lv.in_f / 64; p.w_cols = lv.in_f;
                 p.n_total = lv.out_f; p.shards = K;
-                b->bn = 64;
-                const int widest = cdiv_i(lv.out_f, K);
-                p.tiles_per_shard = cdiv_i(widest, b->bn);
+                p.tiles_per_shard = cdiv_i(cdiv_i(lv.out_f, K), g.fwd.bn);
                 p.epi = UEPI_BIAS_ACT; p.relu = lv.relu ? 1 : 0; p.out_f32 = lv.kind == SB_FC; p.out = lv.act; p.ldc = lv.out_f;
                 p.bias = mv.Wm + lv.p_b; p.status = mv.status;
-                b->grid = dim3((unsigned)m_tiles, (unsigned)(p.tiles_per_shard * K), 1);
+                apply_plan(b, g.fwd, p.kchunks, m_tiles, p.tiles_per_shard * K, mv.ws, (size_t)B);
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->bn)) return fail_plan();
                 um.fwd.enabled = true;
@@ -730,12 +824,11 @@ sb_status umma_plan_layers(sb_model* m)
                 p.mode = MODE_DGRAD; p.ntaps = 1; p.bw = 1; p.bh = 1; p.bn = 128; p.W = 1; p.H = 1; p.N = B;
                 p.tiles_w = 1; p.tiles_h = 1; p.tiles_n = m_tiles; p.kchunks = cdiv_i(lv.out_f, 64); p.w_cols = lv.in_f;
                 p.n_total = lv.in_f; p.shards = 1;
-                b->bn = 64;
-                p.tiles_per_shard = cdiv_i(lv.in_f, b->bn);
+                p.tiles_per_shard = cdiv_i(lv.in_f, g.dgrad.bn);
                 p.epi = UEPI_MASK; p.out = lv.d_below; p.ldc = lv.in_f;
                 p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
                 p.status = mv.status;
-                b->grid = dim3((unsigned)m_tiles, (unsigned)p.tiles_per_shard, 1);
+                apply_plan(b, g.dgrad, p.kchunks, m_tiles, p.tiles_per_shard, mv.ws, (size_t)B);
                 if (!act_map(&um.dgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, 64)) return fail_plan();
                 um.dgrad.enabled = true;
@@ -755,6 +848,7 @@ sb_status umma_plan_layers(sb_model* m)
                 b->bn = lv.in_f >= 256 ? 256 : (lv.in_f >= 128 ? 128 : 64);
                 const int n_tiles = cdiv_i(lv.in_f, b->bn);
                 p.splits = 1; p.chunks_per_split = p.total_chunks;
+                p.stages = p.total_chunks < 4 ? p.total_chunks : 4;
                 p.epi = UEPI_F32; p.ldc = lv.in_f; p.split_stride = 0;
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
                 p.out = (void*)(mv.Gm + lv.p_w);
@@ -769,10 +863,10 @@ sb_status umma_plan_layers(sb_model* m)
     return SB_OK;
 }
 
-sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st); }
-sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st); }
-sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st); }
-sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st); }
+sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st, launch_counter(m)); }
+sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st, launch_counter(m)); }
+sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st, launch_counter(m)); }
+sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st, launch_counter(m)); }
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->wgrad, st); }
 
 sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part)
