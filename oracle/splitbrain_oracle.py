@@ -172,10 +172,15 @@ class OracleModel:
     """The partitioned network: one copy of the (replicated, always in-sync) conv parameters,
     K shards of every FC layer, momentum buffers of the same shapes."""
 
-    def __init__(self, layers, H, W, C, b, R, K, real="float", bf16=False):
+    def __init__(self, layers, H, W, C, b, R, K, real="float", bf16=False, loss_B=None):
         self.layers = list(layers)
         self.H, self.W, self.C, self.b, self.R, self.K = H, W, C, b, R, K
         self.B = b * R
+        # loss_B: size of the batch the mean loss is taken over.  It defaults to this model's own batch; a
+        # test that follows a few sampled images of a larger batch sets it to that batch size, so that the
+        # per-row gradients (softmax - onehot)/loss_B are the ones those rows have inside the large batch
+        # (every row's forward and activation-gradient computation is independent of the other rows).
+        self.loss_B = loss_B if loss_B is not None else self.B
         self.P = Prims(real)
         self.dt = self.P.dt
         self.bf16 = bf16
@@ -282,7 +287,7 @@ class OracleModel:
             elif kind == LOSS:
                 # 5. log-softmax + NLL, mean over the full batch
                 self.logits = X
-                self.row_loss, self.dZ = P.softmax_xent(X, labels, 1.0 / self.B)
+                self.row_loss, self.dZ = P.softmax_xent(X, labels, 1.0 / self.loss_B)
                 self.loss = self.dt(np.sum(self.row_loss, dtype=self.dt) / self.dt(self.B))
         return self.loss
 
@@ -363,5 +368,5 @@ class OracleModel:
         return loss
 
 
-def from_workload(wl, real="float", bf16=False) -> OracleModel:
-    return OracleModel(wl.layers, wl.H, wl.W, wl.C, wl.b, wl.R, wl.K, real=real, bf16=bf16)
+def from_workload(wl, real="float", bf16=False, loss_B=None) -> OracleModel:
+    return OracleModel(wl.layers, wl.H, wl.W, wl.C, wl.b, wl.R, wl.K, real=real, bf16=bf16, loss_B=loss_B)

@@ -311,6 +311,23 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         const double flops = 2.0 * B * (double)l.in_f * l.out_f;
         const double bytes = (double)B * l.in_f * e + (double)l.n_w * e + (double)B * l.out_f * (l.kind == SB_FC ? 4.0 : e);
         if (l.um.fwd.enabled) {
+            if (i == 0) {
+                // The tensor-core kernel reads the gathered input through one tensor map: replica buffers that
+                // already lie back to back are used in place; scattered ones are first copied into the staging area.
+                bool contiguous = true;
+                const size_t rep_bytes = (size_t)b * m->in_per_img * m->esz;
+                for (int r = 1; r < m->cfg.R; ++r)
+                    contiguous = contiguous && (const char*)m->x_tab.p[r] == (const char*)m->x_tab.p[0] + (size_t)r * rep_bytes;
+                const void* src = m->x_tab.p[0];
+                if (!contiguous) {
+                    for (int r = 0; r < m->cfg.R; ++r)
+                        if (m->x_tab.p[r] != m->stage_x + (size_t)r * rep_bytes)
+                            CU_TRY(cudaMemcpyAsync(m->stage_x + (size_t)r * rep_bytes, m->x_tab.p[r], rep_bytes, cudaMemcpyDeviceToDevice, st));
+                    src = m->stage_x;
+                }
+                sb_status bs = umma_bind_input(m, src);
+                if (bs != SB_OK) return fail(bs, "%s", umma_last_error());
+            }
             U_TRY("fc_fwd_umma", flops, bytes, umma_fc_fwd(m, i, st));
             ++m->launches;
             break;
@@ -590,7 +607,7 @@ ModelView model_view(sb_model* m)
     ModelView v{};
     v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
     v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; v.ws_floats = m->ws_floats; v.status = m->status;
-    v.input_grad = m->input_grad; v.x_tab = &m->x_tab;
+    v.input_grad = m->input_grad; v.x_tab = &m->x_tab; v.stage_x = m->stage_x;
     return v;
 }
 LayerView layer_view(sb_model* m, int i)

@@ -641,7 +641,8 @@ static bool conv_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
 static bool fc_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
 {
     // TMA needs 16-byte row strides: in and out multiples of 8; the reduce dims multiples of 64 keep every box row in bounds
-    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && layer > 0 && lv.in_f % 64 == 0 && lv.out_f % 8 == 0 && lv.out_f > 16;
+    (void)layer;   // a first-layer FC reads the network input through a tensor map bound at forward time
+    return mv.bf16 && !(mv.cfg->flags & SB_FLAG_FORCE_SIMT) && lv.in_f % 64 == 0 && lv.out_f % 8 == 0 && lv.out_f > 16;
 }
 
 // Geometry shared by the scratch sizing pass and the real planning pass.
@@ -800,6 +801,8 @@ sb_status umma_plan_layers(sb_model* m)
             const int K = mv.cfg->K;
             const FcGeom g = fc_geom(lv, B, K);
             const int m_tiles = g.m_tiles;
+            if (i == 0) lv.in_act = mv.stage_x;   // placeholder; rebound to the caller's input by umma_bind_input
+            const bool fc_in_grad = i > 0 || (mv.cfg->flags & SB_FLAG_INPUT_GRAD);
             // ---- forward: Y[:, shard j] = X W_j^T + b_j ; N tiles enumerated per shard ----
             {
                 OpBlock* b = blk(um.fwd);
@@ -817,7 +820,7 @@ sb_status umma_plan_layers(sb_model* m)
                 um.fwd.enabled = true;
             }
             // ---- data gradient: dX = sum_j dY_j W_j = one reduction over the concatenated width ----
-            if (want_in_grad && lv.out_f % 8 == 0) {
+            if (fc_in_grad && lv.out_f % 8 == 0) {
                 OpBlock* b = blk(um.dgrad);
                 memset(b, 0, sizeof(*b));
                 UmmaParams& p = b->p;
@@ -860,6 +863,18 @@ sb_status umma_plan_layers(sb_model* m)
             }
         }
     }
+    return SB_OK;
+}
+
+sb_status umma_bind_input(sb_model* m, const void* x)
+{
+    ModelView mv = model_view(m);
+    LayerView lv = layer_view(m, 0);
+    UmmaLayer& um = *lv.um;
+    if (um.bound_input == x) return SB_OK;
+    if (um.fwd.enabled && !act_map(&um.fwd.mapA, x, mv.B, 1, 1, lv.in_f, 1, 1, 128)) return SB_ERR_CUDA;
+    if (um.wgrad.enabled && !act_map(&um.wgrad.mapB, x, mv.B, 1, 1, lv.in_f, 1, 1, 64)) return SB_ERR_CUDA;
+    um.bound_input = x;
     return SB_OK;
 }
 

@@ -16,6 +16,7 @@ struct UmmaOp {
 };
 struct UmmaLayer {
     UmmaOp fwd, dgrad, wgrad;
+    const void* bound_input = nullptr;   // layer 0 only: the input buffer the tensor maps currently point at
 };
 
 // Read-only views of the model for the planner in sb_umma.cu.
@@ -30,6 +31,7 @@ struct ModelView {
     uint32_t* status;
     char* input_grad;
     const PtrTab* x_tab;
+    char* stage_x;        // contiguous [B, input] staging area inside the arena
 };
 struct LayerView {
     int kind, H, W, Cin, Cout, in_f, out_f;
@@ -56,6 +58,8 @@ sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st);
 // Launches the weight-gradient kernel; *splits > 1 means it wrote split partial sums at *part
 // (to be reduced in split order by the caller), else it wrote the gradient itself.
 sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part);
+// First-layer FC: points the tensor maps that read the network input at `x` ([B, in] contiguous, bf16).
+sb_status umma_bind_input(sb_model* m, const void* x);
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);

@@ -267,3 +267,22 @@ def test_bf16_mode_stays_close_to_fp32_mode():
     for ga, gb in zip(a.full_grads(), b_.full_grads()):
         if ga is not None:
             assert np.linalg.norm(gb["w"] - ga["w"]) / np.linalg.norm(ga["w"]) < 0.2
+
+
+def test_sampled_rows_of_a_large_batch_are_independent():
+    """A sub-batch run with loss_B = size of the full batch reproduces the full batch's activations and
+    activation gradients for those rows (pins the sampled-image parity tests used at full sizes)."""
+    full = si.Workload("full", small_net(), 8, 8, 3, 6, 1, 2)
+    params = si.make_params(full, bias_std=0.3)
+    x, y = si.make_batch(full)
+    mf = so.from_workload(full, real="double"); mf.load_params(params)
+    mf.forward([x], [y]); mf.backward()
+    pick = [1, 4]
+    sub = si.Workload("sub", small_net(), 8, 8, 3, len(pick), 1, 2)
+    ms = so.from_workload(sub, real="double", loss_B=full.B); ms.load_params(params)
+    ms.forward([x[pick]], [y[pick]]); ms.backward()
+    assert np.array_equal(ms.logits, mf.logits[pick])
+    np.testing.assert_allclose(ms.row_loss, mf.row_loss[pick], rtol=1e-14)
+    for li in range(5):
+        assert np.array_equal(ms.conv_out[0][li], mf.conv_out[0][li][pick])
+        np.testing.assert_allclose(ms.d_conv[0][li], mf.d_conv[0][li][pick], rtol=1e-13, atol=1e-18)
