@@ -681,6 +681,77 @@ conv_in_fwd_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* 
     store8(y + (size_t)pix * Cout + kg, acc);
 }
 
+// Forward, 4 pixels per thread (W a multiple of 4): a thread owns 4 horizontally adjacent pixels and 8 output
+// channels.  The 3 x 6 x CIN input window of the 4 pixels sits in registers, so each pair of 16-byte weight
+// reads from shared memory feeds 32 FMAs (the 1-pixel kernel above is bound by those reads).
+template <typename T, int CIN, bool TAB>
+__global__ void __launch_bounds__(256)
+conv_in_fwd4_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ wt, const float* __restrict__ bias,
+                    T* __restrict__ y, long nquads, int H, int W, int Cout, int relu)
+{
+    extern __shared__ float s_wf[];            // [9*CIN][Cout] then bias [Cout]
+    float* s_b = s_wf + 9 * CIN * Cout;
+    for (int e = threadIdx.x; e < 9 * CIN * Cout; e += 256) {
+        int k = e % Cout, j = e / Cout;
+        s_wf[e] = ldf(wt + (size_t)k * 9 * CIN + j);
+    }
+    for (int e = threadIdx.x; e < Cout; e += 256) s_b[e] = bias[e];
+    __syncthreads();
+    const int groups = Cout / 8;
+    const long t = blockIdx.x * 256L + threadIdx.x;
+    const long quad = t / groups;
+    const int kg = (int)(t % groups) * 8;
+    if (quad >= nquads) return;
+    const int wq = W / 4;
+    const int w0 = (int)(quad % wq) * 4;
+    const long q2 = quad / wq;
+    const int h = (int)(q2 % H);
+    const long n = q2 / H;
+    const T* img = TAB ? (const T*)tab.p[n / b_per_rep] + (size_t)(n % b_per_rep) * H * W * CIN : x + (size_t)n * H * W * CIN;
+    float win[3][6 * CIN];                     // rows h-1..h+1, columns w0-1..w0+4
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int hh = h + r - 1;
+#pragma unroll
+        for (int c6 = 0; c6 < 6; ++c6) {
+            const int ww = w0 + c6 - 1;
+            const bool in = hh >= 0 && hh < H && ww >= 0 && ww < W;
+#pragma unroll
+            for (int c = 0; c < CIN; ++c) win[r][c6 * CIN + c] = in ? ldf(img + ((size_t)hh * W + ww) * CIN + c) : 0.f;
+        }
+    }
+    float acc[4][8];
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[p][i] = s_b[kg + i];
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int sc = 0; sc < 3 * CIN; ++sc) {          // sc = s*CIN + c
+            const int j = r * 3 * CIN + sc;
+            const float4 w0v = *(const float4*)(s_wf + j * Cout + kg), w1v = *(const float4*)(s_wf + j * Cout + kg + 4);
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const float xv = win[r][p * CIN + sc];
+                acc[p][0] = fmaf(xv, w0v.x, acc[p][0]); acc[p][1] = fmaf(xv, w0v.y, acc[p][1]);
+                acc[p][2] = fmaf(xv, w0v.z, acc[p][2]); acc[p][3] = fmaf(xv, w0v.w, acc[p][3]);
+                acc[p][4] = fmaf(xv, w1v.x, acc[p][4]); acc[p][5] = fmaf(xv, w1v.y, acc[p][5]);
+                acc[p][6] = fmaf(xv, w1v.z, acc[p][6]); acc[p][7] = fmaf(xv, w1v.w, acc[p][7]);
+            }
+        }
+    const size_t pix0 = ((size_t)n * H + h) * W + w0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        if (relu) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (!(acc[p][i] > 0.f)) acc[p][i] = 0.f;
+        }
+        store8(y + (pix0 + p) * Cout + kg, acc[p]);
+    }
+}
+
 // Weight + bias gradient: block = 64 output channels x 4 pixel lanes; per 64-pixel chunk the block stages
 // the patches in shared memory, then thread (k, q) accumulates dy[pix,k] * patch[pix,:] over its pixels.
 // part[block][k][9*CIN] and part_b[block][k] are reduced afterwards in block order.
@@ -700,27 +771,57 @@ conv_in_wgrad_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T
     const long nchunks = (npix + 63) / 64;
     for (long ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
         const long p0 = ch * 64;
-        if (threadIdx.x < 64) {
-            float patch[9 * CIN];
-            const long pix = p0 + threadIdx.x;
-            if (pix < npix) load_patch<T, CIN, TAB>(patch, x, tab, b_per_rep, pix, H, W);
-            else {
+        {
+            // staging: thread (pixel pp, filter row r) writes the 3 taps x CIN values of that row; lane group 3
+            // clears the padding columns
+            const int pp = threadIdx.x % 64, r = threadIdx.x / 64;
+            const long pix = p0 + pp;
+            if (r < 3) {
+                const int w_ = (int)(pix % W);
+                const long t = pix / W;
+                const int h_ = (int)(t % H);
+                const long n_ = t / H;
+                const int hh = h_ + r - 1;
+                const bool row_in = pix < npix && hh >= 0 && hh < H;
+                const T* img = nullptr;
+                if (row_in)
+                    img = (TAB ? (const T*)tab.p[n_ / b_per_rep] + (size_t)(n_ % b_per_rep) * H * W * CIN : x + (size_t)n_ * H * W * CIN) +
+                          (size_t)hh * W * CIN;
 #pragma unroll
-                for (int j = 0; j < 9 * CIN; ++j) patch[j] = 0.f;
+                for (int sdx = 0; sdx < 3; ++sdx) {
+                    const int ww = w_ + sdx - 1;
+                    const bool in = row_in && ww >= 0 && ww < W;
+#pragma unroll
+                    for (int c = 0; c < CIN; ++c) s_patch[pp][(r * 3 + sdx) * CIN + c] = in ? ldf(img + (size_t)ww * CIN + c) : 0.f;
+                }
+            } else {
+#pragma unroll
+                for (int j = 9 * CIN; j < PJ; ++j) s_patch[pp][j] = 0.f;
             }
-#pragma unroll
-            for (int j = 0; j < 9 * CIN; ++j) s_patch[threadIdx.x][j] = patch[j];
         }
         __syncthreads();
         if (k0 + k < Cout) {
-#pragma unroll 4
-            for (int pp = q; pp < 64; pp += 4) {
-                const long pix = p0 + pp;
-                if (pix >= npix) break;
-                const float d = ldf(dy + (size_t)pix * Cout + k0 + k);
-                accb += d;
+            // this thread's 16 pixels of the chunk, 4 at a time so that 4 dy loads are in flight together
+            for (int pg = 0; pg < 4; ++pg) {
+                float d[4];
 #pragma unroll
-                for (int j = 0; j < 9 * CIN; ++j) acc[j] = fmaf(d, s_patch[pp][j], acc[j]);
+                for (int u = 0; u < 4; ++u) {
+                    const long pix = p0 + q + 4 * (pg * 4 + u);
+                    d[u] = pix < npix ? ldf(dy + (size_t)pix * Cout + k0 + k) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int pp = q + 4 * (pg * 4 + u);
+                    accb += d[u];
+                    float pv[PJ];
+#pragma unroll
+                    for (int j4 = 0; j4 < PJ / 4; ++j4) {
+                        const float4 v = *(const float4*)&s_patch[pp][j4 * 4];
+                        pv[j4 * 4] = v.x; pv[j4 * 4 + 1] = v.y; pv[j4 * 4 + 2] = v.z; pv[j4 * 4 + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 9 * CIN; ++j) acc[j] = fmaf(d[u], pv[j], acc[j]);
+                }
             }
         }
         __syncthreads();
@@ -749,6 +850,13 @@ static cudaError_t launch_conv_in_fwd_t(const ConvSimtArgs& a, cudaStream_t st)
     const size_t smem = (size_t)(9 * CIN * a.Cout + a.Cout) * 4;
     PtrTab tab{};
     if (a.tab) tab = *a.tab;
+    if (a.W % 4 == 0) {
+        const long nquads = npix / 4;
+        const int qblocks = (int)((nquads * (a.Cout / 8) + 255) / 256);
+        if (a.tab) conv_in_fwd4_kernel<T, CIN, true><<<qblocks, 256, smem, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
+        else conv_in_fwd4_kernel<T, CIN, false><<<qblocks, 256, smem, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
+        return cudaGetLastError();
+    }
     if (a.tab) conv_in_fwd_kernel<T, CIN, true><<<blocks, 256, smem, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
     else conv_in_fwd_kernel<T, CIN, false><<<blocks, 256, smem, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
     return cudaGetLastError();
@@ -763,7 +871,7 @@ cudaError_t launch_conv_in_fwd(const ConvSimtArgs& a, bool bf16, cudaStream_t st
 int conv_in_wgrad_blocks(int B, int H, int W)
 {
     long chunks = ((long)B * H * W + 63) / 64;
-    return (int)(chunks < 148 * 2 ? chunks : 148 * 2);
+    return (int)(chunks < 148 * 4 ? chunks : 148 * 4);
 }
 template <typename T, int CIN>
 static cudaError_t launch_conv_in_wgrad_t(const WgradSimtArgs& a, cudaStream_t st)
@@ -793,70 +901,122 @@ cudaError_t launch_conv_in_wgrad(const WgradSimtArgs& a, bool bf16, cudaStream_t
 // =============================================================================================
 constexpr int NARROW_MAX = 16;
 
-template <typename T, bool TAB>
-__global__ void __launch_bounds__(256)
+// Forward: one warp per batch row, 8 rows per block; a lane walks the reduction in steps of 8 values
+// (one 16-byte load of X and of each weight row for bf16), then the warp shuffle-reduces its out_f sums.
+template <typename T> struct Vec8;
+template <> struct Vec8<float> { static constexpr int N = 4; typedef float4 V; };
+template <> struct Vec8<__nv_bfloat16> { static constexpr int N = 8; typedef uint4 V; };
+
+// Block = 2 batch rows x 4 reduction quarters (one warp each).  A lane issues all its 16-byte loads of X and
+// of the out_f weight rows for its slice up front (many loads in flight: the kernel is pure latency), the warp
+// shuffle-reduces, and the 4 quarters of a row are added in order through shared memory.
+template <typename T, bool TAB, int KS, bool VEC>
+__global__ void __launch_bounds__(64 * KS)
 fc_narrow_fwd_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ Wt, const float* __restrict__ bias,
-                     T* __restrict__ Y, float* __restrict__ Y32, int in_f, int out_f, int relu)
+                     T* __restrict__ Y, float* __restrict__ Y32, int B, int in_f, int out_f, int relu)
 {
-    __shared__ float s_red[8][NARROW_MAX];
-    const int g = blockIdx.x;
-    const T* xr = TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f;
+    constexpr int VN = Vec8<T>::N;
+    typedef typename Vec8<T>::V V;
+    __shared__ float s_part[2][KS][NARROW_MAX];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int rl = warp / KS, ks = warp % KS;
+    const int g = blockIdx.x * 2 + rl;
+    const int kq = in_f / KS;                 // reduction elements of this warp (multiple of 32*VN or handled by the tail loop)
     float acc[NARROW_MAX];
 #pragma unroll
     for (int j = 0; j < NARROW_MAX; ++j) acc[j] = 0.f;
-    for (int k = threadIdx.x; k < in_f; k += 256) {
-        const float xv = ldf(xr + k);
+    if (g < B) {
+        const T* xr = (TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f) + (size_t)ks * kq;
+        const T* wr = Wt + (size_t)ks * kq;
+        if (VEC) {
+            // 16-byte loads: the host only selects this variant when every row and every slice starts 16-byte aligned
+            for (int k = lane * VN; k + VN <= kq; k += 32 * VN) {
+                const V xv = *(const V*)(xr + k);
+                V wv[NARROW_MAX];
 #pragma unroll
-        for (int j = 0; j < NARROW_MAX; ++j)
-            if (j < out_f) acc[j] = fmaf(xv, ldf(Wt + (size_t)j * in_f + k), acc[j]);
+                for (int j = 0; j < NARROW_MAX; ++j)
+                    if (j < out_f) wv[j] = *(const V*)(wr + (size_t)j * in_f + k);
+#pragma unroll
+                for (int j = 0; j < NARROW_MAX; ++j)
+                    if (j < out_f) {
+#pragma unroll
+                        for (int i = 0; i < VN; ++i) acc[j] = fmaf(ldf((const T*)&xv + i), ldf((const T*)&wv[j] + i), acc[j]);
+                    }
+            }
+        } else {
+            for (int k = lane; k < kq; k += 32) {
+                const float xv = ldf(xr + k);
+#pragma unroll
+                for (int j = 0; j < NARROW_MAX; ++j)
+                    if (j < out_f) acc[j] = fmaf(xv, ldf(wr + (size_t)j * in_f + k), acc[j]);
+            }
+        }
     }
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 #pragma unroll
     for (int j = 0; j < NARROW_MAX; ++j) {
         float v = acc[j];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) s_red[warp][j] = v;
+        if (lane == 0) s_part[rl][ks][j] = v;
     }
     __syncthreads();
-    if (threadIdx.x < out_f) {
-        float v = bias[threadIdx.x];
+    if (threadIdx.x < 2 * NARROW_MAX) {
+        const int r2 = threadIdx.x / NARROW_MAX, j = threadIdx.x % NARROW_MAX;
+        const int g2 = blockIdx.x * 2 + r2;
+        if (g2 < B && j < out_f) {
+            float v = bias[j];
 #pragma unroll
-        for (int w = 0; w < 8; ++w) v += s_red[w][threadIdx.x];
-        if (relu && !(v > 0.f)) v = 0.f;
-        if (Y32) Y32[(size_t)g * out_f + threadIdx.x] = v;
-        if (Y) stf(Y + (size_t)g * out_f + threadIdx.x, v);
+            for (int q = 0; q < KS; ++q) v += s_part[r2][q][j];
+            if (relu && !(v > 0.f)) v = 0.f;
+            if (Y32) Y32[(size_t)g2 * out_f + j] = v;
+            if (Y) stf(Y + (size_t)g2 * out_f + j, v);
+        }
     }
 }
 
+// Weight + bias gradient: block = 32 input columns x 8 row lanes; lane l sums batch rows l, l+8, ... for its
+// column, then the 8 lanes are combined in lane order through shared memory (deterministic).
 template <typename T, bool TAB>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
 fc_narrow_wgrad_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ dY, float* __restrict__ dW,
                        float* __restrict__ db, int B, int in_f, int out_f)
 {
-    extern __shared__ float s_dy[];   // [B][out_f]
-    for (int e = threadIdx.x; e < B * out_f; e += 128) s_dy[e] = ldf(dY + e);
+    extern __shared__ float s_dy[];   // [B][out_f], then the reduction buffer [8][32][NARROW_MAX]
+    float* s_red = s_dy + B * out_f;
+    for (int e = threadIdx.x; e < B * out_f; e += 256) s_dy[e] = ldf(dY + e);
     __syncthreads();
-    const int i = blockIdx.x * 128 + threadIdx.x;
+    const int col = threadIdx.x % 32, lane = threadIdx.x / 32;
+    const int i = blockIdx.x * 32 + col;
     if (blockIdx.x == 0 && threadIdx.x < out_f) {
         float t = 0.f;
         for (int g = 0; g < B; ++g) t += s_dy[g * out_f + threadIdx.x];
         db[threadIdx.x] = t;
     }
-    if (i >= in_f) return;
     float acc[NARROW_MAX];
 #pragma unroll
     for (int j = 0; j < NARROW_MAX; ++j) acc[j] = 0.f;
-    for (int g = 0; g < B; ++g) {
-        const T* xr = TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f;
-        const float xv = ldf(xr + i);
+    if (i < in_f) {
+        for (int g = lane; g < B; g += 8) {
+            const T* xr = TAB ? (const T*)tab.p[g / tab_b] + (size_t)(g % tab_b) * in_f : X + (size_t)g * in_f;
+            const float xv = ldf(xr + i);
 #pragma unroll
-        for (int j = 0; j < NARROW_MAX; ++j)
-            if (j < out_f) acc[j] = fmaf(s_dy[g * out_f + j], xv, acc[j]);
+            for (int j = 0; j < NARROW_MAX; ++j)
+                if (j < out_f) acc[j] = fmaf(s_dy[g * out_f + j], xv, acc[j]);
+        }
     }
 #pragma unroll
-    for (int j = 0; j < NARROW_MAX; ++j)
-        if (j < out_f) dW[(size_t)j * in_f + i] = acc[j];
+    for (int j = 0; j < NARROW_MAX; ++j) s_red[(lane * 32 + col) * NARROW_MAX + j] = acc[j];
+    __syncthreads();
+    if (lane == 0 && i < in_f) {
+#pragma unroll
+        for (int j = 0; j < NARROW_MAX; ++j)
+            if (j < out_f) {
+                float t = 0.f;
+#pragma unroll
+                for (int l = 0; l < 8; ++l) t += s_red[(l * 32 + col) * NARROW_MAX + j];
+                dW[(size_t)j * in_f + i] = t;
+            }
+    }
 }
 
 template <typename T>
@@ -878,7 +1038,7 @@ fc_narrow_dgrad_kernel(const T* __restrict__ dY, const T* __restrict__ Wt, const
     stf(dX + (size_t)g * in_f + i, acc);
 }
 
-bool fc_narrow_supported(int out_f, int B) { return out_f <= NARROW_MAX && (size_t)B * out_f * 4 <= 40 * 1024; }
+bool fc_narrow_supported(int out_f, int B) { return out_f <= NARROW_MAX && (size_t)B * out_f * 4 <= 24 * 1024; }
 
 template <typename T>
 static cudaError_t launch_fc_narrow_t(const FcNarrowArgs& a, cudaStream_t st)
@@ -887,13 +1047,23 @@ static cudaError_t launch_fc_narrow_t(const FcNarrowArgs& a, cudaStream_t st)
     if (a.tab) tab = *a.tab;
     const int tb = a.tab_b > 0 ? a.tab_b : 1;
     if (a.pass == 0) {
-        if (a.tab) fc_narrow_fwd_kernel<T, true><<<a.B, 256, 0, st>>>(nullptr, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.in_f, a.out_f, a.relu);
-        else fc_narrow_fwd_kernel<T, false><<<a.B, 256, 0, st>>>((const T*)a.X, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.in_f, a.out_f, a.relu);
+        const int blocks = (a.B + 1) / 2;
+        // 16-byte loads need every row (and every quarter of a row) to start on a 16-byte boundary
+        const bool aligned_ptrs = (((uintptr_t)a.W | (uintptr_t)a.X) & 15) == 0 && !a.tab;
+        const bool vec = aligned_ptrs && a.in_f % Vec8<T>::N == 0;
+        const bool quarters = vec && a.in_f % (4 * Vec8<T>::N) == 0;
+#define SB_NF(TABF, KS, VECF) fc_narrow_fwd_kernel<T, TABF, KS, VECF><<<blocks, 64 * KS, 0, st>>>( \
+            (const T*)a.X, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.B, a.in_f, a.out_f, a.relu)
+        if (quarters) SB_NF(false, 4, true);
+        else if (vec) SB_NF(false, 1, true);
+        else if (a.tab) SB_NF(true, 1, false);
+        else SB_NF(false, 1, false);
+#undef SB_NF
     } else if (a.pass == 1) {
-        const size_t smem = (size_t)a.B * a.out_f * 4;
-        const int blocks = (a.in_f + 127) / 128;
-        if (a.tab) fc_narrow_wgrad_kernel<T, true><<<blocks, 128, smem, st>>>(nullptr, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
-        else fc_narrow_wgrad_kernel<T, false><<<blocks, 128, smem, st>>>((const T*)a.X, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+        const size_t smem = (size_t)a.B * a.out_f * 4 + 8 * 32 * NARROW_MAX * 4;
+        const int blocks = (a.in_f + 31) / 32;
+        if (a.tab) fc_narrow_wgrad_kernel<T, true><<<blocks, 256, smem, st>>>(nullptr, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+        else fc_narrow_wgrad_kernel<T, false><<<blocks, 256, smem, st>>>((const T*)a.X, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
     } else {
         dim3 grid((a.in_f + 255) / 256, a.B);
         fc_narrow_dgrad_kernel<T><<<grid, 256, 0, st>>>((const T*)a.dY, (const T*)a.W, (const T*)a.ref, (T*)a.dX, a.in_f, a.out_f);
