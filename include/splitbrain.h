@@ -154,6 +154,17 @@ sb_status sb_backward(sb_model* m, void* stream);
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream);
 
 /*
+ * One whole iteration (sb_forward + sb_backward + sb_sgd_step on device-resident inputs) replayed as a CUDA
+ * graph: the first call runs the three passes directly, the second captures them on `stream` (thread-local
+ * capture mode) and every later call with the same input pointers, lr and momentum is one graph launch, which
+ * removes the per-kernel launch cost that dominates at small batch sizes.  Different pointers or
+ * hyper-parameters re-capture.  `stream` must not be the legacy default stream (NULL runs the passes directly).
+ * Arguments as for sb_forward / sb_sgd_step.  Results are identical to the three separate calls.
+ */
+sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum,
+                        void* stream);
+
+/*
  * Mean loss of the last sb_forward.  Synchronises `stream`, copies 4 bytes to host_loss (HOST),
  * and checks the device status word: returns SB_ERR_TIMEOUT if any kernel gave up on a bounded
  * wait since the last call.
@@ -164,7 +175,9 @@ sb_status sb_loss(sb_model* m, void* stream, float* host_loss);
  * One whole iteration from HOST buffers (forward, backward, SGD step, loss read-back): the
  * end-to-end call.  host_x: [B,H,W,C] in the activation dtype, rows r*b..(r+1)*b-1 = replica r;
  * host_labels: int32 [B].  Both are copied host->device on `stream` into staging space inside
- * the arena (pinned host memory makes the copies asynchronous).  Synchronises `stream`.
+ * the arena (pinned host memory makes the copies asynchronous).  Synchronises `stream`.  From the second call on,
+ * the copies, the iteration and the read-back of the loss are replayed as one CUDA graph keyed by the two host
+ * pointers, lr and momentum (the host buffers must then stay at the same addresses; new addresses re-capture).
  */
 sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels,
                              float lr, float momentum, void* stream, float* host_loss);
@@ -221,6 +234,13 @@ typedef struct {
 } sb_profile_entry;
 sb_status sb_profile_begin(sb_model* m, void* stream);
 sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32_t max_entries, int32_t* n);
+
+/*
+ * Debug aid for kernel tuning: dev_buffer = DEVICE buffer of 1024*8 uint64 (or NULL to switch off).  While set,
+ * the first 1024 CTAs of every tensor-core launch record the global nanosecond timer at their phase boundaries
+ * (start, set-up done, first operands landed, last operands landed, accumulator complete, epilogue done).
+ */
+sb_status sb_debug_cta_timing(void* dev_buffer);
 
 /* Number of kernels the last sb_forward + sb_backward + sb_sgd_step enqueued (host counter). */
 sb_status sb_launch_count(const sb_model* m, int64_t* launches);

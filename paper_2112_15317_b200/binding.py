@@ -61,6 +61,7 @@ def _load():
         "sb_model_destroy": [c_void_p],
         "sb_forward": [c_void_p, P(c_void_p), P(c_void_p), c_void_p],
         "sb_backward": [c_void_p, c_void_p],
+        "sb_graph_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
         "sb_sgd_step": [c_void_p, c_float, c_float, c_void_p],
         "sb_loss": [c_void_p, c_void_p, P(c_float)],
         "sb_train_step_host": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p, P(c_float)],
@@ -73,6 +74,7 @@ def _load():
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
         "sb_launch_count": [c_void_p, P(c_int64)],
         "sb_conv_in_wgrad_static": [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p],
+        "sb_debug_cta_timing": [c_void_p],
         "sb_profile_begin": [c_void_p, c_void_p],
         "sb_profile_end": [c_void_p, c_void_p, P(sb_profile_entry), c_int32, P(c_int32)],
     }
@@ -96,6 +98,7 @@ sb_model_create = _lib.sb_model_create
 sb_model_destroy = _lib.sb_model_destroy
 sb_forward = _lib.sb_forward
 sb_backward = _lib.sb_backward
+sb_graph_step = _lib.sb_graph_step
 sb_sgd_step = _lib.sb_sgd_step
 sb_loss = _lib.sb_loss
 sb_train_step_host = _lib.sb_train_step_host
@@ -108,6 +111,7 @@ sb_backward_layers = _lib.sb_backward_layers
 sb_param_bytes = _lib.sb_param_bytes
 sb_launch_count = _lib.sb_launch_count
 sb_conv_in_wgrad_static = _lib.sb_conv_in_wgrad_static
+sb_debug_cta_timing = _lib.sb_debug_cta_timing
 sb_profile_begin = _lib.sb_profile_begin
 sb_profile_end = _lib.sb_profile_end
 
@@ -220,6 +224,11 @@ class Model:
 
     def backward(self):
         _check(sb_backward(self.h, self._stream()))
+
+    def graph_step(self, xs, labels, lr, momentum):
+        """forward + backward + sgd_step as one CUDA-graph launch (captured by the library on the second call)."""
+        xp, lp = self._ptr_arrays(xs, labels)
+        _check(sb_graph_step(self.h, xp, lp, c_float(lr), c_float(momentum), self._stream()))
 
     def sgd_step(self, lr, momentum):
         _check(sb_sgd_step(self.h, c_float(lr), c_float(momentum), self._stream()))

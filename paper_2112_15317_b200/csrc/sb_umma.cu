@@ -58,6 +58,7 @@ struct UmmaParams {
     int bias_fused;       // WGRAD: the centre-tap CTAs of the first N tile also sum dy over the pixels (the bias gradient)
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
+    unsigned long long* timing;   // optional (SB_UMMA_TIMING=1): per-CTA phase timestamps, 8 per CTA, first 1024 CTAs
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -201,6 +202,9 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     float* s_bias = (float*)(ctrl + 512);             // [BN]
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+    unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 8ull * cta_lin : nullptr;
+    if (tlog && threadIdx.x == 0) tlog[0] = globaltimer_ns();
 
     // ---- tile coordinates ---------------------------------------------------------------------
     int tap_fixed = 0, split = 0;
@@ -259,6 +263,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (tlog && threadIdx.x == 0) tlog[1] = globaltimer_ns();   // set-up done
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
@@ -305,6 +310,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
+                if (tlog && it == 0) tlog[2] = globaltimer_ns();            // first operands landed
+                if (tlog && it == n_iters - 1) tlog[3] = globaltimer_ns();  // last operands landed
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
 #pragma unroll
@@ -353,6 +360,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
+            if (tlog && threadIdx.x == 64) tlog[4] = globaltimer_ns();      // accumulator complete
             tc_fence_after();
             bool row_ok;
             size_t row_off;
@@ -447,6 +455,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
     tc_fence_before();
     __syncthreads();
+    if (tlog && threadIdx.x == 0) tlog[5] = globaltimer_ns();               // epilogue done
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
@@ -572,13 +581,18 @@ static_assert(sizeof(OpBlock) <= sizeof(((UmmaOp*)nullptr)->blob), "UmmaOp::blob
 static OpBlock* blk(UmmaOp& op) { return (OpBlock*)op.blob; }
 static const OpBlock* blk(const UmmaOp& op) { return (const OpBlock*)op.blob; }
 
+static unsigned long long* g_timing = nullptr;   // debug only: set through umma_set_timing_buffer
+void umma_set_timing_buffer(void* dev_ptr) { g_timing = (unsigned long long*)dev_ptr; }
+
 static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr)
 {
     const OpBlock* b = blk(op);
     cudaError_t e;
-    if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, b->p, b->grid, st);
-    else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, b->p, b->grid, st);
-    else e = launch_mode<MODE_WGRAD>(b->bn, op, b->p, b->grid, st);
+    UmmaParams pp = b->p;
+    pp.timing = g_timing;
+    if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
+    else e = launch_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
     if (e == cudaSuccess && b->p.mode != MODE_WGRAD && b->p.splits > 1) {
         // ordered sum of the split partial sums + the epilogue the tensor-core kernel skipped
         SplitKEpiArgs a{};

@@ -274,6 +274,37 @@ def test_train_step_host_matches_device_path():
     g1.close(); g2.close()
 
 
+def test_graph_step_and_graph_host_step_match_separate_calls():
+    """On a side stream the library replays the iteration as a CUDA graph (captured on the second call): weights
+    and losses must be bit-identical to the three separate calls, also after the inputs move (re-capture)."""
+    import torch
+    b = sb()
+    wl = WORKLOADS["tensor_core"]()
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    g1 = gpu_model(wl, params, b.SB_BF16)
+    g2 = gpu_model(wl, params, b.SB_BF16)
+    g3 = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    xs2 = [t.clone() for t in xs]                      # same values at other addresses
+    hx = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    hy = torch.from_numpy(y).pin_memory()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for it in range(5):
+            g1.forward(xs, ys); g1.backward(); g1.sgd_step(0.02, 0.9); l1 = g1.loss()
+            g2.graph_step(xs if it < 3 else xs2, ys, 0.02, 0.9); l2 = g2.loss()
+            l3 = g3.train_step_host(hx, hy, 0.02, 0.9)
+            assert l1 == l2 == l3, (it, l1, l2, l3)
+        side.synchronize()
+    w1 = g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)
+    for other in (g2, g3):
+        for a, c in zip(w1, other.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+            if a is not None:
+                assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    g1.close(); g2.close(); g3.close()
+
+
 def test_state_and_argument_errors():
     b = sb()
     wl = si.config(0)
