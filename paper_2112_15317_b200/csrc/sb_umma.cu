@@ -204,7 +204,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
     unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 8ull * cta_lin : nullptr;
-    if (tlog && threadIdx.x == 0) tlog[0] = globaltimer_ns();
+    if (tlog && threadIdx.x == 0) { tlog[0] = globaltimer_ns(); tlog[6] = (unsigned long long)clock64(); }
 
     // ---- tile coordinates ---------------------------------------------------------------------
     int tap_fixed = 0, split = 0;
@@ -242,6 +242,38 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int n_iters = k_end - k_begin;
     const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? 4 : 0);
 
+    // Operand loads of k-iteration `it` of this CTA into ring slot it % STAGES (executed by the producer thread).
+    auto issue_loads = [&](int it) {
+        const int s = it % STAGES;
+        uint8_t* sa = smem + s * C::STAGE_BYTES;
+        uint8_t* sb = sa + A_STAGE_BYTES;
+        mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES);
+        const int kit = k_begin + it;
+        if (MODE == MODE_WGRAD) {
+            // pixel chunk kit -> box origin; A = dy (two 64-channel boxes), B = shifted activations
+            const int cw = (kit % p.tiles_w) * p.bw, ch = ((kit / p.tiles_w) % p.tiles_h) * p.bh;
+            const int cn = (kit / (p.tiles_w * p.tiles_h)) * p.bn;
+            const int dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
+            tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
+            tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + ds, ch + dr, cn);
+        } else {
+            const int tap = kit / p.kchunks, kc = kit % p.kchunks;
+            int dr = 0, ds = 0;
+            if (p.ntaps == 9) { dr = tap / 3 - 1; ds = tap % 3 - 1; }
+            if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
+            tma_load_4d(&mapA, sa, &full[s], kc * 64, pw0 + ds, ph0 + dr, pn0);
+            if (MODE == MODE_FWD) {
+                tma_load_4d(&mapB, sb, &full[s], tap * p.w_cols + kc * 64, n0, 0, 0);
+            } else {
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0);
+            }
+        }
+    };
+    const int preloaded = n_iters < STAGES ? n_iters : STAGES;
+
     // ---- one-time setup -----------------------------------------------------------------------
     if (threadIdx.x == 0) {
         // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
@@ -249,8 +281,9 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapA) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapB) : "memory");
+        // The first ring-full of loads needs nothing but the barriers this thread has just initialised: start
+        // them now, so that their latency overlaps the TMEM allocation and the rest of the set-up.
+        for (int it = 0; it < preloaded; ++it) issue_loads(it);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -263,42 +296,17 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    if (tlog && threadIdx.x == 0) tlog[1] = globaltimer_ns();   // set-up done
+    if (tlog && threadIdx.x == 0) tlog[1] = (unsigned long long)clock64();   // set-up done
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
         if (lane == 0) {
-            for (int it = 0; it < n_iters; ++it) {
+            for (int it = preloaded; it < n_iters; ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
                 if (*abort_flag) break;
-                uint8_t* sa = smem + s * C::STAGE_BYTES;
-                uint8_t* sb = sa + A_STAGE_BYTES;
-                mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES);
-                const int kit = k_begin + it;
-                if (MODE == MODE_WGRAD) {
-                    // pixel chunk kit -> box origin; A = dy (two 64-channel boxes), B = shifted activations
-                    const int cw = (kit % p.tiles_w) * p.bw, ch = ((kit / p.tiles_w) % p.tiles_h) * p.bh;
-                    const int cn = (kit / (p.tiles_w * p.tiles_h)) * p.bn;
-                    const int dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
-                    tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
-                    tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
-#pragma unroll
-                    for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + ds, ch + dr, cn);
-                } else {
-                    const int tap = kit / p.kchunks, kc = kit % p.kchunks;
-                    int dr = 0, ds = 0;
-                    if (p.ntaps == 9) { dr = tap / 3 - 1; ds = tap % 3 - 1; }
-                    if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
-                    tma_load_4d(&mapA, sa, &full[s], kc * 64, pw0 + ds, ph0 + dr, pn0);
-                    if (MODE == MODE_FWD) {
-                        tma_load_4d(&mapB, sb, &full[s], tap * p.w_cols + kc * 64, n0, 0, 0);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0);
-                    }
-                }
+                issue_loads(it);
             }
         }
     } else if (warp == 1) {
@@ -310,8 +318,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
-                if (tlog && it == 0) tlog[2] = globaltimer_ns();            // first operands landed
-                if (tlog && it == n_iters - 1) tlog[3] = globaltimer_ns();  // last operands landed
+                if (tlog && it == 0) tlog[2] = (unsigned long long)clock64();            // first operands landed
+                if (tlog && it == n_iters - 1) tlog[3] = (unsigned long long)clock64();  // last operands landed
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
 #pragma unroll
@@ -360,7 +368,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
-            if (tlog && threadIdx.x == 64) tlog[4] = globaltimer_ns();      // accumulator complete
+            if (tlog && threadIdx.x == 64) tlog[4] = (unsigned long long)clock64();      // accumulator complete
             tc_fence_after();
             bool row_ok;
             size_t row_off;
@@ -455,7 +463,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
     tc_fence_before();
     __syncthreads();
-    if (tlog && threadIdx.x == 0) tlog[5] = globaltimer_ns();               // epilogue done
+    if (tlog && threadIdx.x == 0) { tlog[5] = (unsigned long long)clock64(); tlog[7] = globaltimer_ns(); }   // epilogue done
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
