@@ -7,9 +7,47 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <cstdlib>
+#include <utility>
+
 namespace sb {
 
 constexpr int MAX_PARTS = 64;  // upper bound on R and K
+
+// ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_prologue(): it waits until the
+// kernels it depends on have completed (griddepcontrol.wait, a no-op for a normally launched kernel) and
+// then lets the next kernel in the stream start launching (griddepcontrol.launch_dependents), so that the
+// next kernel's launch latency and set-up overlap this kernel's execution.  Nothing is read from or written
+// to global memory before the wait.  SB_PDL=0 in the environment launches everything the classic way.
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_prologue() { pdl_wait(); pdl_trigger(); }
+#endif
+inline bool pdl_enabled()
+{
+    static const bool on = [] { const char* e = getenv("SB_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t pdl_launch(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
+}
+#define SB_LAUNCH(kern, grid, block, smem, st, ...) (void)::sb::pdl_launch((kern), dim3(grid), dim3(block), (size_t)(smem), (st), __VA_ARGS__)
+
 
 // Pointer table for per-replica caller buffers (inputs, labels): passed by value to kernels.
 struct PtrTab {

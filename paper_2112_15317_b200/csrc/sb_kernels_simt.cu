@@ -52,6 +52,7 @@ conv3x3_simt_kernel(const T* __restrict__ in, PtrTab tab, int b_per_rep, const T
                     const float* __restrict__ bias, T* __restrict__ out, const T* __restrict__ mask_ref,
                     int H, int W, int Cred, int Cres, int Cin, int relu)
 {
+    pdl_prologue();
     __shared__ float s_in[CV_TP + 2][CV_TP + 2][CV_CK + 1];
     __shared__ float s_w[9][CV_CK][CV_TC];
     const int tiles_w = (W + CV_TP - 1) / CV_TP;
@@ -141,13 +142,13 @@ static cudaError_t launch_conv_simt_t(const ConvSimtArgs& a, cudaStream_t st)
     PtrTab tab{};
     if (a.tab) tab = *a.tab;
     if (a.dgrad)
-        conv3x3_simt_kernel<T, true, false><<<grid, 128, 0, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
+        SB_LAUNCH((conv3x3_simt_kernel<T, true, false>), grid, 128, 0, st, (const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
                                                                   (T*)a.out, (const T*)a.mask_ref, a.H, a.W, Cred, Cres, a.Cin, 0);
     else if (a.tab)
-        conv3x3_simt_kernel<T, false, true><<<grid, 128, 0, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias,
+        SB_LAUNCH((conv3x3_simt_kernel<T, false, true>), grid, 128, 0, st, nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias,
                                                                   (T*)a.out, nullptr, a.H, a.W, Cred, Cres, a.Cin, a.relu);
     else
-        conv3x3_simt_kernel<T, false, false><<<grid, 128, 0, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
+        SB_LAUNCH((conv3x3_simt_kernel<T, false, false>), grid, 128, 0, st, (const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias,
                                                                    (T*)a.out, nullptr, a.H, a.W, Cred, Cres, a.Cin, a.relu);
     return cudaGetLastError();
 }
@@ -165,6 +166,7 @@ __global__ void __launch_bounds__(256)
 conv3x3_wgrad_simt_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ dy,
                           float* __restrict__ part, int B, int H, int W, int Cin, int Cout, int splits)
 {
+    pdl_prologue();
     __shared__ float s_dy[32][33];
     __shared__ float s_x[32][33];
     const int k0 = blockIdx.x * 32;
@@ -224,7 +226,7 @@ cudaError_t launch_wgrad_simt(const WgradSimtArgs& a, bool bf16, cudaStream_t st
     PtrTab tab{};
     if (a.tab) tab = *a.tab;
 #define SB_WG(T, TABF)                                                                                         \
-    conv3x3_wgrad_simt_kernel<T, TABF><<<grid, 256, 0, st>>>((const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, \
+    SB_LAUNCH((conv3x3_wgrad_simt_kernel<T, TABF>), grid, 256, 0, st, (const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, \
                                                             a.part, a.B, a.H, a.W, a.Cin, a.Cout, a.splits)
     if (bf16) { if (a.tab) SB_WG(__nv_bfloat16, true); else SB_WG(__nv_bfloat16, false); }
     else      { if (a.tab) SB_WG(float, true); else SB_WG(float, false); }
@@ -239,6 +241,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 colsum_kernel(const T* __restrict__ in, float* __restrict__ part, int M, int N, int splits)
 {
+    pdl_prologue();
     __shared__ float s[8][33];
     const int col = blockIdx.x * 32 + threadIdx.x % 32;
     const int lane_row = threadIdx.x / 32;
@@ -259,14 +262,15 @@ colsum_kernel(const T* __restrict__ in, float* __restrict__ part, int M, int N, 
 cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st)
 {
     dim3 grid(cdiv(N, 32), splits);
-    if (bf16) colsum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)in, part, M, N, splits);
-    else colsum_kernel<float><<<grid, 256, 0, st>>>((const float*)in, part, M, N, splits);
+    if (bf16) SB_LAUNCH((colsum_kernel<__nv_bfloat16>), grid, 256, 0, st, (const __nv_bfloat16*)in, part, M, N, splits);
+    else SB_LAUNCH((colsum_kernel<float>), grid, 256, 0, st, (const float*)in, part, M, N, splits);
     return cudaGetLastError();
 }
 
 __global__ void __launch_bounds__(256)
 reduce_partials_kernel(const float* __restrict__ part, size_t stride, float* __restrict__ out, size_t n, int splits)
 {
+    pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         float t = 0.f;
         for (int s = 0; s < splits; ++s) t += part[(size_t)s * stride + i];
@@ -276,6 +280,7 @@ reduce_partials_kernel(const float* __restrict__ part, size_t stride, float* __r
 __global__ void __launch_bounds__(256)
 reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4* __restrict__ out, size_t n4, int splits)
 {
+    pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
         float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s = 0; s < splits; ++s) {
@@ -290,6 +295,7 @@ reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4*
 __global__ void __launch_bounds__(256)
 reduce_partials_many_kernel(const float* __restrict__ part, size_t stride, float* __restrict__ out, size_t n, int splits)
 {
+    pdl_prologue();
     __shared__ float s[8][33];
     const int e = threadIdx.x % 32, lane = threadIdx.x / 32;
     const size_t i = blockIdx.x * 32ull + e;
@@ -308,15 +314,15 @@ reduce_partials_many_kernel(const float* __restrict__ part, size_t stride, float
 cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st)
 {
     if (splits >= 32 && n <= (1u << 20)) {
-        reduce_partials_many_kernel<<<cdiv((long)n, 32), 256, 0, st>>>(part, stride, out, n, splits);
+        SB_LAUNCH((reduce_partials_many_kernel), cdiv((long)n, 32), 256, 0, st, part, stride, out, n, splits);
     } else if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0) {
         int blocks = cdiv((long)(n / 4), 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
-        reduce_partials4_kernel<<<blocks, 256, 0, st>>>((const float4*)part, stride / 4, (float4*)out, n / 4, splits);
+        SB_LAUNCH((reduce_partials4_kernel), blocks, 256, 0, st, (const float4*)part, stride / 4, (float4*)out, n / 4, splits);
     } else {
         int blocks = cdiv((long)n, 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
-        reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, stride, out, n, splits);
+        SB_LAUNCH((reduce_partials_kernel), blocks, 256, 0, st, part, stride, out, n, splits);
     }
     return cudaGetLastError();
 }
@@ -331,6 +337,7 @@ splitk_epilogue_kernel(const float* __restrict__ part, size_t split_stride, int 
                        const float* __restrict__ bias, int relu, const __nv_bfloat16* __restrict__ ref,
                        void* __restrict__ out, int out_f32)
 {
+    pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
         const size_t e = i * 4;
         float4 t = __ldg((const float4*)(part + e));
@@ -373,9 +380,9 @@ cudaError_t launch_splitk_epilogue(const SplitKEpiArgs& a, cudaStream_t st)
     int blocks = cdiv((long)n4, 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
     if (a.epi == EPI_BIAS_ACT)
-        splitk_epilogue_kernel<EPI_BIAS_ACT><<<blocks, 256, 0, st>>>(a.part, a.split_stride, a.splits, n4, a.N, a.bias, a.relu, nullptr, a.out, a.out_f32);
+        SB_LAUNCH((splitk_epilogue_kernel<EPI_BIAS_ACT>), blocks, 256, 0, st, a.part, a.split_stride, a.splits, n4, a.N, a.bias, a.relu, nullptr, a.out, a.out_f32);
     else
-        splitk_epilogue_kernel<EPI_MASK><<<blocks, 256, 0, st>>>(a.part, a.split_stride, a.splits, n4, a.N, nullptr, 0, (const __nv_bfloat16*)a.ref, a.out, 0);
+        SB_LAUNCH((splitk_epilogue_kernel<EPI_MASK>), blocks, 256, 0, st, a.part, a.split_stride, a.splits, n4, a.N, nullptr, 0, (const __nv_bfloat16*)a.ref, a.out, 0);
     return cudaGetLastError();
 }
 
@@ -397,6 +404,7 @@ template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ p, uint8_t* __restrict__ idx, long total, int H, int W, int C)
 {
+    pdl_prologue();
     typedef typename VecT<T, VEC>::type V;
     typedef typename VecU8<VEC>::type VI;
     const int Ho = H / 2, Wo = W / 2, Cv = C / VEC;
@@ -442,6 +450,7 @@ __global__ void __launch_bounds__(256)
 maxpool_bwd_kernel(const T* __restrict__ dp, const uint8_t* __restrict__ idx, const T* __restrict__ p,
                    T* __restrict__ dx, long total, int H, int W, int C)
 {
+    pdl_prologue();
     typedef typename VecT<T, VEC>::type V;
     typedef typename VecU8<VEC>::type VI;
     const int Ho = H / 2, Wo = W / 2, Cv = C / VEC;
@@ -488,11 +497,11 @@ cudaError_t launch_pool_fwd(const PoolArgs& a, bool bf16, cudaStream_t st)
 {
     long pooled = (long)a.B * (a.H / 2) * (a.W / 2) * a.C;
     if (bf16) {
-        if (a.C % 8 == 0) maxpool_fwd_kernel<__nv_bfloat16, 8><<<ew_blocks(pooled / 8), 256, 0, st>>>((const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled / 8, a.H, a.W, a.C);
-        else maxpool_fwd_kernel<__nv_bfloat16, 1><<<ew_blocks(pooled), 256, 0, st>>>((const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled, a.H, a.W, a.C);
+        if (a.C % 8 == 0) SB_LAUNCH((maxpool_fwd_kernel<__nv_bfloat16, 8>), ew_blocks(pooled / 8), 256, 0, st, (const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled / 8, a.H, a.W, a.C);
+        else SB_LAUNCH((maxpool_fwd_kernel<__nv_bfloat16, 1>), ew_blocks(pooled), 256, 0, st, (const __nv_bfloat16*)a.x, (__nv_bfloat16*)a.p, a.idx, pooled, a.H, a.W, a.C);
     } else {
-        if (a.C % 4 == 0) maxpool_fwd_kernel<float, 4><<<ew_blocks(pooled / 4), 256, 0, st>>>((const float*)a.x, (float*)a.p, a.idx, pooled / 4, a.H, a.W, a.C);
-        else maxpool_fwd_kernel<float, 1><<<ew_blocks(pooled), 256, 0, st>>>((const float*)a.x, (float*)a.p, a.idx, pooled, a.H, a.W, a.C);
+        if (a.C % 4 == 0) SB_LAUNCH((maxpool_fwd_kernel<float, 4>), ew_blocks(pooled / 4), 256, 0, st, (const float*)a.x, (float*)a.p, a.idx, pooled / 4, a.H, a.W, a.C);
+        else SB_LAUNCH((maxpool_fwd_kernel<float, 1>), ew_blocks(pooled), 256, 0, st, (const float*)a.x, (float*)a.p, a.idx, pooled, a.H, a.W, a.C);
     }
     return cudaGetLastError();
 }
@@ -500,11 +509,11 @@ cudaError_t launch_pool_bwd(const PoolBwdArgs& a, bool bf16, cudaStream_t st)
 {
     long pooled = (long)a.B * (a.H / 2) * (a.W / 2) * a.C;
     if (bf16) {
-        if (a.C % 8 == 0) maxpool_bwd_kernel<__nv_bfloat16, 8><<<ew_blocks(pooled / 8), 256, 0, st>>>((const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled / 8, a.H, a.W, a.C);
-        else maxpool_bwd_kernel<__nv_bfloat16, 1><<<ew_blocks(pooled), 256, 0, st>>>((const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled, a.H, a.W, a.C);
+        if (a.C % 8 == 0) SB_LAUNCH((maxpool_bwd_kernel<__nv_bfloat16, 8>), ew_blocks(pooled / 8), 256, 0, st, (const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled / 8, a.H, a.W, a.C);
+        else SB_LAUNCH((maxpool_bwd_kernel<__nv_bfloat16, 1>), ew_blocks(pooled), 256, 0, st, (const __nv_bfloat16*)a.dp, a.idx, (const __nv_bfloat16*)a.p, (__nv_bfloat16*)a.dx, pooled, a.H, a.W, a.C);
     } else {
-        if (a.C % 4 == 0) maxpool_bwd_kernel<float, 4><<<ew_blocks(pooled / 4), 256, 0, st>>>((const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled / 4, a.H, a.W, a.C);
-        else maxpool_bwd_kernel<float, 1><<<ew_blocks(pooled), 256, 0, st>>>((const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled, a.H, a.W, a.C);
+        if (a.C % 4 == 0) SB_LAUNCH((maxpool_bwd_kernel<float, 4>), ew_blocks(pooled / 4), 256, 0, st, (const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled / 4, a.H, a.W, a.C);
+        else SB_LAUNCH((maxpool_bwd_kernel<float, 1>), ew_blocks(pooled), 256, 0, st, (const float*)a.dp, a.idx, (const float*)a.p, (float*)a.dx, pooled, a.H, a.W, a.C);
     }
     return cudaGetLastError();
 }
@@ -518,6 +527,7 @@ __global__ void __launch_bounds__(256)
 softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_rep, float* __restrict__ row_loss,
                     float* __restrict__ loss, T* __restrict__ dZ, unsigned int* __restrict__ counter, int B, int C)
 {
+    pdl_prologue();
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int g = blockIdx.x * 8 + warp;
     if (g < B) {
@@ -559,8 +569,8 @@ softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_r
 cudaError_t launch_softmax_xent(const XentArgs& a, bool bf16, cudaStream_t st)
 {
     int blocks = cdiv(a.B, 8);
-    if (bf16) softmax_xent_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (__nv_bfloat16*)a.dZ, a.counter, a.B, a.C);
-    else softmax_xent_kernel<float><<<blocks, 256, 0, st>>>(a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (float*)a.dZ, a.counter, a.B, a.C);
+    if (bf16) SB_LAUNCH((softmax_xent_kernel<__nv_bfloat16>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (__nv_bfloat16*)a.dZ, a.counter, a.B, a.C);
+    else SB_LAUNCH((softmax_xent_kernel<float>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (float*)a.dZ, a.counter, a.B, a.C);
     return cudaGetLastError();
 }
 
@@ -573,6 +583,7 @@ __global__ void __launch_bounds__(256)
 sgd_kernel(float4* __restrict__ w, float4* __restrict__ v, const float4* __restrict__ g,
            uint2* __restrict__ shadow, size_t n4, float lr, float mu)
 {
+    pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
         float4 ww = w[i], vv = v[i], gg = __ldg(g + i);
         vv.x = fmaf(mu, vv.x, gg.x); vv.y = fmaf(mu, vv.y, gg.y); vv.z = fmaf(mu, vv.z, gg.z); vv.w = fmaf(mu, vv.w, gg.w);
@@ -592,14 +603,15 @@ cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow
 {
     size_t n4 = n / 4;
     int blocks = ew_blocks((long)n4);
-    if (shadow) sgd_kernel<true><<<blocks, 256, 0, st>>>((float4*)w, (float4*)v, (const float4*)g, (uint2*)shadow, n4, lr, mu);
-    else sgd_kernel<false><<<blocks, 256, 0, st>>>((float4*)w, (float4*)v, (const float4*)g, nullptr, n4, lr, mu);
+    if (shadow) SB_LAUNCH((sgd_kernel<true>), blocks, 256, 0, st, (float4*)w, (float4*)v, (const float4*)g, (uint2*)shadow, n4, lr, mu);
+    else SB_LAUNCH((sgd_kernel<false>), blocks, 256, 0, st, (float4*)w, (float4*)v, (const float4*)g, nullptr, n4, lr, mu);
     return cudaGetLastError();
 }
 
 __global__ void __launch_bounds__(256)
 to_bf16_kernel(const float4* __restrict__ w, uint2* __restrict__ shadow, size_t n4)
 {
+    pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
         float4 ww = w[i];
         __nv_bfloat162 lo = __floats2bfloat162_rn(ww.x, ww.y), hi = __floats2bfloat162_rn(ww.z, ww.w);
@@ -611,7 +623,7 @@ to_bf16_kernel(const float4* __restrict__ w, uint2* __restrict__ shadow, size_t 
 }
 cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cudaStream_t st)
 {
-    to_bf16_kernel<<<ew_blocks((long)(n / 4)), 256, 0, st>>>((const float4*)w, (uint2*)shadow, n / 4);
+    SB_LAUNCH((to_bf16_kernel), ew_blocks((long)(n / 4)), 256, 0, st, (const float4*)w, (uint2*)shadow, n / 4);
     return cudaGetLastError();
 }
 
@@ -647,6 +659,7 @@ __global__ void __launch_bounds__(256)
 conv_in_fwd_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ wt, const float* __restrict__ bias,
                    T* __restrict__ y, long npix, int H, int W, int Cout, int relu)
 {
+    pdl_prologue();
     extern __shared__ float s_wf[];            // [9*CIN][Cout] then bias [Cout]
     float* s_b = s_wf + 9 * CIN * Cout;
     for (int e = threadIdx.x; e < 9 * CIN * Cout; e += 256) {
@@ -689,6 +702,7 @@ __global__ void __launch_bounds__(256)
 conv_in_fwd4_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ wt, const float* __restrict__ bias,
                     T* __restrict__ y, long nquads, int H, int W, int Cout, int relu)
 {
+    pdl_prologue();
     extern __shared__ float s_wf[];            // [9*CIN][Cout] then bias [Cout]
     float* s_b = s_wf + 9 * CIN * Cout;
     for (int e = threadIdx.x; e < 9 * CIN * Cout; e += 256) {
@@ -760,6 +774,7 @@ __global__ void __launch_bounds__(256)
 conv_in_wgrad_kernel(const T* __restrict__ x, PtrTab tab, int b_per_rep, const T* __restrict__ dy, float* __restrict__ part,
                      long npix, int H, int W, int Cout, long stride_floats)
 {
+    pdl_prologue();
     constexpr int PJ = (9 * CIN + 3) / 4 * 4;   // padded patch length (16-byte rows)
     __shared__ __align__(16) float s_patch[64][PJ];
     __shared__ float s_red[3][64][9 * CIN + 1];
@@ -853,12 +868,12 @@ static cudaError_t launch_conv_in_fwd_t(const ConvSimtArgs& a, cudaStream_t st)
     if (a.W % 4 == 0) {
         const long nquads = npix / 4;
         const int qblocks = (int)((nquads * (a.Cout / 8) + 255) / 256);
-        if (a.tab) conv_in_fwd4_kernel<T, CIN, true><<<qblocks, 256, smem, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
-        else conv_in_fwd4_kernel<T, CIN, false><<<qblocks, 256, smem, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
+        if (a.tab) SB_LAUNCH((conv_in_fwd4_kernel<T, CIN, true>), qblocks, 256, smem, st, nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
+        else SB_LAUNCH((conv_in_fwd4_kernel<T, CIN, false>), qblocks, 256, smem, st, (const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, nquads, a.H, a.W, a.Cout, a.relu);
         return cudaGetLastError();
     }
-    if (a.tab) conv_in_fwd_kernel<T, CIN, true><<<blocks, 256, smem, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
-    else conv_in_fwd_kernel<T, CIN, false><<<blocks, 256, smem, st>>>((const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
+    if (a.tab) SB_LAUNCH((conv_in_fwd_kernel<T, CIN, true>), blocks, 256, smem, st, nullptr, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
+    else SB_LAUNCH((conv_in_fwd_kernel<T, CIN, false>), blocks, 256, smem, st, (const T*)a.in, tab, a.b_per_rep, (const T*)a.w, a.bias, (T*)a.out, npix, a.H, a.W, a.Cout, a.relu);
     return cudaGetLastError();
 }
 bool conv_in_supported(int Cin, int Cout) { return (Cin == 1 || Cin == 3 || Cin == 4) && Cout % 8 == 0 && Cout <= 256; }
@@ -881,8 +896,8 @@ static cudaError_t launch_conv_in_wgrad_t(const WgradSimtArgs& a, cudaStream_t s
     const long stride = (long)a.Cout * 9 * CIN + a.Cout;
     PtrTab tab{};
     if (a.tab) tab = *a.tab;
-    if (a.tab) conv_in_wgrad_kernel<T, CIN, true><<<grid, 256, 0, st>>>(nullptr, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
-    else conv_in_wgrad_kernel<T, CIN, false><<<grid, 256, 0, st>>>((const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
+    if (a.tab) SB_LAUNCH((conv_in_wgrad_kernel<T, CIN, true>), grid, 256, 0, st, nullptr, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
+    else SB_LAUNCH((conv_in_wgrad_kernel<T, CIN, false>), grid, 256, 0, st, (const T*)a.x, tab, a.b_per_rep, (const T*)a.dy, a.part, npix, a.H, a.W, a.Cout, stride);
     return cudaGetLastError();
 }
 // part: [conv_in_wgrad_blocks][Cout*9*Cin + Cout] floats (weights then bias), to be reduced in block order.
@@ -915,6 +930,7 @@ __global__ void __launch_bounds__(64 * KS)
 fc_narrow_fwd_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ Wt, const float* __restrict__ bias,
                      T* __restrict__ Y, float* __restrict__ Y32, int B, int in_f, int out_f, int relu)
 {
+    pdl_prologue();
     constexpr int VN = Vec8<T>::N;
     typedef typename Vec8<T>::V V;
     __shared__ float s_part[2][KS][NARROW_MAX];
@@ -981,6 +997,7 @@ __global__ void __launch_bounds__(256)
 fc_narrow_wgrad_kernel(const T* __restrict__ X, PtrTab tab, int tab_b, const T* __restrict__ dY, float* __restrict__ dW,
                        float* __restrict__ db, int B, int in_f, int out_f)
 {
+    pdl_prologue();
     extern __shared__ float s_dy[];   // [B][out_f], then the reduction buffer [8][32][NARROW_MAX]
     float* s_red = s_dy + B * out_f;
     for (int e = threadIdx.x; e < B * out_f; e += 256) s_dy[e] = ldf(dY + e);
@@ -1024,6 +1041,7 @@ __global__ void __launch_bounds__(256)
 fc_narrow_dgrad_kernel(const T* __restrict__ dY, const T* __restrict__ Wt, const T* __restrict__ ref, T* __restrict__ dX,
                        int in_f, int out_f)
 {
+    pdl_prologue();
     __shared__ float s_d[NARROW_MAX];
     const int g = blockIdx.y;
     if (threadIdx.x < out_f) s_d[threadIdx.x] = ldf(dY + (size_t)g * out_f + threadIdx.x);
@@ -1052,7 +1070,7 @@ static cudaError_t launch_fc_narrow_t(const FcNarrowArgs& a, cudaStream_t st)
         const bool aligned_ptrs = (((uintptr_t)a.W | (uintptr_t)a.X) & 15) == 0 && !a.tab;
         const bool vec = aligned_ptrs && a.in_f % Vec8<T>::N == 0;
         const bool quarters = vec && a.in_f % (4 * Vec8<T>::N) == 0;
-#define SB_NF(TABF, KS, VECF) fc_narrow_fwd_kernel<T, TABF, KS, VECF><<<blocks, 64 * KS, 0, st>>>( \
+#define SB_NF(TABF, KS, VECF) SB_LAUNCH((fc_narrow_fwd_kernel<T, TABF, KS, VECF>), blocks, 64 * KS, 0, st,  \
             (const T*)a.X, tab, tb, (const T*)a.W, a.bias, (T*)a.Y, a.Y32, a.B, a.in_f, a.out_f, a.relu)
         if (quarters) SB_NF(false, 4, true);
         else if (vec) SB_NF(false, 1, true);
@@ -1062,11 +1080,11 @@ static cudaError_t launch_fc_narrow_t(const FcNarrowArgs& a, cudaStream_t st)
     } else if (a.pass == 1) {
         const size_t smem = (size_t)a.B * a.out_f * 4 + 8 * 32 * NARROW_MAX * 4;
         const int blocks = (a.in_f + 31) / 32;
-        if (a.tab) fc_narrow_wgrad_kernel<T, true><<<blocks, 256, smem, st>>>(nullptr, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
-        else fc_narrow_wgrad_kernel<T, false><<<blocks, 256, smem, st>>>((const T*)a.X, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+        if (a.tab) SB_LAUNCH((fc_narrow_wgrad_kernel<T, true>), blocks, 256, smem, st, nullptr, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
+        else SB_LAUNCH((fc_narrow_wgrad_kernel<T, false>), blocks, 256, smem, st, (const T*)a.X, tab, tb, (const T*)a.dY, a.dW, a.db, a.B, a.in_f, a.out_f);
     } else {
         dim3 grid((a.in_f + 255) / 256, a.B);
-        fc_narrow_dgrad_kernel<T><<<grid, 256, 0, st>>>((const T*)a.dY, (const T*)a.W, (const T*)a.ref, (T*)a.dX, a.in_f, a.out_f);
+        SB_LAUNCH((fc_narrow_dgrad_kernel<T>), grid, 256, 0, st, (const T*)a.dY, (const T*)a.W, (const T*)a.ref, (T*)a.dX, a.in_f, a.out_f);
     }
     return cudaGetLastError();
 }
@@ -1089,6 +1107,7 @@ gemm_simt_kernel(const T* __restrict__ A, long sAm, long sAk, const T* __restric
                  const float* __restrict__ bias, int relu, const T* __restrict__ ref, long ldref,
                  int shard_dim, int shards, PtrTab tab, int tab_mode, int tab_b)
 {
+    pdl_prologue();
     __shared__ float As[16][65];
     __shared__ float Bs[16][65];
     int m_lo = 0, m_hi = M, n_lo = 0, n_hi = N;
@@ -1179,7 +1198,7 @@ static cudaError_t launch_gemm_simt_t(const GemmSimtArgs& a, cudaStream_t st)
     if (a.tab) tab = *a.tab;
     const int tab_mode = a.tab ? a.tab_mode : 0;
 #define SB_GM(E)                                                                                                    \
-    gemm_simt_kernel<T, E><<<grid, 256, 0, st>>>((const T*)a.A, a.sAm, a.sAk, (const T*)a.B, a.sBn, a.sBk, a.M, a.N, a.K, \
+    SB_LAUNCH((gemm_simt_kernel<T, E>), grid, 256, 0, st, (const T*)a.A, a.sAm, a.sAk, (const T*)a.B, a.sBn, a.sBk, a.M, a.N, a.K, \
                                                  a.C, a.ldc, a.C32, a.bias, a.relu, (const T*)a.ref, a.ldref, a.shard_dim, shards, \
                                                  tab, tab_mode, a.tab_b > 0 ? a.tab_b : 1)
     if (a.epi == EPI_BIAS_ACT) SB_GM(EPI_BIAS_ACT);

@@ -275,12 +275,16 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int preloaded = n_iters < STAGES ? n_iters : STAGES;
 
     // ---- one-time setup -----------------------------------------------------------------------
+    // (programmatic dependent launch: everything up to pdl_wait() touches only shared memory and TMEM, so it
+    // may run while the kernel this one depends on is still finishing)
     if (threadIdx.x == 0) {
         // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pdl_wait();
+        pdl_trigger();
         // The first ring-full of loads needs nothing but the barriers this thread has just initialised: start
         // them now, so that their latency overlaps the TMEM allocation and the rest of the set-up.
         for (int it = 0; it < preloaded; ++it) issue_loads(it);
@@ -289,6 +293,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         tmem_alloc(tmem_slot, C::TMEM_COLS);
         tmem_relinquish();
     }
+    if (threadIdx.x != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
     if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
         for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
     }
@@ -563,8 +568,7 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
         attr_set = true;
     }
     if (p.stages < 1 || p.stages > Cfg<MODE, BN>::MAX_STAGES_FIT) return cudaErrorInvalidValue;
-    umma_kernel<MODE, BN><<<grid, UMMA_THREADS, Cfg<MODE, BN>::smem_bytes(p.stages), st>>>(op.mapA, op.mapB, p);
-    return cudaGetLastError();
+    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, p);
 }
 
 template <int MODE>
