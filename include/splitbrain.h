@@ -236,7 +236,7 @@ sb_status sb_profile_begin(sb_model* m, void* stream);
 sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32_t max_entries, int32_t* n);
 
 /*
- * Debug aid for kernel tuning: dev_buffer = DEVICE buffer of 1024*8 uint64 (or NULL to switch off).  While set,
+ * Debug aid for kernel tuning: dev_buffer = DEVICE buffer of 1024*16 uint64 (or NULL to switch off).  While set,
  * the first 1024 CTAs of every tensor-core launch record the global nanosecond timer at their phase boundaries
  * (start, set-up done, first operands landed, last operands landed, accumulator complete, epilogue done).
  */

@@ -282,10 +282,15 @@ reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4*
 {
     pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        // loads go out in batches of 8 (independent, all in flight together); the additions keep split order
         float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < splits; ++s) {
-            const float4 v = __ldg(part + (size_t)s * stride4 + i);
-            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        for (int s0 = 0; s0 < splits; s0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[u] = (s0 + u < splits) ? __ldg(part + (size_t)(s0 + u) * stride4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { t.x += v[u].x; t.y += v[u].y; t.z += v[u].z; t.w += v[u].w; }
         }
         out[i] = t;
     }
@@ -340,10 +345,15 @@ splitk_epilogue_kernel(const float* __restrict__ part, size_t split_stride, int 
     pdl_prologue();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
         const size_t e = i * 4;
-        float4 t = __ldg((const float4*)(part + e));
-        for (int s = 1; s < splits; ++s) {
-            const float4 v = __ldg((const float4*)(part + (size_t)s * split_stride + e));
-            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        // loads go out in batches of 8 (independent, all in flight together); the additions keep split order
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = 0; s0 < splits; s0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[u] = (s0 + u < splits) ? __ldg((const float4*)(part + (size_t)(s0 + u) * split_stride + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { t.x += v[u].x; t.y += v[u].y; t.z += v[u].z; t.w += v[u].w; }
         }
         if (EPI == EPI_BIAS_ACT) {
             const float4 b = *(const float4*)(bias + (e % (size_t)N));

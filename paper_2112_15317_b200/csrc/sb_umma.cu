@@ -203,7 +203,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-    unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 8ull * cta_lin : nullptr;
+    unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 16ull * cta_lin : nullptr;
     if (tlog && threadIdx.x == 0) { tlog[0] = globaltimer_ns(); tlog[6] = (unsigned long long)clock64(); }
 
     // ---- tile coordinates ---------------------------------------------------------------------
@@ -242,26 +242,32 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int n_iters = k_end - k_begin;
     const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? 4 : 0);
 
-    // Operand loads of k-iteration `it` of this CTA into ring slot it % STAGES (executed by the producer thread).
+    // Operand loads of the next k-iteration into ring slot `s` (executed by the producer thread, iterations in
+    // order).  The iteration's coordinates are carried in counters, so the issue path has no integer division.
+    int ld_a = 0, ld_b = 0, ld_c = 0;   // WGRAD: pixel-box indices (w, h, n); FWD/DGRAD: (k-chunk, tap, unused)
+    if (MODE == MODE_WGRAD) {
+        ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
+    } else {
+        ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+    }
+    const int wg_dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, wg_ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
     auto issue_loads = [&](int it) {
         const int s = it % STAGES;
         uint8_t* sa = smem + s * C::STAGE_BYTES;
         uint8_t* sb = sa + A_STAGE_BYTES;
         mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES);
-        const int kit = k_begin + it;
         if (MODE == MODE_WGRAD) {
-            // pixel chunk kit -> box origin; A = dy (two 64-channel boxes), B = shifted activations
-            const int cw = (kit % p.tiles_w) * p.bw, ch = ((kit / p.tiles_w) % p.tiles_h) * p.bh;
-            const int cn = (kit / (p.tiles_w * p.tiles_h)) * p.bn;
-            const int dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
+            // pixel chunk -> box origin; A = dy (two 64-channel boxes), B = shifted activations
+            const int cw = ld_a * p.bw, ch = ld_b * p.bh, cn = ld_c * p.bn;
             tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
             tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + ds, ch + dr, cn);
+            for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn);
+            if (++ld_a == p.tiles_w) { ld_a = 0; if (++ld_b == p.tiles_h) { ld_b = 0; ++ld_c; } }
         } else {
-            const int tap = kit / p.kchunks, kc = kit % p.kchunks;
+            const int kc = ld_a, tap = ld_b;
             int dr = 0, ds = 0;
-            if (p.ntaps == 9) { dr = tap / 3 - 1; ds = tap % 3 - 1; }
+            if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
             if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
             tma_load_4d(&mapA, sa, &full[s], kc * 64, pw0 + ds, ph0 + dr, pn0);
             if (MODE == MODE_FWD) {
@@ -270,6 +276,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #pragma unroll
                 for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0);
             }
+            if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
         }
     };
     const int preloaded = n_iters < STAGES ? n_iters : STAGES;
@@ -283,20 +290,25 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (tlog) tlog[8] = (unsigned long long)clock64();    // barriers initialised
         pdl_wait();
         pdl_trigger();
+        if (tlog) tlog[9] = (unsigned long long)clock64();    // predecessor kernel complete
         // The first ring-full of loads needs nothing but the barriers this thread has just initialised: start
         // them now, so that their latency overlaps the TMEM allocation and the rest of the set-up.
         for (int it = 0; it < preloaded; ++it) issue_loads(it);
+        if (tlog) tlog[10] = (unsigned long long)clock64();   // first ring of loads issued
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, C::TMEM_COLS);
         tmem_relinquish();
+        if (tlog && lane == 0) tlog[11] = (unsigned long long)clock64();   // TMEM allocated
     }
     if (threadIdx.x != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
     if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
         for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
     }
+    if (tlog && threadIdx.x == 64) tlog[12] = (unsigned long long)clock64();   // bias staged
     tc_fence_before();
     __syncthreads();
     tc_fence_after();

@@ -65,7 +65,7 @@ sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
 
 const char* umma_last_error();
-// Debug aid: when set to a device buffer of 1024*8 uint64, every tensor-core CTA (first 1024 of a launch)
+// Debug aid: when set to a device buffer of 1024*16 uint64, every tensor-core CTA (first 1024 of a launch)
 // records %globaltimer at its phase boundaries: start, set-up done, first / last operands landed,
 // accumulator complete, epilogue done.
 void umma_set_timing_buffer(void* dev_ptr);
