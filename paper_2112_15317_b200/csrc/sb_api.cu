@@ -74,8 +74,14 @@ struct sb_model {
     size_t P = 0;  // padded parameter element count
     float *Wm = nullptr, *Vm = nullptr, *Gm = nullptr;
     __nv_bfloat16* Sm = nullptr;
-    float* ws = nullptr;
+    float* ws = nullptr;    // scratch of the data-side kernels (split partial sums of forward / data gradient)
+    float* ws_w = nullptr;  // scratch of the weight-side kernels (split partial sums of weight / bias gradients), so that
+                            // the two sides can run concurrently in the backward pass
     size_t ws_floats = 0;
+    // backward-pass concurrency: weight-gradient work runs on a second stream, ordered by events
+    cudaStream_t wstream = nullptr;
+    cudaEvent_t ev_join = nullptr;
+    std::vector<cudaEvent_t> ev_ready;   // one per layer: "the gradient w.r.t. this layer's output is ready"
     float *row_loss = nullptr, *loss = nullptr;
     unsigned int* counter = nullptr;
     uint32_t* status = nullptr;
@@ -117,6 +123,9 @@ struct sb_model {
     ~sb_model()
     {
         for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
+        for (cudaEvent_t e : ev_ready) cudaEventDestroy(e);
+        if (ev_join) cudaEventDestroy(ev_join);
+        if (wstream) cudaStreamDestroy(wstream);
         if (g_dev.exec) cudaGraphExecDestroy(g_dev.exec);
         if (g_host.exec) cudaGraphExecDestroy(g_host.exec);
     }
@@ -239,6 +248,7 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     if (um_ws > ws_floats) ws_floats = um_ws;
     m->ws_floats = ws_floats;
     m->ws = (float*)take(ws_floats * 4);
+    m->ws_w = (float*)take(ws_floats * 4);
     m->row_loss = (float*)take(B * 4);
     m->loss = (float*)take(256);
     m->counter = (unsigned int*)take(256);
@@ -379,7 +389,10 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
     return SB_OK;
 }
 
-sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
+// part: 1 = weight-side work (weight / bias gradients), 2 = data-side work (input gradient), 3 = both.
+// The two sides of a layer only share read-only inputs, so they may run on different streams.
+enum { SIDE_W = 1, SIDE_D = 2, SIDE_BOTH = 3 };
+sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BOTH)
 {
     Layer& l = m->L[i];
     m->cur_layer = i;
@@ -404,14 +417,15 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             FcNarrowArgs a{};
             a.pass = 1; a.X = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.tab_b = b;
             a.dY = l.dact; a.dW = m->Gm + l.p_w; a.db = m->Gm + l.p_b; a.B = B; a.in_f = l.in_f; a.out_f = l.out_f;
-            L_TRY("fc_narrow_wgrad", flops, act_bytes + (double)l.n_w * 4.0, launch_fc_narrow(a, bf, st));
-            if (want_in_grad) {
+            if (part & SIDE_W) L_TRY("fc_narrow_wgrad", flops, act_bytes + (double)l.n_w * 4.0, launch_fc_narrow(a, bf, st));
+            if (want_in_grad && (part & SIDE_D)) {
                 a.pass = 2; a.W = wts; a.ref = below_relu ? m->L[i - 1].act : nullptr; a.dX = d_below;
                 L_TRY("fc_narrow_dgrad", flops, act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0), launch_fc_narrow(a, bf, st));
             }
             break;
         }
-        if (l.um.wgrad.enabled) {
+        if (!(part & SIDE_W)) {
+        } else if (l.um.wgrad.enabled) {
             U_TRY("fc_wgrad_umma", flops, act_bytes + (double)l.n_w * 4.0, umma_fc_wgrad(m, i, st));
             ++m->launches;
         } else {
@@ -424,9 +438,9 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 2; a.tab_b = b; }
             L_TRY("fc_wgrad_simt", flops, act_bytes + (double)l.n_w * 4.0, launch_gemm_simt(a, bf, st));
         }
-        if (!l.um.wgrad.enabled)   // the tensor-core weight-gradient kernel also produces the bias gradient
+        if (!l.um.wgrad.enabled && (part & SIDE_W))   // the tensor-core weight-gradient kernel also produces the bias gradient
             L_TRY("bias_grad", 0.0, (double)B * l.out_f * e + 4.0 * l.out_f, launch_colsum(l.dact, bf, m->Gm + l.p_b, B, l.out_f, 1, st));
-        if (want_in_grad) {
+        if (want_in_grad && (part & SIDE_D)) {
             // shard-layer / modulo-layer backward: dX = sum_j dY_j W_j, rows stay with their replica
             const double bytes = act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0);
             if (l.um.dgrad.enabled) {
@@ -446,6 +460,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         break;
     }
     case SB_MAXPOOL2: {
+        if (!(part & SIDE_D)) break;
         PoolBwdArgs a{l.dact, l.idx, below_relu ? l.act : nullptr, d_below, B, l.H, l.W, l.Cin};
         const double pooled = (double)B * l.out_per_img;
         L_TRY("pool_bwd", 0.0, pooled * (e + 1 + (below_relu ? e : 0.0) + 4 * e), launch_pool_bwd(a, bf, st));
@@ -456,16 +471,17 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
         const double pix = (double)B * l.H * l.W;
         const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
         // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
-        if (l.thin_input) {
+        if (!(part & SIDE_W)) {
+        } else if (l.thin_input) {
             // input-layer kernel: weight and bias partial sums per block, then one ordered reduce each
             WgradSimtArgs a{};
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
-            a.dy = l.dact; a.part = m->ws; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
+            a.dy = l.dact; a.part = m->ws_w; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
             const int nb = conv_in_wgrad_blocks(B, l.H, l.W);
             const size_t stride = l.n_w + l.n_b;
             L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(m->ws, stride, m->Gm + l.p_w, l.n_w, nb, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(m->ws + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(m->ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(m->ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
         } else if (l.um.wgrad.enabled) {
             int S = 1;
             float* part = nullptr;
@@ -478,21 +494,21 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st)
             const int S = l.wg_splits;
             WgradSimtArgs a{};
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
-            a.dy = l.dact; a.part = S > 1 ? m->ws : m->Gm + l.p_w;
+            a.dy = l.dact; a.part = S > 1 ? m->ws_w : m->Gm + l.p_w;
             a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
             L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws_w, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
         }
-        if (!l.thin_input && !l.um.wgrad.enabled) {
+        if (!l.thin_input && !l.um.wgrad.enabled && (part & SIDE_W)) {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
             const long M = (long)B * l.H * l.W;
             // (stream order makes it safe to reuse the scratch the weight-gradient reduce just read)
             const int S = l.bg_splits;
-            float* part = S > 1 ? m->ws : m->Gm + l.p_b;
+            float* part = S > 1 ? m->ws_w : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
             if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, l.n_b, m->Gm + l.p_b, l.n_b, S, st));
         }
-        if (want_in_grad) {
+        if (want_in_grad && (part & SIDE_D)) {
             const double bytes = pix * (l.Cin + l.Cout) * e + (double)l.n_w * e + (below_relu ? pix * l.Cin * e : 0.0);
             if (l.um.dgrad.enabled) {
                 U_TRY("conv_dgrad_umma", flops, bytes, umma_conv_dgrad(m, i, st));
@@ -620,7 +636,7 @@ ModelView model_view(sb_model* m)
 {
     ModelView v{};
     v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
-    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; v.ws_floats = m->ws_floats; v.status = m->status;
+    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; v.ws_w = m->ws_w; v.ws_floats = m->ws_floats; v.status = m->status;
     v.input_grad = m->input_grad; v.x_tab = &m->x_tab; v.stage_x = m->stage_x;
     return v;
 }
@@ -664,6 +680,15 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     m->arena_bytes = need;
     const char* dbg = getenv("SB_DEBUG_SYNC");
     m->debug_sync = dbg && dbg[0] == '1';
+    const char* one = getenv("SB_ONE_STREAM");
+    if (!(one && one[0] == '1')) {
+        // second stream + ordering events for the backward pass (host objects; no device memory)
+        bool ok_ = cudaStreamCreateWithFlags(&m->wstream, cudaStreamNonBlocking) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) == cudaSuccess;
+        m->ev_ready.assign(n, nullptr);
+        for (int i = 0; ok_ && i < n; ++i) ok_ = cudaEventCreateWithFlags(&m->ev_ready[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok_) { delete m; return fail(SB_ERR_CUDA, "creating the backward-pass stream / events failed"); }
+    }
     cudaError_t e = cudaMemset(arena, 0, need);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }
@@ -725,9 +750,30 @@ sb_status sb_backward(sb_model* m, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (!m->have_fwd) return fail(SB_ERR_STATE, "sb_backward needs a preceding sb_forward");
+    cudaStream_t st = (cudaStream_t)stream;
+    // The weight-gradient work of a layer (and its split reduce) only has to be finished before the update,
+    // while the input-gradient chain is the critical path: the former runs on the model's second stream,
+    // ordered by one event per layer ("the gradient w.r.t. this layer's output is ready") and joined at the
+    // end.  Profiling and debug-sync modes keep everything on one stream.
+    const bool two_streams = m->wstream != nullptr && !m->profiling && !m->debug_sync;
     for (int i = m->n_layers - 1; i >= 0; --i) {
-        sb_status s = backward_layer(m, i, (cudaStream_t)stream);
-        if (s != SB_OK) return s;
+        const int kind = m->L[i].kind;
+        const bool has_params = kind == SB_CONV3X3_RELU || kind == SB_FC_RELU || kind == SB_FC;
+        if (two_streams && has_params) {
+            CU_TRY(cudaEventRecord(m->ev_ready[i], st));
+            CU_TRY(cudaStreamWaitEvent(m->wstream, m->ev_ready[i], 0));
+            sb_status s = backward_layer(m, i, m->wstream, SIDE_W);
+            if (s != SB_OK) return s;
+            s = backward_layer(m, i, st, SIDE_D);
+            if (s != SB_OK) return s;
+        } else {
+            sb_status s = backward_layer(m, i, st, SIDE_BOTH);
+            if (s != SB_OK) return s;
+        }
+    }
+    if (two_streams) {
+        CU_TRY(cudaEventRecord(m->ev_join, m->wstream));
+        CU_TRY(cudaStreamWaitEvent(st, m->ev_join, 0));
     }
     return SB_OK;
 }

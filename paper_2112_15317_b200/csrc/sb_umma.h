@@ -26,7 +26,8 @@ struct ModelView {
     int B, n_layers, first_fc;
     float *Wm, *Gm;
     __nv_bfloat16* Sm;
-    float* ws;
+    float* ws;      // data-side scratch
+    float* ws_w;    // weight-side scratch
     size_t ws_floats;
     uint32_t* status;
     char* input_grad;
