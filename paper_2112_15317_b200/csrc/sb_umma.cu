@@ -24,6 +24,7 @@
 #include "sb_umma.h"
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 namespace sb {
@@ -643,7 +644,16 @@ const char* umma_last_error() { return g_umma_err; }
 //  * ring depth = k-iterations per CTA, capped by what fits; for grids of several waves the ring is kept
 //    shallow enough that two CTAs share an SM, so one CTA's epilogue overlaps the other's main loop.
 struct TilePlan { int bn, splits, cps, stages; };
-static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters)
+// Backward kernels of the two concurrent streams share SMs only if two CTAs fit side by side (shared
+// memory <= ~110 KB each, TMEM columns <= 256 each): SB_BWD_COHABIT=0 gives every kernel the full ring again.
+static bool bwd_cohabit()
+{
+    static const bool on = [] { const char* e = getenv("SB_BWD_COHABIT"); return !(e && e[0] == '0'); }();
+    return on;
+}
+static int cohabit_stages(int bn) { return bn >= 256 ? 2 : (bn >= 128 ? 3 : 4); }
+
+static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward = false)
 {
     TilePlan t;
     t.bn = n_cols_per_shard >= 256 ? 256 : (n_cols_per_shard >= 128 ? 128 : 64);
@@ -658,6 +668,8 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         const int two = t.bn >= 256 ? 2 : (t.bn >= 128 ? 3 : 4);
         if (t.bn < 256 && st > two) st = two;
     }
+    static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
+    if ((backward || fwd_too) && bwd_cohabit() && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     t.stages = st < 1 ? 1 : st;
     return t;
 }
@@ -698,7 +710,7 @@ static ConvGeom conv_geom(const LayerView& lv, int B)
     g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
     g.m_tiles = (long)g.tw * g.th * g.tn;
     g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64));
-    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64));
+    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64), true);
     choose_box(lv.W, lv.H, B, 64, &g.cw, &g.ch, &g.cn);
     g.ctw = cdiv_i(lv.W, g.cw); g.cth = cdiv_i(lv.H, g.ch); g.ctn = cdiv_i(B, g.cn);
     g.total_chunks = g.ctw * g.cth * g.ctn;
@@ -719,7 +731,7 @@ static FcGeom fc_geom(const LayerView& lv, int B, int K)
     FcGeom g;
     g.m_tiles = cdiv_i(B, 128);
     g.fwd = plan_tiles(cdiv_i(lv.out_f, K), K, g.m_tiles, lv.in_f / 64);
-    g.dgrad = plan_tiles(lv.in_f, 1, g.m_tiles, cdiv_i(lv.out_f, 64));
+    g.dgrad = plan_tiles(lv.in_f, 1, g.m_tiles, cdiv_i(lv.out_f, 64), true);
     return g;
 }
 
@@ -822,6 +834,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.splits = g.wg_splits;
                 p.chunks_per_split = g.wg_cps;
                 p.stages = g.wg_cps < (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8)) ? g.wg_cps : (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8));
+                if (bwd_cohabit() && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
                 // the bias gradient rides along: in the parameter arena the bias vector directly follows the
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
@@ -890,6 +903,7 @@ sb_status umma_plan_layers(sb_model* m)
                 const int n_tiles = cdiv_i(lv.in_f, b->bn);
                 p.splits = 1; p.chunks_per_split = p.total_chunks;
                 p.stages = p.total_chunks < 4 ? p.total_chunks : 4;
+                if (bwd_cohabit() && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
                 p.epi = UEPI_F32; p.ldc = lv.in_f; p.split_stride = 0;
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
                 p.out = (void*)(mv.Gm + lv.p_w);
