@@ -75,13 +75,20 @@ struct sb_model {
     float *Wm = nullptr, *Vm = nullptr, *Gm = nullptr;
     __nv_bfloat16* Sm = nullptr;
     float* ws = nullptr;    // scratch of the data-side kernels (split partial sums of forward / data gradient)
+    float* ws_wk[4] = {nullptr, nullptr, nullptr, nullptr};   // one weight-side scratch region per weight stream
     float* ws_w = nullptr;  // scratch of the weight-side kernels (split partial sums of weight / bias gradients), so that
                             // the two sides can run concurrently in the backward pass
     size_t ws_floats = 0;
     // backward-pass concurrency: weight-gradient work runs on a second stream, ordered by events
-    cudaStream_t wstream = nullptr;
-    cudaEvent_t ev_join = nullptr;
+    static constexpr int MAX_WSTREAMS = 4;
+    int n_wstreams = 0;                          // weight-gradient work of layer i runs on wstreams[i % n_wstreams]
+    cudaStream_t wstreams[MAX_WSTREAMS] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_wjoin[MAX_WSTREAMS] = {nullptr, nullptr, nullptr, nullptr};
+    cudaStream_t ustream = nullptr;   // parameter updates folded into the backward pass
+    cudaEvent_t ev_join = nullptr, ev_ujoin = nullptr;
     std::vector<cudaEvent_t> ev_ready;   // one per layer: "the gradient w.r.t. this layer's output is ready"
+    std::vector<cudaEvent_t> ev_dgrad;   // one per layer: "this layer's input gradient has been computed"
+    std::vector<cudaEvent_t> ev_wdone;   // one per layer: "this layer's weight and bias gradients are complete"
     float *row_loss = nullptr, *loss = nullptr;
     unsigned int* counter = nullptr;
     uint32_t* status = nullptr;
@@ -124,8 +131,12 @@ struct sb_model {
     {
         for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
         for (cudaEvent_t e : ev_ready) cudaEventDestroy(e);
+        for (cudaEvent_t e : ev_dgrad) cudaEventDestroy(e);
+        for (cudaEvent_t e : ev_wdone) cudaEventDestroy(e);
+        if (ev_ujoin) cudaEventDestroy(ev_ujoin);
+        if (ustream) cudaStreamDestroy(ustream);
         if (ev_join) cudaEventDestroy(ev_join);
-        if (wstream) cudaStreamDestroy(wstream);
+        for (int k = 0; k < MAX_WSTREAMS; ++k) { if (wstreams[k]) cudaStreamDestroy(wstreams[k]); if (ev_wjoin[k]) cudaEventDestroy(ev_wjoin[k]); }
         if (g_dev.exec) cudaGraphExecDestroy(g_dev.exec);
         if (g_host.exec) cudaGraphExecDestroy(g_host.exec);
     }
@@ -248,7 +259,8 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     if (um_ws > ws_floats) ws_floats = um_ws;
     m->ws_floats = ws_floats;
     m->ws = (float*)take(ws_floats * 4);
-    m->ws_w = (float*)take(ws_floats * 4);
+    for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) m->ws_wk[k] = (float*)take(ws_floats * 4);
+    m->ws_w = m->ws_wk[0];
     m->row_loss = (float*)take(B * 4);
     m->loss = (float*)take(256);
     m->counter = (unsigned int*)take(256);
@@ -404,6 +416,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
     char* d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
     const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
     const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
+    float* const ws_w = m->ws_wk[i % sb_model::MAX_WSTREAMS];   // this layer's weight-side scratch (fixed per layer)
     switch (l.kind) {
     case SB_SOFTMAX_XENT:
         break;  // dZ was produced by the forward loss kernel
@@ -476,12 +489,12 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             // input-layer kernel: weight and bias partial sums per block, then one ordered reduce each
             WgradSimtArgs a{};
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
-            a.dy = l.dact; a.part = m->ws_w; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
+            a.dy = l.dact; a.part = ws_w; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
             const int nb = conv_in_wgrad_blocks(B, l.H, l.W);
             const size_t stride = l.n_w + l.n_b;
             L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(m->ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(m->ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
+            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
         } else if (l.um.wgrad.enabled) {
             int S = 1;
             float* part = nullptr;
@@ -494,17 +507,17 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             const int S = l.wg_splits;
             WgradSimtArgs a{};
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
-            a.dy = l.dact; a.part = S > 1 ? m->ws_w : m->Gm + l.p_w;
+            a.dy = l.dact; a.part = S > 1 ? ws_w : m->Gm + l.p_w;
             a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
             L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(m->ws_w, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
+            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(ws_w, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
         }
         if (!l.thin_input && !l.um.wgrad.enabled && (part & SIDE_W)) {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
             const long M = (long)B * l.H * l.W;
             // (stream order makes it safe to reuse the scratch the weight-gradient reduce just read)
             const int S = l.bg_splits;
-            float* part = S > 1 ? m->ws_w : m->Gm + l.p_b;
+            float* part = S > 1 ? ws_w : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
             if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, l.n_b, m->Gm + l.p_b, l.n_b, S, st));
         }
@@ -636,7 +649,7 @@ ModelView model_view(sb_model* m)
 {
     ModelView v{};
     v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
-    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; v.ws_w = m->ws_w; v.ws_floats = m->ws_floats; v.status = m->status;
+    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) v.ws_wk[k] = m->ws_wk[k]; v.ws_floats = m->ws_floats; v.status = m->status;
     v.input_grad = m->input_grad; v.x_tab = &m->x_tab; v.stage_x = m->stage_x;
     return v;
 }
@@ -683,10 +696,24 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     const char* one = getenv("SB_ONE_STREAM");
     if (!(one && one[0] == '1')) {
         // second stream + ordering events for the backward pass (host objects; no device memory)
-        bool ok_ = cudaStreamCreateWithFlags(&m->wstream, cudaStreamNonBlocking) == cudaSuccess &&
-                   cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) == cudaSuccess;
+        const char* nws = getenv("SB_WSTREAMS");
+        m->n_wstreams = nws ? atoi(nws) : 3;
+        if (m->n_wstreams < 1) m->n_wstreams = 1;
+        if (m->n_wstreams > sb_model::MAX_WSTREAMS) m->n_wstreams = sb_model::MAX_WSTREAMS;
+        bool ok_ = true;
+        for (int k = 0; ok_ && k < m->n_wstreams; ++k)
+            ok_ = cudaStreamCreateWithFlags(&m->wstreams[k], cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&m->ev_wjoin[k], cudaEventDisableTiming) == cudaSuccess;
+        ok_ = ok_ && cudaStreamCreateWithFlags(&m->ustream, cudaStreamNonBlocking) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&m->ev_ujoin, cudaEventDisableTiming) == cudaSuccess;
         m->ev_ready.assign(n, nullptr);
-        for (int i = 0; ok_ && i < n; ++i) ok_ = cudaEventCreateWithFlags(&m->ev_ready[i], cudaEventDisableTiming) == cudaSuccess;
+        m->ev_dgrad.assign(n, nullptr);
+        m->ev_wdone.assign(n, nullptr);
+        for (int i = 0; ok_ && i < n; ++i)
+            ok_ = cudaEventCreateWithFlags(&m->ev_ready[i], cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&m->ev_dgrad[i], cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&m->ev_wdone[i], cudaEventDisableTiming) == cudaSuccess;
         if (!ok_) { delete m; return fail(SB_ERR_CUDA, "creating the backward-pass stream / events failed"); }
     }
     cudaError_t e = cudaMemset(arena, 0, need);
@@ -746,36 +773,81 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
     return SB_OK;
 }
 
-sb_status sb_backward(sb_model* m, void* stream)
+// Backward pass; with `fuse_update` the SGD update of each layer's parameters is enqueued on the weight-side
+// stream as soon as that layer's gradients are complete and its input gradient (which reads the weights) has
+// been computed, so the bandwidth-bound update overlaps the rest of the backward pass.  Element for element the
+// update is the one sb_sgd_step does.  Returns *updated = true if the update was done here.
+static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, float lr, float mu, bool* updated)
 {
-    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
-    if (!m->have_fwd) return fail(SB_ERR_STATE, "sb_backward needs a preceding sb_forward");
-    cudaStream_t st = (cudaStream_t)stream;
     // The weight-gradient work of a layer (and its split reduce) only has to be finished before the update,
     // while the input-gradient chain is the critical path: the former runs on the model's second stream,
     // ordered by one event per layer ("the gradient w.r.t. this layer's output is ready") and joined at the
     // end.  Profiling and debug-sync modes keep everything on one stream.
-    const bool two_streams = m->wstream != nullptr && !m->profiling && !m->debug_sync;
+    const bool two_streams = m->n_wstreams > 0 && !m->profiling && !m->debug_sync;
+    const bool fuse = fuse_update && two_streams;
+    if (updated) *updated = fuse;
     for (int i = m->n_layers - 1; i >= 0; --i) {
-        const int kind = m->L[i].kind;
-        const bool has_params = kind == SB_CONV3X3_RELU || kind == SB_FC_RELU || kind == SB_FC;
+        Layer& l = m->L[i];
+        const bool has_params = l.kind == SB_CONV3X3_RELU || l.kind == SB_FC_RELU || l.kind == SB_FC;
         if (two_streams && has_params) {
+            cudaStream_t wst = m->wstreams[i % m->n_wstreams];
             CU_TRY(cudaEventRecord(m->ev_ready[i], st));
-            CU_TRY(cudaStreamWaitEvent(m->wstream, m->ev_ready[i], 0));
-            sb_status s = backward_layer(m, i, m->wstream, SIDE_W);
+            CU_TRY(cudaStreamWaitEvent(wst, m->ev_ready[i], 0));
+            sb_status s = backward_layer(m, i, wst, SIDE_W);
             if (s != SB_OK) return s;
             s = backward_layer(m, i, st, SIDE_D);
             if (s != SB_OK) return s;
+            if (fuse) {
+                // The update of this layer runs on a third stream: after the layer's gradients are complete (weight
+                // stream) and after its input-gradient kernel, which reads the weights the update rewrites (main stream).
+                CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
+                CU_TRY(cudaEventRecord(m->ev_wdone[i], wst));
+                CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_dgrad[i], 0));
+                CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_wdone[i], 0));
+                const size_t off = l.p_w, cnt = (l.p_b - l.p_w) + align_up(l.n_b, 64);
+                {
+                    cudaStream_t st = m->ustream;   // the launch bracket below records on the stream it launches on
+                    m->cur_layer = i;
+                    L_TRY("sgd", 0.0, (double)cnt * (m->bf16 ? 22.0 : 20.0),
+                          launch_sgd(m->Wm + off, m->Vm + off, m->Gm + off, m->Sm ? m->Sm + off : nullptr, cnt, lr, mu, st));
+                }
+            }
         } else {
             sb_status s = backward_layer(m, i, st, SIDE_BOTH);
             if (s != SB_OK) return s;
         }
     }
     if (two_streams) {
-        CU_TRY(cudaEventRecord(m->ev_join, m->wstream));
-        CU_TRY(cudaStreamWaitEvent(st, m->ev_join, 0));
+        for (int k = 0; k < m->n_wstreams; ++k) {
+            CU_TRY(cudaEventRecord(m->ev_wjoin[k], m->wstreams[k]));
+            CU_TRY(cudaStreamWaitEvent(st, m->ev_wjoin[k], 0));
+        }
+    }
+    if (fuse) {
+        CU_TRY(cudaEventRecord(m->ev_ujoin, m->ustream));
+        CU_TRY(cudaStreamWaitEvent(st, m->ev_ujoin, 0));
+        m->last_step_launches = m->launches;
     }
     return SB_OK;
+}
+
+sb_status sb_backward(sb_model* m, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (!m->have_fwd) return fail(SB_ERR_STATE, "sb_backward needs a preceding sb_forward");
+    return backward_pass(m, (cudaStream_t)stream, false, 0.f, 0.f, nullptr);
+}
+
+// forward + backward + update of one iteration, with the update folded into the backward pass when possible
+static sb_status whole_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float mu, void* stream)
+{
+    sb_status s = sb_forward(m, x, labels, stream);
+    if (s != SB_OK) return s;
+    bool updated = false;
+    s = backward_pass(m, (cudaStream_t)stream, true, lr, mu, &updated);
+    if (s != SB_OK) return s;
+    if (!updated) s = sb_sgd_step(m, lr, mu, stream);
+    return s;
 }
 
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)
@@ -839,9 +911,7 @@ sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const*
     const bool eager = m->profiling || m->debug_sync || !G.warmed || st == nullptr;
     if (eager) {
         // first use (one-time function attributes are set by the first launches), or a mode that needs every launch visible
-        sb_status s = sb_forward(m, x, labels, stream);
-        if (s == SB_OK) s = sb_backward(m, stream);
-        if (s == SB_OK) s = sb_sgd_step(m, lr, momentum, stream);
+        sb_status s = whole_step(m, x, labels, lr, momentum, stream);
         if (s == SB_OK) G.warmed = true;
         return s;
     }
@@ -849,9 +919,7 @@ sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const*
     if (!hit) {
         if (G.exec) { cudaGraphExecDestroy(G.exec); G.exec = nullptr; }
         CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        sb_status s = sb_forward(m, x, labels, stream);
-        if (s == SB_OK) s = sb_backward(m, stream);
-        if (s == SB_OK) s = sb_sgd_step(m, lr, momentum, stream);
+        sb_status s = whole_step(m, x, labels, lr, momentum, stream);
         if (s != SB_OK) { abandon_capture(st); return s; }
         cudaGraph_t graph = nullptr;
         CU_TRY(cudaStreamEndCapture(st, &graph));
@@ -883,11 +951,7 @@ sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* hos
     if (eager) {
         CU_TRY(cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st));
         CU_TRY(cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st));
-        sb_status s = sb_forward(m, xp, lp, stream);
-        if (s != SB_OK) return s;
-        s = sb_backward(m, stream);
-        if (s != SB_OK) return s;
-        s = sb_sgd_step(m, lr, momentum, stream);
+        sb_status s = whole_step(m, xp, lp, lr, momentum, stream);
         if (s != SB_OK) return s;
         G.warmed = true;
         return sb_loss(m, stream, host_loss);
@@ -900,9 +964,7 @@ sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* hos
         cudaError_t e = cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) e = cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st);
         sb_status s = e == cudaSuccess ? SB_OK : fail(SB_ERR_CUDA, "capturing the input copies: %s", cudaGetErrorString(e));
-        if (s == SB_OK) s = sb_forward(m, xp, lp, stream);
-        if (s == SB_OK) s = sb_backward(m, stream);
-        if (s == SB_OK) s = sb_sgd_step(m, lr, momentum, stream);
+        if (s == SB_OK) s = whole_step(m, xp, lp, lr, momentum, stream);
         if (s == SB_OK) {
             e = cudaMemcpyAsync(&m->host_result[0], m->loss, 4, cudaMemcpyDeviceToHost, st);
             if (e == cudaSuccess) e = cudaMemcpyAsync(&m->host_result[1], m->status, 4, cudaMemcpyDeviceToHost, st);

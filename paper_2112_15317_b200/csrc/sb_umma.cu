@@ -840,7 +840,7 @@ sb_status umma_plan_layers(sb_model* m)
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
                 p.split_stride = (long)(lv.n_w + lv.n_b);
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
-                p.out = p.splits > 1 ? (void*)mv.ws_w : (void*)(mv.Gm + lv.p_w);
+                p.out = p.splits > 1 ? (void*)mv.ws_wk[i % 4] : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
                 b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 * p.splits));
                 if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;

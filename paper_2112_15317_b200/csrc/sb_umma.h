@@ -27,7 +27,7 @@ struct ModelView {
     float *Wm, *Gm;
     __nv_bfloat16* Sm;
     float* ws;      // data-side scratch
-    float* ws_w;    // weight-side scratch
+    float* ws_wk[4];  // weight-side scratch regions; layer i uses ws_wk[i % 4]
     size_t ws_floats;
     uint32_t* status;
     char* input_grad;
