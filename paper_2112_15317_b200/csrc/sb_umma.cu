@@ -653,14 +653,40 @@ static bool bwd_cohabit()
 }
 static int cohabit_stages(int bn) { return bn >= 256 ? 2 : (bn >= 128 ? 3 : 4); }
 
+// Cost model behind the tile plan (micro-seconds, calibrated on per-CTA phase timings at VGG-16/CIFAR sizes):
+// a CTA costs ~3 us of fixed work (cold start, first loads, drain, epilogue) plus ~0.4 us per k-iteration (the
+// operand ring is latency / L2-bandwidth bound, almost independently of the tile width); CTAs run in waves of one
+// per SM (two when the ring is shallow); a split reduction adds a second kernel (~8 us with its launch gap).
+static double plan_cost(int bn, int s, int n_cols_per_shard, int shards, long m_tiles, int k_iters)
+{
+    const long ctas = m_tiles * cdiv_i(n_cols_per_shard, bn) * shards * s;
+    const double per_sm = (bn < 256 && ctas >= 296) ? 2.0 : 1.0;
+    const double waves = (double)cdiv_i(ctas, (long)(148 * per_sm));
+    const double t_iter = bn >= 256 ? 0.41 : (bn >= 128 ? 0.37 : 0.33);
+    return waves * (cdiv_i(k_iters, s) * t_iter * (per_sm > 1.0 ? 1.6 : 1.0) + 3.0) + (s > 1 ? 8.0 : 0.0);
+}
 static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward = false)
 {
     TilePlan t;
-    t.bn = n_cols_per_shard >= 256 ? 256 : (n_cols_per_shard >= 128 ? 128 : 64);
+    static const bool legacy = [] { const char* e = getenv("SB_PLAN_LEGACY"); return e && e[0] == '1'; }();
+    int best_bn = 64, best_s = 1;
+    if (legacy) {
+        best_bn = n_cols_per_shard >= 256 ? 256 : (n_cols_per_shard >= 128 ? 128 : 64);
+        const long tiles = m_tiles * cdiv_i(n_cols_per_shard, best_bn) * shards;
+        while (tiles * best_s < 120 && k_iters / (best_s * 2) >= 4) best_s *= 2;
+    } else {
+        double best = 1e300;
+        for (int bn = 64; bn <= 256; bn *= 2) {
+            if (bn > 64 && bn / 2 >= n_cols_per_shard) break;      // never wider than the columns need
+            for (int s = 1; s <= 32 && (s == 1 || k_iters / s >= 4); s *= 2) {
+                const double c = plan_cost(bn, s, n_cols_per_shard, shards, m_tiles, k_iters);
+                if (c < best - 1e-9) { best = c; best_bn = bn; best_s = s; }
+            }
+        }
+    }
+    t.bn = best_bn;
     const long tiles = m_tiles * cdiv_i(n_cols_per_shard, t.bn) * shards;
-    int s = 1;
-    while (tiles * s < 120 && k_iters / (s * 2) >= 4) s *= 2;
-    t.cps = cdiv_i(k_iters, s);
+    t.cps = cdiv_i(k_iters, best_s);
     t.splits = cdiv_i(k_iters, t.cps);
     const int fit = t.bn >= 256 ? 4 : (t.bn >= 128 ? 6 : 8);
     int st = t.cps < fit ? t.cps : fit;
@@ -671,6 +697,8 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
     if ((backward || fwd_too) && bwd_cohabit() && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     t.stages = st < 1 ? 1 : st;
+    static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
+    if (verbose) fprintf(stderr, "plan: N/shard=%d shards=%d m_tiles=%ld k_iters=%d -> bn=%d splits=%d stages=%d\n", n_cols_per_shard, shards, m_tiles, k_iters, t.bn, t.splits, t.stages);
     return t;
 }
 
