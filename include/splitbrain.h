@@ -69,7 +69,10 @@ enum { SB_FP32 = 0, SB_BF16 = 1 };
 enum {
     SB_FLAG_INPUT_GRAD = 1,  /* also compute the gradient w.r.t. the network input (layer 0 dgrad) */
     SB_FLAG_FORCE_SIMT = 2,  /* use the CUDA-core kernels for every layer (cross-check / debugging) */
-    SB_FLAG_PROFILE_LAYERS = 4 /* sb_profile_end reports one entry per (kernel class, layer): "name#layer" */
+    SB_FLAG_PROFILE_LAYERS = 4, /* sb_profile_end reports one entry per (kernel class, layer): "name#layer" */
+    SB_FLAG_FORCE_PAIR = 8   /* run every forward / data-gradient GEMM whose N tile is 128 or 256 wide on CTA pairs
+                                (tcgen05 cta_group::2), whatever the grid size; by default the planner uses pairs only
+                                where they pay (256-wide tiles, at least one wave of CTAs) */
 };
 
 typedef struct {

@@ -55,7 +55,7 @@ struct PtrTab {
 };
 
 // Device status word codes (written by kernels that give up on a bounded wait).
-enum : uint32_t { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3 };
+enum : uint32_t { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_PAIR_TMEM = 4 };
 
 // ---------------------------------------------------------------------------------------------
 // CUDA-core ("SIMT") kernels: the float mode, odd channel counts, and the cross-check path.

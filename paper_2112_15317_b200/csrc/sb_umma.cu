@@ -20,7 +20,12 @@
 // Hang safety: every mbarrier wait is bounded (iteration cap and a wall-clock deadline); a wait
 // that gives up records a code in the model's device status word and the CTA drains and exits
 // normally (TMEM is always released), so a broken pipeline turns into SB_ERR_TIMEOUT on the
-// host instead of a stuck GPU.  No multicast is used anywhere.
+// host instead of a stuck GPU.
+//
+// Large forward / data-gradient grids with 256-wide N tiles run on CTA pairs (umma_pair_kernel,
+// tcgen05.mma.cta_group::2): two neighbouring M tiles share one fetch of the weight-side operand.
+// No load uses multicast; the only multicast is the pair kernel's tcgen05.commit, which releases a
+// ring slot in both CTAs of the pair.
 #include "sb_umma.h"
 
 #include <cstdio>
@@ -163,11 +168,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)2 << 61;   // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = n.
-__host__ __device__ constexpr uint32_t make_idesc(int n, int a_mn_major, int b_mn_major)
+// Instruction descriptor: bf16 x bf16 -> f32, M = m (128; 256 for a CTA pair), N = n.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int a_mn_major, int b_mn_major, int m = 128)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 constexpr int UMMA_THREADS = 192;
@@ -182,6 +187,89 @@ template <int MODE, int BN> struct Cfg {
     static constexpr int TMEM_COLS = BN;
     static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES; }
 };
+
+// Epilogue of one accumulator row: reads BN columns of this warp's TMEM lane quadrant (16 at a time) and
+// writes them as raw split partial sums, or with bias + ReLU / the ReLU mask applied, as float or bf16.
+template <int MODE, int BN>
+__device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, bool row_ok, size_t row_off, int n0, int n_hi,
+                                          int split, const float* s_bias)
+{
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c0, v);     // warp-collective: executed by all lanes regardless of row_ok
+        tmem_ld_wait();
+        if (!row_ok || n0 + c0 >= n_hi) continue;
+        float f[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
+        const int ncol = n0 + c0;
+        const bool full16 = ncol + 16 <= n_hi;
+        if (MODE != MODE_WGRAD && p.splits > 1) {
+            // split reduction: raw partial sums; bias / ReLU / mask / rounding happen in the reduce kernel
+            float* op = p.part + (size_t)split * p.split_stride + row_off + ncol;   // ldc == n_total in these modes
+            if (full16 && ((p.n_total & 3) == 0) && ((ncol & 3) == 0)) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (ncol + j < n_hi) op[j] = f[j];
+            }
+            continue;
+        }
+        if (p.epi == UEPI_BIAS_ACT) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                f[j] += s_bias[c0 + j];
+                if (p.relu && !(f[j] > 0.f)) f[j] = 0.f;
+            }
+        } else if (p.epi == UEPI_MASK && p.ref != nullptr) {
+            const __nv_bfloat16* rp = p.ref + row_off + ncol;
+            if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
+                uint4 r0 = *(const uint4*)rp, r1 = *(const uint4*)(rp + 8);
+                const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
+                const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
+                    if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (ncol + j < n_hi && !(__bfloat162float(rp[j]) > 0.f)) f[j] = 0.f;
+            }
+        }
+        if (p.epi == UEPI_F32 || p.out_f32) {
+            float* op = (float*)p.out + row_off + ncol;
+            if (full16 && ((p.ldc & 3) == 0) && ((ncol & 3) == 0) && ((((size_t)p.split_stride) & 3) == 0) && ((p.w_cols & 3) == 0 || MODE != MODE_WGRAD)) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (ncol + j < n_hi) op[j] = f[j];
+            }
+        } else {
+            __nv_bfloat16* op = (__nv_bfloat16*)p.out + row_off + ncol;
+            if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+                    pk[j] = *(uint32_t*)&t;
+                }
+                ((uint4*)op)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                ((uint4*)op)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (ncol + j < n_hi) op[j] = __float2bfloat16_rn(f[j]);
+            }
+        }
+    }
+}
 
 // ------------------------------------------------------------------------------------------------
 // The kernel
@@ -400,81 +488,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld16(taddr + c0, v);     // warp-collective: executed by all lanes regardless of row_ok
-                tmem_ld_wait();
-                if (!row_ok || n0 + c0 >= n_hi) continue;
-                float f[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
-                const int ncol = n0 + c0;
-                const bool full16 = ncol + 16 <= n_hi;
-                if (MODE != MODE_WGRAD && p.splits > 1) {
-                    // split reduction: raw partial sums; bias / ReLU / mask / rounding happen in the reduce kernel
-                    float* op = p.part + (size_t)split * p.split_stride + row_off + ncol;   // ldc == n_total in these modes
-                    if (full16 && ((p.n_total & 3) == 0) && ((ncol & 3) == 0)) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (ncol + j < n_hi) op[j] = f[j];
-                    }
-                    continue;
-                }
-                if (p.epi == UEPI_BIAS_ACT) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        f[j] += s_bias[c0 + j];
-                        if (p.relu && !(f[j] > 0.f)) f[j] = 0.f;
-                    }
-                } else if (p.epi == UEPI_MASK && p.ref != nullptr) {
-                    const __nv_bfloat16* rp = p.ref + row_off + ncol;
-                    if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
-                        uint4 r0 = *(const uint4*)rp, r1 = *(const uint4*)(rp + 8);
-                        const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
-                        const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
-                            if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (ncol + j < n_hi && !(__bfloat162float(rp[j]) > 0.f)) f[j] = 0.f;
-                    }
-                }
-                if (p.epi == UEPI_F32 || p.out_f32) {
-                    float* op = (float*)p.out + row_off + ncol;
-                    if (full16 && ((p.ldc & 3) == 0) && ((ncol & 3) == 0) && ((((size_t)p.split_stride) & 3) == 0) && ((p.w_cols & 3) == 0 || MODE != MODE_WGRAD)) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) ((float4*)op)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (ncol + j < n_hi) op[j] = f[j];
-                    }
-                } else {
-                    __nv_bfloat16* op = (__nv_bfloat16*)p.out + row_off + ncol;
-                    if (full16 && ((p.ldc & 7) == 0) && ((ncol & 7) == 0)) {
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
-                            pk[j] = *(uint32_t*)&t;
-                        }
-                        ((uint4*)op)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        ((uint4*)op)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (ncol + j < n_hi) op[j] = __float2bfloat16_rn(f[j]);
-                    }
-                }
-            }
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias);
         }
     }
 
@@ -491,6 +505,238 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The CTA-pair kernel (FWD / DGRAD): tcgen05.mma.cta_group::2
+// ------------------------------------------------------------------------------------------------
+// Two CTAs of a cluster -- neighbouring M tiles with the same N tile and split -- run as one 256 x BN MMA.
+// Each CTA fetches its own 128-row A tile but only HALF of the B tile (BN/2 columns); the tensor core reads
+// both halves across the pair, so the weight-side operand crosses L2 -> shared memory once per pair instead
+// of once per CTA (the operand ring is bound by each SM's L2 read bandwidth).  Protocol:
+//   * both producers aim their TMA completions at the LEADER's (cluster rank 0) full[s] barrier, which
+//     expects the bytes of both CTAs;
+//   * the leader's MMA thread issues cta_group::2 MMAs (D rows 0..127 land in the leader's TMEM, rows
+//     128..255 in the peer's, same column range) and releases ring slot s in BOTH CTAs with a multicast commit;
+//   * each CTA's epilogue warps read their own TMEM and write their own 128 output rows.
+// No load uses multicast.  All waits are bounded as in the single-CTA kernel.
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t caddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(caddr) : "memory");
+    return v;
+}
+// TMA load whose completion may signal a barrier in the peer CTA (`bar_caddr` is a shared::cluster address)
+__device__ __forceinline__ void tma_load_4d_pair(const CUtensorMap* map, void* dst, uint32_t bar_caddr, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(bar_caddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar)
+{
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+}
+
+template <int BN> struct PairCfg {
+    static constexpr int B_HALF_BYTES = BN * 64;                       // BN/2 rows (or K x BN/2 columns) of 128 bytes
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_HALF_BYTES;
+    static constexpr int MAX_STAGES_FIT = (BN >= 256) ? 6 : 8;
+    static constexpr int TMEM_COLS = BN;
+    static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 + CTRL_BYTES; }
+};
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaParams p)
+{
+    static_assert(MODE != MODE_WGRAD && BN >= 128, "pair kernel: FWD / DGRAD with N tiles of 128 or 256");
+    using C = PairCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int STAGES = p.stages;
+    uint8_t* ctrl = smem + STAGES * C::STAGE_BYTES;
+    uint64_t* full = (uint64_t*)ctrl;
+    uint64_t* empty = full + MAX_STAGES;
+    uint64_t* acc_full = empty + MAX_STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(acc_full + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* s_bias = (float*)(ctrl + 512);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t rank = cluster_ctarank();       // 0: leader (issues the MMAs), 1: peer
+    const bool leader = rank == 0;
+
+    // ---- tile coordinates (the pair shares blockIdx.y / blockIdx.z; its M tiles are 2j and 2j+1) ----
+    const int m_idx = blockIdx.x, n_idx = blockIdx.y, split = blockIdx.z;
+    const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
+    const int lo = (int)(((long)sh * p.n_total) / p.shards), n_hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
+    const int n0 = lo + t * BN;
+    if (n0 >= n_hi) return;   // uniform over the pair, before any barrier or TMEM allocation
+    // an M index past the last tile (odd tile count) lands wholly out of bounds: zero loads, no stores
+    const int pw0 = (m_idx % p.tiles_w) * p.bw;
+    const int ph0 = ((m_idx / p.tiles_w) % p.tiles_h) * p.bh;
+    const int pn0 = (m_idx / (p.tiles_w * p.tiles_h)) * p.bn;
+    const int k_begin = split * p.chunks_per_split;
+    const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
+    const int n_iters = k_end - k_begin;
+
+    int ld_a = k_begin % p.kchunks, ld_b = k_begin / p.kchunks;   // (k-chunk, tap) of the next load
+    const int nb0 = n0 + (int)rank * (BN / 2);                     // first B column this CTA fetches
+    const uint32_t full0_leader = map_to_cta(smem_u32(&full[0]), 0);
+    auto issue_loads = [&](int it) {
+        const int s = it % STAGES;
+        uint8_t* sa = smem + s * C::STAGE_BYTES;
+        uint8_t* sb = sa + A_STAGE_BYTES;
+        const uint32_t bar = full0_leader + (uint32_t)s * 8u;
+        if (leader) mbar_expect_tx(&full[s], 2u * (uint32_t)C::STAGE_BYTES);
+        const int kc = ld_a, tap = ld_b;
+        int dr = 0, ds = 0;
+        if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
+        if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
+        tma_load_4d_pair(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0);
+        if (MODE == MODE_FWD) {
+            tma_load_4d_pair(&mapB, sb, bar, tap * p.w_cols + kc * 64, nb0, 0, 0);     // box of BN/2 rows
+        } else {
+#pragma unroll
+            for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair(&mapB, sb + j * 8192, bar, tap * p.w_cols + nb0 + 64 * j, kc * 64, 0, 0);
+        }
+        if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
+    };
+    const int preloaded = n_iters < STAGES ? n_iters : STAGES;
+
+    // ---- one-time setup -----------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    cluster_sync_all();    // both CTAs' barriers exist before any copy or commit can signal them
+    if (threadIdx.x == 0) {
+        pdl_wait();
+        pdl_trigger();
+        for (int it = 0; it < preloaded; ++it) issue_loads(it);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, C::TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    if (threadIdx.x != 0) pdl_wait();
+    if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
+        for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();    // the peer's accumulator columns are allocated before the leader's first MMA writes them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = preloaded; it < n_iters; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+                if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
+                if (*abort_flag) break;
+                issue_loads(it);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = make_idesc(BN, 0, MODE != MODE_FWD, 256);
+            // the MMA addresses both accumulators with one TMEM address: the pair must have been given the same columns
+            bool ok = ld_cluster_u32(map_to_cta(smem_u32(tmem_slot), 1)) == tmem_base;
+            if (!ok) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_PAIR_TMEM); }
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+                if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ad = make_desc(sa + kk * 32, 16);
+                    const uint64_t bd = (MODE == MODE_FWD) ? make_desc(sb + kk * 32, 16) : make_desc(sb + kk * 2048, 8192);
+                    umma_bf16_pair(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit_pair(&empty[s]);
+            }
+            if (ok) umma_commit_pair(acc_full);
+        }
+    } else {
+        const int q = warp % 4;
+        const int row = q * 32 + lane;
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(acc_full, 0);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) {
+            if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+        } else {
+            tc_fence_after();
+            const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
+            const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+            const bool row_ok = w < p.W && h < p.H && n < p.N;
+            const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias);
+        }
+    }
+
+    // ---- teardown ------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) { }
+        __syncthreads();
+    }
+    cluster_sync_all();    // neither CTA leaves (or frees TMEM) while its partner may still signal or read it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
     }
 }
 
@@ -584,6 +830,42 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
     return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, p);
 }
 
+// CTA-pair launch: clusters of two CTAs along x, programmatic dependent launch as everywhere else.
+template <int MODE, int BN>
+static cudaError_t launch_pair_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             PairCfg<BN>::smem_bytes(PairCfg<BN>::MAX_STAGES_FIT));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (p.stages < 1 || p.stages > PairCfg<BN>::MAX_STAGES_FIT || (grid.x & 1u)) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(UMMA_THREADS);
+    cfg.dynamicSmemBytes = (size_t)PairCfg<BN>::smem_bytes(p.stages);
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<MODE, BN>, op.mapA, op.mapB, p);
+}
+template <int MODE>
+static cudaError_t launch_pair_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    switch (bn) {
+    case 128: return launch_pair_one<MODE, 128>(op, p, grid, st);
+    case 256: return launch_pair_one<MODE, 256>(op, p, grid, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
 template <int MODE>
 static cudaError_t launch_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
 {
@@ -599,6 +881,7 @@ static cudaError_t launch_mode(int bn, const UmmaOp& op, const UmmaParams& p, di
 struct OpBlock {
     UmmaParams p;
     int bn;
+    int pair;      // FWD / DGRAD: run as CTA pairs (umma_pair_kernel); grid.x is then even
     dim3 grid;
     long rows;     // output rows (pixels / batch rows) of a FWD / DGRAD op
 };
@@ -615,7 +898,9 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     cudaError_t e;
     UmmaParams pp = b->p;
     pp.timing = g_timing;
-    if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    else if (b->pair && b->p.mode == MODE_DGRAD) e = launch_pair_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
+    else if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
     else e = launch_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
     if (e == cudaSuccess && b->p.mode != MODE_WGRAD && b->p.splits > 1) {
@@ -643,7 +928,7 @@ const char* umma_last_error() { return g_umma_err; }
 //    reduced in split order by splitk_epilogue) while every CTA keeps at least 4 k-iterations,
 //  * ring depth = k-iterations per CTA, capped by what fits; for grids of several waves the ring is kept
 //    shallow enough that two CTAs share an SM, so one CTA's epilogue overlaps the other's main loop.
-struct TilePlan { int bn, splits, cps, stages; };
+struct TilePlan { int bn, splits, cps, stages, pair; };
 // Backward kernels of the two concurrent streams share SMs only if two CTAs fit side by side (shared
 // memory <= ~110 KB each, TMEM columns <= 256 each): SB_BWD_COHABIT=0 gives every kernel the full ring again.
 static bool bwd_cohabit()
@@ -665,7 +950,7 @@ static double plan_cost(int bn, int s, int n_cols_per_shard, int shards, long m_
     const double t_iter = bn >= 256 ? 0.41 : (bn >= 128 ? 0.37 : 0.33);
     return waves * (cdiv_i(k_iters, s) * t_iter * (per_sm > 1.0 ? 1.6 : 1.0) + 3.0) + (s > 1 ? 8.0 : 0.0);
 }
-static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward = false)
+static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward, bool force_pair)
 {
     TilePlan t;
     static const bool legacy = [] { const char* e = getenv("SB_PLAN_LEGACY"); return e && e[0] == '1'; }();
@@ -678,6 +963,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         double best = 1e300;
         for (int bn = 64; bn <= 256; bn *= 2) {
             if (bn > 64 && bn / 2 >= n_cols_per_shard) break;      // never wider than the columns need
+            if (force_pair && bn < 256 && bn < n_cols_per_shard) continue;   // forced pairs: the widest tile only
             for (int s = 1; s <= 32 && (s == 1 || k_iters / s >= 4); s *= 2) {
                 const double c = plan_cost(bn, s, n_cols_per_shard, shards, m_tiles, k_iters);
                 if (c < best - 1e-9) { best = c; best_bn = bn; best_s = s; }
@@ -697,19 +983,60 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
     if ((backward || fwd_too) && bwd_cohabit() && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     t.stages = st < 1 ? 1 : st;
+    // CTA pairs: half the weight-side operand per CTA (a smaller stage, so a deeper ring).  Measured at VGG-16 /
+    // ImageNet sizes the pair kernel is 1.2-1.3x faster where the N tile is 256 wide and the grid fills the
+    // machine, slower for 128-wide tiles and for grids of less than a wave (two cluster barriers of fixed cost).
+    // SB_PAIR=0 turns it off, SB_PAIR_MIN_CTAS moves the grid-size threshold.
+    static const bool pair_on = [] { const char* e = getenv("SB_PAIR"); return !(e && e[0] == '0'); }();
+    static const long pair_min_ctas = [] { const char* e = getenv("SB_PAIR_MIN_CTAS"); return e ? atol(e) : 148L; }();
+    t.pair = 0;
+    // (SB_FLAG_FORCE_PAIR: every 128- or 256-wide tile, whatever the grid -- for tests at small sizes)
+    if ((pair_on && t.bn == 256 && m_tiles % 2 == 0 && tiles * t.splits >= pair_min_ctas) || (force_pair && t.bn >= 128)) {
+        t.pair = 1;
+        const int pfit = t.bn >= 256 ? 6 : 8;
+        int pst = t.cps < pfit ? t.cps : pfit;
+        const int ptwo = t.bn >= 256 ? 3 : 4;      // two resident CTAs per SM
+        if ((backward || fwd_too) && bwd_cohabit() && pst > ptwo) pst = ptwo;
+        t.stages = pst < 1 ? 1 : pst;
+    }
     static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
-    if (verbose) fprintf(stderr, "plan: N/shard=%d shards=%d m_tiles=%ld k_iters=%d -> bn=%d splits=%d stages=%d\n", n_cols_per_shard, shards, m_tiles, k_iters, t.bn, t.splits, t.stages);
+    if (verbose) fprintf(stderr, "plan: N/shard=%d shards=%d m_tiles=%ld k_iters=%d -> bn=%d splits=%d stages=%d pair=%d\n", n_cols_per_shard, shards, m_tiles, k_iters, t.bn, t.splits, t.stages, t.pair);
     return t;
 }
 
-// Conv weight-gradient split count: fill the machine once (148 CTAs), keep at least 4 pixel chunks per
-// CTA, and never write more split buffers than the pixel work justifies (each split costs a full
-// float copy of the weight gradient in traffic).
-static int wgrad_splits(long ctas_without_split, int total_chunks)
+// Conv weight-gradient split count. Splitting the pixel (K) dimension fills more SMs but every split
+// writes a float copy of the weight gradient and the ordered reduce reads them all back, so the choice is
+// a small cost model: waves x (chunks per CTA x per-chunk operand time + fixed CTA cost) for the GEMM
+// plus, when split, (S + 1) gradient copies through HBM/L2 and one more launch for the reduce.
+// SB_WGRAD_SPLITS=legacy restores the older rule (fill 148 CTAs, at least 4 chunks per CTA).
+static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_t grad_floats)
 {
-    int s = 1;
-    while (ctas_without_split * s < 148 && total_chunks / (s * 2) >= 4) s *= 2;
-    return s;
+    static const bool legacy = [] { const char* e = getenv("SB_WGRAD_SPLITS"); return e && e[0] == 'l'; }();
+    if (legacy) {
+        int s = 1;
+        while (ctas_without_split * s < 148 && total_chunks / (s * 2) >= 4) s *= 2;
+        return s;
+    }
+    static const double reduce_gbs = [] { const char* e = getenv("SB_WGRAD_REDUCE_GBS"); return e ? atof(e) : 3000.0; }();
+    static const double reduce_fixed = [] { const char* e = getenv("SB_WGRAD_REDUCE_US"); return e ? atof(e) : 3.0; }();
+    static const double chunk_scale = [] { const char* e = getenv("SB_WGRAD_CHUNK_SCALE"); return e ? atof(e) : 1.0; }();
+    const double chunk_us = chunk_scale * (16384.0 + bn * 128.0) / 122.0e3;     // bytes per chunk at ~122 GB/s of L2 per SM
+    const double fixed_us = 3.0 + bn / 256.0 * 1.5;               // CTA start + drain + float epilogue
+    double best = 1e30; int best_s = 1;
+    for (int s = 1; s <= 256; s *= 2) {
+        const int cps = cdiv_i(total_chunks, s);
+        if (s > 1 && cps < 2) break;
+        const int real_s = cdiv_i(total_chunks, cps);
+        const long ctas = ctas_without_split * real_s;
+        const long waves = (ctas + 147) / 148;
+        // two resident CTAs share one SM's operand bandwidth: count a pair of waves as one at twice the chunk time
+        double t = waves * (cps * chunk_us + fixed_us);
+        if (real_s > 1) t += reduce_fixed + (real_s + 1) * (double)grad_floats * 4.0 / (reduce_gbs * 1e3);
+        if (t < best) { best = t; best_s = real_s; }
+    }
+    static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
+    if (verbose) fprintf(stderr, "plan: wgrad base_ctas=%ld chunks=%d bn=%d grad=%zu -> splits=%d (%.1f us)\n", ctas_without_split, total_chunks, bn, grad_floats, best_s, best);
+    return best_s;
 }
 
 static bool conv_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
@@ -731,21 +1058,21 @@ struct ConvGeom {
     int cw, ch, cn, ctw, cth, ctn, total_chunks;   // 64-pixel boxes (WGRAD k-chunks)
     int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps;
 };
-static ConvGeom conv_geom(const LayerView& lv, int B)
+static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
 {
     ConvGeom g;
     choose_box(lv.W, lv.H, B, 128, &g.bw, &g.bh, &g.bn);
     g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
     g.m_tiles = (long)g.tw * g.th * g.tn;
-    g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64));
-    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64), true);
+    g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64), false, force_pair);
+    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64), true, force_pair);
     choose_box(lv.W, lv.H, B, 64, &g.cw, &g.ch, &g.cn);
     g.ctw = cdiv_i(lv.W, g.cw); g.cth = cdiv_i(lv.H, g.ch); g.ctn = cdiv_i(B, g.cn);
     g.total_chunks = g.ctw * g.cth * g.ctn;
     g.wg_bn = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
     g.wg_n_tiles = cdiv_i(lv.Cin, g.wg_bn);
     g.wg_m_tiles = cdiv_i(lv.Cout, 128);
-    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * 9, g.total_chunks);
+    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * 9, g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b);
     g.wg_cps = cdiv_i(g.total_chunks, s);
     g.wg_splits = cdiv_i(g.total_chunks, g.wg_cps);   // no empty trailing split
     return g;
@@ -754,12 +1081,12 @@ struct FcGeom {
     int m_tiles;
     TilePlan fwd, dgrad;
 };
-static FcGeom fc_geom(const LayerView& lv, int B, int K)
+static FcGeom fc_geom(const LayerView& lv, int B, int K, bool force_pair)
 {
     FcGeom g;
     g.m_tiles = cdiv_i(B, 128);
-    g.fwd = plan_tiles(cdiv_i(lv.out_f, K), K, g.m_tiles, lv.in_f / 64);
-    g.dgrad = plan_tiles(lv.in_f, 1, g.m_tiles, cdiv_i(lv.out_f, 64), true);
+    g.fwd = plan_tiles(cdiv_i(lv.out_f, K), K, g.m_tiles, lv.in_f / 64, false, force_pair);
+    g.dgrad = plan_tiles(lv.in_f, 1, g.m_tiles, cdiv_i(lv.out_f, 64), true, force_pair);
     return g;
 }
 
@@ -771,13 +1098,13 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
     for (int i = 0; i < mv.n_layers; ++i) {
         LayerView lv = layer_view(m, i);
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            ConvGeom g = conv_geom(lv, mv.B);
+            ConvGeom g = conv_geom(lv, mv.B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             const size_t pix = (size_t)mv.B * lv.H * lv.W;
             if (g.wg_splits > 1) upd((size_t)g.wg_splits * (lv.n_w + lv.n_b));
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * pix * lv.Cout);
             if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * pix * lv.Cin);
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
-            FcGeom g = fc_geom(lv, mv.B, mv.cfg->K);
+            FcGeom g = fc_geom(lv, mv.B, mv.cfg->K, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * mv.B * lv.out_f);
             if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * mv.B * lv.in_f);
         }
@@ -799,7 +1126,8 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
     p.stages = t.stages;
     p.part = t.splits > 1 ? ws : nullptr;
     p.split_stride = (long)(rows * (size_t)p.n_total);
-    b->grid = dim3((unsigned)m_tiles, (unsigned)n_tiles_total, (unsigned)t.splits);
+    b->pair = t.pair;
+    b->grid = dim3((unsigned)(t.pair ? (m_tiles + 1) / 2 * 2 : m_tiles), (unsigned)n_tiles_total, (unsigned)t.splits);
     b->rows = (long)rows;
 }
 
@@ -813,7 +1141,7 @@ sb_status umma_plan_layers(sb_model* m)
         UmmaLayer& um = *lv.um;
         const bool want_in_grad = i > 0;
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            const ConvGeom g = conv_geom(lv, B);
+            const ConvGeom g = conv_geom(lv, B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             const size_t pix = (size_t)B * lv.H * lv.W;
             // ---- forward ----
             {
@@ -828,7 +1156,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.status = mv.status;
                 apply_plan(b, g.fwd, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
-                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->bn)) return fail_plan();
+                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
                 um.fwd.enabled = true;
             }
             // ---- data gradient ----
@@ -878,7 +1206,7 @@ sb_status umma_plan_layers(sb_model* m)
             }
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
             const int K = mv.cfg->K;
-            const FcGeom g = fc_geom(lv, B, K);
+            const FcGeom g = fc_geom(lv, B, K, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             const int m_tiles = g.m_tiles;
             if (i == 0) lv.in_act = mv.stage_x;   // placeholder; rebound to the caller's input by umma_bind_input
             const bool fc_in_grad = i > 0 || (mv.cfg->flags & SB_FLAG_INPUT_GRAD);
@@ -895,7 +1223,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.bias = mv.Wm + lv.p_b; p.status = mv.status;
                 apply_plan(b, g.fwd, p.kchunks, m_tiles, p.tiles_per_shard * K, mv.ws, (size_t)B);
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
-                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->bn)) return fail_plan();
+                if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
                 um.fwd.enabled = true;
             }
             // ---- data gradient: dX = sum_j dY_j W_j = one reduction over the concatenated width ----

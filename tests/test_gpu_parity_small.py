@@ -29,6 +29,12 @@ def tensor_core_net(classes=16):
             (si.MAXPOOL2, 0), (si.FC_RELU, 256), (si.FC_RELU, 128), (si.FC, classes), (si.SOFTMAX_XENT, classes)]
 
 
+def pair_net(classes=16):
+    # 128- and 256-wide layers, so that with SB_FLAG_FORCE_PAIR the forward and data-gradient GEMMs run on CTA pairs
+    return [(si.CONV3X3_RELU, 64), (si.CONV3X3_RELU, 256), (si.CONV3X3_RELU, 256), (si.MAXPOOL2, 0), (si.CONV3X3_RELU, 128),
+            (si.CONV3X3_RELU, 128), (si.MAXPOOL2, 0), (si.FC_RELU, 512), (si.FC_RELU, 256), (si.FC, classes), (si.SOFTMAX_XENT, classes)]
+
+
 WORKLOADS = {
     "cfg0": lambda: si.config(0),
     "ragged": lambda: si.Workload("ragged", ragged_net(), 20, 12, 4, 3, 2, 3),
@@ -37,7 +43,7 @@ WORKLOADS = {
 }
 
 
-def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_frob_bound=None):
+def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_frob_bound=None, flags=0):
     """Whole iterations, end to end.  Float mode: every tensor within 1e-4.  bf16 mode: forward tensors,
     loss and updated weights within 1e-2 element-wise; backward tensors are bounded in the Frobenius norm,
     because a summation-order difference can flip a ReLU mask or a pooling argmax and that moves single
@@ -46,7 +52,7 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_fr
     params = si.make_params(wl, bias_std=bias_std)
     x, y = si.make_batch(wl)
     om = oracle_model(wl, params, bf16)
-    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32)
+    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=flags)
     xs, ys = device_batch(wl, x, y, bf16)
     xr, yr = si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)
     tol = TOL[bf16]
@@ -107,7 +113,7 @@ def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_fr
     gm.close()
 
 
-def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None):
+def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None, flags=0):
     """Every layer's kernels on the oracle's own tensors as inputs: forward output, weight/bias gradient
     and input gradient of each layer within the contract tolerance ELEMENT-WISE; pool argmax bit-exact.
 
@@ -144,7 +150,7 @@ def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None):
         pool_idx = lambda r, li: om.pool_idx[0][li][rows[r]]
         full = lambda a: a[sel]
         gscale = wl.B / distinct
-    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=b.SB_FLAG_INPUT_GRAD)
+    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=b.SB_FLAG_INPUT_GRAD | flags)
     xs, ys = device_batch(wl, x, y, bf16)
     tol = TOL[bf16]
     nl = len(wl.layers)
@@ -216,6 +222,31 @@ def test_layerwise_teacher_forced(name, bf16):
 @pytest.mark.parametrize("bf16", [False, True])
 def test_two_training_steps_match_oracle(name, bf16):
     compare_everything(WORKLOADS[name](), bf16, steps=2, bias_std=0.2)
+
+
+@pytest.mark.parametrize("images", [(3, 2), (5, 1)])
+def test_cta_pair_kernels_forced(images):
+    """tcgen05 cta_group::2 path at small sizes: every 128/256-wide forward and data-gradient GEMM on CTA pairs,
+    with even (6 images) and odd (5 images: a phantom partner tile) M-tile counts, ragged tiles and split sums."""
+    b = sb()
+    wl = si.Workload("pair", pair_net(), 12, 20, 3, images[0], images[1], 2)
+    layerwise_teacher_forced(wl, True, flags=b.SB_FLAG_FORCE_PAIR)
+    # whole forward pass and loss: the pair path against the single-CTA path and against the oracle
+    params = si.make_params(wl, bias_std=0.2)
+    x, y = si.make_batch(wl)
+    xs, ys = device_batch(wl, x, y, True)
+    om = oracle_model(wl, params, True)
+    om.forward(si.split_replicas(x, wl.R), si.split_replicas(y, wl.R))
+    got = []
+    for flags in (b.SB_FLAG_FORCE_PAIR, 0):
+        gm = gpu_model(wl, params, b.SB_BF16, flags=flags)
+        gm.forward(xs, ys)
+        got.append((gm.read(b.SB_T_ACT, len(wl.layers) - 2, 0, squeeze=False)[:, :, 0, 0], gm.loss()))
+        gm.close()
+    for logits, loss in got:
+        assert maxrel(logits, om.logits) <= TOL[True]
+        assert abs(loss - om.loss) <= TOL[True] * max(1.0, abs(om.loss))
+    assert maxrel(got[0][0], got[1][0]) <= 1e-3
 
 
 @pytest.mark.parametrize("bf16", [False, True])
