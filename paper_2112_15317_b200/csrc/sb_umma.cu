@@ -996,7 +996,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         const int pfit = t.bn >= 256 ? 6 : 8;
         int pst = t.cps < pfit ? t.cps : pfit;
         const int ptwo = t.bn >= 256 ? 3 : 4;      // two resident CTAs per SM
-        if ((backward || fwd_too) && bwd_cohabit() && pst > ptwo) pst = ptwo;
+        if ((tiles * t.splits >= 296 || ((backward || fwd_too) && bwd_cohabit())) && pst > ptwo) pst = ptwo;
         t.stages = pst < 1 ? 1 : pst;
     }
     static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
