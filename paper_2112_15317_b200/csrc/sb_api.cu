@@ -416,7 +416,9 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
     char* d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
     const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
     const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
-    float* const ws_w = m->ws_wk[i % sb_model::MAX_WSTREAMS];   // this layer's weight-side scratch (fixed per layer)
+    // this layer's weight-side scratch: one region per weight stream, so two layers that share a region are
+    // ordered by the stream they share
+    float* const ws_w = m->ws_wk[m->n_wstreams > 0 ? i % m->n_wstreams : 0];
     switch (l.kind) {
     case SB_SOFTMAX_XENT:
         break;  // dZ was produced by the forward loss kernel
@@ -493,8 +495,13 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             const int nb = conv_in_wgrad_blocks(B, l.H, l.W);
             const size_t stride = l.n_w + l.n_b;
             L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
-            L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+            if (l.p_b == l.p_w + l.n_w) {
+                // the bias vector directly follows the weights in the gradient arena, as it does in a partial buffer
+                L_TRY("split_reduce", 0.0, (double)stride * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, stride, nb, st));
+            } else {
+                L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
+                L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+            }
         } else if (l.um.wgrad.enabled) {
             int S = 1;
             float* part = nullptr;
@@ -649,7 +656,7 @@ ModelView model_view(sb_model* m)
 {
     ModelView v{};
     v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
-    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) v.ws_wk[k] = m->ws_wk[k]; v.ws_floats = m->ws_floats; v.status = m->status;
+    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) v.ws_wk[k] = m->ws_wk[k]; v.ws_floats = m->ws_floats; v.n_wstreams = m->n_wstreams; v.status = m->status;
     v.input_grad = m->input_grad; v.x_tab = &m->x_tab; v.stage_x = m->stage_x;
     return v;
 }

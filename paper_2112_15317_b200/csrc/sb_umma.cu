@@ -51,6 +51,7 @@ struct UmmaParams {
     // WGRAD
     int m_total;          // rows of the weight gradient (Cout / out-features)
     int m_shards, m_tiles_per_shard;
+    int tap_group;        // WGRAD: filter taps per CTA: 1, or 3 (one filter row; Cin = 64, N tile = 3 x 64 columns)
     int splits, chunks_per_split, total_chunks;   // split of the reduction (k-iterations) over blockIdx.z
     int stages;           // depth of the shared-memory ring (<= MAX_STAGES)
     float* part;          // FWD/DGRAD with splits > 1: raw float partial sums [split][pixel][n_total]
@@ -183,8 +184,8 @@ constexpr int MAX_STAGES = 8;
 template <int MODE, int BN> struct Cfg {
     static constexpr int B_STAGE_BYTES = BN * 128;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int MAX_STAGES_FIT = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);   // what fits in 227 KB
-    static constexpr int TMEM_COLS = BN;
+    static constexpr int MAX_STAGES_FIT = (BN >= 256) ? 4 : (BN >= 192 ? 5 : (BN >= 128 ? 6 : 8));   // what fits in 227 KB
+    static constexpr int TMEM_COLS = BN == 192 ? 256 : BN;    // allocations are powers of two
     static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES; }
 };
 
@@ -300,10 +301,10 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     int m_idx = blockIdx.x, n_idx = blockIdx.y;
     int n0, n_hi;       // first output column of this tile and one past the last valid column
     if (MODE == MODE_WGRAD) {
-        tap_fixed = blockIdx.z / p.splits;
+        tap_fixed = (blockIdx.z / p.splits) * p.tap_group;   // first tap of this CTA's group
         split = blockIdx.z % p.splits;
         n0 = n_idx * BN;
-        n_hi = p.n_total;
+        n_hi = p.n_total;                                     // tap_group = 3: 3 x Cin (the taps' columns are adjacent)
     } else {
         const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
         const int lo = (int)(((long)sh * p.n_total) / p.shards), hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
@@ -329,7 +330,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int k_begin = split * p.chunks_per_split;
     const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
     const int n_iters = k_end - k_begin;
-    const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? 4 : 0);
+    const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? (p.tap_group == 3 ? 3 : 4) : 0);
 
     // Operand loads of the next k-iteration into ring slot `s` (executed by the producer thread, iterations in
     // order).  The iteration's coordinates are carried in counters, so the issue path has no integer division.
@@ -340,18 +341,27 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
     }
     const int wg_dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, wg_ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
+    // WGRAD with at most 64 gradient rows left in this tile: the second 64-row box of A would be all padding, so it
+    // is not fetched (accumulator rows 64.. then hold garbage that is never stored; MMA rows are independent)
+    const int a_boxes = (MODE == MODE_WGRAD && m0 + 64 >= m_hi) ? 1 : 2;
     auto issue_loads = [&](int it) {
         const int s = it % STAGES;
         uint8_t* sa = smem + s * C::STAGE_BYTES;
         uint8_t* sb = sa + A_STAGE_BYTES;
-        mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES);
+        mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES - (a_boxes == 2 ? 0u : 8192u));
         if (MODE == MODE_WGRAD) {
             // pixel chunk -> box origin; A = dy (two 64-channel boxes), B = shifted activations
             const int cw = ld_a * p.bw, ch = ld_b * p.bh, cn = ld_c * p.bn;
             tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
-            tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
+            if (a_boxes == 2) tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
+            if (BN == 192) {
+                // one filter row: the three taps' activation boxes are the same pixels shifted by -1, 0, +1 in w
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn);
+                for (int j = 0; j < 3; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], 0, cw + j - 1, ch + wg_dr, cn);
+            } else {
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn);
+            }
             if (++ld_a == p.tiles_w) { ld_a = 0; if (++ld_b == p.tiles_h) { ld_b = 0; ++ld_c; } }
         } else {
             const int kc = ld_a, tap = ld_b;
@@ -869,6 +879,7 @@ static cudaError_t launch_pair_mode(int bn, const UmmaOp& op, const UmmaParams& 
 template <int MODE>
 static cudaError_t launch_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
 {
+    if (MODE == MODE_WGRAD && bn == 192) return launch_one<MODE_WGRAD, 192>(op, p, grid, st);
     switch (bn) {
     case 64: return launch_one<MODE, 64>(op, p, grid, st);
     case 128: return launch_one<MODE, 128>(op, p, grid, st);
@@ -936,7 +947,7 @@ static bool bwd_cohabit()
     static const bool on = [] { const char* e = getenv("SB_BWD_COHABIT"); return !(e && e[0] == '0'); }();
     return on;
 }
-static int cohabit_stages(int bn) { return bn >= 256 ? 2 : (bn >= 128 ? 3 : 4); }
+static int cohabit_stages(int bn) { return bn >= 192 ? 2 : (bn >= 128 ? 3 : 4); }
 
 // Cost model behind the tile plan (micro-seconds, calibrated on per-CTA phase timings at VGG-16/CIFAR sizes):
 // a CTA costs ~3 us of fixed work (cold start, first loads, drain, epilogue) plus ~0.4 us per k-iteration (the
@@ -1056,7 +1067,7 @@ struct ConvGeom {
     long m_tiles;
     TilePlan fwd, dgrad;
     int cw, ch, cn, ctw, cth, ctn, total_chunks;   // 64-pixel boxes (WGRAD k-chunks)
-    int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps;
+    int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps, wg_tap_group;
 };
 static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
 {
@@ -1072,7 +1083,12 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
     g.wg_bn = lv.Cin >= 256 ? 256 : (lv.Cin >= 128 ? 128 : 64);
     g.wg_n_tiles = cdiv_i(lv.Cin, g.wg_bn);
     g.wg_m_tiles = cdiv_i(lv.Cout, 128);
-    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * 9, g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b);
+    // 64 input channels: one CTA takes a whole filter row (three taps = 192 adjacent gradient columns), so the dy
+    // tile is fetched once per three taps (SB_WGRAD_TAPS=1 restores one tap per CTA)
+    static const bool taps1 = [] { const char* e = getenv("SB_WGRAD_TAPS"); return e && e[0] == '1'; }();
+    g.wg_tap_group = (lv.Cin == 64 && !taps1) ? 3 : 1;
+    if (g.wg_tap_group == 3) g.wg_bn = 192;
+    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * (9 / g.wg_tap_group), g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b);
     g.wg_cps = cdiv_i(g.total_chunks, s);
     g.wg_splits = cdiv_i(g.total_chunks, g.wg_cps);   // no empty trailing split
     return g;
@@ -1184,21 +1200,25 @@ sb_status umma_plan_layers(sb_model* m)
                 p.mode = MODE_WGRAD; p.ntaps = 9; p.bw = g.cw; p.bh = g.ch; p.bn = g.cn; p.W = lv.W; p.H = lv.H; p.N = B;
                 p.tiles_w = g.ctw; p.tiles_h = g.cth; p.tiles_n = g.ctn;
                 p.total_chunks = g.total_chunks;
-                p.w_cols = lv.Cin; p.n_total = lv.Cin; p.shards = 1; p.tiles_per_shard = 1;
+                p.w_cols = lv.Cin; p.n_total = lv.Cin * g.wg_tap_group; p.shards = 1; p.tiles_per_shard = 1;
                 p.m_total = lv.Cout; p.m_shards = 1; p.m_tiles_per_shard = g.wg_m_tiles;
+                p.tap_group = g.wg_tap_group;
                 b->bn = g.wg_bn;
                 p.splits = g.wg_splits;
                 p.chunks_per_split = g.wg_cps;
-                p.stages = g.wg_cps < (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8)) ? g.wg_cps : (b->bn >= 256 ? 4 : (b->bn >= 128 ? 6 : 8));
+                {
+                    const int fit = b->bn >= 256 ? 4 : (b->bn >= 192 ? 5 : (b->bn >= 128 ? 6 : 8));
+                    p.stages = g.wg_cps < fit ? g.wg_cps : fit;
+                }
                 if (bwd_cohabit() && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
                 // the bias gradient rides along: in the parameter arena the bias vector directly follows the
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
                 p.split_stride = (long)(lv.n_w + lv.n_b);
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
-                p.out = p.splits > 1 ? (void*)mv.ws_wk[i % 4] : (void*)(mv.Gm + lv.p_w);
+                p.out = p.splits > 1 ? (void*)mv.ws_wk[mv.n_wstreams > 0 ? i % mv.n_wstreams : 0] : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
-                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 * p.splits));
+                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 / p.tap_group * p.splits));
                 if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
                 if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch, g.cn)) return fail_plan();
@@ -1255,6 +1275,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.total_chunks = p.tiles_n;
                 p.w_cols = lv.in_f; p.n_total = lv.in_f; p.shards = 1; p.tiles_per_shard = 1;
                 p.m_total = lv.out_f; p.m_shards = K; p.m_tiles_per_shard = cdiv_i(cdiv_i(lv.out_f, K), 128);
+                p.tap_group = 1;
                 b->bn = lv.in_f >= 256 ? 256 : (lv.in_f >= 128 ? 128 : 64);
                 const int n_tiles = cdiv_i(lv.in_f, b->bn);
                 p.splits = 1; p.chunks_per_split = p.total_chunks;
