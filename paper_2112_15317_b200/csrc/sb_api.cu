@@ -331,7 +331,8 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.in = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
         a.w = wts; a.bias = m->Wm + l.p_b; a.out = l.act; a.mask_ref = nullptr;
         a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 0; a.relu = 1;
-        if (l.thin_input) L_TRY("conv_in_fwd", flops, bytes, launch_conv_in_fwd(a, bf, st));
+        if (l.thin_input && l.um.conv_in) L_TRY("conv_in_fwd_umma", flops, bytes, launch_conv_in_fwd_umma(a, m->status, st));
+        else if (l.thin_input) L_TRY("conv_in_fwd", flops, bytes, launch_conv_in_fwd(a, bf, st));
         else L_TRY("conv_fwd_simt", flops, bytes, launch_conv_simt(a, bf, st));
         break;
     }
@@ -492,9 +493,12 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             WgradSimtArgs a{};
             a.x = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
             a.dy = l.dact; a.part = ws_w; a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout;
-            const int nb = conv_in_wgrad_blocks(B, l.H, l.W);
+            const int nb = l.um.conv_in ? conv_in_umma_wgrad_blocks((long)B * l.H * l.W) : conv_in_wgrad_blocks(B, l.H, l.W);
             const size_t stride = l.n_w + l.n_b;
-            L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
+            if (l.um.conv_in)
+                L_TRY("conv_in_wgrad_umma", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad_umma(a, l.um.wgrad.mapA, m->status, st));
+            else
+                L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
             if (l.p_b == l.p_w + l.n_w) {
                 // the bias vector directly follows the weights in the gradient arena, as it does in a partial buffer
                 L_TRY("split_reduce", 0.0, (double)stride * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, stride, nb, st));

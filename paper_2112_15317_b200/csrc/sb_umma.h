@@ -16,6 +16,7 @@ struct UmmaOp {
 };
 struct UmmaLayer {
     UmmaOp fwd, dgrad, wgrad;
+    bool conv_in = false;                // input-layer conv on the tensor cores (wgrad.mapA then maps this layer's dy)
     const void* bound_input = nullptr;   // layer 0 only: the input buffer the tensor maps currently point at
 };
 
@@ -65,6 +66,13 @@ sb_status umma_bind_input(sb_model* m, const void* x);
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
+
+// Input-layer convolution (1, 3 or 4 input channels, 64 output channels, bf16) on the tensor cores.
+bool conv_in_umma_supported(int Cin, int Cout);
+// Partial buffers the weight-gradient kernel writes ([blocks][Cout*9*Cin + Cout] floats, reduced in block order).
+int conv_in_umma_wgrad_blocks(long npix);
+cudaError_t launch_conv_in_fwd_umma(const ConvSimtArgs& a, uint32_t* status, cudaStream_t st);
+cudaError_t launch_conv_in_wgrad_umma(const WgradSimtArgs& a, const CUtensorMap& mapDy, uint32_t* status, cudaStream_t st);
 
 const char* umma_last_error();
 // Debug aid: when set to a device buffer of 1024*16 uint64, every tensor-core CTA (first 1024 of a launch)
