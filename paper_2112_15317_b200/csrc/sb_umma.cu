@@ -842,17 +842,23 @@ static bool bwd_cohabit()
 }
 static int cohabit_stages(int bn) { return bn >= 192 ? 2 : (bn >= 128 ? 3 : 4); }
 
-// Cost model behind the tile plan (micro-seconds, calibrated on per-CTA phase timings at VGG-16/CIFAR sizes):
-// a CTA costs ~3 us of fixed work (cold start, first loads, drain, epilogue) plus ~0.4 us per k-iteration (the
-// operand ring is latency / L2-bandwidth bound, almost independently of the tile width); CTAs run in waves of one
-// per SM (two when the ring is shallow); a split reduction adds a second kernel (~8 us with its launch gap).
+// Cost model behind the tile plan (micro-seconds), fitted to a sweep of N-tile width x split count over the
+// VGG-16 / CIFAR layers (isolated launches, 5 us of event overhead removed):
+//   * one k-iteration of a CTA that has an SM to itself costs ~0.45 us whatever the tile width (0.46 / 0.45 / 0.43
+//     for 256 / 128 / 64 columns): the 128-row A tile, the barrier round trip and the four MMAs dominate;
+//   * two CTAs sharing an SM each run at ~1/1.6 of that rate;
+//   * a CTA carries ~3 us of fixed work (start, first loads, drain, epilogue);
+//   * a split reduction costs a second kernel (~4 us) plus ~0.5 us per MB of float partial sums written and read back
+//     (8.4 MB -> 7 us, 16.8 MB -> 9 us, 33.5 MB -> 27 us measured).
 static double plan_cost(int bn, int s, int n_cols_per_shard, int shards, long m_tiles, int k_iters)
 {
     const long ctas = m_tiles * cdiv_i(n_cols_per_shard, bn) * shards * s;
     const double per_sm = (bn < 256 && ctas >= 296) ? 2.0 : 1.0;
     const double waves = (double)cdiv_i(ctas, (long)(148 * per_sm));
-    const double t_iter = bn >= 256 ? 0.41 : (bn >= 128 ? 0.37 : 0.33);
-    return waves * (cdiv_i(k_iters, s) * t_iter * (per_sm > 1.0 ? 1.6 : 1.0) + 3.0) + (s > 1 ? 8.0 : 0.0);
+    const double t_iter = bn >= 256 ? 0.46 : (bn >= 128 ? 0.45 : 0.43);
+    const double partial_mb = (double)s * (double)m_tiles * 128.0 * (double)n_cols_per_shard * shards * 4.0 / 1.0e6;
+    const double mb_us = 0.5;
+    return waves * (cdiv_i(k_iters, s) * t_iter * (per_sm > 1.0 ? 1.6 : 1.0) + 3.0) + (s > 1 ? 4.0 + mb_us * partial_mb : 0.0);
 }
 static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward, bool force_pair)
 {
@@ -886,6 +892,24 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     }
     static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
     if ((backward || fwd_too) && bwd_cohabit() && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
+    // Grids of more than one CTA per SM: measured, the co-residency of CTAs (their set-up, first loads and
+    // epilogues overlap one another's main loops) is worth more than ring depth -- the 1024-CTA 64-wide layer runs
+    // 28 us with 2 stages (4 CTAs per SM) against 37 us with 4 and 60 us with 8; beyond 3 stages no layer gains.
+    // So the ring is cut down until the CTAs the grid asks for fit side by side (shared memory and TMEM columns
+    // permitting), but never below a double buffer.  SB_STAGE_RULE=legacy keeps the older rule above.
+    static const bool legacy_stages = [] { const char* e = getenv("SB_STAGE_RULE"); return e && e[0] == 'l'; }();
+    static const int min_stages = [] { const char* e = getenv("SB_MIN_STAGES"); int k = e ? atoi(e) : 2; return k < 1 ? 1 : k; }();
+    if (!legacy_stages) {
+        const long ctas = tiles * t.splits;
+        long want = (ctas + 147) / 148;
+        if (want > 512 / t.bn) want = 512 / t.bn;
+        if (want > 8) want = 8;
+        const int stage_bytes = 16384 + t.bn * 128;
+        for (; want > 1; --want) {
+            const int st_res = (int)((224 * 1024 / want - 3 * 1024) / stage_bytes);
+            if (st_res >= min_stages) { if (st > st_res) st = st_res; break; }
+        }
+    }
     t.stages = st < 1 ? 1 : st;
     // CTA pairs: half the weight-side operand per CTA (a smaller stage, so a deeper ring).  Measured at VGG-16 /
     // ImageNet sizes the pair kernel is 1.2-1.3x faster where the N tile is 256 wide and the grid fills the
