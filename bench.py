@@ -268,7 +268,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": wl.name, "network": "VGG-16 (13 conv3x3 + 3 FC), 32x32x3 inputs, 10 classes",
+        "config": {"workload": wl.name, "network": f"{sum(1 for k, _ in wl.layers if k == si.CONV3X3_RELU)} conv3x3 + {sum(1 for k, _ in wl.layers if k in (si.FC_RELU, si.FC))} FC, {wl.H}x{wl.W}x{wl.C} inputs, {wl.classes} classes",
                    "global_batch": imgs, "batch_per_gpu": wl.B, "R": wl.R, "K": wl.K, "b": wl.b,
                    "precision": "bf16 operands, fp32 accumulate, fp32 master weights",
                    "launch": "one CUDA graph per step (sb_graph_step); per-kernel times from a separate event-bracketed pass",

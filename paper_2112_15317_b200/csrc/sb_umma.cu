@@ -320,28 +320,40 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_WGRAD, MODE != MODE_FWD);
-            bool ok = true;
-            for (int it = 0; it < n_iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-                if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
-                if (tlog && it == 0) tlog[2] = (unsigned long long)clock64();            // first operands landed
-                if (tlog && it == n_iters - 1) tlog[3] = (unsigned long long)clock64();  // last operands landed
-                tc_fence_after();
-                const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    // K-major: 16 elements = 32 bytes along the row; MN-major: 16 k-rows = 2048 bytes
-                    const uint64_t ad = (MODE == MODE_WGRAD) ? make_desc(sa + kk * 2048, 8192) : make_desc(sa + kk * 32, 16);
-                    const uint64_t bd = (MODE == MODE_FWD) ? make_desc(sb + kk * 32, 16) : make_desc(sb + kk * 2048, 8192);
-                    umma_bf16(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
-                }
-                umma_commit(&empty[s]);      // stage reusable once these MMAs have read it
+        // The whole warp walks the ring in lock-step (barrier waits, descriptor words and ring counters are the same
+        // in every lane, so they live in uniform registers); one elected lane issues the MMAs and the commits.
+        constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_WGRAD, MODE != MODE_FWD);
+        const uint32_t elected = elect_one() ? 1u : 0u;
+        const uint32_t sa0 = smem_u32(smem);
+        // K-major: 16 elements = 32 bytes along the row; MN-major: 16 k-rows = 2048 bytes
+        const uint64_t dA0 = (MODE == MODE_WGRAD) ? make_desc(sa0, 8192) : make_desc(sa0, 16);
+        const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(sa0 + A_STAGE_BYTES, 16) : make_desc(sa0 + A_STAGE_BYTES, 8192);
+        const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
+        const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
+        constexpr uint32_t A_STEP = ((MODE == MODE_WGRAD) ? 2048u : 32u) >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
+        constexpr uint32_t STAGE16 = (uint32_t)C::STAGE_BYTES >> 4;     // the address field counts 16-byte units
+        int s = 0;
+        uint32_t ph = 0, off = 0;
+        bool ok = true;
+        for (int it = 0; it < n_iters; ++it) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
+            if (!ok) {
+                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
+                break;
             }
-            if (ok) umma_commit(acc_full);   // accumulator complete
+            if (tlog && lane == 0 && it == 0) tlog[2] = (unsigned long long)clock64();            // first operands landed
+            if (tlog && lane == 0 && it == n_iters - 1) tlog[3] = (unsigned long long)clock64();  // last operands landed
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_lohi(tmem_base, a_lo0 + off + kk * A_STEP, a_hi, b_lo0 + off + kk * B_STEP, b_hi, idesc, (it > 0 || kk > 0) ? 1u : 0u, elected);
+            if (elected) umma_commit(&empty[s]);      // stage reusable once these MMAs have read it
+            __syncwarp();
+            ++s; off += STAGE16;
+            if (s == STAGES) { s = 0; off = 0; ph ^= 1u; }
         }
+        if (ok && elected) umma_commit(acc_full);   // accumulator complete
+        __syncwarp();
     } else {
         // =========================== epilogue ===================================================
         const int q = warp % 4;               // TMEM lane quadrant of this warp
@@ -588,26 +600,39 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && leader) {
+        if (leader) {
+            // (converged warp, elected issue: see the single-CTA kernel)
             constexpr uint32_t idesc = make_idesc(BN, 0, MODE != MODE_FWD, 256);
+            const uint32_t elected = elect_one() ? 1u : 0u;
             // the MMA addresses both accumulators with one TMEM address: the pair must have been given the same columns
             bool ok = ld_cluster_u32(map_to_cta(smem_u32(tmem_slot), 1)) == tmem_base;
-            if (!ok) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_PAIR_TMEM); }
+            if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_PAIR_TMEM); }
+            const uint32_t sa0 = smem_u32(smem);
+            const uint64_t dA0 = make_desc(sa0, 16);
+            const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(sa0 + A_STAGE_BYTES, 16) : make_desc(sa0 + A_STAGE_BYTES, 8192);
+            const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
+            constexpr uint32_t A_STEP = 32u >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
+            constexpr uint32_t STAGE16 = (uint32_t)C::STAGE_BYTES >> 4;
+            int s = 0;
+            uint32_t ph = 0, off = 0;
             for (int it = 0; it < n_iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-                if (!mbar_wait(&full[s], ph)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); ok = false; break; }
-                tc_fence_after();
-                const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES), sb = sa + A_STAGE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ad = make_desc(sa + kk * 32, 16);
-                    const uint64_t bd = (MODE == MODE_FWD) ? make_desc(sb + kk * 32, 16) : make_desc(sb + kk * 2048, 8192);
-                    umma_bf16_pair(tmem_base, ad, bd, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
+                if (!ok) {
+                    if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
+                    break;
                 }
-                umma_commit_pair(&empty[s]);
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_pair_lohi(tmem_base, a_lo0 + off + kk * A_STEP, a_hi, b_lo0 + off + kk * B_STEP, b_hi, idesc, (it > 0 || kk > 0) ? 1u : 0u, elected);
+                if (elected) umma_commit_pair(&empty[s]);
+                __syncwarp();
+                ++s; off += STAGE16;
+                if (s == STAGES) { s = 0; off = 0; ph ^= 1u; }
             }
-            if (ok) umma_commit_pair(acc_full);
+            if (ok && elected) umma_commit_pair(acc_full);
+            __syncwarp();
         }
     } else {
         const int q = warp % 4;
@@ -916,7 +941,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     // machine, slower for 128-wide tiles and for grids of less than a wave (two cluster barriers of fixed cost).
     // SB_PAIR=0 turns it off, SB_PAIR_MIN_CTAS moves the grid-size threshold.
     static const bool pair_on = [] { const char* e = getenv("SB_PAIR"); return !(e && e[0] == '0'); }();
-    static const long pair_min_ctas = [] { const char* e = getenv("SB_PAIR_MIN_CTAS"); return e ? atol(e) : 148L; }();
+    static const long pair_min_ctas = [] { const char* e = getenv("SB_PAIR_MIN_CTAS"); return e ? atol(e) : 1L; }();
     t.pair = 0;
     // (SB_FLAG_FORCE_PAIR: every 128- or 256-wide tile, whatever the grid -- for tests at small sizes)
     if ((pair_on && t.bn == 256 && m_tiles % 2 == 0 && tiles * t.splits >= pair_min_ctas) || (force_pair && t.bn >= 128)) {
