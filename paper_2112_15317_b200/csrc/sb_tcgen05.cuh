@@ -57,6 +57,21 @@ __device__ __forceinline__ void tma_load_4d(const CUtensorMap* map, void* dst, u
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// Predicated forms for a converged producer warp: every lane executes the slot, the lane with `elected` != 0 issues.
+__device__ __forceinline__ void mbar_expect_tx_el(uint32_t bar_saddr, uint32_t bytes, uint32_t elected)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
+                 ::"r"(bar_saddr), "r"(bytes), "r"(elected) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_el(const CUtensorMap* map, uint32_t dst_saddr, uint32_t bar_saddr, int c0, int c1, int c2, int c3,
+                                               uint32_t elected)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+        "@q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n\t}"
+        ::"r"(dst_saddr), "l"(map), "r"(bar_saddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");

@@ -237,23 +237,26 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     // WGRAD with at most 64 gradient rows left in this tile: the second 64-row box of A would be all padding, so it
     // is not fetched (accumulator rows 64.. then hold garbage that is never stored; MMA rows are independent)
     const int a_boxes = (MODE == MODE_WGRAD && m0 + 64 >= m_hi) ? 1 : 2;
-    auto issue_loads = [&](int it) {
-        const int s = it % STAGES;
-        uint8_t* sa = smem + s * C::STAGE_BYTES;
-        uint8_t* sb = sa + A_STAGE_BYTES;
-        mbar_expect_tx(&full[s], (uint32_t)C::STAGE_BYTES - (a_boxes == 2 ? 0u : 8192u));
+    // (executed by the whole producer warp in lock-step: every value below is the same in all lanes, the lane with
+    // el != 0 issues; ring slot and smem offset are carried in counters)
+    int ld_s = 0;
+    uint32_t ld_off = 0;
+    const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(&full[0]);
+    auto issue_loads = [&](uint32_t el) {
+        const uint32_t sa = smem0 + ld_off, sb = sa + A_STAGE_BYTES, bar = full0 + 8u * (uint32_t)ld_s;
+        mbar_expect_tx_el(bar, (uint32_t)C::STAGE_BYTES - (a_boxes == 2 ? 0u : 8192u), el);
         if (MODE == MODE_WGRAD) {
             // pixel chunk -> box origin; A = dy (two 64-channel boxes), B = shifted activations
             const int cw = ld_a * p.bw, ch = ld_b * p.bh, cn = ld_c * p.bn;
-            tma_load_4d(&mapA, sa, &full[s], m0, cw, ch, cn);
-            if (a_boxes == 2) tma_load_4d(&mapA, sa + 8192, &full[s], m0 + 64, cw, ch, cn);
+            tma_load_4d_el(&mapA, sa, bar, m0, cw, ch, cn, el);
+            if (a_boxes == 2) tma_load_4d_el(&mapA, sa + 8192, bar, m0 + 64, cw, ch, cn, el);
             if (BN == 192) {
                 // one filter row: the three taps' activation boxes are the same pixels shifted by -1, 0, +1 in w
 #pragma unroll
-                for (int j = 0; j < 3; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], 0, cw + j - 1, ch + wg_dr, cn);
+                for (int j = 0; j < 3; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, 0, cw + j - 1, ch + wg_dr, cn, el);
             } else {
 #pragma unroll
-                for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn);
+                for (int j = 0; j < BN / 64; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn, el);
             }
             if (++ld_a == p.tiles_w) { ld_a = 0; if (++ld_b == p.tiles_h) { ld_b = 0; ++ld_c; } }
         } else {
@@ -261,42 +264,49 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             int dr = 0, ds = 0;
             if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
             if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
-            tma_load_4d(&mapA, sa, &full[s], kc * 64, pw0 + ds, ph0 + dr, pn0);
+            tma_load_4d_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
             if (MODE == MODE_FWD) {
-                tma_load_4d(&mapB, sb, &full[s], tap * p.w_cols + kc * 64, n0, 0, 0);
+                tma_load_4d_el(&mapB, sb, bar, tap * p.w_cols + kc * 64, n0, 0, 0, el);
             } else {
 #pragma unroll
-                for (int j = 0; j < BN / 64; ++j) tma_load_4d(&mapB, sb + j * 8192, &full[s], tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0);
+                for (int j = 0; j < BN / 64; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, tap * p.w_cols + n0 + 64 * j, kc * 64, 0, 0, el);
             }
             if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
         }
+        ++ld_s; ld_off += (uint32_t)C::STAGE_BYTES;
+        if (ld_s == STAGES) { ld_s = 0; ld_off = 0; }
     };
     const int preloaded = n_iters < STAGES ? n_iters : STAGES;
 
     // ---- one-time setup -----------------------------------------------------------------------
     // (programmatic dependent launch: everything up to pdl_wait() touches only shared memory and TMEM, so it
     // may run while the kernel this one depends on is still finishing)
-    if (threadIdx.x == 0) {
-        // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
-        mbar_init(acc_full, 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (tlog) tlog[8] = (unsigned long long)clock64();    // barriers initialised
+    uint32_t prod_el = 0;
+    if (warp == 0) {
+        if (lane == 0) {
+            // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
+            for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
+            mbar_init(acc_full, 1);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            if (tlog) tlog[8] = (unsigned long long)clock64();    // barriers initialised
+        }
+        __syncwarp();
         pdl_wait();
         pdl_trigger();
-        if (tlog) tlog[9] = (unsigned long long)clock64();    // predecessor kernel complete
-        // The first ring-full of loads needs nothing but the barriers this thread has just initialised: start
-        // them now, so that their latency overlaps the TMEM allocation and the rest of the set-up.
-        for (int it = 0; it < preloaded; ++it) issue_loads(it);
-        if (tlog) tlog[10] = (unsigned long long)clock64();   // first ring of loads issued
+        if (tlog && lane == 0) tlog[9] = (unsigned long long)clock64();    // predecessor kernel complete
+        // The first ring-full of loads needs nothing but the barriers just initialised: start them now, so that
+        // their latency overlaps the TMEM allocation and the rest of the set-up.
+        prod_el = elect_one() ? 1u : 0u;
+        for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
+        if (tlog && lane == 0) tlog[10] = (unsigned long long)clock64();   // first ring of loads issued
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, C::TMEM_COLS);
         tmem_relinquish();
         if (tlog && lane == 0) tlog[11] = (unsigned long long)clock64();   // TMEM allocated
     }
-    if (threadIdx.x != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
+    if (warp != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
     if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
         for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
     }
@@ -309,15 +319,20 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
-        if (lane == 0) {
-            for (int it = preloaded; it < n_iters; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-                if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
-                if (*abort_flag) break;
-                issue_loads(it);
+        // the whole warp in lock-step; slot `ws` is free once the MMAs that read it have completed
+        int ws = 0;
+        uint32_t wph = 0;
+        for (int it = preloaded; it < n_iters; ++it) {
+            const bool got = __all_sync(0xffffffffu, mbar_wait(&empty[ws], wph) ? 1 : 0) != 0;
+            if (!got) {
+                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+                break;
             }
+            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
+            issue_loads(prod_el);
+            if (++ws == STAGES) { ws = 0; wph ^= 1u; }
         }
+        __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
         // The whole warp walks the ring in lock-step (barrier waits, descriptor words and ring counters are the same
@@ -466,6 +481,15 @@ __device__ __forceinline__ void tma_load_4d_pair(const CUtensorMap* map, void* d
         ::"r"(smem_u32(dst)), "l"(map), "r"(bar_caddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_4d_pair_el(const CUtensorMap* map, uint32_t dst_saddr, uint32_t bar_caddr, int c0, int c1, int c2, int c3,
+                                                    uint32_t elected)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+        "@q cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n\t}"
+        ::"r"(dst_saddr), "l"(map), "r"(bar_caddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
@@ -541,24 +565,28 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     int ld_a = k_begin % p.kchunks, ld_b = k_begin / p.kchunks;   // (k-chunk, tap) of the next load
     const int nb0 = n0 + (int)rank * (BN / 2);                     // first B column this CTA fetches
     const uint32_t full0_leader = map_to_cta(smem_u32(&full[0]), 0);
-    auto issue_loads = [&](int it) {
-        const int s = it % STAGES;
-        uint8_t* sa = smem + s * C::STAGE_BYTES;
-        uint8_t* sb = sa + A_STAGE_BYTES;
-        const uint32_t bar = full0_leader + (uint32_t)s * 8u;
-        if (leader) mbar_expect_tx(&full[s], 2u * (uint32_t)C::STAGE_BYTES);
+    // (whole producer warp in lock-step, elected issue: see the single-CTA kernel)
+    int ld_s = 0;
+    uint32_t ld_off = 0;
+    const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(&full[0]);
+    auto issue_loads = [&](uint32_t el) {
+        const uint32_t sa = smem0 + ld_off, sb = sa + A_STAGE_BYTES;
+        const uint32_t bar = full0_leader + (uint32_t)ld_s * 8u;
+        if (leader) mbar_expect_tx_el(full0 + 8u * (uint32_t)ld_s, 2u * (uint32_t)C::STAGE_BYTES, el);
         const int kc = ld_a, tap = ld_b;
         int dr = 0, ds = 0;
         if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
         if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
-        tma_load_4d_pair(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0);
+        tma_load_4d_pair_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
         if (MODE == MODE_FWD) {
-            tma_load_4d_pair(&mapB, sb, bar, tap * p.w_cols + kc * 64, nb0, 0, 0);     // box of BN/2 rows
+            tma_load_4d_pair_el(&mapB, sb, bar, tap * p.w_cols + kc * 64, nb0, 0, 0, el);     // box of BN/2 rows
         } else {
 #pragma unroll
-            for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair(&mapB, sb + j * 8192, bar, tap * p.w_cols + nb0 + 64 * j, kc * 64, 0, 0);
+            for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair_el(&mapB, sb + j * 8192, bar, tap * p.w_cols + nb0 + 64 * j, kc * 64, 0, 0, el);
         }
         if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
+        ++ld_s; ld_off += (uint32_t)C::STAGE_BYTES;
+        if (ld_s == STAGES) { ld_s = 0; ld_off = 0; }
     };
     const int preloaded = n_iters < STAGES ? n_iters : STAGES;
 
@@ -570,16 +598,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     cluster_sync_all();    // both CTAs' barriers exist before any copy or commit can signal them
-    if (threadIdx.x == 0) {
+    uint32_t prod_el = 0;
+    if (warp == 0) {
         pdl_wait();
         pdl_trigger();
-        for (int it = 0; it < preloaded; ++it) issue_loads(it);
+        prod_el = elect_one() ? 1u : 0u;
+        for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
     }
     if (warp == 1) {
         tmem_alloc_pair(tmem_slot, C::TMEM_COLS);
         tmem_relinquish_pair();
     }
-    if (threadIdx.x != 0) pdl_wait();
+    if (warp != 0) pdl_wait();
     if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
         for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
     }
@@ -590,15 +620,19 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int it = preloaded; it < n_iters; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-                if (!mbar_wait(&empty[s], ph ^ 1u)) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); break; }
-                if (*abort_flag) break;
-                issue_loads(it);
+        int ws = 0;
+        uint32_t wph = 0;
+        for (int it = preloaded; it < n_iters; ++it) {
+            const bool got = __all_sync(0xffffffffu, mbar_wait(&empty[ws], wph) ? 1 : 0) != 0;
+            if (!got) {
+                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+                break;
             }
+            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
+            issue_loads(prod_el);
+            if (++ws == STAGES) { ws = 0; wph ^= 1u; }
         }
+        __syncwarp();
     } else if (warp == 1) {
         if (leader) {
             // (converged warp, elected issue: see the single-CTA kernel)
