@@ -75,15 +75,15 @@ struct sb_model {
     float *Wm = nullptr, *Vm = nullptr, *Gm = nullptr;
     __nv_bfloat16* Sm = nullptr;
     float* ws = nullptr;    // scratch of the data-side kernels (split partial sums of forward / data gradient)
-    float* ws_wk[4] = {nullptr, nullptr, nullptr, nullptr};   // one weight-side scratch region per weight stream
+    float* ws_wk[8] = {};   // one weight-side scratch region per weight stream
     float* ws_w = nullptr;  // scratch of the weight-side kernels (split partial sums of weight / bias gradients), so that
                             // the two sides can run concurrently in the backward pass
     size_t ws_floats = 0;
     // backward-pass concurrency: weight-gradient work runs on a second stream, ordered by events
-    static constexpr int MAX_WSTREAMS = 4;
+    static constexpr int MAX_WSTREAMS = 8;
     int n_wstreams = 0;                          // weight-gradient work of layer i runs on wstreams[i % n_wstreams]
-    cudaStream_t wstreams[MAX_WSTREAMS] = {nullptr, nullptr, nullptr, nullptr};
-    cudaEvent_t ev_wjoin[MAX_WSTREAMS] = {nullptr, nullptr, nullptr, nullptr};
+    cudaStream_t wstreams[MAX_WSTREAMS] = {};
+    cudaEvent_t ev_wjoin[MAX_WSTREAMS] = {};
     cudaStream_t ustream = nullptr;   // parameter updates folded into the backward pass
     cudaEvent_t ev_join = nullptr, ev_ujoin = nullptr;
     std::vector<cudaEvent_t> ev_ready;   // one per layer: "the gradient w.r.t. this layer's output is ready"
@@ -708,7 +708,7 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     if (!(one && one[0] == '1')) {
         // second stream + ordering events for the backward pass (host objects; no device memory)
         const char* nws = getenv("SB_WSTREAMS");
-        m->n_wstreams = nws ? atoi(nws) : 3;
+        m->n_wstreams = nws ? atoi(nws) : 4;
         if (m->n_wstreams < 1) m->n_wstreams = 1;
         if (m->n_wstreams > sb_model::MAX_WSTREAMS) m->n_wstreams = sb_model::MAX_WSTREAMS;
         bool ok_ = true;
@@ -797,11 +797,13 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
     const bool two_streams = m->n_wstreams > 0 && !m->profiling && !m->debug_sync;
     const bool fuse = fuse_update && two_streams;
     if (updated) *updated = fuse;
+    unsigned used_streams = 0;   // weight streams that received work in this pass (only those are joined)
     for (int i = m->n_layers - 1; i >= 0; --i) {
         Layer& l = m->L[i];
         const bool has_params = l.kind == SB_CONV3X3_RELU || l.kind == SB_FC_RELU || l.kind == SB_FC;
         if (two_streams && has_params) {
             cudaStream_t wst = m->wstreams[i % m->n_wstreams];
+            used_streams |= 1u << (i % m->n_wstreams);
             CU_TRY(cudaEventRecord(m->ev_ready[i], st));
             CU_TRY(cudaStreamWaitEvent(wst, m->ev_ready[i], 0));
             sb_status s = backward_layer(m, i, wst, SIDE_W);
@@ -830,6 +832,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
     }
     if (two_streams) {
         for (int k = 0; k < m->n_wstreams; ++k) {
+            if (!(used_streams & (1u << k))) continue;
             CU_TRY(cudaEventRecord(m->ev_wjoin[k], m->wstreams[k]));
             CU_TRY(cudaStreamWaitEvent(st, m->ev_wjoin[k], 0));
         }

@@ -28,7 +28,7 @@ struct ModelView {
     float *Wm, *Gm;
     __nv_bfloat16* Sm;
     float* ws;      // data-side scratch
-    float* ws_wk[4];  // weight-side scratch regions, one per weight stream: layer i uses ws_wk[i % n_wstreams]
+    float* ws_wk[8];  // weight-side scratch regions, one per weight stream: layer i uses ws_wk[i % n_wstreams]
     int n_wstreams;   // 0: everything runs on the caller's stream (region 0)
     size_t ws_floats;
     uint32_t* status;
