@@ -903,8 +903,9 @@ static int cohabit_stages(int bn) { return bn >= 192 ? 2 : (bn >= 128 ? 3 : 4); 
 
 // Cost model behind the tile plan (micro-seconds), fitted to a sweep of N-tile width x split count over the
 // VGG-16 / CIFAR layers (isolated launches, 5 us of event overhead removed):
-//   * one k-iteration of a CTA that has an SM to itself costs ~0.45 us whatever the tile width (0.46 / 0.45 / 0.43
-//     for 256 / 128 / 64 columns): the 128-row A tile, the barrier round trip and the four MMAs dominate;
+//   * one k-iteration of a CTA that has an SM to itself costs 0.38 / 0.315 / 0.245 us for 256 / 128 / 64 columns
+//     (operand bytes through the SM's L2 port; before the MMAs were issued from a converged warp it was ~0.45 us
+//     whatever the width);
 //   * two CTAs sharing an SM each run at ~1/1.6 of that rate;
 //   * a CTA carries ~3 us of fixed work (start, first loads, drain, epilogue);
 //   * a split reduction costs a second kernel (~4 us) plus ~0.5 us per MB of float partial sums written and read back
@@ -914,7 +915,7 @@ static double plan_cost(int bn, int s, int n_cols_per_shard, int shards, long m_
     const long ctas = m_tiles * cdiv_i(n_cols_per_shard, bn) * shards * s;
     const double per_sm = (bn < 256 && ctas >= 296) ? 2.0 : 1.0;
     const double waves = (double)cdiv_i(ctas, (long)(148 * per_sm));
-    const double t_iter = bn >= 256 ? 0.46 : (bn >= 128 ? 0.45 : 0.43);
+    const double t_iter = bn >= 256 ? 0.38 : (bn >= 128 ? 0.315 : 0.245);
     const double partial_mb = (double)s * (double)m_tiles * 128.0 * (double)n_cols_per_shard * shards * 4.0 / 1.0e6;
     const double mb_us = 0.5;
     return waves * (cdiv_i(k_iters, s) * t_iter * (per_sm > 1.0 ? 1.6 : 1.0) + 3.0) + (s > 1 ? 4.0 + mb_us * partial_mb : 0.0);

@@ -246,7 +246,8 @@ def test_cta_pair_kernels_forced(images):
     for logits, loss in got:
         assert maxrel(logits, om.logits) <= TOL[True]
         assert abs(loss - om.loss) <= TOL[True] * max(1.0, abs(om.loss))
-    assert maxrel(got[0][0], got[1][0]) <= 1e-3
+    # the two plans may split reductions differently, so their bf16 roundings differ: same bound as against the oracle
+    assert maxrel(got[0][0], got[1][0]) <= TOL[True]
 
 
 @pytest.mark.parametrize("bf16", [False, True])
