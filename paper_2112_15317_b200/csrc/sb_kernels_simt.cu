@@ -603,7 +603,8 @@ __device__ __forceinline__ void sgd_apply(float4& ww, float4& vv, const float4& 
 }
 // Grid-stride blocks with four independent 16-byte triples in flight per thread.  (Measured: the update does not
 // hide behind the backward pass's tensor-core kernels whatever the grid size -- 16, 8, 4, 2 or 1 blocks per SM
-// all give the same step time -- because both are bound by the SM <-> L2 path; SB_SGD_BLOCKS_PER_SM changes the grid.)
+// all give the same step time, and confined to 32 or 64 blocks the update overlaps but is itself too slow;
+// streaming (evict-first) loads and stores make no difference either.  SB_SGD_BLOCKS_PER_SM changes the grid.)
 template <bool SHADOW>
 __global__ void __launch_bounds__(256)
 sgd_kernel(float4* __restrict__ w, float4* __restrict__ v, const float4* __restrict__ g,
@@ -615,19 +616,19 @@ sgd_kernel(float4* __restrict__ w, float4* __restrict__ v, const float4* __restr
     for (; i + 3 * stride < n4; i += 4 * stride) {
         float4 ww[4], vv[4], gg[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { ww[u] = w[i + u * stride]; vv[u] = v[i + u * stride]; gg[u] = __ldg(g + i + u * stride); }
+        for (int u = 0; u < 4; ++u) { ww[u] = __ldcs(w + i + u * stride); vv[u] = __ldcs(v + i + u * stride); gg[u] = __ldcs(g + i + u * stride); }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             sgd_apply<SHADOW>(ww[u], vv[u], gg[u], lr, mu, SHADOW ? shadow + i + u * stride : nullptr);
-            v[i + u * stride] = vv[u];
-            w[i + u * stride] = ww[u];
+            __stcs(v + i + u * stride, vv[u]);
+            __stcs(w + i + u * stride, ww[u]);
         }
     }
     for (; i < n4; i += stride) {
-        float4 ww = w[i], vv = v[i], gg = __ldg(g + i);
+        float4 ww = __ldcs(w + i), vv = __ldcs(v + i), gg = __ldcs(g + i);
         sgd_apply<SHADOW>(ww, vv, gg, lr, mu, SHADOW ? shadow + i : nullptr);
-        v[i] = vv;
-        w[i] = ww;
+        __stcs(v + i, vv);
+        __stcs(w + i, ww);
     }
 }
 cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n, float lr, float mu, cudaStream_t st)
