@@ -997,12 +997,13 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
 // a small cost model: waves x (chunks per CTA x per-chunk operand time + fixed CTA cost) for the GEMM
 // plus, when split, (S + 1) gradient copies through HBM/L2 and one more launch for the reduce.
 // SB_WGRAD_SPLITS=legacy restores the older rule (fill 148 CTAs, at least 4 chunks per CTA).
-static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_t grad_floats)
+static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_t grad_floats, double* cost_out = nullptr)
 {
     static const bool legacy = [] { const char* e = getenv("SB_WGRAD_SPLITS"); return e && e[0] == 'l'; }();
     if (legacy) {
         int s = 1;
         while (ctas_without_split * s < 148 && total_chunks / (s * 2) >= 4) s *= 2;
+        if (cost_out) *cost_out = bn >= 256 ? 0.0 : 1.0;    // legacy: widest tile
         return s;
     }
     static const double reduce_gbs = [] { const char* e = getenv("SB_WGRAD_REDUCE_GBS"); return e ? atof(e) : 3000.0; }();
@@ -1024,6 +1025,7 @@ static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_
     }
     static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
     if (verbose) fprintf(stderr, "plan: wgrad base_ctas=%ld chunks=%d bn=%d grad=%zu -> splits=%d (%.1f us)\n", ctas_without_split, total_chunks, bn, grad_floats, best_s, best);
+    if (cost_out) *cost_out = best;
     return best_s;
 }
 
@@ -1065,7 +1067,17 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
     static const bool taps1 = [] { const char* e = getenv("SB_WGRAD_TAPS"); return e && e[0] == '1'; }();
     g.wg_tap_group = (lv.Cin == 64 && !taps1) ? 3 : 1;
     if (g.wg_tap_group == 3) g.wg_bn = 192;
-    const int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * (9 / g.wg_tap_group), g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b);
+    double cost = 0.0;
+    int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * (9 / g.wg_tap_group), g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b, &cost);
+    // a narrower N tile doubles the CTAs of a grid that leaves SMs idle (e.g. 512 channels at 4x4: 72 CTAs of 256
+    // columns against 144 of 128): take it when the same model says it is faster (SB_WGRAD_NARROW=0 keeps the widest)
+    static const bool narrow = [] { const char* e = getenv("SB_WGRAD_NARROW"); return !(e && e[0] == '0'); }();
+    if (narrow && g.wg_tap_group == 1 && g.wg_bn == 256) {
+        double cost2 = 0.0;
+        const int n2 = cdiv_i(lv.Cin, 128);
+        const int s2 = wgrad_splits((long)g.wg_m_tiles * n2 * 9, g.total_chunks, 128, (size_t)lv.n_w + lv.n_b, &cost2);
+        if (cost2 < cost) { g.wg_bn = 128; g.wg_n_tiles = n2; s = s2; }
+    }
     g.wg_cps = cdiv_i(g.total_chunks, s);
     g.wg_splits = cdiv_i(g.total_chunks, g.wg_cps);   // no empty trailing split
     return g;
