@@ -27,6 +27,13 @@ Readings taken where the paper is silent (stated in full in the design notes): o
 pass over all R*b rows instead of K sub-iterations with gradients divided by K; R and K are
 independent; every FC layer is sharded with boundaries floor(j*out/K).
 
+step_modulo() is the other schedule, the paper's own [Modulo Layer]: the FC stack runs K
+sub-iterations on b/K examples of every replica and updates the FC parameters after each with
+gradients divided by K; the conv stack back-propagates once, after the K-th.  It is not equal to the
+unpartitioned step for K > 1, so its parity is against this algorithm only; it is pinned by K = 1
+(identical to step()), by lr = 0 (gradients add up to the synchronous ones), by re-composition
+out of forward()/backward() calls on the sub-batches, and by the paper's worked B = 2, K = 2 example.
+
 `bf16=True` switches on the mixed-precision contract of the CUDA library: operands of every
 contraction (stored activations, stored activation gradients, the weight copies used in the
 contractions) are rounded to bfloat16 (round-to-nearest-even) at the points where the library
@@ -366,6 +373,132 @@ class OracleModel:
         self.backward()
         self.sgd_step(lr, mu)
         return loss
+
+    # ---- the modulo layer's own schedule [Modulo Layer] ------------------------------------
+    def modulo_rows(self, k):
+        """Rows (in gather order g = r*b + i) that sub-iteration k sends through the FC stack: every replica's k-th
+        slice of b/K local examples, replica-major -- row p of the sub-batch comes from replica p // (b/K)."""
+        bk = self.b // self.K
+        return np.array([r * self.b + k * bk + i for r in range(self.R) for i in range(bk)], dtype=np.int64)
+
+    def step_modulo(self, x_list, labels_list, lr, mu):
+        """One iteration in the paper's schedule: the conv stack runs once on the whole local batches, then the FC
+        stack runs K sub-iterations, each on a distinct b/K examples of every replica; the FC parameters are
+        updated after every sub-iteration with gradients divided by K, the conv parameters once at the end.
+
+        Normalisation: every row's loss gradient is (softmax - onehot)/B, B = R*b.  For the FC parameters that is
+        the mean over the sub-batch divided by K (the paper's compensation); for the conv stack it is what the
+        synchronous iteration uses, so with K = 1 this is step().  Returns the mean of the B row losses (each
+        taken with the FC parameters of its own sub-iteration)."""
+        P, R, b, K = self.P, self.R, self.b, self.K
+        assert b % K == 0, "the modulo schedule needs b divisible by K"
+        nl = len(self.layers)
+        first_fc = next(i for i, (k, _) in enumerate(self.layers) if k in (FC_RELU, FC))
+        assert first_fc > 0, "the modulo layer sits between a conv-side stack and the FC stack"
+        self.first_fc = first_fc
+        # 1. conv stack forward, all rows, once (as in forward())
+        self.x_in = [self._q(np.array(x, self.dt)) for x in x_list]
+        self.conv_out = [[None] * nl for _ in range(R)]
+        self.pool_idx = [[None] * nl for _ in range(R)]
+        feats = []
+        for r in range(R):
+            a = self.x_in[r]
+            for li in range(first_fc):
+                kind, _ = self.layers[li]
+                if kind == CONV:
+                    a = self._q(P.conv_fwd(a, self._q(self.params[li]["w"]), self.params[li]["b"], relu=True))
+                else:
+                    a, self.pool_idx[r][li] = P.pool_fwd(a)
+                self.conv_out[r][li] = a
+            feats.append(a.reshape(b, -1))
+        self.feat_shape = a.shape
+        D = feats[0].shape[1]
+        X_all = np.empty((self.B, D), self.dt)
+        labels_all = np.empty((self.B,), np.int32)
+        for g in range(self.B):
+            X_all[g, :] = feats[g // b][g % b, :]
+            labels_all[g] = labels_list[g // b][g % b]
+        dX_all = np.zeros((self.B, D), self.dt)
+        row_loss_all = np.zeros((self.B,), self.dt)
+        self.mod_fc_grads = []            # per sub-iteration: the FC gradients that were applied (for tests)
+        # 2. K sub-iterations of the FC stack
+        for k in range(K):
+            rows = self.modulo_rows(k)
+            X = np.ascontiguousarray(X_all[rows])
+            labels = np.ascontiguousarray(labels_all[rows])
+            fc_in, fc_out = {}, {}
+            for li in range(first_fc, nl):
+                kind, out = self.layers[li]
+                if kind in (FC_RELU, FC):
+                    fc_in[li] = X
+                    cb = self.bounds[li]
+                    Y = np.empty((X.shape[0], out), self.dt)
+                    for j in range(K):
+                        sh = self.params[li][j]
+                        Y[:, cb[j]:cb[j + 1]] = P.fc_fwd(X, self._q(sh["w"]), sh["b"], relu=(kind == FC_RELU))
+                    if kind == FC_RELU:
+                        Y = self._q(Y)
+                    fc_out[li] = Y
+                    X = Y
+                else:
+                    row_loss, dZ = P.softmax_xent(X, labels, 1.0 / self.B)
+                    row_loss_all[rows] = row_loss
+            dY = self._q(dZ)
+            g_k = {}
+            for li in range(nl - 2, first_fc - 1, -1):
+                cb = self.bounds[li]
+                Xin = fc_in[li]
+                g = []
+                dX = np.zeros_like(Xin)
+                for j in range(K):
+                    sh = self.params[li][j]
+                    dWj, dbj, dXj = P.fc_bwd(Xin, self._q(sh["w"]), np.ascontiguousarray(dY[:, cb[j]:cb[j + 1]]))
+                    g.append({"w": dWj, "b": dbj})
+                    dX = dX + dXj
+                g_k[li] = g
+                if li > first_fc:
+                    dY = self._q(dX * (fc_out[li - 1] > 0))
+            dX_all[rows] = dX
+            self.mod_fc_grads.append(g_k)
+            for li, g in g_k.items():     # FC update of this sub-iteration
+                self.grads[li] = g
+                for j in range(K):
+                    for key in ("w", "b"):
+                        P.sgd(self.params[li][j][key], self.mom[li][j][key], g[j][key], lr, mu)
+        self.row_loss = row_loss_all
+        self.loss = self.dt(np.sum(row_loss_all, dtype=self.dt) / self.dt(self.B))
+        # 3. modulo layer backward + conv stack backward on all rows, DP reduce, conv update (as in backward())
+        dfeat = [np.empty((b,) + self.feat_shape[1:], self.dt) for _ in range(R)]
+        for g_ in range(self.B):
+            dfeat[g_ // b][g_ % b] = dX_all[g_].reshape(self.feat_shape[1:])
+        self.mod_dfeat = dfeat
+        rep_grads = []
+        for r in range(R):
+            d = dfeat[r]
+            gr = {}
+            for li in range(first_fc - 1, -1, -1):
+                kind, _ = self.layers[li]
+                below = self.conv_out[r][li - 1] if li > 0 else self.x_in[r]
+                if kind == POOL:
+                    d = P.pool_bwd(self._q(d), self.pool_idx[r][li])
+                else:
+                    d = self._q(d * (self.conv_out[r][li] > 0))
+                    dw, db = P.conv_wgrad(below, d)
+                    gr[li] = {"w": dw, "b": db}
+                    if li > 0:
+                        d = P.conv_dgrad(d, self._q(self.params[li]["w"]))
+            rep_grads.append(gr)
+        for li in range(first_fc):
+            if self.layers[li][0] == CONV:
+                gw = np.zeros_like(self.params[li]["w"])
+                gb = np.zeros_like(self.params[li]["b"])
+                for r in range(R):
+                    gw = gw + rep_grads[r][li]["w"]
+                    gb = gb + rep_grads[r][li]["b"]
+                self.grads[li] = {"w": gw, "b": gb}
+                for key in ("w", "b"):
+                    P.sgd(self.params[li][key], self.mom[li][key], self.grads[li][key], lr, mu)
+        return self.loss
 
 
 def from_workload(wl, real="float", bf16=False, loss_B=None) -> OracleModel:
