@@ -38,6 +38,10 @@ import sb_inputs as si  # noqa: E402
 METRIC = "training images/sec (VGG-16 CIFAR shape)"
 UNIT = "images/s"
 LR, MU = 0.01, 0.9
+# ImageNet-shape configuration: He-normal weights without normalisation layers make plain SGD at 0.01 diverge on the
+# synthetic batch (loss 11 -> 18 -> 274 in three steps); the step time does not depend on the values, but a finite loss is
+# reported, so that configuration trains at a smaller rate
+LR_BY_CONFIG = {3: 1.0e-4}
 
 
 def peaks():
@@ -163,6 +167,7 @@ def run_ours(args):
     from paper_2112_15317_b200 import binding as sb
 
     wl = workload(args.config)
+    lr = LR_BY_CONFIG.get(args.config, LR)
     params = si.make_params(wl)
     x, y = si.make_batch(wl, seed=si.SEED_DATA + rank)
     m = sb.Model.from_workload(wl, precision=sb.SB_BF16, device=f"cuda:{local}")
@@ -177,12 +182,12 @@ def run_ours(args):
     torch.cuda.set_stream(side)
 
     def step():
-        m.graph_step(xs, ys, LR, MU)
+        m.graph_step(xs, ys, lr, MU)
 
     def step_eager():
         m.forward(xs, ys)
         m.backward()
-        m.sgd_step(LR, MU)
+        m.sgd_step(lr, MU)
 
     def barrier():
         torch.cuda.synchronize()
@@ -209,11 +214,11 @@ def run_ours(args):
 
     # end to end through the host-buffer entry point
     for _ in range(max(1, min(args.warmup, 3))):
-        m.train_step_host(hx, hy, LR, MU)
+        m.train_step_host(hx, hy, lr, MU)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        m.train_step_host(hx, hy, LR, MU)
+        m.train_step_host(hx, hy, lr, MU)
     torch.cuda.synchronize()
     ms_e2e = (time.perf_counter() - t0) * 1e3
     barrier()
@@ -269,7 +274,7 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": wl.name, "network": f"{sum(1 for k, _ in wl.layers if k == si.CONV3X3_RELU)} conv3x3 + {sum(1 for k, _ in wl.layers if k in (si.FC_RELU, si.FC))} FC, {wl.H}x{wl.W}x{wl.C} inputs, {wl.classes} classes",
-                   "global_batch": imgs, "batch_per_gpu": wl.B, "R": wl.R, "K": wl.K, "b": wl.b,
+                   "global_batch": imgs, "batch_per_gpu": wl.B, "R": wl.R, "K": wl.K, "b": wl.b, "lr": lr, "momentum": MU,
                    "precision": "bf16 operands, fp32 accumulate, fp32 master weights",
                    "launch": "one CUDA graph per step (sb_graph_step); per-kernel times from a separate event-bracketed pass",
                    "l2": "per-step working set (activations+gradients+weights, >1 GB) exceeds the 126 MB L2; no flush",

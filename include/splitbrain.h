@@ -70,9 +70,11 @@ enum {
     SB_FLAG_INPUT_GRAD = 1,  /* also compute the gradient w.r.t. the network input (layer 0 dgrad) */
     SB_FLAG_FORCE_SIMT = 2,  /* use the CUDA-core kernels for every layer (cross-check / debugging) */
     SB_FLAG_PROFILE_LAYERS = 4, /* sb_profile_end reports one entry per (kernel class, layer): "name#layer" */
-    SB_FLAG_FORCE_PAIR = 8   /* run every forward / data-gradient GEMM whose N tile is 128 or 256 wide on CTA pairs
+    SB_FLAG_FORCE_PAIR = 8,  /* run every forward / data-gradient GEMM whose N tile is 128 or 256 wide on CTA pairs
                                 (tcgen05 cta_group::2), whatever the grid size; by default the planner uses pairs only
                                 where they pay (256-wide tiles, at least one wave of CTAs) */
+    SB_FLAG_MODULO_SCHEDULE = 16 /* reserve the buffers and plan the sub-batch kernels sb_modulo_step needs
+                                (batch_per_replica must be a multiple of K; the first layer must not be an FC layer) */
 };
 
 typedef struct {
@@ -155,6 +157,23 @@ sb_status sb_backward(sb_model* m, void* stream);
  * v <- momentum*v + g ; w <- w - lr*v ; in SB_BF16 mode also refreshes the bf16 weight copies.
  */
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream);
+
+/*
+ * One iteration in the modulo layer's own schedule [Modulo Layer: "The stateful scheduling for the K iterations"]:
+ * the conv-side layers run forward once on all R*b rows; the FC stack then runs K sub-iterations, sub-iteration k
+ * on the k-th slice of b/K examples of every replica (inside a sub-batch the row at position p belongs to replica
+ * p / (b/K)); every row's loss gradient is (softmax - onehot)/(R*b), which for the FC parameters is the mean over
+ * the sub-batch divided by K, and the FC parameters take an SGD-momentum update after every sub-iteration, so K
+ * per iteration; after the K-th the conv-side layers back-propagate once over all rows and take their update.
+ * With K = 1 the result is that of sb_forward + sb_backward + sb_sgd_step; with K > 1 it is a different
+ * algorithm (the FC weights move between sub-iterations).  sb_loss afterwards returns the mean of the R*b row
+ * losses.  Needs SB_FLAG_MODULO_SCHEDULE at creation (SB_ERR_STATE otherwise).  Arguments as for sb_forward /
+ * sb_sgd_step; runs on `stream`, asynchronous.  Afterwards SB_T_ROW_LOSS and the FC activation tensors hold their
+ * rows in sub-iteration order (position k*(R*b/K) + r*(b/K) + i = example k*(b/K) + i of replica r), the FC
+ * activations as left by the sub-iteration that wrote them; sb_backward needs a new sb_forward.
+ */
+sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum,
+                         void* stream);
 
 /*
  * One whole iteration (sb_forward + sb_backward + sb_sgd_step on device-resident inputs) replayed as a CUDA

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(HERE, "libsplitbrain.so")
 SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
 SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT = 1, 2, 3, 4, 5
-SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR = 1, 2, 4, 8
+SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE = 1, 2, 4, 8, 16
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
 SB_DT_F32, SB_DT_BF16, SB_DT_U8, SB_DT_I32 = 0, 1, 2, 3
@@ -62,6 +62,7 @@ def _load():
         "sb_forward": [c_void_p, P(c_void_p), P(c_void_p), c_void_p],
         "sb_backward": [c_void_p, c_void_p],
         "sb_graph_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
+        "sb_modulo_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
         "sb_sgd_step": [c_void_p, c_float, c_float, c_void_p],
         "sb_loss": [c_void_p, c_void_p, P(c_float)],
         "sb_train_step_host": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p, P(c_float)],
@@ -99,6 +100,7 @@ sb_model_destroy = _lib.sb_model_destroy
 sb_forward = _lib.sb_forward
 sb_backward = _lib.sb_backward
 sb_graph_step = _lib.sb_graph_step
+sb_modulo_step = _lib.sb_modulo_step
 sb_sgd_step = _lib.sb_sgd_step
 sb_loss = _lib.sb_loss
 sb_train_step_host = _lib.sb_train_step_host
@@ -229,6 +231,11 @@ class Model:
         """forward + backward + sgd_step as one CUDA-graph launch (captured by the library on the second call)."""
         xp, lp = self._ptr_arrays(xs, labels)
         _check(sb_graph_step(self.h, xp, lp, c_float(lr), c_float(momentum), self._stream()))
+
+    def modulo_step(self, xs, labels, lr, momentum):
+        """One iteration in the modulo layer's sub-iteration schedule (model created with SB_FLAG_MODULO_SCHEDULE)."""
+        xp, lp = self._ptr_arrays(xs, labels)
+        _check(sb_modulo_step(self.h, xp, lp, c_float(lr), c_float(momentum), self._stream()))
 
     def sgd_step(self, lr, momentum):
         _check(sb_sgd_step(self.h, c_float(lr), c_float(momentum), self._stream()))

@@ -57,6 +57,10 @@ struct Layer {
     bool narrow = false;                        // FC with out <= 16: dedicated narrow kernels
     int act_dt = SB_DT_F32;
     UmmaLayer um;                               // tensor-core plan of this layer (tcgen05 path)
+    // Sub-batch copies of the first FC layer (modulo schedule): where its input comes from and where its input
+    // gradient goes, instead of the layer below's buffers
+    char* in_override = nullptr;
+    char* dbelow_override = nullptr;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -97,6 +101,14 @@ struct sb_model {
     char* input_grad = nullptr;
     PtrTab x_tab{}, label_tab{};
     bool have_x = false, have_labels = false, have_fwd = false;
+    // Modulo schedule (SB_FLAG_MODULO_SCHEDULE): the FC input / its gradient in sub-iteration order, the labels in
+    // that order, and per sub-iteration a copy of the layer table whose FC layers address B/K rows of the buffers.
+    // While a sub-iteration runs, L and B are those of the sub-batch (sub_active, sub_row0 say so).
+    char *mod_x = nullptr, *mod_dx = nullptr;
+    int32_t* mod_labels = nullptr;
+    std::vector<std::vector<Layer>> mod_L;
+    bool sub_active = false;
+    int sub_row0 = 0, full_B = 0;
     int64_t launches = 0, last_step_launches = 0;
     // CUDA graphs of a whole iteration (sb_graph_step, sb_train_step_host), re-captured when their key changes
     struct StepGraph {
@@ -268,6 +280,15 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     m->stage_x = take(B * m->in_per_img * m->esz);
     m->stage_labels = (int32_t*)take(B * 4);
     m->input_grad = (cfg->flags & SB_FLAG_INPUT_GRAD) ? take(B * m->in_per_img * m->esz) : nullptr;
+    if (cfg->flags & SB_FLAG_MODULO_SCHEDULE) {
+        if (m->first_fc == 0) return fail(SB_ERR_UNSUPPORTED, "the modulo schedule needs a conv-side stack below the FC stack");
+        if (cfg->batch_per_replica % cfg->K != 0) return fail(SB_ERR_UNSUPPORTED, "the modulo schedule needs batch_per_replica divisible by K");
+        const size_t D = (size_t)m->L[m->first_fc].in_f;
+        if ((D * m->esz) % 16 != 0) return fail(SB_ERR_UNSUPPORTED, "the modulo schedule needs feature rows of a multiple of 16 bytes");
+        m->mod_x = take(B * D * m->esz);
+        m->mod_dx = take(B * D * m->esz);
+        m->mod_labels = (int32_t*)take(B * sizeof(int32_t));
+    }
     *total = off;
     return SB_OK;
 }
@@ -306,7 +327,7 @@ inline int shard_lo(int j, int total, int K) { return (int)(((long)j * total) / 
     } while (0)
 
 // Which buffer holds the input of layer i: the previous layer's output, or the caller's images.
-inline const char* layer_input(const sb_model* m, int i) { return i > 0 ? m->L[i - 1].act : nullptr; }
+inline const char* layer_input(const sb_model* m, int i) { return m->L[i].in_override ? m->L[i].in_override : (i > 0 ? m->L[i - 1].act : nullptr); }
 
 sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
 {
@@ -395,6 +416,15 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.logits = (const float*)fc.act; a.labels = m->label_tab; a.b_per_rep = b;
         a.row_loss = m->row_loss; a.loss = m->loss; a.dZ = fc.dact; a.counter = m->counter;
         a.B = B; a.C = l.out;
+        if (m->sub_active) {
+            // rows [sub_row0, sub_row0 + B) of the full batch, labels already in sub-iteration order; every row's
+            // gradient carries 1/full_B and the mean loss is taken over all rows written so far and before
+            a.labels = PtrTab{};
+            a.labels.p[0] = m->mod_labels + m->sub_row0;
+            a.b_per_rep = B;
+            a.row_loss = m->row_loss + m->sub_row0;
+            a.scale_B = m->full_B; a.loss_base = m->row_loss; a.loss_rows = m->full_B;
+        }
         L_TRY("softmax_xent", 0.0, (double)B * l.out * (4.0 + e) + 8.0 * B, launch_softmax_xent(a, bf, st));
         break;
     }
@@ -414,7 +444,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
     const double e = (double)m->esz;
     const bool want_in_grad = i > 0 || (m->cfg.flags & SB_FLAG_INPUT_GRAD);
     // where the gradient w.r.t. this layer's input goes, and whether the layer below applied a ReLU
-    char* d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
+    char* d_below = l.dbelow_override ? l.dbelow_override : (i > 0 ? m->L[i - 1].dact : m->input_grad);
     const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
     const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
     // this layer's weight-side scratch: one region per weight stream, so two layers that share a region are
@@ -435,7 +465,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             a.dY = l.dact; a.dW = m->Gm + l.p_w; a.db = m->Gm + l.p_b; a.B = B; a.in_f = l.in_f; a.out_f = l.out_f;
             if (part & SIDE_W) L_TRY("fc_narrow_wgrad", flops, act_bytes + (double)l.n_w * 4.0, launch_fc_narrow(a, bf, st));
             if (want_in_grad && (part & SIDE_D)) {
-                a.pass = 2; a.W = wts; a.ref = below_relu ? m->L[i - 1].act : nullptr; a.dX = d_below;
+                a.pass = 2; a.W = wts; a.ref = below_relu ? layer_input(m, i) : nullptr; a.dX = d_below;
                 L_TRY("fc_narrow_dgrad", flops, act_bytes + (double)l.n_w * e + (below_relu ? (double)B * l.in_f * e : 0.0), launch_fc_narrow(a, bf, st));
             }
             break;
@@ -468,7 +498,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
                 a.B = wts; a.sBn = 1; a.sBk = l.in_f;
                 a.M = B; a.N = l.in_f; a.K = l.out_f;
                 a.epi = EPI_MASK; a.C = d_below; a.ldc = l.in_f;
-                a.ref = below_relu ? m->L[i - 1].act : nullptr; a.ldref = l.in_f;
+                a.ref = below_relu ? layer_input(m, i) : nullptr; a.ldref = l.in_f;
                 a.shard_dim = 2; a.shards = m->cfg.K;
                 L_TRY("fc_dgrad_simt", flops, bytes, launch_gemm_simt(a, bf, st));
             }
@@ -671,8 +701,8 @@ LayerView layer_view(sb_model* m, int i)
     v.kind = l.kind; v.H = l.H; v.W = l.W; v.Cin = l.Cin; v.Cout = l.Cout; v.in_f = l.in_f; v.out_f = l.out_f; v.relu = l.relu;
     v.p_w = l.p_w; v.p_b = l.p_b; v.n_w = l.n_w; v.n_b = l.n_b;
     v.act = l.act; v.dact = l.dact; v.um = &l.um;
-    v.in_act = i > 0 ? m->L[i - 1].act : nullptr;
-    v.d_below = i > 0 ? m->L[i - 1].dact : m->input_grad;
+    v.in_act = l.in_override ? l.in_override : (i > 0 ? m->L[i - 1].act : nullptr);
+    v.d_below = l.dbelow_override ? l.dbelow_override : (i > 0 ? m->L[i - 1].dact : m->input_grad);
     v.below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
     return v;
 }
@@ -730,8 +760,37 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     cudaError_t e = cudaMemset(arena, 0, need);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }
-    s = umma_plan_layers(m);
+    s = umma_plan_layers(m, 0);
     if (s != SB_OK) { delete m; return fail(s, "tensor-core planning failed: %s", umma_last_error()); }
+    if (m->cfg.flags & SB_FLAG_MODULO_SCHEDULE) {
+        // One layer table per sub-iteration: its FC layers address rows [k*B/K, (k+1)*B/K) of the same buffers, the
+        // first of them reads / writes the permuted feature buffers; their tensor-core ops are planned for B/K rows.
+        const int K = m->cfg.K, Bk = m->B / K;
+        const size_t D = (size_t)m->L[m->first_fc].in_f;
+        m->full_B = m->B;
+        for (int k = 0; k < K; ++k) {
+            std::vector<Layer> Lk = m->L;
+            const size_t row0 = (size_t)k * Bk;
+            for (int i = m->first_fc; i < m->n_layers; ++i) {
+                Layer& l = Lk[i];
+                if (l.kind != SB_FC_RELU && l.kind != SB_FC) continue;
+                l.act += row0 * l.out_per_img * (l.act_dt == SB_DT_F32 ? 4 : m->esz);
+                l.dact += row0 * l.out_per_img * m->esz;
+                l.um = UmmaLayer{};
+            }
+            Lk[m->first_fc].in_override = m->mod_x + row0 * D * m->esz;
+            Lk[m->first_fc].dbelow_override = m->mod_dx + row0 * D * m->esz;
+            m->mod_L.push_back(std::move(Lk));
+        }
+        for (int k = 0; k < K && s == SB_OK; ++k) {
+            std::swap(m->L, m->mod_L[k]);
+            m->B = Bk;
+            s = umma_plan_layers(m, m->first_fc);
+            m->B = m->full_B;
+            std::swap(m->L, m->mod_L[k]);
+        }
+        if (s != SB_OK) { delete m; return fail(s, "tensor-core planning of the sub-batches failed: %s", umma_last_error()); }
+    }
     *out = m;
     return SB_OK;
 }
@@ -862,6 +921,62 @@ static sb_status whole_step(sb_model* m, const void* const* x, const int32_t* co
     if (s != SB_OK) return s;
     if (!updated) s = sb_sgd_step(m, lr, mu, stream);
     return s;
+}
+
+// One iteration in the modulo layer's own schedule [Modulo Layer]: the conv-side stack runs forward once on all
+// R*b rows; the modulo layer copies the feature rows into sub-iteration order (replica r's k-th slice of b/K rows
+// -> rows k*B/K + r*b/K ...); the FC stack then runs K sub-iterations (forward, loss with 1/B per row, backward,
+// SGD update of the FC parameters), each on B/K rows; the input gradients are copied back into row order and the
+// conv-side stack back-propagates once and takes its update.  Everything runs on the caller's stream.
+sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (!(m->cfg.flags & SB_FLAG_MODULO_SCHEDULE)) return fail(SB_ERR_STATE, "the model was created without SB_FLAG_MODULO_SCHEDULE");
+    if (!x || !labels) return fail(SB_ERR_INVALID_ARG, "x or labels is null");
+    if (m->sub_active) return fail(SB_ERR_STATE, "a sub-iteration is in progress");
+    cudaStream_t st = (cudaStream_t)stream;
+    sb_status s = set_inputs(m, x, labels);
+    if (s != SB_OK) return s;
+    m->launches = 0;
+    const int ff = m->first_fc, K = m->cfg.K, R = m->cfg.R, b = m->cfg.batch_per_replica, Bk = m->B / K;
+    const size_t D = (size_t)m->L[ff].in_f;
+    for (int i = 0; i < ff; ++i) {
+        s = forward_layer(m, i, st);
+        if (s != SB_OK) return s;
+    }
+    m->cur_layer = ff;
+    {
+        ModuloCopyArgs a{m->L[ff - 1].act, m->mod_x, D * m->esz, R, b, K, 0, &m->label_tab, m->mod_labels};
+        L_TRY("modulo_gather", 0.0, 2.0 * m->B * D * m->esz, launch_modulo_copy(a, st));
+    }
+    const size_t fc_off = m->L[ff].p_w, fc_cnt = m->P - fc_off;
+    for (int k = 0; k < K; ++k) {
+        std::swap(m->L, m->mod_L[k]);
+        m->B = Bk; m->sub_active = true; m->sub_row0 = k * Bk;
+        s = SB_OK;
+        for (int i = ff; i < m->n_layers && s == SB_OK; ++i) s = forward_layer(m, i, st);
+        for (int i = m->n_layers - 1; i >= ff && s == SB_OK; --i) s = backward_layer(m, i, st, SIDE_BOTH);
+        m->B = m->full_B; m->sub_active = false; m->sub_row0 = 0;
+        std::swap(m->L, m->mod_L[k]);
+        if (s != SB_OK) return s;
+        m->cur_layer = -1;
+        L_TRY("sgd", 0.0, (double)fc_cnt * (m->bf16 ? 22.0 : 20.0),
+              launch_sgd(m->Wm + fc_off, m->Vm + fc_off, m->Gm + fc_off, m->Sm ? m->Sm + fc_off : nullptr, fc_cnt, lr, momentum, st));
+    }
+    m->cur_layer = ff;
+    {
+        ModuloCopyArgs a{m->mod_dx, m->L[ff - 1].dact, D * m->esz, R, b, K, 1, nullptr, nullptr};
+        L_TRY("modulo_scatter", 0.0, 2.0 * m->B * D * m->esz, launch_modulo_copy(a, st));
+    }
+    for (int i = ff - 1; i >= 0; --i) {
+        s = backward_layer(m, i, st, SIDE_BOTH);
+        if (s != SB_OK) return s;
+    }
+    m->cur_layer = -1;
+    L_TRY("sgd", 0.0, (double)fc_off * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, fc_off, lr, momentum, st));
+    m->have_fwd = false;   // the FC activations hold the last sub-iteration only: sb_backward has nothing consistent to use
+    m->last_step_launches = m->launches;
+    return SB_OK;
 }
 
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream)

@@ -139,8 +139,27 @@ struct XentArgs {
     void* dZ;             // [B,C] activation dtype: (softmax - onehot)/B
     unsigned int* counter; // zero-initialised word; left at zero
     int B, C;
+    // Sub-batch use (modulo schedule): the rows above are a slice of a larger batch.  scale_B > 0 replaces B in the
+    // 1/B of dZ; loss_rows > 0 makes the mean loss the sum of loss_base[0 .. loss_rows) divided by loss_rows.
+    int scale_B = 0;
+    const float* loss_base = nullptr;
+    int loss_rows = 0;
 };
 cudaError_t launch_softmax_xent(const XentArgs& a, bool bf16, cudaStream_t st);
+
+// Modulo layer as an explicit copy (sub-iteration schedule): R replicas of b rows, K slices of b/K rows each.
+// gather : dst[k*(R*b/K) + r*(b/K) + i] = src[r*b + k*(b/K) + i]   (rows of `row_bytes` bytes, a multiple of 16)
+// scatter: the inverse.  labels (optional, gather only): int32 per row, read through the per-replica table.
+struct ModuloCopyArgs {
+    const void* src;
+    void* dst;
+    size_t row_bytes;
+    int R, b, K;
+    int scatter;               // 0: gather, 1: scatter
+    const PtrTab* labels;      // gather only: R pointers to int32 [b]; nullptr = no labels
+    int32_t* labels_out;       // [R*b] in sub-iteration order
+};
+cudaError_t launch_modulo_copy(const ModuloCopyArgs& a, cudaStream_t st);
 
 cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n,
                        float lr, float mu, cudaStream_t st);

@@ -535,7 +535,8 @@ cudaError_t launch_pool_bwd(const PoolBwdArgs& a, bool bf16, cudaStream_t st)
 template <typename T>
 __global__ void __launch_bounds__(256)
 softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_rep, float* __restrict__ row_loss,
-                    float* __restrict__ loss, T* __restrict__ dZ, unsigned int* __restrict__ counter, int B, int C)
+                    float* __restrict__ loss, T* __restrict__ dZ, unsigned int* __restrict__ counter, int B, int C,
+                    int scale_B, const float* __restrict__ loss_base, int loss_rows)
 {
     pdl_prologue();
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -552,7 +553,7 @@ softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_r
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         const float lse = m + logf(s);
-        const float invB = 1.0f / (float)B;
+        const float invB = 1.0f / (float)scale_B;
         for (int c = lane; c < C; c += 32) {
             float pr = expf(z[c] - lse);
             stf(dZ + (size_t)g * C + c, (pr - (c == y ? 1.f : 0.f)) * invB);
@@ -567,20 +568,52 @@ softmax_xent_kernel(const float* __restrict__ logits, PtrTab labels, int b_per_r
     if (last && warp == 0) {
         __threadfence();
         float t = 0.f;
-        for (int i0 = 0; i0 < B; i0 += 32) {           // fixed order: chunks of 32 rows, tree inside
-            float v = (i0 + lane < B) ? ((volatile float*)row_loss)[i0 + lane] : 0.f;
+        for (int i0 = 0; i0 < loss_rows; i0 += 32) {   // fixed order: chunks of 32 rows, tree inside
+            float v = (i0 + lane < loss_rows) ? ((volatile const float*)loss_base)[i0 + lane] : 0.f;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
             t += v;
         }
-        if (lane == 0) { *loss = t / (float)B; *counter = 0u; }
+        if (lane == 0) { *loss = t / (float)loss_rows; *counter = 0u; }
     }
 }
 cudaError_t launch_softmax_xent(const XentArgs& a, bool bf16, cudaStream_t st)
 {
     int blocks = cdiv(a.B, 8);
-    if (bf16) SB_LAUNCH((softmax_xent_kernel<__nv_bfloat16>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (__nv_bfloat16*)a.dZ, a.counter, a.B, a.C);
-    else SB_LAUNCH((softmax_xent_kernel<float>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (float*)a.dZ, a.counter, a.B, a.C);
+    const int scale_B = a.scale_B > 0 ? a.scale_B : a.B;
+    const float* loss_base = a.loss_rows > 0 ? a.loss_base : a.row_loss;
+    const int loss_rows = a.loss_rows > 0 ? a.loss_rows : a.B;
+    if (bf16) SB_LAUNCH((softmax_xent_kernel<__nv_bfloat16>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (__nv_bfloat16*)a.dZ, a.counter, a.B, a.C, scale_B, loss_base, loss_rows);
+    else SB_LAUNCH((softmax_xent_kernel<float>), blocks, 256, 0, st, a.logits, a.labels, a.b_per_rep, a.row_loss, a.loss, (float*)a.dZ, a.counter, a.B, a.C, scale_B, loss_base, loss_rows);
+    return cudaGetLastError();
+}
+
+// Modulo layer as a row permutation (see ModuloCopyArgs): one block column per row, 16-byte chunks.
+__global__ void __launch_bounds__(256)
+modulo_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t row_vecs, int R, int b, int K, int scatter,
+                   PtrTab labels, int has_labels, int32_t* __restrict__ labels_out)
+{
+    pdl_prologue();
+    const int bk = b / K;
+    const int nat = blockIdx.y;                                  // natural row index r*b + k*bk + i
+    const int r = nat / b, k = (nat % b) / bk, i = nat % bk;
+    const int sub = k * (R * bk) + r * bk + i;                   // sub-iteration order
+    const uint4* s = src + (size_t)(scatter ? sub : nat) * row_vecs;
+    uint4* d = dst + (size_t)(scatter ? nat : sub) * row_vecs;
+    for (size_t v = blockIdx.x * (size_t)blockDim.x + threadIdx.x; v < row_vecs; v += (size_t)gridDim.x * blockDim.x) d[v] = s[v];
+    if (has_labels && !scatter && blockIdx.x == 0 && threadIdx.x == 0) labels_out[sub] = ((const int32_t*)labels.p[r])[nat % b];
+}
+cudaError_t launch_modulo_copy(const ModuloCopyArgs& a, cudaStream_t st)
+{
+    if (a.row_bytes % 16 != 0 || a.K < 1 || a.b % a.K != 0) return cudaErrorInvalidValue;
+    const size_t row_vecs = a.row_bytes / 16;
+    int bx = (int)((row_vecs + 255) / 256);
+    if (bx > 32) bx = 32;
+    if (bx < 1) bx = 1;
+    PtrTab tab{};
+    if (a.labels) tab = *a.labels;
+    SB_LAUNCH((modulo_copy_kernel), dim3(bx, a.R * a.b), 256, 0, st, (const uint4*)a.src, (uint4*)a.dst, row_vecs, a.R, a.b, a.K, a.scatter, tab,
+              a.labels ? 1 : 0, a.labels_out);
     return cudaGetLastError();
 }
 

@@ -1123,6 +1123,7 @@ static sb_status fail_plan() { return SB_ERR_CUDA; }
 // Fills the split / ring fields of a FWD or DGRAD op from its tile plan.
 static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles, int n_tiles_total, float* ws, size_t rows)
 {
+    // (the scratch for split partial sums was sized by umma_plan_scratch for the full batch; sub-batch plans are checked by the caller)
     UmmaParams& p = b->p;
     b->bn = t.bn;
     p.total_chunks = k_iters;
@@ -1136,12 +1137,12 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
     b->rows = (long)rows;
 }
 
-sb_status umma_plan_layers(sb_model* m)
+sb_status umma_plan_layers(sb_model* m, int first_layer)
 {
     ModelView mv = model_view(m);
     if (!mv.bf16 || (mv.cfg->flags & SB_FLAG_FORCE_SIMT)) return SB_OK;
     const int B = mv.B;
-    for (int i = 0; i < mv.n_layers; ++i) {
+    for (int i = first_layer; i < mv.n_layers; ++i) {
         LayerView lv = layer_view(m, i);
         UmmaLayer& um = *lv.um;
         const bool want_in_grad = i > 0;
@@ -1239,6 +1240,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.epi = UEPI_BIAS_ACT; p.relu = lv.relu ? 1 : 0; p.out_f32 = lv.kind == SB_FC; p.out = lv.act; p.ldc = lv.out_f;
                 p.bias = mv.Wm + lv.p_b; p.status = mv.status;
                 apply_plan(b, g.fwd, p.kchunks, m_tiles, p.tiles_per_shard * K, mv.ws, (size_t)B);
+                if (p.splits > 1 && (size_t)p.splits * (size_t)p.split_stride > mv.ws_floats) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
                 um.fwd.enabled = true;
@@ -1256,6 +1258,7 @@ sb_status umma_plan_layers(sb_model* m)
                 p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
                 p.status = mv.status;
                 apply_plan(b, g.dgrad, p.kchunks, m_tiles, p.tiles_per_shard, mv.ws, (size_t)B);
+                if (p.splits > 1 && (size_t)p.splits * (size_t)p.split_stride > mv.ws_floats) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.dgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, 64)) return fail_plan();
                 um.dgrad.enabled = true;

@@ -53,8 +53,8 @@ int64_t* launch_counter(sb_model* m);
 // Scratch floats the tensor-core path needs (split partial sums); called during planning,
 // before the arena exists (pointers in the views are null or unset).
 sb_status umma_plan_scratch(sb_model* m, size_t* floats);
-// Encodes tensor maps and decides, per layer and pass, whether the tensor-core kernel runs.
-sb_status umma_plan_layers(sb_model* m);
+// Encodes tensor maps and decides, per layer and pass, whether the tensor-core kernel runs (layers first_layer..).
+sb_status umma_plan_layers(sb_model* m, int first_layer);
 
 sb_status umma_conv_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st);
