@@ -168,7 +168,8 @@ sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream);
  * With K = 1 the result is that of sb_forward + sb_backward + sb_sgd_step; with K > 1 it is a different
  * algorithm (the FC weights move between sub-iterations).  sb_loss afterwards returns the mean of the R*b row
  * losses.  Needs SB_FLAG_MODULO_SCHEDULE at creation (SB_ERR_STATE otherwise).  Arguments as for sb_forward /
- * sb_sgd_step; runs on `stream`, asynchronous.  Afterwards SB_T_ROW_LOSS and the FC activation tensors hold their
+ * sb_sgd_step; runs on `stream`, asynchronous; like sb_graph_step the second call captures the iteration as a CUDA
+ * graph and later calls with the same pointers and hyper-parameters replay it.  Afterwards SB_T_ROW_LOSS and the FC activation tensors hold their
  * rows in sub-iteration order (position k*(R*b/K) + r*(b/K) + i = example k*(b/K) + i of replica r), the FC
  * activations as left by the sub-iteration that wrote them; sb_backward needs a new sb_forward.
  */

@@ -120,7 +120,7 @@ struct sb_model {
         float lr = 0.f, mu = 0.f;
         bool warmed = false;
     };
-    StepGraph g_dev, g_host;
+    StepGraph g_dev, g_host, g_mod;
     uint32_t host_result[2] = {0, 0};   // loss bits and device status word written by the host-step graph
     // per-launch event recording (sb_profile_begin / sb_profile_end)
     struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; int layer; };
@@ -151,6 +151,7 @@ struct sb_model {
         for (int k = 0; k < MAX_WSTREAMS; ++k) { if (wstreams[k]) cudaStreamDestroy(wstreams[k]); if (ev_wjoin[k]) cudaEventDestroy(ev_wjoin[k]); }
         if (g_dev.exec) cudaGraphExecDestroy(g_dev.exec);
         if (g_host.exec) cudaGraphExecDestroy(g_host.exec);
+        if (g_mod.exec) cudaGraphExecDestroy(g_mod.exec);
     }
 };
 
@@ -847,8 +848,9 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
 // stream as soon as that layer's gradients are complete and its input gradient (which reads the weights) has
 // been computed, so the bandwidth-bound update overlaps the rest of the backward pass.  Element for element the
 // update is the one sb_sgd_step does.  Returns *updated = true if the update was done here.
-static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, float lr, float mu, bool* updated)
+static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, float lr, float mu, bool* updated, int hi = -1, int lo = 0)
 {
+    if (hi < 0) hi = m->n_layers - 1;     // layers hi .. lo, top down
     // The weight-gradient work of a layer (and its split reduce) only has to be finished before the update,
     // while the input-gradient chain is the critical path: the former runs on the model's second stream,
     // ordered by one event per layer ("the gradient w.r.t. this layer's output is ready") and joined at the
@@ -857,7 +859,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
     const bool fuse = fuse_update && two_streams;
     if (updated) *updated = fuse;
     unsigned used_streams = 0;   // weight streams that received work in this pass (only those are joined)
-    for (int i = m->n_layers - 1; i >= 0; --i) {
+    for (int i = hi; i >= lo; --i) {
         Layer& l = m->L[i];
         const bool has_params = l.kind == SB_CONV3X3_RELU || l.kind == SB_FC_RELU || l.kind == SB_FC;
         if (two_streams && has_params) {
@@ -928,7 +930,7 @@ static sb_status whole_step(sb_model* m, const void* const* x, const int32_t* co
 // -> rows k*B/K + r*b/K ...); the FC stack then runs K sub-iterations (forward, loss with 1/B per row, backward,
 // SGD update of the FC parameters), each on B/K rows; the input gradients are copied back into row order and the
 // conv-side stack back-propagates once and takes its update.  Everything runs on the caller's stream.
-sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
+static sb_status modulo_step_direct(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (!(m->cfg.flags & SB_FLAG_MODULO_SCHEDULE)) return fail(SB_ERR_STATE, "the model was created without SB_FLAG_MODULO_SCHEDULE");
@@ -968,12 +970,12 @@ sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const
         ModuloCopyArgs a{m->mod_dx, m->L[ff - 1].dact, D * m->esz, R, b, K, 1, nullptr, nullptr};
         L_TRY("modulo_scatter", 0.0, 2.0 * m->B * D * m->esz, launch_modulo_copy(a, st));
     }
-    for (int i = ff - 1; i >= 0; --i) {
-        s = backward_layer(m, i, st, SIDE_BOTH);
-        if (s != SB_OK) return s;
-    }
+    // conv-side stack: the multi-stream backward pass with the per-layer updates folded in, as in the synchronous step
+    bool updated = false;
+    s = backward_pass(m, st, true, lr, momentum, &updated, ff - 1, 0);
+    if (s != SB_OK) return s;
     m->cur_layer = -1;
-    L_TRY("sgd", 0.0, (double)fc_off * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, fc_off, lr, momentum, st));
+    if (!updated) L_TRY("sgd", 0.0, (double)fc_off * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm, m->Vm, m->Gm, m->Sm, fc_off, lr, momentum, st));
     m->have_fwd = false;   // the FC activations hold the last sub-iteration only: sb_backward has nothing consistent to use
     m->last_step_launches = m->launches;
     return SB_OK;
@@ -1029,18 +1031,21 @@ static void abandon_capture(cudaStream_t st)
     cudaGetLastError();
 }
 
-sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
+// An iteration on device-resident inputs replayed as a CUDA graph: the first call runs `step` directly, the second
+// captures it, later calls with the same pointers and hyper-parameters are one graph launch.
+typedef sb_status (*StepFn)(sb_model*, const void* const*, const int32_t* const*, float, float, void*);
+static sb_status graph_replay(sb_model* m, sb_model::StepGraph& G, StepFn step, const void* const* x, const int32_t* const* labels,
+                              float lr, float momentum, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (!x || !labels) return fail(SB_ERR_INVALID_ARG, "x or labels is null");
     cudaStream_t st = (cudaStream_t)stream;
-    sb_model::StepGraph& G = m->g_dev;
     PtrTab xt{}, lt{};
     for (int r = 0; r < m->cfg.R; ++r) { xt.p[r] = x[r]; lt.p[r] = labels[r]; }
     const bool eager = m->profiling || m->debug_sync || !G.warmed || st == nullptr;
     if (eager) {
         // first use (one-time function attributes are set by the first launches), or a mode that needs every launch visible
-        sb_status s = whole_step(m, x, labels, lr, momentum, stream);
+        sb_status s = step(m, x, labels, lr, momentum, stream);
         if (s == SB_OK) G.warmed = true;
         return s;
     }
@@ -1048,7 +1053,7 @@ sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const*
     if (!hit) {
         if (G.exec) { cudaGraphExecDestroy(G.exec); G.exec = nullptr; }
         CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        sb_status s = whole_step(m, x, labels, lr, momentum, stream);
+        sb_status s = step(m, x, labels, lr, momentum, stream);
         if (s != SB_OK) { abandon_capture(st); return s; }
         cudaGraph_t graph = nullptr;
         CU_TRY(cudaStreamEndCapture(st, &graph));
@@ -1058,8 +1063,24 @@ sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const*
         G.x = xt; G.labels = lt; G.lr = lr; G.mu = momentum;
     }
     CU_TRY(cudaGraphLaunch(G.exec, st));
-    m->have_fwd = true;
     return SB_OK;
+}
+
+sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    sb_status s = graph_replay(m, m->g_dev, whole_step, x, labels, lr, momentum, stream);
+    if (s == SB_OK) m->have_fwd = true;
+    return s;
+}
+
+sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (!(m->cfg.flags & SB_FLAG_MODULO_SCHEDULE)) return fail(SB_ERR_STATE, "the model was created without SB_FLAG_MODULO_SCHEDULE");
+    sb_status s = graph_replay(m, m->g_mod, modulo_step_direct, x, labels, lr, momentum, stream);
+    if (s == SB_OK) m->have_fwd = false;
+    return s;
 }
 
 sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum,
