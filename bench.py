@@ -312,17 +312,85 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_fc_sweep(args):
+    """Configuration 4: the sharded-FC sweep (one 25088 -> 4096 layer; forward + data gradient + weight gradient) at
+    batch {32, 128, 512} x K {1, 2, 4, 8} x R {1, 4}: TFLOP/s of each point against the dense bf16 peak.  The
+    equality across K is a parity test (tests/test_gpu_parity_configs.py); this only times."""
+    import torch
+
+    import __graft_entry__ as ge
+    if int(os.environ.get("RANK", 0)) != 0:
+        return
+    ge.build()
+    torch.cuda.set_device(0)
+    from paper_2112_15317_b200 import binding as sb
+    import numpy as np
+
+    d_in, d_out = 25088, 4096
+    pk = peaks()
+    side = torch.cuda.Stream()
+    torch.cuda.set_stream(side)
+    layers = [(si.FC, d_out), (si.SOFTMAX_XENT, d_out)]
+    steps, warm = max(3, min(args.steps, 50)), max(3, min(args.warmup, 10))
+    points = []
+    sampler = ClockSampler(0)
+    t_wall0 = time.time()
+    for B in (32, 128, 512):
+        w, x, dy = si.fc_sweep_case(B)
+        xt = torch.from_numpy(x).cuda().to(torch.bfloat16)
+        params = [{"w": w, "b": np.zeros(d_out, np.float32)}, None]
+        for R in (1, 4):
+            for K in (1, 2, 4, 8):
+                wl = si.Workload(f"fc_sweep_B{B}_R{R}_K{K}", layers, 1, 1, d_in, B // R, R, K)
+                m = sb.Model.from_workload(wl, precision=sb.SB_BF16, flags=sb.SB_FLAG_INPUT_GRAD)
+                m.load_params(params, si.shard_bounds)
+                xs = [xt[r * wl.b:(r + 1) * wl.b] for r in range(R)]
+                m.forward_layers(0, 0, xs, None)
+                m.write(sb.SB_T_DACT, 0, 0, dy)
+                for _ in range(warm):
+                    m.forward_layers(0, 0, xs, None); m.backward_layers(0, 0)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                side.synchronize()
+                e0.record(side)
+                for _ in range(steps):
+                    m.forward_layers(0, 0, xs, None); m.backward_layers(0, 0)
+                e1.record(side)
+                side.synchronize()
+                ms = e0.elapsed_time(e1) / steps
+                flops = 3 * 2.0 * B * d_in * d_out
+                # weights read twice (forward, data gradient) + the float weight gradient written once + activations
+                byts = 2 * d_in * d_out * 2 + d_in * d_out * 4 + B * (3 * d_in + 2 * d_out) * 2
+                t_roof = max(flops / (pk["tf_sustained"] * 1e12), byts / (pk["hbm_gbs"] * 1e9)) * 1e3
+                points.append(dict(B=B, R=R, K=K, ms=ms, tflops=flops / ms / 1e9, frac_of_tensor_peak=flops / ms / 1e9 / pk["tf_sustained"],
+                                   roofline_ms=t_roof, frac_of_roofline=t_roof / ms))
+                m.close()
+    clocks = sampler.stop(t_wall0, time.time())
+    best = max(points, key=lambda p_: p_["tflops"])
+    print(json.dumps({
+        "metric": "sharded FC forward + dgrad + wgrad throughput", "value": best["tflops"], "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": best["ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg4_sharded_fc_sweep", "layer": "FC 25088 -> 4096, bf16 operands, fp32 accumulate, fp32 weight gradient",
+                   "points": "B in {32,128,512} x R in {1,4} x K in {1,2,4,8}; value = best point", "launch": "separate calls (no graph), one stream",
+                   "l2": "the 205 MB bf16 weight matrix and the 411 MB gradient exceed the 126 MB L2; no flush"},
+        "peak": {"tensor_tflops": pk["tf_sustained"], "hbm_gbs": pk["hbm_gbs"], "source": pk["source"]},
+        "clocks": clocks, "sweep": points}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3],
-                    help="1 = VGG-16 CIFAR shape, batch 128 (the metric's configuration); 0/2/3 = the other configurations")
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4],
+                    help="1 = VGG-16 CIFAR shape, batch 128 (the metric's configuration); 0/2/3 = the other configurations; "
+                         "4 = the sharded-FC sweep (TFLOP/s per point)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 4:
+        run_fc_sweep(args)
     else:
         run_ours(args)
 
