@@ -951,7 +951,9 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         if (t.bn < 256 && st > two) st = two;
     }
     static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
-    if ((backward || fwd_too) && bwd_cohabit() && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
+    // (a grid that leaves SMs idle need not share its SMs: the other stream's CTAs find free ones; SB_COHABIT_MIN_CTAS)
+    static const long cohabit_min = [] { const char* e = getenv("SB_COHABIT_MIN_CTAS"); return e ? atol(e) : 0L; }();
+    if ((backward || fwd_too) && bwd_cohabit() && tiles * t.splits >= cohabit_min && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     // Grids of more than one CTA per SM: measured, the co-residency of CTAs (their set-up, first loads and
     // epilogues overlap one another's main loops) is worth more than ring depth -- the 1024-CTA 64-wide layer runs
     // 28 us with 2 stages (4 CTAs per SM) against 37 us with 4 and 60 us with 8; beyond 3 stages no layer gains.
@@ -984,7 +986,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         const int pfit = t.bn >= 256 ? 6 : 8;
         int pst = t.cps < pfit ? t.cps : pfit;
         const int ptwo = t.bn >= 256 ? 3 : 4;      // two resident CTAs per SM
-        if ((tiles * t.splits >= 296 || ((backward || fwd_too) && bwd_cohabit())) && pst > ptwo) pst = ptwo;
+        if ((tiles * t.splits >= 296 || ((backward || fwd_too) && bwd_cohabit() && tiles * t.splits >= cohabit_min)) && pst > ptwo) pst = ptwo;
         t.stages = pst < 1 ? 1 : pst;
     }
     static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
@@ -1208,7 +1210,12 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     const int fit = b->bn >= 256 ? 4 : (b->bn >= 192 ? 5 : (b->bn >= 128 ? 6 : 8));
                     p.stages = g.wg_cps < fit ? g.wg_cps : fit;
                 }
-                if (bwd_cohabit() && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
+                {
+                    // grids of fewer than ~100 CTAs leave the other streams whole SMs: no need to keep the ring shallow (measured: -1.5 % step)
+                    static const long wg_cohabit_min = [] { const char* e = getenv("SB_WG_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
+                    const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * (9 / p.tap_group) * p.splits;
+                    if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
+                }
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
                 // the bias gradient rides along: in the parameter arena the bias vector directly follows the
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
