@@ -952,7 +952,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     }
     static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
     // (a grid that leaves SMs idle need not share its SMs: the other stream's CTAs find free ones; SB_COHABIT_MIN_CTAS)
-    static const long cohabit_min = [] { const char* e = getenv("SB_COHABIT_MIN_CTAS"); return e ? atol(e) : 0L; }();
+    static const long cohabit_min = [] { const char* e = getenv("SB_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
     if ((backward || fwd_too) && bwd_cohabit() && tiles * t.splits >= cohabit_min && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     // Grids of more than one CTA per SM: measured, the co-residency of CTAs (their set-up, first loads and
     // epilogues overlap one another's main loops) is worth more than ring depth -- the 1024-CTA 64-wide layer runs
