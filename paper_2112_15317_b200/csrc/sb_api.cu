@@ -353,7 +353,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.in = layer_input(m, i); a.tab = i == 0 ? &m->x_tab : nullptr; a.b_per_rep = b;
         a.w = wts; a.bias = m->Wm + l.p_b; a.out = l.act; a.mask_ref = nullptr;
         a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.dgrad = 0; a.relu = 1;
-        if (l.thin_input && l.um.conv_in) L_TRY("conv_in_fwd_umma", flops, bytes, launch_conv_in_fwd_umma(a, m->status, st));
+        if (l.thin_input && l.um.conv_in) L_TRY("conv_in_fwd_umma", flops, bytes, launch_conv_in_fwd_umma(a, &l.um.fwd.mapA, m->status, st));
         else if (l.thin_input) L_TRY("conv_in_fwd", flops, bytes, launch_conv_in_fwd(a, bf, st));
         else L_TRY("conv_fwd_simt", flops, bytes, launch_conv_simt(a, bf, st));
         break;

@@ -18,6 +18,7 @@
 #include "sb_tcgen05.cuh"
 
 #include <cstdio>
+#include <cstdlib>
 
 namespace sb {
 
@@ -60,14 +61,67 @@ __device__ __forceinline__ uint4 patch_chunk(const __nv_bfloat16* img, int h, in
     return make_uint4(pk[0], pk[1], pk[2], pk[3]);
 }
 
+// Staged variant: the pixels a tile's 3x3 neighbourhoods touch are one contiguous range of the image (flat pixels
+// [first - W - 1, last + W + 1], clipped to the image), so the CTA first copies that range into shared memory with
+// coalesced 4-byte loads and the patch rows are gathered from there (27 two-byte global loads per pixel become ~7
+// four-byte loads per thread).  `win` holds the elements from index e_start of the image on.
+template <int CIN>
+__device__ __forceinline__ uint4 patch_chunk_win(const __nv_bfloat16* win, long e_start, int h, int w, int H, int W, int k0, int ones_col)
+{
+    uint32_t pk[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        uint32_t two[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int k = k0 + 2 * e + u;
+            uint32_t bits = 0;
+            if (k < 9 * CIN) {
+                const int tap = k / CIN, c = k - tap * CIN;
+                const int r3 = tap / 3, hh = h + r3 - 1, ww = w + (tap - 3 * r3) - 1;
+                if (hh >= 0 && hh < H && ww >= 0 && ww < W)
+                    bits = (uint32_t)__bfloat16_as_ushort(win[((long)hh * W + ww) * CIN + c - e_start]);
+            } else if (k == ones_col) {
+                bits = 0x3F80u;   // bf16 1.0
+            }
+            two[u] = bits;
+        }
+        pk[e] = two[0] | (two[1] << 16);
+    }
+    return make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+// Copies the window of `count` pixels starting at pixel p_in of the image `img` (H*W*CIN elements, an even number,
+// 4-byte aligned) into `win`; returns the element index the window starts at.  Called by all CI_THREADS threads.
+template <int CIN>
+__device__ __forceinline__ long stage_window(const __nv_bfloat16* img, __nv_bfloat16* win, long p_in, int count, int H, int W)
+{
+    const long HW = (long)H * W;
+    long lo = p_in - W - 1, hi = p_in + count + W + 1;
+    if (lo < 0) lo = 0;
+    if (hi > HW) hi = HW;
+    const long e_start = (lo * CIN) & ~1L, e_end = hi * CIN;       // e_end <= H*W*CIN, which is even: whole words stay inside
+    const int words = (int)((e_end - e_start + 1) / 2);
+    const uint32_t* src = (const uint32_t*)(img + e_start);
+    uint32_t* dst = (uint32_t*)win;
+    for (int i = threadIdx.x; i < words; i += CI_THREADS) dst[i] = src[i];
+    return e_start;
+}
+// Shared-memory bytes of the window for `count` pixels per tile; 0 = too large, gather from global memory instead.
+static size_t window_bytes(int count, int W, int Cin)
+{
+    const size_t b = ((size_t)(count + 2 * W + 2) * Cin + 2) * 2;
+    return b <= 24576 ? (b + 15) / 16 * 16 : 0;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Forward: persistent CTAs, one 128-pixel tile (flat pixel index) per iteration
 // ------------------------------------------------------------------------------------------------
 template <int CIN, bool TAB>
 __global__ void __launch_bounds__(CI_THREADS)
-conv_in_fwd_umma_kernel(const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_per_rep, const __nv_bfloat16* __restrict__ wt,
+conv_in_fwd_umma_kernel(const __grid_constant__ CUtensorMap mapY, int tma_out, const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_per_rep,
+                        const __nv_bfloat16* __restrict__ wt,
                         const float* __restrict__ bias, __nv_bfloat16* __restrict__ y, long npix, int H, int W, int Cout, int relu,
-                        long n_tiles, uint32_t tmem_cols, uint32_t* status)
+                        long n_tiles, uint32_t tmem_cols, uint32_t* status, int use_window)
 {
     constexpr int KSTEPS = (9 * CIN + 15) / 16;      // 16-wide MMA k-steps that hold data
     constexpr int CHUNKS = 2 * KSTEPS;               // 16-byte chunks per row that hold data
@@ -79,6 +133,7 @@ conv_in_fwd_umma_kernel(const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_p
     uint64_t* bar = (uint64_t*)(s_bias + Cout);
     uint32_t* tmem_slot = (uint32_t*)(bar + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    __nv_bfloat16* win = (__nv_bfloat16*)(((uintptr_t)(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // input window (use_window)
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32, r = threadIdx.x;
     if (threadIdx.x == 0) {
@@ -116,8 +171,9 @@ conv_in_fwd_umma_kernel(const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_p
     const size_t img_elems = (size_t)H * W * CIN;
     uint32_t phase = 0;
 
+    const long HW = (long)H * W;
     for (long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const long P = tile * 128 + r;
+        const long P0 = tile * 128, P = P0 + r;
         const bool valid = P < npix;
         int w = 0, h = 0;
         const __nv_bfloat16* img = x;
@@ -127,10 +183,27 @@ conv_in_fwd_umma_kernel(const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_p
             h = (int)(q % H);
             img = image_ptr<TAB>(x, tab, b_per_rep, q / H, img_elems);
         }
+        // a tile that lies inside one image (uniform over the CTA) gathers from the staged window
+        const long p_in = P0 % HW;
+        const bool staged = use_window && p_in + 128 <= HW && P0 + 128 <= npix;
+        if (tma_out) {
+            // the previous tile's output was staged in sA: its TMA store must have read it before sA is rewritten
+            if (threadIdx.x == 0) tma_store_wait_read();
+            __syncthreads();
+        }
+        if (staged) {
+            const __nv_bfloat16* img0 = image_ptr<TAB>(x, tab, b_per_rep, P0 / HW, img_elems);
+            const long e_start = stage_window<CIN>(img0, win, p_in, 128, H, W);
+            __syncthreads();
 #pragma unroll
-        for (int j = 0; j < CHUNKS; ++j) {
-            const uint4 v = valid ? patch_chunk<CIN>(img, h, w, H, W, 8 * j, -1) : make_uint4(0u, 0u, 0u, 0u);
-            *(uint4*)(sA + r * 128 + ((j ^ (r & 7)) << 4)) = v;
+            for (int j = 0; j < CHUNKS; ++j)
+                *(uint4*)(sA + r * 128 + ((j ^ (r & 7)) << 4)) = patch_chunk_win<CIN>(win, e_start, h, w, H, W, 8 * j, -1);
+        } else {
+#pragma unroll
+            for (int j = 0; j < CHUNKS; ++j) {
+                const uint4 v = valid ? patch_chunk<CIN>(img, h, w, H, W, 8 * j, -1) : make_uint4(0u, 0u, 0u, 0u);
+                *(uint4*)(sA + r * 128 + ((j ^ (r & 7)) << 4)) = v;
+            }
         }
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
         __syncthreads();
@@ -164,14 +237,28 @@ conv_in_fwd_umma_kernel(const __nv_bfloat16* __restrict__ x, PtrTab tab, int b_p
                     __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
                     pk[j] = *(uint32_t*)&t;
                 }
-                ((uint4*)(yr + c0))[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                ((uint4*)(yr + c0))[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                if (tma_out) {
+                    // output row r = 128 bytes (64 channels), staged in the A tile's buffer (the MMA has consumed it) in
+                    // the same 128-byte swizzle, so that one TMA store writes the tile's 16 KB in full lines
+                    const int j0 = c0 >> 3;
+                    *(uint4*)(sA + r * 128 + (((j0) ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *(uint4*)(sA + r * 128 + (((j0 + 1) ^ (r & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                } else {
+                    ((uint4*)(yr + c0))[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    ((uint4*)(yr + c0))[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
             }
         }
+        if (tma_out) fence_async_smem();
         tc_fence_before();
         __syncthreads();             // accumulator drained and A tile consumed before the next tile overwrites them
         if (*abort_flag) break;
+        if (tma_out && threadIdx.x == 0) {
+            tma_store_4d(&mapY, smem_u32(sA), 0, (int)P0, 0, 0);     // rows past the last pixel are clipped by the tensor map
+            tma_store_commit();
+        }
     }
+    if (tma_out && threadIdx.x == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -352,28 +439,37 @@ int conv_in_umma_wgrad_blocks(long npix)
 }
 
 template <int CIN>
-static cudaError_t launch_fwd_t(const ConvSimtArgs& a, uint32_t* status, cudaStream_t st)
+static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, uint32_t* status, cudaStream_t st)
 {
     const long npix = (long)a.B * a.H * a.W;
     const long n_tiles = (npix + 127) / 128;
     const int grid = (int)(n_tiles < 148 * 6 ? n_tiles : 148 * 6);
-    const size_t smem = 1024 + 16384 + (size_t)a.Cout * 128 + (size_t)a.Cout * 4 + 64;
+    // the staged gather needs images of an even number of elements (4-byte loads) and a window that fits
+    static const bool no_window = [] { const char* e = getenv("SB_CONV_IN_WINDOW"); return e && e[0] == '0'; }();
+    const size_t wbytes = (!no_window && ((size_t)a.H * a.W * CIN) % 2 == 0) ? window_bytes(128, a.W, CIN) : 0;
+    const size_t smem = 1024 + 16384 + (size_t)a.Cout * 128 + (size_t)a.Cout * 4 + 64 + wbytes;
+    const int use_window = wbytes > 0 ? 1 : 0;
     PtrTab tab{};
     if (a.tab) tab = *a.tab;
     const uint32_t cols = pow2_cols(a.Cout);
+    // the output goes out by TMA store when the caller made a tensor map for it (64 channels: one 128-byte row per pixel)
+    static const bool no_tma_out = [] { const char* e = getenv("SB_CONV_IN_TMA_OUT"); return e && e[0] == '0'; }();
+    const int tma_out = (mapY && a.Cout == 64 && !no_tma_out) ? 1 : 0;
+    CUtensorMap dummy{};
+    const CUtensorMap& my = tma_out ? *mapY : dummy;
     if (a.tab)
-        return pdl_launch(conv_in_fwd_umma_kernel<CIN, true>, dim3(grid), dim3(CI_THREADS), smem, st, (const __nv_bfloat16*)nullptr, tab, a.b_per_rep,
-                          (const __nv_bfloat16*)a.w, a.bias, (__nv_bfloat16*)a.out, npix, a.H, a.W, a.Cout, a.relu, n_tiles, cols, status);
-    return pdl_launch(conv_in_fwd_umma_kernel<CIN, false>, dim3(grid), dim3(CI_THREADS), smem, st, (const __nv_bfloat16*)a.in, tab, a.b_per_rep,
-                      (const __nv_bfloat16*)a.w, a.bias, (__nv_bfloat16*)a.out, npix, a.H, a.W, a.Cout, a.relu, n_tiles, cols, status);
+        return pdl_launch(conv_in_fwd_umma_kernel<CIN, true>, dim3(grid), dim3(CI_THREADS), smem, st, my, tma_out, (const __nv_bfloat16*)nullptr, tab, a.b_per_rep,
+                          (const __nv_bfloat16*)a.w, a.bias, (__nv_bfloat16*)a.out, npix, a.H, a.W, a.Cout, a.relu, n_tiles, cols, status, use_window);
+    return pdl_launch(conv_in_fwd_umma_kernel<CIN, false>, dim3(grid), dim3(CI_THREADS), smem, st, my, tma_out, (const __nv_bfloat16*)a.in, tab, a.b_per_rep,
+                      (const __nv_bfloat16*)a.w, a.bias, (__nv_bfloat16*)a.out, npix, a.H, a.W, a.Cout, a.relu, n_tiles, cols, status, use_window);
 }
 
-cudaError_t launch_conv_in_fwd_umma(const ConvSimtArgs& a, uint32_t* status, cudaStream_t st)
+cudaError_t launch_conv_in_fwd_umma(const ConvSimtArgs& a, const CUtensorMap* mapY, uint32_t* status, cudaStream_t st)
 {
     switch (a.Cin) {
-    case 1: return launch_fwd_t<1>(a, status, st);
-    case 3: return launch_fwd_t<3>(a, status, st);
-    case 4: return launch_fwd_t<4>(a, status, st);
+    case 1: return launch_fwd_t<1>(a, mapY, status, st);
+    case 3: return launch_fwd_t<3>(a, mapY, status, st);
+    case 4: return launch_fwd_t<4>(a, mapY, status, st);
     default: return cudaErrorInvalidValue;
     }
 }

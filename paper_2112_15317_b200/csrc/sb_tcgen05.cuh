@@ -72,6 +72,19 @@ __device__ __forceinline__ void tma_load_4d_el(const CUtensorMap* map, uint32_t 
         ::"r"(dst_saddr), "l"(map), "r"(bar_saddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
         : "memory");
 }
+// TMA store of one box from shared memory (bulk async-group completion) through a rank-4 tensor map (the rank of the
+// instruction must be the map's: every map of this library is encoded with four dimensions); elements beyond the
+// tensor are clipped.  Coordinates must not be negative, c0 * element size a multiple of 16 bytes.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src_saddr, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src_saddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all committed stores have finished READING shared memory (the buffer may be overwritten)
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all committed stores are complete
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");

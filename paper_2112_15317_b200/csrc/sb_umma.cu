@@ -1153,6 +1153,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
             static const bool off = [] { const char* e = getenv("SB_CONV_IN_UMMA"); return e && e[0] == '0'; }();
             if (!off) {
                 if (!mat_map(&um.wgrad.mapA, lv.dact, (long)B * lv.H * lv.W, lv.Cout, 64)) return fail_plan();
+                if (!mat_map(&um.fwd.mapA, lv.act, (long)B * lv.H * lv.W, lv.Cout, 128)) return fail_plan();
                 um.conv_in = true;
             }
         }

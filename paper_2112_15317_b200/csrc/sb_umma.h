@@ -16,7 +16,8 @@ struct UmmaOp {
 };
 struct UmmaLayer {
     UmmaOp fwd, dgrad, wgrad;
-    bool conv_in = false;                // input-layer conv on the tensor cores (wgrad.mapA then maps this layer's dy)
+    bool conv_in = false;                // input-layer conv on the tensor cores (wgrad.mapA then maps this layer's dy,
+                                         // fwd.mapA its output for the TMA store)
     const void* bound_input = nullptr;   // layer 0 only: the input buffer the tensor maps currently point at
 };
 
@@ -71,7 +72,8 @@ sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
 bool conv_in_umma_supported(int Cin, int Cout);
 // Partial buffers the weight-gradient kernel writes ([blocks][Cout*9*Cin + Cout] floats, reduced in block order).
 int conv_in_umma_wgrad_blocks(long npix);
-cudaError_t launch_conv_in_fwd_umma(const ConvSimtArgs& a, uint32_t* status, cudaStream_t st);
+// mapY: optional tensor map of the output as [pixels][Cout] with a (64, 128) box (nullptr: plain stores)
+cudaError_t launch_conv_in_fwd_umma(const ConvSimtArgs& a, const CUtensorMap* mapY, uint32_t* status, cudaStream_t st);
 cudaError_t launch_conv_in_wgrad_umma(const WgradSimtArgs& a, const CUtensorMap& mapDy, uint32_t* status, cudaStream_t st);
 
 const char* umma_last_error();
