@@ -58,6 +58,7 @@ struct UmmaParams {
     float* part;          // FWD/DGRAD with splits > 1: raw float partial sums [split][pixel][n_total]
     // epilogue
     int epi, relu, out_f32;
+    int tma_out;          // FWD/DGRAD, bf16 output, no split: the tile is staged in shared memory and written by TMA stores (map C)
     void* out;            // FWD/DGRAD: [pixels][ldc] bf16 (or float when out_f32); WGRAD: float partial sums
     long ldc;
     const float* bias;
@@ -86,7 +87,7 @@ template <int MODE, int BN> struct Cfg {
 // writes them as raw split partial sums, or with bias + ReLU / the ReLU mask applied, as float or bf16.
 template <int MODE, int BN>
 __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, bool row_ok, size_t row_off, int n0, int n_hi,
-                                          int split, const float* s_bias)
+                                          int split, const float* s_bias, uint8_t* stage = nullptr, int row = 0)
 {
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 16) {
@@ -154,8 +155,16 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
                     __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
                     pk[j] = *(uint32_t*)&t;
                 }
-                ((uint4*)op)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                ((uint4*)op)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                if (stage != nullptr) {
+                    // TMA-store staging: 64-column slabs of 128 rows x 128 bytes in the 128-byte swizzle of the tensor map
+                    uint8_t* slab = stage + (c0 >> 6) * 16384 + row * 128;
+                    const int j0 = (c0 & 63) >> 3;
+                    *(uint4*)(slab + ((j0 ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *(uint4*)(slab + (((j0 + 1) ^ (row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                } else {
+                    ((uint4*)op)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    ((uint4*)op)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
             } else {
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
@@ -170,7 +179,8 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
 // ------------------------------------------------------------------------------------------------
 template <int MODE, int BN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
-umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaParams p)
+umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+            const UmmaParams p)
 {
     using C = Cfg<MODE, BN>;
     extern __shared__ uint8_t smem_raw[];
@@ -418,13 +428,23 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias);
+            // (the operand ring is idle once the accumulator is complete: its first bytes stage the output tile)
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, (MODE != MODE_WGRAD && p.tma_out) ? smem : nullptr, row);
+            if (MODE != MODE_WGRAD && p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
 
     // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
     tc_fence_before();
     __syncthreads();
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) {
+        // one 64-column slab per store: rows outside the image and columns outside the tensor are clipped
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j)
+            if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(smem) + j * 16384, n0 + 64 * j, pw0, ph0, pn0);
+        tma_store_commit();
+        tma_store_wait_all();
+    }
     if (tlog && threadIdx.x == 0) { tlog[5] = (unsigned long long)clock64(); tlog[7] = globaltimer_ns(); }   // epilogue done
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
@@ -529,7 +549,8 @@ template <int BN> struct PairCfg {
 
 template <int MODE, int BN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
-umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaParams p)
+umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+                 const UmmaParams p)
 {
     static_assert(MODE != MODE_WGRAD && BN >= 128, "pair kernel: FWD / DGRAD with N tiles of 128 or 256");
     using C = PairCfg<BN>;
@@ -683,7 +704,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             const bool row_ok = w < p.W && h < p.H && n < p.N;
             const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, p.tma_out ? smem : nullptr, row);
+            if (p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
 
@@ -696,6 +718,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         __syncthreads();
     }
     cluster_sync_all();    // neither CTA leaves (or frees TMEM) while its partner may still signal or read it
+    if (p.tma_out && threadIdx.x == 64 && !*abort_flag) {
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j)
+            if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(smem) + j * 16384, n0 + 64 * j, pw0, ph0, pn0);
+        tma_store_commit();
+        tma_store_wait_all();
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
@@ -789,7 +818,7 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
         attr_set = true;
     }
     if (p.stages < 1 || p.stages > Cfg<MODE, BN>::MAX_STAGES_FIT) return cudaErrorInvalidValue;
-    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, p);
+    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, op.mapC, p);
 }
 
 // CTA-pair launch: clusters of two CTAs along x, programmatic dependent launch as everywhere else.
@@ -816,7 +845,7 @@ static cudaError_t launch_pair_one(const UmmaOp& op, const UmmaParams& p, dim3 g
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<MODE, BN>, op.mapA, op.mapB, p);
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<MODE, BN>, op.mapA, op.mapB, op.mapC, p);
 }
 template <int MODE>
 static cudaError_t launch_pair_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
@@ -1139,6 +1168,20 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
     b->rows = (long)rows;
 }
 
+// TMA-store epilogue of a FWD / DGRAD op: possible when the output is bf16, the reduction is not split, every N tile
+// ends on a 64-column slab boundary inside its shard, and the idle operand ring can hold the staged tile.
+// SB_TMA_OUT=0 keeps the direct row stores.
+static bool tma_out_ok(const OpBlock* b, int cols_per_shard, int shards)
+{
+    static const bool off = [] { const char* e = getenv("SB_TMA_OUT"); return e && e[0] == '0'; }();
+    const UmmaParams& p = b->p;
+    if (off || p.out_f32 || p.splits > 1 || p.epi == UEPI_F32) return false;
+    if (p.n_total % 64 != 0 || p.ldc % 64 != 0) return false;
+    if (shards > 1 && (cols_per_shard % b->bn != 0 || p.n_total % shards != 0)) return false;
+    const long stage_bytes = b->pair ? 16384 + b->bn * 64 : 16384 + b->bn * 128;
+    return (long)p.stages * stage_bytes >= (long)(b->bn / 64) * 16384;
+}
+
 sb_status umma_plan_layers(sb_model* m, int first_layer)
 {
     ModelView mv = model_view(m);
@@ -1174,6 +1217,10 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 apply_plan(b, g.fwd, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
+                if (tma_out_ok(b, lv.Cout, 1)) {
+                    if (!act_map(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
+                    p.tma_out = 1;
+                }
                 um.fwd.enabled = true;
             }
             // ---- data gradient ----
@@ -1191,6 +1238,10 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 apply_plan(b, g.dgrad, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
                 if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, 64)) return fail_plan();
+                if (tma_out_ok(b, lv.Cin, 1)) {
+                    if (!act_map(&um.dgrad.mapC, lv.d_below, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
+                    p.tma_out = 1;
+                }
                 um.dgrad.enabled = true;
             }
             // ---- weight gradient ----
@@ -1251,6 +1302,10 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 if (p.splits > 1 && (size_t)p.splits * (size_t)p.split_stride > mv.ws_floats) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.fwd.mapA, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
+                if (tma_out_ok(b, cdiv_i(lv.out_f, K), K)) {
+                    if (!act_map(&um.fwd.mapC, lv.act, B, 1, 1, lv.out_f, 1, 1, 128)) return fail_plan();
+                    p.tma_out = 1;
+                }
                 um.fwd.enabled = true;
             }
             // ---- data gradient: dX = sum_j dY_j W_j = one reduction over the concatenated width ----
@@ -1269,6 +1324,10 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 if (p.splits > 1 && (size_t)p.splits * (size_t)p.split_stride > mv.ws_floats) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.dgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 128)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.out_f, lv.in_f, 64)) return fail_plan();
+                if (tma_out_ok(b, lv.in_f, 1)) {
+                    if (!act_map(&um.dgrad.mapC, lv.d_below, B, 1, 1, lv.in_f, 1, 1, 128)) return fail_plan();
+                    p.tma_out = 1;
+                }
                 um.dgrad.enabled = true;
             }
             // ---- weight gradient: dW_j = dY_j^T X ; M tiles enumerated per shard (needs 16-byte aligned shard starts) ----
