@@ -42,7 +42,7 @@ LR, MU = 0.01, 0.9
 # layers: plain SGD at 0.01 is at its stability limit there (at the ImageNet shape it diverges within three steps, loss
 # 11 -> 18 -> 274; at the CIFAR shape some summation orders diverge after several hundred repetitions).  The step time
 # does not depend on the values, but a finite, falling loss is reported, so the VGG configurations train at smaller rates.
-LR_BY_CONFIG = {1: 2.0e-3, 2: 2.0e-3, 3: 1.0e-4}
+LR_BY_CONFIG = {1: 2.0e-3, 2: 1.0e-3, 3: 1.0e-4}
 
 
 def peaks():
