@@ -265,6 +265,15 @@ sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32
  */
 sb_status sb_debug_cta_timing(void* dev_buffer);
 
+/*
+ * Self-test of the hang-safety path.  Every wait inside the library's kernels is bounded; a wait that runs out makes
+ * the kernel record a code in the model's device status word and return normally, and the next sb_loss (or
+ * sb_train_step_host) returns SB_ERR_TIMEOUT and clears the word.  This call enqueues one CTA that waits limit_ms
+ * (1..1000) on a barrier that nothing completes and then reports in that way, so that a caller (or a test) can see
+ * the whole path work without a stalled pipeline.  The GPU context stays usable.  No counterpart in the paper.
+ */
+sb_status sb_debug_wait_probe(sb_model* m, int32_t limit_ms, void* stream);
+
 /* Number of kernels the last sb_forward + sb_backward + sb_sgd_step enqueued (host counter). */
 sb_status sb_launch_count(const sb_model* m, int64_t* launches);
 

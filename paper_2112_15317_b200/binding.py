@@ -63,6 +63,7 @@ def _load():
         "sb_backward": [c_void_p, c_void_p],
         "sb_graph_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
         "sb_modulo_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
+        "sb_debug_wait_probe": [c_void_p, c_int32, c_void_p],
         "sb_sgd_step": [c_void_p, c_float, c_float, c_void_p],
         "sb_loss": [c_void_p, c_void_p, P(c_float)],
         "sb_train_step_host": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p, P(c_float)],
@@ -101,6 +102,7 @@ sb_forward = _lib.sb_forward
 sb_backward = _lib.sb_backward
 sb_graph_step = _lib.sb_graph_step
 sb_modulo_step = _lib.sb_modulo_step
+sb_debug_wait_probe = _lib.sb_debug_wait_probe
 sb_sgd_step = _lib.sb_sgd_step
 sb_loss = _lib.sb_loss
 sb_train_step_host = _lib.sb_train_step_host
@@ -236,6 +238,10 @@ class Model:
         """One iteration in the modulo layer's sub-iteration schedule (model created with SB_FLAG_MODULO_SCHEDULE)."""
         xp, lp = self._ptr_arrays(xs, labels)
         _check(sb_modulo_step(self.h, xp, lp, c_float(lr), c_float(momentum), self._stream()))
+
+    def debug_wait_probe(self, limit_ms=20):
+        """Enqueue the bounded-wait self-test; the next loss() raises SB_ERR_TIMEOUT."""
+        _check(sb_debug_wait_probe(self.h, c_int32(limit_ms), self._stream()))
 
     def sgd_step(self, lr, momentum):
         _check(sb_sgd_step(self.h, c_float(lr), c_float(momentum), self._stream()))

@@ -1238,6 +1238,14 @@ sb_status sb_debug_cta_timing(void* dev_buffer)
     return SB_OK;
 }
 
+sb_status sb_debug_wait_probe(sb_model* m, int32_t limit_ms, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    if (limit_ms < 1 || limit_ms > 1000) return fail(SB_ERR_INVALID_ARG, "limit_ms must be in 1..1000");
+    CU_TRY(launch_wait_probe(m->status, (unsigned long long)limit_ms * 1000000ull, (cudaStream_t)stream));
+    return SB_OK;
+}
+
 sb_status sb_launch_count(const sb_model* m, int64_t* launches)
 {
     if (!m || !launches) return fail(SB_ERR_INVALID_ARG, "null argument");

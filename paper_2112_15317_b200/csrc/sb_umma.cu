@@ -914,6 +914,30 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
 
 const char* umma_last_error() { return g_umma_err; }
 
+// Self-test of the bounded-wait path: one CTA waits on an mbarrier that nothing will ever complete, with the same
+// polling loop as the pipeline waits but a limit of `limit_ns`; when the limit passes it records DEV_TIMEOUT_EPI in the
+// status word and returns normally, exactly as a stalled pipeline would.
+__global__ void __launch_bounds__(32) wait_probe_kernel(uint32_t* status, unsigned long long limit_ns)
+{
+    __shared__ uint64_t never;
+    if (threadIdx.x == 0) {
+        mbar_init(&never, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint64_t t0 = globaltimer_ns();
+        bool done = false;
+        for (uint32_t it = 0; it < (1u << 28) && !done; ++it) {
+            done = mbar_try_wait(&never, 0);
+            if ((it & 255u) == 255u && globaltimer_ns() - t0 > limit_ns) break;
+        }
+        if (!done) atomicMax(status, (uint32_t)DEV_TIMEOUT_EPI);
+    }
+}
+cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cudaStream_t st)
+{
+    wait_probe_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 // Tile plan of a FWD / DGRAD GEMM: N tile, reduction split and ring depth.
 //  * N tile as wide as the column count allows (operand traffic from L2 per FLOP falls with the tile width),
 //  * if that leaves fewer CTAs than ~0.8 waves, split the reduction over blockIdx.z (float partial sums,

@@ -349,3 +349,22 @@ def test_state_and_argument_errors():
     with pytest.raises(b.SBError):
         gm.read(b.SB_T_WEIGHT, 4, 5)          # shard out of range
     gm.close()
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """The hang-safety path end to end: a wait that runs out (20 ms, on a barrier nothing completes) becomes
+    SB_ERR_TIMEOUT at the next sb_loss, the status word is cleared, and the model keeps working."""
+    b = sb()
+    wl = WORKLOADS["cfg0"]()
+    params = si.make_params(wl)
+    x, y = si.make_batch(wl)
+    gm = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    gm.forward(xs, ys)
+    good = gm.loss()
+    gm.debug_wait_probe(20)
+    with pytest.raises(b.SBError, match="SB_ERR_TIMEOUT"):
+        gm.loss()
+    gm.forward(xs, ys)
+    assert gm.loss() == good          # status cleared, same result as before
+    gm.close()
