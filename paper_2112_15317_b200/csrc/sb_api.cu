@@ -554,11 +554,19 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
             if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(ws_w, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
         }
-        if (!l.thin_input && !l.um.wgrad.enabled && (part & SIDE_W)) {
+        if (!l.thin_input && (part & SIDE_W) && (!l.um.wgrad.enabled || !umma_wgrad_bias_fused(m, i))) {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
             const long M = (long)B * l.H * l.W;
             // (stream order makes it safe to reuse the scratch the weight-gradient reduce just read)
-            const int S = l.bg_splits;
+            int S = l.bg_splits;
+            if (bf && l.Cout % 8 == 0) {
+                // the vectorised column-sum kernel covers 256 columns per block column: split the rows finely enough to
+                // fill the machine (its splits need not be whole images), within the scratch
+                long want = 592 / ((l.Cout / 8 + 31) / 32);
+                if (want > M / 64) want = M / 64;
+                if (want > (long)(m->ws_floats / l.n_b)) want = (long)(m->ws_floats / l.n_b);
+                S = want < 1 ? 1 : (int)want;
+            }
             float* part = S > 1 ? ws_w : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
             if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, l.n_b, m->Gm + l.p_b, l.n_b, S, st));

@@ -259,8 +259,60 @@ colsum_kernel(const T* __restrict__ in, float* __restrict__ part, int M, int N, 
         part[(size_t)sp * N + col] = t;
     }
 }
+// bf16, N a multiple of 8: a thread owns 8 adjacent columns (one 16-byte load per row), 8 row lanes per block take rows
+// r0 + lane_row, + 8, ... with four independent loads in flight and are combined in lane order (deterministic).
+__global__ void __launch_bounds__(256)
+colsum_vec_kernel(const uint4* __restrict__ in, float* __restrict__ part, int M, int N, int splits)
+{
+    pdl_prologue();
+    __shared__ float s[8][32][9];
+    const int nv = N / 8;
+    const int vc = blockIdx.x * 32 + threadIdx.x % 32;
+    const int lane_row = threadIdx.x / 32;
+    const int sp = blockIdx.y;
+    const long rows = (M + splits - 1) / splits, r0 = (long)sp * rows;
+    const long r1 = r0 + rows < M ? r0 + rows : M;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (vc < nv) {
+        long r = r0 + lane_row;
+        for (; r + 24 < r1; r += 32) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldg(in + (r + 8 * u) * nv + vc);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const __nv_bfloat16* h = (const __nv_bfloat16*)&v[u];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[j] += __bfloat162float(h[j]);
+            }
+        }
+        for (; r < r1; r += 8) {
+            const uint4 v = __ldg(in + r * nv + vc);
+            const __nv_bfloat16* h = (const __nv_bfloat16*)&v;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += __bfloat162float(h[j]);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[lane_row][threadIdx.x % 32][j] = acc[j];
+    __syncthreads();
+    if (lane_row == 0 && vc < nv) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float t = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t += s[i][threadIdx.x][j];
+            part[(size_t)sp * N + vc * 8 + j] = t;
+        }
+    }
+}
 cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st)
 {
+    if (bf16 && N % 8 == 0 && (((uintptr_t)in) & 15) == 0) {
+        dim3 vgrid(cdiv(N / 8, 32), splits);
+        SB_LAUNCH((colsum_vec_kernel), vgrid, 256, 0, st, (const uint4*)in, part, M, N, splits);
+        return cudaGetLastError();
+    }
     dim3 grid(cdiv(N, 32), splits);
     if (bf16) SB_LAUNCH((colsum_kernel<__nv_bfloat16>), grid, 256, 0, st, (const __nv_bfloat16*)in, part, M, N, splits);
     else SB_LAUNCH((colsum_kernel<float>), grid, 256, 0, st, (const float*)in, part, M, N, splits);

@@ -552,7 +552,7 @@ __global__ void __launch_bounds__(UMMA_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
                  const UmmaParams p)
 {
-    static_assert(MODE != MODE_WGRAD && BN >= 128, "pair kernel: FWD / DGRAD with N tiles of 128 or 256");
+    static_assert(BN == 128 || BN == 256, "pair kernel: N tiles of 128 or 256");
     using C = PairCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -570,10 +570,21 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const bool leader = rank == 0;
 
     // ---- tile coordinates (the pair shares blockIdx.y / blockIdx.z; its M tiles are 2j and 2j+1) ----
-    const int m_idx = blockIdx.x, n_idx = blockIdx.y, split = blockIdx.z;
-    const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
-    const int lo = (int)(((long)sh * p.n_total) / p.shards), n_hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
-    const int n0 = lo + t * BN;
+    // FWD / DGRAD: M tile = a 128-pixel box, N tile inside a shard.  WGRAD (conv layers, one tap per CTA, unsharded): M
+    // tile = 128 gradient rows (output channels), N tile = BN input channels, blockIdx.z = tap * splits + split.
+    const int m_idx = blockIdx.x, n_idx = blockIdx.y;
+    int split = blockIdx.z, tap_fixed = 0, n0, n_hi, m0 = 0, m_hi = 0;
+    if (MODE == MODE_WGRAD) {
+        tap_fixed = blockIdx.z / p.splits;
+        split = blockIdx.z % p.splits;
+        n0 = n_idx * BN; n_hi = p.n_total;
+        m0 = m_idx * 128; m_hi = p.m_total;
+    } else {
+        const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
+        const int lo = (int)(((long)sh * p.n_total) / p.shards);
+        n_hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
+        n0 = lo + t * BN;
+    }
     if (n0 >= n_hi) return;   // uniform over the pair, before any barrier or TMEM allocation
     // an M index past the last tile (odd tile count) lands wholly out of bounds: zero loads, no stores
     const int pw0 = (m_idx % p.tiles_w) * p.bw;
@@ -583,7 +594,14 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
     const int n_iters = k_end - k_begin;
 
-    int ld_a = k_begin % p.kchunks, ld_b = k_begin / p.kchunks;   // (k-chunk, tap) of the next load
+    // next load: FWD / DGRAD (k-chunk, tap); WGRAD pixel-box indices (w, h, n)
+    int ld_a, ld_b, ld_c = 0;
+    if (MODE == MODE_WGRAD) {
+        ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
+    } else {
+        ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+    }
+    const int wg_dr = tap_fixed / 3 - 1, wg_ds = tap_fixed % 3 - 1;
     const int nb0 = n0 + (int)rank * (BN / 2);                     // first B column this CTA fetches
     const uint32_t full0_leader = map_to_cta(smem_u32(&full[0]), 0);
     // (whole producer warp in lock-step, elected issue: see the single-CTA kernel)
@@ -594,18 +612,28 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const uint32_t sa = smem0 + ld_off, sb = sa + A_STAGE_BYTES;
         const uint32_t bar = full0_leader + (uint32_t)ld_s * 8u;
         if (leader) mbar_expect_tx_el(full0 + 8u * (uint32_t)ld_s, 2u * (uint32_t)C::STAGE_BYTES, el);
-        const int kc = ld_a, tap = ld_b;
-        int dr = 0, ds = 0;
-        if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
-        if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
-        tma_load_4d_pair_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
-        if (MODE == MODE_FWD) {
-            tma_load_4d_pair_el(&mapB, sb, bar, tap * p.w_cols + kc * 64, nb0, 0, 0, el);     // box of BN/2 rows
-        } else {
+        if (MODE == MODE_WGRAD) {
+            // A = this CTA's 128 gradient rows of dy (two 64-channel boxes), B = its half of the shifted activations
+            const int cw = ld_a * p.bw, ch = ld_b * p.bh, cn = ld_c * p.bn;
+            tma_load_4d_pair_el(&mapA, sa, bar, m0, cw, ch, cn, el);
+            tma_load_4d_pair_el(&mapA, sa + 8192, bar, m0 + 64, cw, ch, cn, el);
 #pragma unroll
-            for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair_el(&mapB, sb + j * 8192, bar, tap * p.w_cols + nb0 + 64 * j, kc * 64, 0, 0, el);
+            for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair_el(&mapB, sb + j * 8192, bar, nb0 + 64 * j, cw + wg_ds, ch + wg_dr, cn, el);
+            if (++ld_a == p.tiles_w) { ld_a = 0; if (++ld_b == p.tiles_h) { ld_b = 0; ++ld_c; } }
+        } else {
+            const int kc = ld_a, tap = ld_b;
+            int dr = 0, ds = 0;
+            if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
+            if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
+            tma_load_4d_pair_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
+            if (MODE == MODE_FWD) {
+                tma_load_4d_pair_el(&mapB, sb, bar, tap * p.w_cols + kc * 64, nb0, 0, 0, el);     // box of BN/2 rows
+            } else {
+#pragma unroll
+                for (int j = 0; j < BN / 128; ++j) tma_load_4d_pair_el(&mapB, sb + j * 8192, bar, tap * p.w_cols + nb0 + 64 * j, kc * 64, 0, 0, el);
+            }
+            if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
         }
-        if (++ld_a == p.kchunks) { ld_a = 0; ++ld_b; }
         ++ld_s; ld_off += (uint32_t)C::STAGE_BYTES;
         if (ld_s == STAGES) { ld_s = 0; ld_off = 0; }
     };
@@ -657,17 +685,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     } else if (warp == 1) {
         if (leader) {
             // (converged warp, elected issue: see the single-CTA kernel)
-            constexpr uint32_t idesc = make_idesc(BN, 0, MODE != MODE_FWD, 256);
+            constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_WGRAD, MODE != MODE_FWD, 256);
             const uint32_t elected = elect_one() ? 1u : 0u;
             // the MMA addresses both accumulators with one TMEM address: the pair must have been given the same columns
             bool ok = ld_cluster_u32(map_to_cta(smem_u32(tmem_slot), 1)) == tmem_base;
             if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_PAIR_TMEM); }
             const uint32_t sa0 = smem_u32(smem);
-            const uint64_t dA0 = make_desc(sa0, 16);
+            const uint64_t dA0 = (MODE == MODE_WGRAD) ? make_desc(sa0, 8192) : make_desc(sa0, 16);
             const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(sa0 + A_STAGE_BYTES, 16) : make_desc(sa0 + A_STAGE_BYTES, 8192);
             const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
             const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
-            constexpr uint32_t A_STEP = 32u >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
+            constexpr uint32_t A_STEP = ((MODE == MODE_WGRAD) ? 2048u : 32u) >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
             constexpr uint32_t STAGE16 = (uint32_t)C::STAGE_BYTES >> 4;
             int s = 0;
             uint32_t ph = 0, off = 0;
@@ -699,13 +727,21 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
             tc_fence_after();
-            const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
-            const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
-            const bool row_ok = w < p.W && h < p.H && n < p.N;
-            const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+            bool row_ok;
+            size_t row_off;
+            if (MODE == MODE_WGRAD) {
+                row_ok = (m0 + row) < m_hi;
+                row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
+            } else {
+                const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
+                const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+                row_ok = w < p.W && h < p.H && n < p.N;
+                row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, p.tma_out ? smem : nullptr, row);
-            if (p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const bool staged_out = MODE != MODE_WGRAD && p.tma_out;
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, staged_out ? smem : nullptr, row);
+            if (staged_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
 
@@ -718,7 +754,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         __syncthreads();
     }
     cluster_sync_all();    // neither CTA leaves (or frees TMEM) while its partner may still signal or read it
-    if (p.tma_out && threadIdx.x == 64 && !*abort_flag) {
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) {
 #pragma unroll
         for (int j = 0; j < BN / 64; ++j)
             if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(smem) + j * 16384, n0 + 64 * j, pw0, ph0, pn0);
@@ -892,6 +928,7 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     pp.timing = g_timing;
     if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_DGRAD) e = launch_pair_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
+    else if (b->pair && b->p.mode == MODE_WGRAD) e = launch_pair_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
     else if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->p.mode == MODE_DGRAD) e = launch_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
     else e = launch_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
@@ -1297,6 +1334,21 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 // weights (Cout*9*Cin is a multiple of 64 here), and a split buffer uses the same layout
                 p.split_stride = (long)(lv.n_w + lv.n_b);
                 p.bias_fused = 1; p.bias_off = (long)lv.n_w;
+                {
+                    // CTA pairs over two neighbouring blocks of 128 output channels: each CTA fetches half of the
+                    // activation tile (a smaller stage, a deeper ring in the same shared memory).  The pair kernel
+                    // does not sum dy on the side, so the bias gradient is taken by a column-sum kernel (wgrad_pair).
+                    static const bool wg_pair = [] { const char* e = getenv("SB_WG_PAIR"); return !(e && e[0] == '0'); }();
+                    if (wg_pair && p.tap_group == 1 && (b->bn == 128 || b->bn == 256) && g.wg_m_tiles % 2 == 0 && lv.Cout % 128 == 0) {
+                        b->pair = 1;
+                        p.bias_fused = 0;
+                        const int pfit = b->bn >= 256 ? 6 : 8, ptwo = b->bn >= 256 ? 3 : 4;
+                        int pst = g.wg_cps < pfit ? g.wg_cps : pfit;
+                        const long ctas = (long)g.wg_m_tiles * g.wg_n_tiles * 9 * p.splits;
+                        if (bwd_cohabit() && ctas >= 100 && pst > ptwo) pst = ptwo;
+                        p.stages = pst < 1 ? 1 : pst;
+                    }
+                }
                 p.out = p.splits > 1 ? (void*)mv.ws_wk[mv.n_wstreams > 0 ? i % mv.n_wstreams : 0] : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
                 b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 / p.tap_group * p.splits));
@@ -1403,6 +1455,12 @@ sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st) { return laun
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st, launch_counter(m)); }
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st, launch_counter(m)); }
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->wgrad, st); }
+
+bool umma_wgrad_bias_fused(sb_model* m, int layer)
+{
+    const UmmaLayer& um = *layer_view(m, layer).um;
+    return um.wgrad.enabled && blk(um.wgrad)->p.bias_fused != 0;
+}
 
 sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part)
 {

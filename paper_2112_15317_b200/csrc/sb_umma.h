@@ -63,6 +63,8 @@ sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st);
 // Launches the weight-gradient kernel; *splits > 1 means it wrote split partial sums at *part
 // (to be reduced in split order by the caller), else it wrote the gradient itself.
 sb_status umma_conv_wgrad_launch(sb_model* m, int layer, cudaStream_t st, int* splits, float** part);
+// false: the layer's weight-gradient kernel (CTA-pair variant) leaves the bias gradient to a column-sum kernel
+bool umma_wgrad_bias_fused(sb_model* m, int layer);
 // First-layer FC: points the tensor maps that read the network input at `x` ([B, in] contiguous, bf16).
 sb_status umma_bind_input(sb_model* m, const void* x);
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
