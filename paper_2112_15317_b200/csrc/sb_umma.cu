@@ -1104,9 +1104,13 @@ static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_
     const double chunk_us = chunk_scale * (16384.0 + bn * 128.0) / 122.0e3;     // bytes per chunk at ~122 GB/s of L2 per SM
     const double fixed_us = 3.0 + bn / 256.0 * 1.5;               // CTA start + drain + float epilogue
     double best = 1e30; int best_s = 1;
-    for (int s = 1; s <= 256; s *= 2) {
+    for (int s = 1; s <= 256; ++s) {
         const int cps = cdiv_i(total_chunks, s);
         if (s > 1 && cps < 2) break;
+        // Short kernels may take any split count (3 tap rows x 48 splits = 144 CTAs fill the machine: -1.2 % step at
+        // CIFAR size); long ones (>= 256 chunks per CTA, ImageNet size) keep to powers of two, which leaves a third of
+        // the SMs to the data-gradient kernel they run beside (filling the machine there measured +2.5 % step).
+        if ((s & (s - 1)) != 0 && cps >= 256) continue;
         const int real_s = cdiv_i(total_chunks, cps);
         const long ctas = ctas_without_split * real_s;
         const long waves = (ctas + 147) / 148;
