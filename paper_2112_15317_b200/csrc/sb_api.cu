@@ -96,6 +96,10 @@ struct sb_model {
     float *row_loss = nullptr, *loss = nullptr;
     unsigned int* counter = nullptr;
     uint32_t* status = nullptr;
+    // Set by the multi-stream backward pass while it enqueues the weight side of one conv layer: the layer's split
+    // reduces then apply the update themselves (launch_reduce_sgd) once `ev` (the layer's input-gradient kernel, which
+    // reads the weights) has passed; `covered` counts the parameters updated that way.
+    struct { bool on = false; float lr = 0.f, mu = 0.f; cudaEvent_t ev = nullptr; bool waited = false; size_t covered = 0; } fuse;
     char* stage_x = nullptr;
     int32_t* stage_labels = nullptr;
     char* input_grad = nullptr;
@@ -517,6 +521,26 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
         if (i == 0 && !m->have_x) return fail(SB_ERR_STATE, "layer 0 needs input pointers");
         const double pix = (double)B * l.H * l.W;
         const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
+        // End of a gradient range [goff, goff + n) of this layer: S > 1 partial copies at `src` are reduced in order into
+        // the gradient arena -- or, when the backward pass folds the update in, reduced and applied in one kernel (S = 1:
+        // the gradient is already in the arena and takes a plain update).
+        const bool fuse = m->fuse.on && (part & SIDE_W) && !(part & SIDE_D) && l.n_w % 4 == 0 && l.n_b % 4 == 0 && l.p_w % 4 == 0 && l.p_b % 4 == 0;
+        auto finish = [&](const float* src, size_t stride, size_t goff, size_t n, int S) -> sb_status {
+            if (!fuse) {
+                if (S > 1) L_TRY("split_reduce", 0.0, (double)n * 4.0 * (S + 1), launch_reduce_partials(src, stride, m->Gm + goff, n, S, st));
+                return SB_OK;
+            }
+            if (!m->fuse.waited) { CU_TRY(cudaStreamWaitEvent(st, m->fuse.ev, 0)); m->fuse.waited = true; }
+            __nv_bfloat16* sh = m->Sm ? m->Sm + goff : nullptr;
+            if (S > 1)
+                L_TRY("split_reduce_sgd", 0.0, (double)n * (4.0 * S + (m->bf16 ? 18.0 : 16.0)),
+                      launch_reduce_sgd(src, stride, n, S, m->Wm + goff, m->Vm + goff, sh, m->fuse.lr, m->fuse.mu, st));
+            else
+                L_TRY("sgd", 0.0, (double)n * (m->bf16 ? 22.0 : 20.0), launch_sgd(m->Wm + goff, m->Vm + goff, m->Gm + goff, sh, n, m->fuse.lr, m->fuse.mu, st));
+            m->fuse.covered += n;
+            return SB_OK;
+        };
+        sb_status fs = SB_OK;
         // weight gradient over all replicas' pixels (the DP reduce is the sum over image ranges)
         if (!(part & SIDE_W)) {
         } else if (l.thin_input) {
@@ -532,19 +556,23 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
                 L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
             if (l.p_b == l.p_w + l.n_w) {
                 // the bias vector directly follows the weights in the gradient arena, as it does in a partial buffer
-                L_TRY("split_reduce", 0.0, (double)stride * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, stride, nb, st));
+                if ((fs = finish(ws_w, stride, l.p_w, stride, nb)) != SB_OK) return fs;
             } else {
-                L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (nb + 1), launch_reduce_partials(ws_w, stride, m->Gm + l.p_w, l.n_w, nb, st));
-                L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (nb + 1), launch_reduce_partials(ws_w + l.n_w, stride, m->Gm + l.p_b, l.n_b, nb, st));
+                if ((fs = finish(ws_w, stride, l.p_w, l.n_w, nb)) != SB_OK) return fs;
+                if ((fs = finish(ws_w + l.n_w, stride, l.p_b, l.n_b, nb)) != SB_OK) return fs;
             }
         } else if (l.um.wgrad.enabled) {
             int S = 1;
             float* part = nullptr;
             U_TRY("conv_wgrad_umma", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, umma_conv_wgrad_launch(m, i, st, &S, &part));
             ++m->launches;
-            // weights and bias gradient reduce together (same layout in the split buffers and in the arena)
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)(l.n_w + l.n_b) * 4.0 * (S + 1),
-                             launch_reduce_partials(part, l.n_w + l.n_b, m->Gm + l.p_w, l.n_w + l.n_b, S, st));
+            // weights and bias gradient reduce together (same layout in the split buffers and in the arena); a kernel
+            // that leaves the bias gradient to the column-sum pass below reduces (or updates) the weights only
+            const bool with_bias = umma_wgrad_bias_fused(m, i) && l.p_b == l.p_w + l.n_w;
+            if (with_bias || S > 1 || fuse) {
+                if (with_bias || !fuse) { if ((fs = finish(part, l.n_w + l.n_b, l.p_w, l.n_w + l.n_b, S)) != SB_OK) return fs; }
+                else if ((fs = finish(part, l.n_w + l.n_b, l.p_w, l.n_w, S)) != SB_OK) return fs;
+            }
         } else {
             const int S = l.wg_splits;
             WgradSimtArgs a{};
@@ -552,7 +580,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             a.dy = l.dact; a.part = S > 1 ? ws_w : m->Gm + l.p_w;
             a.B = B; a.H = l.H; a.W = l.W; a.Cin = l.Cin; a.Cout = l.Cout; a.splits = S;
             L_TRY("conv_wgrad_simt", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_wgrad_simt(a, bf, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_w * 4.0 * (S + 1), launch_reduce_partials(ws_w, l.n_w, m->Gm + l.p_w, l.n_w, S, st));
+            if ((fs = finish(ws_w, l.n_w, l.p_w, l.n_w, S)) != SB_OK) return fs;
         }
         if (!l.thin_input && (part & SIDE_W) && (!l.um.wgrad.enabled || !umma_wgrad_bias_fused(m, i))) {
             // bias gradient: column sums of dY over image-range splits, then the same ordered reduce
@@ -569,7 +597,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             }
             float* part = S > 1 ? ws_w : m->Gm + l.p_b;
             L_TRY("bias_grad", 0.0, pix * l.Cout * e, launch_colsum(l.dact, bf, part, (int)M, l.Cout, S, st));
-            if (S > 1) L_TRY("split_reduce", 0.0, (double)l.n_b * 4.0 * (S + 1), launch_reduce_partials(part, l.n_b, m->Gm + l.p_b, l.n_b, S, st));
+            if ((fs = finish(part, l.n_b, l.p_b, l.n_b, S)) != SB_OK) return fs;
         }
         if (want_in_grad && (part & SIDE_D)) {
             const double bytes = pix * (l.Cin + l.Cout) * e + (double)l.n_w * e + (below_relu ? pix * l.Cin * e : 0.0);
@@ -875,14 +903,31 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
             used_streams |= 1u << (i % m->n_wstreams);
             CU_TRY(cudaEventRecord(m->ev_ready[i], st));
             CU_TRY(cudaStreamWaitEvent(wst, m->ev_ready[i], 0));
-            sb_status s = backward_layer(m, i, wst, SIDE_W);
-            if (s != SB_OK) return s;
-            s = backward_layer(m, i, st, SIDE_D);
-            if (s != SB_OK) return s;
+            // Conv layers in a fused pass: the input-gradient kernel is enqueued first and its event recorded, so that the
+            // layer's split reduces on the weight stream can wait for it and apply the update themselves.
+            static const bool reduce_updates = [] { const char* e = getenv("SB_REDUCE_SGD"); return !(e && e[0] == '0'); }();
+            const bool in_reduce = fuse && reduce_updates && l.kind == SB_CONV3X3_RELU;
+            sb_status s = SB_OK;
+            if (in_reduce) {
+                s = backward_layer(m, i, st, SIDE_D);
+                if (s != SB_OK) return s;
+                CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
+                m->fuse.on = true; m->fuse.lr = lr; m->fuse.mu = mu; m->fuse.ev = m->ev_dgrad[i]; m->fuse.waited = false; m->fuse.covered = 0;
+                s = backward_layer(m, i, wst, SIDE_W);
+                m->fuse.on = false;
+                if (s != SB_OK) return s;
+                if (m->fuse.covered == l.n_w + l.n_b) continue;     // every parameter of the layer has taken its update
+                if (m->fuse.covered != 0) return fail(SB_ERR_STATE, "layer %d: update folded into part of its reduces only", i);
+            } else {
+                s = backward_layer(m, i, wst, SIDE_W);
+                if (s != SB_OK) return s;
+                s = backward_layer(m, i, st, SIDE_D);
+                if (s != SB_OK) return s;
+            }
             if (fuse) {
                 // The update of this layer runs on a third stream: after the layer's gradients are complete (weight
                 // stream) and after its input-gradient kernel, which reads the weights the update rewrites (main stream).
-                CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
+                if (!in_reduce) CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
                 CU_TRY(cudaEventRecord(m->ev_wdone[i], wst));
                 CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_dgrad[i], 0));
                 CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_wdone[i], 0));

@@ -113,6 +113,9 @@ cudaError_t launch_fc_narrow(const FcNarrowArgs& a, bool bf16, cudaStream_t st);
 cudaError_t launch_colsum(const void* in, bool bf16, float* part, int M, int N, int splits, cudaStream_t st);
 // out[i] = sum_{s<splits} part[s*stride + i], s ascending.
 cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st);
+// the same ordered sum, consumed at once by the SGD step of the n parameters at w / v (shadow: their bf16 copies or nullptr)
+cudaError_t launch_reduce_sgd(const float* part, size_t stride, size_t n, int splits, float* w, float* v, __nv_bfloat16* shadow,
+                              float lr, float mu, cudaStream_t st);
 
 struct PoolArgs {
     const void* x;  // [B,H,W,C]

@@ -716,6 +716,88 @@ sgd_kernel(float4* __restrict__ w, float4* __restrict__ v, const float4* __restr
         __stcs(w + i, ww);
     }
 }
+// Ordered split reduce and update in one pass: g = sum_s part[s] (the same kernels' split order as
+// launch_reduce_partials, so the gradient has the same bits), then the SGD step on w, v (and the bf16 copy) without
+// the gradient ever being written to or read back from the gradient arena.
+template <bool SHADOW>
+__global__ void __launch_bounds__(256)
+reduce_sgd4_kernel(const float4* __restrict__ part, size_t stride4, int splits, float4* __restrict__ w, float4* __restrict__ v,
+                   uint2* __restrict__ shadow, size_t n4, float lr, float mu)
+{
+    pdl_prologue();
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 ww = w[i], vv = v[i];
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = 0; s0 < splits; s0 += 8) {
+            float4 pv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                pv[u] = (s0 + u < splits) ? __ldg(part + (size_t)(s0 + u) * stride4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { t.x += pv[u].x; t.y += pv[u].y; t.z += pv[u].z; t.w += pv[u].w; }
+        }
+        sgd_apply<SHADOW>(ww, vv, t, lr, mu, SHADOW ? shadow + i : nullptr);
+        v[i] = vv;
+        w[i] = ww;
+    }
+}
+__device__ __forceinline__ void sgd_apply_scalar(float* w, float* v, float g, __nv_bfloat16* shadow, size_t i, float lr, float mu)
+{
+    const float vv = fmaf(mu, v[i], g), ww = fmaf(-lr, vv, w[i]);
+    v[i] = vv;
+    w[i] = ww;
+    if (shadow) shadow[i] = __float2bfloat16_rn(ww);
+}
+__global__ void __launch_bounds__(256)
+reduce_sgd_many_kernel(const float* __restrict__ part, size_t stride, int splits, float* __restrict__ w, float* __restrict__ v,
+                       __nv_bfloat16* __restrict__ shadow, size_t n, float lr, float mu)
+{
+    pdl_prologue();
+    __shared__ float s[8][33];
+    const int e = threadIdx.x % 32, lane = threadIdx.x / 32;
+    const size_t i = blockIdx.x * 32ull + e;
+    float t = 0.f;
+    if (i < n)
+        for (int sp = lane; sp < splits; sp += 8) t += part[(size_t)sp * stride + i];
+    s[lane][e] = t;
+    __syncthreads();
+    if (lane == 0 && i < n) {
+        float r = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r += s[j][e];
+        sgd_apply_scalar(w, v, r, shadow, i, lr, mu);
+    }
+}
+__global__ void __launch_bounds__(256)
+reduce_sgd_kernel(const float* __restrict__ part, size_t stride, int splits, float* __restrict__ w, float* __restrict__ v,
+                  __nv_bfloat16* __restrict__ shadow, size_t n, float lr, float mu)
+{
+    pdl_prologue();
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float t = 0.f;
+        for (int sp = 0; sp < splits; ++sp) t += part[(size_t)sp * stride + i];
+        sgd_apply_scalar(w, v, t, shadow, i, lr, mu);
+    }
+}
+cudaError_t launch_reduce_sgd(const float* part, size_t stride, size_t n, int splits, float* w, float* v, __nv_bfloat16* shadow,
+                              float lr, float mu, cudaStream_t st)
+{
+    // (the same case split as launch_reduce_partials: each case sums in the same order there and here)
+    if (splits >= 32 && n <= (1u << 20)) {
+        SB_LAUNCH((reduce_sgd_many_kernel), cdiv((long)n, 32), 256, 0, st, part, stride, splits, w, v, shadow, n, lr, mu);
+    } else if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)w | (uintptr_t)v) & 15) == 0 && (((uintptr_t)shadow) & 7) == 0) {
+        int blocks = cdiv((long)(n / 4), 256);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        if (shadow) SB_LAUNCH((reduce_sgd4_kernel<true>), blocks, 256, 0, st, (const float4*)part, stride / 4, splits, (float4*)w, (float4*)v, (uint2*)shadow, n / 4, lr, mu);
+        else SB_LAUNCH((reduce_sgd4_kernel<false>), blocks, 256, 0, st, (const float4*)part, stride / 4, splits, (float4*)w, (float4*)v, nullptr, n / 4, lr, mu);
+    } else {
+        int blocks = cdiv((long)n, 256);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        SB_LAUNCH((reduce_sgd_kernel), blocks, 256, 0, st, part, stride, splits, w, v, shadow, n, lr, mu);
+    }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n, float lr, float mu, cudaStream_t st)
 {
     size_t n4 = n / 4;

@@ -306,12 +306,16 @@ def test_train_step_host_matches_device_path():
     g1.close(); g2.close()
 
 
-def test_graph_step_and_graph_host_step_match_separate_calls():
+@pytest.mark.parametrize("net", ["tensor_core", "pair"])
+def test_graph_step_and_graph_host_step_match_separate_calls(net):
     """On a side stream the library replays the iteration as a CUDA graph (captured on the second call): weights
-    and losses must be bit-identical to the three separate calls, also after the inputs move (re-capture)."""
+    and losses must be bit-identical to the three separate calls, also after the inputs move (re-capture).  The graph
+    step folds the conv layers' update into their split reduces (one kernel sums the partial weight gradients in
+    order and applies SGD); the separate calls store the gradient and update afterwards.  "pair" adds layers whose
+    weight gradient runs on CTA pairs and whose bias gradient comes from the column-sum kernel."""
     import torch
     b = sb()
-    wl = WORKLOADS["tensor_core"]()
+    wl = WORKLOADS["tensor_core"]() if net == "tensor_core" else si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2)
     params = si.make_params(wl, bias_std=0.1)
     x, y = si.make_batch(wl)
     g1 = gpu_model(wl, params, b.SB_BF16)
