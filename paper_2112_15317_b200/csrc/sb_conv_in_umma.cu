@@ -326,11 +326,10 @@ conv_in_wgrad_umma_kernel(const __grid_constant__ CUtensorMap mapDy, const __nv_
     const size_t img_elems = (size_t)H * W * CIN;
     const int row = threadIdx.x >> 1, half = threadIdx.x & 1;     // two threads per pixel row
 
-    for (int it = 0; it < n_iters; ++it) {
-        const int s = it & 1;
-        uint8_t* sa = stage0 + s * 16384;
-        uint8_t* sb = sa + 8192;
-        // (stage s is free: thread 0 waited for the MMAs of chunk it-2 before the barrier that ended iteration it-1)
+    // This thread's 16-byte chunks of the patch row of pixel chunk `it`, gathered into registers: the gather of chunk
+    // it + 1 is issued before chunk it is stored and multiplied, so its load latency overlaps that work.
+    constexpr int NJ = (CHUNKS + 1) / 2;
+    auto gather = [&](int it, uint4 (&out)[NJ]) {
         const long P = (c_begin + it) * 64 + row;
         const bool valid = P < npix;
         int w = 0, h = 0;
@@ -342,13 +341,28 @@ conv_in_wgrad_umma_kernel(const __grid_constant__ CUtensorMap mapDy, const __nv_
             img = image_ptr<TAB>(x, tab, b_per_rep, q / H, img_elems);
         }
 #pragma unroll
-        for (int jj = 0; jj < (CHUNKS + 1) / 2; ++jj) {
+        for (int jj = 0; jj < NJ; ++jj) {
             const int j = 2 * jj + half;
-            if (j < CHUNKS) {
-                const uint4 v = valid ? patch_chunk<CIN>(img, h, w, H, W, 8 * j, NK) : make_uint4(0u, 0u, 0u, 0u);
-                *(uint4*)(sb + row * 128 + ((j ^ (row & 7)) << 4)) = v;
-            }
+            out[jj] = (j < CHUNKS && valid) ? patch_chunk<CIN>(img, h, w, H, W, 8 * j, NK) : make_uint4(0u, 0u, 0u, 0u);
         }
+    };
+    uint4 cur[NJ], nxt[NJ];
+    gather(0, cur);
+#pragma unroll
+    for (int jj = 0; jj < NJ; ++jj) nxt[jj] = make_uint4(0u, 0u, 0u, 0u);
+    for (int it = 0; it < n_iters; ++it) {
+        const int s = it & 1;
+        uint8_t* sa = stage0 + s * 16384;
+        uint8_t* sb = sa + 8192;
+        if (it + 1 < n_iters) gather(it + 1, nxt);
+        // (stage s is free: thread 0 waited for the MMAs of chunk it-2 before the barrier that ended iteration it-1)
+#pragma unroll
+        for (int jj = 0; jj < NJ; ++jj) {
+            const int j = 2 * jj + half;
+            if (j < CHUNKS) *(uint4*)(sb + row * 128 + ((j ^ (row & 7)) << 4)) = cur[jj];
+        }
+#pragma unroll
+        for (int jj = 0; jj < NJ; ++jj) cur[jj] = nxt[jj];
         fence_async_smem();
         __syncthreads();
         if (threadIdx.x == 0) {

@@ -138,6 +138,9 @@ def config(i: int) -> Workload:
         return Workload("cfg2_vgg16_cifar_b256", vgg16_layers(1, 10), 32, 32, 3, 32, 8, 8)
     if i == 3:
         return Workload("cfg3_vgg16_imagenet_b64", vgg16_layers(7, 1000), 224, 224, 3, 16, 4, 4)
+    if i == 5:
+        # the paper's own evaluation network (Table 1), one MP group of four workers: mp = 4, 32 images per worker
+        return Workload("cfg5_paper_vgg_cifar_b128", paper_vgg_variant_layers(), 32, 32, 3, 32, 4, 4)
     raise ValueError("config 4 is the FC sweep: see fc_sweep_case()")
 
 

@@ -112,6 +112,18 @@ def test_cfg2_full_size_sampled_images_and_partition_invariance():
     g1.close()
 
 
+def test_cfg5_paper_vgg_variant_every_layer_and_sampled_images():
+    """The paper's own evaluation network (Table 1: 7 conv + 3 FC layers on 32x32 images) as one MP group of four
+    workers: every layer's kernels element-wise at the full batch, then a full-size forward + backward with sampled
+    images followed by the oracle, and one whole training step at a reduced batch."""
+    from test_gpu_parity_small import compare_everything, layerwise_teacher_forced
+    wl = si.config(5)
+    layerwise_teacher_forced(wl, bf16=True, bias_std=0.05, distinct=4)
+    gm, _, _ = sampled_image_check(wl, [0, 77])
+    gm.close()
+    compare_everything(wl.with_batch(4), bf16=True, steps=1, bias_std=0.0, grad_frob_bound=0.3)
+
+
 def test_cfg3_full_size_sampled_image():
     gm, _, _ = sampled_image_check(si.config(3), [21])
     gm.close()
