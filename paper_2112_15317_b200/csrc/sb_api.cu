@@ -96,6 +96,7 @@ struct sb_model {
     float *row_loss = nullptr, *loss = nullptr;
     unsigned int* counter = nullptr;
     uint32_t* status = nullptr;
+    int pooled_by_conv = -1;   // index of the pool layer whose output the conv kernel just before it has already written (same forward call)
     // Set by the multi-stream backward pass while it enqueues the weight side of one conv layer: the layer's split
     // reduces then apply the update themselves (launch_reduce_sgd) once `ev` (the layer's input-gradient kernel, which
     // reads the weights) has passed; `covered` counts the parameters updated that way.
@@ -349,8 +350,10 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         const double flops = 2.0 * pix * l.Cout * 9.0 * l.Cin;
         const double bytes = pix * l.Cin * e + (double)l.n_w * e + pix * l.Cout * e;
         if (l.um.fwd.enabled) {
-            U_TRY("conv_fwd_umma", flops, bytes, umma_conv_fwd(m, i, st));
+            const double pool_bytes = l.um.pool_fused ? pix / 4.0 * l.Cout * (e + 1.0) : 0.0;
+            U_TRY("conv_fwd_umma", flops, bytes + pool_bytes, umma_conv_fwd(m, i, st));
             ++m->launches;
+            if (l.um.pool_fused) m->pooled_by_conv = i + 1;
             break;
         }
         ConvSimtArgs a{};
@@ -363,6 +366,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         break;
     }
     case SB_MAXPOOL2: {
+        if (m->pooled_by_conv == i) { m->pooled_by_conv = -1; break; }   // the conv kernel below has written this layer's output
         PoolArgs a{layer_input(m, i), l.act, l.idx, B, l.H, l.W, l.Cin};
         const double pooled = (double)B * l.out_per_img;
         L_TRY("pool_fwd", 0.0, pooled * (4 * e + e + 1), launch_pool_fwd(a, bf, st));
@@ -737,7 +741,7 @@ LayerView layer_view(sb_model* m, int i)
     LayerView v{};
     v.kind = l.kind; v.H = l.H; v.W = l.W; v.Cin = l.Cin; v.Cout = l.Cout; v.in_f = l.in_f; v.out_f = l.out_f; v.relu = l.relu;
     v.p_w = l.p_w; v.p_b = l.p_b; v.n_w = l.n_w; v.n_b = l.n_b;
-    v.act = l.act; v.dact = l.dact; v.um = &l.um;
+    v.act = l.act; v.dact = l.dact; v.um = &l.um; v.pool_idx = l.idx;
     v.in_act = l.in_override ? l.in_override : (i > 0 ? m->L[i - 1].act : nullptr);
     v.d_below = l.dbelow_override ? l.dbelow_override : (i > 0 ? m->L[i - 1].dact : m->input_grad);
     v.below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
@@ -847,10 +851,12 @@ sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void
         sb_status s = set_inputs(m, x, labels);
         if (s != SB_OK) return s;
     }
+    m->pooled_by_conv = -1;     // a pool layer run on its own (or first in the range) computes its output itself
     for (int i = first; i <= last; ++i) {
         sb_status s = forward_layer(m, i, (cudaStream_t)stream);
         if (s != SB_OK) return s;
     }
+    m->pooled_by_conv = -1;
     return SB_OK;
 }
 
@@ -872,10 +878,12 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
     sb_status s = set_inputs(m, x, labels);
     if (s != SB_OK) return s;
     m->launches = 0;
+    m->pooled_by_conv = -1;
     for (int i = 0; i < m->n_layers; ++i) {
         s = forward_layer(m, i, (cudaStream_t)stream);
         if (s != SB_OK) return s;
     }
+    m->pooled_by_conv = -1;
     m->have_fwd = true;
     return SB_OK;
 }
@@ -993,6 +1001,7 @@ static sb_status modulo_step_direct(sb_model* m, const void* const* x, const int
     sb_status s = set_inputs(m, x, labels);
     if (s != SB_OK) return s;
     m->launches = 0;
+    m->pooled_by_conv = -1;
     const int ff = m->first_fc, K = m->cfg.K, R = m->cfg.R, b = m->cfg.batch_per_replica, Bk = m->B / K;
     const size_t D = (size_t)m->L[ff].in_f;
     for (int i = 0; i < ff; ++i) {

@@ -60,6 +60,8 @@ struct UmmaParams {
     int epi, relu, out_f32;
     int tma_out;          // FWD/DGRAD, bf16 output, no split: the tile is staged in shared memory and written by TMA stores (map C)
     void* out;            // FWD/DGRAD: [pixels][ldc] bf16 (or float when out_f32); WGRAD: float partial sums
+    __nv_bfloat16* pool_out;   // FWD with tma_out, conv layer followed by a 2x2 max-pool: the pool layer's output [N][H/2][W/2][ldc]
+    uint8_t* pool_idx;         // ... and its argmax bytes (dh*2+dw), same shape; nullptr = no fused pool
     long ldc;
     const float* bias;
     const __nv_bfloat16* ref;   // UEPI_MASK: same layout as out; nullptr = no mask
@@ -171,6 +173,54 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
                     if (ncol + j < n_hi) op[j] = __float2bfloat16_rn(f[j]);
             }
         }
+    }
+}
+
+// 2x2 max-pool of the output tile staged for the TMA store (64-column slabs of 128 rows x 128 bytes, 16-byte chunks
+// XOR-swizzled by row % 8; tile row = wi + bw * (hi + bh * ni) with bw, bh even, so every pooling window lies inside
+// the tile).  One task = one pooled pixel x 8 channels: four 16-byte shared-memory reads, one 16-byte store of the
+// maxima and one 8-byte store of the argmax positions (dh*2+dw, the first maximum wins: the same rule and the same
+// bf16 inputs as the stand-alone pooling kernel, so the bytes are identical).  Called by the 128 epilogue threads.
+template <int BN>
+__device__ __forceinline__ void pool_from_stage(const UmmaParams& p, const uint8_t* stage, int t128, int n0, int n_hi, int pw0, int ph0, int pn0)
+{
+    constexpr int CH = BN / 8;
+    const int wb = p.bw / 2, hb = p.bh / 2, Ho = p.H / 2, Wo = p.W / 2;
+    for (int t = t128; t < 32 * CH; t += 128) {
+        const int c = t % CH, pr = t / CH;
+        const int wl = pr % wb, hl = (pr / wb) % hb, nl = pr / (wb * hb);
+        const int w = pw0 + 2 * wl, h = ph0 + 2 * hl, n = pn0 + nl, ncol = n0 + 8 * c;
+        if (w >= p.W || h >= p.H || n >= p.N || ncol >= n_hi) continue;
+        const int r00 = 2 * wl + p.bw * (2 * hl + p.bh * nl);
+        const uint8_t* slab = stage + (c >> 3) * 16384;
+        const int cj = c & 7;
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int r = r00 + (j & 1) + (j >> 1) * p.bw;
+            v[j] = *(const uint4*)(slab + r * 128 + ((cj ^ (r & 7)) << 4));
+        }
+        uint4 outv;
+        uint2 outi;
+        __nv_bfloat16* ov = (__nv_bfloat16*)&outv;
+        uint8_t* oi = (uint8_t*)&outi;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            __nv_bfloat16 bestv = ((const __nv_bfloat16*)&v[0])[k];
+            float best = __bfloat162float(bestv);
+            int bi = 0;
+#pragma unroll
+            for (int j = 1; j < 4; ++j) {
+                const __nv_bfloat16 cand = ((const __nv_bfloat16*)&v[j])[k];
+                const float f = __bfloat162float(cand);
+                if (f > best) { best = f; bi = j; bestv = cand; }
+            }
+            ov[k] = bestv;
+            oi[k] = (uint8_t)bi;
+        }
+        const size_t o = (((size_t)n * Ho + (h >> 1)) * Wo + (w >> 1)) * (size_t)p.ldc + ncol;
+        *(uint4*)(p.pool_out + o) = outv;
+        *(uint2*)(p.pool_idx + o) = outi;
     }
 }
 
@@ -443,8 +493,10 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         for (int j = 0; j < BN / 64; ++j)
             if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(smem) + j * 16384, n0 + 64 * j, pw0, ph0, pn0);
         tma_store_commit();
-        tma_store_wait_all();
     }
+    if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
+        pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);     // reads the stage while the TMA stores read it too
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_all();
     if (tlog && threadIdx.x == 0) { tlog[5] = (unsigned long long)clock64(); tlog[7] = globaltimer_ns(); }   // epilogue done
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
@@ -759,8 +811,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         for (int j = 0; j < BN / 64; ++j)
             if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(smem) + j * 16384, n0 + 64 * j, pw0, ph0, pn0);
         tma_store_commit();
-        tma_store_wait_all();
     }
+    if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
+        pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_all();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
@@ -1285,6 +1339,17 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 if (tma_out_ok(b, lv.Cout, 1)) {
                     if (!act_map(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                     p.tma_out = 1;
+                    // a 2x2 max-pool right above: pooled from the staged tile in the same kernel (SB_POOL_FUSE=0: separate kernel)
+                    static const bool pool_fuse = [] { const char* e = getenv("SB_POOL_FUSE"); return !(e && e[0] == '0'); }();
+                    um.pool_fused = false;
+                    if (pool_fuse && i + 1 < mv.n_layers && g.bw % 2 == 0 && g.bh % 2 == 0 && lv.W % 2 == 0 && lv.H % 2 == 0 && lv.Cout % 8 == 0) {
+                        LayerView nx = layer_view(m, i + 1);
+                        if (nx.kind == SB_MAXPOOL2 && nx.pool_idx != nullptr) {
+                            p.pool_out = (__nv_bfloat16*)nx.act;
+                            p.pool_idx = nx.pool_idx;
+                            um.pool_fused = true;
+                        }
+                    }
                 }
                 um.fwd.enabled = true;
             }

@@ -20,6 +20,8 @@ struct UmmaLayer {
     bool conv_in = false;                // input-layer conv on the tensor cores (wgrad.mapA then maps this layer's dy,
                                          // fwd.mapA its output for the TMA store)
     const void* bound_input = nullptr;   // layer 0 only: the input buffer the tensor maps currently point at
+    bool pool_fused = false;             // conv layer followed by a 2x2 max-pool: the forward kernel also writes the pool layer's
+                                         // output and argmax bytes from its staged output tile
 };
 
 // Read-only views of the model for the planner in sb_umma.cu.
@@ -43,6 +45,7 @@ struct LayerView {
     bool relu;
     size_t p_w, p_b, n_w, n_b;
     char *act, *dact;
+    unsigned char* pool_idx;   // pool layers: argmax bytes
     const char* in_act;   // previous layer's output (nullptr for layer 0)
     char* d_below;        // where the input gradient goes
     bool below_relu;

@@ -341,6 +341,34 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
     g1.close(); g2.close(); g3.close()
 
 
+@pytest.mark.parametrize("net", ["tensor_core", "pair", "cfg1_b4"])
+def test_pool_written_by_the_conv_kernel_equals_the_pooling_kernel(net):
+    """A conv layer followed by a 2x2 max-pool writes the pool layer's output and argmax bytes from its own staged
+    output tile.  Run on its own (a layer range that starts at the pool layer) the pool layer uses the stand-alone
+    pooling kernel on the same conv output: maxima and argmax bytes must be identical, ragged tiles included."""
+    b = sb()
+    if net == "cfg1_b4":
+        wl = si.config(1).with_batch(4)
+    else:
+        wl = WORKLOADS["tensor_core"]() if net == "tensor_core" else si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2)
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    gm = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    gm.forward(xs, ys)
+    pools = [li for li, (kind, _) in enumerate(wl.layers) if kind == si.MAXPOOL2]
+    assert pools
+    fused = {li: [(gm.read(b.SB_T_ACT, li, r, squeeze=False), gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)) for r in range(wl.R)] for li in pools}
+    for li in pools:
+        gm.forward_layers(li, li)
+        for r in range(wl.R):
+            act, idx = fused[li][r]
+            assert np.array_equal(act, gm.read(b.SB_T_ACT, li, r, squeeze=False)), (li, r)
+            assert np.array_equal(idx, gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)), (li, r)
+            assert idx.max() <= 3
+    gm.close()
+
+
 def test_state_and_argument_errors():
     b = sb()
     wl = si.config(0)
