@@ -903,6 +903,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
     const bool fuse = fuse_update && two_streams;
     if (updated) *updated = fuse;
     unsigned used_streams = 0;   // weight streams that received work in this pass (only those are joined)
+    bool used_ustream = false;   // likewise the update stream
     for (int i = hi; i >= lo; --i) {
         Layer& l = m->L[i];
         const bool has_params = l.kind == SB_CONV3X3_RELU || l.kind == SB_FC_RELU || l.kind == SB_FC;
@@ -939,6 +940,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
                 CU_TRY(cudaEventRecord(m->ev_wdone[i], wst));
                 CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_dgrad[i], 0));
                 CU_TRY(cudaStreamWaitEvent(m->ustream, m->ev_wdone[i], 0));
+                used_ustream = true;
                 const size_t off = l.p_w, cnt = (l.p_b - l.p_w) + align_up(l.n_b, 64);
                 {
                     cudaStream_t st = m->ustream;   // the launch bracket below records on the stream it launches on
@@ -960,8 +962,10 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
         }
     }
     if (fuse) {
-        CU_TRY(cudaEventRecord(m->ev_ujoin, m->ustream));
-        CU_TRY(cudaStreamWaitEvent(st, m->ev_ujoin, 0));
+        if (used_ustream) {
+            CU_TRY(cudaEventRecord(m->ev_ujoin, m->ustream));
+            CU_TRY(cudaStreamWaitEvent(st, m->ev_ujoin, 0));
+        }
         m->last_step_launches = m->launches;
     }
     return SB_OK;

@@ -100,6 +100,34 @@ def test_modulo_step_with_K1_equals_the_synchronous_calls():
             assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
 
 
+def test_modulo_step_replayed_as_a_graph_equals_the_direct_calls():
+    """On a side stream sb_modulo_step captures the iteration on its second call and replays it afterwards (all weight
+    streams joined, the conv layers' updates applied inside their split reduces): losses and parameters must be
+    bit-identical to the same steps enqueued directly on the default stream."""
+    import torch
+    b = sb()
+    wl = si.Workload("modulo_graph", tensor_core_net(), 12, 20, 3, 4, 2, 2)
+    params = si.make_params(wl, bias_std=0.2)
+    x, y = si.make_batch(wl)
+    xs, ys = device_batch(wl, x, y, True)
+    g1 = gpu_model(wl, params, b.SB_BF16, flags=b.SB_FLAG_MODULO_SCHEDULE)
+    g2 = gpu_model(wl, params, b.SB_BF16, flags=b.SB_FLAG_MODULO_SCHEDULE)
+    losses1 = []
+    for _ in range(4):
+        g1.modulo_step(xs, ys, 0.02, 0.9); losses1.append(g1.loss())
+    side = torch.cuda.Stream()
+    losses2 = []
+    with torch.cuda.stream(side):
+        for _ in range(4):
+            g2.modulo_step(xs, ys, 0.02, 0.9); losses2.append(g2.loss())
+        side.synchronize()
+    assert losses1 == losses2
+    for a, c in zip(g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), g2.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    g1.close(); g2.close()
+
+
 def test_modulo_step_needs_the_flag_and_a_divisible_batch():
     b = sb()
     wl = si.Workload("modulo_noflag", tensor_core_net(), 8, 8, 3, 4, 2, 2)
