@@ -347,31 +347,45 @@ reduce_partials4_kernel(const float4* __restrict__ part, size_t stride4, float4*
         out[i] = t;
     }
 }
-// Many splits, few elements: 32 elements per block, 8 lanes share the splits of each element and are
-// combined in lane order (fixed order -> deterministic).
-__global__ void __launch_bounds__(256)
+// Many splits, few elements: 32 elements per block, LANES lanes share the splits of each element (lane l takes
+// splits l, l + LANES, ... in order, four loads in flight) and are combined in lane order: a fixed order, so the
+// result is deterministic.  LANES = 8, or 32 from 128 splits on (the input layer's per-block partial sums).
+template <int LANES>
+__device__ __forceinline__ float many_lane_sum(const float* __restrict__ part, size_t stride, size_t i, int lane, int splits)
+{
+    float t = 0.f;
+    int sp = lane;
+    for (; sp + 3 * LANES < splits; sp += 4 * LANES) {
+        const float a = part[(size_t)sp * stride + i], b = part[(size_t)(sp + LANES) * stride + i];
+        const float c = part[(size_t)(sp + 2 * LANES) * stride + i], d = part[(size_t)(sp + 3 * LANES) * stride + i];
+        t += a; t += b; t += c; t += d;
+    }
+    for (; sp < splits; sp += LANES) t += part[(size_t)sp * stride + i];
+    return t;
+}
+template <int LANES>
+__global__ void __launch_bounds__(32 * LANES)
 reduce_partials_many_kernel(const float* __restrict__ part, size_t stride, float* __restrict__ out, size_t n, int splits)
 {
     pdl_prologue();
-    __shared__ float s[8][33];
+    __shared__ float s[LANES][33];
     const int e = threadIdx.x % 32, lane = threadIdx.x / 32;
     const size_t i = blockIdx.x * 32ull + e;
-    float t = 0.f;
-    if (i < n)
-        for (int sp = lane; sp < splits; sp += 8) t += part[(size_t)sp * stride + i];
-    s[lane][e] = t;
+    s[lane][e] = i < n ? many_lane_sum<LANES>(part, stride, i, lane, splits) : 0.f;
     __syncthreads();
     if (lane == 0 && i < n) {
         float r = 0.f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) r += s[j][e];
+        for (int j = 0; j < LANES; ++j) r += s[j][e];
         out[i] = r;
     }
 }
 cudaError_t launch_reduce_partials(const float* part, size_t stride, float* out, size_t n, int splits, cudaStream_t st)
 {
-    if (splits >= 32 && n <= (1u << 20)) {
-        SB_LAUNCH((reduce_partials_many_kernel), cdiv((long)n, 32), 256, 0, st, part, stride, out, n, splits);
+    if (splits >= 128 && n <= (1u << 20)) {
+        SB_LAUNCH((reduce_partials_many_kernel<32>), cdiv((long)n, 32), 1024, 0, st, part, stride, out, n, splits);
+    } else if (splits >= 32 && n <= (1u << 20)) {
+        SB_LAUNCH((reduce_partials_many_kernel<8>), cdiv((long)n, 32), 256, 0, st, part, stride, out, n, splits);
     } else if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0) {
         int blocks = cdiv((long)(n / 4), 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
@@ -748,23 +762,21 @@ __device__ __forceinline__ void sgd_apply_scalar(float* w, float* v, float g, __
     w[i] = ww;
     if (shadow) shadow[i] = __float2bfloat16_rn(ww);
 }
-__global__ void __launch_bounds__(256)
+template <int LANES>
+__global__ void __launch_bounds__(32 * LANES)
 reduce_sgd_many_kernel(const float* __restrict__ part, size_t stride, int splits, float* __restrict__ w, float* __restrict__ v,
                        __nv_bfloat16* __restrict__ shadow, size_t n, float lr, float mu)
 {
     pdl_prologue();
-    __shared__ float s[8][33];
+    __shared__ float s[LANES][33];
     const int e = threadIdx.x % 32, lane = threadIdx.x / 32;
     const size_t i = blockIdx.x * 32ull + e;
-    float t = 0.f;
-    if (i < n)
-        for (int sp = lane; sp < splits; sp += 8) t += part[(size_t)sp * stride + i];
-    s[lane][e] = t;
+    s[lane][e] = i < n ? many_lane_sum<LANES>(part, stride, i, lane, splits) : 0.f;
     __syncthreads();
     if (lane == 0 && i < n) {
         float r = 0.f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) r += s[j][e];
+        for (int j = 0; j < LANES; ++j) r += s[j][e];
         sgd_apply_scalar(w, v, r, shadow, i, lr, mu);
     }
 }
@@ -783,8 +795,10 @@ cudaError_t launch_reduce_sgd(const float* part, size_t stride, size_t n, int sp
                               float lr, float mu, cudaStream_t st)
 {
     // (the same case split as launch_reduce_partials: each case sums in the same order there and here)
-    if (splits >= 32 && n <= (1u << 20)) {
-        SB_LAUNCH((reduce_sgd_many_kernel), cdiv((long)n, 32), 256, 0, st, part, stride, splits, w, v, shadow, n, lr, mu);
+    if (splits >= 128 && n <= (1u << 20)) {
+        SB_LAUNCH((reduce_sgd_many_kernel<32>), cdiv((long)n, 32), 1024, 0, st, part, stride, splits, w, v, shadow, n, lr, mu);
+    } else if (splits >= 32 && n <= (1u << 20)) {
+        SB_LAUNCH((reduce_sgd_many_kernel<8>), cdiv((long)n, 32), 256, 0, st, part, stride, splits, w, v, shadow, n, lr, mu);
     } else if (n % 4 == 0 && stride % 4 == 0 && (((uintptr_t)part | (uintptr_t)w | (uintptr_t)v) & 15) == 0 && (((uintptr_t)shadow) & 7) == 0) {
         int blocks = cdiv((long)(n / 4), 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
