@@ -10,7 +10,7 @@
 // Every operand tile is a set of 128-byte rows fetched by TMA (cp.async.bulk.tensor, 4-D boxes,
 // SWIZZLE_128B; out-of-bounds coordinates read zeros, which implements the convolution padding,
 // ragged tile edges and ragged reduction tails) into a ring of shared-memory stages guarded by
-// mbarriers.  One thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) into a TMEM
+// mbarriers.  One elected lane issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) into a TMEM
 // accumulator; tcgen05.commit releases a stage back to the TMA producer; four epilogue warps read
 // the accumulator with tcgen05.ld and apply bias+ReLU / the ReLU mask / the split-sum store.
 //
@@ -22,10 +22,17 @@
 // normally (TMEM is always released), so a broken pipeline turns into SB_ERR_TIMEOUT on the
 // host instead of a stuck GPU.
 //
-// Large forward / data-gradient grids with 256-wide N tiles run on CTA pairs (umma_pair_kernel,
-// tcgen05.mma.cta_group::2): two neighbouring M tiles share one fetch of the weight-side operand.
+// Large forward / data-gradient grids with 256-wide N tiles, and the weight gradients of layers with
+// 256+ output channels, run on CTA pairs (umma_pair_kernel, tcgen05.mma.cta_group::2): two
+// neighbouring M tiles share one fetch of the other operand, half of it per CTA.
 // No load uses multicast; the only multicast is the pair kernel's tcgen05.commit, which releases a
 // ring slot in both CTAs of the pair.
+//
+// Epilogues: bf16 output tiles with whole rows are staged in the drained operand ring and leave by
+// TMA stores; a forward tile of a layer that a 2x2 max-pool follows is pooled from that stage in the
+// same kernel (pool_from_stage); split reductions write float partial tiles that an ordered reduce
+// kernel finishes.  The MMA and TMA issue loops run as converged warps with the instruction
+// predicated on one elected lane (descriptors in uniform registers).
 #include "sb_umma.h"
 #include "sb_tcgen05.cuh"
 

@@ -369,6 +369,20 @@ def test_pool_written_by_the_conv_kernel_equals_the_pooling_kernel(net):
     gm.close()
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_maximum_partition_counts(bf16):
+    """R = 64 replicas of one image and K = 64 shards (the largest counts the library accepts): FC shards of one or
+    two columns (70 and 130 columns over 64 shards: uneven boundaries c_j = floor(j*out/K)), 64 input pointers."""
+    net = [(si.CONV3X3_RELU, 64), (si.CONV3X3_RELU, 64), (si.MAXPOOL2, 0), (si.FC_RELU, 130), (si.FC_RELU, 70), (si.FC, 64),
+           (si.SOFTMAX_XENT, 64)]
+    wl = si.Workload("max_parts", net, 8, 8, 3, 1, 64, 64)
+    layerwise_teacher_forced(wl, bf16, bias_std=0.1)
+    compare_everything(wl, bf16, steps=1, bias_std=0.1, grad_frob_bound=0.3 if bf16 else None)
+    b = sb()
+    with pytest.raises(b.SBError, match="SB_ERR_SHAPE"):
+        gpu_model(si.Workload("too_many", net, 8, 8, 3, 1, 65, 64), si.make_params(wl), b.SB_FP32)
+
+
 def test_state_and_argument_errors():
     b = sb()
     wl = si.config(0)
