@@ -258,7 +258,7 @@ conv_in_fwd_umma_kernel(const __grid_constant__ CUtensorMap mapY, int tma_out, c
             tma_store_commit();
         }
     }
-    if (tma_out && threadIdx.x == 0) tma_store_wait_all();
+    if (tma_out && threadIdx.x == 0) tma_store_wait_read();   // shared memory may be released once the stores have read it; the writes complete with the grid
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {

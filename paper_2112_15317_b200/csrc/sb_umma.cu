@@ -503,7 +503,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     }
     if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
         pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);     // reads the stage while the TMA stores read it too
-    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_all();
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();   // shared memory may be released once the stores have read it; the writes complete with the grid
     if (tlog && threadIdx.x == 0) { tlog[5] = (unsigned long long)clock64(); tlog[7] = globaltimer_ns(); }   // epilogue done
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
@@ -821,7 +821,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     }
     if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
         pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);
-    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_all();
+    if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();   // shared memory may be released once the stores have read it; the writes complete with the grid
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
