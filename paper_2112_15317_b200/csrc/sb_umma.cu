@@ -76,8 +76,14 @@ struct UmmaParams {
     int bias_fused;       // WGRAD: the centre-tap CTAs of the first N tile also sum dy over the pixels (the bias gradient)
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
+    // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
+    // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
+    uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
     unsigned long long* timing;   // optional (SB_UMMA_TIMING=1): per-CTA phase timestamps, 8 per CTA, first 1024 CTAs
 };
+
+__host__ __device__ __forceinline__ uint32_t fast_rcp(uint32_t d) { return d <= 1u ? 0u : (uint32_t)(0x100000000ull / d) + 1u; }
+__device__ __forceinline__ int fast_div(int n, uint32_t mul) { return mul == 0u ? n : (int)__umulhi((uint32_t)n, mul); }
 
 constexpr int UMMA_THREADS = 192;
 constexpr int A_STAGE_BYTES = 16384;   // 128 rows x 128 B (K-major) or 2 boxes of 64 rows x 128 B (MN-major)
@@ -195,7 +201,8 @@ __device__ __forceinline__ void pool_from_stage(const UmmaParams& p, const uint8
     const int wb = p.bw / 2, hb = p.bh / 2, Ho = p.H / 2, Wo = p.W / 2;
     for (int t = t128; t < 32 * CH; t += 128) {
         const int c = t % CH, pr = t / CH;
-        const int wl = pr % wb, hl = (pr / wb) % hb, nl = pr / (wb * hb);
+        const int pq = fast_div(pr, p.rcp_wb), nl = fast_div(pr, p.rcp_wbhb);
+        const int wl = pr - pq * wb, hl = pq - nl * hb;
         const int w = pw0 + 2 * wl, h = ph0 + 2 * hl, n = pn0 + nl, ncol = n0 + 8 * c;
         if (w >= p.W || h >= p.H || n >= p.N || ncol >= n_hi) continue;
         const int r00 = 2 * wl + p.bw * (2 * hl + p.bh * nl);
@@ -266,10 +273,15 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         n0 = n_idx * BN;
         n_hi = p.n_total;                                     // tap_group = 3: 3 x Cin (the taps' columns are adjacent)
     } else {
-        const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
-        const int lo = (int)(((long)sh * p.n_total) / p.shards), hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
-        n0 = lo + t * BN;
-        n_hi = hi;
+        if (p.shards == 1) {
+            n0 = n_idx * BN;
+            n_hi = p.n_total;
+        } else {
+            const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
+            const int lo = (int)(((long)sh * p.n_total) / p.shards), hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
+            n0 = lo + t * BN;
+            n_hi = hi;
+        }
         if (n0 >= n_hi) return;   // uniform over the CTA, before any barrier or TMEM allocation
     }
     // FWD/DGRAD: the M tile is one pixel box; WGRAD: the M tile is 128 gradient rows of one shard
@@ -281,9 +293,10 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         m_hi = hi;
         if (m0 >= m_hi) return;
     } else {
-        pw0 = (m_idx % p.tiles_w) * p.bw;
-        ph0 = ((m_idx / p.tiles_w) % p.tiles_h) * p.bh;
-        pn0 = (m_idx / (p.tiles_w * p.tiles_h)) * p.bn;
+        const int q1 = fast_div(m_idx, p.rcp_tiles_w), q2 = fast_div(m_idx, p.rcp_tiles_wh);
+        pw0 = (m_idx - q1 * p.tiles_w) * p.bw;
+        ph0 = (q1 - q2 * p.tiles_h) * p.bh;
+        pn0 = q2 * p.bn;
     }
     if (MODE != MODE_WGRAD) split = blockIdx.z;
     // k-iterations of this CTA: a contiguous range of the reduction
@@ -295,10 +308,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     // Operand loads of the next k-iteration into ring slot `s` (executed by the producer thread, iterations in
     // order).  The iteration's coordinates are carried in counters, so the issue path has no integer division.
     int ld_a = 0, ld_b = 0, ld_c = 0;   // WGRAD: pixel-box indices (w, h, n); FWD/DGRAD: (k-chunk, tap, unused)
-    if (MODE == MODE_WGRAD) {
-        ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
-    } else {
-        ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+    if (k_begin != 0) {      // (an unsplit reduction starts at zero: no division on that path)
+        if (MODE == MODE_WGRAD) {
+            ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
+        } else {
+            ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+        }
     }
     const int wg_dr = p.ntaps == 9 ? tap_fixed / 3 - 1 : 0, wg_ds = p.ntaps == 9 ? tap_fixed % 3 - 1 : 0;
     // WGRAD with at most 64 gradient rows left in this tile: the second 64-row box of A would be all padding, so it
@@ -441,6 +456,19 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         const int q = warp % 4;               // TMEM lane quadrant of this warp
         const int row = q * 32 + lane;        // accumulator row handled by this thread
         bool ok = true;
+        // where this thread's accumulator row goes (computed while the main loop runs)
+        bool row_ok;
+        size_t row_off;
+        if (MODE == MODE_WGRAD) {
+            row_ok = (m0 + row) < m_hi;
+            row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
+        } else {
+            const int r1 = fast_div(row, p.rcp_bw), ni = fast_div(row, p.rcp_bwbh);
+            const int wi = row - r1 * p.bw, hi_ = r1 - ni * p.bh;
+            const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+            row_ok = w < p.W && h < p.H && n < p.N;
+            row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+        }
         if (MODE == MODE_WGRAD && do_bias) {
             // Bias gradient: thread `row` sums dy[pixel, m0 + row] over this CTA's pixel chunks, reading the A
             // stage (64 pixel rows of 128 bytes per 64-channel box, 16-byte chunks XOR-swizzled by row % 8)
@@ -473,17 +501,6 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         } else {
             if (tlog && threadIdx.x == 64) tlog[4] = (unsigned long long)clock64();      // accumulator complete
             tc_fence_after();
-            bool row_ok;
-            size_t row_off;
-            if (MODE == MODE_WGRAD) {
-                row_ok = (m0 + row) < m_hi;
-                row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
-            } else {
-                const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
-                const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
-                row_ok = w < p.W && h < p.H && n < p.N;
-                row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
-            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             // (the operand ring is idle once the accumulator is complete: its first bytes stage the output tile)
             store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, (MODE != MODE_WGRAD && p.tma_out) ? smem : nullptr, row);
@@ -639,26 +656,34 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         n0 = n_idx * BN; n_hi = p.n_total;
         m0 = m_idx * 128; m_hi = p.m_total;
     } else {
-        const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
-        const int lo = (int)(((long)sh * p.n_total) / p.shards);
-        n_hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
-        n0 = lo + t * BN;
+        if (p.shards == 1) {
+            n0 = n_idx * BN;
+            n_hi = p.n_total;
+        } else {
+            const int sh = n_idx / p.tiles_per_shard, t = n_idx % p.tiles_per_shard;
+            const int lo = (int)(((long)sh * p.n_total) / p.shards);
+            n_hi = (int)(((long)(sh + 1) * p.n_total) / p.shards);
+            n0 = lo + t * BN;
+        }
     }
     if (n0 >= n_hi) return;   // uniform over the pair, before any barrier or TMEM allocation
     // an M index past the last tile (odd tile count) lands wholly out of bounds: zero loads, no stores
-    const int pw0 = (m_idx % p.tiles_w) * p.bw;
-    const int ph0 = ((m_idx / p.tiles_w) % p.tiles_h) * p.bh;
-    const int pn0 = (m_idx / (p.tiles_w * p.tiles_h)) * p.bn;
+    const int mq1 = fast_div(m_idx, p.rcp_tiles_w), mq2 = fast_div(m_idx, p.rcp_tiles_wh);
+    const int pw0 = (m_idx - mq1 * p.tiles_w) * p.bw;
+    const int ph0 = (mq1 - mq2 * p.tiles_h) * p.bh;
+    const int pn0 = mq2 * p.bn;
     const int k_begin = split * p.chunks_per_split;
     const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
     const int n_iters = k_end - k_begin;
 
     // next load: FWD / DGRAD (k-chunk, tap); WGRAD pixel-box indices (w, h, n)
-    int ld_a, ld_b, ld_c = 0;
-    if (MODE == MODE_WGRAD) {
-        ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
-    } else {
-        ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+    int ld_a = 0, ld_b = 0, ld_c = 0;
+    if (k_begin != 0) {
+        if (MODE == MODE_WGRAD) {
+            ld_a = k_begin % p.tiles_w; ld_b = (k_begin / p.tiles_w) % p.tiles_h; ld_c = k_begin / (p.tiles_w * p.tiles_h);
+        } else {
+            ld_a = k_begin % p.kchunks; ld_b = k_begin / p.kchunks;
+        }
     }
     const int wg_dr = tap_fixed / 3 - 1, wg_ds = tap_fixed % 3 - 1;
     const int nb0 = n0 + (int)rank * (BN / 2);                     // first B column this CTA fetches
@@ -780,23 +805,25 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const int q = warp % 4;
         const int row = q * 32 + lane;
         bool ok = true;
+        // where this thread's accumulator row goes (computed while the main loop runs)
+        bool row_ok;
+        size_t row_off;
+        if (MODE == MODE_WGRAD) {
+            row_ok = (m0 + row) < m_hi;
+            row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
+        } else {
+            const int r1 = fast_div(row, p.rcp_bw), ni = fast_div(row, p.rcp_bwbh);
+            const int wi = row - r1 * p.bw, hi_ = r1 - ni * p.bh;
+            const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+            row_ok = w < p.W && h < p.H && n < p.N;
+            row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+        }
         if (lane == 0) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
             tc_fence_after();
-            bool row_ok;
-            size_t row_off;
-            if (MODE == MODE_WGRAD) {
-                row_ok = (m0 + row) < m_hi;
-                row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
-            } else {
-                const int wi = row % p.bw, hi_ = (row / p.bw) % p.bh, ni = row / (p.bw * p.bh);
-                const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
-                row_ok = w < p.W && h < p.H && n < p.N;
-                row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
-            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             const bool staged_out = MODE != MODE_WGRAD && p.tma_out;
             store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, staged_out ? smem : nullptr, row);
@@ -987,6 +1014,14 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     cudaError_t e;
     UmmaParams pp = b->p;
     pp.timing = g_timing;
+    if (pp.mode != MODE_WGRAD) {
+        pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
+        pp.rcp_tiles_wh = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h));
+        pp.rcp_bw = fast_rcp((uint32_t)pp.bw);
+        pp.rcp_bwbh = fast_rcp((uint32_t)(pp.bw * pp.bh));
+        pp.rcp_wb = fast_rcp((uint32_t)(pp.bw / 2));
+        pp.rcp_wbhb = fast_rcp((uint32_t)((pp.bw / 2) * (pp.bh / 2)));
+    }
     if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_DGRAD) e = launch_pair_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_WGRAD) e = launch_pair_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
