@@ -29,9 +29,19 @@ constexpr int CI_THREADS = 128;
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 template <bool TAB>
-__device__ __forceinline__ const __nv_bfloat16* image_ptr(const __nv_bfloat16* x, const PtrTab& tab, int b_per_rep, long n, size_t img_elems)
+__device__ __forceinline__ const __nv_bfloat16* image_ptr(const __nv_bfloat16* x, const PtrTab& tab, int b_per_rep, uint32_t n, size_t img_elems)
 {
-    return TAB ? (const __nv_bfloat16*)tab.p[n / b_per_rep] + (size_t)(n % b_per_rep) * img_elems : x + (size_t)n * img_elems;
+    if (!TAB) return x + (size_t)n * img_elems;
+    const uint32_t rep = n / (uint32_t)b_per_rep;
+    return (const __nv_bfloat16*)tab.p[rep] + (size_t)(n - rep * (uint32_t)b_per_rep) * img_elems;
+}
+// flat pixel index (< 2^31: checked by the launchers) -> column, row, image; 32-bit divisions only
+__device__ __forceinline__ void pixel_coords(uint32_t P, int W, int H, int& w, int& h, uint32_t& n)
+{
+    const uint32_t q = P / (uint32_t)W;
+    w = (int)(P - q * (uint32_t)W);
+    n = q / (uint32_t)H;
+    h = (int)(q - n * (uint32_t)H);
 }
 
 // k-values [k0, k0 + 8) of pixel (h, w) of image `img` as one 16-byte chunk; `ones_col` (or -1) is the k index that holds 1.
@@ -178,13 +188,13 @@ conv_in_fwd_umma_kernel(const __grid_constant__ CUtensorMap mapY, int tma_out, c
         int w = 0, h = 0;
         const __nv_bfloat16* img = x;
         if (valid) {
-            w = (int)(P % W);
-            const long q = P / W;
-            h = (int)(q % H);
-            img = image_ptr<TAB>(x, tab, b_per_rep, q / H, img_elems);
+            uint32_t n;
+            pixel_coords((uint32_t)P, W, H, w, h, n);
+            img = image_ptr<TAB>(x, tab, b_per_rep, n, img_elems);
         }
         // a tile that lies inside one image (uniform over the CTA) gathers from the staged window
-        const long p_in = P0 % HW;
+        const uint32_t n0_img = (uint32_t)P0 / (uint32_t)HW;
+        const long p_in = (long)((uint32_t)P0 - n0_img * (uint32_t)HW);
         const bool staged = use_window && p_in + 128 <= HW && P0 + 128 <= npix;
         if (tma_out) {
             // the previous tile's output was staged in sA: its TMA store must have read it before sA is rewritten
@@ -192,7 +202,7 @@ conv_in_fwd_umma_kernel(const __grid_constant__ CUtensorMap mapY, int tma_out, c
             __syncthreads();
         }
         if (staged) {
-            const __nv_bfloat16* img0 = image_ptr<TAB>(x, tab, b_per_rep, P0 / HW, img_elems);
+            const __nv_bfloat16* img0 = image_ptr<TAB>(x, tab, b_per_rep, n0_img, img_elems);
             const long e_start = stage_window<CIN>(img0, win, p_in, 128, H, W);
             __syncthreads();
 #pragma unroll
@@ -335,10 +345,9 @@ conv_in_wgrad_umma_kernel(const __grid_constant__ CUtensorMap mapDy, const __nv_
         int w = 0, h = 0;
         const __nv_bfloat16* img = x;
         if (valid) {
-            w = (int)(P % W);
-            const long q = P / W;
-            h = (int)(q % H);
-            img = image_ptr<TAB>(x, tab, b_per_rep, q / H, img_elems);
+            uint32_t n;
+            pixel_coords((uint32_t)P, W, H, w, h, n);
+            img = image_ptr<TAB>(x, tab, b_per_rep, n, img_elems);
         }
 #pragma unroll
         for (int jj = 0; jj < NJ; ++jj) {
@@ -456,6 +465,7 @@ template <int CIN>
 static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, uint32_t* status, cudaStream_t st)
 {
     const long npix = (long)a.B * a.H * a.W;
+    if (npix + 128 >= (1L << 31)) return cudaErrorInvalidValue;     // the kernel's pixel arithmetic is 32-bit
     const long n_tiles = (npix + 127) / 128;
     const int grid = (int)(n_tiles < 148 * 6 ? n_tiles : 148 * 6);
     // the staged gather needs images of an even number of elements (4-byte loads) and a window that fits
@@ -492,6 +502,7 @@ template <int CIN>
 static cudaError_t launch_wgrad_t(const WgradSimtArgs& a, const CUtensorMap& mapDy, uint32_t* status, cudaStream_t st)
 {
     const long npix = (long)a.B * a.H * a.W;
+    if (npix + 128 >= (1L << 31)) return cudaErrorInvalidValue;     // the kernel's pixel arithmetic is 32-bit
     const long chunks = (npix + 63) / 64;
     const int grid = conv_in_umma_wgrad_blocks(npix);
     const long cpc = (chunks + grid - 1) / grid;
