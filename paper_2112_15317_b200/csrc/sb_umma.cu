@@ -104,6 +104,83 @@ template <int MODE, int BN>
 __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, bool row_ok, size_t row_off, int n0, int n_hi,
                                           int split, const float* s_bias, uint8_t* stage = nullptr, int row = 0)
 {
+    if (MODE != MODE_WGRAD && stage != nullptr) {
+        // Staged bf16 tile for the TMA store (the planner only selects it for unsplit bf16 outputs whose columns end on
+        // 64-column slabs): every decision is taken once, outside the loop -- an epilogue warp runs alone on its
+        // scheduler, so every branch and every dependent instruction in the loop costs its full latency.
+        const bool bias_act = p.epi == UEPI_BIAS_ACT, relu = p.relu != 0;
+        const __nv_bfloat16* refrow = (p.epi == UEPI_MASK && p.ref != nullptr && row_ok) ? p.ref + row_off + n0 : nullptr;
+        const uint32_t bias_s = smem_u32(s_bias);
+        const uint32_t row_s = smem_u32(stage) + (uint32_t)row * 128u;
+        const uint32_t sw = (uint32_t)(row & 7);
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(taddr + c0, v);     // warp-collective
+            tmem_ld_wait();
+            if (n0 + c0 >= n_hi) continue;            // (uniform: whole 64-column slabs)
+            float f[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
+            if (bias_act) {
+#pragma unroll
+                for (int j4 = 0; j4 < 4; ++j4) {
+                    float b0, b1, b2, b3;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(bias_s + (uint32_t)(c0 + 4 * j4) * 4u));
+                    f[4 * j4] += b0; f[4 * j4 + 1] += b1; f[4 * j4 + 2] += b2; f[4 * j4 + 3] += b3;
+                }
+                if (relu) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) f[j] = f[j] > 0.f ? f[j] : 0.f;     // (NaN -> 0, as the reference path)
+                }
+            } else if (refrow != nullptr) {
+                const uint4 r0 = *(const uint4*)(refrow + c0), r1 = *(const uint4*)(refrow + c0 + 8);
+                const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
+                const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
+                    if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
+                }
+            }
+            uint32_t pk[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+                pk[j] = *(uint32_t*)&t;
+            }
+            // 64-column slabs of 128 rows x 128 bytes in the 128-byte swizzle of the tensor map
+            const uint32_t slab = row_s + (uint32_t)(c0 >> 6) * 16384u, j0 = (uint32_t)(c0 & 63) >> 3;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((j0 ^ sw) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + (((j0 + 1u) ^ sw) << 4)), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+        }
+        return;
+    }
+    const bool raw_partials = MODE != MODE_WGRAD && p.splits > 1;
+    if (raw_partials || p.epi == UEPI_F32) {
+        // Float rows without any arithmetic: the split partial sums of a forward / data-gradient op, or a weight-gradient
+        // tile (straight into the gradient or into a split copy).  Destination and vector-store decision taken once.
+        float* dst = raw_partials ? p.part + (size_t)split * p.split_stride + row_off + n0 : (float*)p.out + row_off + n0;
+        const bool vec = raw_partials ? ((p.n_total & 3) == 0 && (n0 & 3) == 0)
+                                      : ((p.ldc & 3) == 0 && (n0 & 3) == 0 && ((((size_t)p.split_stride) & 3) == 0) && ((p.w_cols & 3) == 0 || MODE != MODE_WGRAD));
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(taddr + c0, v);     // warp-collective: executed by all lanes regardless of row_ok
+            tmem_ld_wait();
+            if (!row_ok || n0 + c0 >= n_hi) continue;
+            if (vec && n0 + c0 + 16 <= n_hi) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    ((float4*)(dst + c0))[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (n0 + c0 + j < n_hi) dst[c0 + j] = __uint_as_float(v[j]);
+            }
+        }
+        return;
+    }
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 16) {
         uint32_t v[16];
