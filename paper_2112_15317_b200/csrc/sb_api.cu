@@ -18,6 +18,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <algorithm>
 #include <vector>
 
 using namespace sb;
@@ -266,7 +267,8 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
             if ((size_t)sb_ * l.n_b > ws_floats) ws_floats = (size_t)sb_ * l.n_b;
             l.thin_input = conv_in_supported(l.Cin, l.Cout);
             if (l.thin_input) {
-                size_t nd = (size_t)conv_in_wgrad_blocks((int)B, l.H, l.W) * (l.n_w + l.n_b);
+                const int nblk = std::max(conv_in_wgrad_blocks((int)B, l.H, l.W), conv_in_umma_wgrad_blocks((long)B * l.H * l.W));
+                size_t nd = (size_t)nblk * (l.n_w + l.n_b);
                 if (nd > ws_floats) ws_floats = nd;
             }
         }

@@ -455,7 +455,7 @@ int conv_in_umma_wgrad_blocks(long npix)
 {
     const long chunks = (npix + 63) / 64;
     long ctas = chunks / 4;                       // at least ~4 chunks per CTA
-    if (ctas > 148 * 4) ctas = 148 * 4;
+    if (ctas > 148 * 6) ctas = 148 * 6;           // six CTAs per SM overlap one another's gather / MMA / barrier chains (4: +15 % time)
     if (ctas < 1) ctas = 1;
     const long cpc = (chunks + ctas - 1) / ctas;
     return (int)((chunks + cpc - 1) / cpc);       // no empty trailing CTA
