@@ -84,6 +84,15 @@ struct UmmaParams {
 
 __host__ __device__ __forceinline__ uint32_t fast_rcp(uint32_t d) { return d <= 1u ? 0u : (uint32_t)(0x100000000ull / d) + 1u; }
 __device__ __forceinline__ int fast_div(int n, uint32_t mul) { return mul == 0u ? n : (int)__umulhi((uint32_t)n, mul); }
+// the same with one correction step: the estimate is never low and at most one high for any n < 2^31, so this is exact
+// for every tile index (fast_div alone is exact while n * d < 2^32: rows of a tile, pooled pixels of a tile)
+__device__ __forceinline__ int fast_div_exact(int n, uint32_t mul, int d)
+{
+    if (mul == 0u) return n;
+    uint32_t q = __umulhi((uint32_t)n, mul);
+    if (q * (uint32_t)d > (uint32_t)n) --q;
+    return (int)q;
+}
 
 constexpr int UMMA_THREADS = 192;
 constexpr int A_STAGE_BYTES = 16384;   // 128 rows x 128 B (K-major) or 2 boxes of 64 rows x 128 B (MN-major)
@@ -370,7 +379,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         m_hi = hi;
         if (m0 >= m_hi) return;
     } else {
-        const int q1 = fast_div(m_idx, p.rcp_tiles_w), q2 = fast_div(m_idx, p.rcp_tiles_wh);
+        const int q1 = fast_div_exact(m_idx, p.rcp_tiles_w, p.tiles_w), q2 = fast_div_exact(m_idx, p.rcp_tiles_wh, p.tiles_w * p.tiles_h);
         pw0 = (m_idx - q1 * p.tiles_w) * p.bw;
         ph0 = (q1 - q2 * p.tiles_h) * p.bh;
         pn0 = q2 * p.bn;
@@ -745,7 +754,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     }
     if (n0 >= n_hi) return;   // uniform over the pair, before any barrier or TMEM allocation
     // an M index past the last tile (odd tile count) lands wholly out of bounds: zero loads, no stores
-    const int mq1 = fast_div(m_idx, p.rcp_tiles_w), mq2 = fast_div(m_idx, p.rcp_tiles_wh);
+    const int mq1 = fast_div_exact(m_idx, p.rcp_tiles_w, p.tiles_w), mq2 = fast_div_exact(m_idx, p.rcp_tiles_wh, p.tiles_w * p.tiles_h);
     const int pw0 = (m_idx - mq1 * p.tiles_w) * p.bw;
     const int ph0 = (mq1 - mq2 * p.tiles_h) * p.bh;
     const int pn0 = mq2 * p.bn;
