@@ -306,7 +306,7 @@ def test_train_step_host_matches_device_path():
     g1.close(); g2.close()
 
 
-@pytest.mark.parametrize("net", ["tensor_core", "pair"])
+@pytest.mark.parametrize("net", ["tensor_core", "pair", "tensor_core_fp32", "ragged_fp32"])
 def test_graph_step_and_graph_host_step_match_separate_calls(net):
     """On a side stream the library replays the iteration as a CUDA graph (captured on the second call): weights
     and losses must be bit-identical to the three separate calls, also after the inputs move (re-capture).  The graph
@@ -315,15 +315,20 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
     weight gradient runs on CTA pairs and whose bias gradient comes from the column-sum kernel."""
     import torch
     b = sb()
-    wl = WORKLOADS["tensor_core"]() if net == "tensor_core" else si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2)
+    bf16 = not net.endswith("_fp32")            # float mode: the CUDA-core kernels, their split reduces fold the update in too
+    if net.startswith("ragged"):
+        wl = WORKLOADS["ragged"]()
+    else:
+        wl = WORKLOADS["tensor_core"]() if net.startswith("tensor_core") else si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2)
     params = si.make_params(wl, bias_std=0.1)
     x, y = si.make_batch(wl)
-    g1 = gpu_model(wl, params, b.SB_BF16)
-    g2 = gpu_model(wl, params, b.SB_BF16)
-    g3 = gpu_model(wl, params, b.SB_BF16)
-    xs, ys = device_batch(wl, x, y, True)
+    prec = b.SB_BF16 if bf16 else b.SB_FP32
+    g1 = gpu_model(wl, params, prec)
+    g2 = gpu_model(wl, params, prec)
+    g3 = gpu_model(wl, params, prec)
+    xs, ys = device_batch(wl, x, y, bf16)
     xs2 = [t.clone() for t in xs]                      # same values at other addresses
-    hx = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    hx = (torch.from_numpy(x).to(torch.bfloat16) if bf16 else torch.from_numpy(x)).pin_memory()
     hy = torch.from_numpy(y).pin_memory()
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
