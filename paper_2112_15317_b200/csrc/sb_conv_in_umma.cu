@@ -467,7 +467,6 @@ static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, 
     const long npix = (long)a.B * a.H * a.W;
     if (npix + 128 >= (1L << 31)) return cudaErrorInvalidValue;     // the kernel's pixel arithmetic is 32-bit
     const long n_tiles = (npix + 127) / 128;
-    const int grid = (int)(n_tiles < 148 * 6 ? n_tiles : 148 * 6);
     // the staged gather needs images of an even number of elements (4-byte loads) and a window that fits
     static const bool no_window = [] { const char* e = getenv("SB_CONV_IN_WINDOW"); return e && e[0] == '0'; }();
     const size_t wbytes = (!no_window && ((size_t)a.H * a.W * CIN) % 2 == 0) ? window_bytes(128, a.W, CIN) : 0;
@@ -481,6 +480,13 @@ static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, 
     const int tma_out = (mapY && a.Cout == 64 && !no_tma_out) ? 1 : 0;
     CUtensorMap dummy{};
     const CUtensorMap& my = tma_out ? *mapY : dummy;
+    // persistent CTAs, as many as are resident at once (7 per SM for 64 output channels; their TMEM columns also fit:
+    // 8 x 64): one CTA more per SM than fits means a second wave (measured 159 us with 7, 228 us with 8 at ImageNet size)
+    long per_sm = (227L * 1024) / (long)(smem + 1024);       // shared memory (1 KB per CTA is reserved by the system)
+    if (per_sm > 512 / (long)cols) per_sm = 512 / (long)cols;    // TMEM columns
+    if (per_sm > 8) per_sm = 8;
+    if (per_sm < 1) per_sm = 1;
+    const int grid = (int)(n_tiles < 148L * per_sm ? n_tiles : 148L * per_sm);
     if (a.tab)
         return pdl_launch(conv_in_fwd_umma_kernel<CIN, true>, dim3(grid), dim3(CI_THREADS), smem, st, my, tma_out, (const __nv_bfloat16*)nullptr, tab, a.b_per_rep,
                           (const __nv_bfloat16*)a.w, a.bias, (__nv_bfloat16*)a.out, npix, a.H, a.W, a.Cout, a.relu, n_tiles, cols, status, use_window);
