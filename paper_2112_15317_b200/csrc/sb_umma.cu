@@ -59,7 +59,8 @@ struct UmmaParams {
     // WGRAD
     int m_total;          // rows of the weight gradient (Cout / out-features)
     int m_shards, m_tiles_per_shard;
-    int tap_group;        // WGRAD: filter taps per CTA: 1, or 3 (one filter row; Cin = 64, N tile = 3 x 64 columns)
+    int tap_group;        // WGRAD: filter taps per CTA: 1, 3 (one filter row; Cin = 64, N tile = 3 x 64 columns) or 2 (Cin = 128,
+                          // N tile = 2 x 128 columns; the fifth group holds tap 8 alone)
     int splits, chunks_per_split, total_chunks;   // split of the reduction (k-iterations) over blockIdx.z
     int stages;           // depth of the shared-memory ring (<= MAX_STAGES)
     float* part;          // FWD/DGRAD with splits > 1: raw float partial sums [split][pixel][n_total]
@@ -358,6 +359,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         split = blockIdx.z % p.splits;
         n0 = n_idx * BN;
         n_hi = p.n_total;                                     // tap_group = 3: 3 x Cin (the taps' columns are adjacent)
+        if (p.tap_group == 2) n_hi = min(p.n_total, (9 - tap_fixed) * p.w_cols);   // the last pair of taps has one member
     } else {
         if (p.shards == 1) {
             n0 = n_idx * BN;
@@ -389,6 +391,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int k_begin = split * p.chunks_per_split;
     const int k_end = min(k_begin + p.chunks_per_split, p.total_chunks);
     const int n_iters = k_end - k_begin;
+    // (tap groups {3,4,5} and {4,5} both start with a tap every CTA grid has exactly once per M tile and split)
     const bool do_bias = MODE == MODE_WGRAD && p.bias_fused && n_idx == 0 && tap_fixed == (p.ntaps == 9 ? (p.tap_group == 3 ? 3 : 4) : 0);
 
     // Operand loads of the next k-iteration into ring slot `s` (executed by the producer thread, iterations in
@@ -422,6 +425,14 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 // one filter row: the three taps' activation boxes are the same pixels shifted by -1, 0, +1 in w
 #pragma unroll
                 for (int j = 0; j < 3; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, 0, cw + j - 1, ch + wg_dr, cn, el);
+            } else if (BN == 256 && p.tap_group == 2) {
+                // two adjacent taps of a 128-input-channel layer: boxes 0, 1 = channels 0-63, 64-127 of tap t, boxes 2, 3 of
+                // tap t + 1 (tap 9 does not exist: its rows lie outside the image and read as zeros, its columns are not stored)
+                const int t1 = tap_fixed + 1, dr1 = t1 / 3 - 1, ds1 = t1 % 3 - 1;
+                tma_load_4d_el(&mapB, sb, bar, 0, cw + wg_ds, ch + wg_dr, cn, el);
+                tma_load_4d_el(&mapB, sb + 8192, bar, 64, cw + wg_ds, ch + wg_dr, cn, el);
+                tma_load_4d_el(&mapB, sb + 16384, bar, 0, cw + ds1, ch + dr1, cn, el);
+                tma_load_4d_el(&mapB, sb + 24576, bar, 64, cw + ds1, ch + dr1, cn, el);
             } else {
 #pragma unroll
                 for (int j = 0; j < BN / 64; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn, el);
@@ -1345,8 +1356,15 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
     static const bool taps1 = [] { const char* e = getenv("SB_WGRAD_TAPS"); return e && e[0] == '1'; }();
     g.wg_tap_group = (lv.Cin == 64 && !taps1) ? 3 : 1;
     if (g.wg_tap_group == 3) g.wg_bn = 192;
+    // 128 input channels and at most 128 output channels (one M tile, so no CTA pair): two adjacent taps per CTA as one
+    // 256-column tile (dy fetched once per two taps; five tap groups, the last with tap 8 alone).  SB_WGRAD_TAPS=1 turns it off.
+    // Taken for long reductions only (ImageNet-size layers: 613 -> 290 us alone); at CIFAR size the kernel alone is 15 %
+    // faster but the step is not (its 96 KB ring and 256 TMEM columns leave the data-gradient kernel less room beside it).
+    static const int taps2_min_chunks = [] { const char* e = getenv("SB_WGRAD_TAPS2_MIN_CHUNKS"); return e ? atoi(e) : 2048; }();
+    if (lv.Cin == 128 && lv.Cout <= 128 && !taps1 && g.total_chunks >= taps2_min_chunks) { g.wg_tap_group = 2; g.wg_bn = 256; g.wg_n_tiles = 1; }
+    const int tap_groups = (9 + g.wg_tap_group - 1) / g.wg_tap_group;
     double cost = 0.0;
-    int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * (9 / g.wg_tap_group), g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b, &cost);
+    int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * tap_groups, g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b, &cost);
     // a narrower N tile doubles the CTAs of a grid that leaves SMs idle (e.g. 512 channels at 4x4: 72 CTAs of 256
     // columns against 144 of 128): take it when the same model says it is faster (SB_WGRAD_NARROW=0 keeps the widest)
     static const bool narrow = [] { const char* e = getenv("SB_WGRAD_NARROW"); return !(e && e[0] == '0'); }();
@@ -1523,7 +1541,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 {
                     // grids of fewer than ~100 CTAs leave the other streams whole SMs: no need to keep the ring shallow (measured: -1.5 % step)
                     static const long wg_cohabit_min = [] { const char* e = getenv("SB_WG_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
-                    const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * (9 / p.tap_group) * p.splits;
+                    const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * ((9 + p.tap_group - 1) / p.tap_group) * p.splits;
                     if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
                 }
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
@@ -1548,7 +1566,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 }
                 p.out = p.splits > 1 ? (void*)mv.ws_wk[mv.n_wstreams > 0 ? i % mv.n_wstreams : 0] : (void*)(mv.Gm + lv.p_w);
                 p.status = mv.status;
-                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)(9 / p.tap_group * p.splits));
+                b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)((9 + p.tap_group - 1) / p.tap_group * p.splits));
                 if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
                 if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
                 if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch, g.cn)) return fail_plan();
