@@ -1542,7 +1542,12 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     // grids of fewer than ~100 CTAs leave the other streams whole SMs: no need to keep the ring shallow (measured: -1.5 % step)
                     static const long wg_cohabit_min = [] { const char* e = getenv("SB_WG_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
                     const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * ((9 + p.tap_group - 1) / p.tap_group) * p.splits;
-                    if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cohabit_stages(b->bn)) p.stages = cohabit_stages(b->bn);
+                    // (the filter-row kernel of a short reduction keeps a third 40 KB stage: CIFAR-size steps -1 to -2.7 %; a long
+                    // one leaves the room to the data-gradient kernel beside it: ImageNet-size step +1.9 % with three)
+                    static const int row3_max_cps = [] { const char* e = getenv("SB_WGRAD_ROW3_MAX_CHUNKS"); return e ? atoi(e) : 128; }();
+                    int cap = cohabit_stages(b->bn);
+                    if (b->bn == 192 && g.wg_cps <= row3_max_cps) cap = 3;
+                    if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cap) p.stages = cap;
                 }
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;
                 // the bias gradient rides along: in the parameter arena the bias vector directly follows the
