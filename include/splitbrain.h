@@ -262,13 +262,6 @@ sb_status sb_profile_begin(sb_model* m, void* stream);
 sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32_t max_entries, int32_t* n);
 
 /*
- * Debug aid for kernel tuning: dev_buffer = DEVICE buffer of 1024*16 uint64 (or NULL to switch off).  While set,
- * the first 1024 CTAs of every tensor-core launch record the global nanosecond timer at their phase boundaries
- * (start, set-up done, first operands landed, last operands landed, accumulator complete, epilogue done).
- */
-sb_status sb_debug_cta_timing(void* dev_buffer);
-
-/*
  * Self-test of the hang-safety path.  Every wait inside the library's kernels is bounded; a wait that runs out makes
  * the kernel record a code in the model's device status word and return normally, and the next sb_loss (or
  * sb_train_step_host) returns SB_ERR_TIMEOUT and clears the word.  This call enqueues one CTA that waits limit_ms

@@ -76,7 +76,6 @@ def _load():
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
         "sb_launch_count": [c_void_p, P(c_int64)],
         "sb_conv_in_wgrad_static": [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p],
-        "sb_debug_cta_timing": [c_void_p],
         "sb_profile_begin": [c_void_p, c_void_p],
         "sb_profile_end": [c_void_p, c_void_p, P(sb_profile_entry), c_int32, P(c_int32)],
     }
@@ -115,7 +114,6 @@ sb_backward_layers = _lib.sb_backward_layers
 sb_param_bytes = _lib.sb_param_bytes
 sb_launch_count = _lib.sb_launch_count
 sb_conv_in_wgrad_static = _lib.sb_conv_in_wgrad_static
-sb_debug_cta_timing = _lib.sb_debug_cta_timing
 sb_profile_begin = _lib.sb_profile_begin
 sb_profile_end = _lib.sb_profile_end
 

@@ -9,11 +9,10 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsplitbrain.so")
 SOURCES = ["sb_api.cu", "sb_kernels_simt.cu", "sb_umma.cu", "sb_noalloc.cu", "sb_conv_in_umma.cu"]
-# stand-alone timing program (tcgen05.mma issue rate); not part of the library
-TOOL_SRC = "mma_issue_rate.cu"
-TOOL = os.path.join(HERE, "mma_issue_rate")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC"]
+# development builds: extra compiler flags, e.g. SB_NVCC_EXTRA="-DSB_DEV_TUNING -DSB_CTA_TIMING"
+NVCC_FLAGS += os.environ.get("SB_NVCC_EXTRA", "").split()
 
 
 def sources():
@@ -45,21 +44,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
-    tool_src = os.path.join(CSRC, TOOL_SRC)
-    tool_proc = None
-    if os.path.exists(tool_src):
-        tool_cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-cudart", "static",
-                    tool_src, "-o", TOOL + f".tmp{os.getpid()}"]
-        tool_proc = (tool_cmd, subprocess.Popen(tool_cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
     tmp = LIB + f".tmp{os.getpid()}"
     subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-cudart", "static"], check=True)
     os.replace(tmp, LIB)
-    if tool_proc:
-        out, _ = tool_proc[1].communicate()
-        if tool_proc[1].returncode != 0:
-            sys.stderr.write(out)
-            raise RuntimeError("nvcc failed: " + " ".join(tool_proc[0]))
-        os.replace(TOOL + f".tmp{os.getpid()}", TOOL)
     return LIB
 
 

@@ -780,8 +780,7 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     const char* one = getenv("SB_ONE_STREAM");
     if (!(one && one[0] == '1')) {
         // second stream + ordering events for the backward pass (host objects; no device memory)
-        const char* nws = getenv("SB_WSTREAMS");
-        m->n_wstreams = nws ? atoi(nws) : 4;
+        m->n_wstreams = (int)tune("SB_WSTREAMS", 4);
         if (m->n_wstreams < 1) m->n_wstreams = 1;
         if (m->n_wstreams > sb_model::MAX_WSTREAMS) m->n_wstreams = sb_model::MAX_WSTREAMS;
         bool ok_ = true;
@@ -916,7 +915,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
             CU_TRY(cudaStreamWaitEvent(wst, m->ev_ready[i], 0));
             // Conv layers in a fused pass: the input-gradient kernel is enqueued first and its event recorded, so that the
             // layer's split reduces on the weight stream can wait for it and apply the update themselves.
-            static const bool reduce_updates = [] { const char* e = getenv("SB_REDUCE_SGD"); return !(e && e[0] == '0'); }();
+            static const bool reduce_updates = tune("SB_REDUCE_SGD", 1) != 0;
             const bool in_reduce = fuse && reduce_updates && l.kind == SB_CONV3X3_RELU;
             sb_status s = SB_OK;
             if (in_reduce) {
@@ -1300,11 +1299,14 @@ sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32
     return SB_OK;
 }
 
-sb_status sb_debug_cta_timing(void* dev_buffer)
+#ifdef SB_CTA_TIMING
+// development builds only (not in the public header): hands the tensor-core kernels a device buffer for per-CTA clock stamps
+extern "C" sb_status sb_debug_cta_timing(void* dev_buffer)
 {
     umma_set_timing_buffer(dev_buffer);
     return SB_OK;
 }
+#endif
 
 sb_status sb_debug_wait_probe(sb_model* m, int32_t limit_ms, void* stream)
 {

@@ -468,7 +468,7 @@ static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, 
     if (npix + 128 >= (1L << 31)) return cudaErrorInvalidValue;     // the kernel's pixel arithmetic is 32-bit
     const long n_tiles = (npix + 127) / 128;
     // the staged gather needs images of an even number of elements (4-byte loads) and a window that fits
-    static const bool no_window = [] { const char* e = getenv("SB_CONV_IN_WINDOW"); return e && e[0] == '0'; }();
+    static const bool no_window = tune("SB_CONV_IN_WINDOW", 1) == 0;
     const size_t wbytes = (!no_window && ((size_t)a.H * a.W * CIN) % 2 == 0) ? window_bytes(128, a.W, CIN) : 0;
     const size_t smem = 1024 + 16384 + (size_t)a.Cout * 128 + (size_t)a.Cout * 4 + 64 + wbytes;
     const int use_window = wbytes > 0 ? 1 : 0;
@@ -476,7 +476,7 @@ static cudaError_t launch_fwd_t(const ConvSimtArgs& a, const CUtensorMap* mapY, 
     if (a.tab) tab = *a.tab;
     const uint32_t cols = pow2_cols(a.Cout);
     // the output goes out by TMA store when the caller made a tensor map for it (64 channels: one 128-byte row per pixel)
-    static const bool no_tma_out = [] { const char* e = getenv("SB_CONV_IN_TMA_OUT"); return e && e[0] == '0'; }();
+    static const bool no_tma_out = tune("SB_CONV_IN_TMA_OUT", 1) == 0;
     const int tma_out = (mapY && a.Cout == 64 && !no_tma_out) ? 1 : 0;
     CUtensorMap dummy{};
     const CUtensorMap& my = tma_out ? *mapY : dummy;

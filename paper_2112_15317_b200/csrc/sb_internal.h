@@ -26,6 +26,18 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_prologue() { pdl_wait(); pdl_trigger(); }
 #endif
+// Tuning constants of the planner.  The shipped library uses the compiled-in defaults; a development build
+// (-DSB_DEV_TUNING) lets an environment variable of the same name override each one for A/B measurements.
+inline double tune(const char* name, double dflt)
+{
+#ifdef SB_DEV_TUNING
+    const char* e = getenv(name);
+    return e ? atof(e) : dflt;
+#else
+    (void)name;
+    return dflt;
+#endif
+}
 inline bool pdl_enabled()
 {
     static const bool on = [] { const char* e = getenv("SB_PDL"); return !(e && e[0] == '0'); }();

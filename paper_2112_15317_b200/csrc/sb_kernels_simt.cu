@@ -815,7 +815,7 @@ cudaError_t launch_reduce_sgd(const float* part, size_t stride, size_t n, int sp
 cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n, float lr, float mu, cudaStream_t st)
 {
     size_t n4 = n / 4;
-    static const int per_sm = [] { const char* e = getenv("SB_SGD_BLOCKS_PER_SM"); int k = e ? atoi(e) : 16; return k < 1 ? 1 : k; }();
+    static const int per_sm = (int)tune("SB_SGD_BLOCKS_PER_SM", 16);
     long blocks = ((long)n4 + 255) / 256;
     if (blocks > 148L * per_sm) blocks = 148L * per_sm;
     if (blocks < 1) blocks = 1;

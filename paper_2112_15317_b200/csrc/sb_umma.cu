@@ -80,8 +80,22 @@ struct UmmaParams {
     // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
     // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
     uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
-    unsigned long long* timing;   // optional (SB_UMMA_TIMING=1): per-CTA phase timestamps, 8 per CTA, first 1024 CTAs
+    // Halo variant of the 3x3 FWD / DGRAD kernel (umma_halo_kernel): the pixel box lies in shared memory as [h][n][w] rows
+    // (tile row = wi + bw * (ni + bn * hi)), one activation fetch of bh + 2 image rows serves the three taps of a filter column.
+    int hn_order;         // 1: tile rows in (h, n, w) order; 0: (n, h, w)
+    int a_stages;         // depth of the activation (halo) ring; `stages` is then the depth of the weight ring
+    uint32_t rcp_bwbn;    // reciprocal of bw * bn (hn_order)
+#ifdef SB_CTA_TIMING
+    unsigned long long* timing;   // development builds only: per-CTA phase timestamps, 16 per CTA, first 1024 CTAs
+#endif
 };
+
+// Per-CTA phase stamps: compiled in only with -DSB_CTA_TIMING (a development aid; the shipped kernels carry none).
+#ifdef SB_CTA_TIMING
+#define SB_TLOG(cond, slot, val) do { if (tlog && (cond)) tlog[slot] = (unsigned long long)(val); } while (0)
+#else
+#define SB_TLOG(cond, slot, val) do { } while (0)
+#endif
 
 __host__ __device__ __forceinline__ uint32_t fast_rcp(uint32_t d) { return d <= 1u ? 0u : (uint32_t)(0x100000000ull / d) + 1u; }
 __device__ __forceinline__ int fast_div(int n, uint32_t mul) { return mul == 0u ? n : (int)__umulhi((uint32_t)n, mul); }
@@ -277,8 +291,8 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
 }
 
 // 2x2 max-pool of the output tile staged for the TMA store (64-column slabs of 128 rows x 128 bytes, 16-byte chunks
-// XOR-swizzled by row % 8; tile row = wi + bw * (hi + bh * ni) with bw, bh even, so every pooling window lies inside
-// the tile).  One task = one pooled pixel x 8 channels: four 16-byte shared-memory reads, one 16-byte store of the
+// XOR-swizzled by row % 8; tile row = wi + bw * (hi + bh * ni), or wi + bw * (ni + bn * hi) in the halo kernel's order,
+// with bw, bh even, so every pooling window lies inside the tile).  One task = one pooled pixel x 8 channels: four 16-byte shared-memory reads, one 16-byte store of the
 // maxima and one 8-byte store of the argmax positions (dh*2+dw, the first maximum wins: the same rule and the same
 // bf16 inputs as the stand-alone pooling kernel, so the bytes are identical).  Called by the 128 epilogue threads.
 template <int BN>
@@ -286,19 +300,21 @@ __device__ __forceinline__ void pool_from_stage(const UmmaParams& p, const uint8
 {
     constexpr int CH = BN / 8;
     const int wb = p.bw / 2, hb = p.bh / 2, Ho = p.H / 2, Wo = p.W / 2;
+    // tile row of pixel (wi, hi, ni) = wi + h_step * hi + n_step * ni
+    const int h_step = p.hn_order ? p.bw * p.bn : p.bw, n_step = p.hn_order ? p.bw : p.bw * p.bh;
     for (int t = t128; t < 32 * CH; t += 128) {
         const int c = t % CH, pr = t / CH;
         const int pq = fast_div(pr, p.rcp_wb), nl = fast_div(pr, p.rcp_wbhb);
         const int wl = pr - pq * wb, hl = pq - nl * hb;
         const int w = pw0 + 2 * wl, h = ph0 + 2 * hl, n = pn0 + nl, ncol = n0 + 8 * c;
         if (w >= p.W || h >= p.H || n >= p.N || ncol >= n_hi) continue;
-        const int r00 = 2 * wl + p.bw * (2 * hl + p.bh * nl);
+        const int r00 = 2 * wl + h_step * 2 * hl + n_step * nl;
         const uint8_t* slab = stage + (c >> 3) * 16384;
         const int cj = c & 7;
         uint4 v[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int r = r00 + (j & 1) + (j >> 1) * p.bw;
+            const int r = r00 + (j & 1) + (j >> 1) * h_step;
             v[j] = *(const uint4*)(slab + r * 128 + ((cj ^ (r & 7)) << 4));
         }
         uint4 outv;
@@ -347,8 +363,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+#ifdef SB_CTA_TIMING
     unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 16ull * cta_lin : nullptr;
-    if (tlog && threadIdx.x == 0) { tlog[0] = globaltimer_ns(); tlog[6] = (unsigned long long)clock64(); }
+#endif
+    (void)cta_lin;
+    SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TLOG(threadIdx.x == 0, 6, clock64());
 
     // ---- tile coordinates ---------------------------------------------------------------------
     int tap_fixed = 0, split = 0;
@@ -468,33 +488,33 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             mbar_init(acc_full, 1);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            if (tlog) tlog[8] = (unsigned long long)clock64();    // barriers initialised
+            SB_TLOG(true, 8, clock64());    // barriers initialised
         }
         __syncwarp();
         pdl_wait();
         pdl_trigger();
-        if (tlog && lane == 0) tlog[9] = (unsigned long long)clock64();    // predecessor kernel complete
+        SB_TLOG(lane == 0, 9, clock64());    // predecessor kernel complete
         // The first ring-full of loads needs nothing but the barriers just initialised: start them now, so that
         // their latency overlaps the TMEM allocation and the rest of the set-up.
         prod_el = elect_one() ? 1u : 0u;
         for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
-        if (tlog && lane == 0) tlog[10] = (unsigned long long)clock64();   // first ring of loads issued
+        SB_TLOG(lane == 0, 10, clock64());   // first ring of loads issued
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, C::TMEM_COLS);
         tmem_relinquish();
-        if (tlog && lane == 0) tlog[11] = (unsigned long long)clock64();   // TMEM allocated
+        SB_TLOG(lane == 0, 11, clock64());   // TMEM allocated
     }
     if (warp != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
     if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
         for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
     }
-    if (tlog && threadIdx.x == 64) tlog[12] = (unsigned long long)clock64();   // bias staged
+    SB_TLOG(threadIdx.x == 64, 12, clock64());   // bias staged
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    if (tlog && threadIdx.x == 0) tlog[1] = (unsigned long long)clock64();   // set-up done
+    SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
@@ -535,8 +555,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
                 break;
             }
-            if (tlog && lane == 0 && it == 0) tlog[2] = (unsigned long long)clock64();            // first operands landed
-            if (tlog && lane == 0 && it == n_iters - 1) tlog[3] = (unsigned long long)clock64();  // last operands landed
+            SB_TLOG(lane == 0 && it == 0, 2, clock64());            // first operands landed
+            SB_TLOG(lane == 0 && it == n_iters - 1, 3, clock64());  // last operands landed
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
@@ -596,7 +616,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
-            if (tlog && threadIdx.x == 64) tlog[4] = (unsigned long long)clock64();      // accumulator complete
+            SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             // (the operand ring is idle once the accumulator is complete: its first bytes stage the output tile)
@@ -618,7 +638,254 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
         pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);     // reads the stage while the TMA stores read it too
     if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();   // shared memory may be released once the stores have read it; the writes complete with the grid
-    if (tlog && threadIdx.x == 0) { tlog[5] = (unsigned long long)clock64(); tlog[7] = globaltimer_ns(); }   // epilogue done
+    SB_TLOG(threadIdx.x == 0, 5, clock64());   // epilogue done
+    SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
+    if (*abort_flag) {
+        // give copies that may still be in flight time to land before shared memory is released
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The halo kernel (3x3 FWD / DGRAD): one activation fetch per filter column
+// ------------------------------------------------------------------------------------------------
+// In umma_kernel every (tap, 64-channel chunk) fetches its own 128-pixel activation box, so each activation pixel
+// crosses L2 -> shared memory nine times per chunk and the main loop runs at the rate one SM pulls operands from L2.
+// Here the three taps of one filter COLUMN (same shift in w, shifts -1, 0, +1 in h) share one fetch: the box carries
+// bh + 2 image rows (a halo row above and below), it lies in shared memory as [h][n][w] rows of 128 bytes -- the
+// tensor map lists the dimensions as (c, w, n, h) -- and tap row j = 0, 1, 2 reads the 128 tile rows that start
+// j * bw * bn rows into it.  bw * bn is a multiple of 8, so that start is a whole number of 8-row swizzle groups and
+// only the start address of the shared-memory descriptor moves.  Per 64-channel chunk the activations cross three
+// times (once per shift in w) with (bh + 2) / bh of the box each, instead of nine times.  Zero padding, ragged tile
+// edges and images past the batch are the TMA's out-of-bounds zero fill, as before.
+//
+// Two rings: activation halos (a_stages slots, one per (chunk, w shift) group, released after its three taps) and
+// weight tiles (stages slots, one per tap, as in umma_kernel).  Warp roles, bounded waits, epilogues, the pooled
+// output and programmatic dependent launch are those of umma_kernel; tile row = wi + bw * (ni + bn * hi).
+constexpr int MAX_A_STAGES = 4;
+template <int BN> struct HaloCfg {
+    static constexpr int B_STAGE_BYTES = BN * 128;
+    static constexpr int TMEM_COLS = BN;
+    static constexpr int smem_bytes(int a_stages, int a_slot_bytes, int b_stages)
+    {
+        return a_stages * a_slot_bytes + b_stages * B_STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES;
+    }
+};
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+                 const UmmaParams p)
+{
+    static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "halo kernel: forward and data gradient only");
+    using C = HaloCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int SA = p.a_stages, SB = p.stages;
+    const uint32_t row_step = (uint32_t)(p.bw * p.bn) * 128u;          // bytes between halo rows (a multiple of 1024)
+    const uint32_t a_slot = (uint32_t)(p.bh + 2) * row_step;
+    uint8_t* b_ring = smem + (size_t)SA * a_slot;
+    uint8_t* ctrl = b_ring + (size_t)SB * C::B_STAGE_BYTES;
+    uint64_t* b_full = (uint64_t*)ctrl;               // [MAX_STAGES]
+    uint64_t* b_empty = b_full + MAX_STAGES;          // [MAX_STAGES]
+    uint64_t* a_full = b_empty + MAX_STAGES;          // [MAX_A_STAGES]
+    uint64_t* a_empty = a_full + MAX_A_STAGES;        // [MAX_A_STAGES]
+    uint64_t* acc_full = a_empty + MAX_A_STAGES;      // [1]
+    uint32_t* tmem_slot = (uint32_t*)(acc_full + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* s_bias = (float*)(ctrl + 512);             // [BN]
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+    // ---- tile coordinates ---------------------------------------------------------------------
+    const int m_idx = blockIdx.x, split = blockIdx.z;
+    const int n0 = blockIdx.y * BN, n_hi = p.n_total;
+    if (n0 >= n_hi) return;   // uniform over the CTA, before any barrier or TMEM allocation
+    const int q1 = fast_div_exact(m_idx, p.rcp_tiles_w, p.tiles_w), q2 = fast_div_exact(m_idx, p.rcp_tiles_wh, p.tiles_w * p.tiles_h);
+    const int pw0 = (m_idx - q1 * p.tiles_w) * p.bw;
+    const int ph0 = (q1 - q2 * p.tiles_h) * p.bh;
+    const int pn0 = q2 * p.bn;
+    // this CTA's groups: a contiguous range of the 3 * kchunks (chunk, w shift) groups
+    const int g_begin = split * p.chunks_per_split;
+    const int g_end = min(g_begin + p.chunks_per_split, p.total_chunks);
+    const int n_groups = g_end - g_begin;
+
+    // ---- producer state (whole warp in lock-step, elected issue: see umma_kernel) -----------------
+    int ld_kc = 0, ld_dsi = 0;
+    if (g_begin != 0) { ld_kc = g_begin / 3; ld_dsi = g_begin % 3; }
+    int la_s = 0, lb_s = 0;
+    uint32_t la_off = 0, lb_off = 0;
+    const uint32_t smem0 = smem_u32(smem), bring0 = smem_u32(b_ring);
+    const uint32_t afull0 = smem_u32(&a_full[0]), bfull0 = smem_u32(&b_full[0]);
+    auto issue_halo = [&](uint32_t el) {
+        const uint32_t bar = afull0 + 8u * (uint32_t)la_s;
+        mbar_expect_tx_el(bar, a_slot, el);
+        tma_load_4d_el(&mapA, smem0 + la_off, bar, ld_kc * 64, pw0 + ld_dsi - 1, pn0, ph0 - 1, el);    // (c, w, n, h)
+        ++la_s; la_off += a_slot;
+        if (la_s == SA) { la_s = 0; la_off = 0; }
+    };
+    auto issue_weights = [&](int j, uint32_t el) {
+        // halo row j and w shift ld_dsi - 1 belong to filter tap (r, s) = (j, dsi) in the forward pass and, the
+        // shifts being mirrored, to (2 - j, 2 - dsi) in the data gradient
+        const int tap = MODE == MODE_FWD ? 3 * j + ld_dsi : 3 * (2 - j) + (2 - ld_dsi);
+        const uint32_t dst = bring0 + lb_off, bar = bfull0 + 8u * (uint32_t)lb_s;
+        mbar_expect_tx_el(bar, (uint32_t)C::B_STAGE_BYTES, el);
+        if (MODE == MODE_FWD) {
+            tma_load_4d_el(&mapB, dst, bar, tap * p.w_cols + ld_kc * 64, n0, 0, 0, el);
+        } else {
+#pragma unroll
+            for (int jj = 0; jj < BN / 64; ++jj) tma_load_4d_el(&mapB, dst + jj * 8192, bar, tap * p.w_cols + n0 + 64 * jj, ld_kc * 64, 0, 0, el);
+        }
+        ++lb_s; lb_off += (uint32_t)C::B_STAGE_BYTES;
+        if (lb_s == SB) { lb_s = 0; lb_off = 0; }
+    };
+    auto next_group = [&]() { if (++ld_dsi == 3) { ld_dsi = 0; ++ld_kc; } };
+    // whole groups that fit into both rings without waiting for a release
+    int preloaded = SA < SB / 3 ? SA : SB / 3;
+    if (preloaded > n_groups) preloaded = n_groups;
+
+    // ---- one-time setup -----------------------------------------------------------------------
+    uint32_t prod_el = 0;
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < SB; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
+            for (int s = 0; s < SA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
+            mbar_init(acc_full, 1);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        pdl_wait();
+        pdl_trigger();
+        prod_el = elect_one() ? 1u : 0u;
+        for (int g = 0; g < preloaded; ++g) {
+            issue_halo(prod_el);
+#pragma unroll
+            for (int j = 0; j < 3; ++j) issue_weights(j, prod_el);
+            next_group();
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (warp != 0) pdl_wait();   // every thread that will touch global memory waits for the predecessor kernel
+    if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT && warp >= 2) {
+        for (int c = threadIdx.x - 64; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // =========================== TMA producer ===============================================
+        // slot use counts decide whether a release has to be awaited: use u of a slot waits for release u - 1
+        bool ok = true;
+        for (int g = preloaded; g < n_groups && ok; ++g) {
+            if (g >= SA) {
+                const uint32_t par = (uint32_t)((g / SA - 1) & 1);
+                ok = __all_sync(0xffffffffu, mbar_wait(&a_empty[la_s], par) ? 1 : 0) != 0;
+                if (!ok) break;
+            }
+            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
+            issue_halo(prod_el);
+#pragma unroll 1
+            for (int j = 0; j < 3 && ok; ++j) {
+                const int it = 3 * g + j;
+                if (it >= SB) {
+                    const uint32_t par = (uint32_t)((it / SB - 1) & 1);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&b_empty[lb_s], par) ? 1 : 0) != 0;
+                    if (!ok) break;
+                }
+                issue_weights(j, prod_el);
+            }
+            next_group();
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        __syncwarp();
+    } else if (warp == 1) {
+        // =========================== MMA issuer =================================================
+        constexpr uint32_t idesc = make_idesc(BN, 0, MODE != MODE_FWD);
+        const uint32_t elected = elect_one() ? 1u : 0u;
+        const uint64_t dA0 = make_desc(smem0, 16);
+        const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(bring0, 16) : make_desc(bring0, 8192);
+        const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
+        const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
+        constexpr uint32_t A_STEP = 32u >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
+        constexpr uint32_t BSTAGE16 = (uint32_t)C::B_STAGE_BYTES >> 4;     // the address field counts 16-byte units
+        const uint32_t aslot16 = a_slot >> 4, rowstep16 = row_step >> 4;
+        int sa = 0, sb_ = 0;
+        uint32_t pha = 0, phb = 0, aoff = 0, boff = 0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&a_full[sa], pha) ? 1 : 0) != 0;
+            if (!ok) break;
+#pragma unroll 1
+            for (int j = 0; j < 3; ++j) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&b_full[sb_], phb) ? 1 : 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t alo = a_lo0 + aoff + (uint32_t)j * rowstep16;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_lohi(tmem_base, alo + kk * A_STEP, a_hi, b_lo0 + boff + kk * B_STEP, b_hi, idesc, (g > 0 || j > 0 || kk > 0) ? 1u : 0u, elected);
+                if (elected) umma_commit(&b_empty[sb_]);      // weight slot reusable once these MMAs have read it
+                __syncwarp();
+                ++sb_; boff += BSTAGE16;
+                if (sb_ == SB) { sb_ = 0; boff = 0; phb ^= 1u; }
+            }
+            if (!ok) break;
+            if (elected) umma_commit(&a_empty[sa]);           // halo slot reusable once its three taps have read it
+            __syncwarp();
+            ++sa; aoff += aslot16;
+            if (sa == SA) { sa = 0; aoff = 0; pha ^= 1u; }
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
+        if (ok && elected) umma_commit(acc_full);   // accumulator complete
+        __syncwarp();
+    } else {
+        // =========================== epilogue ===================================================
+        const int q = warp % 4;               // TMEM lane quadrant of this warp
+        const int row = q * 32 + lane;        // accumulator row handled by this thread
+        // tile row = wi + bw * (ni + bn * hi)
+        const int r1 = fast_div(row, p.rcp_bw), hi_ = fast_div(row, p.rcp_bwbn);
+        const int wi = row - r1 * p.bw, ni = r1 - hi_ * p.bn;
+        const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+        const bool row_ok = w < p.W && h < p.H && n < p.N;
+        const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(acc_full, 0);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) {
+            if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+        } else {
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+            // (the rings are idle once the accumulator is complete: their first bytes stage the output tile)
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, p.tma_out ? smem : nullptr, row);
+            if (p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+    }
+
+    // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (p.tma_out && threadIdx.x == 64 && !*abort_flag) {
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j)
+            if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem0 + j * 16384, n0 + 64 * j, pw0, pn0, ph0);    // (c, w, n, h)
+        tma_store_commit();
+    }
+    if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
+        pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);     // reads the stage while the TMA stores read it too
+    if (p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
@@ -1102,15 +1369,19 @@ static_assert(sizeof(OpBlock) <= sizeof(((UmmaOp*)nullptr)->blob), "UmmaOp::blob
 static OpBlock* blk(UmmaOp& op) { return (OpBlock*)op.blob; }
 static const OpBlock* blk(const UmmaOp& op) { return (const OpBlock*)op.blob; }
 
-static unsigned long long* g_timing = nullptr;   // debug only: set through umma_set_timing_buffer
+#ifdef SB_CTA_TIMING
+static unsigned long long* g_timing = nullptr;   // development builds only: set through umma_set_timing_buffer
 void umma_set_timing_buffer(void* dev_ptr) { g_timing = (unsigned long long*)dev_ptr; }
+#endif
 
 static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr)
 {
     const OpBlock* b = blk(op);
     cudaError_t e;
     UmmaParams pp = b->p;
+#ifdef SB_CTA_TIMING
     pp.timing = g_timing;
+#endif
     if (pp.mode != MODE_WGRAD) {
         pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
         pp.rcp_tiles_wh = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h));
@@ -1179,7 +1450,7 @@ struct TilePlan { int bn, splits, cps, stages, pair; };
 // memory <= ~110 KB each, TMEM columns <= 256 each): SB_BWD_COHABIT=0 gives every kernel the full ring again.
 static bool bwd_cohabit()
 {
-    static const bool on = [] { const char* e = getenv("SB_BWD_COHABIT"); return !(e && e[0] == '0'); }();
+    static const bool on = tune("SB_BWD_COHABIT", 1) != 0;
     return on;
 }
 static int cohabit_stages(int bn) { return bn >= 192 ? 2 : (bn >= 128 ? 3 : 4); }
@@ -1206,13 +1477,8 @@ static double plan_cost(int bn, int s, int n_cols_per_shard, int shards, long m_
 static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k_iters, bool backward, bool force_pair)
 {
     TilePlan t;
-    static const bool legacy = [] { const char* e = getenv("SB_PLAN_LEGACY"); return e && e[0] == '1'; }();
     int best_bn = 64, best_s = 1;
-    if (legacy) {
-        best_bn = n_cols_per_shard >= 256 ? 256 : (n_cols_per_shard >= 128 ? 128 : 64);
-        const long tiles = m_tiles * cdiv_i(n_cols_per_shard, best_bn) * shards;
-        while (tiles * best_s < 120 && k_iters / (best_s * 2) >= 4) best_s *= 2;
-    } else {
+    {
         double best = 1e300;
         for (int bn = 64; bn <= 256; bn *= 2) {
             if (bn > 64 && bn / 2 >= n_cols_per_shard) break;      // never wider than the columns need
@@ -1233,18 +1499,17 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         const int two = t.bn >= 256 ? 2 : (t.bn >= 128 ? 3 : 4);
         if (t.bn < 256 && st > two) st = two;
     }
-    static const bool fwd_too = [] { const char* e = getenv("SB_FWD_COHABIT"); return e && e[0] == '1'; }();
+    static const bool fwd_too = tune("SB_FWD_COHABIT", 0) != 0;
     // (a grid that leaves SMs idle need not share its SMs: the other stream's CTAs find free ones; SB_COHABIT_MIN_CTAS)
-    static const long cohabit_min = [] { const char* e = getenv("SB_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
+    static const long cohabit_min = (long)tune("SB_COHABIT_MIN_CTAS", 100);
     if ((backward || fwd_too) && bwd_cohabit() && tiles * t.splits >= cohabit_min && st > cohabit_stages(t.bn)) st = cohabit_stages(t.bn);
     // Grids of more than one CTA per SM: measured, the co-residency of CTAs (their set-up, first loads and
     // epilogues overlap one another's main loops) is worth more than ring depth -- the 1024-CTA 64-wide layer runs
     // 28 us with 2 stages (4 CTAs per SM) against 37 us with 4 and 60 us with 8; beyond 3 stages no layer gains.
     // So the ring is cut down until the CTAs the grid asks for fit side by side (shared memory and TMEM columns
     // permitting), but never below a double buffer.  SB_STAGE_RULE=legacy keeps the older rule above.
-    static const bool legacy_stages = [] { const char* e = getenv("SB_STAGE_RULE"); return e && e[0] == 'l'; }();
-    static const int min_stages = [] { const char* e = getenv("SB_MIN_STAGES"); int k = e ? atoi(e) : 2; return k < 1 ? 1 : k; }();
-    if (!legacy_stages) {
+    static const int min_stages = (int)tune("SB_MIN_STAGES", 2);
+    {
         const long ctas = tiles * t.splits;
         long want = (ctas + 147) / 148;
         if (want > 512 / t.bn) want = 512 / t.bn;
@@ -1260,8 +1525,8 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     // ImageNet sizes the pair kernel is 1.2-1.3x faster where the N tile is 256 wide and the grid fills the
     // machine, slower for 128-wide tiles and for grids of less than a wave (two cluster barriers of fixed cost).
     // SB_PAIR=0 turns it off, SB_PAIR_MIN_CTAS moves the grid-size threshold.
-    static const bool pair_on = [] { const char* e = getenv("SB_PAIR"); return !(e && e[0] == '0'); }();
-    static const long pair_min_ctas = [] { const char* e = getenv("SB_PAIR_MIN_CTAS"); return e ? atol(e) : 1L; }();
+    static const bool pair_on = tune("SB_PAIR", 1) != 0;
+    static const long pair_min_ctas = (long)tune("SB_PAIR_MIN_CTAS", 1);
     t.pair = 0;
     // (SB_FLAG_FORCE_PAIR: every 128- or 256-wide tile, whatever the grid -- for tests at small sizes)
     if ((pair_on && t.bn == 256 && m_tiles % 2 == 0 && tiles * t.splits >= pair_min_ctas) || (force_pair && t.bn >= 128)) {
@@ -1272,7 +1537,7 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
         if ((tiles * t.splits >= 296 || ((backward || fwd_too) && bwd_cohabit() && tiles * t.splits >= cohabit_min)) && pst > ptwo) pst = ptwo;
         t.stages = pst < 1 ? 1 : pst;
     }
-    static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
+    static const bool verbose = tune("SB_PLAN_VERBOSE", 0) != 0;
     if (verbose) fprintf(stderr, "plan: N/shard=%d shards=%d m_tiles=%ld k_iters=%d -> bn=%d splits=%d stages=%d pair=%d\n", n_cols_per_shard, shards, m_tiles, k_iters, t.bn, t.splits, t.stages, t.pair);
     return t;
 }
@@ -1284,16 +1549,9 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
 // SB_WGRAD_SPLITS=legacy restores the older rule (fill 148 CTAs, at least 4 chunks per CTA).
 static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_t grad_floats, double* cost_out = nullptr)
 {
-    static const bool legacy = [] { const char* e = getenv("SB_WGRAD_SPLITS"); return e && e[0] == 'l'; }();
-    if (legacy) {
-        int s = 1;
-        while (ctas_without_split * s < 148 && total_chunks / (s * 2) >= 4) s *= 2;
-        if (cost_out) *cost_out = bn >= 256 ? 0.0 : 1.0;    // legacy: widest tile
-        return s;
-    }
-    static const double reduce_gbs = [] { const char* e = getenv("SB_WGRAD_REDUCE_GBS"); return e ? atof(e) : 3000.0; }();
-    static const double reduce_fixed = [] { const char* e = getenv("SB_WGRAD_REDUCE_US"); return e ? atof(e) : 3.0; }();
-    static const double chunk_scale = [] { const char* e = getenv("SB_WGRAD_CHUNK_SCALE"); return e ? atof(e) : 1.0; }();
+    static const double reduce_gbs = tune("SB_WGRAD_REDUCE_GBS", 3000.0);
+    static const double reduce_fixed = tune("SB_WGRAD_REDUCE_US", 3.0);
+    static const double chunk_scale = tune("SB_WGRAD_CHUNK_SCALE", 1.0);
     const double chunk_us = chunk_scale * (16384.0 + bn * 128.0) / 122.0e3;     // bytes per chunk at ~122 GB/s of L2 per SM
     const double fixed_us = 3.0 + bn / 256.0 * 1.5;               // CTA start + drain + float epilogue
     double best = 1e30; int best_s = 1;
@@ -1312,7 +1570,7 @@ static int wgrad_splits(long ctas_without_split, int total_chunks, int bn, size_
         if (real_s > 1) t += reduce_fixed + (real_s + 1) * (double)grad_floats * 4.0 / (reduce_gbs * 1e3);
         if (t < best) { best = t; best_s = real_s; }
     }
-    static const bool verbose = [] { const char* e = getenv("SB_PLAN_VERBOSE"); return e && e[0] == '1'; }();
+    static const bool verbose = tune("SB_PLAN_VERBOSE", 0) != 0;
     if (verbose) fprintf(stderr, "plan: wgrad base_ctas=%ld chunks=%d bn=%d grad=%zu -> splits=%d (%.1f us)\n", ctas_without_split, total_chunks, bn, grad_floats, best_s, best);
     if (cost_out) *cost_out = best;
     return best_s;
@@ -1353,21 +1611,21 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
     g.wg_m_tiles = cdiv_i(lv.Cout, 128);
     // 64 input channels: one CTA takes a whole filter row (three taps = 192 adjacent gradient columns), so the dy
     // tile is fetched once per three taps (SB_WGRAD_TAPS=1 restores one tap per CTA)
-    static const bool taps1 = [] { const char* e = getenv("SB_WGRAD_TAPS"); return e && e[0] == '1'; }();
+    static const bool taps1 = tune("SB_WGRAD_TAPS", 0) == 1;
     g.wg_tap_group = (lv.Cin == 64 && !taps1) ? 3 : 1;
     if (g.wg_tap_group == 3) g.wg_bn = 192;
     // 128 input channels and at most 128 output channels (one M tile, so no CTA pair): two adjacent taps per CTA as one
     // 256-column tile (dy fetched once per two taps; five tap groups, the last with tap 8 alone).  SB_WGRAD_TAPS=1 turns it off.
     // Taken for long reductions only (ImageNet-size layers: 613 -> 290 us alone); at CIFAR size the kernel alone is 15 %
     // faster but the step is not (its 96 KB ring and 256 TMEM columns leave the data-gradient kernel less room beside it).
-    static const int taps2_min_chunks = [] { const char* e = getenv("SB_WGRAD_TAPS2_MIN_CHUNKS"); return e ? atoi(e) : 2048; }();
+    static const int taps2_min_chunks = (int)tune("SB_WGRAD_TAPS2_MIN_CHUNKS", 2048);
     if (lv.Cin == 128 && lv.Cout <= 128 && !taps1 && g.total_chunks >= taps2_min_chunks) { g.wg_tap_group = 2; g.wg_bn = 256; g.wg_n_tiles = 1; }
     const int tap_groups = (9 + g.wg_tap_group - 1) / g.wg_tap_group;
     double cost = 0.0;
     int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * tap_groups, g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b, &cost);
     // a narrower N tile doubles the CTAs of a grid that leaves SMs idle (e.g. 512 channels at 4x4: 72 CTAs of 256
     // columns against 144 of 128): take it when the same model says it is faster (SB_WGRAD_NARROW=0 keeps the widest)
-    static const bool narrow = [] { const char* e = getenv("SB_WGRAD_NARROW"); return !(e && e[0] == '0'); }();
+    static const bool narrow = tune("SB_WGRAD_NARROW", 1) != 0;
     if (narrow && g.wg_tap_group == 1 && g.wg_bn == 256) {
         double cost2 = 0.0;
         const int n2 = cdiv_i(lv.Cin, 128);
@@ -1438,7 +1696,7 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
 // SB_TMA_OUT=0 keeps the direct row stores.
 static bool tma_out_ok(const OpBlock* b, int cols_per_shard, int shards)
 {
-    static const bool off = [] { const char* e = getenv("SB_TMA_OUT"); return e && e[0] == '0'; }();
+    static const bool off = tune("SB_TMA_OUT", 1) == 0;
     const UmmaParams& p = b->p;
     if (off || p.out_f32 || p.splits > 1 || p.epi == UEPI_F32) return false;
     if (p.n_total % 64 != 0 || p.ldc % 64 != 0) return false;
@@ -1458,7 +1716,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
         const bool want_in_grad = i > 0;
         if (lv.kind == SB_CONV3X3_RELU && !conv_umma_ok(mv, lv, i) && conv_in_umma_supported(lv.Cin, lv.Cout)) {
             // input layer: the weight-gradient kernel fetches dy as [pixels][64] rows, 64 pixels per box
-            static const bool off = [] { const char* e = getenv("SB_CONV_IN_UMMA"); return e && e[0] == '0'; }();
+            static const bool off = tune("SB_CONV_IN_UMMA", 1) == 0;
             if (!off) {
                 if (!mat_map(&um.wgrad.mapA, lv.dact, (long)B * lv.H * lv.W, lv.Cout, 64)) return fail_plan();
                 if (!mat_map(&um.fwd.mapA, lv.act, (long)B * lv.H * lv.W, lv.Cout, 128)) return fail_plan();
@@ -1486,7 +1744,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     if (!act_map(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                     p.tma_out = 1;
                     // a 2x2 max-pool right above: pooled from the staged tile in the same kernel (SB_POOL_FUSE=0: separate kernel)
-                    static const bool pool_fuse = [] { const char* e = getenv("SB_POOL_FUSE"); return !(e && e[0] == '0'); }();
+                    static const bool pool_fuse = tune("SB_POOL_FUSE", 1) != 0;
                     um.pool_fused = false;
                     if (pool_fuse && i + 1 < mv.n_layers && g.bw % 2 == 0 && g.bh % 2 == 0 && lv.W % 2 == 0 && lv.H % 2 == 0 && lv.Cout % 8 == 0) {
                         LayerView nx = layer_view(m, i + 1);
@@ -1540,11 +1798,11 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 }
                 {
                     // grids of fewer than ~100 CTAs leave the other streams whole SMs: no need to keep the ring shallow (measured: -1.5 % step)
-                    static const long wg_cohabit_min = [] { const char* e = getenv("SB_WG_COHABIT_MIN_CTAS"); return e ? atol(e) : 100L; }();
+                    static const long wg_cohabit_min = (long)tune("SB_WG_COHABIT_MIN_CTAS", 100);
                     const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * ((9 + p.tap_group - 1) / p.tap_group) * p.splits;
                     // (the filter-row kernel of a short reduction keeps a third 40 KB stage: CIFAR-size steps -1 to -2.7 %; a long
                     // one leaves the room to the data-gradient kernel beside it: ImageNet-size step +1.9 % with three)
-                    static const int row3_max_cps = [] { const char* e = getenv("SB_WGRAD_ROW3_MAX_CHUNKS"); return e ? atoi(e) : 128; }();
+                    static const int row3_max_cps = (int)tune("SB_WGRAD_ROW3_MAX_CHUNKS", 128);
                     int cap = cohabit_stages(b->bn);
                     if (b->bn == 192 && g.wg_cps <= row3_max_cps) cap = 3;
                     if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cap) p.stages = cap;
@@ -1558,7 +1816,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     // CTA pairs over two neighbouring blocks of 128 output channels: each CTA fetches half of the
                     // activation tile (a smaller stage, a deeper ring in the same shared memory).  The pair kernel
                     // does not sum dy on the side, so the bias gradient is taken by a column-sum kernel (wgrad_pair).
-                    static const bool wg_pair = [] { const char* e = getenv("SB_WG_PAIR"); return !(e && e[0] == '0'); }();
+                    static const bool wg_pair = tune("SB_WG_PAIR", 1) != 0;
                     if (wg_pair && p.tap_group == 1 && (b->bn == 128 || b->bn == 256) && g.wg_m_tiles % 2 == 0 && lv.Cout % 128 == 0) {
                         b->pair = 1;
                         p.bias_fused = 0;

@@ -85,9 +85,10 @@ cudaError_t launch_conv_in_wgrad_umma(const WgradSimtArgs& a, const CUtensorMap&
 const char* umma_last_error();
 // One CTA that waits (bounded by limit_ns) on a barrier nothing completes, then reports through the status word.
 cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cudaStream_t st);
-// Debug aid: when set to a device buffer of 1024*16 uint64, every tensor-core CTA (first 1024 of a launch)
-// records %globaltimer at its phase boundaries: start, set-up done, first / last operands landed,
-// accumulator complete, epilogue done.
+#ifdef SB_CTA_TIMING
+// Development builds only: when set to a device buffer of 1024*16 uint64, every tensor-core CTA (first 1024 of a launch)
+// records clock stamps at its phase boundaries.
 void umma_set_timing_buffer(void* dev_ptr);
+#endif
 
 }  // namespace sb

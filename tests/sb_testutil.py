@@ -27,6 +27,25 @@ def outlier_fraction(a, ref, tol):
     return float(np.mean(np.abs(a - ref) > tol * (np.max(np.abs(ref)) + 1e-30)))
 
 
+class Checks:
+    """Collects (name, value, bound) comparisons so that one run reports every violation, not just the first.
+    `log` keeps everything that was measured (a probe can print it); finish() asserts that nothing exceeded its bound."""
+
+    def __init__(self):
+        self.log = []
+
+    def le(self, name, value, bound):
+        self.log.append((name, float(value), float(bound)))
+
+    def worst(self, prefix):
+        vals = [v for n, v, _ in self.log if str(n).startswith(prefix)]
+        return max(vals) if vals else 0.0
+
+    def finish(self):
+        bad = [(n, v, b) for n, v, b in self.log if not v <= b]
+        assert not bad, "parity bounds exceeded: " + "; ".join(f"{n}: {v:.3e} > {b:.1e}" for n, v, b in bad[:12])
+
+
 def oracle_model(wl, params, bf16, real="float"):
     from oracle import splitbrain_oracle as so
     m = so.from_workload(wl, real=real, bf16=bf16)

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 import sb_inputs as si
-from sb_testutil import device_batch, frob, gpu_model, maxrel, oracle_model, outlier_fraction
+from sb_testutil import Checks, device_batch, gpu_model, maxrel, oracle_model
 
 pytestmark = pytest.mark.gpu
 
@@ -43,113 +43,131 @@ WORKLOADS = {
 }
 
 
-def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, grad_frob_bound=None, flags=0):
-    """Whole iterations, end to end.  Float mode: every tensor within 1e-4.  bf16 mode: forward tensors,
-    loss and updated weights within 1e-2 element-wise; backward tensors are bounded in the Frobenius norm,
-    because a summation-order difference can flip a ReLU mask or a pooling argmax and that moves single
-    gradient elements by their full size (test_layerwise_teacher_forced holds the element-wise bound)."""
+# End-to-end comparisons of whole iterations.
+#
+# Float mode: every tensor of both passes element-wise within 1e-4, the oracle running entirely on its own.
+#
+# bf16 mode.  Forward tensors, row losses and the loss: element-wise max|err|/max|ref| <= 1e-2, the oracle running on
+# its own.  The backward pass is a discontinuous function of the forward tensors: every ReLU mask and pooling route is
+# decided by a stored bf16 activation, and the loss gradient softmax(z) - onehot amplifies a 0.5 % difference of the
+# logits by |z|.  The two forward passes agree only to bf16 rounding (a different fp32 summation order moves a stored
+# value across a rounding boundary now and then, and after a few layers the two runs are two independent roundings of
+# the same network), and on untrained He-initialised networks that is enough to move gradients by 10 - 70 % of their
+# maximum (the oracle's own bf16 and float modes differ by as much: test_oracle_model).  No implementation could hold an
+# element-wise bound there, and a norm-wise bound loose enough to pass is too loose to catch a wrong kernel.  So both
+# sides take the discrete decisions on the SAME stored values: after the forward comparison the oracle adopts the
+# GPU's stored forward state (activations, argmax bytes, logits; all within 1e-2 of its own) and runs ITS backward pass
+# from there.  Then every weight / bias gradient, momentum and updated weight of the GPU's end-to-end backward chain
+# must match element-wise within 1e-2, and every activation gradient within 2e-2: the chain stores up to 18 gradients
+# in bf16 one after the other, and where the two sides round a value to different neighbours the difference (2^-8 of
+# the value) is carried down the chain; 1.03e-2 was measured at the bottom of the 13 conv layers at ImageNet size.
+# Layer by layer, on forced inputs, every one of these tensors holds 1e-2 (layerwise_teacher_forced).
+TOL_DACT_CHAIN = {False: 1e-4, True: 2e-2}
+
+
+def adopt_forward_state(ref, gm, checks=None):
+    """Copies the GPU model's stored forward tensors into ref.om (the oracle), so that the oracle's backward() runs on
+    the same stored activations, pooling routes and logits as the GPU's.  With repeated images (ref.first is set) every
+    copy of an image must be bit-identical on the GPU; the first copy is the one adopted."""
     b = sb()
-    params = si.make_params(wl, bias_std=bias_std)
-    x, y = si.make_batch(wl)
-    om = oracle_model(wl, params, bf16)
-    gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=flags)
-    xs, ys = device_batch(wl, x, y, bf16)
-    xr, yr = si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)
-    tol = TOL[bf16]
+    wl, om = ref.wl, ref.om
+    first_fc = om.first_fc
+    nl = len(wl.layers)
 
-    def check_grad(a, ref, what):
-        if bf16:
-            # flips compound once the weights themselves have drifted: only a sanity bound after step 0
-            bound = (grad_frob_bound or 3 * tol) if what[1] == 0 else 0.3
-            assert frob(a, ref) <= bound, (what, frob(a, ref))
+    def rows_for_oracle(full):          # [B, ...] in GPU batch order -> what the oracle holds
+        if ref.first is None:
+            return [np.ascontiguousarray(full[r * wl.b:(r + 1) * wl.b]) for r in range(wl.R)]
+        if checks is not None:
+            checks.le(("copies of one image identical",), float(not np.array_equal(full, full[ref.first][ref.sel])), 0.0)
+        return [np.ascontiguousarray(full[ref.first])]
+
+    for li in range(first_fc):
+        full = np.concatenate([gm.read(b.SB_T_ACT, li, r, squeeze=False) for r in range(wl.R)])
+        for r, a in enumerate(rows_for_oracle(full)):
+            om.conv_out[r][li] = a.astype(om.dt)
+        if wl.layers[li][0] == si.MAXPOOL2:
+            full = np.concatenate([gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False) for r in range(wl.R)])
+            for r, a in enumerate(rows_for_oracle(full)):
+                om.pool_idx[r][li] = a
+    X = np.concatenate([om.conv_out[r][first_fc - 1].reshape(om.conv_out[r][first_fc - 1].shape[0], -1) for r in range(om.R)])
+    for li in range(first_fc, nl - 1):
+        om.fc_in[li] = X
+        full = gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0]
+        X = rows_for_oracle(full)
+        X = np.concatenate(X).astype(om.dt)
+        om.fc_out[li] = X
+    om.logits = X
+    om.row_loss, om.dZ = om.P.softmax_xent(X, om.labels, 1.0 / om.loss_B)
+
+
+def compare_everything(wl, bf16, steps=2, lr=0.01, mu=0.9, bias_std=0.0, flags=0, checks=None):
+    """Whole iterations, end to end, every tensor of every layer against the oracle (see the comment above)."""
+    ref = Ref(wl, bf16, bias_std, run=False)
+    return end_to_end_vs_ref(ref, steps=steps, lr=lr, mu=mu, checks=checks, flags=flags)
+
+
+class Ref:
+    """The oracle's tensors for one workload, laid out as the GPU holds them (per replica rows).
+
+    distinct = d (full-size runs): the batch is made of d different seeded images, each used B/d times; batch row g
+    holds image (g + g // b) mod d, so the images on the two sides of a replica boundary differ and the copies of one
+    image sit at different positions in different replicas (d = B: all rows distinct).  The oracle then only has to
+    follow d images (with the loss scale 1/B of the full batch); every copy on the GPU must match its original
+    element-wise, and the weight gradients are B/d times those of the d-image batch (the gradient is a sum over
+    rows, and equal rows contribute equally)."""
+
+    def __init__(self, wl, bf16, bias_std, distinct=None, run=True):
+        self.wl, self.bf16 = wl, bf16
+        self.params = si.make_params(wl, bias_std=bias_std)
+        x, y = si.make_batch(wl)
+        self.first = self.sel = None
+        self.ran = run
+        if distinct is None:
+            om = oracle_model(wl, self.params, bf16)
+            self.inputs = (si.split_replicas(x, wl.R), si.split_replicas(y, wl.R))
+            if run:
+                om.forward(*self.inputs)
+                om.backward()
+            self.rows = [np.arange(r * wl.b, (r + 1) * wl.b) for r in range(wl.R)]
+            self.conv_out = lambda r, li: om.conv_out[r][li]
+            self.d_conv = lambda r, li: om.d_conv[r][li]
+            self.pool_idx = lambda r, li: om.pool_idx[r][li]
+            self.full = lambda a: a
+            self.gscale = 1.0
         else:
-            assert maxrel(a, ref) <= tol, (what, maxrel(a, ref))
-
-    for step in range(steps):
-        lo = om.forward(xr, yr)
-        om.backward()
-        gm.forward(xs, ys)
-        gm.backward()
-        lg = gm.loss()
-        assert abs(lg - float(lo)) <= tol * max(1.0, abs(float(lo))), (step, lg, lo)
-        nl = len(wl.layers)
-        for li, (kind, out) in enumerate(wl.layers):
-            if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
-                for r in range(wl.R):
-                    a = gm.read(b.SB_T_ACT, li, r, squeeze=False)
-                    assert maxrel(a, om.conv_out[r][li]) <= tol, ("act", step, li, r)
-                    check_grad(gm.read(b.SB_T_DACT, li, r, squeeze=False), om.d_conv[r][li], ("dact", step, li, r))
-                    if kind == si.MAXPOOL2:
-                        idx = gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False)
-                        mism = float(np.mean(idx != om.pool_idx[r][li]))
-                        # bit-exact in float mode; in bf16 mode end to end a one-ulp difference of a stored activation may move
-                        # an argmax between near-equal neighbours (the layer-wise test checks exactness on forced inputs)
-                        assert mism <= (1e-2 if bf16 else 0.0), ("pool idx", step, li, r, mism)
-            elif kind in (si.FC_RELU, si.FC):
-                a = gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0]
-                assert maxrel(a, om.fc_out[li]) <= tol, ("fc act", step, li)
-                check_grad(gm.read(b.SB_T_DACT, li, 0, squeeze=False)[:, :, 0, 0], om.d_pre[li], ("fc dact", step, li))
-        rl = gm.read(b.SB_T_ROW_LOSS, nl - 1, 0)
-        assert maxrel(rl, om.row_loss) <= tol
-        gg = gm.gather_params(b.SB_T_GRAD_W, b.SB_T_GRAD_B)
-        for li, (a, ref) in enumerate(zip(gg, om.full_grads())):
-            if ref is not None:
-                check_grad(a["w"].reshape(ref["w"].shape), ref["w"], ("grad w", step, li))
-                check_grad(a["b"], ref["b"], ("grad b", step, li))
-        om.sgd_step(lr, mu)
-        gm.sgd_step(lr, mu)
-        for what_w, what_b, ref_list, is_mom in ((b.SB_T_WEIGHT, b.SB_T_BIAS, om.full_params(), False),
-                                                 (b.SB_T_MOM_W, b.SB_T_MOM_B, om.full_mom(), True)):
-            got = gm.gather_params(what_w, what_b)
-            for li, (a, ref) in enumerate(zip(got, ref_list)):
-                if ref is not None:
-                    if is_mom:
-                        check_grad(a["w"].reshape(ref["w"].shape), ref["w"], ("mom w", step, li))
-                    else:
-                        assert maxrel(a["w"].reshape(ref["w"].shape), ref["w"]) <= tol, ("weight", step, li)
-                        if np.max(np.abs(ref["b"])) > 0:
-                            # a bias that started at zero is -lr * (its gradient): same bound as the gradients
-                            check_grad(a["b"], ref["b"], ("bias", step, li))
-    gm.close()
+            assert wl.B % distinct == 0 and (distinct == wl.B or wl.b % distinct == 0)
+            from oracle import splitbrain_oracle as so
+            sub = si.Workload(wl.name + "_distinct", wl.layers, wl.H, wl.W, wl.C, distinct, 1, wl.K)
+            om = so.from_workload(sub, real="float", bf16=bf16, loss_B=wl.B)
+            om.load_params(self.params)
+            self.inputs = ([x[:distinct]], [y[:distinct]])
+            if run:
+                om.forward(*self.inputs)
+                om.backward()
+            g_idx = np.arange(wl.B)
+            sel = (g_idx + g_idx // wl.b) % distinct if distinct < wl.B else g_idx
+            assert (np.bincount(sel, minlength=distinct) == wl.B // distinct).all()
+            self.sel = sel
+            self.first = np.array([int(np.argmax(sel == i)) for i in range(distinct)])
+            x, y = x[sel], y[sel]
+            rows = [sel[r * wl.b:(r + 1) * wl.b] for r in range(wl.R)]
+            self.rows = rows
+            self.conv_out = lambda r, li: om.conv_out[0][li][rows[r]]
+            self.d_conv = lambda r, li: om.d_conv[0][li][rows[r]]
+            self.pool_idx = lambda r, li: om.pool_idx[0][li][rows[r]]
+            self.full = lambda a: a[sel]
+            self.gscale = wl.B / distinct
+        self.om, self.x, self.y = om, x, y
 
 
-def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None, flags=0):
+def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None, flags=0, ref=None):
     """Every layer's kernels on the oracle's own tensors as inputs: forward output, weight/bias gradient
     and input gradient of each layer within the contract tolerance ELEMENT-WISE; pool argmax bit-exact.
-
-    distinct = d (full-size runs): the batch is d different seeded images repeated B/d times.  The oracle then
-    only has to follow d images (with the loss scale 1/B of the full batch); every copy on the GPU must match
-    its original element-wise, and the weight gradients are B/d times those of the d-image batch (the
-    gradient is a sum over rows, and equal rows contribute equally)."""
+    (distinct: see Ref.)"""
     b = sb()
-    params = si.make_params(wl, bias_std=bias_std)
-    x, y = si.make_batch(wl)
-    if distinct is None:
-        om = oracle_model(wl, params, bf16)
-        om.forward(si.split_replicas(x, wl.R), si.split_replicas(y, wl.R))
-        om.backward()
-        rows = [np.arange(r * wl.b, (r + 1) * wl.b) for r in range(wl.R)]
-        conv_out = lambda r, li: om.conv_out[r][li]
-        d_conv = lambda r, li: om.d_conv[r][li]
-        pool_idx = lambda r, li: om.pool_idx[r][li]
-        full = lambda a: a
-        gscale = 1.0
-    else:
-        assert wl.B % distinct == 0
-        from oracle import splitbrain_oracle as so
-        sub = si.Workload(wl.name + "_distinct", wl.layers, wl.H, wl.W, wl.C, distinct, 1, wl.K)
-        om = so.from_workload(sub, real="float", bf16=bf16, loss_B=wl.B)
-        om.load_params(params)
-        om.forward([x[:distinct]], [y[:distinct]])
-        om.backward()
-        sel = np.arange(wl.B) % distinct
-        x, y = x[sel], y[sel]
-        rows = [sel[r * wl.b:(r + 1) * wl.b] for r in range(wl.R)]
-        conv_out = lambda r, li: om.conv_out[0][li][rows[r]]
-        d_conv = lambda r, li: om.d_conv[0][li][rows[r]]
-        pool_idx = lambda r, li: om.pool_idx[0][li][rows[r]]
-        full = lambda a: a[sel]
-        gscale = wl.B / distinct
+    ref = ref or Ref(wl, bf16, bias_std, distinct)
+    om, params, x, y = ref.om, ref.params, ref.x, ref.y
+    conv_out, d_conv, pool_idx, full, gscale = ref.conv_out, ref.d_conv, ref.pool_idx, ref.full, ref.gscale
     gm = gpu_model(wl, params, b.SB_BF16 if bf16 else b.SB_FP32, flags=b.SB_FLAG_INPUT_GRAD | flags)
     xs, ys = device_batch(wl, x, y, bf16)
     tol = TOL[bf16]
@@ -212,6 +230,66 @@ def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None, flags=0):
     gm.close()
 
 
+def end_to_end_vs_ref(ref, steps=1, lr=0.01, mu=0.9, checks=None, flags=0):
+    """Whole iterations on the GPU (forward, backward, update) against the oracle, every row of every tensor, all
+    element-wise.  bf16 mode: the oracle's backward pass runs on the GPU's stored forward state (adopt_forward_state)."""
+    b = sb()
+    wl, bf16, om = ref.wl, ref.bf16, ref.om
+    tol = TOL[bf16]
+    ck = checks if checks is not None else Checks()
+    gm = gpu_model(wl, ref.params, b.SB_BF16 if bf16 else b.SB_FP32, flags=flags)
+    xs, ys = device_batch(wl, ref.x, ref.y, bf16)
+    nl = len(wl.layers)
+    for step in range(steps):
+        if step > 0 or not ref.ran:
+            om.forward(*ref.inputs)
+        gm.forward(xs, ys)
+        gm.backward()
+        ref_loss = float(np.mean(ref.full(om.row_loss)))
+        ck.le(("loss", step), abs(gm.loss() - ref_loss) / max(1.0, abs(ref_loss)), tol)
+        for li, (kind, out) in enumerate(wl.layers):
+            if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
+                for r in range(wl.R):
+                    ck.le(("act", step, li, r), maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), ref.conv_out(r, li)), tol)
+                    if kind == si.MAXPOOL2 and not bf16:
+                        ck.le(("pool idx", step, li, r), float(np.mean(gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False) != ref.pool_idx(r, li))), 0.0)
+            elif kind in (si.FC_RELU, si.FC):
+                ck.le(("fc act", step, li), maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], ref.full(om.fc_out[li])), tol)
+        ck.le(("row loss", step), maxrel(gm.read(b.SB_T_ROW_LOSS, nl - 1, 0), ref.full(om.row_loss)), tol)
+        if bf16:
+            adopt_forward_state(ref, gm, ck)
+        om.backward()
+        for li, (kind, out) in enumerate(wl.layers):
+            if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
+                for r in range(wl.R):
+                    ck.le(("dact", step, li, r), maxrel(gm.read(b.SB_T_DACT, li, r, squeeze=False), ref.d_conv(r, li)), TOL_DACT_CHAIN[bf16])
+            elif kind in (si.FC_RELU, si.FC):
+                ck.le(("fc dact", step, li), maxrel(gm.read(b.SB_T_DACT, li, 0, squeeze=False)[:, :, 0, 0], ref.full(om.d_pre[li])), TOL_DACT_CHAIN[bf16])
+        # with repeated rows the gradient is gscale times the oracle's (equal rows contribute equally): scale the oracle's
+        # gradients in place, so that its own SGD step then yields the momentum and weights to compare with
+        for g in om.grads:
+            for part in (g if isinstance(g, list) else [g] if g is not None else []):
+                part["w"] *= om.dt(ref.gscale)
+                part["b"] *= om.dt(ref.gscale)
+        for li, (a, g) in enumerate(zip(gm.gather_params(b.SB_T_GRAD_W, b.SB_T_GRAD_B), om.full_grads())):
+            if g is not None:
+                ck.le(("grad w", step, li), maxrel(a["w"].reshape(g["w"].shape), g["w"]), tol)
+                ck.le(("grad b", step, li), maxrel(a["b"], g["b"]), tol)
+        om.sgd_step(lr, mu)
+        gm.sgd_step(lr, mu)
+        for what_w, what_b, ref_list, name in ((b.SB_T_WEIGHT, b.SB_T_BIAS, om.full_params(), "weight"),
+                                               (b.SB_T_MOM_W, b.SB_T_MOM_B, om.full_mom(), "mom")):
+            for li, (a, g) in enumerate(zip(gm.gather_params(what_w, what_b), ref_list)):
+                if g is not None:
+                    ck.le((name + " w", step, li), maxrel(a["w"].reshape(g["w"].shape), g["w"]), tol)
+                    if np.max(np.abs(g["b"])) > 0:
+                        ck.le((name + " b", step, li), maxrel(a["b"], g["b"]), tol)
+    gm.close()
+    if checks is None:
+        ck.finish()
+    return ck
+
+
 @pytest.mark.parametrize("name", list(WORKLOADS))
 @pytest.mark.parametrize("bf16", [False, True])
 def test_layerwise_teacher_forced(name, bf16):
@@ -222,6 +300,35 @@ def test_layerwise_teacher_forced(name, bf16):
 @pytest.mark.parametrize("bf16", [False, True])
 def test_two_training_steps_match_oracle(name, bf16):
     compare_everything(WORKLOADS[name](), bf16, steps=2, bias_std=0.2)
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1_b4", "cfg5_b4"])
+def test_bf16_path_against_the_oracle_in_plain_float(name):
+    """The bf16 CUDA path against the oracle WITHOUT any rounding on the oracle's side (float arithmetic throughout):
+    every forward tensor, the logits, the row losses and the loss within 1e-2 element-wise.  (Gradients are not
+    compared here: rounding the stored activations moves ReLU masks and pooling routes, so the gradients of the
+    bf16 network are those of a slightly different function -- the oracle's own bf16 mode, pinned on the CPU side,
+    is the comparand for them.)"""
+    b = sb()
+    wl = si.config(0) if name == "cfg0" else si.config(int(name[3])).with_batch(4)
+    params = si.make_params(wl)
+    x, y = si.make_batch(wl)
+    om = oracle_model(wl, params, False)
+    lo = float(om.forward(si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)))
+    gm = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    gm.forward(xs, ys)
+    ck = Checks()
+    ck.le(("loss",), abs(gm.loss() - lo) / max(1.0, abs(lo)), 1e-2)
+    for li, (kind, out) in enumerate(wl.layers):
+        if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
+            for r in range(wl.R):
+                ck.le(("act", li, r), maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), om.conv_out[r][li]), 1e-2)
+        elif kind in (si.FC_RELU, si.FC):
+            ck.le(("fc act", li), maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], om.fc_out[li]), 1e-2)
+    ck.le(("row loss",), maxrel(gm.read(b.SB_T_ROW_LOSS, len(wl.layers) - 1, 0), om.row_loss), 1e-2)
+    gm.close()
+    ck.finish()
 
 
 @pytest.mark.parametrize("images", [(3, 2), (5, 1)])
@@ -382,7 +489,7 @@ def test_maximum_partition_counts(bf16):
            (si.SOFTMAX_XENT, 64)]
     wl = si.Workload("max_parts", net, 8, 8, 3, 1, 64, 64)
     layerwise_teacher_forced(wl, bf16, bias_std=0.1)
-    compare_everything(wl, bf16, steps=1, bias_std=0.1, grad_frob_bound=0.3 if bf16 else None)
+    compare_everything(wl, bf16, steps=1, bias_std=0.1)
     b = sb()
     with pytest.raises(b.SBError, match="SB_ERR_SHAPE"):
         gpu_model(si.Workload("too_many", net, 8, 8, 3, 1, 65, 64), si.make_params(wl), b.SB_FP32)
