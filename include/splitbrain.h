@@ -70,11 +70,15 @@ enum {
     SB_FLAG_INPUT_GRAD = 1,  /* also compute the gradient w.r.t. the network input (layer 0 dgrad) */
     SB_FLAG_FORCE_SIMT = 2,  /* use the CUDA-core kernels for every layer (cross-check / debugging) */
     SB_FLAG_PROFILE_LAYERS = 4, /* sb_profile_end reports one entry per (kernel class, layer): "name#layer" */
-    SB_FLAG_FORCE_PAIR = 8,  /* run every forward / data-gradient GEMM whose N tile is 128 or 256 wide on CTA pairs
-                                (tcgen05 cta_group::2), whatever the grid size; by default the planner uses pairs only
-                                where they pay (256-wide tiles, at least one wave of CTAs) */
-    SB_FLAG_MODULO_SCHEDULE = 16 /* reserve the buffers and plan the sub-batch kernels sb_modulo_step needs
+    SB_FLAG_FORCE_PAIR = 8,  /* run every forward / data-gradient GEMM whose N tile is 128 or 256 wide, and every conv weight
+                                gradient with 256+ output channels, on CTA pairs (tcgen05 cta_group::2), whatever the size;
+                                by default the planner uses pairs only where they pay (256-wide tiles and at least one wave
+                                of CTAs; weight gradients with long reductions) */
+    SB_FLAG_MODULO_SCHEDULE = 16, /* reserve the buffers and plan the sub-batch kernels sb_modulo_step needs
                                 (batch_per_replica must be a multiple of K; the first layer must not be an FC layer) */
+    SB_FLAG_NO_HALO = 32     /* 3x3 forward / data-gradient GEMMs on the kernel that fetches an activation box per filter tap
+                                instead of the default one that shares a fetch of bh + 2 image rows between the three taps of
+                                a filter column (for tests: both kernels must give the same results) */
 };
 
 typedef struct {

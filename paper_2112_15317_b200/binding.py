@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(HERE, "libsplitbrain.so")
 SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
 SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT = 1, 2, 3, 4, 5
-SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE = 1, 2, 4, 8, 16
+SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO = 1, 2, 4, 8, 16, 32
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
 SB_DT_F32, SB_DT_BF16, SB_DT_U8, SB_DT_I32 = 0, 1, 2, 3

@@ -87,6 +87,8 @@ struct UmmaParams {
     uint32_t rcp_bwbn;    // reciprocal of bw * bn (hn_order)
 #ifdef SB_CTA_TIMING
     unsigned long long* timing;   // development builds only: per-CTA phase timestamps, 16 per CTA, first 1024 CTAs
+    int dbg_skip;                 // development builds only (halo kernel, timing experiments, WRONG results): bit 0 = no activation
+                                  // loads after the first ring, bit 1 = no weight loads after the first ring
 #endif
 };
 
@@ -519,18 +521,31 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (warp == 0) {
         // =========================== TMA producer ===============================================
         // the whole warp in lock-step; slot `ws` is free once the MMAs that read it have completed
+        // Rings of four or more stages are refilled two slots per round: both releases are polled together (two
+        // independent barrier reads in flight) and the loads of both iterations go out back to back.  Taken one slot
+        // at a time, the wait -> issue chain of this warp, not the operand bytes, set the pace of the main loop
+        // (measured with the loads switched off: the same time per iteration).  Shallow rings keep the one-slot step: a
+        // producer that waits for two free slots out of two or three would stall the MMA warp.
         int ws = 0;
         uint32_t wph = 0;
-        for (int it = preloaded; it < n_iters; ++it) {
-            const bool got = __all_sync(0xffffffffu, mbar_wait(&empty[ws], wph) ? 1 : 0) != 0;
-            if (!got) {
-                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
-                break;
+        const int batch = STAGES >= 4 ? 2 : 1;
+        bool got = true;
+        for (int it = preloaded; it < n_iters;) {
+            const int nb = (batch == 2 && it + 1 < n_iters) ? 2 : 1;
+            const int s2 = ws + 1 == STAGES ? 0 : ws + 1;
+            const uint32_t p2 = s2 == 0 ? wph ^ 1u : wph;
+            const bool w1 = mbar_try_wait(&empty[ws], wph), w2 = nb == 2 ? mbar_try_wait(&empty[s2], p2) : true;
+            if (!__all_sync(0xffffffffu, (w1 && w2) ? 1 : 0)) {
+                got = __all_sync(0xffffffffu, (mbar_wait(&empty[ws], wph) && (nb == 1 || mbar_wait(&empty[s2], p2))) ? 1 : 0) != 0;
+                if (!got) break;
             }
-            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
             issue_loads(prod_el);
-            if (++ws == STAGES) { ws = 0; wph ^= 1u; }
+            if (nb == 2) issue_loads(prod_el);
+            if (nb == 2) { ws = s2 + 1; wph = p2; } else { ws = ws + 1; }
+            if (ws == STAGES) { ws = 0; wph ^= 1u; }
+            it += nb;
         }
+        if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -549,23 +564,43 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         int s = 0;
         uint32_t ph = 0, off = 0;
         bool ok = true;
-        for (int it = 0; it < n_iters; ++it) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
-            if (!ok) {
-                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
-                break;
+        // two ring slots per round where the ring is deep enough (see the producer): both full barriers are polled together
+        // and the eight MMAs go out back to back
+        const int batch = STAGES >= 4 ? 2 : 1;
+        for (int it = 0; it < n_iters;) {
+            const int nb = (batch == 2 && it + 1 < n_iters) ? 2 : 1;
+            const int s2 = s + 1 == STAGES ? 0 : s + 1;
+            const uint32_t p2 = s2 == 0 ? ph ^ 1u : ph, off2 = s2 == 0 ? 0u : off + STAGE16;
+            const bool w1 = mbar_try_wait(&full[s], ph), w2 = nb == 2 ? mbar_try_wait(&full[s2], p2) : true;
+            if (!__all_sync(0xffffffffu, w1 ? 1 : 0)) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
+                if (!ok) break;
             }
             SB_TLOG(lane == 0 && it == 0, 2, clock64());            // first operands landed
-            SB_TLOG(lane == 0 && it == n_iters - 1, 3, clock64());  // last operands landed
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
                 umma_bf16_lohi(tmem_base, a_lo0 + off + kk * A_STEP, a_hi, b_lo0 + off + kk * B_STEP, b_hi, idesc, (it > 0 || kk > 0) ? 1u : 0u, elected);
             if (elected) umma_commit(&empty[s]);      // stage reusable once these MMAs have read it
+            if (nb == 2) {
+                if (!__all_sync(0xffffffffu, w2 ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&full[s2], p2) ? 1 : 0) != 0;
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_lohi(tmem_base, a_lo0 + off2 + kk * A_STEP, a_hi, b_lo0 + off2 + kk * B_STEP, b_hi, idesc, 1u, elected);
+                if (elected) umma_commit(&empty[s2]);
+                s = s2; off = off2; ph = p2;
+            }
+            SB_TLOG(lane == 0 && it + nb >= n_iters, 3, clock64());  // last operands landed
             __syncwarp();
             ++s; off += STAGE16;
             if (s == STAGES) { s = 0; off = 0; ph ^= 1u; }
+            it += nb;
         }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
         if (ok && elected) umma_commit(acc_full);   // accumulator complete
         __syncwarp();
     } else {
@@ -702,6 +737,12 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     float* s_bias = (float*)(ctrl + 512);             // [BN]
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+#ifdef SB_CTA_TIMING
+    const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+    unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 16ull * cta_lin : nullptr;
+#endif
+    SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TLOG(threadIdx.x == 0, 6, clock64());
 
     // ---- tile coordinates ---------------------------------------------------------------------
     const int m_idx = blockIdx.x, split = blockIdx.z;
@@ -723,10 +764,19 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     uint32_t la_off = 0, lb_off = 0;
     const uint32_t smem0 = smem_u32(smem), bring0 = smem_u32(b_ring);
     const uint32_t afull0 = smem_u32(&a_full[0]), bfull0 = smem_u32(&b_full[0]);
+    int dbg_a = 0, dbg_b = 0;
+    (void)dbg_a; (void)dbg_b;
     auto issue_halo = [&](uint32_t el) {
         const uint32_t bar = afull0 + 8u * (uint32_t)la_s;
+#ifdef SB_CTA_TIMING
+        if ((p.dbg_skip & 1) && dbg_a++ >= SA) mbar_expect_tx_el(bar, 0u, el);
+        else {
+#endif
         mbar_expect_tx_el(bar, a_slot, el);
         tma_load_4d_el(&mapA, smem0 + la_off, bar, ld_kc * 64, pw0 + ld_dsi - 1, pn0, ph0 - 1, el);    // (c, w, n, h)
+#ifdef SB_CTA_TIMING
+        }
+#endif
         ++la_s; la_off += a_slot;
         if (la_s == SA) { la_s = 0; la_off = 0; }
     };
@@ -735,6 +785,10 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         // shifts being mirrored, to (2 - j, 2 - dsi) in the data gradient
         const int tap = MODE == MODE_FWD ? 3 * j + ld_dsi : 3 * (2 - j) + (2 - ld_dsi);
         const uint32_t dst = bring0 + lb_off, bar = bfull0 + 8u * (uint32_t)lb_s;
+#ifdef SB_CTA_TIMING
+        if ((p.dbg_skip & 2) && dbg_b++ >= SB) mbar_expect_tx_el(bar, 0u, el);
+        else {
+#endif
         mbar_expect_tx_el(bar, (uint32_t)C::B_STAGE_BYTES, el);
         if (MODE == MODE_FWD) {
             tma_load_4d_el(&mapB, dst, bar, tap * p.w_cols + ld_kc * 64, n0, 0, 0, el);
@@ -742,6 +796,9 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 #pragma unroll
             for (int jj = 0; jj < BN / 64; ++jj) tma_load_4d_el(&mapB, dst + jj * 8192, bar, tap * p.w_cols + n0 + 64 * jj, ld_kc * 64, 0, 0, el);
         }
+#ifdef SB_CTA_TIMING
+        }
+#endif
         ++lb_s; lb_off += (uint32_t)C::B_STAGE_BYTES;
         if (lb_s == SB) { lb_s = 0; lb_off = 0; }
     };
@@ -783,29 +840,36 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
-        // slot use counts decide whether a release has to be awaited: use u of a slot waits for release u - 1
+        // One group per round: the releases of its halo slot and of its three weight slots are polled together (four
+        // independent barrier reads in flight instead of four waits one after the other), then the four copies are
+        // issued.  A barrier that has not completed a phase yet reports the phase before its first as complete, so
+        // the first pass over a ring waits for parity 1 and falls through; the parity flips at every wrap.  (Taken
+        // tap by tap, with the wait parities recomputed by division, this loop was what set the pace of the whole
+        // main loop: ~135 cycles per MMA against ~85 this way.)
+        // (the preloaded groups took first uses only: preloaded <= SA and 3 * preloaded <= SB; a ring they filled exactly
+        // has wrapped to slot 0, and its next use waits for the first release)
+        uint32_t pa_par = (preloaded > 0 && la_s == 0) ? 0u : 1u, pb_par = (preloaded > 0 && lb_s == 0) ? 0u : 1u;
         bool ok = true;
-        for (int g = preloaded; g < n_groups && ok; ++g) {
-            if (g >= SA) {
-                const uint32_t par = (uint32_t)((g / SA - 1) & 1);
-                ok = __all_sync(0xffffffffu, mbar_wait(&a_empty[la_s], par) ? 1 : 0) != 0;
+        for (int g = preloaded; g < n_groups; ++g) {
+            const int s1 = lb_s, s2 = s1 + 1 == SB ? 0 : s1 + 1, s3 = s2 + 1 == SB ? 0 : s2 + 1;
+            const uint32_t p1 = pb_par, p2 = s2 == 0 ? p1 ^ 1u : p1, p3 = s3 == 0 ? p2 ^ 1u : p2;
+            const bool w0 = mbar_try_wait(&a_empty[la_s], pa_par), w1 = mbar_try_wait(&b_empty[s1], p1),
+                       w2 = mbar_try_wait(&b_empty[s2], p2), w3 = mbar_try_wait(&b_empty[s3], p3);
+            if (!__all_sync(0xffffffffu, (w0 && w1 && w2 && w3) ? 1 : 0)) {
+                ok = __all_sync(0xffffffffu, (mbar_wait(&a_empty[la_s], pa_par) && mbar_wait(&b_empty[s1], p1) &&
+                                              mbar_wait(&b_empty[s2], p2) && mbar_wait(&b_empty[s3], p3)) ? 1 : 0) != 0;
                 if (!ok) break;
             }
-            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
+            const bool a_wraps = la_s + 1 == SA;
             issue_halo(prod_el);
-#pragma unroll 1
-            for (int j = 0; j < 3 && ok; ++j) {
-                const int it = 3 * g + j;
-                if (it >= SB) {
-                    const uint32_t par = (uint32_t)((it / SB - 1) & 1);
-                    ok = __all_sync(0xffffffffu, mbar_wait(&b_empty[lb_s], par) ? 1 : 0) != 0;
-                    if (!ok) break;
-                }
-                issue_weights(j, prod_el);
-            }
+            if (a_wraps) pa_par ^= 1u;
+#pragma unroll
+            for (int j = 0; j < 3; ++j) issue_weights(j, prod_el);
+            pb_par = (s3 + 1 == SB) ? p3 ^ 1u : p3;
             next_group();
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
@@ -824,26 +888,50 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         int sa = 0, sb_ = 0;
         uint32_t pha = 0, phb = 0, aoff = 0, boff = 0;
         bool ok = true;
-        for (int g = 0; g < n_groups && ok; ++g) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&a_full[sa], pha) ? 1 : 0) != 0;
-            if (!ok) break;
-#pragma unroll 1
-            for (int j = 0; j < 3; ++j) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&b_full[sb_], phb) ? 1 : 0) != 0;
+        // One group per round: the four full barriers are polled together, then the twelve MMAs go out back to back
+        // (a tap whose weights had not landed at the poll is waited for just before its own four).
+        for (int g = 0; g < n_groups; ++g) {
+            const int s1 = sb_, s2 = s1 + 1 == SB ? 0 : s1 + 1, s3 = s2 + 1 == SB ? 0 : s2 + 1;
+            const uint32_t p1 = phb, p2 = s2 == 0 ? p1 ^ 1u : p1, p3 = s3 == 0 ? p2 ^ 1u : p2;
+            const uint32_t o1 = boff, o2 = s2 == 0 ? 0u : o1 + BSTAGE16, o3 = s3 == 0 ? 0u : o2 + BSTAGE16;
+            const bool w0 = mbar_try_wait(&a_full[sa], pha), w1 = mbar_try_wait(&b_full[s1], p1), w2 = mbar_try_wait(&b_full[s2], p2),
+                       w3 = mbar_try_wait(&b_full[s3], p3);
+            if (!__all_sync(0xffffffffu, (w0 && w1) ? 1 : 0)) {
+                ok = __all_sync(0xffffffffu, (mbar_wait(&a_full[sa], pha) && mbar_wait(&b_full[s1], p1)) ? 1 : 0) != 0;
+                if (!ok) break;
+            }
+            SB_TLOG(lane == 0 && g == 0, 2, clock64());                    // first operands landed
+            tc_fence_after();
+            const uint32_t alo = a_lo0 + aoff;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_lohi(tmem_base, alo + kk * A_STEP, a_hi, b_lo0 + o1 + kk * B_STEP, b_hi, idesc, (g > 0 || kk > 0) ? 1u : 0u, elected);
+            if (elected) umma_commit(&b_empty[s1]);      // weight slot reusable once these MMAs have read it
+            if (!__all_sync(0xffffffffu, w2 ? 1 : 0)) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&b_full[s2], p2) ? 1 : 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t alo = a_lo0 + aoff + (uint32_t)j * rowstep16;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16_lohi(tmem_base, alo + kk * A_STEP, a_hi, b_lo0 + boff + kk * B_STEP, b_hi, idesc, (g > 0 || j > 0 || kk > 0) ? 1u : 0u, elected);
-                if (elected) umma_commit(&b_empty[sb_]);      // weight slot reusable once these MMAs have read it
-                __syncwarp();
-                ++sb_; boff += BSTAGE16;
-                if (sb_ == SB) { sb_ = 0; boff = 0; phb ^= 1u; }
             }
-            if (!ok) break;
-            if (elected) umma_commit(&a_empty[sa]);           // halo slot reusable once its three taps have read it
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_lohi(tmem_base, alo + rowstep16 + kk * A_STEP, a_hi, b_lo0 + o2 + kk * B_STEP, b_hi, idesc, 1u, elected);
+            if (elected) umma_commit(&b_empty[s2]);
+            if (!__all_sync(0xffffffffu, w3 ? 1 : 0)) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&b_full[s3], p3) ? 1 : 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+            }
+            SB_TLOG(lane == 0 && g == n_groups - 1, 3, clock64());         // last operands landed
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_lohi(tmem_base, alo + 2 * rowstep16 + kk * A_STEP, a_hi, b_lo0 + o3 + kk * B_STEP, b_hi, idesc, 1u, elected);
+            if (elected) {
+                umma_commit(&b_empty[s3]);
+                umma_commit(&a_empty[sa]);               // halo slot reusable once its three taps have read it
+            }
             __syncwarp();
+            sb_ = s3 + 1; boff = o3 + BSTAGE16; phb = p3;
+            if (sb_ == SB) { sb_ = 0; boff = 0; phb ^= 1u; }
             ++sa; aoff += aslot16;
             if (sa == SA) { sa = 0; aoff = 0; pha ^= 1u; }
         }
@@ -866,6 +954,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         if (!ok) {
             if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         } else {
+            SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             // (the rings are idle once the accumulator is complete: their first bytes stage the output tile)
@@ -886,6 +975,8 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     if (MODE == MODE_FWD && p.tma_out && p.pool_out != nullptr && warp >= 2 && !*abort_flag)
         pool_from_stage<BN>(p, smem, threadIdx.x - 64, n0, n_hi, pw0, ph0, pn0);     // reads the stage while the TMA stores read it too
     if (p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();
+    SB_TLOG(threadIdx.x == 0, 5, clock64());   // epilogue done
+    SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
@@ -1117,18 +1208,27 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
+        // (two slots per round on rings of four or more stages: see the single-CTA kernel)
         int ws = 0;
         uint32_t wph = 0;
-        for (int it = preloaded; it < n_iters; ++it) {
-            const bool got = __all_sync(0xffffffffu, mbar_wait(&empty[ws], wph) ? 1 : 0) != 0;
-            if (!got) {
-                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
-                break;
+        const int batch = STAGES >= 4 ? 2 : 1;
+        bool got = true;
+        for (int it = preloaded; it < n_iters;) {
+            const int nb = (batch == 2 && it + 1 < n_iters) ? 2 : 1;
+            const int s2 = ws + 1 == STAGES ? 0 : ws + 1;
+            const uint32_t p2 = s2 == 0 ? wph ^ 1u : wph;
+            const bool w1 = mbar_try_wait(&empty[ws], wph), w2 = nb == 2 ? mbar_try_wait(&empty[s2], p2) : true;
+            if (!__all_sync(0xffffffffu, (w1 && w2) ? 1 : 0)) {
+                got = __all_sync(0xffffffffu, (mbar_wait(&empty[ws], wph) && (nb == 1 || mbar_wait(&empty[s2], p2))) ? 1 : 0) != 0;
+                if (!got) break;
             }
-            if (__any_sync(0xffffffffu, *abort_flag ? 1 : 0)) break;
             issue_loads(prod_el);
-            if (++ws == STAGES) { ws = 0; wph ^= 1u; }
+            if (nb == 2) issue_loads(prod_el);
+            if (nb == 2) { ws = s2 + 1; wph = p2; } else { ws = ws + 1; }
+            if (ws == STAGES) { ws = 0; wph ^= 1u; }
+            it += nb;
         }
+        if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
         __syncwarp();
     } else if (warp == 1) {
         if (leader) {
@@ -1147,21 +1247,40 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             constexpr uint32_t STAGE16 = (uint32_t)C::STAGE_BYTES >> 4;
             int s = 0;
             uint32_t ph = 0, off = 0;
-            for (int it = 0; it < n_iters && ok; ++it) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
-                if (!ok) {
-                    if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
-                    break;
+            const int batch = STAGES >= 4 ? 2 : 1;
+            const bool tmem_ok = ok;
+            for (int it = 0; it < n_iters && ok;) {
+                const int nb = (batch == 2 && it + 1 < n_iters) ? 2 : 1;
+                const int s2 = s + 1 == STAGES ? 0 : s + 1;
+                const uint32_t p2 = s2 == 0 ? ph ^ 1u : ph, off2 = s2 == 0 ? 0u : off + STAGE16;
+                const bool w1 = mbar_try_wait(&full[s], ph), w2 = nb == 2 ? mbar_try_wait(&full[s2], p2) : true;
+                if (!__all_sync(0xffffffffu, w1 ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&full[s], ph) ? 1 : 0) != 0;
+                    if (!ok) break;
                 }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     umma_bf16_pair_lohi(tmem_base, a_lo0 + off + kk * A_STEP, a_hi, b_lo0 + off + kk * B_STEP, b_hi, idesc, (it > 0 || kk > 0) ? 1u : 0u, elected);
                 if (elected) umma_commit_pair(&empty[s]);
+                if (nb == 2) {
+                    if (!__all_sync(0xffffffffu, w2 ? 1 : 0)) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&full[s2], p2) ? 1 : 0) != 0;
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_bf16_pair_lohi(tmem_base, a_lo0 + off2 + kk * A_STEP, a_hi, b_lo0 + off2 + kk * B_STEP, b_hi, idesc, 1u, elected);
+                    if (elected) umma_commit_pair(&empty[s2]);
+                    s = s2; off = off2; ph = p2;
+                }
                 __syncwarp();
                 ++s; off += STAGE16;
                 if (s == STAGES) { s = 0; off = 0; ph ^= 1u; }
+                it += nb;
             }
+            if (tmem_ok && !ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
             if (ok && elected) umma_commit_pair(acc_full);
             __syncwarp();
         }
@@ -1268,6 +1387,15 @@ static bool act_map(CUtensorMap* map, const void* ptr, int N, int H, int W, int 
     uint32_t b[4] = {64, (uint32_t)bw, (uint32_t)bh, (uint32_t)bn};
     return encode_map(map, ptr, d, s, b);
 }
+// The same tensor with the dimensions listed as (C, W, N, H) and a (64, bw, bn, bh) box: the box then lies in shared
+// memory as [h][n][w] rows, which is what the halo kernel wants (a shift in h is a whole number of bw * bn rows).
+static bool act_map_hn(CUtensorMap* map, const void* ptr, int N, int H, int W, int C, int bw, int bh, int bn)
+{
+    uint64_t d[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)N, (uint64_t)H};
+    uint64_t s[3] = {(uint64_t)C * 2, (uint64_t)H * W * C * 2, (uint64_t)W * C * 2};
+    uint32_t b[4] = {64, (uint32_t)bw, (uint32_t)bn, (uint32_t)bh};
+    return encode_map(map, ptr, d, s, b);
+}
 // Row-major matrix [rows][cols] bf16 -> map (cols, rows, 1, 1) with a (64, box_rows, 1, 1) box.
 static bool mat_map(CUtensorMap* map, const void* ptr, long rows, long cols, int box_rows)
 {
@@ -1298,27 +1426,66 @@ static void choose_box(int W, int H, int N, int target, int* bw, int* bh, int* b
 template <int MODE, int BN>
 static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Cfg<MODE, BN>::smem_bytes(Cfg<MODE, BN>::MAX_STAGES_FIT));
+    // (the attribute belongs to the device's copy of the function: set it once per device)
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg<MODE, BN>::smem_bytes(Cfg<MODE, BN>::MAX_STAGES_FIT));
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     if (p.stages < 1 || p.stages > Cfg<MODE, BN>::MAX_STAGES_FIT) return cudaErrorInvalidValue;
     return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, op.mapC, p);
+}
+
+template <int MODE, int BN>
+static cudaError_t launch_halo_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    const int a_slot = (p.bh + 2) * p.bw * p.bn * 128;
+    const int smem = HaloCfg<BN>::smem_bytes(p.a_stages, a_slot, p.stages);
+    if (p.a_stages < 1 || p.a_stages > MAX_A_STAGES || p.stages < 1 || p.stages > MAX_STAGES || smem > 227 * 1024) return cudaErrorInvalidValue;
+    // (the attribute belongs to the device's copy of the function: set it once per device)
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(umma_halo_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    return pdl_launch(umma_halo_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)smem, st, op.mapA, op.mapB, op.mapC, p);
+}
+template <int MODE>
+static cudaError_t launch_halo_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    switch (bn) {
+    case 64: return launch_halo_one<MODE, 64>(op, p, grid, st);
+    case 128: return launch_halo_one<MODE, 128>(op, p, grid, st);
+    case 256: return launch_halo_one<MODE, 256>(op, p, grid, st);
+    default: return cudaErrorInvalidValue;
+    }
 }
 
 // CTA-pair launch: clusters of two CTAs along x, programmatic dependent launch as everywhere else.
 template <int MODE, int BN>
 static cudaError_t launch_pair_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             PairCfg<BN>::smem_bytes(PairCfg<BN>::MAX_STAGES_FIT));
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(umma_pair_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PairCfg<BN>::smem_bytes(PairCfg<BN>::MAX_STAGES_FIT));
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     if (p.stages < 1 || p.stages > PairCfg<BN>::MAX_STAGES_FIT || (grid.x & 1u)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
@@ -1362,6 +1529,7 @@ struct OpBlock {
     UmmaParams p;
     int bn;
     int pair;      // FWD / DGRAD: run as CTA pairs (umma_pair_kernel); grid.x is then even
+    int halo;      // 3x3 FWD / DGRAD: umma_halo_kernel (activation halos shared by the three taps of a filter column)
     dim3 grid;
     long rows;     // output rows (pixels / batch rows) of a FWD / DGRAD op
 };
@@ -1381,6 +1549,7 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     UmmaParams pp = b->p;
 #ifdef SB_CTA_TIMING
     pp.timing = g_timing;
+    pp.dbg_skip = (int)tune("SB_HALO_SKIP", 0);
 #endif
     if (pp.mode != MODE_WGRAD) {
         pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
@@ -1389,8 +1558,11 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
         pp.rcp_bwbh = fast_rcp((uint32_t)(pp.bw * pp.bh));
         pp.rcp_wb = fast_rcp((uint32_t)(pp.bw / 2));
         pp.rcp_wbhb = fast_rcp((uint32_t)((pp.bw / 2) * (pp.bh / 2)));
+        pp.rcp_bwbn = fast_rcp((uint32_t)(pp.bw * pp.bn));
     }
-    if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    if (b->halo && b->p.mode == MODE_FWD) e = launch_halo_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    else if (b->halo && b->p.mode == MODE_DGRAD) e = launch_halo_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
+    else if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_DGRAD) e = launch_pair_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_WGRAD) e = launch_pair_mode<MODE_WGRAD>(b->bn, op, pp, b->grid, st);
     else if (b->p.mode == MODE_FWD) e = launch_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
@@ -1445,7 +1617,7 @@ cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cud
 //    reduced in split order by splitk_epilogue) while every CTA keeps at least 4 k-iterations,
 //  * ring depth = k-iterations per CTA, capped by what fits; for grids of several waves the ring is kept
 //    shallow enough that two CTAs share an SM, so one CTA's epilogue overlaps the other's main loop.
-struct TilePlan { int bn, splits, cps, stages, pair; };
+struct TilePlan { int bn, splits, cps, stages, pair, halo, a_stages; };
 // Backward kernels of the two concurrent streams share SMs only if two CTAs fit side by side (shared
 // memory <= ~110 KB each, TMEM columns <= 256 each): SB_BWD_COHABIT=0 gives every kernel the full ring again.
 static bool bwd_cohabit()
@@ -1528,6 +1700,8 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     static const bool pair_on = tune("SB_PAIR", 1) != 0;
     static const long pair_min_ctas = (long)tune("SB_PAIR_MIN_CTAS", 1);
     t.pair = 0;
+    t.halo = 0;
+    t.a_stages = 0;
     // (SB_FLAG_FORCE_PAIR: every 128- or 256-wide tile, whatever the grid -- for tests at small sizes)
     if ((pair_on && t.bn == 256 && m_tiles % 2 == 0 && tiles * t.splits >= pair_min_ctas) || (force_pair && t.bn >= 128)) {
         t.pair = 1;
@@ -1539,6 +1713,90 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     }
     static const bool verbose = tune("SB_PLAN_VERBOSE", 0) != 0;
     if (verbose) fprintf(stderr, "plan: N/shard=%d shards=%d m_tiles=%ld k_iters=%d -> bn=%d splits=%d stages=%d pair=%d\n", n_cols_per_shard, shards, m_tiles, k_iters, t.bn, t.splits, t.stages, t.pair);
+    return t;
+}
+
+// Pixel box of the halo kernel: bw * bh * bn = 128 (powers of two) with bw * bn a multiple of 8 (a shift by one image
+// row is then a whole number of 8-row swizzle groups) and bh even (pooling windows inside the tile).  Least padded
+// volume, weighted by the halo rows a box of that height fetches on top of its own ((bh + 2) / bh, of which the
+// activations are about half of a CTA's operand bytes).
+static bool choose_box_halo(int W, int H, int N, int* bw, int* bh, int* bn)
+{
+    double best = 1e300;
+    bool found = false;
+    for (int w = 1; w <= 128; w *= 2)
+        for (int h = 2; w * h <= 128; h *= 2) {
+            const int n = 128 / (w * h);
+            if ((w * n) % 8 != 0 || n > 256 || w > 256) continue;
+            const double vol = (double)cdiv_i(W, w) * w * cdiv_i(H, h) * h * cdiv_i(N, n) * n;
+            const double score = vol * (1.0 + 1.0 / h) * (1.0 - 1e-6 * w);
+            if (score < best) { best = score; *bw = w; *bh = h; *bn = n; found = true; }
+        }
+    return found;
+}
+// Tile plan of a halo-kernel op (see plan_tiles for the ideas): the reduction is 3 * kchunks groups of three taps.  The
+// main loop is paced by the issuing warps, not by operand bytes: measured with the loads switched off it takes as long as
+// with them, ~70 / 85 / 145 cycles per MMA for 64 / 128 / 256 columns (four MMAs per tap) once the producer and the
+// MMA warp handle a whole group per round; the rings must then hold two groups of weight tiles or the producer, which
+// waits for a whole group of free slots, falls behind (a ring of 4 runs at half the rate of a ring of 8).
+static TilePlan plan_tiles_halo(int n_cols, long m_tiles, int kchunks, int a_slot_bytes, bool backward)
+{
+    TilePlan t{};
+    t.halo = 1;
+    const int groups = 3 * kchunks;
+    double best = 1e300;
+    int best_bn = 64, best_s = 1;
+    static const double fixed_us = tune("SB_HALO_FIXED_US", 3.0), share_factor = tune("SB_HALO_SHARE", 1.6);
+    static const double tap64 = tune("SB_HALO_TAP64", 0.16), tap128 = tune("SB_HALO_TAP128", 0.19), tap256 = tune("SB_HALO_TAP256", 0.33);
+    for (int bn = 64; bn <= 256; bn *= 2) {
+        if (bn > 64 && bn / 2 >= n_cols) break;
+        const double t_tap = bn >= 256 ? tap256 : (bn >= 128 ? tap128 : tap64);
+        for (int s = 1; s <= 32 && (s == 1 || groups / s >= 2); s *= 2) {
+            const long ctas = m_tiles * cdiv_i(n_cols, bn) * s;
+            const double per_sm = (bn < 256 && ctas >= 296) ? 2.0 : 1.0;
+            const double waves = (double)cdiv_i(ctas, (long)(148 * per_sm));
+            const double partial_mb = (double)s * (double)m_tiles * 128.0 * (double)n_cols * 4.0 / 1.0e6;
+            const double c = waves * (cdiv_i(groups, s) * 3.0 * t_tap * (per_sm > 1.0 ? share_factor : 1.0) + fixed_us) + (s > 1 ? 4.0 + 0.5 * partial_mb : 0.0);
+            if (c < best - 1e-9) { best = c; best_bn = bn; best_s = s; }
+        }
+    }
+    {
+        static const int f_bn = (int)tune("SB_HALO_BN", 0);
+        if (f_bn > 0 && f_bn <= n_cols) { best_bn = f_bn; }
+    }
+    t.bn = best_bn;
+    t.cps = cdiv_i(groups, best_s);            // groups per CTA
+    t.splits = cdiv_i(groups, t.cps);
+    const long ctas = m_tiles * cdiv_i(n_cols, t.bn) * t.splits;
+    // Rings: as many CTAs side by side as the grid has per SM (TMEM columns and a two-group weight ring permitting, four
+    // at most; backward grids of 100 CTAs or more leave room for a CTA of the weight-gradient streams), and within that
+    // share of the shared memory the deepest rings.
+    static const long cohabit_min = (long)tune("SB_COHABIT_MIN_CTAS", 100);
+    long want = (ctas + 147) / 148;
+    if (want > 512 / t.bn) want = 512 / t.bn;
+    if (want > 4) want = 4;
+    if (want < 2 && backward && bwd_cohabit() && ctas >= cohabit_min && t.bn < 256) want = 2;
+    const int b_stage = t.bn * 128;
+    int sa = 2, sb = 0;
+    for (; want >= 1; --want) {
+        const int budget = (int)(227 * 1024 / want) - 4 * 1024;
+        sb = (budget - 2 * a_slot_bytes) / b_stage;
+        if (sb >= 6 || want == 1) break;
+    }
+    if (sb > MAX_STAGES) sb = MAX_STAGES;
+    if (sb < 3) sb = 3;
+    if (want <= 1 && 227 * 1024 - 4 * 1024 - 3 * a_slot_bytes - sb * b_stage >= 0) sa = 3;
+    {
+        static const int f_sa = (int)tune("SB_HALO_SA", 0), f_sb = (int)tune("SB_HALO_SB", 0);
+        if (f_sa > 0) sa = f_sa;
+        if (f_sb > 0) sb = f_sb;
+    }
+    if (sa > t.cps) sa = t.cps;
+    if (sb > 3 * t.cps) sb = 3 * t.cps;
+    t.a_stages = sa;
+    t.stages = sb;
+    static const bool verbose = tune("SB_PLAN_VERBOSE", 0) != 0;
+    if (verbose) fprintf(stderr, "plan: halo N=%d m_tiles=%ld kchunks=%d a_slot=%d -> bn=%d splits=%d a_stages=%d b_stages=%d (%.1f us)\n", n_cols, m_tiles, kchunks, a_slot_bytes, t.bn, t.splits, t.a_stages, t.stages, best);
     return t;
 }
 
@@ -1590,19 +1848,43 @@ static bool fc_umma_ok(const ModelView& mv, const LayerView& lv, int layer)
 // Geometry shared by the scratch sizing pass and the real planning pass.
 struct ConvGeom {
     int bw, bh, bn, tw, th, tn;      // 128-pixel boxes (FWD / DGRAD M tiles)
+    int halo;                        // the forward / data-gradient ops run on umma_halo_kernel (box chosen for it)
     long m_tiles;
     TilePlan fwd, dgrad;
     int cw, ch, cn, ctw, cth, ctn, total_chunks;   // 64-pixel boxes (WGRAD k-chunks)
     int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps, wg_tap_group;
 };
-static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair)
+static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_halo)
 {
     ConvGeom g;
-    choose_box(lv.W, lv.H, B, 128, &g.bw, &g.bh, &g.bn);
-    g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
-    g.m_tiles = (long)g.tw * g.th * g.tn;
-    g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64), false, force_pair);
-    g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64), true, force_pair);
+    static const bool halo_on = tune("SB_HALO", 1) != 0;
+    g.halo = 0;
+    // The halo kernel wants deep rings (two groups of weight tiles in flight), so one CTA fills an SM's shared memory; a
+    // grid of several CTAs per SM does better on the per-tap kernel, whose two-stage rings let four CTAs share an SM and
+    // overlap their set-up and epilogue phases (measured at CIFAR size: 1024 tiles of 64 columns 25 us against 29 us).
+    static const long halo_max_tiles = (long)tune("SB_HALO_MAX_TILES", 160);
+    int hbw = 0, hbh = 0, hbn = 0;
+    bool halo = halo_on && !force_pair && !no_halo && choose_box_halo(lv.W, lv.H, B, &hbw, &hbh, &hbn);
+    if (halo) {
+        const long mt = (long)cdiv_i(lv.W, hbw) * cdiv_i(lv.H, hbh) * cdiv_i(B, hbn);
+        const int widest = lv.Cout < lv.Cin ? lv.Cout : lv.Cin;
+        if (mt * cdiv_i(widest, widest >= 128 ? 128 : 64) > halo_max_tiles) halo = false;
+    }
+    if (halo) {
+        g.bw = hbw; g.bh = hbh; g.bn = hbn;
+        g.halo = 1;
+        g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
+        g.m_tiles = (long)g.tw * g.th * g.tn;
+        const int a_slot = (g.bh + 2) * g.bw * g.bn * 128;
+        g.fwd = plan_tiles_halo(lv.Cout, g.m_tiles, lv.Cin / 64, a_slot, false);
+        g.dgrad = plan_tiles_halo(lv.Cin, g.m_tiles, lv.Cout / 64, a_slot, true);
+    } else {
+        choose_box(lv.W, lv.H, B, 128, &g.bw, &g.bh, &g.bn);
+        g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
+        g.m_tiles = (long)g.tw * g.th * g.tn;
+        g.fwd = plan_tiles(lv.Cout, 1, g.m_tiles, 9 * (lv.Cin / 64), false, force_pair);
+        g.dgrad = plan_tiles(lv.Cin, 1, g.m_tiles, 9 * (lv.Cout / 64), true, force_pair);
+    }
     choose_box(lv.W, lv.H, B, 64, &g.cw, &g.ch, &g.cn);
     g.ctw = cdiv_i(lv.W, g.cw); g.cth = cdiv_i(lv.H, g.ch); g.ctn = cdiv_i(B, g.cn);
     g.total_chunks = g.ctw * g.cth * g.ctn;
@@ -1657,7 +1939,7 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
     for (int i = 0; i < mv.n_layers; ++i) {
         LayerView lv = layer_view(m, i);
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            ConvGeom g = conv_geom(lv, mv.B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
+            ConvGeom g = conv_geom(lv, mv.B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0);
             const size_t pix = (size_t)mv.B * lv.H * lv.W;
             if (g.wg_splits > 1) upd((size_t)g.wg_splits * (lv.n_w + lv.n_b));
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * pix * lv.Cout);
@@ -1684,6 +1966,9 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
     p.chunks_per_split = t.cps;
     p.splits = t.splits;
     p.stages = t.stages;
+    p.a_stages = t.a_stages;
+    p.hn_order = t.halo;
+    b->halo = t.halo;
     p.part = t.splits > 1 ? ws : nullptr;
     p.split_stride = (long)(rows * (size_t)p.n_total);
     b->pair = t.pair;
@@ -1701,6 +1986,7 @@ static bool tma_out_ok(const OpBlock* b, int cols_per_shard, int shards)
     if (off || p.out_f32 || p.splits > 1 || p.epi == UEPI_F32) return false;
     if (p.n_total % 64 != 0 || p.ldc % 64 != 0) return false;
     if (shards > 1 && (cols_per_shard % b->bn != 0 || p.n_total % shards != 0)) return false;
+    if (b->halo) return (long)p.a_stages * (p.bh + 2) * p.bw * p.bn * 128 + (long)p.stages * b->bn * 128 >= (long)(b->bn / 64) * 16384;
     const long stage_bytes = b->pair ? 16384 + b->bn * 64 : 16384 + b->bn * 128;
     return (long)p.stages * stage_bytes >= (long)(b->bn / 64) * 16384;
 }
@@ -1724,7 +2010,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
             }
         }
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            const ConvGeom g = conv_geom(lv, B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
+            const ConvGeom g = conv_geom(lv, B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0);
             const size_t pix = (size_t)B * lv.H * lv.W;
             // ---- forward ----
             {
@@ -1737,11 +2023,15 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 p.tiles_per_shard = cdiv_i(lv.Cout, g.fwd.bn);
                 p.epi = UEPI_BIAS_ACT; p.relu = 1; p.out_f32 = 0; p.out = lv.act; p.ldc = lv.Cout; p.bias = mv.Wm + lv.p_b;
                 p.status = mv.status;
-                apply_plan(b, g.fwd, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
-                if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
+                apply_plan(b, g.fwd, g.halo ? 3 * p.kchunks : 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
+                if (g.halo) {
+                    if (!act_map_hn(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh + 2, g.bn)) return fail_plan();
+                } else if (!act_map(&um.fwd.mapA, lv.in_act, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.fwd.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, b->pair ? b->bn / 2 : b->bn)) return fail_plan();
                 if (tma_out_ok(b, lv.Cout, 1)) {
-                    if (!act_map(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
+                    if (g.halo) {
+                        if (!act_map_hn(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
+                    } else if (!act_map(&um.fwd.mapC, lv.act, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                     p.tma_out = 1;
                     // a 2x2 max-pool right above: pooled from the staged tile in the same kernel (SB_POOL_FUSE=0: separate kernel)
                     static const bool pool_fuse = tune("SB_POOL_FUSE", 1) != 0;
@@ -1769,11 +2059,15 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 p.epi = UEPI_MASK; p.out = lv.d_below; p.ldc = lv.Cin;
                 p.ref = lv.below_relu ? (const __nv_bfloat16*)lv.in_act : nullptr;
                 p.status = mv.status;
-                apply_plan(b, g.dgrad, 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
-                if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
+                apply_plan(b, g.dgrad, g.halo ? 3 * p.kchunks : 9 * p.kchunks, g.m_tiles, p.tiles_per_shard, mv.ws, pix);
+                if (g.halo) {
+                    if (!act_map_hn(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.bw, g.bh + 2, g.bn)) return fail_plan();
+                } else if (!act_map(&um.dgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.bw, g.bh, g.bn)) return fail_plan();
                 if (!mat_map(&um.dgrad.mapB, mv.Sm + lv.p_w, lv.Cout, 9L * lv.Cin, 64)) return fail_plan();
                 if (tma_out_ok(b, lv.Cin, 1)) {
-                    if (!act_map(&um.dgrad.mapC, lv.d_below, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
+                    if (g.halo) {
+                        if (!act_map_hn(&um.dgrad.mapC, lv.d_below, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
+                    } else if (!act_map(&um.dgrad.mapC, lv.d_below, B, lv.H, lv.W, lv.Cin, g.bw, g.bh, g.bn)) return fail_plan();
                     p.tma_out = 1;
                 }
                 um.dgrad.enabled = true;
@@ -1817,7 +2111,11 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     // activation tile (a smaller stage, a deeper ring in the same shared memory).  The pair kernel
                     // does not sum dy on the side, so the bias gradient is taken by a column-sum kernel (wgrad_pair).
                     static const bool wg_pair = tune("SB_WG_PAIR", 1) != 0;
-                    if (wg_pair && p.tap_group == 1 && (b->bn == 128 || b->bn == 256) && g.wg_m_tiles % 2 == 0 && lv.Cout % 128 == 0) {
+                    // (long reductions only: below ~160 pixel chunks the pair's two cluster barriers and the separate column-sum
+                    // kernel cost more than the halved activation fetch saves: CIFAR shape at batch 128 -1.4 % step with pairs,
+                    // batch 256 +0.4 %, ImageNet shape +1.9 %)
+                    static const int wg_pair_min_chunks = (int)tune("SB_WG_PAIR_MIN_CHUNKS", 160);
+                    if (wg_pair && (g.total_chunks >= wg_pair_min_chunks || (mv.cfg->flags & SB_FLAG_FORCE_PAIR)) && p.tap_group == 1 && (b->bn == 128 || b->bn == 256) && g.wg_m_tiles % 2 == 0 && lv.Cout % 128 == 0) {
                         b->pair = 1;
                         p.bias_fused = 0;
                         const int pfit = b->bn >= 256 ? 6 : 8, ptwo = b->bn >= 256 ? 3 : 4;

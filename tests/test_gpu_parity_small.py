@@ -296,6 +296,30 @@ def test_layerwise_teacher_forced(name, bf16):
     layerwise_teacher_forced(WORKLOADS[name](), bf16)
 
 
+@pytest.mark.parametrize("name", ["tensor_core", "pair_net", "cfg1_b4"])
+def test_per_tap_kernel_layerwise_and_against_the_halo_kernel(name):
+    """SB_FLAG_NO_HALO: the 3x3 forward / data-gradient GEMMs on the kernel that fetches one activation box per filter
+    tap.  Every layer element-wise against the oracle, and a whole forward + backward against the default (halo)
+    kernels: both sum the same products in another order, so stored bf16 values may differ by one rounding step."""
+    b = sb()
+    wl = {"tensor_core": WORKLOADS["tensor_core"], "pair_net": lambda: si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2),
+          "cfg1_b4": lambda: si.config(1).with_batch(4)}[name]()
+    layerwise_teacher_forced(wl, True, flags=b.SB_FLAG_NO_HALO)
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    xs, ys = device_batch(wl, x, y, True)
+    got = []
+    for flags in (b.SB_FLAG_NO_HALO, 0):
+        gm = gpu_model(wl, params, b.SB_BF16, flags=flags)
+        gm.forward(xs, ys)
+        convs = [li for li, (k, _) in enumerate(wl.layers) if k == si.CONV3X3_RELU]
+        got.append(([gm.read(b.SB_T_ACT, li, 0, squeeze=False) for li in convs], gm.loss()))
+        gm.close()
+    for a, c in zip(got[0][0], got[1][0]):
+        assert maxrel(a, c) <= TOL[True]
+    assert abs(got[0][1] - got[1][1]) <= TOL[True] * max(1.0, abs(got[1][1]))
+
+
 @pytest.mark.parametrize("name", list(WORKLOADS))
 @pytest.mark.parametrize("bf16", [False, True])
 def test_two_training_steps_match_oracle(name, bf16):
@@ -413,7 +437,7 @@ def test_train_step_host_matches_device_path():
     g1.close(); g2.close()
 
 
-@pytest.mark.parametrize("net", ["tensor_core", "pair", "tensor_core_fp32", "ragged_fp32"])
+@pytest.mark.parametrize("net", ["tensor_core", "pair", "pair_forced", "tensor_core_fp32", "ragged_fp32"])
 def test_graph_step_and_graph_host_step_match_separate_calls(net):
     """On a side stream the library replays the iteration as a CUDA graph (captured on the second call): weights
     and losses must be bit-identical to the three separate calls, also after the inputs move (re-capture).  The graph
@@ -430,9 +454,10 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
     params = si.make_params(wl, bias_std=0.1)
     x, y = si.make_batch(wl)
     prec = b.SB_BF16 if bf16 else b.SB_FP32
-    g1 = gpu_model(wl, params, prec)
-    g2 = gpu_model(wl, params, prec)
-    g3 = gpu_model(wl, params, prec)
+    flags = b.SB_FLAG_FORCE_PAIR if net == "pair_forced" else 0      # weight gradients on CTA pairs + the column-sum kernel
+    g1 = gpu_model(wl, params, prec, flags=flags)
+    g2 = gpu_model(wl, params, prec, flags=flags)
+    g3 = gpu_model(wl, params, prec, flags=flags)
     xs, ys = device_batch(wl, x, y, bf16)
     xs2 = [t.clone() for t in xs]                      # same values at other addresses
     hx = (torch.from_numpy(x).to(torch.bfloat16) if bf16 else torch.from_numpy(x)).pin_memory()
