@@ -55,7 +55,10 @@ typedef enum {
     SB_MAXPOOL2 = 2,     /* 2x2 max, stride 2 */
     SB_FC_RELU = 3,      /* fully connected + bias + ReLU, column-sharded K ways */
     SB_FC = 4,           /* fully connected + bias (the logits layer) */
-    SB_SOFTMAX_XENT = 5  /* log-softmax + negative log-likelihood, mean over the batch */
+    SB_SOFTMAX_XENT = 5, /* log-softmax + negative log-likelihood, mean over the batch */
+    SB_FC_RELU_WHOLE = 6, /* SB_FC_RELU kept whole on every worker: the "do not partition" outcome of the paper's
+                             computation-to-communication test for this layer [Layer Partitioning] */
+    SB_FC_WHOLE = 7       /* SB_FC (logits layer) kept whole */
 } sb_layer_kind;
 
 typedef struct {
@@ -240,6 +243,59 @@ sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void
 sb_status sb_backward_layers(sb_model* m, int32_t last, int32_t first, void* stream);
 
 /*
+ * Layer partitioning as a table [Listing 1 "Layer Partitioning"; Layer Partitioning paragraph].  Walks the sequential
+ * layer list and returns the transformed network: every input layer in order (SB_NODE_LAYER, with the number of
+ * column shards it is split into: K for SB_FC_RELU / SB_FC when K > 1, else 1), a SB_NODE_MODULO node in front of the
+ * first split layer (its input is whole: the MP group gathers the replicas' rows there), and a SB_NODE_SHARD node in
+ * front of every layer, the loss included, whose input arrives as column slices.  dim / dimF are the widths, per
+ * example, of the node's OUTPUT as one worker holds it and in full (dim = ceil(out / K) for a split layer).
+ * Convolution / pooling layers are never split and refuse a partitioned input (SB_ERR_UNSUPPORTED).
+ * Host-only: no CUDA call, usable without a GPU.  sb_model_create consumes the same table (per-layer shard counts).
+ *   layers, cfg : HOST, as for sb_model_create (H, W, C, K are read).
+ *   out         : HOST array of max_nodes entries, or NULL to query the count;  n_nodes : HOST, receives the count.
+ * Errors: as sb_model_bytes for the layer list; SB_ERR_INVALID_ARG if max_nodes is too small.  Message: sb_partition_last_error().
+ */
+typedef enum { SB_NODE_LAYER = 0, SB_NODE_MODULO = 1, SB_NODE_SHARD = 2 } sb_node_kind;
+typedef struct {
+    int32_t node;   /* sb_node_kind */
+    int32_t layer;  /* SB_NODE_LAYER: index into the input list; MODULO / SHARD: the layer it is inserted in front of */
+    int32_t shards; /* SB_NODE_LAYER: 1 = whole on every worker, K = split by output column; inserted nodes: K */
+    int32_t reserved;
+    int64_t dim;    /* output width one worker holds */
+    int64_t dimF;   /* full output width */
+} sb_plan_node;
+sb_status sb_partition(const sb_layer* layers, int32_t n, const sb_config* cfg, sb_plan_node* out, int32_t max_nodes, int32_t* n_nodes);
+const char* sb_partition_last_error(void);
+
+/*
+ * Exchange schedule of ONE MP group of G = R = K workers, worker i being data replica i and model shard i
+ * [Modulo Layer, Shard Layer; Distributed Machine Learning: reduce].  Lists every block that travels between two
+ * workers in one synchronous iteration, forward pass first, then the backward pass in execution order:
+ *   SB_X_GATHER_ROWS : modulo layer, forward.  src sends its b feature rows [row0,row1) x all D columns to dst.
+ *   SB_X_GATHER_COLS : shard layer, forward.  src sends its column slice [col0,col1) of layer `layer`'s [B,width] output.
+ *   SB_X_REDUCE_COLS : shard layer, backward.  src sends columns [col0,col1) (dst's slice) of its full-width partial
+ *                      gradient w.r.t. layer `layer`'s output; dst adds the G partial results in worker order 0..G-1.
+ *   SB_X_REDUCE_ROWS : modulo layer, backward.  src sends rows [row0,row1) (dst's examples) of its full-width partial
+ *                      gradient w.r.t. the features; dst adds the G partial results in worker order.
+ *   SB_X_ALLREDUCE   : the parameters of layer `layer` are held by every worker and trained on its own rows (conv stack):
+ *                      their gradients are summed over all workers (src = dst = -1).
+ * On one GPU every one of these is addressing inside one device buffer; this table is the contract a multi-GPU
+ * runtime has to carry out (it has been executed by CPU worker processes in the tests, not on several GPUs).
+ * Host-only.  out may be NULL to query the count.
+ */
+typedef enum { SB_X_GATHER_ROWS = 1, SB_X_GATHER_COLS = 2, SB_X_REDUCE_COLS = 3, SB_X_REDUCE_ROWS = 4, SB_X_ALLREDUCE = 5 } sb_exchange_kind;
+typedef struct {
+    int32_t kind;   /* sb_exchange_kind */
+    int32_t layer;  /* layer whose output (or parameters) the block belongs to; for the modulo layer: the first split FC layer */
+    int32_t pass;   /* 0 forward, 1 backward */
+    int32_t src, dst;
+    int32_t reserved;
+    int64_t row0, row1, col0, col1; /* block of the [B, width] matrix */
+    int64_t width;
+} sb_exchange_msg;
+sb_status sb_exchange_plan(const sb_layer* layers, int32_t n, const sb_config* cfg, sb_exchange_msg* out, int32_t max_msgs, int32_t* n_msgs);
+
+/*
  * Parameter bytes (float master copies) one worker of an MP group of size K holds: all conv
  * parameters plus shard `shard` of every FC layer [Evaluation: parameter-memory saving].
  */
@@ -273,6 +329,19 @@ sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32
  * the whole path work without a stalled pipeline.  The GPU context stays usable.  No counterpart in the paper.
  */
 sb_status sb_debug_wait_probe(sb_model* m, int32_t limit_ms, void* stream);
+
+/*
+ * Debug aids that stand in for a memory checker (no counterpart in the paper).
+ * sb_debug_poison fills every buffer a training step rewrites -- activations, activation gradients, pooling argmax bytes,
+ * split partial sums and the other scratch regions; not the parameters, momentum or gradients of parameters -- with 0xFF
+ * bytes (NaN in float and bfloat16), on `stream`.  A kernel that reads an element nothing wrote in the same step then
+ * produces NaN instead of silently re-using the previous step's value.  The next call must be sb_forward / a whole step.
+ * sb_debug_check_guards synchronises `stream` and checks the guard bytes the library keeps behind every region of the
+ * arena (256 bytes or more of a fixed pattern, written at creation): n_bad (HOST) receives the number of regions whose
+ * guard was overwritten, first_bad_offset (HOST, may be NULL) the arena offset of the first damaged byte or -1.
+ */
+sb_status sb_debug_poison(sb_model* m, void* stream);
+sb_status sb_debug_check_guards(sb_model* m, void* stream, int32_t* n_bad, int64_t* first_bad_offset);
 
 /* Number of kernels the last sb_forward + sb_backward + sb_sgd_step enqueued (host counter). */
 sb_status sb_launch_count(const sb_model* m, int64_t* launches);

@@ -19,7 +19,9 @@ LIB_PATH = os.path.join(HERE, "libsplitbrain.so")
 
 SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
-SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT = 1, 2, 3, 4, 5
+SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT, SB_FC_RELU_WHOLE, SB_FC_WHOLE = 1, 2, 3, 4, 5, 6, 7
+SB_NODE_LAYER, SB_NODE_MODULO, SB_NODE_SHARD = 0, 1, 2
+SB_X_GATHER_ROWS, SB_X_GATHER_COLS, SB_X_REDUCE_COLS, SB_X_REDUCE_ROWS, SB_X_ALLREDUCE = 1, 2, 3, 4, 5
 SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO = 1, 2, 4, 8, 16, 32
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
@@ -35,6 +37,15 @@ class sb_layer(ctypes.Structure):
 class sb_config(ctypes.Structure):
     _fields_ = [("H", c_int32), ("W", c_int32), ("C", c_int32), ("batch_per_replica", c_int32),
                 ("R", c_int32), ("K", c_int32), ("precision", c_int32), ("flags", c_int32)]
+
+
+class sb_plan_node(ctypes.Structure):
+    _fields_ = [("node", c_int32), ("layer", c_int32), ("shards", c_int32), ("reserved", c_int32), ("dim", c_int64), ("dimF", c_int64)]
+
+
+class sb_exchange_msg(ctypes.Structure):
+    _fields_ = [("kind", c_int32), ("layer", c_int32), ("pass_", c_int32), ("src", c_int32), ("dst", c_int32), ("reserved", c_int32),
+                ("row0", c_int64), ("row1", c_int64), ("col0", c_int64), ("col1", c_int64), ("width", c_int64)]
 
 
 class sb_profile_entry(ctypes.Structure):
@@ -64,6 +75,8 @@ def _load():
         "sb_graph_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
         "sb_modulo_step": [c_void_p, P(c_void_p), P(c_void_p), c_float, c_float, c_void_p],
         "sb_debug_wait_probe": [c_void_p, c_int32, c_void_p],
+        "sb_debug_poison": [c_void_p, c_void_p],
+        "sb_debug_check_guards": [c_void_p, c_void_p, P(c_int32), P(c_int64)],
         "sb_sgd_step": [c_void_p, c_float, c_float, c_void_p],
         "sb_loss": [c_void_p, c_void_p, P(c_float)],
         "sb_train_step_host": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p, P(c_float)],
@@ -76,6 +89,8 @@ def _load():
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
         "sb_launch_count": [c_void_p, P(c_int64)],
         "sb_conv_in_wgrad_static": [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p],
+        "sb_partition": [P(sb_layer), c_int32, P(sb_config), P(sb_plan_node), c_int32, P(c_int32)],
+        "sb_exchange_plan": [P(sb_layer), c_int32, P(sb_config), P(sb_exchange_msg), c_int32, P(c_int32)],
         "sb_profile_begin": [c_void_p, c_void_p],
         "sb_profile_end": [c_void_p, c_void_p, P(sb_profile_entry), c_int32, P(c_int32)],
     }
@@ -87,11 +102,13 @@ def _load():
     lib.sb_last_error.restype = c_char_p
     lib.sb_static_last_error.argtypes = []
     lib.sb_static_last_error.restype = c_char_p
+    lib.sb_partition_last_error.argtypes = []
+    lib.sb_partition_last_error.restype = c_char_p
     return lib, sigs
 
 
 _lib, _SIGS = _load()
-EXPORTED = sorted(list(_SIGS) + ["sb_last_error", "sb_static_last_error"])
+EXPORTED = sorted(list(_SIGS) + ["sb_last_error", "sb_static_last_error", "sb_partition_last_error"])
 
 # Same-named module-level entry points (raw status codes).
 sb_model_bytes = _lib.sb_model_bytes
@@ -102,6 +119,8 @@ sb_backward = _lib.sb_backward
 sb_graph_step = _lib.sb_graph_step
 sb_modulo_step = _lib.sb_modulo_step
 sb_debug_wait_probe = _lib.sb_debug_wait_probe
+sb_debug_poison = _lib.sb_debug_poison
+sb_debug_check_guards = _lib.sb_debug_check_guards
 sb_sgd_step = _lib.sb_sgd_step
 sb_loss = _lib.sb_loss
 sb_train_step_host = _lib.sb_train_step_host
@@ -116,6 +135,39 @@ sb_launch_count = _lib.sb_launch_count
 sb_conv_in_wgrad_static = _lib.sb_conv_in_wgrad_static
 sb_profile_begin = _lib.sb_profile_begin
 sb_profile_end = _lib.sb_profile_end
+sb_partition = _lib.sb_partition
+sb_exchange_plan = _lib.sb_exchange_plan
+
+
+def partition(layers, H, W, C, K):
+    """The transformed network of sb_partition as a list of dicts (host-only; no GPU needed)."""
+    arr = _layers_array(layers)
+    cfg = sb_config(H, W, C, 1, K, K, SB_FP32, 0)
+    n = c_int32()
+    st = sb_partition(arr, len(layers), byref(cfg), None, 0, byref(n))
+    if st != SB_OK:
+        raise SBError(st, _lib.sb_partition_last_error().decode())
+    out = (sb_plan_node * n.value)()
+    st = sb_partition(arr, len(layers), byref(cfg), out, n.value, byref(n))
+    if st != SB_OK:
+        raise SBError(st, _lib.sb_partition_last_error().decode())
+    return [dict(node=o.node, layer=o.layer, shards=o.shards, dim=o.dim, dimF=o.dimF) for o in out]
+
+
+def exchange_plan(layers, H, W, C, b, G):
+    """The exchange schedule of one MP group of G workers (sb_exchange_plan) as a list of dicts (host-only)."""
+    arr = _layers_array(layers)
+    cfg = sb_config(H, W, C, b, G, G, SB_FP32, 0)
+    n = c_int32()
+    st = sb_exchange_plan(arr, len(layers), byref(cfg), None, 0, byref(n))
+    if st != SB_OK:
+        raise SBError(st, _lib.sb_partition_last_error().decode())
+    out = (sb_exchange_msg * max(n.value, 1))()
+    st = sb_exchange_plan(arr, len(layers), byref(cfg), out, n.value, byref(n))
+    if st != SB_OK:
+        raise SBError(st, _lib.sb_partition_last_error().decode())
+    return [dict(kind=o.kind, layer=o.layer, backward=o.pass_, src=o.src, dst=o.dst, rows=(o.row0, o.row1), cols=(o.col0, o.col1),
+                 width=o.width) for o in out[:n.value]]
 
 
 def sb_last_error() -> str:
@@ -305,9 +357,10 @@ class Model:
             if kind == SB_CONV3X3_RELU:
                 self.write(SB_T_WEIGHT, li, 0, p["w"])
                 self.write(SB_T_BIAS, li, 0, p["b"])
-            elif kind in (SB_FC_RELU, SB_FC):
-                cb = bounds_fn(out, self.K)
-                for j in range(self.K):
+            elif kind in (SB_FC_RELU, SB_FC, SB_FC_RELU_WHOLE, SB_FC_WHOLE):
+                K = self.K if kind in (SB_FC_RELU, SB_FC) else 1       # a layer kept whole has one shard
+                cb = bounds_fn(out, K)
+                for j in range(K):
                     self.write(SB_T_WEIGHT, li, j, p["w"][cb[j]:cb[j + 1]])
                     self.write(SB_T_BIAS, li, j, p["b"][cb[j]:cb[j + 1]])
         self.refresh_shadow()
@@ -319,13 +372,23 @@ class Model:
         for li, (kind, _) in enumerate(self.layers):
             if kind == SB_CONV3X3_RELU:
                 out.append({"w": self.read(what_w, li, 0, squeeze=False), "b": self.read(what_b, li, 0)})
-            elif kind in (SB_FC_RELU, SB_FC):
-                ws = [self.read(what_w, li, j, squeeze=False)[:, :, 0, 0] for j in range(self.K)]
-                bs = [self.read(what_b, li, j, squeeze=False)[:, 0, 0, 0] for j in range(self.K)]
+            elif kind in (SB_FC_RELU, SB_FC, SB_FC_RELU_WHOLE, SB_FC_WHOLE):
+                K = self.K if kind in (SB_FC_RELU, SB_FC) else 1
+                ws = [self.read(what_w, li, j, squeeze=False)[:, :, 0, 0] for j in range(K)]
+                bs = [self.read(what_b, li, j, squeeze=False)[:, 0, 0, 0] for j in range(K)]
                 out.append({"w": np.concatenate(ws, 0), "b": np.concatenate(bs, 0)})
             else:
                 out.append(None)
         return out
+
+    def debug_poison(self):
+        _check(sb_debug_poison(self.h, self._stream()))
+
+    def debug_check_guards(self):
+        """(number of damaged guard regions, arena offset of the first damaged byte or -1)"""
+        n, off = c_int32(), c_int64()
+        _check(sb_debug_check_guards(self.h, self._stream(), byref(n), byref(off)))
+        return n.value, off.value
 
     def param_bytes(self, shard=0) -> int:
         v = c_size_t()

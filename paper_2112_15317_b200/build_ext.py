@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsplitbrain.so")
-SOURCES = ["sb_api.cu", "sb_kernels_simt.cu", "sb_umma.cu", "sb_noalloc.cu", "sb_conv_in_umma.cu"]
+SOURCES = ["sb_api.cu", "sb_kernels_simt.cu", "sb_umma.cu", "sb_noalloc.cu", "sb_conv_in_umma.cu", "sb_partition.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 # development builds: extra compiler flags, e.g. SB_NVCC_EXTRA="-DSB_DEV_TUNING -DSB_CTA_TIMING"

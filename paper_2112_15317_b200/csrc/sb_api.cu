@@ -56,6 +56,7 @@ struct Layer {
     int bg_splits = 1;                          // conv bias-gradient row splits
     bool thin_input = false;                    // conv with Cin of 1/3/4: dedicated input-layer kernels
     bool narrow = false;                        // FC with out <= 16: dedicated narrow kernels
+    int K = 1;                                  // FC: column shards of this layer (the model's K, or 1 for a layer kept whole)
     int act_dt = SB_DT_F32;
     UmmaLayer um;                               // tensor-core plan of this layer (tcgen05 path)
     // Sub-batch copies of the first FC layer (modulo schedule): where its input comes from and where its input
@@ -127,6 +128,11 @@ struct sb_model {
         bool warmed = false;
     };
     StepGraph g_dev, g_host, g_mod;
+    // Debug aids that stand in for a memory checker: every arena region is followed by a 256-byte guard holding a fixed
+    // pattern (sb_debug_check_guards), and the regions a step overwrites are listed so that they can be filled with NaN
+    // bit patterns before a step (sb_debug_poison).
+    struct Region { size_t off, bytes; bool scratch; };
+    std::vector<Region> regions;
     uint32_t host_result[2] = {0, 0};   // loss bits and device status word written by the host-step graph
     // per-launch event recording (sb_profile_begin / sb_profile_end)
     struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; int layer; };
@@ -188,6 +194,9 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
         l.kind = layers[i].kind;
         l.out = layers[i].out;
         l.act_dt = m->bf16 ? SB_DT_BF16 : SB_DT_F32;
+        // an FC layer kept whole is the same layer with one shard: from here on only the shard count tells them apart
+        const bool whole = l.kind == SB_FC_RELU_WHOLE || l.kind == SB_FC_WHOLE;
+        if (whole) l.kind = l.kind == SB_FC_RELU_WHOLE ? SB_FC_RELU : SB_FC;
         switch (l.kind) {
         case SB_CONV3X3_RELU:
             if (feat >= 0) return fail(SB_ERR_SHAPE, "layer %d: convolution after a fully-connected layer", i);
@@ -208,7 +217,7 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
         case SB_FC_RELU:
         case SB_FC:
             if (l.out < 1) return fail(SB_ERR_SHAPE, "layer %d: FC width must be positive", i);
-            if (cfg->K > l.out) return fail(SB_ERR_SHAPE, "layer %d: K=%d exceeds the FC width %d", i, cfg->K, l.out);
+            if (!whole && cfg->K > l.out) return fail(SB_ERR_SHAPE, "layer %d: K=%d exceeds the FC width %d", i, cfg->K, l.out);
             if (feat < 0) { feat = (long)H * W * C; first_fc = i; }
             l.in_f = (int)feat; l.out_f = l.out; l.relu = l.kind == SB_FC_RELU;
             l.n_w = (size_t)l.in_f * l.out_f; l.n_b = l.out_f;
@@ -232,16 +241,36 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
         }
     }
     if (m->L[n - 1].kind != SB_SOFTMAX_XENT) return fail(SB_ERR_SHAPE, "the last layer must be SB_SOFTMAX_XENT");
+    {
+        // The partitioning table [Listing 1] decides how many column shards every layer has.  On one GPU its MODULO and SHARD
+        // nodes are addressing inside one device buffer (row g of the gathered matrix is row g of the batch-major activation
+        // buffer, a column slice is a column range), so only the per-layer shard counts are consumed here.
+        std::vector<sb_plan_node> nodes((size_t)2 * n + 2);
+        int32_t nn = 0;
+        sb_status ps = sb_partition(layers, n, cfg, nodes.data(), (int32_t)nodes.size(), &nn);
+        if (ps != SB_OK) return fail(ps, "%s", sb_partition_last_error());
+        for (int32_t k = 0; k < nn; ++k)
+            if (nodes[k].node == SB_NODE_LAYER) m->L[nodes[k].layer].K = nodes[k].shards;
+    }
     m->first_fc = first_fc;
     m->P = P;
 
     // ---- arena carve-up -------------------------------------------------------------------
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return base ? base + o : (char*)nullptr; };
+    // every region starts on a 256-byte boundary and is followed by at least 256 guard bytes that no kernel may touch
+    bool scratch_region = false;
+    m->regions.clear();
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        m->regions.push_back({o, bytes, scratch_region});
+        off = align_up(off + bytes, 256) + 256;
+        return base ? base + o : (char*)nullptr;
+    };
     m->Wm = (float*)take(P * 4);
     m->Vm = (float*)take(P * 4);
     m->Gm = (float*)take(P * 4);
     m->Sm = m->bf16 ? (__nv_bfloat16*)take(P * 2) : nullptr;
+    scratch_region = true;      // from here on: activations, gradients of activations, scratch -- everything a step rewrites
     const size_t B = m->B;
     size_t ws_floats = 1024;
     for (int i = 0; i < n; ++i) {
@@ -282,6 +311,7 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) m->ws_wk[k] = (float*)take(ws_floats * 4);
     m->ws_w = m->ws_wk[0];
     m->row_loss = (float*)take(B * 4);
+    scratch_region = false;     // (loss, counter and status words keep their values between calls)
     m->loss = (float*)take(256);
     m->counter = (unsigned int*)take(256);
     m->status = (uint32_t*)take(256);
@@ -415,7 +445,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         a.M = B; a.N = l.out_f; a.K = l.in_f;
         a.epi = EPI_BIAS_ACT; a.ldc = l.out_f; a.bias = m->Wm + l.p_b; a.relu = l.relu;
         if (l.kind == SB_FC) { a.C = nullptr; a.C32 = (float*)l.act; } else { a.C = l.act; a.C32 = nullptr; }
-        a.shard_dim = 1; a.shards = m->cfg.K;
+        a.shard_dim = 1; a.shards = l.K;
         if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 1; a.tab_b = b; }
         L_TRY("fc_fwd_simt", flops, bytes, launch_gemm_simt(a, bf, st));
         break;
@@ -491,7 +521,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             a.B = layer_input(m, i); a.sBn = 1; a.sBk = l.in_f;
             a.M = l.out_f; a.N = l.in_f; a.K = B;
             a.epi = EPI_F32; a.C = m->Gm + l.p_w; a.ldc = l.in_f;
-            a.shard_dim = 3; a.shards = m->cfg.K;
+            a.shard_dim = 3; a.shards = l.K;
             if (i == 0) { a.tab = &m->x_tab; a.tab_mode = 2; a.tab_b = b; }
             L_TRY("fc_wgrad_simt", flops, act_bytes + (double)l.n_w * 4.0, launch_gemm_simt(a, bf, st));
         }
@@ -510,7 +540,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
                 a.M = B; a.N = l.in_f; a.K = l.out_f;
                 a.epi = EPI_MASK; a.C = d_below; a.ldc = l.in_f;
                 a.ref = below_relu ? layer_input(m, i) : nullptr; a.ldref = l.in_f;
-                a.shard_dim = 2; a.shards = m->cfg.K;
+                a.shard_dim = 2; a.shards = l.K;
                 L_TRY("fc_dgrad_simt", flops, bytes, launch_gemm_simt(a, bf, st));
             }
         }
@@ -531,14 +561,17 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
         // the gradient arena -- or, when the backward pass folds the update in, reduced and applied in one kernel (S = 1:
         // the gradient is already in the arena and takes a plain update).
         const bool fuse = m->fuse.on && (part & SIDE_W) && !(part & SIDE_D) && l.n_w % 4 == 0 && l.n_b % 4 == 0 && l.p_w % 4 == 0 && l.p_b % 4 == 0;
-        auto finish = [&](const float* src, size_t stride, size_t goff, size_t n, int S) -> sb_status {
+        // (in_place: with S = 1 the kernel wrote the gradient into the arena itself; the input-layer kernels always write
+        // partial buffers, so a single one still has to be carried over)
+        auto finish = [&](const float* src, size_t stride, size_t goff, size_t n, int S, bool in_place = true) -> sb_status {
+            const bool reduce = S > 1 || !in_place;
             if (!fuse) {
-                if (S > 1) L_TRY("split_reduce", 0.0, (double)n * 4.0 * (S + 1), launch_reduce_partials(src, stride, m->Gm + goff, n, S, st));
+                if (reduce) L_TRY("split_reduce", 0.0, (double)n * 4.0 * (S + 1), launch_reduce_partials(src, stride, m->Gm + goff, n, S, st));
                 return SB_OK;
             }
             if (!m->fuse.waited) { CU_TRY(cudaStreamWaitEvent(st, m->fuse.ev, 0)); m->fuse.waited = true; }
             __nv_bfloat16* sh = m->Sm ? m->Sm + goff : nullptr;
-            if (S > 1)
+            if (reduce)
                 L_TRY("split_reduce_sgd", 0.0, (double)n * (4.0 * S + (m->bf16 ? 18.0 : 16.0)),
                       launch_reduce_sgd(src, stride, n, S, m->Wm + goff, m->Vm + goff, sh, m->fuse.lr, m->fuse.mu, st));
             else
@@ -562,10 +595,10 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
                 L_TRY("conv_in_wgrad", flops, pix * (l.Cin + l.Cout) * e + (double)l.n_w * 4.0, launch_conv_in_wgrad(a, bf, st));
             if (l.p_b == l.p_w + l.n_w) {
                 // the bias vector directly follows the weights in the gradient arena, as it does in a partial buffer
-                if ((fs = finish(ws_w, stride, l.p_w, stride, nb)) != SB_OK) return fs;
+                if ((fs = finish(ws_w, stride, l.p_w, stride, nb, false)) != SB_OK) return fs;
             } else {
-                if ((fs = finish(ws_w, stride, l.p_w, l.n_w, nb)) != SB_OK) return fs;
-                if ((fs = finish(ws_w + l.n_w, stride, l.p_b, l.n_b, nb)) != SB_OK) return fs;
+                if ((fs = finish(ws_w, stride, l.p_w, l.n_w, nb, false)) != SB_OK) return fs;
+                if ((fs = finish(ws_w + l.n_w, stride, l.p_b, l.n_b, nb, false)) != SB_OK) return fs;
             }
         } else if (l.um.wgrad.enabled) {
             int S = 1;
@@ -648,7 +681,7 @@ sb_status resolve(sb_model* m, int what, int li, int part, char** ptr, int64_t s
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (li < 0 || li >= m->n_layers) return fail(SB_ERR_INVALID_ARG, "layer %d out of range", li);
     Layer& l = m->L[li];
-    const int b = m->cfg.batch_per_replica, R = m->cfg.R, K = m->cfg.K;
+    const int b = m->cfg.batch_per_replica, R = m->cfg.R, K = l.K;      // (K: this layer's own shard count)
     int64_t sh[4] = {1, 1, 1, 1};
     char* p = nullptr;
     int dt = SB_DT_F32;
@@ -741,6 +774,7 @@ LayerView layer_view(sb_model* m, int i)
 {
     Layer& l = m->L[i];
     LayerView v{};
+    v.K = l.K;
     v.kind = l.kind; v.H = l.H; v.W = l.W; v.Cin = l.Cin; v.Cout = l.Cout; v.in_f = l.in_f; v.out_f = l.out_f; v.relu = l.relu;
     v.p_w = l.p_w; v.p_b = l.p_b; v.n_w = l.n_w; v.n_b = l.n_b;
     v.act = l.act; v.dact = l.dact; v.um = &l.um; v.pool_idx = l.idx;
@@ -800,6 +834,11 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
         if (!ok_) { delete m; return fail(SB_ERR_CUDA, "creating the backward-pass stream / events failed"); }
     }
     cudaError_t e = cudaMemset(arena, 0, need);
+    // the guard bytes behind every region (checked by sb_debug_check_guards)
+    for (size_t k = 0; e == cudaSuccess && k < m->regions.size(); ++k) {
+        const size_t g0 = m->regions[k].off + m->regions[k].bytes, g1 = align_up(g0, 256) + 256;
+        e = cudaMemset((char*)arena + g0, 0xA5, g1 - g0);
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete m; return fail(SB_ERR_CUDA, "clearing the arena: %s", cudaGetErrorString(e)); }
     s = umma_plan_layers(m, 0);
@@ -1249,7 +1288,8 @@ sb_status sb_param_bytes(const sb_model* m, int32_t shard, size_t* bytes)
     for (const Layer& l : m->L) {
         if (l.kind == SB_CONV3X3_RELU) n += l.n_w + l.n_b;
         else if (l.kind == SB_FC_RELU || l.kind == SB_FC) {
-            size_t rows = shard_lo(shard + 1, l.out_f, m->cfg.K) - shard_lo(shard, l.out_f, m->cfg.K);
+            // a layer kept whole is held in full by every worker
+            size_t rows = l.K == 1 ? (size_t)l.out_f : (size_t)(shard_lo(shard + 1, l.out_f, l.K) - shard_lo(shard, l.out_f, l.K));
             n += rows * l.in_f + rows;
         }
     }
@@ -1313,6 +1353,37 @@ sb_status sb_debug_wait_probe(sb_model* m, int32_t limit_ms, void* stream)
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (limit_ms < 1 || limit_ms > 1000) return fail(SB_ERR_INVALID_ARG, "limit_ms must be in 1..1000");
     CU_TRY(launch_wait_probe(m->status, (unsigned long long)limit_ms * 1000000ull, (cudaStream_t)stream));
+    return SB_OK;
+}
+
+sb_status sb_debug_poison(sb_model* m, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    // 0xFF bytes are NaN in float and in bfloat16, and an impossible argmax byte
+    for (const sb_model::Region& r : m->regions)
+        if (r.scratch && r.bytes) CU_TRY(cudaMemsetAsync(m->arena + r.off, 0xFF, r.bytes, (cudaStream_t)stream));
+    m->have_fwd = false;
+    return SB_OK;
+}
+
+sb_status sb_debug_check_guards(sb_model* m, void* stream, int32_t* n_bad, int64_t* first_bad_offset)
+{
+    if (!m || !n_bad) return fail(SB_ERR_INVALID_ARG, "null argument");
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    *n_bad = 0;
+    if (first_bad_offset) *first_bad_offset = -1;
+    std::vector<unsigned char> h;
+    for (const sb_model::Region& r : m->regions) {
+        const size_t g0 = r.off + r.bytes, g1 = align_up(r.off + r.bytes, 256) + 256;
+        h.resize(g1 - g0);
+        CU_TRY(cudaMemcpy(h.data(), m->arena + g0, g1 - g0, cudaMemcpyDeviceToHost));
+        for (size_t k = 0; k < h.size(); ++k)
+            if (h[k] != 0xA5) {
+                if (*n_bad == 0 && first_bad_offset) *first_bad_offset = (int64_t)(g0 + k);
+                ++*n_bad;
+                break;
+            }
+    }
     return SB_OK;
 }
 

@@ -1945,7 +1945,7 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * pix * lv.Cout);
             if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * pix * lv.Cin);
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
-            FcGeom g = fc_geom(lv, mv.B, mv.cfg->K, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
+            FcGeom g = fc_geom(lv, mv.B, lv.K, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * mv.B * lv.out_f);
             if (g.dgrad.splits > 1) upd((size_t)g.dgrad.splits * mv.B * lv.in_f);
         }
@@ -2134,7 +2134,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 um.wgrad.enabled = true;
             }
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
-            const int K = mv.cfg->K;
+            const int K = lv.K;
             const FcGeom g = fc_geom(lv, B, K, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0);
             const int m_tiles = g.m_tiles;
             if (i == 0) lv.in_act = mv.stage_x;   // placeholder; rebound to the caller's input by umma_bind_input

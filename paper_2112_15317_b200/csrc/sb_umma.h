@@ -42,6 +42,7 @@ struct ModelView {
 };
 struct LayerView {
     int kind, H, W, Cin, Cout, in_f, out_f;
+    int K;                // FC: this layer's column shards
     bool relu;
     size_t p_w, p_b, n_w, n_b;
     char *act, *dact;

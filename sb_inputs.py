@@ -27,6 +27,8 @@ MAXPOOL2 = 2
 FC_RELU = 3
 FC = 4
 SOFTMAX_XENT = 5
+FC_RELU_WHOLE = 6   # FC + ReLU that the partitioning keeps whole on every worker
+FC_WHOLE = 7
 
 SEED_WEIGHTS = 2112
 SEED_DATA = 15317
@@ -86,9 +88,10 @@ def layer_shapes(wl: Workload):
             out.append(dict(kind=kind, H=H, W=W, C=C))
             H //= 2
             W //= 2
-        elif kind in (FC_RELU, FC):
+        elif kind in (FC_RELU, FC, FC_RELU_WHOLE, FC_WHOLE):
             if feat is None:
                 feat = H * W * C
+            kind = FC_RELU if kind in (FC_RELU, FC_RELU_WHOLE) else FC      # (shapes and initial values do not depend on the split)
             out.append({"kind": kind, "in": feat, "out": o, "relu": kind == FC_RELU})
             feat = o
         elif kind == SOFTMAX_XENT:

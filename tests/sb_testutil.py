@@ -46,9 +46,16 @@ class Checks:
         assert not bad, "parity bounds exceeded: " + "; ".join(f"{n}: {v:.3e} > {b:.1e}" for n, v, b in bad[:12])
 
 
+def all_split(wl):
+    """The same workload with every FC layer split K ways (an FC layer kept whole computes the same function: the oracle,
+    which splits every FC layer, serves as the reference for both)."""
+    kinds = {si.FC_RELU_WHOLE: si.FC_RELU, si.FC_WHOLE: si.FC}
+    return si.Workload(wl.name, [(kinds.get(k, k), o) for k, o in wl.layers], wl.H, wl.W, wl.C, wl.b, wl.R, wl.K)
+
+
 def oracle_model(wl, params, bf16, real="float"):
     from oracle import splitbrain_oracle as so
-    m = so.from_workload(wl, real=real, bf16=bf16)
+    m = so.from_workload(all_split(wl), real=real, bf16=bf16)
     m.load_params(params)
     return m
 

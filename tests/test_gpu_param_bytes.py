@@ -52,3 +52,18 @@ def test_param_bytes_per_worker_match_table1(K):
             assert round(100.0 * (1.0 - got / (4.0 * (conv + fc))), 1) == 65.8
     if K == 1:
         assert per_shard[0] == 4 * 6990666
+
+
+def test_layers_kept_whole_are_counted_in_full_for_every_worker():
+    """An FC layer that the partitioning keeps whole (SB_FC_RELU_WHOLE) is held in full by every worker."""
+    from paper_2112_15317_b200 import binding as sb
+    K = 4
+    layers = [(si.CONV3X3_RELU, 16), (si.MAXPOOL2, 0), (si.FC_RELU_WHOLE, 48), (si.FC_RELU, 64), (si.FC, 12), (si.SOFTMAX_XENT, 12)]
+    wl = si.Workload("whole", layers, 8, 8, 3, 2, 1, K)
+    m = sb.Model.from_workload(wl, precision=sb.SB_FP32)
+    conv = 16 * 27 + 16
+    fc_whole = 48 * (4 * 4 * 16) + 48
+    for j in range(K):
+        want = conv + fc_whole + (64 // K) * (48 + 1) + (12 // K) * (64 + 1)
+        assert m.param_bytes(j) == 4 * want
+    m.close()

@@ -10,6 +10,7 @@ from sb_testutil import Checks, device_batch, gpu_model, maxrel, oracle_model
 pytestmark = pytest.mark.gpu
 
 TOL = {False: 1e-4, True: 1e-2}
+FC_KINDS = (si.FC_RELU, si.FC, si.FC_RELU_WHOLE, si.FC_WHOLE)
 
 
 def sb():
@@ -194,7 +195,7 @@ def layerwise_teacher_forced(wl, bf16, bias_std=0.2, distinct=None, flags=0, ref
                 assert maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), conv_out(r, li)) <= tol, ("act", li, r)
                 if kind == si.MAXPOOL2:
                     assert np.array_equal(gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False), pool_idx(r, li)), ("idx", li, r)
-        elif kind in (si.FC_RELU, si.FC):
+        elif kind in FC_KINDS:
             assert maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], full(om.fc_out[li])) <= tol, ("fc act", li)
         else:
             assert maxrel(gm.read(b.SB_T_ROW_LOSS, li, 0), full(om.row_loss)) <= tol
@@ -253,7 +254,7 @@ def end_to_end_vs_ref(ref, steps=1, lr=0.01, mu=0.9, checks=None, flags=0):
                     ck.le(("act", step, li, r), maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), ref.conv_out(r, li)), tol)
                     if kind == si.MAXPOOL2 and not bf16:
                         ck.le(("pool idx", step, li, r), float(np.mean(gm.read(b.SB_T_POOL_IDX, li, r, squeeze=False) != ref.pool_idx(r, li))), 0.0)
-            elif kind in (si.FC_RELU, si.FC):
+            elif kind in FC_KINDS:
                 ck.le(("fc act", step, li), maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], ref.full(om.fc_out[li])), tol)
         ck.le(("row loss", step), maxrel(gm.read(b.SB_T_ROW_LOSS, nl - 1, 0), ref.full(om.row_loss)), tol)
         if bf16:
@@ -263,7 +264,7 @@ def end_to_end_vs_ref(ref, steps=1, lr=0.01, mu=0.9, checks=None, flags=0):
             if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
                 for r in range(wl.R):
                     ck.le(("dact", step, li, r), maxrel(gm.read(b.SB_T_DACT, li, r, squeeze=False), ref.d_conv(r, li)), TOL_DACT_CHAIN[bf16])
-            elif kind in (si.FC_RELU, si.FC):
+            elif kind in FC_KINDS:
                 ck.le(("fc dact", step, li), maxrel(gm.read(b.SB_T_DACT, li, 0, squeeze=False)[:, :, 0, 0], ref.full(om.d_pre[li])), TOL_DACT_CHAIN[bf16])
         # with repeated rows the gradient is gscale times the oracle's (equal rows contribute equally): scale the oracle's
         # gradients in place, so that its own SGD step then yields the momentum and weights to compare with
@@ -348,7 +349,7 @@ def test_bf16_path_against_the_oracle_in_plain_float(name):
         if kind in (si.CONV3X3_RELU, si.MAXPOOL2):
             for r in range(wl.R):
                 ck.le(("act", li, r), maxrel(gm.read(b.SB_T_ACT, li, r, squeeze=False), om.conv_out[r][li]), 1e-2)
-        elif kind in (si.FC_RELU, si.FC):
+        elif kind in FC_KINDS:
             ck.le(("fc act", li), maxrel(gm.read(b.SB_T_ACT, li, 0, squeeze=False)[:, :, 0, 0], om.fc_out[li]), 1e-2)
     ck.le(("row loss",), maxrel(gm.read(b.SB_T_ROW_LOSS, len(wl.layers) - 1, 0), om.row_loss), 1e-2)
     gm.close()
@@ -379,6 +380,29 @@ def test_cta_pair_kernels_forced(images):
         assert abs(loss - om.loss) <= TOL[True] * max(1.0, abs(om.loss))
     # the two plans may split reductions differently, so their bf16 roundings differ: same bound as against the oracle
     assert maxrel(got[0][0], got[1][0]) <= TOL[True]
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_fc_layers_kept_whole_compute_the_same_network(bf16):
+    """SB_FC_RELU_WHOLE / SB_FC_WHOLE (the partitioning table's "do not split" outcome): every layer element-wise
+    against the oracle, whole iterations end to end, and the forward pass bit-identical to the all-split model."""
+    b = sb()
+    mixed = [(si.CONV3X3_RELU, 64), (si.MAXPOOL2, 0), (si.FC_RELU_WHOLE, 128), (si.FC_RELU, 256), (si.FC_RELU_WHOLE, 64), (si.FC_WHOLE, 16),
+             (si.SOFTMAX_XENT, 16)]
+    wl = si.Workload("whole_fc", mixed, 8, 8, 3, 3, 2, 4)
+    layerwise_teacher_forced(wl, bf16)
+    compare_everything(wl, bf16, steps=2, bias_std=0.1)
+    from sb_testutil import all_split
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    xs, ys = device_batch(wl, x, y, bf16)
+    logits = []
+    for w in (wl, all_split(wl)):
+        gm = gpu_model(w, params, b.SB_BF16 if bf16 else b.SB_FP32)
+        gm.forward(xs, ys)
+        logits.append(gm.read(b.SB_T_ACT, len(w.layers) - 2, 0, squeeze=False)[:, :, 0, 0])
+        gm.close()
+    assert np.array_equal(logits[0], logits[1])
 
 
 @pytest.mark.parametrize("bf16", [False, True])
@@ -518,6 +542,61 @@ def test_maximum_partition_counts(bf16):
     b = sb()
     with pytest.raises(b.SBError, match="SB_ERR_SHAPE"):
         gpu_model(si.Workload("too_many", net, 8, 8, 3, 1, 65, 64), si.make_params(wl), b.SB_FP32)
+
+
+@pytest.mark.parametrize("name", ["tensor_core", "ragged", "pair_forced", "cfg1_b4", "ragged_fp32"])
+def test_poisoned_buffers_and_guard_bytes(name):
+    """Stand-ins for a memory checker.  (1) Every buffer a step rewrites is filled with NaN bit patterns before each
+    step: a kernel that read an element nothing wrote in that step (a ragged tile tail, an unwritten split partial sum,
+    a stale argmax byte) would carry the NaN into the loss or the parameters; results must stay bit-identical to the
+    unpoisoned run.  (2) The guard bytes behind every arena region must be untouched after whole training steps."""
+    import torch
+    b = sb()
+    bf16 = not name.endswith("_fp32")
+    flags = b.SB_FLAG_FORCE_PAIR if name == "pair_forced" else 0
+    wl = {"tensor_core": WORKLOADS["tensor_core"], "ragged": WORKLOADS["ragged"], "ragged_fp32": WORKLOADS["ragged"],
+          "pair_forced": lambda: si.Workload("pair", pair_net(), 12, 20, 3, 3, 2, 2), "cfg1_b4": lambda: si.config(1).with_batch(4)}[name]()
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    xs, ys = device_batch(wl, x, y, bf16)
+    prec = b.SB_BF16 if bf16 else b.SB_FP32
+    clean, dirty = gpu_model(wl, params, prec, flags=flags), gpu_model(wl, params, prec, flags=flags)
+    for step in range(2):
+        clean.forward(xs, ys); clean.backward(); clean.sgd_step(0.01, 0.9)
+        dirty.debug_poison()
+        dirty.forward(xs, ys); dirty.backward(); dirty.sgd_step(0.01, 0.9)
+        assert clean.loss() == dirty.loss() and np.isfinite(dirty.loss()), step
+    # the fused step (CUDA graph on a side stream) on poisoned buffers as well
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for step in range(3):
+            clean.graph_step(xs, ys, 0.01, 0.9)
+            dirty.debug_poison()
+            dirty.graph_step(xs, ys, 0.01, 0.9)
+            assert clean.loss() == dirty.loss(), step
+        side.synchronize()
+    for a, c in zip(clean.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), dirty.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    assert clean.debug_check_guards() == (0, -1) and dirty.debug_check_guards() == (0, -1)
+    clean.close(); dirty.close()
+
+
+def test_guard_check_reports_a_damaged_guard():
+    """The checker itself: one byte set just past a tensor (from the host, inside the arena's guard area) is found."""
+    cudart = pytest.importorskip("cuda.cudart")
+    b = sb()
+    wl = WORKLOADS["cfg0"]()
+    gm = gpu_model(wl, si.make_params(wl), b.SB_FP32)
+    assert gm.debug_check_guards() == (0, -1)
+    ptr, shape, _ = gm.tensor_info(b.SB_T_ROW_LOSS, len(wl.layers) - 1, 0)
+    end = ptr + 4 * int(np.prod(shape))
+    (err,) = cudart.cudaMemset(end + 3, 0, 1)
+    assert int(err) == 0
+    n_bad, off = gm.debug_check_guards()
+    arena_base = (gm.arena.data_ptr() + 255) // 256 * 256
+    assert n_bad == 1 and off == end + 3 - arena_base
+    gm.close()
 
 
 def test_state_and_argument_errors():
