@@ -79,9 +79,12 @@ enum {
                                 of CTAs; weight gradients with long reductions) */
     SB_FLAG_MODULO_SCHEDULE = 16, /* reserve the buffers and plan the sub-batch kernels sb_modulo_step needs
                                 (batch_per_replica must be a multiple of K; the first layer must not be an FC layer) */
-    SB_FLAG_NO_HALO = 32     /* 3x3 forward / data-gradient GEMMs on the kernel that fetches an activation box per filter tap
+    SB_FLAG_NO_HALO = 32,    /* 3x3 forward / data-gradient GEMMs on the kernel that fetches an activation box per filter tap
                                 instead of the default one that shares a fetch of bh + 2 image rows between the three taps of
                                 a filter column (for tests: both kernels must give the same results) */
+    SB_FLAG_FORCE_PERSIST = 64 /* 3x3 forward / data-gradient GEMMs of layers up to 128 channels wide on the persistent kernel
+                                (a few CTAs walk all output tiles, two accumulators in turn), whatever the layer's size; by
+                                default only layers with several tiles per SM use it (for tests at small sizes) */
 };
 
 typedef struct {

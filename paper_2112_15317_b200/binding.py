@@ -22,7 +22,7 @@ SB_FP32, SB_BF16 = 0, 1
 SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT, SB_FC_RELU_WHOLE, SB_FC_WHOLE = 1, 2, 3, 4, 5, 6, 7
 SB_NODE_LAYER, SB_NODE_MODULO, SB_NODE_SHARD = 0, 1, 2
 SB_X_GATHER_ROWS, SB_X_GATHER_COLS, SB_X_REDUCE_COLS, SB_X_REDUCE_ROWS, SB_X_ALLREDUCE = 1, 2, 3, 4, 5
-SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO = 1, 2, 4, 8, 16, 32
+SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO, SB_FLAG_FORCE_PERSIST = 1, 2, 4, 8, 16, 32, 64
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
 SB_DT_F32, SB_DT_BF16, SB_DT_U8, SB_DT_I32 = 0, 1, 2, 3

@@ -85,6 +85,7 @@ struct UmmaParams {
     int hn_order;         // 1: tile rows in (h, n, w) order; 0: (n, h, w)
     int a_stages;         // depth of the activation (halo) ring; `stages` is then the depth of the weight ring
     uint32_t rcp_bwbn;    // reciprocal of bw * bn (hn_order)
+    uint32_t rcp_mtiles;  // reciprocal of tiles_w * tiles_h * tiles_n (persistent halo kernel: tile index -> N tile)
 #ifdef SB_CTA_TIMING
     unsigned long long* timing;   // development builds only: per-CTA phase timestamps, 16 per CTA, first 1024 CTAs
     int dbg_skip;                 // development builds only (halo kernel, timing experiments, WRONG results): bit 0 = no activation
@@ -990,6 +991,288 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 }
 
 // ------------------------------------------------------------------------------------------------
+// The persistent halo kernel: one CTA walks many output tiles
+// ------------------------------------------------------------------------------------------------
+// A layer of many tiles (several per SM) spends, one tile per CTA, more time in per-CTA fixed work -- barrier and TMEM
+// set-up (~1.3 us), the first operand round trip (~0.4 us), the accumulator drain and the epilogue (~1.5 us) -- than in
+// a short main loop (1 - 3 us at 64 - 128 input channels).  Here a CTA is launched once per SM slot and walks the tiles
+// t = blockIdx.x, blockIdx.x + gridDim.x, ... with
+//   * the operand rings running on across tile boundaries (the producer warp starts the next tile's first groups while
+//     the last ones of the current tile are still being multiplied), and
+//   * two TMEM accumulators: the MMA warp fills accumulator (i & 1) for the i-th tile while the four epilogue warps
+//     drain the other one (tcgen05.ld, bias + ReLU / mask, staging, TMA store, fused 2x2 pool), handing it back through
+//     acc_empty[].
+// The output tile is staged in its own shared-memory buffer (the rings are never idle here).  Unsplit reductions with
+// the TMA-store epilogue only (the planner checks); everything else as in umma_halo_kernel, every wait bounded.
+template <int BN> struct HaloPersistCfg {
+    static constexpr int B_STAGE_BYTES = BN * 128;
+    static constexpr int STAGE_OUT_BYTES = (BN / 64) * 16384;
+    static constexpr int TMEM_COLS = 2 * BN;                 // 128, 256 or 512: powers of two
+    static constexpr int smem_bytes(int a_stages, int a_slot_bytes, int b_stages)
+    {
+        return a_stages * a_slot_bytes + b_stages * B_STAGE_BYTES + STAGE_OUT_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES;
+    }
+};
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 128 epilogue threads
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+                         const UmmaParams p)
+{
+    static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "halo kernel: forward and data gradient only");
+    using C = HaloPersistCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int SA = p.a_stages, SB = p.stages;
+    const uint32_t row_step = (uint32_t)(p.bw * p.bn) * 128u;
+    const uint32_t a_slot = (uint32_t)(p.bh + 2) * row_step;
+    uint8_t* b_ring = smem + (size_t)SA * a_slot;
+    uint8_t* stage_out = b_ring + (size_t)SB * C::B_STAGE_BYTES;
+    uint8_t* ctrl = stage_out + C::STAGE_OUT_BYTES;
+    uint64_t* b_full = (uint64_t*)ctrl;               // [MAX_STAGES]
+    uint64_t* b_empty = b_full + MAX_STAGES;          // [MAX_STAGES]
+    uint64_t* a_full = b_empty + MAX_STAGES;          // [MAX_A_STAGES]
+    uint64_t* a_empty = a_full + MAX_A_STAGES;        // [MAX_A_STAGES]
+    uint64_t* acc_full = a_empty + MAX_A_STAGES;      // [2]
+    uint64_t* acc_empty = acc_full + 2;               // [2]
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* s_bias = (float*)(ctrl + 512);             // [BN]
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+#ifdef SB_CTA_TIMING
+    unsigned long long* tlog = (p.timing != nullptr && blockIdx.x < 1024) ? p.timing + 16ull * blockIdx.x : nullptr;
+#endif
+    SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TLOG(threadIdx.x == 0, 6, clock64());
+    const int m_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
+    const int n_tiles_total = m_tiles * p.tiles_per_shard;       // (tiles_per_shard = N tiles; conv layers have one shard)
+    const int n_groups = p.total_chunks;                         // 3 * kchunks groups per tile
+    const uint32_t smem0 = smem_u32(smem), bring0 = smem_u32(b_ring);
+
+    // tile index -> pixel-box origin and first output column
+    auto tile_coords = [&](int t, int& pw0, int& ph0, int& pn0, int& n0) {
+        const int n_idx = fast_div_exact(t, p.rcp_mtiles, m_tiles);
+        const int m_idx = t - n_idx * m_tiles;
+        const int q1 = fast_div_exact(m_idx, p.rcp_tiles_w, p.tiles_w), q2 = fast_div_exact(m_idx, p.rcp_tiles_wh, p.tiles_w * p.tiles_h);
+        pw0 = (m_idx - q1 * p.tiles_w) * p.bw;
+        ph0 = (q1 - q2 * p.tiles_h) * p.bh;
+        pn0 = q2 * p.bn;
+        n0 = n_idx * BN;
+    };
+
+    // ---- one-time setup -----------------------------------------------------------------------
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < SB; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
+            for (int s = 0; s < SA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
+            for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 1); }
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    pdl_wait();          // every thread that touches global memory waits for the predecessor kernel
+    if (warp == 0) pdl_trigger();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
+
+    if (warp == 0) {
+        // =========================== TMA producer ===============================================
+        // (whole warp in lock-step, elected issue, one group per round: see umma_halo_kernel; the rings never reset)
+        const uint32_t prod_el = elect_one() ? 1u : 0u;
+        const uint32_t afull0 = smem_u32(&a_full[0]), bfull0 = smem_u32(&b_full[0]);
+        int la_s = 0, lb_s = 0;
+        uint32_t la_off = 0, lb_off = 0, pa_par = 1u, pb_par = 1u;
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
+            int pw0, ph0, pn0, n0;
+            tile_coords(t, pw0, ph0, pn0, n0);
+            int kc = 0, dsi = 0;
+            for (int g = 0; g < n_groups; ++g) {
+                const int s1 = lb_s, s2 = s1 + 1 == SB ? 0 : s1 + 1, s3 = s2 + 1 == SB ? 0 : s2 + 1;
+                const uint32_t p1 = pb_par, p2 = s2 == 0 ? p1 ^ 1u : p1, p3 = s3 == 0 ? p2 ^ 1u : p2;
+                const bool w0 = mbar_try_wait(&a_empty[la_s], pa_par), w1 = mbar_try_wait(&b_empty[s1], p1),
+                           w2 = mbar_try_wait(&b_empty[s2], p2), w3 = mbar_try_wait(&b_empty[s3], p3);
+                if (!__all_sync(0xffffffffu, (w0 && w1 && w2 && w3) ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, (mbar_wait(&a_empty[la_s], pa_par) && mbar_wait(&b_empty[s1], p1) &&
+                                                  mbar_wait(&b_empty[s2], p2) && mbar_wait(&b_empty[s3], p3)) ? 1 : 0) != 0;
+                    if (!ok) break;
+                }
+                {
+                    const uint32_t bar = afull0 + 8u * (uint32_t)la_s;
+                    mbar_expect_tx_el(bar, a_slot, prod_el);
+                    tma_load_4d_el(&mapA, smem0 + la_off, bar, kc * 64, pw0 + dsi - 1, pn0, ph0 - 1, prod_el);    // (c, w, n, h)
+                    ++la_s; la_off += a_slot;
+                    if (la_s == SA) { la_s = 0; la_off = 0; pa_par ^= 1u; }
+                }
+#pragma unroll
+                for (int j = 0; j < 3; ++j) {
+                    const int tap = MODE == MODE_FWD ? 3 * j + dsi : 3 * (2 - j) + (2 - dsi);
+                    const uint32_t dst = bring0 + lb_off, bar = bfull0 + 8u * (uint32_t)lb_s;
+                    mbar_expect_tx_el(bar, (uint32_t)C::B_STAGE_BYTES, prod_el);
+                    if (MODE == MODE_FWD) {
+                        tma_load_4d_el(&mapB, dst, bar, tap * p.w_cols + kc * 64, n0, 0, 0, prod_el);
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < BN / 64; ++jj)
+                            tma_load_4d_el(&mapB, dst + jj * 8192, bar, tap * p.w_cols + n0 + 64 * jj, kc * 64, 0, 0, prod_el);
+                    }
+                    ++lb_s; lb_off += (uint32_t)C::B_STAGE_BYTES;
+                    if (lb_s == SB) { lb_s = 0; lb_off = 0; pb_par ^= 1u; }
+                }
+                if (++dsi == 3) { dsi = 0; ++kc; }
+            }
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        __syncwarp();
+    } else if (warp == 1) {
+        // =========================== MMA issuer =================================================
+        constexpr uint32_t idesc = make_idesc(BN, 0, MODE != MODE_FWD);
+        const uint32_t elected = elect_one() ? 1u : 0u;
+        const uint64_t dA0 = make_desc(smem0, 16);
+        const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(bring0, 16) : make_desc(bring0, 8192);
+        const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
+        const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
+        constexpr uint32_t A_STEP = 32u >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
+        constexpr uint32_t BSTAGE16 = (uint32_t)C::B_STAGE_BYTES >> 4;
+        const uint32_t aslot16 = a_slot >> 4, rowstep16 = row_step >> 4;
+        int sa = 0, sb_ = 0;
+        uint32_t pha = 0, phb = 0, aoff = 0, boff = 0;
+        bool ok = true;
+        int i = 0;                                  // tiles this CTA has started
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++i) {
+            const int buf = i & 1;
+            // the epilogue must have drained this accumulator's previous tile (use u of a buffer waits for release u - 1;
+            // a fresh barrier reports the phase before its first as complete)
+            ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[buf], (uint32_t)(((i >> 1) + 1) & 1)) ? 1 : 0) != 0;
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+            for (int g = 0; g < n_groups; ++g) {
+                const int s1 = sb_, s2 = s1 + 1 == SB ? 0 : s1 + 1, s3 = s2 + 1 == SB ? 0 : s2 + 1;
+                const uint32_t p1 = phb, p2 = s2 == 0 ? p1 ^ 1u : p1, p3 = s3 == 0 ? p2 ^ 1u : p2;
+                const uint32_t o1 = boff, o2 = s2 == 0 ? 0u : o1 + BSTAGE16, o3 = s3 == 0 ? 0u : o2 + BSTAGE16;
+                const bool w0 = mbar_try_wait(&a_full[sa], pha), w1 = mbar_try_wait(&b_full[s1], p1), w2 = mbar_try_wait(&b_full[s2], p2),
+                           w3 = mbar_try_wait(&b_full[s3], p3);
+                if (!__all_sync(0xffffffffu, (w0 && w1) ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, (mbar_wait(&a_full[sa], pha) && mbar_wait(&b_full[s1], p1)) ? 1 : 0) != 0;
+                    if (!ok) break;
+                }
+                tc_fence_after();
+                const uint32_t alo = a_lo0 + aoff;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_lohi(d_tmem, alo + kk * A_STEP, a_hi, b_lo0 + o1 + kk * B_STEP, b_hi, idesc, (g > 0 || kk > 0) ? 1u : 0u, elected);
+                if (elected) umma_commit(&b_empty[s1]);
+                if (!__all_sync(0xffffffffu, w2 ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&b_full[s2], p2) ? 1 : 0) != 0;
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_lohi(d_tmem, alo + rowstep16 + kk * A_STEP, a_hi, b_lo0 + o2 + kk * B_STEP, b_hi, idesc, 1u, elected);
+                if (elected) umma_commit(&b_empty[s2]);
+                if (!__all_sync(0xffffffffu, w3 ? 1 : 0)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&b_full[s3], p3) ? 1 : 0) != 0;
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_lohi(d_tmem, alo + 2 * rowstep16 + kk * A_STEP, a_hi, b_lo0 + o3 + kk * B_STEP, b_hi, idesc, 1u, elected);
+                if (elected) {
+                    umma_commit(&b_empty[s3]);
+                    umma_commit(&a_empty[sa]);
+                }
+                __syncwarp();
+                sb_ = s3 + 1; boff = o3 + BSTAGE16; phb = p3;
+                if (sb_ == SB) { sb_ = 0; boff = 0; phb ^= 1u; }
+                ++sa; aoff += aslot16;
+                if (sa == SA) { sa = 0; aoff = 0; pha ^= 1u; }
+            }
+            if (!ok) break;
+            if (elected) umma_commit(&acc_full[buf]);   // this tile's accumulator is complete once the MMAs above have run
+            __syncwarp();
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_MMA); }
+        __syncwarp();
+    } else {
+        // =========================== epilogue ===================================================
+        const int q = warp % 4;               // TMEM lane quadrant of this warp
+        const int row = q * 32 + lane;        // accumulator row handled by this thread
+        const int t128 = threadIdx.x - 64;
+        // tile row = wi + bw * (ni + bn * hi): the same for every tile
+        const int r1 = fast_div(row, p.rcp_bw), hi_ = fast_div(row, p.rcp_bwbn);
+        const int wi = row - r1 * p.bw, ni = r1 - hi_ * p.bn;
+        bool ok = true;
+        int i = 0;
+        for (int t = blockIdx.x; t < n_tiles_total; t += gridDim.x, ++i) {
+            const int buf = i & 1;
+            int pw0, ph0, pn0, n0;
+            tile_coords(t, pw0, ph0, pn0, n0);
+            const int n_hi = p.n_total;
+            const int w = pw0 + wi, h = ph0 + hi_, n = pn0 + ni;
+            const bool row_ok = w < p.W && h < p.H && n < p.N;
+            const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
+            if (MODE == MODE_FWD && p.epi == UEPI_BIAS_ACT) {
+                // (the previous tile's epilogue has passed its last barrier: nobody still reads the old bias values)
+                for (int c = t128; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
+            }
+            if (lane == 0) ok = mbar_wait(&acc_full[buf], (uint32_t)((i >> 1) & 1));
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) {
+                if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+            }
+            epi_bar_sync();                       // bias staged; a timeout seen by any epilogue warp is seen by all below
+            if (*abort_flag) break;
+            SB_TLOG(t128 == 0 && i < 4, 8 + 2 * i, clock64());      // accumulator of tile i complete
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, 0, s_bias, stage_out, row);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            tc_fence_before();
+            epi_bar_sync();                       // the tile is staged and every warp has finished reading the accumulator
+            if (t128 == 0) {
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&acc_empty[buf])) : "memory");   // accumulator free
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j)
+                    if (n0 + 64 * j < n_hi) tma_store_4d(&mapC, smem_u32(stage_out) + j * 16384, n0 + 64 * j, pw0, pn0, ph0);    // (c, w, n, h)
+                tma_store_commit();
+            }
+            if (MODE == MODE_FWD && p.pool_out != nullptr) pool_from_stage<BN>(p, stage_out, t128, n0, n_hi, pw0, ph0, pn0);
+            if (t128 == 0) tma_store_wait_read();
+            epi_bar_sync();                       // the stage may be overwritten by the next tile
+            SB_TLOG(t128 == 0 && i < 4, 9 + 2 * i, clock64());      // epilogue of tile i done
+        }
+    }
+
+    // ---- teardown: everyone meets here; TMEM is released on every path ----------------------------
+    tc_fence_before();
+    __syncthreads();
+    SB_TLOG(threadIdx.x == 0, 5, clock64());
+    SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
+    if (*abort_flag) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // The CTA-pair kernel (FWD / DGRAD): tcgen05.mma.cta_group::2
 // ------------------------------------------------------------------------------------------------
 // Two CTAs of a cluster -- neighbouring M tiles with the same N tile and split -- run as one 256 x BN MMA.
@@ -1472,6 +1755,36 @@ static cudaError_t launch_halo_mode(int bn, const UmmaOp& op, const UmmaParams& 
     }
 }
 
+template <int MODE, int BN>
+static cudaError_t launch_halo_persist_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    const int a_slot = (p.bh + 2) * p.bw * p.bn * 128;
+    const int smem = HaloPersistCfg<BN>::smem_bytes(p.a_stages, a_slot, p.stages);
+    if (p.a_stages < 1 || p.a_stages > MAX_A_STAGES || p.stages < 3 || p.stages > MAX_STAGES || smem > 227 * 1024 || !p.tma_out || p.splits != 1)
+        return cudaErrorInvalidValue;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(umma_halo_persist_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    return pdl_launch(umma_halo_persist_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)smem, st, op.mapA, op.mapB, op.mapC, p);
+}
+template <int MODE>
+static cudaError_t launch_halo_persist_mode(int bn, const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
+{
+    switch (bn) {
+    case 64: return launch_halo_persist_one<MODE, 64>(op, p, grid, st);
+    case 128: return launch_halo_persist_one<MODE, 128>(op, p, grid, st);
+    case 256: return launch_halo_persist_one<MODE, 256>(op, p, grid, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
 // CTA-pair launch: clusters of two CTAs along x, programmatic dependent launch as everywhere else.
 template <int MODE, int BN>
 static cudaError_t launch_pair_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, cudaStream_t st)
@@ -1530,6 +1843,7 @@ struct OpBlock {
     int bn;
     int pair;      // FWD / DGRAD: run as CTA pairs (umma_pair_kernel); grid.x is then even
     int halo;      // 3x3 FWD / DGRAD: umma_halo_kernel (activation halos shared by the three taps of a filter column)
+    int persist;   // ... its persistent variant: grid.x CTAs walk all tiles (umma_halo_persist_kernel)
     dim3 grid;
     long rows;     // output rows (pixels / batch rows) of a FWD / DGRAD op
 };
@@ -1549,6 +1863,10 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     UmmaParams pp = b->p;
 #ifdef SB_CTA_TIMING
     pp.timing = g_timing;
+    {
+        static const int only_mode = (int)tune("SB_TLOG_MODE", -1);      // log only kernels of one mode (0 fwd, 1 dgrad, 2 wgrad)
+        if (only_mode >= 0 && pp.mode != only_mode) pp.timing = nullptr;
+    }
     pp.dbg_skip = (int)tune("SB_HALO_SKIP", 0);
 #endif
     if (pp.mode != MODE_WGRAD) {
@@ -1559,8 +1877,11 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
         pp.rcp_wb = fast_rcp((uint32_t)(pp.bw / 2));
         pp.rcp_wbhb = fast_rcp((uint32_t)((pp.bw / 2) * (pp.bh / 2)));
         pp.rcp_bwbn = fast_rcp((uint32_t)(pp.bw * pp.bn));
+        pp.rcp_mtiles = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h * pp.tiles_n));
     }
-    if (b->halo && b->p.mode == MODE_FWD) e = launch_halo_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    if (b->halo && b->persist && b->p.mode == MODE_FWD) e = launch_halo_persist_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
+    else if (b->halo && b->persist && b->p.mode == MODE_DGRAD) e = launch_halo_persist_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
+    else if (b->halo && b->p.mode == MODE_FWD) e = launch_halo_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->halo && b->p.mode == MODE_DGRAD) e = launch_halo_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_FWD) e = launch_pair_mode<MODE_FWD>(b->bn, op, pp, b->grid, st);
     else if (b->pair && b->p.mode == MODE_DGRAD) e = launch_pair_mode<MODE_DGRAD>(b->bn, op, pp, b->grid, st);
@@ -1617,7 +1938,7 @@ cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cud
 //    reduced in split order by splitk_epilogue) while every CTA keeps at least 4 k-iterations,
 //  * ring depth = k-iterations per CTA, capped by what fits; for grids of several waves the ring is kept
 //    shallow enough that two CTAs share an SM, so one CTA's epilogue overlaps the other's main loop.
-struct TilePlan { int bn, splits, cps, stages, pair, halo, a_stages; };
+struct TilePlan { int bn, splits, cps, stages, pair, halo, a_stages, persist, persist_ctas; };
 // Backward kernels of the two concurrent streams share SMs only if two CTAs fit side by side (shared
 // memory <= ~110 KB each, TMEM columns <= 256 each): SB_BWD_COHABIT=0 gives every kernel the full ring again.
 static bool bwd_cohabit()
@@ -1702,6 +2023,8 @@ static TilePlan plan_tiles(int n_cols_per_shard, int shards, long m_tiles, int k
     t.pair = 0;
     t.halo = 0;
     t.a_stages = 0;
+    t.persist = 0;
+    t.persist_ctas = 0;
     // (SB_FLAG_FORCE_PAIR: every 128- or 256-wide tile, whatever the grid -- for tests at small sizes)
     if ((pair_on && t.bn == 256 && m_tiles % 2 == 0 && tiles * t.splits >= pair_min_ctas) || (force_pair && t.bn >= 128)) {
         t.pair = 1;
@@ -1800,6 +2123,45 @@ static TilePlan plan_tiles_halo(int n_cols, long m_tiles, int kchunks, int a_slo
     return t;
 }
 
+// Plan of the persistent halo kernel (layers of several tiles per SM, unsplit): 128-wide tiles where the layer has the
+// columns (one CTA per SM with the deepest rings), 64-wide ones otherwise (two CTAs per SM with two-group rings).
+static TilePlan plan_tiles_halo_persist(int n_cols, long m_tiles, int kchunks, int a_slot_bytes)
+{
+    TilePlan t{};
+    t.halo = 1;
+    t.persist = 1;
+    static const int f_bn = (int)tune("SB_PERSIST_BN", 0);
+    t.bn = f_bn > 0 ? f_bn : (n_cols >= 128 ? 128 : 64);
+    t.splits = 1;
+    t.cps = 3 * kchunks;
+    const int b_stage = t.bn * 128, stage_out = (t.bn / 64) * 16384;
+    int per_sm = 1, sa = 2, sb = 6;
+    if (2 * (2 * a_slot_bytes + 6 * b_stage + stage_out + 4 * 1024) <= 227 * 1024 && 2 * 2 * t.bn <= 512) {
+        per_sm = 2;
+        sb = ((227 * 1024 / 2) - 4 * 1024 - stage_out - 2 * a_slot_bytes) / b_stage;
+    } else {
+        sa = 3;
+        sb = (227 * 1024 - 4 * 1024 - stage_out - 3 * a_slot_bytes) / b_stage;
+        if (sb < 6) { sa = 2; sb = (227 * 1024 - 4 * 1024 - stage_out - 2 * a_slot_bytes) / b_stage; }
+    }
+    if (sb > MAX_STAGES) sb = MAX_STAGES;
+    if (sb < 3) sb = 3;
+    {
+        static const int f_sa = (int)tune("SB_PERSIST_SA", 0), f_sb = (int)tune("SB_PERSIST_SB", 0), f_per = (int)tune("SB_PERSIST_PER_SM", 0);
+        if (f_sa > 0) sa = f_sa;
+        if (f_sb > 0) sb = f_sb;
+        if (f_per > 0) per_sm = f_per;
+    }
+    t.a_stages = sa;
+    t.stages = sb;
+    const long tiles = m_tiles * cdiv_i(n_cols, t.bn);
+    const long slots = 148L * per_sm;
+    t.persist_ctas = (int)(tiles < slots ? tiles : slots);
+    static const bool verbose = tune("SB_PLAN_VERBOSE", 0) != 0;
+    if (verbose) fprintf(stderr, "plan: halo persistent N=%d m_tiles=%ld kchunks=%d -> bn=%d a_stages=%d b_stages=%d ctas=%d (%ld tiles)\n", n_cols, m_tiles, kchunks, t.bn, t.a_stages, t.stages, t.persist_ctas, tiles);
+    return t;
+}
+
 // Conv weight-gradient split count. Splitting the pixel (K) dimension fills more SMs but every split
 // writes a float copy of the weight gradient and the ordered reduce reads them all back, so the choice is
 // a small cost model: waves x (chunks per CTA x per-chunk operand time + fixed CTA cost) for the GEMM
@@ -1854,7 +2216,7 @@ struct ConvGeom {
     int cw, ch, cn, ctw, cth, ctn, total_chunks;   // 64-pixel boxes (WGRAD k-chunks)
     int wg_bn, wg_n_tiles, wg_m_tiles, wg_splits, wg_cps, wg_tap_group;
 };
-static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_halo)
+static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_halo, bool force_persist)
 {
     ConvGeom g;
     static const bool halo_on = tune("SB_HALO", 1) != 0;
@@ -1865,10 +2227,23 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_h
     static const long halo_max_tiles = (long)tune("SB_HALO_MAX_TILES", 160);
     int hbw = 0, hbh = 0, hbn = 0;
     bool halo = halo_on && !force_pair && !no_halo && choose_box_halo(lv.W, lv.H, B, &hbw, &hbh, &hbn);
+    static const bool persist_on = tune("SB_HALO_PERSIST", 1) != 0;
+    static const long persist_max_width = (long)tune("SB_PERSIST_MAX_WIDTH", 128);
+    bool persist = false;
     if (halo) {
         const long mt = (long)cdiv_i(lv.W, hbw) * cdiv_i(lv.H, hbh) * cdiv_i(B, hbn);
         const int widest = lv.Cout < lv.Cin ? lv.Cout : lv.Cin;
-        if (mt * cdiv_i(widest, widest >= 128 ? 128 : 64) > halo_max_tiles) halo = false;
+        const long tiles = mt * cdiv_i(widest, widest >= 128 ? 128 : 64);
+        if (tiles > halo_max_tiles || force_persist) {
+            // Four or more tiles per SM: the persistent variant (layers up to 128 channels wide; wider ones do better on the
+            // per-tap kernel's CTA pairs with 256-column tiles).  Measured at CIFAR size, batch 128: the 1024-tile layer
+            // 20.3 -> 16.3 us, the 256-tile layers 7.3 -> 9.0 and 12.8 -> 13.5 us (one or two tiles per CTA do not repay the
+            // second accumulator's set-up); ImageNet-size step -3.6 %, batch 256 -2 %.
+            static const long persist_min_tiles = (long)tune("SB_PERSIST_MIN_TILES", 4 * 148);
+            persist = persist_on && (tiles >= persist_min_tiles || force_persist) && lv.Cout <= persist_max_width && lv.Cin <= persist_max_width &&
+                      lv.Cout % 64 == 0 && lv.Cin % 64 == 0;
+            if (!persist) halo = false;
+        }
     }
     if (halo) {
         g.bw = hbw; g.bh = hbh; g.bn = hbn;
@@ -1876,8 +2251,17 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_h
         g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
         g.m_tiles = (long)g.tw * g.th * g.tn;
         const int a_slot = (g.bh + 2) * g.bw * g.bn * 128;
-        g.fwd = plan_tiles_halo(lv.Cout, g.m_tiles, lv.Cin / 64, a_slot, false);
-        g.dgrad = plan_tiles_halo(lv.Cin, g.m_tiles, lv.Cout / 64, a_slot, true);
+        if (persist) {
+            g.fwd = plan_tiles_halo_persist(lv.Cout, g.m_tiles, lv.Cin / 64, a_slot);
+            g.dgrad = plan_tiles_halo_persist(lv.Cin, g.m_tiles, lv.Cout / 64, a_slot);
+            if (force_persist) {      // (tests at small sizes: few CTAs, so that each walks several tiles and reuses both accumulators)
+                if (g.fwd.persist_ctas > 3) g.fwd.persist_ctas = 3;
+                if (g.dgrad.persist_ctas > 3) g.dgrad.persist_ctas = 3;
+            }
+        } else {
+            g.fwd = plan_tiles_halo(lv.Cout, g.m_tiles, lv.Cin / 64, a_slot, false);
+            g.dgrad = plan_tiles_halo(lv.Cin, g.m_tiles, lv.Cout / 64, a_slot, true);
+        }
     } else {
         choose_box(lv.W, lv.H, B, 128, &g.bw, &g.bh, &g.bn);
         g.tw = cdiv_i(lv.W, g.bw); g.th = cdiv_i(lv.H, g.bh); g.tn = cdiv_i(B, g.bn);
@@ -1939,7 +2323,7 @@ sb_status umma_plan_scratch(sb_model* m, size_t* floats)
     for (int i = 0; i < mv.n_layers; ++i) {
         LayerView lv = layer_view(m, i);
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            ConvGeom g = conv_geom(lv, mv.B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0);
+            ConvGeom g = conv_geom(lv, mv.B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0, (mv.cfg->flags & SB_FLAG_FORCE_PERSIST) != 0);
             const size_t pix = (size_t)mv.B * lv.H * lv.W;
             if (g.wg_splits > 1) upd((size_t)g.wg_splits * (lv.n_w + lv.n_b));
             if (g.fwd.splits > 1) upd((size_t)g.fwd.splits * pix * lv.Cout);
@@ -1969,10 +2353,12 @@ static void apply_plan(OpBlock* b, const TilePlan& t, int k_iters, long m_tiles,
     p.a_stages = t.a_stages;
     p.hn_order = t.halo;
     b->halo = t.halo;
+    b->persist = t.persist;
     p.part = t.splits > 1 ? ws : nullptr;
     p.split_stride = (long)(rows * (size_t)p.n_total);
     b->pair = t.pair;
     b->grid = dim3((unsigned)(t.pair ? (m_tiles + 1) / 2 * 2 : m_tiles), (unsigned)n_tiles_total, (unsigned)t.splits);
+    if (t.persist) b->grid = dim3((unsigned)t.persist_ctas, 1, 1);
     b->rows = (long)rows;
 }
 
@@ -1986,6 +2372,7 @@ static bool tma_out_ok(const OpBlock* b, int cols_per_shard, int shards)
     if (off || p.out_f32 || p.splits > 1 || p.epi == UEPI_F32) return false;
     if (p.n_total % 64 != 0 || p.ldc % 64 != 0) return false;
     if (shards > 1 && (cols_per_shard % b->bn != 0 || p.n_total % shards != 0)) return false;
+    if (b->halo && b->persist) return true;
     if (b->halo) return (long)p.a_stages * (p.bh + 2) * p.bw * p.bn * 128 + (long)p.stages * b->bn * 128 >= (long)(b->bn / 64) * 16384;
     const long stage_bytes = b->pair ? 16384 + b->bn * 64 : 16384 + b->bn * 128;
     return (long)p.stages * stage_bytes >= (long)(b->bn / 64) * 16384;
@@ -2010,7 +2397,7 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
             }
         }
         if (lv.kind == SB_CONV3X3_RELU && conv_umma_ok(mv, lv, i)) {
-            const ConvGeom g = conv_geom(lv, B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0);
+            const ConvGeom g = conv_geom(lv, B, (mv.cfg->flags & SB_FLAG_FORCE_PAIR) != 0, (mv.cfg->flags & SB_FLAG_NO_HALO) != 0, (mv.cfg->flags & SB_FLAG_FORCE_PERSIST) != 0);
             const size_t pix = (size_t)B * lv.H * lv.W;
             // ---- forward ----
             {
