@@ -212,6 +212,8 @@ def run_ours(args):
     t_wall0 = time.time()
     blocks = [timed_block(step)]
     want = max_over_ranks([min(200.0, max(1.0, np.ceil(500.0 / max(blocks[0], 1e-3))))], world, "cuda")[0]
+    if args.repeats > 0:
+        want = args.repeats
     for _ in range(int(want) - 1):
         blocks.append(timed_block(step))
     t_wall1 = time.time()
@@ -406,6 +408,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="number of timed blocks of --steps steps (0 = as many as cover half a second; 1 for a profiler capture)")
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4, 5],
                     help="1 = VGG-16 CIFAR shape, batch 128 (the metric's configuration); 0/2/3 = the other configurations; "
                          "4 = the sharded-FC sweep (TFLOP/s per point); 5 = the paper's own 7-conv / 3-FC CIFAR network (its Table 1), "
