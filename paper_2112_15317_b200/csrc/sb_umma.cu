@@ -77,6 +77,7 @@ struct UmmaParams {
     int bias_fused;       // WGRAD: the centre-tap CTAs of the first N tile also sum dy over the pixels (the bias gradient)
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
+    int wg_sweep;         // WGRAD: the float tile leaves through shared memory in contiguous row segments (wgrad_sweep_epilogue)
     // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
     // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
     uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
@@ -124,6 +125,54 @@ template <int MODE, int BN> struct Cfg {
     static constexpr int TMEM_COLS = BN == 192 ? 256 : BN;    // allocations are powers of two
     static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES; }
 };
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 128 epilogue threads (warps 2..5)
+
+// Weight-gradient epilogue through shared memory: the float tile leaves in whole, contiguous row segments.
+// The accumulator row of a thread is one gradient ROW (ldc floats apart from the next thread's), so storing it
+// straight from registers gives every warp instruction 32 separate 16-byte pieces (measured 2.3 TB/s on a 411 MB
+// gradient).  Here the tile goes through the drained operand ring in slabs of 64 columns -- thread r writes its 64 floats
+// as 16-byte chunks, chunk c at position c ^ (r & 7) of its 8-chunk group, which spreads a warp's stores over all banks
+// -- and is then swept row by row: half a warp takes one row's 256 contiguous bytes, so every global access of a warp
+// is two whole 256-byte runs.
+template <int BN>
+__device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32_t taddr, uint8_t* stage, int row, int m0, int m_hi,
+                                                      int n0, int n_hi, size_t tile_off)
+{
+    const int t128 = threadIdx.x - 64, q = t128 >> 5, lane = t128 & 31;
+    const int hl = lane & 15, sub = lane >> 4;
+    const uint32_t stage_s = smem_u32(stage);
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+        if (n0 + c0 >= n_hi) break;                       // (uniform)
+#pragma unroll
+        for (int cc = 0; cc < 64; cc += 16) {
+            uint32_t v[16];
+            tmem_ld16(taddr + c0 + cc, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t ch = (uint32_t)(cc / 4 + j);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_s + (uint32_t)row * 256u + ((ch ^ (uint32_t)(row & 7)) << 4)),
+                             "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
+            }
+        }
+        epi_bar_sync();
+        const int col = n0 + c0 + 4 * hl;
+        if (col < n_hi) {
+#pragma unroll 2
+            for (int rr = q * 2 + sub; rr < 128; rr += 8) {
+                if (m0 + rr >= m_hi) break;
+                float4 g;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(g.x), "=f"(g.y), "=f"(g.z), "=f"(g.w)
+                             : "r"(stage_s + (uint32_t)rr * 256u + (((uint32_t)hl ^ (uint32_t)(rr & 7)) << 4)));
+                const size_t off = tile_off + (size_t)rr * p.ldc + c0 + 4 * hl;
+                *(float4*)((float*)p.out + off) = g;
+            }
+        }
+        epi_bar_sync();                                   // the slab may be overwritten
+    }
+}
 
 // Epilogue of one accumulator row: reads BN columns of this warp's TMEM lane quadrant (16 at a time) and
 // writes them as raw split partial sums, or with bias + ReLU / the ReLU mask applied, as float or bf16.
@@ -649,9 +698,18 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
         if (lane == 0 && ok) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) {
-            if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
-        } else {
+        if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
+        if (MODE == MODE_WGRAD && p.wg_sweep) {
+            // (the four epilogue warps work on the tile together: all of them reach this barrier, also after a timeout)
+            epi_bar_sync();
+            if (!*abort_flag) {
+                SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+                wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
+                                         (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0);
+            }
+        } else if (ok) {
             SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -1013,7 +1071,6 @@ template <int BN> struct HaloPersistCfg {
         return a_stages * a_slot_bytes + b_stages * B_STAGE_BYTES + STAGE_OUT_BYTES + 1024 /*alignment slack*/ + CTRL_BYTES;
     }
 };
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 128 epilogue threads
 
 template <int MODE, int BN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
@@ -1861,6 +1918,13 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     const OpBlock* b = blk(op);
     cudaError_t e;
     UmmaParams pp = b->p;
+    if (pp.mode == MODE_WGRAD && !b->pair) {
+        static const bool sweep_on = tune("SB_WGRAD_SWEEP", 1) != 0;
+        const bool aligned = (pp.ldc & 3) == 0 && (pp.w_cols & 3) == 0 && (pp.n_total & 3) == 0 && (pp.split_stride & 3) == 0 &&
+                             (((uintptr_t)pp.out) & 15) == 0;
+        const long ring = (long)pp.stages * (A_STAGE_BYTES + b->bn * 128);
+        pp.wg_sweep = (sweep_on && aligned && ring >= 32768) ? 1 : 0;
+    }
 #ifdef SB_CTA_TIMING
     pp.timing = g_timing;
     {
