@@ -271,22 +271,31 @@ sb_status sb_partition(const sb_layer* layers, int32_t n, const sb_config* cfg, 
 const char* sb_partition_last_error(void);
 
 /*
- * Exchange schedule of ONE MP group of G = R = K workers, worker i being data replica i and model shard i
- * [Modulo Layer, Shard Layer; Distributed Machine Learning: reduce].  Lists every block that travels between two
- * workers in one synchronous iteration, forward pass first, then the backward pass in execution order:
- *   SB_X_GATHER_ROWS : modulo layer, forward.  src sends its b feature rows [row0,row1) x all D columns to dst.
- *   SB_X_GATHER_COLS : shard layer, forward.  src sends its column slice [col0,col1) of layer `layer`'s [B,width] output.
+ * Exchange schedule of N = R workers in R / K MP groups of K = mp workers each [Modulo Layer, Shard Layer, Group MP
+ * Extension; Distributed Machine Learning: reduce].  Worker p is data replica p (rows [p*b, (p+1)*b) of the N*b-row
+ * batch), belongs to group gid = p / K and holds model shard off = p % K of that group; R must be a multiple of K
+ * (R = K: a single group; K = 1: pure data parallelism).  Lists every block that travels between two workers in one
+ * synchronous iteration, forward pass first, then the backward pass in execution order; src and dst are worker ids,
+ * rows are rows of the whole batch:
+ *   SB_X_GATHER_ROWS : modulo layer, forward.  src sends its b feature rows [row0,row1) x all D columns to dst (same group).
+ *   SB_X_GATHER_COLS : shard layer, forward.  src sends its column slice [col0,col1) of layer `layer`'s output for the
+ *                      group's rows [row0,row1).
  *   SB_X_REDUCE_COLS : shard layer, backward.  src sends columns [col0,col1) (dst's slice) of its full-width partial
- *                      gradient w.r.t. layer `layer`'s output; dst adds the G partial results in worker order 0..G-1.
+ *                      gradient w.r.t. layer `layer`'s output; dst adds the K partial results in worker order.
  *   SB_X_REDUCE_ROWS : modulo layer, backward.  src sends rows [row0,row1) (dst's examples) of its full-width partial
- *                      gradient w.r.t. the features; dst adds the G partial results in worker order.
+ *                      gradient w.r.t. the features; dst adds the K partial results in worker order.
  *   SB_X_ALLREDUCE   : the parameters of layer `layer` are held by every worker and trained on its own rows (conv stack):
- *                      their gradients are summed over all workers (src = dst = -1).
- * On one GPU every one of these is addressing inside one device buffer; this table is the contract a multi-GPU
- * runtime has to carry out (it has been executed by CPU worker processes in the tests, not on several GPUs).
+ *                      their gradients are summed over all N workers (src = dst = -1).
+ *   SB_X_ALLREDUCE_GROUPS : more than one group only.  Shard src (= offset inside a group; -1: a layer kept whole, every
+ *                      offset) of FC layer `layer`, output columns [col0,col1), was trained by each group on that group's
+ *                      rows: its gradients are summed over the workers gid*K + src of all groups, in group order.
+ * On one GPU every one of these is addressing inside one device buffer (the arithmetic of N workers in groups of mp is
+ * sb_config's R = N, K = mp); this table is the contract a multi-GPU runtime has to carry out (it has been executed
+ * by CPU worker processes in the tests, not on several GPUs).
  * Host-only.  out may be NULL to query the count.
  */
-typedef enum { SB_X_GATHER_ROWS = 1, SB_X_GATHER_COLS = 2, SB_X_REDUCE_COLS = 3, SB_X_REDUCE_ROWS = 4, SB_X_ALLREDUCE = 5 } sb_exchange_kind;
+typedef enum { SB_X_GATHER_ROWS = 1, SB_X_GATHER_COLS = 2, SB_X_REDUCE_COLS = 3, SB_X_REDUCE_ROWS = 4, SB_X_ALLREDUCE = 5,
+               SB_X_ALLREDUCE_GROUPS = 6 } sb_exchange_kind;
 typedef struct {
     int32_t kind;   /* sb_exchange_kind */
     int32_t layer;  /* layer whose output (or parameters) the block belongs to; for the modulo layer: the first split FC layer */

@@ -21,7 +21,7 @@ SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
 SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT, SB_FC_RELU_WHOLE, SB_FC_WHOLE = 1, 2, 3, 4, 5, 6, 7
 SB_NODE_LAYER, SB_NODE_MODULO, SB_NODE_SHARD = 0, 1, 2
-SB_X_GATHER_ROWS, SB_X_GATHER_COLS, SB_X_REDUCE_COLS, SB_X_REDUCE_ROWS, SB_X_ALLREDUCE = 1, 2, 3, 4, 5
+SB_X_GATHER_ROWS, SB_X_GATHER_COLS, SB_X_REDUCE_COLS, SB_X_REDUCE_ROWS, SB_X_ALLREDUCE, SB_X_ALLREDUCE_GROUPS = 1, 2, 3, 4, 5, 6
 SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO, SB_FLAG_FORCE_PERSIST = 1, 2, 4, 8, 16, 32, 64
 (SB_T_WEIGHT, SB_T_BIAS, SB_T_GRAD_W, SB_T_GRAD_B, SB_T_MOM_W, SB_T_MOM_B, SB_T_ACT, SB_T_DACT,
  SB_T_POOL_IDX, SB_T_ROW_LOSS, SB_T_INPUT_GRAD, SB_T_SHADOW_W) = range(12)
@@ -154,10 +154,11 @@ def partition(layers, H, W, C, K):
     return [dict(node=o.node, layer=o.layer, shards=o.shards, dim=o.dim, dimF=o.dimF) for o in out]
 
 
-def exchange_plan(layers, H, W, C, b, G):
-    """The exchange schedule of one MP group of G workers (sb_exchange_plan) as a list of dicts (host-only)."""
+def exchange_plan(layers, H, W, C, b, N, mp=None):
+    """The exchange schedule of N workers in MP groups of mp (default: one group of N) from sb_exchange_plan, as a list
+    of dicts (host-only)."""
     arr = _layers_array(layers)
-    cfg = sb_config(H, W, C, b, G, G, SB_FP32, 0)
+    cfg = sb_config(H, W, C, b, N, N if mp is None else mp, SB_FP32, 0)
     n = c_int32()
     st = sb_exchange_plan(arr, len(layers), byref(cfg), None, 0, byref(n))
     if st != SB_OK:

@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
     tmp = LIB + f".tmp{os.getpid()}"
-    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-cudart", "static"], check=True)
+    subprocess.run([nvcc, "-shared"] + NVCC_FLAGS[:2] + ["-o", tmp] + objs + ["-cudart", "static"], check=True)
     os.replace(tmp, LIB)
     return LIB
 

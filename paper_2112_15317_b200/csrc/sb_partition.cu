@@ -13,11 +13,15 @@
 // dim with dimF; the surrounding text compares the two widths of the layer's INPUT ("if the input dimension has been
 // partitioned, a shard layer is inserted"), which is what is done here.
 //
-// sb_exchange_plan lists, for an MP group of G workers in which worker i is data replica i and model shard i
-// (R = K = G), every block of every matrix that has to travel between two workers in one synchronous iteration
-// [Modulo Layer and Shard Layer paragraphs and their figures]: the modulo layer's gather of feature rows and the
-// return of gradient rows, the shard layer's gather of column slices and the reduce of gradient column slices, and
-// the replicas' parameter reduce [Distributed Machine Learning: reduce].
+// sb_exchange_plan lists, for N = R workers arranged in R / K MP groups of K = mp workers each [Group MP Extension], every
+// block of every matrix that has to travel between two workers in one synchronous iteration [Modulo Layer and Shard
+// Layer paragraphs and their figures]: the modulo layer's gather of feature rows and the return of gradient rows, the
+// shard layer's gather of column slices and the reduce of gradient column slices -- all of them inside one group --
+// and the two parameter reduces [Distributed Machine Learning: reduce; Implementation]: the conv stack over all N
+// workers, and each FC shard over the workers that hold the same shard in the other groups.  Worker p belongs to group
+// gid = p / mp and is data replica p and model shard off = p % mp of that group (the lost figure's mapping, taken from
+// the text: the group a worker belongs to, and its offset inside it); with R = K there is a single group, with K = 1
+// the schedule is pure data parallelism.
 #include "../../include/splitbrain.h"
 
 #include <cstdarg>
@@ -118,10 +122,11 @@ extern "C" sb_status sb_exchange_plan(const sb_layer* layers, int32_t n, const s
     std::vector<sb_plan_node> net;
     sb_status s = walk(layers, n, cfg, net);
     if (s != SB_OK) return s;
-    if (cfg->R != cfg->K) return fail(SB_ERR_UNSUPPORTED, "an MP group has one replica and one shard per worker: R (%d) must equal K (%d)", cfg->R, cfg->K);
+    if (cfg->R < 1 || cfg->R % cfg->K != 0)
+        return fail(SB_ERR_UNSUPPORTED, "the R (%d) workers form groups of K (%d): R must be a multiple of K", cfg->R, cfg->K);
     if (cfg->batch_per_replica < 1) return fail(SB_ERR_SHAPE, "batch_per_replica must be positive");
-    const int G = cfg->K;
-    const int64_t b = cfg->batch_per_replica, B = b * G;
+    const int mp = cfg->K, N = cfg->R, G = N / mp;                    // group size, workers, groups
+    const int64_t b = cfg->batch_per_replica, Bg = b * mp;             // rows one worker owns, rows one group works on
     std::vector<sb_exchange_msg> fwd;
     std::vector<std::vector<sb_exchange_msg>> bwd_blocks;      // one block per node, in forward order
     auto msg = [&](int kind, int layer, int pass, int src, int dst, int64_t r0, int64_t r1, int64_t c0, int64_t c1, int64_t width) {
@@ -130,44 +135,60 @@ extern "C" sb_status sb_exchange_plan(const sb_layer* layers, int32_t n, const s
         m.row0 = r0; m.row1 = r1; m.col0 = c0; m.col1 = c1; m.width = width;
         return m;
     };
-    bool gathered = false;      // the modulo layer has run: every worker holds all B rows from here on
+    bool gathered = false;      // the modulo layer has run: every worker holds all rows of its group from here on
     for (size_t k = 0; k < net.size(); ++k) {
         const sb_plan_node& nd = net[k];
         bwd_blocks.emplace_back();
         std::vector<sb_exchange_msg>& bwd_rev = bwd_blocks.back();
         if (nd.node == SB_NODE_MODULO) {
-            // forward: worker i owns rows [i*b, (i+1)*b) of the [B, D] feature matrix and sends them to every other worker;
-            // backward: worker src holds a full-width partial gradient for ALL rows and returns rows [dst*b, (dst+1)*b) to
-            // their owner, which sums the G partial results in worker order
-            for (int src = 0; src < G; ++src)
-                for (int dst = 0; dst < G; ++dst) {
-                    if (src == dst) continue;
-                    fwd.push_back(msg(SB_X_GATHER_ROWS, nd.layer, 0, src, dst, src * b, (src + 1) * b, 0, nd.dimF, nd.dimF));
-                    bwd_rev.push_back(msg(SB_X_REDUCE_ROWS, nd.layer, 1, src, dst, dst * b, (dst + 1) * b, 0, nd.dimF, nd.dimF));
-                }
+            // forward: worker p owns rows [p*b, (p+1)*b) of the feature matrix and sends them to every other worker of its
+            // group; backward: worker src holds a full-width partial gradient for ALL rows of the group and returns dst's rows
+            // to their owner, which sums the mp partial results in worker order
+            for (int gid = 0; gid < G; ++gid)
+                for (int so = 0; so < mp; ++so)
+                    for (int d_o = 0; d_o < mp; ++d_o) {
+                        if (so == d_o) continue;
+                        const int src = gid * mp + so, dst = gid * mp + d_o;
+                        fwd.push_back(msg(SB_X_GATHER_ROWS, nd.layer, 0, src, dst, src * b, (src + 1) * b, 0, nd.dimF, nd.dimF));
+                        bwd_rev.push_back(msg(SB_X_REDUCE_ROWS, nd.layer, 1, src, dst, dst * b, (dst + 1) * b, 0, nd.dimF, nd.dimF));
+                    }
             gathered = true;
         } else if (nd.node == SB_NODE_SHARD) {
-            // the layer below (nd.layer - 1) is split: worker i holds columns [c_i, c_{i+1}) of its [B, width] output
+            // the layer below (nd.layer - 1) is split: the worker at offset o holds columns [c_o, c_{o+1}) of its group's
+            // [Bg, width] output
             const int below = nd.layer - 1;
             const int64_t width = nd.dimF;
             const bool consumer_split = layers[nd.layer].kind == SB_FC_RELU || layers[nd.layer].kind == SB_FC;
-            for (int src = 0; src < G; ++src)
-                for (int dst = 0; dst < G; ++dst) {
-                    if (src == dst) continue;
-                    fwd.push_back(msg(SB_X_GATHER_COLS, below, 0, src, dst, 0, B, lo(src, width, G), lo(src + 1, width, G), width));
-                    // backward: a split consumer computes a full-width partial input gradient on every worker; the slice that
-                    // belongs to worker dst travels there and is summed in worker order.  A whole consumer (and the loss, which
-                    // every worker evaluates on the full logits) yields the same full gradient everywhere: each worker just
-                    // keeps its own column slice, nothing travels.
-                    if (consumer_split)
-                        bwd_rev.push_back(msg(SB_X_REDUCE_COLS, below, 1, src, dst, 0, B, lo(dst, width, G), lo(dst + 1, width, G), width));
-                }
+            for (int gid = 0; gid < G; ++gid)
+                for (int so = 0; so < mp; ++so)
+                    for (int d_o = 0; d_o < mp; ++d_o) {
+                        if (so == d_o) continue;
+                        const int src = gid * mp + so, dst = gid * mp + d_o;
+                        const int64_t r0 = gid * Bg, r1 = (gid + 1) * Bg;
+                        fwd.push_back(msg(SB_X_GATHER_COLS, below, 0, src, dst, r0, r1, lo(so, width, mp), lo(so + 1, width, mp), width));
+                        // backward: a split consumer computes a full-width partial input gradient on every worker; the slice that
+                        // belongs to worker dst travels there and is summed in worker order.  A whole consumer (and the loss, which
+                        // every worker evaluates on the full logits) yields the same full gradient everywhere in the group: each
+                        // worker just keeps its own column slice, nothing travels.
+                        if (consumer_split)
+                            bwd_rev.push_back(msg(SB_X_REDUCE_COLS, below, 1, src, dst, r0, r1, lo(d_o, width, mp), lo(d_o + 1, width, mp), width));
+                    }
         } else {
             const int kind = layers[nd.layer].kind;
-            // parameters that every worker holds AND trains on its own rows are reduced over the replicas: the conv stack, and
-            // an FC layer kept whole below the modulo layer.  (Above it every worker sees all B rows: the copies stay equal.)
-            const bool dp_params = kind == SB_CONV3X3_RELU || (is_whole(kind) && !gathered);
-            if (dp_params && G > 1) bwd_rev.push_back(msg(SB_X_ALLREDUCE, nd.layer, 1, -1, -1, 0, 0, 0, 0, 0));
+            // parameters that every worker holds AND trains on its own rows are reduced over all N workers: the conv stack, and
+            // an FC layer kept whole below the modulo layer (every FC layer when K = 1).
+            const bool dp_params = kind == SB_CONV3X3_RELU || (is_fc(kind) && nd.shards == 1 && !gathered);
+            if (dp_params && N > 1) bwd_rev.push_back(msg(SB_X_ALLREDUCE, nd.layer, 1, -1, -1, 0, 0, 0, 0, 0));
+            // above the modulo layer a group trains its FC parameters on the group's rows only: shard o is summed over the
+            // workers at offset o of every group (src = o); a layer kept whole there is equal on all workers of a group and
+            // is summed over the groups likewise (src = -1: every offset)
+            if (is_fc(kind) && !dp_params && G > 1) {
+                if (nd.shards > 1)
+                    for (int o = 0; o < mp; ++o)
+                        bwd_rev.push_back(msg(SB_X_ALLREDUCE_GROUPS, nd.layer, 1, o, -1, 0, 0, lo(o, nd.dimF, mp), lo(o + 1, nd.dimF, mp), nd.dimF));
+                else
+                    bwd_rev.push_back(msg(SB_X_ALLREDUCE_GROUPS, nd.layer, 1, -1, -1, 0, 0, 0, nd.dimF, nd.dimF));
+            }
         }
     }
     std::vector<sb_exchange_msg> all(fwd);

@@ -2545,11 +2545,9 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                     // grids of fewer than ~100 CTAs leave the other streams whole SMs: no need to keep the ring shallow (measured: -1.5 % step)
                     static const long wg_cohabit_min = (long)tune("SB_WG_COHABIT_MIN_CTAS", 100);
                     const long ctas = (long)p.m_tiles_per_shard * g.wg_n_tiles * ((9 + p.tap_group - 1) / p.tap_group) * p.splits;
-                    // (the filter-row kernel of a short reduction keeps a third 40 KB stage: CIFAR-size steps -1 to -2.7 %; a long
-                    // one leaves the room to the data-gradient kernel beside it: ImageNet-size step +1.9 % with three)
-                    static const int row3_max_cps = (int)tune("SB_WGRAD_ROW3_MAX_CHUNKS", 128);
-                    int cap = cohabit_stages(b->bn);
-                    if (b->bn == 192 && g.wg_cps <= row3_max_cps) cap = 3;
+                    // (the filter-row kernel keeps its whole five-stage ring: with two slots per round the deeper ring is worth more
+                    // than a neighbour on the SM -- steps -0.2 to -1.6 % against a ring cut to two or three 40 KB stages)
+                    const int cap = b->bn == 192 ? 5 : cohabit_stages(b->bn);
                     if (bwd_cohabit() && ctas >= wg_cohabit_min && p.stages > cap) p.stages = cap;
                 }
                 p.epi = UEPI_F32; p.ldc = 9L * lv.Cin;

@@ -134,10 +134,55 @@ def test_exchange_plan_blocks_tile_every_matrix(G, b_):
                 assert all(m["cols"] == (cb[dst], cb[dst + 1]) and m["rows"] == (0, B) for m in got)  # every sender's copy of MY slice
             else:
                 assert all(m["rows"] == (dst * b_, (dst + 1) * b_) and m["cols"] == (0, width) for m in got)
-    with pytest.raises(bnd.SBError, match="must equal K"):
+    with pytest.raises(bnd.SBError, match="multiple of K"):
         arr = bnd._layers_array(wl.layers)
         import ctypes
         cfg = bnd.sb_config(32, 32, 3, 4, 2, 4, 0, 0)
         n = ctypes.c_int32()
         st = bnd.sb_exchange_plan(arr, len(wl.layers), ctypes.byref(cfg), None, 0, ctypes.byref(n))
         raise bnd.SBError(st, bnd._lib.sb_partition_last_error().decode())
+
+
+@pytest.mark.parametrize("N,mp_,b_", [(4, 2, 3), (8, 2, 4), (8, 4, 2), (6, 3, 5)])
+def test_exchange_plan_with_several_mp_groups(N, mp_, b_):
+    """Group MP Extension: N workers in N / mp groups.  Worker p belongs to group p // mp at offset p % mp; the modulo
+    and shard layers' blocks stay inside a group and cover that group's rows only; the conv stack is reduced over all N
+    workers, every FC shard over the workers at the same offset of all groups."""
+    bnd = binding()
+    wl = si.config(5)
+    msgs = bnd.exchange_plan(wl.layers, 32, 32, 3, b_, N, mp_)
+    G = N // mp_
+    fc = [li for li, (k, _) in enumerate(wl.layers) if k in (si.FC_RELU, si.FC)]
+    conv = [li for li, (k, _) in enumerate(wl.layers) if k == si.CONV3X3_RELU]
+    p2p = [m for m in msgs if m["kind"] in (bnd.SB_X_GATHER_ROWS, bnd.SB_X_GATHER_COLS, bnd.SB_X_REDUCE_COLS, bnd.SB_X_REDUCE_ROWS)]
+    assert all(m["src"] // mp_ == m["dst"] // mp_ and m["src"] != m["dst"] for m in p2p)          # nothing crosses a group
+    for m in p2p:
+        gid = m["dst"] // mp_
+        g0, g1 = gid * mp_ * b_, (gid + 1) * mp_ * b_
+        if m["kind"] == bnd.SB_X_GATHER_ROWS:
+            assert m["rows"] == (m["src"] * b_, (m["src"] + 1) * b_) and g0 <= m["rows"][0] < g1  # owner of row g: worker g // b
+        elif m["kind"] == bnd.SB_X_REDUCE_ROWS:
+            assert m["rows"] == (m["dst"] * b_, (m["dst"] + 1) * b_)
+        else:
+            cb = si.shard_bounds(m["width"], mp_)
+            who = m["src"] if m["kind"] == bnd.SB_X_GATHER_COLS else m["dst"]
+            assert m["rows"] == (g0, g1) and m["cols"] == (cb[who % mp_], cb[who % mp_ + 1])
+    for kind, layers_ in [(bnd.SB_X_GATHER_ROWS, fc[:1]), (bnd.SB_X_REDUCE_ROWS, fc[:1]), (bnd.SB_X_GATHER_COLS, fc), (bnd.SB_X_REDUCE_COLS, fc[:-1])]:
+        for li in layers_:
+            assert len([m for m in p2p if m["kind"] == kind and m["layer"] == li]) == G * mp_ * (mp_ - 1)
+    # one group's traffic does not grow with the number of groups (the point of the extension): per worker, the modulo
+    # and shard layers receive (mp - 1) / mp of each matrix whatever N is
+    one = bnd.exchange_plan(wl.layers, 32, 32, 3, b_, mp_, mp_)
+    per_worker = lambda ms, w: sum((m["rows"][1] - m["rows"][0]) * (m["cols"][1] - m["cols"][0]) for m in ms if m["dst"] == w)
+    assert per_worker(p2p, N - 1) == per_worker([m for m in one if m["dst"] >= 0], mp_ - 1)
+    # parameter reduces
+    assert [m["layer"] for m in msgs if m["kind"] == bnd.SB_X_ALLREDUCE] == list(reversed(conv))
+    gr = [m for m in msgs if m["kind"] == bnd.SB_X_ALLREDUCE_GROUPS]
+    assert [(m["layer"], m["src"]) for m in gr] == [(li, o) for li in reversed(fc) for o in range(mp_)]
+    for m in gr:
+        cb = si.shard_bounds(m["width"], mp_)
+        assert m["cols"] == (cb[m["src"]], cb[m["src"] + 1]) and m["backward"] == 1
+    # a single group has no such entry; K = 1 is pure data parallelism: nothing but reduces over all workers, FC layers included
+    assert not [m for m in bnd.exchange_plan(wl.layers, 32, 32, 3, b_, mp_, mp_) if m["kind"] == bnd.SB_X_ALLREDUCE_GROUPS]
+    dp = bnd.exchange_plan(wl.layers, 32, 32, 3, b_, N, 1)
+    assert all(m["kind"] == bnd.SB_X_ALLREDUCE for m in dp) and [m["layer"] for m in dp] == list(reversed(sorted(conv + fc)))
