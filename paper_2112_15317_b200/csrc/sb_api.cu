@@ -814,7 +814,7 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
     const char* one = getenv("SB_ONE_STREAM");
     if (!(one && one[0] == '1')) {
         // second stream + ordering events for the backward pass (host objects; no device memory)
-        m->n_wstreams = (int)tune("SB_WSTREAMS", 4);
+        m->n_wstreams = (int)tune("SB_WSTREAMS", 6);
         if (m->n_wstreams < 1) m->n_wstreams = 1;
         if (m->n_wstreams > sb_model::MAX_WSTREAMS) m->n_wstreams = sb_model::MAX_WSTREAMS;
         bool ok_ = true;
@@ -1344,6 +1344,11 @@ sb_status sb_profile_end(sb_model* m, void* stream, sb_profile_entry* out, int32
 extern "C" sb_status sb_debug_cta_timing(void* dev_buffer)
 {
     umma_set_timing_buffer(dev_buffer);
+    return SB_OK;
+}
+extern "C" sb_status sb_debug_cta_trace(void* dev_buffer)
+{
+    umma_set_trace_buffer(dev_buffer);
     return SB_OK;
 }
 #endif

@@ -91,14 +91,24 @@ struct UmmaParams {
     unsigned long long* timing;   // development builds only: per-CTA phase timestamps, 16 per CTA, first 1024 CTAs
     int dbg_skip;                 // development builds only (halo kernel, timing experiments, WRONG results): bit 0 = no activation
                                   // loads after the first ring, bit 1 = no weight loads after the first ring
+    unsigned long long* trace;    // development builds only: [0] = record counter, records of 4 words from word 8 on (one per CTA)
 #endif
 };
 
 // Per-CTA phase stamps: compiled in only with -DSB_CTA_TIMING (a development aid; the shipped kernels carry none).
 #ifdef SB_CTA_TIMING
 #define SB_TLOG(cond, slot, val) do { if (tlog && (cond)) tlog[slot] = (unsigned long long)(val); } while (0)
+#define SB_TRACE_BEGIN() const unsigned long long trace_t0 = globaltimer_ns()
+#define SB_TRACE_END(kind) do { if (p.trace != nullptr && threadIdx.x == 0) { \
+        const unsigned long long ti_ = atomicAdd(p.trace, 1ull); \
+        if (ti_ < 60000ull) { unsigned long long* r_ = p.trace + 8 + 4 * ti_; unsigned smid_; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_)); \
+            r_[0] = trace_t0; r_[1] = globaltimer_ns(); \
+            r_[2] = (unsigned long long)smid_ | ((unsigned long long)(kind) << 16) | ((unsigned long long)p.mode << 24) | ((unsigned long long)(gridDim.x * gridDim.y * gridDim.z) << 32); \
+            r_[3] = (unsigned long long)(unsigned)p.total_chunks | ((unsigned long long)(unsigned)p.n_total << 32); } } } while (0)
 #else
 #define SB_TLOG(cond, slot, val) do { } while (0)
+#define SB_TRACE_BEGIN() do { } while (0)
+#define SB_TRACE_END(kind) do { } while (0)
 #endif
 
 __host__ __device__ __forceinline__ uint32_t fast_rcp(uint32_t d) { return d <= 1u ? 0u : (uint32_t)(0x100000000ull / d) + 1u; }
@@ -420,6 +430,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #endif
     (void)cta_lin;
     SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TRACE_BEGIN();
     SB_TLOG(threadIdx.x == 0, 6, clock64());
 
     // ---- tile coordinates ---------------------------------------------------------------------
@@ -734,6 +745,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (MODE != MODE_WGRAD && p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();   // shared memory may be released once the stores have read it; the writes complete with the grid
     SB_TLOG(threadIdx.x == 0, 5, clock64());   // epilogue done
     SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
+    SB_TRACE_END(0);
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
@@ -801,6 +813,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     unsigned long long* tlog = (p.timing != nullptr && cta_lin < 1024) ? p.timing + 16ull * cta_lin : nullptr;
 #endif
     SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TRACE_BEGIN();
     SB_TLOG(threadIdx.x == 0, 6, clock64());
 
     // ---- tile coordinates ---------------------------------------------------------------------
@@ -1036,6 +1049,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     if (p.tma_out && threadIdx.x == 64 && !*abort_flag) tma_store_wait_read();
     SB_TLOG(threadIdx.x == 0, 5, clock64());   // epilogue done
     SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
+    SB_TRACE_END(2);
     if (*abort_flag) {
         // give copies that may still be in flight time to land before shared memory is released
         const uint64_t t0 = globaltimer_ns();
@@ -1102,6 +1116,7 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
     unsigned long long* tlog = (p.timing != nullptr && blockIdx.x < 1024) ? p.timing + 16ull * blockIdx.x : nullptr;
 #endif
     SB_TLOG(threadIdx.x == 0, 0, globaltimer_ns());
+    SB_TRACE_BEGIN();
     SB_TLOG(threadIdx.x == 0, 6, clock64());
     const int m_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
     const int n_tiles_total = m_tiles * p.tiles_per_shard;       // (tiles_per_shard = N tiles; conv layers have one shard)
@@ -1318,6 +1333,7 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
     __syncthreads();
     SB_TLOG(threadIdx.x == 0, 5, clock64());
     SB_TLOG(threadIdx.x == 0, 7, globaltimer_ns());
+    SB_TRACE_END(3);
     if (*abort_flag) {
         const uint64_t t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 200000ull) { }
@@ -1910,7 +1926,9 @@ static const OpBlock* blk(const UmmaOp& op) { return (const OpBlock*)op.blob; }
 
 #ifdef SB_CTA_TIMING
 static unsigned long long* g_timing = nullptr;   // development builds only: set through umma_set_timing_buffer
+static unsigned long long* g_trace = nullptr;
 void umma_set_timing_buffer(void* dev_ptr) { g_timing = (unsigned long long*)dev_ptr; }
+void umma_set_trace_buffer(void* dev_ptr) { g_trace = (unsigned long long*)dev_ptr; }
 #endif
 
 static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr)
@@ -1927,6 +1945,7 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     }
 #ifdef SB_CTA_TIMING
     pp.timing = g_timing;
+    pp.trace = g_trace;
     {
         static const int only_mode = (int)tune("SB_TLOG_MODE", -1);      // log only kernels of one mode (0 fwd, 1 dgrad, 2 wgrad)
         if (only_mode >= 0 && pp.mode != only_mode) pp.timing = nullptr;

@@ -90,6 +90,7 @@ cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cud
 // Development builds only: when set to a device buffer of 1024*16 uint64, every tensor-core CTA (first 1024 of a launch)
 // records clock stamps at its phase boundaries.
 void umma_set_timing_buffer(void* dev_ptr);
+void umma_set_trace_buffer(void* dev_ptr);
 #endif
 
 }  // namespace sb
