@@ -226,18 +226,38 @@ def run_ours(args):
     for _ in range(max(1, min(args.warmup, 3))):
         m.train_step_host(hx, hy, lr, MU)
 
-    def host_block():
+    def host_block(prefetch):
+        # `prefetch`: the input copies are started ahead (sb_prefetch_host, copy stream) and the iterations are launched without
+        # waiting (sb_train_step_host_async / _wait); every step still copies its inputs from pinned host memory and has its
+        # loss read back and collected on the host, all inside the timed region
         barrier()
         t0 = time.perf_counter()
-        for _ in range(args.steps):
-            m.train_step_host(hx, hy, lr, MU)
+        if prefetch:
+            # two iterations in flight: iteration i + 1 is launched before the loss of iteration i is collected, the inputs
+            # of iteration i + 2 are copied while i + 1 computes
+            n = args.steps
+            m.prefetch_host(hx, hy)
+            if n > 1:
+                m.prefetch_host(hx, hy)
+            m.train_step_host_async(hx, hy, lr, MU)
+            for i in range(1, n):
+                m.train_step_host_async(hx, hy, lr, MU)
+                m.train_step_host_wait()
+                if i + 1 < n:
+                    m.prefetch_host(hx, hy)
+            m.train_step_host_wait()
+        else:
+            for i in range(args.steps):
+                m.train_step_host(hx, hy, lr, MU)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) * 1e3
         barrier()
         return dt
 
-    e2e_blocks = [host_block() for _ in range(min(len(blocks), 50))]
+    host_block(True)
+    e2e_blocks = [host_block(True) for _ in range(min(len(blocks), 50))]
     ms_e2e = float(np.median(e2e_blocks))
+    ms_e2e_plain = float(np.median([host_block(False) for _ in range(min(len(blocks), 20))]))
 
     # Per-kernel-class timing: the kernels of the same fused step (sb_graph_step), enqueued eagerly on ONE stream with a pair of
     # CUDA events around every launch (the library's profiling mode), at most 50 steps.  Same kernels as the timed graph,
@@ -248,7 +268,7 @@ def run_ours(args):
         step()
     prof = m.profile_end()
 
-    ms, ms_e2e = max_over_ranks([ms, ms_e2e], world, "cuda")
+    ms, ms_e2e, ms_e2e_plain = max_over_ranks([ms, ms_e2e, ms_e2e_plain], world, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -299,7 +319,13 @@ def run_ours(args):
                    "l2": f"per-step working set (activations + gradients + parameters: arena of {m.arena_bytes / 1e6:.0f} MB) exceeds the 126 MB L2; no flush",
                    "parallelism": "1 GPU: R logical replicas x K logical shards" if world == 1 else f"{world} independent replicas of the 1-GPU job"},
         "e2e": {"value": imgs / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": int(hx.numel() * 2 + hy.numel() * 4), "d2h_bytes_per_step": 8},
+                "h2d_bytes_per_step": int(hx.numel() * 2 + hy.numel() * 4), "d2h_bytes_per_step": 8,
+                "path": "sb_prefetch_host (inputs copied from pinned host memory one to two iterations ahead, on a copy stream) + "
+                        "sb_train_step_host_async / sb_train_step_host_wait (one CUDA graph per iteration: the iteration and the loss / status "
+                        "read-back into pinned memory; two iterations in flight, every loss collected on the host); wall clock over `steps` "
+                        "steps, median block",
+                "value_synchronous": imgs / (ms_e2e_plain / args.steps * 1e-3),
+                "synchronous_path": "sb_train_step_host: copies, iteration, read-back and a stream synchronise per call"},
         "gpu_launches": int(launches * args.steps),
         "repeats": len(blocks), "block_ms_min": float(min(blocks)), "block_ms_max": float(max(blocks)),
         "value_path": "median of `repeats` blocks of `steps` CUDA-graph replays of sb_graph_step (backward on several streams inside the graph), CUDA events",

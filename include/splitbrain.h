@@ -219,6 +219,34 @@ sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* hos
                              float lr, float momentum, void* stream, float* host_loss);
 
 /*
+ * Input prefetch for sb_train_step_host: starts the host->device copy of a LATER iteration's inputs into the second of
+ * two staging areas inside the arena, on a copy stream of the library's own, and returns at once, so that the copy runs
+ * while the current iteration computes.  Staged batches (two at most) are consumed in order: the next
+ * sb_train_step_host / sb_train_step_host_async call must name the same host_x / host_labels, waits for the staged copy on the device instead of
+ * copying, and is otherwise the same call (same result bits).  The host buffers must stay unchanged until that call
+ * returns; pinned host memory makes the copy asynchronous.
+ *   host_x, host_labels : HOST, as for sb_train_step_host.
+ * Errors: SB_ERR_STATE with two batches already staged; sb_train_step_host returns SB_ERR_STATE when a batch is
+ * staged and it is called with other host buffers.
+ */
+sb_status sb_prefetch_host(sb_model* m, const void* host_x, const int32_t* host_labels);
+
+/*
+ * sb_train_step_host without the wait: launches the iteration on `stream` and returns; sb_train_step_host_wait
+ * blocks until the OLDEST launched iteration has finished and returns its loss (and SB_ERR_TIMEOUT if one of its kernels
+ * gave up on a bounded wait).  Two iterations may be in flight, so that the host's launch and wake-up latency and the
+ * read-back of one iteration hide behind the next one.  The iteration must have been staged by sb_prefetch_host (one
+ * staging area and one pair of pinned result words per iteration in flight); without a staged batch, on the first
+ * call of a model and in the diagnostic modes the call runs the iteration to completion itself and the wait returns
+ * its result at once.  Iterations run in launch order on `stream`; results equal those of sb_train_step_host bit
+ * for bit.
+ * Errors: SB_ERR_STATE with two iterations in flight, with none to wait for, when a staged batch's host buffers are
+ * not the ones named, and when sb_train_step_host is called while iterations are in flight.
+ */
+sb_status sb_train_step_host_async(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum, void* stream);
+sb_status sb_train_step_host_wait(sb_model* m, void* stream, float* host_loss);
+
+/*
  * Introspection for parity tests and checkpointing: a borrowed DEVICE pointer to one tensor.
  *   what  : SB_T_*;  layer : index into the layer list;
  *   part  : replica r for conv-side activations, shard j for FC parameters.

@@ -80,6 +80,9 @@ def _load():
         "sb_sgd_step": [c_void_p, c_float, c_float, c_void_p],
         "sb_loss": [c_void_p, c_void_p, P(c_float)],
         "sb_train_step_host": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p, P(c_float)],
+        "sb_prefetch_host": [c_void_p, c_void_p, c_void_p],
+        "sb_train_step_host_async": [c_void_p, c_void_p, c_void_p, c_float, c_float, c_void_p],
+        "sb_train_step_host_wait": [c_void_p, c_void_p, P(c_float)],
         "sb_tensor": [c_void_p, c_int32, c_int32, c_int32, P(c_void_p), P(c_int64), P(c_int32)],
         "sb_tensor_read": [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_size_t],
         "sb_tensor_write": [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_size_t],
@@ -124,6 +127,9 @@ sb_debug_check_guards = _lib.sb_debug_check_guards
 sb_sgd_step = _lib.sb_sgd_step
 sb_loss = _lib.sb_loss
 sb_train_step_host = _lib.sb_train_step_host
+sb_prefetch_host = _lib.sb_prefetch_host
+sb_train_step_host_async = _lib.sb_train_step_host_async
+sb_train_step_host_wait = _lib.sb_train_step_host_wait
 sb_tensor = _lib.sb_tensor
 sb_tensor_read = _lib.sb_tensor_read
 sb_tensor_write = _lib.sb_tensor_write
@@ -308,6 +314,24 @@ class Model:
         px = host_x.data_ptr() if hasattr(host_x, "data_ptr") else host_x.ctypes.data
         pl = host_labels.data_ptr() if hasattr(host_labels, "data_ptr") else host_labels.ctypes.data
         _check(sb_train_step_host(self.h, c_void_p(px), c_void_p(pl), c_float(lr), c_float(momentum), self._stream(), byref(v)))
+        return v.value
+
+    def prefetch_host(self, host_x, host_labels):
+        """Start the host->device copy of a later iteration's inputs (consumed by the next train_step_host on the same buffers)."""
+        px = host_x.data_ptr() if hasattr(host_x, "data_ptr") else host_x.ctypes.data
+        pl = host_labels.data_ptr() if hasattr(host_labels, "data_ptr") else host_labels.ctypes.data
+        _check(sb_prefetch_host(self.h, c_void_p(px), c_void_p(pl)))
+
+    def train_step_host_async(self, host_x, host_labels, lr, momentum):
+        """Launch an iteration on a staged batch without waiting; collect its loss with train_step_host_wait()."""
+        px = host_x.data_ptr() if hasattr(host_x, "data_ptr") else host_x.ctypes.data
+        pl = host_labels.data_ptr() if hasattr(host_labels, "data_ptr") else host_labels.ctypes.data
+        _check(sb_train_step_host_async(self.h, c_void_p(px), c_void_p(pl), c_float(lr), c_float(momentum), self._stream()))
+
+    def train_step_host_wait(self) -> float:
+        """Loss of the oldest iteration in flight (blocks until it has finished)."""
+        v = c_float()
+        _check(sb_train_step_host_wait(self.h, self._stream(), byref(v)))
         return v.value
 
     def forward_layers(self, first, last, xs=None, labels=None):

@@ -105,6 +105,23 @@ struct sb_model {
     struct { bool on = false; float lr = 0.f, mu = 0.f; cudaEvent_t ev = nullptr; bool waited = false; size_t covered = 0; } fuse;
     char* stage_x = nullptr;
     int32_t* stage_labels = nullptr;
+    // Input prefetch (sb_prefetch_host): a second staging area, so that the copy of the next iteration's inputs runs on a
+    // copy stream while the current iteration computes.  Staged batches are consumed in order by sb_train_step_host.
+    char* stage_xb[2] = {nullptr, nullptr};          // [0] = stage_x
+    int32_t* stage_lb[2] = {nullptr, nullptr};       // [0] = stage_labels
+    struct Staged { const void* host_x; const void* host_labels; int buf; };
+    Staged staged[2];
+    int n_staged = 0, stage_next = 0;
+    cudaStream_t cpstream = nullptr;
+    cudaEvent_t ev_staged[2] = {nullptr, nullptr};
+    // Iterations in flight (sb_train_step_host_async): at most one per staging area; each writes its loss and the device
+    // status word into its own pair of words of a small pinned host buffer and records ev_done[area].
+    struct Flight { int slot; bool finished; float loss; sb_status status; char msg[160]; };
+    Flight flights[2];
+    int n_flights = 0;
+    bool slot_busy[2] = {false, false};
+    cudaEvent_t ev_done[2] = {nullptr, nullptr};
+    uint32_t* host_res = nullptr;      // pinned host memory: [3][2] words (areas 0, 1; 2 = the call that copies its inputs itself)
     char* input_grad = nullptr;
     PtrTab x_tab{}, label_tab{};
     bool have_x = false, have_labels = false, have_fwd = false;
@@ -128,12 +145,12 @@ struct sb_model {
         bool warmed = false;
     };
     StepGraph g_dev, g_host, g_mod;
+    StepGraph g_pre[2];      // sb_train_step_host on inputs staged by sb_prefetch_host: one graph per staging area
     // Debug aids that stand in for a memory checker: every arena region is followed by a 256-byte guard holding a fixed
     // pattern (sb_debug_check_guards), and the regions a step overwrites are listed so that they can be filled with NaN
     // bit patterns before a step (sb_debug_poison).
     struct Region { size_t off, bytes; bool scratch; };
     std::vector<Region> regions;
-    uint32_t host_result[2] = {0, 0};   // loss bits and device status word written by the host-step graph
     // per-launch event recording (sb_profile_begin / sb_profile_end)
     struct Rec { const char* tag; cudaEvent_t e0, e1; double flops, bytes; int layer; };
     int cur_layer = -1;   // layer whose kernels are being enqueued (profiling detail)
@@ -164,6 +181,13 @@ struct sb_model {
         if (g_dev.exec) cudaGraphExecDestroy(g_dev.exec);
         if (g_host.exec) cudaGraphExecDestroy(g_host.exec);
         if (g_mod.exec) cudaGraphExecDestroy(g_mod.exec);
+        for (int k = 0; k < 2; ++k) {
+            if (g_pre[k].exec) cudaGraphExecDestroy(g_pre[k].exec);
+            if (ev_staged[k]) cudaEventDestroy(ev_staged[k]);
+            if (ev_done[k]) cudaEventDestroy(ev_done[k]);
+        }
+        if (host_res) cudaFreeHost(host_res);
+        if (cpstream) cudaStreamDestroy(cpstream);
     }
 };
 
@@ -317,6 +341,9 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     m->status = (uint32_t*)take(256);
     m->stage_x = take(B * m->in_per_img * m->esz);
     m->stage_labels = (int32_t*)take(B * 4);
+    m->stage_xb[0] = m->stage_x; m->stage_lb[0] = m->stage_labels;
+    m->stage_xb[1] = take(B * m->in_per_img * m->esz);
+    m->stage_lb[1] = (int32_t*)take(B * 4);
     m->input_grad = (cfg->flags & SB_FLAG_INPUT_GRAD) ? take(B * m->in_per_img * m->esz) : nullptr;
     if (cfg->flags & SB_FLAG_MODULO_SCHEDULE) {
         if (m->first_fc == 0) return fail(SB_ERR_UNSUPPORTED, "the modulo schedule needs a conv-side stack below the FC stack");
@@ -419,6 +446,7 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
                     contiguous = contiguous && (const char*)m->x_tab.p[r] == (const char*)m->x_tab.p[0] + (size_t)r * rep_bytes;
                 const void* src = m->x_tab.p[0];
                 if (!contiguous) {
+                    if (m->n_staged > 0) return fail(SB_ERR_STATE, "a batch staged by sb_prefetch_host occupies the staging area: consume it first");
                     for (int r = 0; r < m->cfg.R; ++r)
                         if (m->x_tab.p[r] != m->stage_x + (size_t)r * rep_bytes)
                             CU_TRY(cudaMemcpyAsync(m->stage_x + (size_t)r * rep_bytes, m->x_tab.p[r], rep_bytes, cudaMemcpyDeviceToDevice, st));
@@ -1189,63 +1217,177 @@ sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const
     return s;
 }
 
-sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum,
-                             void* stream, float* host_loss)
+namespace {
+// pinned result words, the copy stream and its events: host-side objects made on first use (no device memory)
+sb_status host_step_objects(sb_model* m)
 {
-    if (!m || !host_x || !host_labels || !host_loss) return fail(SB_ERR_INVALID_ARG, "null argument");
-    cudaStream_t st = (cudaStream_t)stream;
-    const size_t xb = (size_t)m->B * m->in_per_img * m->esz;
-    const void* xp[MAX_PARTS];
-    const int32_t* lp[MAX_PARTS];
-    const int b = m->cfg.batch_per_replica;
-    for (int r = 0; r < m->cfg.R; ++r) {
-        xp[r] = m->stage_x + (size_t)r * b * m->in_per_img * m->esz;
-        lp[r] = m->stage_labels + (size_t)r * b;
+    if (m->host_res) return SB_OK;
+    CU_TRY(cudaHostAlloc((void**)&m->host_res, 6 * sizeof(uint32_t), cudaHostAllocDefault));
+    memset(m->host_res, 0, 6 * sizeof(uint32_t));
+    CU_TRY(cudaStreamCreateWithFlags(&m->cpstream, cudaStreamNonBlocking));
+    for (int k = 0; k < 2; ++k) {
+        CU_TRY(cudaEventCreateWithFlags(&m->ev_staged[k], cudaEventDisableTiming));
+        CU_TRY(cudaEventCreateWithFlags(&m->ev_done[k], cudaEventDisableTiming));
     }
-    sb_model::StepGraph& G = m->g_host;
-    const bool eager = m->profiling || m->debug_sync || !G.warmed || st == nullptr;
-    if (eager) {
-        CU_TRY(cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st));
-        CU_TRY(cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st));
-        sb_status s = whole_step(m, xp, lp, lr, momentum, stream);
-        if (s != SB_OK) return s;
-        G.warmed = true;
-        return sb_loss(m, stream, host_loss);
-    }
-    // One graph per (host buffers, lr, momentum): H2D copies, the whole iteration, and the loss / status read-back.
-    const bool hit = G.exec && G.host_x == host_x && G.host_labels == (const void*)host_labels && G.lr == lr && G.mu == momentum;
-    if (!hit) {
-        if (G.exec) { cudaGraphExecDestroy(G.exec); G.exec = nullptr; }
-        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        cudaError_t e = cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st);
-        sb_status s = e == cudaSuccess ? SB_OK : fail(SB_ERR_CUDA, "capturing the input copies: %s", cudaGetErrorString(e));
-        if (s == SB_OK) s = whole_step(m, xp, lp, lr, momentum, stream);
-        if (s == SB_OK) {
-            e = cudaMemcpyAsync(&m->host_result[0], m->loss, 4, cudaMemcpyDeviceToHost, st);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(&m->host_result[1], m->status, 4, cudaMemcpyDeviceToHost, st);
-            if (e != cudaSuccess) s = fail(SB_ERR_CUDA, "capturing the read-back: %s", cudaGetErrorString(e));
-        }
-        if (s != SB_OK) { abandon_capture(st); return s; }
-        cudaGraph_t graph = nullptr;
-        CU_TRY(cudaStreamEndCapture(st, &graph));
-        e = cudaGraphInstantiate(&G.exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) { G.exec = nullptr; return fail(SB_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e)); }
-        G.host_x = host_x; G.host_labels = host_labels; G.lr = lr; G.mu = momentum;
-    }
-    CU_TRY(cudaGraphLaunch(G.exec, st));
-    CU_TRY(cudaStreamSynchronize(st));
-    m->have_fwd = true;
+    return SB_OK;
+}
+sb_status read_result(sb_model* m, int slot, cudaStream_t st, float* host_loss)
+{
     uint32_t status_word;
-    memcpy(host_loss, &m->host_result[0], 4);
-    memcpy(&status_word, &m->host_result[1], 4);
+    memcpy(host_loss, &m->host_res[2 * slot], 4);
+    memcpy(&status_word, &m->host_res[2 * slot + 1], 4);
     if (status_word != DEV_OK) {
         cudaMemsetAsync(m->status, 0, 4, st);
         cudaStreamSynchronize(st);
         return fail(SB_ERR_TIMEOUT, "a kernel gave up on a bounded wait (device status %u)", status_word);
     }
     return SB_OK;
+}
+}  // namespace
+
+sb_status sb_prefetch_host(sb_model* m, const void* host_x, const int32_t* host_labels)
+{
+    if (!m || !host_x || !host_labels) return fail(SB_ERR_INVALID_ARG, "null argument");
+    if (m->n_staged >= 2) return fail(SB_ERR_STATE, "two batches are staged already: consume one with sb_train_step_host first");
+    sb_status hs = host_step_objects(m);
+    if (hs != SB_OK) return hs;
+    // The staging area chosen here is free on the host's side (the iteration that last read it has been launched); on the
+    // device the copy waits for that iteration to finish.
+    const int buf = m->stage_next;
+    const size_t xb = (size_t)m->B * m->in_per_img * m->esz;
+    CU_TRY(cudaStreamWaitEvent(m->cpstream, m->ev_done[buf], 0));      // (an event never recorded counts as complete)
+    CU_TRY(cudaMemcpyAsync(m->stage_xb[buf], host_x, xb, cudaMemcpyHostToDevice, m->cpstream));
+    CU_TRY(cudaMemcpyAsync(m->stage_lb[buf], host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, m->cpstream));
+    CU_TRY(cudaEventRecord(m->ev_staged[buf], m->cpstream));
+    m->staged[m->n_staged++] = sb_model::Staged{host_x, (const void*)host_labels, buf};
+    m->stage_next = buf ^ 1;
+    return SB_OK;
+}
+
+// Launches one iteration from host buffers.  wait = true: synchronises and returns the loss (sb_train_step_host);
+// wait = false: returns after the launch and appends the iteration to the flights (sb_train_step_host_async).
+static sb_status host_step(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum, void* stream, bool wait,
+                           float* host_loss)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    sb_status hs = host_step_objects(m);
+    if (hs != SB_OK) return hs;
+    const size_t xb = (size_t)m->B * m->in_per_img * m->esz;
+    // a batch staged by sb_prefetch_host is consumed by the next call, which must name the same host buffers
+    const bool pre = m->n_staged > 0;
+    int buf = 0;
+    if (pre) {
+        if (m->staged[0].host_x != host_x || m->staged[0].host_labels != (const void*)host_labels)
+            return fail(SB_ERR_STATE, "a batch staged by sb_prefetch_host is pending: the next sb_train_step_host must name its host buffers");
+        buf = m->staged[0].buf;
+        if (m->slot_busy[buf]) return fail(SB_ERR_STATE, "the iteration that used this staging area has not been collected (sb_train_step_host_wait)");
+        m->staged[0] = m->staged[1];
+        --m->n_staged;
+        CU_TRY(cudaStreamWaitEvent(st, m->ev_staged[buf], 0));
+    } else {
+        if (m->n_flights > 0) return fail(SB_ERR_STATE, "iterations are in flight: only staged batches may be launched behind them");
+        m->stage_next = 1;      // (this call copies into staging area 0 itself: the next prefetch goes to area 1)
+    }
+    const int slot = pre ? buf : 2;
+    const void* xp[MAX_PARTS];
+    const int32_t* lp[MAX_PARTS];
+    const int b = m->cfg.batch_per_replica;
+    for (int r = 0; r < m->cfg.R; ++r) {
+        xp[r] = m->stage_xb[buf] + (size_t)r * b * m->in_per_img * m->esz;
+        lp[r] = m->stage_lb[buf] + (size_t)r * b;
+    }
+    sb_model::StepGraph& G = pre ? m->g_pre[buf] : m->g_host;
+    const bool eager = m->profiling || m->debug_sync || !m->g_host.warmed || st == nullptr;
+    sb_status s = SB_OK;
+    bool finished = false;
+    float loss = 0.f;
+    if (eager) {
+        if (!pre) {
+            CU_TRY(cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st));
+            CU_TRY(cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st));
+        }
+        s = whole_step(m, xp, lp, lr, momentum, stream);
+        if (s != SB_OK) return s;
+        m->g_host.warmed = true;
+        if (pre) CU_TRY(cudaEventRecord(m->ev_done[buf], st));
+        s = sb_loss(m, stream, &loss);       // (synchronises: the direct path is the first call and the diagnostic modes)
+        finished = true;
+    } else {
+        // One graph per (host buffers, lr, momentum): H2D copies (unless staged beforehand), the whole iteration, and the
+        // loss / status read-back.  A staged batch has one graph per staging area, keyed by lr and momentum only.
+        const bool hit = G.exec && (pre || (G.host_x == host_x && G.host_labels == (const void*)host_labels)) && G.lr == lr && G.mu == momentum;
+        if (!hit) {
+            if (G.exec) { cudaGraphExecDestroy(G.exec); G.exec = nullptr; }
+            CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+            cudaError_t e = cudaSuccess;
+            if (!pre) {
+                e = cudaMemcpyAsync(m->stage_x, host_x, xb, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(m->stage_labels, host_labels, (size_t)m->B * 4, cudaMemcpyHostToDevice, st);
+            }
+            s = e == cudaSuccess ? SB_OK : fail(SB_ERR_CUDA, "capturing the input copies: %s", cudaGetErrorString(e));
+            if (s == SB_OK) s = whole_step(m, xp, lp, lr, momentum, stream);
+            if (s == SB_OK) {
+                e = cudaMemcpyAsync(&m->host_res[2 * slot], m->loss, 4, cudaMemcpyDeviceToHost, st);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(&m->host_res[2 * slot + 1], m->status, 4, cudaMemcpyDeviceToHost, st);
+                if (e != cudaSuccess) s = fail(SB_ERR_CUDA, "capturing the read-back: %s", cudaGetErrorString(e));
+            }
+            if (s != SB_OK) { abandon_capture(st); return s; }
+            cudaGraph_t graph = nullptr;
+            CU_TRY(cudaStreamEndCapture(st, &graph));
+            e = cudaGraphInstantiate(&G.exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) { G.exec = nullptr; return fail(SB_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e)); }
+            G.host_x = host_x; G.host_labels = host_labels; G.lr = lr; G.mu = momentum;
+        }
+        CU_TRY(cudaGraphLaunch(G.exec, st));
+        if (pre) CU_TRY(cudaEventRecord(m->ev_done[buf], st));
+        m->have_fwd = true;
+        if (wait || !pre) {
+            CU_TRY(cudaStreamSynchronize(st));
+            s = read_result(m, slot, st, &loss);
+            finished = true;
+        }
+    }
+    if (wait) {
+        if (host_loss) *host_loss = loss;
+        return s;
+    }
+    sb_model::Flight& f = m->flights[m->n_flights++];
+    f.slot = slot; f.finished = finished; f.loss = loss; f.status = s;
+    snprintf(f.msg, sizeof(f.msg), "%s", finished && s != SB_OK ? sb_last_error() : "");
+    if (!finished) m->slot_busy[slot] = true;
+    return SB_OK;
+}
+
+sb_status sb_train_step_host(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum,
+                             void* stream, float* host_loss)
+{
+    if (!m || !host_x || !host_labels || !host_loss) return fail(SB_ERR_INVALID_ARG, "null argument");
+    if (m->n_flights > 0) return fail(SB_ERR_STATE, "iterations are in flight: collect them with sb_train_step_host_wait first");
+    return host_step(m, host_x, host_labels, lr, momentum, stream, true, host_loss);
+}
+
+sb_status sb_train_step_host_async(sb_model* m, const void* host_x, const int32_t* host_labels, float lr, float momentum, void* stream)
+{
+    if (!m || !host_x || !host_labels) return fail(SB_ERR_INVALID_ARG, "null argument");
+    if (m->n_flights >= 2) return fail(SB_ERR_STATE, "two iterations are in flight: collect one with sb_train_step_host_wait first");
+    return host_step(m, host_x, host_labels, lr, momentum, stream, false, nullptr);
+}
+
+sb_status sb_train_step_host_wait(sb_model* m, void* stream, float* host_loss)
+{
+    if (!m || !host_loss) return fail(SB_ERR_INVALID_ARG, "null argument");
+    if (m->n_flights == 0) return fail(SB_ERR_STATE, "no iteration in flight");
+    sb_model::Flight f = m->flights[0];
+    m->flights[0] = m->flights[1];
+    --m->n_flights;
+    if (f.finished) {
+        *host_loss = f.loss;
+        return f.status == SB_OK ? SB_OK : fail(f.status, "%s", f.msg);
+    }
+    CU_TRY(cudaEventSynchronize(m->ev_done[f.slot]));
+    m->slot_busy[f.slot] = false;
+    return read_result(m, f.slot, (cudaStream_t)stream, host_loss);
 }
 
 sb_status sb_tensor(sb_model* m, int32_t what, int32_t layer, int32_t part, void** dev_ptr, int64_t shape[4], int32_t* dtype)

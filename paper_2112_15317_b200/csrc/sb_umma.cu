@@ -78,6 +78,7 @@ struct UmmaParams {
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
     int wg_sweep;         // WGRAD: the float tile leaves through shared memory in contiguous row segments (wgrad_sweep_epilogue)
+    int pdl_late;         // the kernel that depends on this one may start once every CTA has ISSUED ALL ITS OPERAND LOADS (not at once)
     // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
     // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
     uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
@@ -98,16 +99,19 @@ struct UmmaParams {
 // Per-CTA phase stamps: compiled in only with -DSB_CTA_TIMING (a development aid; the shipped kernels carry none).
 #ifdef SB_CTA_TIMING
 #define SB_TLOG(cond, slot, val) do { if (tlog && (cond)) tlog[slot] = (unsigned long long)(val); } while (0)
-#define SB_TRACE_BEGIN() const unsigned long long trace_t0 = globaltimer_ns()
+#define SB_TRACE_BEGIN() const unsigned long long trace_t0 = globaltimer_ns(); unsigned long long trace_a = 0, trace_b = 0, trace_c = 0
+#define SB_TRACE_STAMP(var) do { if (p.trace != nullptr && threadIdx.x == 0) var = globaltimer_ns(); } while (0)
 #define SB_TRACE_END(kind) do { if (p.trace != nullptr && threadIdx.x == 0) { \
         const unsigned long long ti_ = atomicAdd(p.trace, 1ull); \
-        if (ti_ < 60000ull) { unsigned long long* r_ = p.trace + 8 + 4 * ti_; unsigned smid_; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_)); \
+        if (ti_ < 40000ull) { unsigned long long* r_ = p.trace + 8 + 6 * ti_; unsigned smid_; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_)); \
             r_[0] = trace_t0; r_[1] = globaltimer_ns(); \
             r_[2] = (unsigned long long)smid_ | ((unsigned long long)(kind) << 16) | ((unsigned long long)p.mode << 24) | ((unsigned long long)(gridDim.x * gridDim.y * gridDim.z) << 32); \
-            r_[3] = (unsigned long long)(unsigned)p.total_chunks | ((unsigned long long)(unsigned)p.n_total << 32); } } } while (0)
+            r_[3] = (unsigned long long)(unsigned)p.total_chunks | ((unsigned long long)(unsigned)p.n_total << 32); \
+            r_[4] = ((trace_a - trace_t0) & 0xffffffffull) | (((trace_b - trace_t0) & 0xffffffffull) << 32); r_[5] = trace_c - trace_t0; } } } while (0)
 #else
 #define SB_TLOG(cond, slot, val) do { } while (0)
 #define SB_TRACE_BEGIN() do { } while (0)
+#define SB_TRACE_STAMP(var) do { } while (0)
 #define SB_TRACE_END(kind) do { } while (0)
 #endif
 
@@ -555,7 +559,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
         __syncwarp();
         pdl_wait();
-        pdl_trigger();
+        if (!p.pdl_late) pdl_trigger();
+        SB_TRACE_STAMP(trace_a);
         SB_TLOG(lane == 0, 9, clock64());    // predecessor kernel complete
         // The first ring-full of loads needs nothing but the barriers just initialised: start them now, so that
         // their latency overlaps the TMEM allocation and the rest of the set-up.
@@ -578,6 +583,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
+    SB_TRACE_STAMP(trace_b);
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
@@ -607,6 +613,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             it += nb;
         }
         if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        SB_TRACE_STAMP(trace_c);
+        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -891,7 +899,8 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         }
         __syncwarp();
         pdl_wait();
-        pdl_trigger();
+        if (!p.pdl_late) pdl_trigger();
+        SB_TRACE_STAMP(trace_a);
         prod_el = elect_one() ? 1u : 0u;
         for (int g = 0; g < preloaded; ++g) {
             issue_halo(prod_el);
@@ -913,6 +922,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
+    SB_TRACE_STAMP(trace_b);
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
@@ -945,6 +955,8 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             next_group();
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        SB_TRACE_STAMP(trace_c);
+        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -1150,12 +1162,14 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
         tmem_relinquish();
     }
     pdl_wait();          // every thread that touches global memory waits for the predecessor kernel
-    if (warp == 0) pdl_trigger();
+    SB_TRACE_STAMP(trace_a);
+    if (warp == 0 && !p.pdl_late) pdl_trigger();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     SB_TLOG(threadIdx.x == 0, 1, clock64());   // set-up done
+    SB_TRACE_STAMP(trace_b);
 
     if (warp == 0) {
         // =========================== TMA producer ===============================================
@@ -1205,6 +1219,8 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
             }
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        SB_TRACE_STAMP(trace_c);
+        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -1545,7 +1561,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     uint32_t prod_el = 0;
     if (warp == 0) {
         pdl_wait();
-        pdl_trigger();
+        if (!p.pdl_late) pdl_trigger();
         prod_el = elect_one() ? 1u : 0u;
         for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
     }
@@ -1585,6 +1601,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             it += nb;
         }
         if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
+        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         if (leader) {
@@ -1952,6 +1969,11 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     }
     pp.dbg_skip = (int)tune("SB_HALO_SKIP", 0);
 #endif
+    {
+        // bit 0: forward, bit 1: data gradient, bit 2: weight gradient kernels release their dependents late
+        static const int pdl_late = (int)tune("SB_PDL_LATE", 0);
+        pp.pdl_late = (pdl_late >> pp.mode) & 1;
+    }
     if (pp.mode != MODE_WGRAD) {
         pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
         pp.rcp_tiles_wh = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h));

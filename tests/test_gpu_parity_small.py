@@ -538,6 +538,76 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
     g1.close(); g2.close(); g3.close()
 
 
+def test_prefetched_host_batches_give_the_same_steps():
+    """sb_prefetch_host stages the inputs of later iterations on a copy stream (two staging areas); sb_train_step_host
+    (or its asynchronous form, two iterations in flight) then consumes them in order.  Six iterations over three DIFFERENT batches, prefetched one and two iterations ahead,
+    must give the same losses and weights, bit for bit, as the same iterations with the copies inside the call; a call
+    that names other host buffers while a batch is staged, and a third staged batch, are refused."""
+    import torch
+    b = sb()
+    wl = WORKLOADS["tensor_core"]()
+    params = si.make_params(wl, bias_std=0.1)
+    g1 = gpu_model(wl, params, b.SB_BF16)
+    g2 = gpu_model(wl, params, b.SB_BF16)
+    batches = []
+    for k in range(3):
+        x, y = si.make_batch(wl, seed=si.SEED_DATA + k)
+        batches.append((torch.from_numpy(x).to(torch.bfloat16).pin_memory(), torch.from_numpy(y).pin_memory()))
+    order = [0, 1, 2, 0, 1, 2]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        plain = [g1.train_step_host(*batches[k], 0.02, 0.9) for k in order]
+        got = []
+        g2.prefetch_host(*batches[order[0]])
+        g2.prefetch_host(*batches[order[1]])                       # two iterations ahead
+        with pytest.raises(b.SBError, match="two batches are staged"):
+            g2.prefetch_host(*batches[order[2]])
+        with pytest.raises(b.SBError, match="must name its host buffers"):
+            g2.train_step_host(*batches[2], 0.02, 0.9)
+        for i, k in enumerate(order):
+            got.append(g2.train_step_host(*batches[k], 0.02, 0.9))
+            if i + 2 < len(order):
+                g2.prefetch_host(*batches[order[i + 2]])           # refill: always one or two batches ahead
+        side.synchronize()
+    assert got == plain, (got, plain)
+    assert len(set(plain)) > 3                                      # (the batches differ: so do the losses)
+    for a, c in zip(g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), g2.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    # with nothing staged the plain call works again on the same model
+    with torch.cuda.stream(side):
+        l1 = g1.train_step_host(*batches[1], 0.02, 0.9)
+        l2 = g2.train_step_host(*batches[1], 0.02, 0.9)
+        side.synchronize()
+    assert l1 == l2
+    # two iterations in flight: launch i + 1 before collecting i; same losses and weights again
+    with torch.cuda.stream(side):
+        plain = [g1.train_step_host(*batches[k], 0.02, 0.9) for k in order]
+        got = []
+        with pytest.raises(b.SBError, match="no iteration in flight"):
+            g2.train_step_host_wait()
+        g2.prefetch_host(*batches[order[0]])
+        g2.prefetch_host(*batches[order[1]])
+        g2.train_step_host_async(*batches[order[0]], 0.02, 0.9)
+        for i in range(1, len(order)):
+            g2.train_step_host_async(*batches[order[i]], 0.02, 0.9)
+            if i == 1:
+                with pytest.raises(b.SBError, match="two iterations are in flight"):
+                    g2.train_step_host_async(*batches[order[i]], 0.02, 0.9)
+                with pytest.raises(b.SBError, match="in flight"):
+                    g2.train_step_host(*batches[order[i]], 0.02, 0.9)
+            got.append(g2.train_step_host_wait())
+            if i + 1 < len(order):
+                g2.prefetch_host(*batches[order[i + 1]])
+        got.append(g2.train_step_host_wait())
+        side.synchronize()
+    assert got == plain, (got, plain)
+    for a, c in zip(g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), g2.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    g1.close(); g2.close()
+
+
 @pytest.mark.parametrize("net", ["tensor_core", "pair", "cfg1_b4"])
 def test_pool_written_by_the_conv_kernel_equals_the_pooling_kernel(net):
     """A conv layer followed by a 2x2 max-pool writes the pool layer's output and argmax bytes from its own staged
