@@ -956,6 +956,16 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
     return SB_OK;
 }
 
+// The weight-side work of layer i (weight / bias gradient, split reduces, folded update) on `wst`; classic = without the
+// programmatic-dependent-launch attribute.
+static sb_status weight_side(sb_model* m, int i, cudaStream_t wst, bool classic)
+{
+    pdl_classic() = classic ? 1 : 0;
+    const sb_status s = backward_layer(m, i, wst, SIDE_W);
+    pdl_classic() = 0;
+    return s;
+}
+
 // Backward pass; with `fuse_update` the SGD update of each layer's parameters is enqueued on the weight-side
 // stream as soon as that layer's gradients are complete and its input gradient (which reads the weights) has
 // been computed, so the bandwidth-bound update overlaps the rest of the backward pass.  Element for element the
@@ -976,6 +986,15 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
         Layer& l = m->L[i];
         const bool has_params = l.kind == SB_CONV3X3_RELU || l.kind == SB_FC_RELU || l.kind == SB_FC;
         if (two_streams && has_params) {
+            // Weight-side kernels of short reductions (FC layers, the 2x2 and 4x4 conv layers) are launched the classic way:
+            // launched early, their CTAs sit on SMs waiting for the stream's previous kernel while the input-gradient chain
+            // needs those SMs (batch 128 / 256 at CIFAR size: -1.9 % step, the 7-conv net -3.9 %; layers of 8192+ rows: +-0 to +1.9 %
+            // without the early launch, so those keep it; so does every layer of a step of long kernels -- ImageNet-size inputs:
+            // +0.6 to +1 % without).
+            static const long classic_max_rows = (long)tune("SB_WSIDE_CLASSIC_MAX_ROWS", 5000);
+            static const long classic_max_input = (long)tune("SB_WSIDE_CLASSIC_MAX_INPUT", 1L << 20);
+            const bool classic = (l.kind == SB_CONV3X3_RELU ? (long)m->B * l.H * l.W : (long)m->B) <= classic_max_rows &&
+                                 (long)m->B * m->cfg.H * m->cfg.W <= classic_max_input;
             cudaStream_t wst = m->wstreams[i % m->n_wstreams];
             used_streams |= 1u << (i % m->n_wstreams);
             CU_TRY(cudaEventRecord(m->ev_ready[i], st));
@@ -990,13 +1009,13 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
                 if (s != SB_OK) return s;
                 CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
                 m->fuse.on = true; m->fuse.lr = lr; m->fuse.mu = mu; m->fuse.ev = m->ev_dgrad[i]; m->fuse.waited = false; m->fuse.covered = 0;
-                s = backward_layer(m, i, wst, SIDE_W);
+                s = weight_side(m, i, wst, classic);
                 m->fuse.on = false;
                 if (s != SB_OK) return s;
                 if (m->fuse.covered == l.n_w + l.n_b) continue;     // every parameter of the layer has taken its update
                 if (m->fuse.covered != 0) return fail(SB_ERR_STATE, "layer %d: update folded into part of its reduces only", i);
             } else {
-                s = backward_layer(m, i, wst, SIDE_W);
+                s = weight_side(m, i, wst, classic);
                 if (s != SB_OK) return s;
                 s = backward_layer(m, i, st, SIDE_D);
                 if (s != SB_OK) return s;

@@ -38,10 +38,12 @@ inline double tune(const char* name, double dflt)
     return dflt;
 #endif
 }
+// (the calling thread can switch the attribute off for the launches it enqueues next: pdl_classic() = 1 ... = 0)
+inline int& pdl_classic() { static thread_local int off = 0; return off; }
 inline bool pdl_enabled()
 {
     static const bool on = [] { const char* e = getenv("SB_PDL"); return !(e && e[0] == '0'); }();
-    return on;
+    return on && !pdl_classic();
 }
 template <typename... KArgs, typename... Args>
 inline cudaError_t pdl_launch(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)

@@ -78,7 +78,6 @@ struct UmmaParams {
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
     int wg_sweep;         // WGRAD: the float tile leaves through shared memory in contiguous row segments (wgrad_sweep_epilogue)
-    int pdl_late;         // the kernel that depends on this one may start once every CTA has ISSUED ALL ITS OPERAND LOADS (not at once)
     // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
     // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
     uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
@@ -559,7 +558,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
         __syncwarp();
         pdl_wait();
-        if (!p.pdl_late) pdl_trigger();
+        pdl_trigger();
         SB_TRACE_STAMP(trace_a);
         SB_TLOG(lane == 0, 9, clock64());    // predecessor kernel complete
         // The first ring-full of loads needs nothing but the barriers just initialised: start them now, so that
@@ -614,7 +613,6 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
         if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
         SB_TRACE_STAMP(trace_c);
-        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -899,7 +897,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         }
         __syncwarp();
         pdl_wait();
-        if (!p.pdl_late) pdl_trigger();
+        pdl_trigger();
         SB_TRACE_STAMP(trace_a);
         prod_el = elect_one() ? 1u : 0u;
         for (int g = 0; g < preloaded; ++g) {
@@ -956,7 +954,6 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
         SB_TRACE_STAMP(trace_c);
-        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -1163,7 +1160,7 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
     }
     pdl_wait();          // every thread that touches global memory waits for the predecessor kernel
     SB_TRACE_STAMP(trace_a);
-    if (warp == 0 && !p.pdl_late) pdl_trigger();
+    if (warp == 0) pdl_trigger();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1220,7 +1217,6 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
         SB_TRACE_STAMP(trace_c);
-        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer =================================================
@@ -1561,7 +1557,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     uint32_t prod_el = 0;
     if (warp == 0) {
         pdl_wait();
-        if (!p.pdl_late) pdl_trigger();
+        pdl_trigger();
         prod_el = elect_one() ? 1u : 0u;
         for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
     }
@@ -1601,7 +1597,6 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             it += nb;
         }
         if (!got && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_TMA); }
-        if (p.pdl_late) pdl_trigger();
         __syncwarp();
     } else if (warp == 1) {
         if (leader) {
@@ -1969,11 +1964,6 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     }
     pp.dbg_skip = (int)tune("SB_HALO_SKIP", 0);
 #endif
-    {
-        // bit 0: forward, bit 1: data gradient, bit 2: weight gradient kernels release their dependents late
-        static const int pdl_late = (int)tune("SB_PDL_LATE", 0);
-        pp.pdl_late = (pdl_late >> pp.mode) & 1;
-    }
     if (pp.mode != MODE_WGRAD) {
         pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
         pp.rcp_tiles_wh = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h));
