@@ -150,7 +150,7 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;"
 // is two whole 256-byte runs.
 template <int BN>
 __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32_t taddr, uint8_t* stage, int row, int m0, int m_hi,
-                                                      int n0, int n_hi, size_t tile_off)
+                                                      int n0, int n_hi, size_t tile_off, int slab_mult = 1)
 {
     const int t128 = threadIdx.x - 64, q = t128 >> 5, lane = t128 & 31;
     const int hl = lane & 15, sub = lane >> 4;
@@ -179,7 +179,7 @@ __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32
                 float4 g;
                 asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(g.x), "=f"(g.y), "=f"(g.z), "=f"(g.w)
                              : "r"(stage_s + (uint32_t)rr * 256u + (((uint32_t)hl ^ (uint32_t)(rr & 7)) << 4)));
-                const size_t off = tile_off + (size_t)rr * p.ldc + c0 + 4 * hl;
+                const size_t off = tile_off + (size_t)rr * p.ldc + (size_t)(c0 * slab_mult) + 4 * hl;   // (slab_mult: 64-column slabs three taps apart)
                 *(float4*)((float*)p.out + off) = g;
             }
         }
@@ -494,6 +494,9 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     // WGRAD with at most 64 gradient rows left in this tile: the second 64-row box of A would be all padding, so it
     // is not fetched (accumulator rows 64.. then hold garbage that is never stored; MMA rows are independent)
     const int a_boxes = (MODE == MODE_WGRAD && m0 + 64 >= m_hi) ? 1 : 2;
+    // filter-column variant of the 64-input-channel weight gradient (BN = 192, hn_order): bytes between image rows of the
+    // activation box, and the box's size with its two halo rows
+    const uint32_t col_row_step = (uint32_t)(p.bw * p.bn) * 128u, col_box_bytes = (uint32_t)(p.bh + 2) * col_row_step;
     // (executed by the whole producer warp in lock-step: every value below is the same in all lanes, the lane with
     // el != 0 issues; ring slot and smem offset are carried in counters)
     int ld_s = 0;
@@ -501,10 +504,18 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(&full[0]);
     auto issue_loads = [&](uint32_t el) {
         const uint32_t sa = smem0 + ld_off, sb = sa + A_STAGE_BYTES, bar = full0 + 8u * (uint32_t)ld_s;
-        mbar_expect_tx_el(bar, (uint32_t)C::STAGE_BYTES - (a_boxes == 2 ? 0u : 8192u), el);
+        mbar_expect_tx_el(bar, (MODE == MODE_WGRAD && BN == 192 && p.hn_order ? (uint32_t)A_STAGE_BYTES + col_box_bytes : (uint32_t)C::STAGE_BYTES) -
+                                   (a_boxes == 2 ? 0u : 8192u), el);
         if (MODE == MODE_WGRAD) {
             // pixel chunk -> box origin; A = dy (two 64-channel boxes), B = shifted activations
             const int cw = ld_a * p.bw, ch = ld_b * p.bh, cn = ld_c * p.bn;
+            if (BN == 192 && p.hn_order) {
+                // one filter COLUMN: tensor maps with the dimensions listed as (c, w, n, h); one activation box with an image row
+                // of halo above and below serves the three taps (the three 64-column panels of B are windows into it, see below)
+                tma_load_4d_el(&mapA, sa, bar, m0, cw, cn, ch, el);
+                if (a_boxes == 2) tma_load_4d_el(&mapA, sa + 8192, bar, m0 + 64, cw, cn, ch, el);
+                tma_load_4d_el(&mapB, sb, bar, 0, cw + tap_fixed / 3 - 1, cn, ch - 1, el);
+            } else {
             tma_load_4d_el(&mapA, sa, bar, m0, cw, ch, cn, el);
             if (a_boxes == 2) tma_load_4d_el(&mapA, sa + 8192, bar, m0 + 64, cw, ch, cn, el);
             if (BN == 192) {
@@ -522,6 +533,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             } else {
 #pragma unroll
                 for (int j = 0; j < BN / 64; ++j) tma_load_4d_el(&mapB, sb + j * 8192, bar, n0 + 64 * j, cw + wg_ds, ch + wg_dr, cn, el);
+            }
             }
             if (++ld_a == p.tiles_w) { ld_a = 0; if (++ld_b == p.tiles_h) { ld_b = 0; ++ld_c; } }
         } else {
@@ -623,7 +635,10 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         const uint32_t sa0 = smem_u32(smem);
         // K-major: 16 elements = 32 bytes along the row; MN-major: 16 k-rows = 2048 bytes
         const uint64_t dA0 = (MODE == MODE_WGRAD) ? make_desc(sa0, 8192) : make_desc(sa0, 16);
-        const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(sa0 + A_STAGE_BYTES, 16) : make_desc(sa0 + A_STAGE_BYTES, 8192);
+        // (filter-column weight gradient: the three 64-column panels of B are the same activation box read one image row
+        // apart -- tap row r starts r * bw * bn rows into it, a whole number of 8-row swizzle groups)
+        const uint64_t dB0 = (MODE == MODE_FWD) ? make_desc(sa0 + A_STAGE_BYTES, 16)
+                                                : make_desc(sa0 + A_STAGE_BYTES, (MODE == MODE_WGRAD && BN == 192 && p.hn_order) ? col_row_step : 8192u);
         const uint32_t a_hi = (uint32_t)(dA0 >> 32), b_hi = (uint32_t)(dB0 >> 32);
         const uint32_t a_lo0 = (uint32_t)dA0, b_lo0 = (uint32_t)dB0;
         constexpr uint32_t A_STEP = ((MODE == MODE_WGRAD) ? 2048u : 32u) >> 4, B_STEP = ((MODE == MODE_FWD) ? 32u : 2048u) >> 4;
@@ -723,8 +738,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-                wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
-                                         (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0);
+                if (BN == 192 && p.hn_order)      // slab j = tap row j of filter column tap_fixed / 3: gradient columns (3 j + column) * Cin ..
+                    wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
+                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)(tap_fixed / 3) * p.w_cols, 3);
+                else
+                    wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
+                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0);
             }
         } else if (ok) {
             SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
@@ -1953,7 +1972,11 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
         const bool aligned = (pp.ldc & 3) == 0 && (pp.w_cols & 3) == 0 && (pp.n_total & 3) == 0 && (pp.split_stride & 3) == 0 &&
                              (((uintptr_t)pp.out) & 15) == 0;
         const long ring = (long)pp.stages * (A_STAGE_BYTES + b->bn * 128);
-        pp.wg_sweep = (sweep_on && aligned && ring >= 32768) ? 1 : 0;
+        pp.wg_sweep = ((sweep_on || pp.hn_order) && aligned && ring >= 32768) ? 1 : 0;
+        if (pp.hn_order && !pp.wg_sweep) {
+            snprintf(g_umma_err, sizeof(g_umma_err), "filter-column weight gradient planned without the staged epilogue");
+            return SB_ERR_CUDA;
+        }
     }
 #ifdef SB_CTA_TIMING
     pp.timing = g_timing;
@@ -2609,8 +2632,19 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 p.status = mv.status;
                 b->grid = dim3((unsigned)p.m_tiles_per_shard, (unsigned)g.wg_n_tiles, (unsigned)((9 + p.tap_group - 1) / p.tap_group * p.splits));
                 if ((size_t)p.splits * (lv.n_w + lv.n_b) > mv.ws_floats && p.splits > 1) return SB_ERR_ARENA_TOO_SMALL;
-                if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
-                if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch, g.cn)) return fail_plan();
+                // 64 input channels: one filter COLUMN per CTA instead of one filter row -- the three taps then share one
+                // activation box with a halo row above and below (the three N panels of the MMA are windows into it) instead
+                // of three boxes shifted in w.  Needs whole 8-row swizzle groups per image row of the box and the sweep epilogue.
+                static const bool col_on = tune("SB_WG_COLUMN", 1) != 0;
+                if (col_on && p.tap_group == 3 && !b->pair && (g.cw * g.cn) % 8 == 0 && (p.split_stride & 3) == 0 && (((uintptr_t)p.out) & 15) == 0 &&
+                    !(mv.cfg->flags & SB_FLAG_NO_HALO)) {
+                    p.hn_order = 1;
+                    if (!act_map_hn(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
+                    if (!act_map_hn(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch + 2, g.cn)) return fail_plan();
+                } else {
+                    if (!act_map(&um.wgrad.mapA, lv.dact, B, lv.H, lv.W, lv.Cout, g.cw, g.ch, g.cn)) return fail_plan();
+                    if (!act_map(&um.wgrad.mapB, lv.in_act, B, lv.H, lv.W, lv.Cin, g.cw, g.ch, g.cn)) return fail_plan();
+                }
                 um.wgrad.enabled = true;
             }
         } else if ((lv.kind == SB_FC_RELU || lv.kind == SB_FC) && fc_umma_ok(mv, lv, i)) {
