@@ -193,9 +193,10 @@ sb_status sb_modulo_step(sb_model* m, const void* const* x, const int32_t* const
  * removes the per-kernel launch cost that dominates at small batch sizes.  Different pointers or
  * hyper-parameters re-capture.  `stream` must not be the legacy default stream (NULL runs the passes directly).
  * Arguments as for sb_forward / sb_sgd_step.  Parameters, momentum, activations and loss are identical to the
- * three separate calls.  SB_T_GRAD_W / SB_T_GRAD_B of the conv layers are unspecified afterwards (here and after
+ * three separate calls.  SB_T_GRAD_W / SB_T_GRAD_B are unspecified afterwards (here and after
  * sb_modulo_step / sb_train_step_host): where a weight gradient is summed from split partial copies, the ordered
- * sum feeds the update directly and is not stored; use sb_backward to read gradients.
+ * sum feeds the update directly and is not stored, and the weight-gradient kernel of a large FC layer applies the
+ * update to its tile itself; use sb_backward to read gradients.
  */
 sb_status sb_graph_step(sb_model* m, const void* const* x, const int32_t* const* labels, float lr, float momentum,
                         void* stream);

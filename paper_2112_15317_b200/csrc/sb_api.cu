@@ -540,6 +540,13 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
             break;
         }
         if (!(part & SIDE_W)) {
+        } else if (l.um.wgrad.enabled && m->fuse.on && !(part & SIDE_D) && umma_fc_wgrad_can_update(m, i)) {
+            // fused pass: the update is applied by the weight-gradient kernel's epilogue (after the layer's input-gradient
+            // kernel, which reads the weights); the gradient itself is never stored
+            if (!m->fuse.waited) { CU_TRY(cudaStreamWaitEvent(st, m->fuse.ev, 0)); m->fuse.waited = true; }
+            U_TRY("fc_wgrad_umma", flops, act_bytes + (double)(l.n_w + l.n_b) * (m->bf16 ? 18.0 : 16.0), umma_fc_wgrad_update(m, i, m->fuse.lr, m->fuse.mu, st));
+            ++m->launches;
+            m->fuse.covered = l.n_w + l.n_b;
         } else if (l.um.wgrad.enabled) {
             U_TRY("fc_wgrad_umma", flops, act_bytes + (double)l.n_w * 4.0, umma_fc_wgrad(m, i, st));
             ++m->launches;
@@ -794,7 +801,7 @@ ModelView model_view(sb_model* m)
 {
     ModelView v{};
     v.cfg = &m->cfg; v.bf16 = m->bf16; v.B = m->B; v.n_layers = m->n_layers; v.first_fc = m->first_fc;
-    v.Wm = m->Wm; v.Gm = m->Gm; v.Sm = m->Sm; v.ws = m->ws; for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) v.ws_wk[k] = m->ws_wk[k]; v.ws_floats = m->ws_floats; v.n_wstreams = m->n_wstreams; v.status = m->status;
+    v.Wm = m->Wm; v.Gm = m->Gm; v.Vm = m->Vm; v.Sm = m->Sm; v.ws = m->ws; for (int k = 0; k < sb_model::MAX_WSTREAMS; ++k) v.ws_wk[k] = m->ws_wk[k]; v.ws_floats = m->ws_floats; v.n_wstreams = m->n_wstreams; v.status = m->status;
     v.input_grad = m->input_grad; v.x_tab = &m->x_tab; v.stage_x = m->stage_x;
     return v;
 }
@@ -1002,7 +1009,10 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
             // Conv layers in a fused pass: the input-gradient kernel is enqueued first and its event recorded, so that the
             // layer's split reduces on the weight stream can wait for it and apply the update themselves.
             static const bool reduce_updates = tune("SB_REDUCE_SGD", 1) != 0;
-            const bool in_reduce = fuse && reduce_updates && l.kind == SB_CONV3X3_RELU;
+            // FC layers whose weight-gradient kernel can carry the update take the same order (SB_FC_WGRAD_UPDATE=0: separate update)
+            static const bool fc_wgrad_update = tune("SB_FC_WGRAD_UPDATE", 1) != 0;
+            const bool in_reduce = fuse && ((reduce_updates && l.kind == SB_CONV3X3_RELU) ||
+                                            (fc_wgrad_update && l.kind != SB_CONV3X3_RELU && !l.narrow && umma_fc_wgrad_can_update(m, i)));
             sb_status s = SB_OK;
             if (in_reduce) {
                 s = backward_layer(m, i, st, SIDE_D);

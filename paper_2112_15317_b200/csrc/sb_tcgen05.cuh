@@ -72,6 +72,21 @@ __device__ __forceinline__ void tma_load_4d_el(const CUtensorMap* map, uint32_t 
         ::"r"(dst_saddr), "l"(map), "r"(bar_saddr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
         : "memory");
 }
+// Untiled bulk copy global -> shared memory, completion counted in bytes on an mbarrier.  Both addresses 16-byte aligned,
+// the size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_load(uint32_t dst_saddr, const void* src, uint32_t bytes, uint32_t bar_saddr)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_saddr), "l"(src), "r"(bytes), "r"(bar_saddr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar_saddr)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_saddr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar_saddr, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_saddr), "r"(bytes) : "memory");
+}
 // TMA store of one box from shared memory (bulk async-group completion) through a rank-4 tensor map (the rank of the
 // instruction must be the map's: every map of this library is encoded with four dimensions); elements beyond the
 // tensor are clipped.  Coordinates must not be negative, c0 * element size a multiple of 16 bytes.

@@ -78,6 +78,11 @@ struct UmmaParams {
     long bias_off;        // WGRAD: float offset of the bias-gradient vector inside one split buffer
     uint32_t* status;
     int wg_sweep;         // WGRAD: the float tile leaves through shared memory in contiguous row segments (wgrad_sweep_epilogue)
+    // WGRAD with the update folded in (sgd_w != nullptr): the sweep applies v <- mu v + g, w <- w - lr v to the parameters at
+    // the tile's offsets (same element offsets as in `out`) and refreshes their bf16 copy instead of storing g
+    float *sgd_w, *sgd_v;
+    __nv_bfloat16* sgd_s;
+    float sgd_lr, sgd_mu;
     // Reciprocals for the divisions on the CTAs' start-up and epilogue paths (filled by launch_op from the fields above):
     // q = n / d as __umulhi(n, mul) with mul = 2^32 / d + 1, exact while n * d < 2^32; mul = 0 stands for d = 1.
     uint32_t rcp_tiles_w, rcp_tiles_wh, rcp_bw, rcp_bwbh, rcp_wb, rcp_wbhb;   // (wb, hb = bw / 2, bh / 2: the pooled box)
@@ -185,6 +190,86 @@ __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32
         }
         epi_bar_sync();                                   // the slab may be overwritten
     }
+}
+
+// The same sweep with the SGD-momentum update folded in (FC layers in the fused step): instead of storing the gradient
+// tile, v <- mu v + g and w <- w - lr v are applied to the parameters at the tile's offsets and their bf16 copy is
+// refreshed -- the operations of the stand-alone update kernel in the same order, so the bits are the same, while the
+// float gradient is neither written nor read back (8 of 26 bytes per parameter).  The w and v rows of a 64-column slab
+// are fetched ahead by bulk copies (one 256-byte row of each per epilogue thread) into two slab buffers behind the
+// control block: slabs 0 and 1 are requested before the main loop starts, slab j + 2 when slab j has been swept, so a
+// CTA has 64 - 128 KB of parameter loads in flight while it multiplies, drains and sweeps.
+constexpr int UPD_SLAB_BYTES = 65536;                 // per slab buffer: w rows [128][256 B], then v rows [128][256 B]
+constexpr int UPD_EXTRA_SMEM = 2 * UPD_SLAB_BYTES;
+__device__ __forceinline__ void upd_request_slab(const UmmaParams& p, uint32_t buf_s, uint32_t bar_s, int row, bool row_ok, size_t row_off)
+{
+    if (row_ok) {
+        mbar_arrive_expect_tx(bar_s, 512u);
+        bulk_load(buf_s + (uint32_t)row * 256u, p.sgd_w + row_off, 256u, bar_s);
+        bulk_load(buf_s + 32768u + (uint32_t)row * 256u, p.sgd_v + row_off, 256u, bar_s);
+    } else {
+        mbar_arrive(bar_s);
+    }
+}
+template <int BN>
+__device__ __forceinline__ bool wgrad_sweep_update_epilogue(const UmmaParams& p, uint32_t taddr, uint8_t* stage, uint32_t slab_s, uint64_t* slab_bar,
+                                                             int row, int m0, int m_hi, int n0, int n_hi, size_t tile_off)
+{
+    const int t128 = threadIdx.x - 64, q = t128 >> 5, lane = t128 & 31;
+    const int hl = lane & 15, sub = lane >> 4;
+    const uint32_t stage_s = smem_u32(stage);
+    const bool row_ok = m0 + row < m_hi;
+    bool ok = true;
+#pragma unroll 1
+    for (int j = 0; j < BN / 64; ++j) {
+        const int c0 = 64 * j;
+        if (n0 + c0 >= n_hi) break;                       // (uniform)
+        const uint32_t buf_s = slab_s + (uint32_t)(j & 1) * (uint32_t)UPD_SLAB_BYTES;
+#pragma unroll
+        for (int cc = 0; cc < 64; cc += 16) {
+            uint32_t v[16];
+            tmem_ld16(taddr + c0 + cc, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t ch = (uint32_t)(cc / 4 + k);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_s + (uint32_t)row * 256u + ((ch ^ (uint32_t)(row & 7)) << 4)),
+                             "r"(v[4 * k]), "r"(v[4 * k + 1]), "r"(v[4 * k + 2]), "r"(v[4 * k + 3]) : "memory");
+            }
+        }
+        // the slab's parameter rows have landed (every thread waits: it reads other threads' rows)
+        if (ok) ok = mbar_wait(&slab_bar[j & 1], (uint32_t)((j >> 1) & 1));
+        epi_bar_sync();
+        if (ok) {
+#pragma unroll 4
+            for (int rr = q * 2 + sub; rr < 128; rr += 8) {
+                if (m0 + rr >= m_hi) break;
+                float4 g, w, v;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(g.x), "=f"(g.y), "=f"(g.z), "=f"(g.w)
+                             : "r"(stage_s + (uint32_t)rr * 256u + (((uint32_t)hl ^ (uint32_t)(rr & 7)) << 4)));
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w)
+                             : "r"(buf_s + (uint32_t)rr * 256u + ((uint32_t)hl << 4)));
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                             : "r"(buf_s + 32768u + (uint32_t)rr * 256u + ((uint32_t)hl << 4)));
+                v.x = fmaf(p.sgd_mu, v.x, g.x); v.y = fmaf(p.sgd_mu, v.y, g.y); v.z = fmaf(p.sgd_mu, v.z, g.z); v.w = fmaf(p.sgd_mu, v.w, g.w);
+                w.x = fmaf(-p.sgd_lr, v.x, w.x); w.y = fmaf(-p.sgd_lr, v.y, w.y); w.z = fmaf(-p.sgd_lr, v.z, w.z); w.w = fmaf(-p.sgd_lr, v.w, w.w);
+                const size_t off = tile_off + (size_t)rr * p.ldc + c0 + 4 * hl;
+                __stcs((float4*)(p.sgd_v + off), v);
+                __stcs((float4*)(p.sgd_w + off), w);
+                if (p.sgd_s != nullptr) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+                    uint2 pk;
+                    pk.x = *(uint32_t*)&lo;
+                    pk.y = *(uint32_t*)&hi;
+                    *(uint2*)(p.sgd_s + off) = pk;
+                }
+            }
+        }
+        epi_bar_sync();                                   // stage and slab buffer may be overwritten
+        if (ok && j + 2 < BN / 64 && n0 + c0 + 128 < n_hi)
+            upd_request_slab(p, buf_s, smem_u32(&slab_bar[j & 1]), row, row_ok, tile_off + (size_t)row * p.ldc + c0 + 128);
+    }
+    return ok;
 }
 
 // Epilogue of one accumulator row: reads BN columns of this warp's TMEM lane quadrant (16 at a time) and
@@ -424,7 +509,9 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     uint64_t* acc_full = empty + MAX_STAGES;          // [1]
     uint32_t* tmem_slot = (uint32_t*)(acc_full + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint64_t* slab_bar = (uint64_t*)(ctrl + 256);     // [2] WGRAD with the update folded in: parameter slabs landed
     float* s_bias = (float*)(ctrl + 512);             // [BN]
+    uint8_t* slab_buf = ctrl + CTRL_BYTES;            // ... and the two slab buffers (only allocated for such launches)
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const unsigned cta_lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
@@ -564,6 +651,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
             for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
             mbar_init(acc_full, 1);
+            if (MODE == MODE_WGRAD && p.sgd_w != nullptr) { mbar_init(&slab_bar[0], 128); mbar_init(&slab_bar[1], 128); }
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             SB_TLOG(true, 8, clock64());    // barriers initialised
@@ -696,6 +784,13 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (MODE == MODE_WGRAD) {
             row_ok = (m0 + row) < m_hi;
             row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
+            if (p.sgd_w != nullptr) {
+                // update folded in: this thread's w and v rows of the first two 64-column slabs are requested now
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    if (j < BN / 64 && n0 + 64 * j < n_hi)
+                        upd_request_slab(p, smem_u32(slab_buf) + (uint32_t)j * (uint32_t)UPD_SLAB_BYTES, smem_u32(&slab_bar[j]), row, row_ok, row_off + n0 + 64 * j);
+            }
         } else {
             const int r1 = fast_div(row, p.rcp_bw), ni = fast_div(row, p.rcp_bwbh);
             const int wi = row - r1 * p.bw, hi_ = r1 - ni * p.bh;
@@ -724,8 +819,17 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[s])) : "memory");
             }
-            if (ok && (m0 + row) < m_hi)
-                ((float*)p.out)[(size_t)split * p.split_stride + p.bias_off + m0 + row] = bsum;
+            if (ok && (m0 + row) < m_hi) {
+                const size_t bo = (size_t)split * p.split_stride + p.bias_off + m0 + row;
+                if (p.sgd_w != nullptr) {
+                    const float vb = fmaf(p.sgd_mu, p.sgd_v[bo], bsum), wb = fmaf(-p.sgd_lr, vb, p.sgd_w[bo]);
+                    p.sgd_v[bo] = vb;
+                    p.sgd_w[bo] = wb;
+                    if (p.sgd_s != nullptr) p.sgd_s[bo] = __float2bfloat16_rn(wb);
+                } else {
+                    ((float*)p.out)[bo] = bsum;
+                }
+            }
             if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         }
         if (lane == 0 && ok) ok = mbar_wait(acc_full, 0);
@@ -738,7 +842,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-                if (BN == 192 && p.hn_order)      // slab j = tap row j of filter column tap_fixed / 3: gradient columns (3 j + column) * Cin ..
+                if (p.sgd_w != nullptr) {
+                    if (!wgrad_sweep_update_epilogue<BN>(p, taddr, smem, smem_u32(slab_buf), slab_bar, row, m0, m_hi, n0, n_hi,
+                                                         (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0) && lane == 0) {
+                        *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI);
+                    }
+                } else if (BN == 192 && p.hn_order)      // slab j = tap row j of filter column tap_fixed / 3: gradient columns (3 j + column) * Cin ..
                     wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
                                              (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)(tap_fixed / 3) * p.w_cols, 3);
                 else
@@ -1821,12 +1930,15 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<MODE, BN>::smem_bytes(Cfg<MODE, BN>::MAX_STAGES_FIT));
+                                 MODE == MODE_WGRAD ? 227 * 1024 : Cfg<MODE, BN>::smem_bytes(Cfg<MODE, BN>::MAX_STAGES_FIT));
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     if (p.stages < 1 || p.stages > Cfg<MODE, BN>::MAX_STAGES_FIT) return cudaErrorInvalidValue;
-    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), (size_t)Cfg<MODE, BN>::smem_bytes(p.stages), st, op.mapA, op.mapB, op.mapC, p);
+    // (a weight gradient with the update folded in carries two parameter slab buffers behind its control block)
+    const size_t smem = (size_t)Cfg<MODE, BN>::smem_bytes(p.stages) + (MODE == MODE_WGRAD && p.sgd_w != nullptr ? (size_t)UPD_EXTRA_SMEM : 0);
+    if (smem > 227 * 1024) return cudaErrorInvalidValue;
+    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), smem, st, op.mapA, op.mapB, op.mapC, p);
 }
 
 template <int MODE, int BN>
@@ -1962,17 +2074,30 @@ void umma_set_timing_buffer(void* dev_ptr) { g_timing = (unsigned long long*)dev
 void umma_set_trace_buffer(void* dev_ptr) { g_trace = (unsigned long long*)dev_ptr; }
 #endif
 
-static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr)
+struct SgdFuse { float *w, *v; __nv_bfloat16* s; float lr, mu; };
+static bool wgrad_sweep_ok(const OpBlock* b)
+{
+    const UmmaParams& pp = b->p;
+    static const bool sweep_on = tune("SB_WGRAD_SWEEP", 1) != 0;
+    const bool aligned = (pp.ldc & 3) == 0 && (pp.w_cols & 3) == 0 && (pp.n_total & 3) == 0 && (pp.split_stride & 3) == 0 &&
+                         (((uintptr_t)pp.out) & 15) == 0;
+    const long ring = (long)pp.stages * (A_STAGE_BYTES + b->bn * 128);
+    return (sweep_on || pp.hn_order) && aligned && ring >= 32768;
+}
+static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches = nullptr, const SgdFuse* fuse = nullptr)
 {
     const OpBlock* b = blk(op);
     cudaError_t e;
     UmmaParams pp = b->p;
+    if (fuse) {
+        if (pp.mode != MODE_WGRAD || b->pair || pp.splits != 1 || !pp.bias_fused || !wgrad_sweep_ok(b)) {
+            snprintf(g_umma_err, sizeof(g_umma_err), "weight gradient with folded update asked for an op that cannot carry it");
+            return SB_ERR_CUDA;
+        }
+        pp.sgd_w = fuse->w; pp.sgd_v = fuse->v; pp.sgd_s = fuse->s; pp.sgd_lr = fuse->lr; pp.sgd_mu = fuse->mu;
+    }
     if (pp.mode == MODE_WGRAD && !b->pair) {
-        static const bool sweep_on = tune("SB_WGRAD_SWEEP", 1) != 0;
-        const bool aligned = (pp.ldc & 3) == 0 && (pp.w_cols & 3) == 0 && (pp.n_total & 3) == 0 && (pp.split_stride & 3) == 0 &&
-                             (((uintptr_t)pp.out) & 15) == 0;
-        const long ring = (long)pp.stages * (A_STAGE_BYTES + b->bn * 128);
-        pp.wg_sweep = ((sweep_on || pp.hn_order) && aligned && ring >= 32768) ? 1 : 0;
+        pp.wg_sweep = wgrad_sweep_ok(b) ? 1 : 0;
         if (pp.hn_order && !pp.wg_sweep) {
             snprintf(g_umma_err, sizeof(g_umma_err), "filter-column weight gradient planned without the staged epilogue");
             return SB_ERR_CUDA;
@@ -2745,6 +2870,27 @@ sb_status umma_conv_dgrad(sb_model* m, int layer, cudaStream_t st) { return laun
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->fwd, st, launch_counter(m)); }
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->dgrad, st, launch_counter(m)); }
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st) { return launch_op(layer_view(m, layer).um->wgrad, st); }
+
+bool umma_fc_wgrad_can_update(sb_model* m, int layer)
+{
+    const LayerView lv = layer_view(m, layer);
+    if (!lv.um->wgrad.enabled) return false;
+    const OpBlock* b = blk(lv.um->wgrad);
+    // (the parameter arenas share the gradient arena's element offsets: 16-byte alignment of `out` carries over)
+    const long smem = (long)b->p.stages * (A_STAGE_BYTES + b->bn * 128) + 1024 + CTRL_BYTES + UPD_EXTRA_SMEM;
+    // (layers of at least two CTAs per SM only: the kernel then holds a whole SM per CTA and has to fill the machine by
+    // itself -- 4096 x 4096: step -2.3 %; 4096 x 512 and the 1024-wide layers of the 7-conv net: +2 % with their 64 - 128 CTAs)
+    static const long min_ctas = (long)tune("SB_FC_UPDATE_MIN_CTAS", 296);
+    return b->p.mode == MODE_WGRAD && !b->pair && b->p.ntaps == 1 && b->bn != 192 && b->p.splits == 1 && b->p.bias_fused && wgrad_sweep_ok(b) &&
+           (lv.p_w & 3) == 0 && (lv.in_f % 64) == 0 && smem <= 227 * 1024 && (long)b->grid.x * b->grid.y * b->grid.z >= min_ctas;
+}
+sb_status umma_fc_wgrad_update(sb_model* m, int layer, float lr, float mu, cudaStream_t st)
+{
+    const ModelView mv = model_view(m);
+    const LayerView lv = layer_view(m, layer);
+    SgdFuse f{mv.Wm + lv.p_w, mv.Vm + lv.p_w, mv.Sm ? mv.Sm + lv.p_w : nullptr, lr, mu};
+    return launch_op(lv.um->wgrad, st, nullptr, &f);
+}
 
 bool umma_wgrad_bias_fused(sb_model* m, int layer)
 {

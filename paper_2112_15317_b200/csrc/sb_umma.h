@@ -29,7 +29,7 @@ struct ModelView {
     const sb_config* cfg;
     bool bf16;
     int B, n_layers, first_fc;
-    float *Wm, *Gm;
+    float *Wm, *Gm, *Vm;
     __nv_bfloat16* Sm;
     float* ws;      // data-side scratch
     float* ws_wk[8];  // weight-side scratch regions, one per weight stream: layer i uses ws_wk[i % n_wstreams]
@@ -74,6 +74,10 @@ sb_status umma_bind_input(sb_model* m, const void* x);
 sb_status umma_fc_fwd(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_dgrad(sb_model* m, int layer, cudaStream_t st);
 sb_status umma_fc_wgrad(sb_model* m, int layer, cudaStream_t st);
+// FC weight gradient with the SGD-momentum update applied in the kernel's epilogue (gradient never stored): possible when
+// umma_fc_wgrad_can_update says so (unsplit reduction, staged epilogue, bias gradient in the same kernel)
+bool umma_fc_wgrad_can_update(sb_model* m, int layer);
+sb_status umma_fc_wgrad_update(sb_model* m, int layer, float lr, float mu, cudaStream_t st);
 
 // Input-layer convolution (1, 3 or 4 input channels, 64 output channels, bf16) on the tensor cores.
 bool conv_in_umma_supported(int Cin, int Cout);
