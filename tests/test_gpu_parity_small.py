@@ -538,6 +538,46 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
     g1.close(); g2.close(); g3.close()
 
 
+def test_large_fc_layer_takes_its_update_inside_the_weight_gradient_kernel():
+    """In the fused step (sb_graph_step) the weight-gradient kernel of a large FC layer (4096 x 4096: two CTAs per SM and
+    more) applies the SGD-momentum update to its tile itself and never stores the gradient; the smaller FC layers keep
+    gradient store + update kernel.  Three steps must leave weights, biases and losses bit-identical to the separate
+    calls (whose update kernel the folded form restates operation for operation), the separate calls are checked
+    against the oracle, and a sentinel written into the gradient tensors shows which layers did not store theirs."""
+    import torch
+    b = sb()
+    net = [(si.CONV3X3_RELU, 64), (si.MAXPOOL2, 0), (si.FC_RELU, 4096), (si.FC_RELU, 4096), (si.FC, 16), (si.SOFTMAX_XENT, 16)]
+    wl = si.Workload("fc4096", net, 8, 8, 3, 4, 2, 2)
+    compare_everything(wl, True, steps=2, lr=0.02, mu=0.9, bias_std=0.1)           # separate calls against the oracle
+    params = si.make_params(wl, bias_std=0.1)
+    x, y = si.make_batch(wl)
+    g1 = gpu_model(wl, params, b.SB_BF16)
+    g2 = gpu_model(wl, params, b.SB_BF16)
+    xs, ys = device_batch(wl, x, y, True)
+    side = torch.cuda.Stream()
+    fc = [2, 3, 4]
+    with torch.cuda.stream(side):
+        for it in range(3):
+            g1.forward(xs, ys); g1.backward(); g1.sgd_step(0.02, 0.9); l1 = g1.loss()
+            if it == 2:
+                for li in fc:
+                    for part in range(wl.K):
+                        _, shape, _ = g2.tensor_info(b.SB_T_GRAD_W, li, part)
+                        g2.write(b.SB_T_GRAD_W, li, part, np.full(shape, 7.0, np.float32))
+            g2.graph_step(xs, ys, 0.02, 0.9); l2 = g2.loss()
+            assert l1 == l2, (it, l1, l2)
+        side.synchronize()
+    for a, c in zip(g1.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS), g2.gather_params(b.SB_T_WEIGHT, b.SB_T_BIAS)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    for a, c in zip(g1.gather_params(b.SB_T_MOM_W, b.SB_T_MOM_B), g2.gather_params(b.SB_T_MOM_W, b.SB_T_MOM_B)):
+        if a is not None:
+            assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
+    kept = {li: all(np.all(g2.read(b.SB_T_GRAD_W, li, part, squeeze=False) == 7.0) for part in range(wl.K)) for li in fc}
+    assert kept == {2: False, 3: True, 4: False}, kept      # only the 4096 x 4096 layer skipped its gradient store
+    g1.close(); g2.close()
+
+
 def test_prefetched_host_batches_give_the_same_steps():
     """sb_prefetch_host stages the inputs of later iterations on a copy stream (two staging areas); sb_train_step_host
     (or its asynchronous form, two iterations in flight) then consumes them in order.  Six iterations over three DIFFERENT batches, prefetched one and two iterations ahead,
