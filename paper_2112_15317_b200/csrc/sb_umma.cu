@@ -195,30 +195,29 @@ __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32
 // The same sweep with the SGD-momentum update folded in (FC layers in the fused step): instead of storing the gradient
 // tile, v <- mu v + g and w <- w - lr v are applied to the parameters at the tile's offsets and their bf16 copy is
 // refreshed -- the operations of the stand-alone update kernel in the same order, so the bits are the same, while the
-// float gradient is neither written nor read back (8 of 26 bytes per parameter).  The w and v rows of a 64-column slab
-// are fetched ahead by bulk copies (one 256-byte row of each per epilogue thread) into two slab buffers behind the
-// control block: slabs 0 and 1 are requested before the main loop starts, slab j + 2 when slab j has been swept, so a
-// CTA has 64 - 128 KB of parameter loads in flight while it multiplies, drains and sweeps.
+// float gradient is neither written nor read back (8 of 26 bytes per parameter).  The w and v boxes of a 64-column slab
+// (128 rows x 256 bytes each, float tensor maps over the master weights and the momentum buffer) are fetched ahead by
+// TMA into two slab buffers behind the control block: slabs 0 and 1 are requested before the main loop starts, slab
+// j + 2 when slab j has been swept, so a CTA has 64 - 128 KB of parameter loads in flight while it multiplies, drains
+// and sweeps.  (One 256-byte bulk copy per row and array, 256 per slab, kept the TMA unit busy for ~5 us per slab.)
 constexpr int UPD_SLAB_BYTES = 65536;                 // per slab buffer: w rows [128][256 B], then v rows [128][256 B]
 constexpr int UPD_EXTRA_SMEM = 2 * UPD_SLAB_BYTES;
-__device__ __forceinline__ void upd_request_slab(const UmmaParams& p, uint32_t buf_s, uint32_t bar_s, int row, bool row_ok, size_t row_off)
+__device__ __forceinline__ void upd_request_slab(const CUtensorMap* mapW, const CUtensorMap* mapV, uint8_t* buf, uint64_t* bar, int col, int m0)
 {
-    if (row_ok) {
-        mbar_arrive_expect_tx(bar_s, 512u);
-        bulk_load(buf_s + (uint32_t)row * 256u, p.sgd_w + row_off, 256u, bar_s);
-        bulk_load(buf_s + 32768u + (uint32_t)row * 256u, p.sgd_v + row_off, 256u, bar_s);
-    } else {
-        mbar_arrive(bar_s);
-    }
+    // one thread: a 64-column x 128-row box of w and one of v (rows past the matrix read as zeros and are never stored)
+    mbar_expect_tx(bar, (uint32_t)UPD_SLAB_BYTES);
+    tma_load_4d(mapW, buf, bar, col, m0, 0, 0);
+    tma_load_4d(mapV, buf + 32768, bar, col, m0, 0, 0);
 }
 template <int BN>
-__device__ __forceinline__ bool wgrad_sweep_update_epilogue(const UmmaParams& p, uint32_t taddr, uint8_t* stage, uint32_t slab_s, uint64_t* slab_bar,
-                                                             int row, int m0, int m_hi, int n0, int n_hi, size_t tile_off)
+__device__ __forceinline__ bool wgrad_sweep_update_epilogue(const UmmaParams& p, const CUtensorMap* mapW, const CUtensorMap* mapV, uint32_t taddr,
+                                                             uint8_t* stage, uint8_t* slab_buf, uint64_t* slab_bar, int row, int m0, int m_hi, int n0,
+                                                             int n_hi, size_t tile_off)
 {
+    const uint32_t slab_s = smem_u32(slab_buf);
     const int t128 = threadIdx.x - 64, q = t128 >> 5, lane = t128 & 31;
     const int hl = lane & 15, sub = lane >> 4;
     const uint32_t stage_s = smem_u32(stage);
-    const bool row_ok = m0 + row < m_hi;
     bool ok = true;
 #pragma unroll 1
     for (int j = 0; j < BN / 64; ++j) {
@@ -266,8 +265,8 @@ __device__ __forceinline__ bool wgrad_sweep_update_epilogue(const UmmaParams& p,
             }
         }
         epi_bar_sync();                                   // stage and slab buffer may be overwritten
-        if (ok && j + 2 < BN / 64 && n0 + c0 + 128 < n_hi)
-            upd_request_slab(p, buf_s, smem_u32(&slab_bar[j & 1]), row, row_ok, tile_off + (size_t)row * p.ldc + c0 + 128);
+        if (ok && threadIdx.x == 64 && j + 2 < BN / 64 && n0 + c0 + 128 < n_hi)
+            upd_request_slab(mapW, mapV, slab_buf + (size_t)(j & 1) * UPD_SLAB_BYTES, &slab_bar[j & 1], n0 + c0 + 128, m0);
     }
     return ok;
 }
@@ -497,7 +496,7 @@ __device__ __forceinline__ void pool_from_stage(const UmmaParams& p, const uint8
 template <int MODE, int BN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
-            const UmmaParams p)
+            const __grid_constant__ CUtensorMap mapD, const UmmaParams p)
 {
     using C = Cfg<MODE, BN>;
     extern __shared__ uint8_t smem_raw[];
@@ -651,7 +650,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             // a stage is released by the MMA commit, plus one arrival per epilogue warp in the CTAs that also sum dy
             for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], do_bias ? 5u : 1u); }
             mbar_init(acc_full, 1);
-            if (MODE == MODE_WGRAD && p.sgd_w != nullptr) { mbar_init(&slab_bar[0], 128); mbar_init(&slab_bar[1], 128); }
+            if (MODE == MODE_WGRAD && p.sgd_w != nullptr) { mbar_init(&slab_bar[0], 1); mbar_init(&slab_bar[1], 1); }
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             SB_TLOG(true, 8, clock64());    // barriers initialised
@@ -784,12 +783,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (MODE == MODE_WGRAD) {
             row_ok = (m0 + row) < m_hi;
             row_off = (size_t)split * p.split_stride + (size_t)(m0 + row) * p.ldc + (size_t)tap_fixed * p.w_cols;
-            if (p.sgd_w != nullptr) {
-                // update folded in: this thread's w and v rows of the first two 64-column slabs are requested now
+            if (p.sgd_w != nullptr && threadIdx.x == 64) {
+                // update folded in: the w and v boxes of the first two 64-column slabs are requested now
 #pragma unroll
                 for (int j = 0; j < 2; ++j)
                     if (j < BN / 64 && n0 + 64 * j < n_hi)
-                        upd_request_slab(p, smem_u32(slab_buf) + (uint32_t)j * (uint32_t)UPD_SLAB_BYTES, smem_u32(&slab_bar[j]), row, row_ok, row_off + n0 + 64 * j);
+                        upd_request_slab(&mapC, &mapD, slab_buf + (size_t)j * UPD_SLAB_BYTES, &slab_bar[j], n0 + 64 * j, m0);
             }
         } else {
             const int r1 = fast_div(row, p.rcp_bw), ni = fast_div(row, p.rcp_bwbh);
@@ -843,7 +842,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
                 if (p.sgd_w != nullptr) {
-                    if (!wgrad_sweep_update_epilogue<BN>(p, taddr, smem, smem_u32(slab_buf), slab_bar, row, m0, m_hi, n0, n_hi,
+                    if (!wgrad_sweep_update_epilogue<BN>(p, &mapC, &mapD, taddr, smem, slab_buf, slab_bar, row, m0, m_hi, n0, n_hi,
                                                          (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0) && lane == 0) {
                         *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI);
                     }
@@ -1901,6 +1900,23 @@ static bool mat_map(CUtensorMap* map, const void* ptr, long rows, long cols, int
     return encode_map(map, ptr, d, s, b);
 }
 
+// Row-major float matrix [rows][cols] -> map (cols, rows, 1, 1) with a (64, 128, 1, 1) box, no swizzle: 128 rows of 256 bytes.
+static bool mat_map_f32(CUtensorMap* map, const void* ptr, long rows, long cols)
+{
+    if (!get_encode()) return false;
+    cuuint64_t gd[4] = {(cuuint64_t)cols, (cuuint64_t)rows, 1, 1};
+    cuuint64_t gs[3] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * cols * 4, (cuuint64_t)rows * cols * 4};
+    cuuint32_t bx[4] = {64, 128, 1, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(ptr), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_umma_err, sizeof(g_umma_err), "cuTensorMapEncodeTiled (float matrix %ld x %ld) failed (%d)", rows, cols, (int)r);
+        return false;
+    }
+    return true;
+}
+
 static int cdiv_i(long a, long b) { return (int)((a + b - 1) / b); }
 
 // Pixel box (bw, bh, bn) with bw*bh*bn = target (a power of two): least padded volume, then widest rows.
@@ -1938,7 +1954,7 @@ static cudaError_t launch_one(const UmmaOp& op, const UmmaParams& p, dim3 grid, 
     // (a weight gradient with the update folded in carries two parameter slab buffers behind its control block)
     const size_t smem = (size_t)Cfg<MODE, BN>::smem_bytes(p.stages) + (MODE == MODE_WGRAD && p.sgd_w != nullptr ? (size_t)UPD_EXTRA_SMEM : 0);
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
-    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), smem, st, op.mapA, op.mapB, op.mapC, p);
+    return pdl_launch(umma_kernel<MODE, BN>, grid, dim3(UMMA_THREADS), smem, st, op.mapA, op.mapB, op.mapC, op.mapD, p);
 }
 
 template <int MODE, int BN>
@@ -2060,6 +2076,7 @@ struct OpBlock {
     int pair;      // FWD / DGRAD: run as CTA pairs (umma_pair_kernel); grid.x is then even
     int halo;      // 3x3 FWD / DGRAD: umma_halo_kernel (activation halos shared by the three taps of a filter column)
     int persist;   // ... its persistent variant: grid.x CTAs walk all tiles (umma_halo_persist_kernel)
+    int upd_maps;  // FC WGRAD: mapC / mapD are float maps over the layer's master weights and momentum
     dim3 grid;
     long rows;     // output rows (pixels / batch rows) of a FWD / DGRAD op
 };
@@ -2090,7 +2107,7 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     cudaError_t e;
     UmmaParams pp = b->p;
     if (fuse) {
-        if (pp.mode != MODE_WGRAD || b->pair || pp.splits != 1 || !pp.bias_fused || !wgrad_sweep_ok(b)) {
+        if (pp.mode != MODE_WGRAD || !b->upd_maps || b->pair || pp.splits != 1 || !pp.bias_fused || !wgrad_sweep_ok(b)) {
             snprintf(g_umma_err, sizeof(g_umma_err), "weight gradient with folded update asked for an op that cannot carry it");
             return SB_ERR_CUDA;
         }
@@ -2846,6 +2863,10 @@ sb_status umma_plan_layers(sb_model* m, int first_layer)
                 b->grid = dim3((unsigned)(p.m_tiles_per_shard * K), (unsigned)n_tiles, 1);
                 if (!act_map(&um.wgrad.mapA, lv.dact, B, 1, 1, lv.out_f, 1, 1, 64)) return fail_plan();
                 if (!act_map(&um.wgrad.mapB, lv.in_act, B, 1, 1, lv.in_f, 1, 1, 64)) return fail_plan();
+                // float maps over the master weights and the momentum buffer, for the weight gradient with the update folded in
+                b->upd_maps = (mv.Vm != nullptr && (lv.p_w & 3) == 0 && lv.in_f % 4 == 0 &&
+                               mat_map_f32(&um.wgrad.mapC, mv.Wm + lv.p_w, lv.out_f, lv.in_f) &&
+                               mat_map_f32(&um.wgrad.mapD, mv.Vm + lv.p_w, lv.out_f, lv.in_f)) ? 1 : 0;
                 um.wgrad.enabled = true;
             }
         }
@@ -2878,10 +2899,10 @@ bool umma_fc_wgrad_can_update(sb_model* m, int layer)
     const OpBlock* b = blk(lv.um->wgrad);
     // (the parameter arenas share the gradient arena's element offsets: 16-byte alignment of `out` carries over)
     const long smem = (long)b->p.stages * (A_STAGE_BYTES + b->bn * 128) + 1024 + CTRL_BYTES + UPD_EXTRA_SMEM;
-    // (layers of at least two CTAs per SM only: the kernel then holds a whole SM per CTA and has to fill the machine by
-    // itself -- 4096 x 4096: step -2.3 %; 4096 x 512 and the 1024-wide layers of the 7-conv net: +2 % with their 64 - 128 CTAs)
-    static const long min_ctas = (long)tune("SB_FC_UPDATE_MIN_CTAS", 296);
-    return b->p.mode == MODE_WGRAD && !b->pair && b->p.ntaps == 1 && b->bn != 192 && b->p.splits == 1 && b->p.bias_fused && wgrad_sweep_ok(b) &&
+    // (not for grids of a few dozen CTAs: the kernel holds a whole SM's shared memory per CTA -- measured per step: 4096 x 4096
+    // (512 CTAs) -3.4 %, 512 -> 4096 (64 CTAs) a further -1.4 %, a 1024 x 1024 layer (32 CTAs) +0.5 %)
+    static const long min_ctas = (long)tune("SB_FC_UPDATE_MIN_CTAS", 64);
+    return b->p.mode == MODE_WGRAD && b->upd_maps && !b->pair && b->p.ntaps == 1 && b->bn != 192 && b->p.splits == 1 && b->p.bias_fused && wgrad_sweep_ok(b) &&
            (lv.p_w & 3) == 0 && (lv.in_f % 64) == 0 && smem <= 227 * 1024 && (long)b->grid.x * b->grid.y * b->grid.z >= min_ctas;
 }
 sb_status umma_fc_wgrad_update(sb_model* m, int layer, float lr, float mu, cudaStream_t st)

@@ -12,7 +12,9 @@ struct UmmaOp {
     bool enabled = false;
     alignas(64) CUtensorMap mapA;
     alignas(64) CUtensorMap mapB;
-    alignas(64) CUtensorMap mapC;          // output tensor, for the TMA-store epilogue (when the op's tma_out is set)
+    alignas(64) CUtensorMap mapC;          // output tensor, for the TMA-store epilogue (when the op's tma_out is set);
+                                           // FC weight gradient: the float master weights [out][in] (update folded in)
+    alignas(64) CUtensorMap mapD;          // FC weight gradient: the momentum buffer, same shape
     alignas(16) unsigned char blob[512];   // kernel parameters, tile width and grid (see sb_umma.cu)
 };
 struct UmmaLayer {

@@ -539,14 +539,14 @@ def test_graph_step_and_graph_host_step_match_separate_calls(net):
 
 
 def test_large_fc_layer_takes_its_update_inside_the_weight_gradient_kernel():
-    """In the fused step (sb_graph_step) the weight-gradient kernel of a large FC layer (4096 x 4096: two CTAs per SM and
-    more) applies the SGD-momentum update to its tile itself and never stores the gradient; the smaller FC layers keep
-    gradient store + update kernel.  Three steps must leave weights, biases and losses bit-identical to the separate
+    """In the fused step (sb_graph_step) the weight-gradient kernel of a large FC layer (64 CTAs and more: 4096 x 4096,
+    1024 -> 4096) applies the SGD-momentum update to its tile itself and never stores the gradient; the smaller FC layers
+    keep gradient store + update kernel.  Three steps must leave weights, biases and losses bit-identical to the separate
     calls (whose update kernel the folded form restates operation for operation), the separate calls are checked
     against the oracle, and a sentinel written into the gradient tensors shows which layers did not store theirs."""
     import torch
     b = sb()
-    net = [(si.CONV3X3_RELU, 64), (si.MAXPOOL2, 0), (si.FC_RELU, 4096), (si.FC_RELU, 4096), (si.FC, 16), (si.SOFTMAX_XENT, 16)]
+    net = [(si.CONV3X3_RELU, 64), (si.MAXPOOL2, 0), (si.FC_RELU, 4096), (si.FC_RELU, 4096), (si.FC_RELU, 256), (si.FC, 16), (si.SOFTMAX_XENT, 16)]
     wl = si.Workload("fc4096", net, 8, 8, 3, 4, 2, 2)
     compare_everything(wl, True, steps=2, lr=0.02, mu=0.9, bias_std=0.1)           # separate calls against the oracle
     params = si.make_params(wl, bias_std=0.1)
@@ -555,7 +555,7 @@ def test_large_fc_layer_takes_its_update_inside_the_weight_gradient_kernel():
     g2 = gpu_model(wl, params, b.SB_BF16)
     xs, ys = device_batch(wl, x, y, True)
     side = torch.cuda.Stream()
-    fc = [2, 3, 4]
+    fc = [2, 3, 4, 5]
     with torch.cuda.stream(side):
         for it in range(3):
             g1.forward(xs, ys); g1.backward(); g1.sgd_step(0.02, 0.9); l1 = g1.loss()
@@ -574,7 +574,7 @@ def test_large_fc_layer_takes_its_update_inside_the_weight_gradient_kernel():
         if a is not None:
             assert np.array_equal(a["w"], c["w"]) and np.array_equal(a["b"], c["b"])
     kept = {li: all(np.all(g2.read(b.SB_T_GRAD_W, li, part, squeeze=False) == 7.0) for part in range(wl.K)) for li in fc}
-    assert kept == {2: False, 3: True, 4: False}, kept      # only the 4096 x 4096 layer skipped its gradient store
+    assert kept == {2: True, 3: True, 4: False, 5: False}, kept      # the two 4096-wide layers skipped their gradient store
     g1.close(); g2.close()
 
 
