@@ -336,9 +336,9 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     m->ws_w = m->ws_wk[0];
     m->row_loss = (float*)take(B * 4);
     scratch_region = false;     // (loss, counter and status words keep their values between calls)
-    m->loss = (float*)take(256);
+    m->loss = (float*)take(256);              // [0] = mean loss, [1] = device status word: adjacent, so that one copy reads both back
+    m->status = base ? (uint32_t*)(m->loss + 1) : nullptr;
     m->counter = (unsigned int*)take(256);
-    m->status = (uint32_t*)take(256);
     m->stage_x = take(B * m->in_per_img * m->esz);
     m->stage_labels = (int32_t*)take(B * 4);
     m->stage_xb[0] = m->stage_x; m->stage_lb[0] = m->stage_labels;
@@ -1356,8 +1356,7 @@ static sb_status host_step(sb_model* m, const void* host_x, const int32_t* host_
             s = e == cudaSuccess ? SB_OK : fail(SB_ERR_CUDA, "capturing the input copies: %s", cudaGetErrorString(e));
             if (s == SB_OK) s = whole_step(m, xp, lp, lr, momentum, stream);
             if (s == SB_OK) {
-                e = cudaMemcpyAsync(&m->host_res[2 * slot], m->loss, 4, cudaMemcpyDeviceToHost, st);
-                if (e == cudaSuccess) e = cudaMemcpyAsync(&m->host_res[2 * slot + 1], m->status, 4, cudaMemcpyDeviceToHost, st);
+                e = cudaMemcpyAsync(&m->host_res[2 * slot], m->loss, 8, cudaMemcpyDeviceToHost, st);      // loss and status word
                 if (e != cudaSuccess) s = fail(SB_ERR_CUDA, "capturing the read-back: %s", cudaGetErrorString(e));
             }
             if (s != SB_OK) { abandon_capture(st); return s; }
