@@ -2551,8 +2551,11 @@ static ConvGeom conv_geom(const LayerView& lv, int B, bool force_pair, bool no_h
     int s = wgrad_splits((long)g.wg_m_tiles * g.wg_n_tiles * tap_groups, g.total_chunks, g.wg_bn, (size_t)lv.n_w + lv.n_b, &cost);
     // a narrower N tile doubles the CTAs of a grid that leaves SMs idle (e.g. 512 channels at 4x4: 72 CTAs of 256
     // columns against 144 of 128): take it when the same model says it is faster (SB_WGRAD_NARROW=0 keeps the widest)
+    // (reductions of 128 pixel chunks or more only: for the short ones -- 512 channels at 4x4 and 2x2, batch 128 / 256 -- the 72
+    // wide CTAs leave half the SMs to the other streams, steps -0.6 %; the long ones of ImageNet-size inputs lose 1.3 % without it)
     static const bool narrow = tune("SB_WGRAD_NARROW", 1) != 0;
-    if (narrow && g.wg_tap_group == 1 && g.wg_bn == 256) {
+    static const int narrow_min_chunks = (int)tune("SB_WGRAD_NARROW_MIN_CHUNKS", 128);
+    if (narrow && g.wg_tap_group == 1 && g.wg_bn == 256 && g.total_chunks >= narrow_min_chunks) {
         double cost2 = 0.0;
         const int n2 = cdiv_i(lv.Cin, 128);
         const int s2 = wgrad_splits((long)g.wg_m_tiles * n2 * 9, g.total_chunks, 128, (size_t)lv.n_w + lv.n_b, &cost2);
