@@ -40,6 +40,14 @@ contractions) are rounded to bfloat16 (round-to-nearest-even) at the points wher
 stores them; accumulators, bias add, ReLU, logits, loss, dW/db, master weights and momentum stay
 in the working precision.
 
+Dropout [Listing 1, case DROPOUT | RELU: a one-to-one functional layer that follows the partitioned width]:
+each shard multiplies its own columns by a keep mask and by 1/(1 - p) (the reading taken: the expectation-
+preserving form, so that nothing changes at evaluation time).  The mask bit of element (global batch row g,
+logical column c) of dropout layer li in iteration t is drawn by the counter-based Philox-4x32-10 generator
+(Salmon et al., "Parallel random numbers: as easy as 1, 2, 3", SC'11) at counter (e mod 2^32, e div 2^32, li, t),
+e = g*width + c, key = the 64-bit seed: it depends on neither R nor K.  The element is kept iff the first output
+word is >= p * 2^32, p given in units of 1/65536.
+
 Parity pins: see tests/test_oracle_*.py (brute-force single-element evaluators, adjoint
 identities, finite differences in double, closed forms, R/K invariance, a float64 autograd
 re-computation of the unpartitioned network).  Unpinned: nothing in this file (group-MP mapping,
@@ -57,6 +65,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 from oracle import build_oracle  # noqa: E402
 
 CONV, POOL, FC_RELU, FC, LOSS = 1, 2, 3, 4, 5
+DROPOUT = 8   # out = drop probability p in units of 1/65536 (1 .. 65535)
 
 _libs = {}
 
@@ -86,6 +95,45 @@ def round_bf16(a: np.ndarray) -> np.ndarray:
 
 def shard_bounds(out: int, K: int):
     return [(j * out) // K for j in range(K + 1)]
+
+
+def philox4x32_10(c0, c1, c2, c3, k0, k1):
+    """Philox-4x32 with 10 rounds (Salmon et al., SC'11, section 3.3 and table 2 constants): counter words c0..c3
+    (uint32 arrays or scalars, broadcast together), key words k0, k1.  Returns the four output words as uint64
+    arrays holding 32-bit values.  One round: with (hi0, lo0) = M0 * c0 and (hi1, lo1) = M1 * c2 as 64-bit
+    products, the new counter is (hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0); the key is bumped by the Weyl
+    constants (golden ratio, sqrt(3) - 1) between rounds."""
+    M0, M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+    W0, W1 = 0x9E3779B9, 0xBB67AE85
+    mask = np.uint64(0xFFFFFFFF)
+    c0, c1, c2, c3 = (np.asarray(c, dtype=np.uint64) & mask for c in (c0, c1, c2, c3))
+    k0, k1 = int(k0) & 0xFFFFFFFF, int(k1) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = M0 * c0            # < 2^64: exact in uint64
+        p1 = M1 * c2
+        hi0, lo0 = p0 >> np.uint64(32), p0 & mask
+        hi1, lo1 = p1 >> np.uint64(32), p1 & mask
+        c0, c1, c2, c3 = hi1 ^ c1 ^ np.uint64(k0), lo1, hi0 ^ c3 ^ np.uint64(k1), lo0
+        k0 = (k0 + W0) & 0xFFFFFFFF
+        k1 = (k1 + W1) & 0xFFFFFFFF
+    return c0, c1, c2, c3
+
+
+def dropout_keep(seed, step, layer, rows, width, units):
+    """Keep mask [len(rows), width] of one dropout layer: element (global row g, column c) is kept iff the first
+    Philox word at counter (e mod 2^32, e div 2^32, layer, step mod 2^32), e = g*width + c, under the key
+    (seed mod 2^32, seed div 2^32) is >= units * 2^16, i.e. with probability 1 - units/65536."""
+    assert 0 < units < 65536
+    rows = np.asarray(rows, dtype=np.uint64)
+    e = rows[:, None] * np.uint64(width) + np.arange(width, dtype=np.uint64)[None, :]
+    x0, _, _, _ = philox4x32_10(e & np.uint64(0xFFFFFFFF), e >> np.uint64(32), layer, int(step) & 0xFFFFFFFF,
+                                int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
+    return x0 >= np.uint64(units << 16)
+
+
+def dropout_scale(units):
+    """1 / (1 - p) as one float32 division of exactly representable integers."""
+    return np.float32(65536.0) / np.float32(65536 - units)
 
 
 class Prims:
@@ -195,11 +243,16 @@ class OracleModel:
         self.mom = [None] * len(layers)
         self.bounds = [None] * len(layers)   # fc: shard column boundaries
         self.grads = [None] * len(layers)
+        self.dropout_seed, self.dropout_step = 0, 0   # key and iteration counter of the dropout masks
 
     # ---- helpers -------------------------------------------------------------------------
     def _q(self, a):
         """Storage rounding of the mixed-precision mode (identity otherwise)."""
         return round_bf16(a) if self.bf16 else a
+
+    def set_dropout(self, seed, step=0):
+        """Key of the dropout masks and the iteration number the next forward pass draws them for."""
+        self.dropout_seed, self.dropout_step = int(seed), int(step)
 
     def load_params(self, full_params):
         """Take the logical (unpartitioned) parameters and split every FC layer by output column
@@ -249,6 +302,7 @@ class OracleModel:
         self.pool_idx = [[None] * nl for _ in range(R)]
         self.fc_in = [None] * nl                          # full-width input of each FC layer [B,in]
         self.fc_out = [None] * nl                         # full-width output (after the shard layer)
+        self.drop_keep = [None] * nl                      # dropout layers: the keep mask [B,width]
         first_fc = next(i for i, (k, _) in enumerate(self.layers) if k in (FC_RELU, FC))
         self.first_fc = first_fc
         # 1. data-parallel convolution stack, one replica at a time
@@ -291,11 +345,28 @@ class OracleModel:
                     Y = self._q(Y)                        # stored activation; logits stay unrounded
                 self.fc_out[li] = Y
                 X = Y
+            elif kind == DROPOUT:
+                # one-to-one layer on the partitioned width: shard j masks and rescales its own columns of the layer
+                # below (an FC + ReLU), before the shard layer gathers them
+                assert self.layers[li - 1][0] == FC_RELU, "dropout follows an FC + ReLU layer"
+                cb = self.bounds[li - 1]
+                width = X.shape[1]
+                keep = dropout_keep(self.dropout_seed, self.dropout_step, li, np.arange(self.B), width, out)
+                scale = dropout_scale(out)
+                Y = np.empty_like(X)
+                for j in range(self.K):
+                    Xj, kj = X[:, cb[j]:cb[j + 1]], keep[:, cb[j]:cb[j + 1]]
+                    Y[:, cb[j]:cb[j + 1]] = self._q(np.where(kj, Xj * self.dt(scale), self.dt(0)))
+                self.drop_keep[li] = keep
+                self.fc_out[li] = Y
+                X = Y
             elif kind == LOSS:
                 # 5. log-softmax + NLL, mean over the full batch
                 self.logits = X
                 self.row_loss, self.dZ = P.softmax_xent(X, labels, 1.0 / self.loss_B)
                 self.loss = self.dt(np.sum(self.row_loss, dtype=self.dt) / self.dt(self.B))
+        if any(k == DROPOUT for k, _ in self.layers):
+            self.dropout_step += 1                        # the next forward pass draws fresh masks
         return self.loss
 
     # ---- backward ------------------------------------------------------------------------
@@ -307,6 +378,13 @@ class OracleModel:
         dY = self._q(self.dZ)         # gradient of the loss w.r.t. the last FC's output
         for li in range(nl - 2, self.first_fc - 1, -1):
             kind, out = self.layers[li]
+            if kind == DROPOUT:
+                # dY is the gradient w.r.t. this layer's output: the kept elements carry it down times 1/(1 - p); the
+                # layer below is an FC + ReLU, whose mask and storage rounding follow
+                self.d_pre[li] = dY
+                dIn = np.where(self.drop_keep[li], dY * self.dt(dropout_scale(out)), self.dt(0))
+                dY = self._q(dIn * (self.fc_out[li - 1] > 0))
+                continue
             cb = self.bounds[li]
             self.d_pre[li] = dY
             X = self.fc_in[li]
@@ -320,7 +398,9 @@ class OracleModel:
                 dX = dX + dXj
             self.grads[li] = g
             self.d_fc_in[li] = dX
-            if li > self.first_fc:
+            if li > self.first_fc and self.layers[li - 1][0] == DROPOUT:
+                dY = self._q(dX)                          # stored gradient w.r.t. the dropout layer's output
+            elif li > self.first_fc:
                 # the layer below is an FC+ReLU: mask by its stored output, then store
                 dY = self._q(dX * (self.fc_out[li - 1] > 0))
         # 7. modulo layer backward: rows back to their owners
@@ -392,6 +472,7 @@ class OracleModel:
         taken with the FC parameters of its own sub-iteration)."""
         P, R, b, K = self.P, self.R, self.b, self.K
         assert b % K == 0, "the modulo schedule needs b divisible by K"
+        assert all(k != DROPOUT for k, _ in self.layers), "dropout is not part of the sub-iteration schedule here"
         nl = len(self.layers)
         first_fc = next(i for i, (k, _) in enumerate(self.layers) if k in (FC_RELU, FC))
         assert first_fc > 0, "the modulo layer sits between a conv-side stack and the FC stack"

@@ -29,6 +29,7 @@ FC = 4
 SOFTMAX_XENT = 5
 FC_RELU_WHOLE = 6   # FC + ReLU that the partitioning keeps whole on every worker
 FC_WHOLE = 7
+DROPOUT = 8         # out = drop probability in units of 1/65536; follows an FC + ReLU layer
 
 SEED_WEIGHTS = 2112
 SEED_DATA = 15317
@@ -73,6 +74,7 @@ def layer_shapes(wl: Workload):
     conv : {'kind','H','W','Cin','Cout'}          (H, W preserved: 3x3, stride 1, zero pad 1)
     pool : {'kind','H','W','C'}                   (input H, W; output H/2, W/2)
     fc   : {'kind','in','out','relu'}
+    dropout : {'kind','width','units'}            (units = drop probability * 65536)
     loss : {'kind','classes'}
     """
     H, W, C = wl.H, wl.W, wl.C
@@ -94,6 +96,9 @@ def layer_shapes(wl: Workload):
             kind = FC_RELU if kind in (FC_RELU, FC_RELU_WHOLE) else FC      # (shapes and initial values do not depend on the split)
             out.append({"kind": kind, "in": feat, "out": o, "relu": kind == FC_RELU})
             feat = o
+        elif kind == DROPOUT:
+            assert feat is not None and 0 < o < 65536
+            out.append(dict(kind=kind, width=feat, units=o))
         elif kind == SOFTMAX_XENT:
             assert feat == o, "loss width must equal last FC width"
             out.append(dict(kind=kind, classes=o))
