@@ -58,12 +58,22 @@ typedef enum {
     SB_SOFTMAX_XENT = 5, /* log-softmax + negative log-likelihood, mean over the batch */
     SB_FC_RELU_WHOLE = 6, /* SB_FC_RELU kept whole on every worker: the "do not partition" outcome of the paper's
                              computation-to-communication test for this layer [Layer Partitioning] */
-    SB_FC_WHOLE = 7       /* SB_FC (logits layer) kept whole */
+    SB_FC_WHOLE = 7,      /* SB_FC (logits layer) kept whole */
+    SB_DROPOUT = 8        /* dropout on the output of the SB_FC_RELU / SB_FC_RELU_WHOLE layer directly below it: a one-to-one
+                             functional layer that follows the partitioned width, no modulo or shard node in between [Listing 1,
+                             case DROPOUT | RELU].  `out` = drop probability p in units of 1/65536 (1..65535).  Element (batch row
+                             g, column c) of the layer's [B, width] input is kept iff the first output word of the
+                             Philox-4x32-10 counter-based generator at counter (e mod 2^32, e div 2^32, layer index, iteration),
+                             e = g*width + c, key = the seed of sb_dropout_seed, is >= p * 2^32; kept elements are multiplied by
+                             1/(1 - p) (float 65536 / (65536 - out)), dropped ones are zero.  The mask depends on the logical
+                             element only, never on R or K.  The iteration counter lives on the device and goes up by one each
+                             time a forward pass has run the network's last dropout layer (graph replays included).  Not
+                             available under SB_FLAG_MODULO_SCHEDULE. */
 } sb_layer_kind;
 
 typedef struct {
     int32_t kind; /* sb_layer_kind */
-    int32_t out;  /* Cout / out-features / number of classes; ignored for SB_MAXPOOL2 */
+    int32_t out;  /* Cout / out-features / number of classes; ignored for SB_MAXPOOL2; SB_DROPOUT: p * 65536 */
 } sb_layer;
 
 enum { SB_FP32 = 0, SB_BF16 = 1 };
@@ -107,7 +117,8 @@ enum {
     SB_T_ACT = 6,      /* layer output.  conv/pool: replica `part`'s [b,H,W,C]; FC: [B,out] (part
                           ignored); activation dtype, except the logits layer which is float */
     SB_T_DACT = 7,     /* gradient w.r.t. the layer's pre-activation output (conv, FC) or w.r.t. its
-                          output (pool); same shape/partitioning as SB_T_ACT; activation dtype */
+                          output (pool, dropout: zero wherever the dropout output is zero); same shape/partitioning as SB_T_ACT;
+                          activation dtype */
     SB_T_POOL_IDX = 8, /* uint8 argmax position (dh*2+dw) per pooled element, replica `part` */
     SB_T_ROW_LOSS = 9, /* float [B]: per-row negative log-likelihood (layer = the loss layer) */
     SB_T_INPUT_GRAD = 10, /* gradient w.r.t. replica `part`'s input (needs SB_FLAG_INPUT_GRAD) */
@@ -263,6 +274,13 @@ sb_status sb_tensor_write(sb_model* m, int32_t what, int32_t layer, int32_t part
 
 /* Rebuild the bf16 weight copies from the float master weights (after sb_tensor_write). */
 sb_status sb_refresh_shadow(sb_model* m, void* stream);
+
+/*
+ * Dropout masks [Listing 1, case DROPOUT | RELU; see SB_DROPOUT]: sets the 64-bit key of the mask generator and the
+ * iteration number (taken modulo 2^32) the next forward pass draws its masks for.  Enqueues one tiny kernel on `stream`
+ * (asynchronous; a model is created with seed 0, iteration 0).  SB_ERR_INVALID_ARG for a null model.
+ */
+sb_status sb_dropout_seed(sb_model* m, uint64_t seed, uint64_t iteration, void* stream);
 
 /*
  * Run a sub-range of layers only, on whatever the arena buffers currently hold ("teacher

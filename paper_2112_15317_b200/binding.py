@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(HERE, "libsplitbrain.so")
 
 SB_OK = 0
 SB_FP32, SB_BF16 = 0, 1
-SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT, SB_FC_RELU_WHOLE, SB_FC_WHOLE = 1, 2, 3, 4, 5, 6, 7
+SB_CONV3X3_RELU, SB_MAXPOOL2, SB_FC_RELU, SB_FC, SB_SOFTMAX_XENT, SB_FC_RELU_WHOLE, SB_FC_WHOLE, SB_DROPOUT = 1, 2, 3, 4, 5, 6, 7, 8
 SB_NODE_LAYER, SB_NODE_MODULO, SB_NODE_SHARD = 0, 1, 2
 SB_X_GATHER_ROWS, SB_X_GATHER_COLS, SB_X_REDUCE_COLS, SB_X_REDUCE_ROWS, SB_X_ALLREDUCE, SB_X_ALLREDUCE_GROUPS = 1, 2, 3, 4, 5, 6
 SB_FLAG_INPUT_GRAD, SB_FLAG_FORCE_SIMT, SB_FLAG_PROFILE_LAYERS, SB_FLAG_FORCE_PAIR, SB_FLAG_MODULO_SCHEDULE, SB_FLAG_NO_HALO, SB_FLAG_FORCE_PERSIST = 1, 2, 4, 8, 16, 32, 64
@@ -87,6 +87,7 @@ def _load():
         "sb_tensor_read": [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_size_t],
         "sb_tensor_write": [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_size_t],
         "sb_refresh_shadow": [c_void_p, c_void_p],
+        "sb_dropout_seed": [c_void_p, ctypes.c_uint64, ctypes.c_uint64, c_void_p],
         "sb_forward_layers": [c_void_p, c_int32, c_int32, P(c_void_p), P(c_void_p), c_void_p],
         "sb_backward_layers": [c_void_p, c_int32, c_int32, c_void_p],
         "sb_param_bytes": [c_void_p, c_int32, P(c_size_t)],
@@ -134,6 +135,7 @@ sb_tensor = _lib.sb_tensor
 sb_tensor_read = _lib.sb_tensor_read
 sb_tensor_write = _lib.sb_tensor_write
 sb_refresh_shadow = _lib.sb_refresh_shadow
+sb_dropout_seed = _lib.sb_dropout_seed
 sb_forward_layers = _lib.sb_forward_layers
 sb_backward_layers = _lib.sb_backward_layers
 sb_param_bytes = _lib.sb_param_bytes
@@ -343,6 +345,9 @@ class Model:
 
     def refresh_shadow(self):
         _check(sb_refresh_shadow(self.h, self._stream()))
+
+    def dropout_seed(self, seed, iteration=0):
+        _check(sb_dropout_seed(self.h, ctypes.c_uint64(seed), ctypes.c_uint64(iteration), self._stream()))
 
     # ---- introspection -----------------------------------------------------------------------
     def tensor_info(self, what, layer, part=0):

@@ -98,6 +98,8 @@ struct sb_model {
     float *row_loss = nullptr, *loss = nullptr;
     unsigned int* counter = nullptr;
     uint32_t* status = nullptr;
+    uint32_t* drop_state = nullptr;   // dropout: {seed lo, seed hi, iteration, 0} (device words, kept between calls)
+    int last_dropout = -1;            // index of the network's last dropout layer: its forward kernel is followed by the iteration bump
     int pooled_by_conv = -1;   // index of the pool layer whose output the conv kernel just before it has already written (same forward call)
     // Set by the multi-stream backward pass while it enqueues the weight side of one conv layer: the layer's split
     // reduces then apply the update themselves (launch_reduce_sgd) once `ev` (the layer's input-gradient kernel, which
@@ -249,6 +251,15 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
             l.out_per_img = l.out;
             if (l.kind == SB_FC) l.act_dt = SB_DT_F32;
             break;
+        case SB_DROPOUT:
+            // one-to-one layer on the output of the FC + ReLU layer below [Listing 1, case DROPOUT | RELU]; out = p * 65536
+            if (i == 0 || m->L[i - 1].kind != SB_FC_RELU) return fail(SB_ERR_UNSUPPORTED, "layer %d: dropout must follow an FC + ReLU layer", i);
+            if (l.out < 1 || l.out > 65535) return fail(SB_ERR_SHAPE, "layer %d: drop probability must be 1..65535 (units of 1/65536)", i);
+            if (cfg->flags & SB_FLAG_MODULO_SCHEDULE) return fail(SB_ERR_UNSUPPORTED, "layer %d: dropout is not available under the modulo schedule", i);
+            l.in_f = l.out_f = (int)feat;
+            l.out_per_img = (size_t)feat;
+            m->last_dropout = i;
+            break;
         case SB_SOFTMAX_XENT:
             if (i != n - 1) return fail(SB_ERR_SHAPE, "the loss must be the last layer");
             if (i == 0 || m->L[i - 1].kind != SB_FC) return fail(SB_ERR_SHAPE, "the loss must follow an SB_FC (logits) layer");
@@ -339,6 +350,7 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
     m->loss = (float*)take(256);              // [0] = mean loss, [1] = device status word: adjacent, so that one copy reads both back
     m->status = base ? (uint32_t*)(m->loss + 1) : nullptr;
     m->counter = (unsigned int*)take(256);
+    m->drop_state = (uint32_t*)take(256);
     m->stage_x = take(B * m->in_per_img * m->esz);
     m->stage_labels = (int32_t*)take(B * 4);
     m->stage_xb[0] = m->stage_x; m->stage_lb[0] = m->stage_labels;
@@ -478,6 +490,12 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
         L_TRY("fc_fwd_simt", flops, bytes, launch_gemm_simt(a, bf, st));
         break;
     }
+    case SB_DROPOUT: {
+        const double n = (double)B * l.out_f;
+        L_TRY("dropout_fwd", 0.0, 2.0 * n * e, launch_dropout_fwd(layer_input(m, i), l.act, (size_t)B, l.out_f, m->drop_state, i, l.out, bf, st));
+        if (i == m->last_dropout) L_TRY("dropout_state", 0.0, 8.0, launch_dropout_state(m->drop_state, 1, 0, 0, st));
+        break;
+    }
     case SB_SOFTMAX_XENT: {
         if (!m->have_labels) return fail(SB_ERR_STATE, "the loss layer needs label pointers");
         Layer& fc = m->L[i - 1];
@@ -514,7 +532,7 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
     const bool want_in_grad = i > 0 || (m->cfg.flags & SB_FLAG_INPUT_GRAD);
     // where the gradient w.r.t. this layer's input goes, and whether the layer below applied a ReLU
     char* d_below = l.dbelow_override ? l.dbelow_override : (i > 0 ? m->L[i - 1].dact : m->input_grad);
-    const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
+    const bool below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU || m->L[i - 1].kind == SB_DROPOUT);
     const void* wts = bf ? (const void*)(m->Sm + l.p_w) : (const void*)(m->Wm + l.p_w);
     // this layer's weight-side scratch: one region per weight stream, so two layers that share a region are
     // ordered by the stream they share
@@ -579,6 +597,15 @@ sb_status backward_layer(sb_model* m, int i, cudaStream_t st, int part = SIDE_BO
                 L_TRY("fc_dgrad_simt", flops, bytes, launch_gemm_simt(a, bf, st));
             }
         }
+        break;
+    }
+    case SB_DROPOUT: {
+        // the layer above wrote the gradient w.r.t. this layer's output, zeroed wherever the output is zero (dropped, or the
+        // ReLU below was inactive): what is left is the scale of the kept elements, and the result is the gradient w.r.t. the
+        // pre-activation output of the FC + ReLU layer below
+        if (!(part & SIDE_D)) break;
+        const double n = (double)B * l.out_f;
+        L_TRY("dropout_bwd", 0.0, 2.0 * n * e, launch_dropout_bwd(l.dact, d_below, (size_t)B * l.out_f, l.out, bf, st));
         break;
     }
     case SB_MAXPOOL2: {
@@ -721,6 +748,7 @@ sb_status resolve(sb_model* m, int what, int li, int part, char** ptr, int64_t s
     char* p = nullptr;
     int dt = SB_DT_F32;
     const bool is_conv = l.kind == SB_CONV3X3_RELU, is_fc = l.kind == SB_FC_RELU || l.kind == SB_FC, is_pool = l.kind == SB_MAXPOOL2;
+    const bool is_flat = is_fc || l.kind == SB_DROPOUT;   // [B, width] activations
     auto param = [&](float* region, bool weight) -> sb_status {
         if (!is_conv && !is_fc) return fail(SB_ERR_INVALID_ARG, "layer %d has no parameters", li);
         if (is_conv) {
@@ -754,7 +782,7 @@ sb_status resolve(sb_model* m, int what, int li, int part, char** ptr, int64_t s
         char* basep = what == SB_T_ACT ? l.act : l.dact;
         dt = what == SB_T_ACT ? l.act_dt : (m->bf16 ? SB_DT_BF16 : SB_DT_F32);
         size_t e = dt == SB_DT_BF16 ? 2 : 4;
-        if (is_fc) { p = basep; sh[0] = m->B; sh[1] = l.out_f; }
+        if (is_flat) { p = basep; sh[0] = m->B; sh[1] = l.out_f; }
         else {
             if (part < 0 || part >= R) return fail(SB_ERR_INVALID_ARG, "replica %d out of range", part);
             p = basep + (size_t)part * b * l.out_per_img * e;
@@ -815,7 +843,7 @@ LayerView layer_view(sb_model* m, int i)
     v.act = l.act; v.dact = l.dact; v.um = &l.um; v.pool_idx = l.idx;
     v.in_act = l.in_override ? l.in_override : (i > 0 ? m->L[i - 1].act : nullptr);
     v.d_below = l.dbelow_override ? l.dbelow_override : (i > 0 ? m->L[i - 1].dact : m->input_grad);
-    v.below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU);
+    v.below_relu = i > 0 && (m->L[i - 1].kind == SB_CONV3X3_RELU || m->L[i - 1].kind == SB_FC_RELU || m->L[i - 1].kind == SB_DROPOUT);
     return v;
 }
 int64_t* launch_counter(sb_model* m) { return &m->launches; }
@@ -1159,6 +1187,15 @@ sb_status sb_refresh_shadow(sb_model* m, void* stream)
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     cudaStream_t st = (cudaStream_t)stream;
     if (m->bf16) L_TRY("to_bf16", 0.0, (double)m->P * 6.0, launch_to_bf16(m->Wm, m->Sm, m->P, st));
+    return SB_OK;
+}
+
+sb_status sb_dropout_seed(sb_model* m, uint64_t seed, uint64_t iteration, void* stream)
+{
+    if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
+    cudaStream_t st = (cudaStream_t)stream;
+    m->cur_layer = -1;
+    L_TRY("dropout_state", 0.0, 16.0, launch_dropout_state(m->drop_state, 0, seed, (uint32_t)iteration, st));
     return SB_OK;
 }
 

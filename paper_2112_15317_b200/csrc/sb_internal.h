@@ -178,6 +178,14 @@ struct ModuloCopyArgs {
 };
 cudaError_t launch_modulo_copy(const ModuloCopyArgs& a, cudaStream_t st);
 
+// Dropout layer on a [rows, width] activation matrix (units = drop probability * 65536): y = keep ? x / (1 - p) : 0 with the
+// keep bit of logical element (row, column) drawn by a counter-based generator from `state` = {seed lo, seed hi, iteration}
+// (device memory) and the layer index; backward: dx = dy / (1 - p) (dy arrives zero where the output was zero).
+cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st);
+cudaError_t launch_dropout_bwd(const void* dy, void* dx, size_t n, int units, bool bf16, cudaStream_t st);
+// mode 0: state <- {seed, iteration}; mode 1: iteration += 1
+cudaError_t launch_dropout_state(uint32_t* state, int mode, uint64_t seed, uint32_t iteration, cudaStream_t st);
+
 cudaError_t launch_sgd(float* w, float* v, const float* g, __nv_bfloat16* shadow, size_t n,
                        float lr, float mu, cudaStream_t st);
 cudaError_t launch_to_bf16(const float* w, __nv_bfloat16* shadow, size_t n, cudaStream_t st);

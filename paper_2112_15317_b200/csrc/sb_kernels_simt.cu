@@ -684,6 +684,74 @@ cudaError_t launch_modulo_copy(const ModuloCopyArgs& a, cudaStream_t st)
 }
 
 // =============================================================================================
+// Dropout [Listing 1, case DROPOUT | RELU]: a one-to-one layer on the (partitioned) width of the FC + ReLU layer below.
+// Element (global batch row g, logical column c) is kept iff the first output word of Philox-4x32-10 (Salmon et al.,
+// SC'11) at counter (e mod 2^32, e div 2^32, layer, iteration), e = g*width + c, under the 64-bit seed as key, is at
+// least p * 2^32; kept elements are multiplied by 1/(1 - p).  state = {seed lo, seed hi, iteration, unused}.
+// =============================================================================================
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1)
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+template <typename T>
+__global__ void __launch_bounds__(256)
+dropout_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, size_t n, const uint32_t* __restrict__ state, uint32_t layer,
+                   uint32_t threshold, float scale)
+{
+    pdl_prologue();
+    const uint32_t k0 = state[0], k1 = state[1], it = state[2];
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t u = philox4x32_10_word0((uint32_t)e, (uint32_t)(e >> 32), layer, it, k0, k1);
+        stf(y + e, u >= threshold ? ldf(x + e) * scale : 0.0f);
+    }
+}
+// y = x * scale (the backward pass of the kept elements; the dropped ones arrive as zeros)
+template <typename T>
+__global__ void __launch_bounds__(256)
+scale_kernel(const T* __restrict__ x, T* __restrict__ y, size_t n, float scale)
+{
+    pdl_prologue();
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) stf(y + e, ldf(x + e) * scale);
+}
+// mode 0: state = {v0, v1, v2, 0};  mode 1: ++iteration
+__global__ void dropout_state_kernel(uint32_t* state, int mode, uint32_t v0, uint32_t v1, uint32_t v2)
+{
+    pdl_prologue();
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (mode == 0) { state[0] = v0; state[1] = v1; state[2] = v2; state[3] = 0u; }
+    else state[2] += 1u;
+}
+cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st)
+{
+    const size_t n = rows * (size_t)width;
+    const uint32_t threshold = (uint32_t)units << 16;
+    const float scale = 65536.0f / (float)(65536 - units);
+    if (bf16) SB_LAUNCH((dropout_fwd_kernel<__nv_bfloat16>), ew_blocks((long)n), 256, 0, st, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, state, (uint32_t)layer, threshold, scale);
+    else SB_LAUNCH((dropout_fwd_kernel<float>), ew_blocks((long)n), 256, 0, st, (const float*)x, (float*)y, n, state, (uint32_t)layer, threshold, scale);
+    return cudaGetLastError();
+}
+cudaError_t launch_dropout_bwd(const void* dy, void* dx, size_t n, int units, bool bf16, cudaStream_t st)
+{
+    const float scale = 65536.0f / (float)(65536 - units);
+    if (bf16) SB_LAUNCH((scale_kernel<__nv_bfloat16>), ew_blocks((long)n), 256, 0, st, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, n, scale);
+    else SB_LAUNCH((scale_kernel<float>), ew_blocks((long)n), 256, 0, st, (const float*)dy, (float*)dx, n, scale);
+    return cudaGetLastError();
+}
+cudaError_t launch_dropout_state(uint32_t* state, int mode, uint64_t seed, uint32_t iteration, cudaStream_t st)
+{
+    SB_LAUNCH((dropout_state_kernel), 1, 32, 0, st, state, mode, (uint32_t)seed, (uint32_t)(seed >> 32), iteration);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
 // SGD with momentum over the whole (padded, 16-byte aligned) parameter arena:
 // v <- mu*v + g ; w <- w - lr*v ; optional bf16 copy of the new w.
 // =============================================================================================

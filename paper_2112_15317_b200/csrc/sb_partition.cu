@@ -7,7 +7,8 @@
 // input), splits fully-connected layers by output column into K shards unless the layer is marked "whole" (the
 // outcome of the paper's computation-to-communication test, for which it gives no formula), puts a MODULO node in
 // front of the first split layer whose input is whole and a SHARD node in front of every layer -- the loss included --
-// whose input arrives partitioned.  ReLU is part of the FC kinds here and follows the partitioned width.
+// whose input arrives partitioned.  ReLU is part of the FC kinds here and follows the partitioned width; so does a
+// dropout layer (the listing's DROPOUT | RELU case: dim and dimF pass through unchanged).
 //
 // Reading of the listing's LINEAR case: as printed it overwrites dimF with the layer's output width BEFORE comparing
 // dim with dimF; the surrounding text compares the two widths of the layer's INPUT ("if the input dimension has been
@@ -86,6 +87,13 @@ sb_status walk(const sb_layer* layers, int32_t n, const sb_config* cfg, std::vec
             dimF = out;
             dim = split ? (out + K - 1) / K : out;                       // "1/K size" (the widest shard when K does not divide out)
             push(SB_NODE_LAYER, i, split ? K : 1, dim, dimF);
+        } else if (kind == SB_DROPOUT) {
+            // one-to-one functional layer: adapts to the (partitioned) width of the layer below, dim and dimF pass through,
+            // no modulo or shard node in front of it
+            if (i == 0 || !(layers[i - 1].kind == SB_FC_RELU || layers[i - 1].kind == SB_FC_RELU_WHOLE))
+                return fail(SB_ERR_UNSUPPORTED, "layer %d: dropout must follow an FC + ReLU layer", i);
+            if (out < 1 || out > 65535) return fail(SB_ERR_SHAPE, "layer %d: drop probability must be 1..65535 (units of 1/65536)", i);
+            push(SB_NODE_LAYER, i, dim != dimF ? K : 1, dim, dimF);
         } else if (kind == SB_SOFTMAX_XENT) {
             if (dim != dimF) push(SB_NODE_SHARD, i, K, dimF, dimF);      // the loss needs the full width
             dim = dimF;

@@ -82,6 +82,30 @@ def test_layers_kept_whole_follow_the_listing():
     assert tokens(b, b.partition(net2, 8, 8, 3, 4), net2, 4) == "C* F F L"
 
 
+def test_dropout_follows_the_partitioned_width_without_communication_nodes():
+    """Listing 1, case DROPOUT | RELU: a one-to-one functional layer takes the width the layer below left (1/K of it
+    behind a split layer), passes dim and dimF on unchanged, and gets neither a modulo nor a shard node in front of it;
+    the shard node goes in front of the next layer that needs the full width."""
+    b = binding()
+    conv = [(si.CONV3X3_RELU, 8), (si.MAXPOOL2, 0)]
+    net = conv + [(si.FC_RELU, 32), (si.DROPOUT, 16384), (si.FC_RELU_WHOLE, 24), (si.DROPOUT, 100), (si.FC, 10), (si.SOFTMAX_XENT, 10)]
+    nodes = b.partition(net, 8, 8, 3, 4)
+    seq = [(nd["node"], nd["layer"], nd["shards"], nd["dim"], nd["dimF"]) for nd in nodes]
+    L, M, S = b.SB_NODE_LAYER, b.SB_NODE_MODULO, b.SB_NODE_SHARD
+    assert seq == [(L, 0, 1, 512, 512), (L, 1, 1, 128, 128),
+                   (M, 2, 4, 128, 128), (L, 2, 4, 8, 32), (L, 3, 4, 8, 32),          # dropout on the 1/K slice
+                   (S, 4, 4, 32, 32), (L, 4, 1, 24, 24), (L, 5, 1, 24, 24),          # whole layer, dropout on the whole width
+                   (L, 6, 4, 3, 10), (S, 7, 4, 10, 10), (L, 7, 1, 10, 10)]
+    # the exchange schedule gathers the dropout layer's column slices (layer 3), not the FC layer's below it
+    msgs = b.exchange_plan(net, 8, 8, 3, 2, 4)
+    gathers = {m["layer"] for m in msgs if m["kind"] == b.SB_X_GATHER_COLS}
+    assert gathers == {3, 6}
+    with pytest.raises(b.SBError, match="must follow an FC"):
+        b.partition(conv + [(si.DROPOUT, 100), (si.FC, 4), (si.SOFTMAX_XENT, 4)], 8, 8, 3, 2)
+    with pytest.raises(b.SBError, match="drop probability"):
+        b.partition(conv + [(si.FC_RELU, 8), (si.DROPOUT, 0), (si.FC, 4), (si.SOFTMAX_XENT, 4)], 8, 8, 3, 2)
+
+
 def test_conv_side_layers_refuse_a_partitioned_input_and_bad_lists_are_rejected():
     b = binding()
     with pytest.raises(b.SBError):
