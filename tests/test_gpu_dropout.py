@@ -163,6 +163,58 @@ def test_graph_replays_advance_the_iteration_and_match_the_oracle():
     assert np.array_equal(fc_act(gm2, b.SB_T_ACT, 5) != 0, om2.fc_out[5] != 0)
 
 
+def test_full_size_vgg16_with_dropout_in_the_classifier():
+    """The metric's network (VGG-16, CIFAR shape, batch 128, R = K = 4, bf16) with p = 0.5 dropout after both 4096-wide FC
+    layers, in the launch configuration the benchmark times (sb_graph_step: multi-stream backward, update folded into the
+    FC weight-gradient kernels).  Forward against the oracle; the dropout layers exactly, on the stored tensors; two
+    graph iterations draw different masks."""
+    from oracle import splitbrain_oracle as so
+    b = sb()
+    base = si.config(1)
+    layers = []
+    for kind, out in base.layers:
+        layers.append((kind, out))
+        if kind == si.FC_RELU:
+            layers.append((si.DROPOUT, P50))
+    wl = si.Workload("cfg1_dropout", layers, base.H, base.W, base.C, base.b, base.R, base.K)
+    params = si.make_params(wl)
+    x, y = si.make_batch(wl)
+    gm = gpu_model(wl, params, b.SB_BF16); gm.dropout_seed(SEED, 100)
+    xs, ys = device_batch(wl, x, y, True)
+    gm.forward(xs, ys)
+    om = oracle_model(wl, params, True); om.set_dropout(SEED, 100)
+    lo = float(om.forward(si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)))
+    assert abs(gm.loss() - lo) / abs(lo) < 1e-2
+    drops = drop_layers(wl)
+    assert len(drops) == 2
+    masks = []
+    for li in drops:
+        below = fc_act(gm, b.SB_T_ACT, li - 1)
+        keep = so.dropout_keep(SEED, 100, li, np.arange(wl.B), 4096, P50)
+        want = so.round_bf16(np.where(keep, below * so.dropout_scale(P50), np.float32(0)))
+        assert np.array_equal(fc_act(gm, b.SB_T_ACT, li), want), li
+        assert abs(keep.mean() - 0.5) < 5 * 0.5 / np.sqrt(keep.size)
+        assert maxrel(fc_act(gm, b.SB_T_ACT, li), om.fc_out[li]) < 2e-2
+        masks.append(keep)
+    # whole iterations through the graph path: iteration 101 (direct), 102 (captured), 103 (replayed)
+    import torch
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for it in (101, 102, 103):
+            gm.graph_step(xs, ys, 1e-3, 0.9)
+            s.synchronize()
+            li = drops[0]
+            below = fc_act(gm, b.SB_T_ACT, li - 1)
+            keep = so.dropout_keep(SEED, it, li, np.arange(wl.B), 4096, P50)
+            assert np.array_equal(fc_act(gm, b.SB_T_ACT, li), so.round_bf16(np.where(keep, below * so.dropout_scale(P50), np.float32(0)))), it
+            assert 0.4 < np.mean(keep != masks[0]) < 0.6
+            # backward through the layer, on the stored gradients
+            dact = fc_act(gm, b.SB_T_DACT, li)
+            assert np.all(dact[fc_act(gm, b.SB_T_ACT, li) == 0] == 0)
+            assert np.array_equal(fc_act(gm, b.SB_T_DACT, li - 1), so.round_bf16(dact * so.dropout_scale(P50))), it
+    assert np.isfinite(gm.loss())
+
+
 def test_dropout_is_refused_where_it_is_not_supported():
     b = sb()
     bad_after_conv = [(si.CONV3X3_RELU, 8), (si.DROPOUT, P25), (si.FC, 4), (si.SOFTMAX_XENT, 4)]
