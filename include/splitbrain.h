@@ -67,8 +67,9 @@ typedef enum {
                              e = g*width + c, key = the seed of sb_dropout_seed, is >= p * 2^32; kept elements are multiplied by
                              1/(1 - p) (float 65536 / (65536 - out)), dropped ones are zero.  The mask depends on the logical
                              element only, never on R or K.  The iteration counter lives on the device and goes up by one each
-                             time a forward pass has run the network's last dropout layer (graph replays included).  Not
-                             available under SB_FLAG_MODULO_SCHEDULE. */
+                             time a forward pass has run the network's last dropout layer (graph replays included); in
+                             sb_modulo_step the K sub-iterations are one iteration and every example meets the mask of its
+                             batch row. */
 } sb_layer_kind;
 
 typedef struct {

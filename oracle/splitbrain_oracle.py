@@ -472,7 +472,6 @@ class OracleModel:
         taken with the FC parameters of its own sub-iteration)."""
         P, R, b, K = self.P, self.R, self.b, self.K
         assert b % K == 0, "the modulo schedule needs b divisible by K"
-        assert all(k != DROPOUT for k, _ in self.layers), "dropout is not part of the sub-iteration schedule here"
         nl = len(self.layers)
         first_fc = next(i for i, (k, _) in enumerate(self.layers) if k in (FC_RELU, FC))
         assert first_fc > 0, "the modulo layer sits between a conv-side stack and the FC stack"
@@ -507,7 +506,7 @@ class OracleModel:
             rows = self.modulo_rows(k)
             X = np.ascontiguousarray(X_all[rows])
             labels = np.ascontiguousarray(labels_all[rows])
-            fc_in, fc_out = {}, {}
+            fc_in, fc_out, drop_keep = {}, {}, {}
             for li in range(first_fc, nl):
                 kind, out = self.layers[li]
                 if kind in (FC_RELU, FC):
@@ -521,12 +520,26 @@ class OracleModel:
                         Y = self._q(Y)
                     fc_out[li] = Y
                     X = Y
+                elif kind == DROPOUT:
+                    # the masks of an iteration belong to the examples (global rows), whichever sub-iteration carries them
+                    cb = self.bounds[li - 1]
+                    keep = dropout_keep(self.dropout_seed, self.dropout_step, li, rows, X.shape[1], out)
+                    Y = np.empty_like(X)
+                    for j in range(K):
+                        Y[:, cb[j]:cb[j + 1]] = self._q(np.where(keep[:, cb[j]:cb[j + 1]], X[:, cb[j]:cb[j + 1]] * self.dt(dropout_scale(out)), self.dt(0)))
+                    drop_keep[li] = keep
+                    fc_out[li] = Y
+                    X = Y
                 else:
                     row_loss, dZ = P.softmax_xent(X, labels, 1.0 / self.B)
                     row_loss_all[rows] = row_loss
             dY = self._q(dZ)
             g_k = {}
             for li in range(nl - 2, first_fc - 1, -1):
+                if self.layers[li][0] == DROPOUT:
+                    dIn = np.where(drop_keep[li], dY * self.dt(dropout_scale(self.layers[li][1])), self.dt(0))
+                    dY = self._q(dIn * (fc_out[li - 1] > 0))
+                    continue
                 cb = self.bounds[li]
                 Xin = fc_in[li]
                 g = []
@@ -537,7 +550,9 @@ class OracleModel:
                     g.append({"w": dWj, "b": dbj})
                     dX = dX + dXj
                 g_k[li] = g
-                if li > first_fc:
+                if li > first_fc and self.layers[li - 1][0] == DROPOUT:
+                    dY = self._q(dX)
+                elif li > first_fc:
                     dY = self._q(dX * (fc_out[li - 1] > 0))
             dX_all[rows] = dX
             self.mod_fc_grads.append(g_k)
@@ -548,6 +563,8 @@ class OracleModel:
                         P.sgd(self.params[li][j][key], self.mom[li][j][key], g[j][key], lr, mu)
         self.row_loss = row_loss_all
         self.loss = self.dt(np.sum(row_loss_all, dtype=self.dt) / self.dt(self.B))
+        if any(k_ == DROPOUT for k_, _ in self.layers):
+            self.dropout_step += 1                        # one iteration = all K sub-iterations
         # 3. modulo layer backward + conv stack backward on all rows, DP reduce, conv update (as in backward())
         dfeat = [np.empty((b,) + self.feat_shape[1:], self.dt) for _ in range(R)]
         for g_ in range(self.B):

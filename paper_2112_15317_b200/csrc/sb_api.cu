@@ -255,7 +255,6 @@ sb_status plan(const sb_layer* layers, int n, const sb_config* cfg, sb_model* m,
             // one-to-one layer on the output of the FC + ReLU layer below [Listing 1, case DROPOUT | RELU]; out = p * 65536
             if (i == 0 || m->L[i - 1].kind != SB_FC_RELU) return fail(SB_ERR_UNSUPPORTED, "layer %d: dropout must follow an FC + ReLU layer", i);
             if (l.out < 1 || l.out > 65535) return fail(SB_ERR_SHAPE, "layer %d: drop probability must be 1..65535 (units of 1/65536)", i);
-            if (cfg->flags & SB_FLAG_MODULO_SCHEDULE) return fail(SB_ERR_UNSUPPORTED, "layer %d: dropout is not available under the modulo schedule", i);
             l.in_f = l.out_f = (int)feat;
             l.out_per_img = (size_t)feat;
             m->last_dropout = i;
@@ -492,8 +491,12 @@ sb_status forward_layer(sb_model* m, int i, cudaStream_t st)
     }
     case SB_DROPOUT: {
         const double n = (double)B * l.out_f;
-        L_TRY("dropout_fwd", 0.0, 2.0 * n * e, launch_dropout_fwd(layer_input(m, i), l.act, (size_t)B, l.out_f, m->drop_state, i, l.out, bf, st));
-        if (i == m->last_dropout) L_TRY("dropout_state", 0.0, 8.0, launch_dropout_state(m->drop_state, 1, 0, 0, st));
+        // (a sub-iteration of the modulo schedule works on b/K rows of every replica: the masks are those of the batch rows,
+        // and the iteration counter moves on after the last sub-iteration)
+        const int sub_bk = m->sub_active ? b / m->cfg.K : 0, sub_k = m->sub_active ? m->sub_row0 / B : 0;
+        L_TRY("dropout_fwd", 0.0, 2.0 * n * e, launch_dropout_fwd(layer_input(m, i), l.act, (size_t)B, l.out_f, m->drop_state, i, l.out, bf, st, sub_bk, b, sub_k));
+        if (i == m->last_dropout && (!m->sub_active || m->sub_row0 + B == m->full_B))
+            L_TRY("dropout_state", 0.0, 8.0, launch_dropout_state(m->drop_state, 1, 0, 0, st));
         break;
     }
     case SB_SOFTMAX_XENT: {
@@ -917,7 +920,7 @@ sb_status sb_model_create(const sb_layer* layers, int32_t n, const sb_config* cf
             const size_t row0 = (size_t)k * Bk;
             for (int i = m->first_fc; i < m->n_layers; ++i) {
                 Layer& l = Lk[i];
-                if (l.kind != SB_FC_RELU && l.kind != SB_FC) continue;
+                if (l.kind != SB_FC_RELU && l.kind != SB_FC && l.kind != SB_DROPOUT) continue;
                 l.act += row0 * l.out_per_img * (l.act_dt == SB_DT_F32 ? 4 : m->esz);
                 l.dact += row0 * l.out_per_img * m->esz;
                 l.um = UmmaLayer{};

@@ -181,7 +181,9 @@ cudaError_t launch_modulo_copy(const ModuloCopyArgs& a, cudaStream_t st);
 // Dropout layer on a [rows, width] activation matrix (units = drop probability * 65536): y = keep ? x / (1 - p) : 0 with the
 // keep bit of logical element (row, column) drawn by a counter-based generator from `state` = {seed lo, seed hi, iteration}
 // (device memory) and the layer index; backward: dx = dy / (1 - p) (dy arrives zero where the output was zero).
-cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st);
+// sub_bk > 0: the rows are sub-iteration sub_k of the modulo schedule (sub_bk rows of each replica's sub_b); masks follow the batch rows
+cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st,
+                               int sub_bk = 0, int sub_b = 0, int sub_k = 0);
 cudaError_t launch_dropout_bwd(const void* dy, void* dx, size_t n, int units, bool bf16, cudaStream_t st);
 // mode 0: state <- {seed, iteration}; mode 1: iteration += 1
 cudaError_t launch_dropout_state(uint32_t* state, int mode, uint64_t seed, uint32_t iteration, cudaStream_t st);

@@ -701,16 +701,24 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
     }
     return c0;
 }
+// sub_bk > 0: the rows are those of sub-iteration sub_k of the modulo layer's schedule (replica r's sub_k-th slice of sub_bk rows,
+// replica-major): buffer row j is batch row (j / sub_bk) * sub_b + sub_k * sub_bk + j % sub_bk, and the mask follows the batch row
 template <typename T>
 __global__ void __launch_bounds__(256)
-dropout_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, size_t n, const uint32_t* __restrict__ state, uint32_t layer,
-                   uint32_t threshold, float scale)
+dropout_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, size_t n, int width, const uint32_t* __restrict__ state, uint32_t layer,
+                   uint32_t threshold, float scale, int sub_bk, int sub_b, int sub_k)
 {
     pdl_prologue();
     const uint32_t k0 = state[0], k1 = state[1], it = state[2];
-    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        size_t e = i;
+        if (sub_bk > 0) {
+            const size_t j = i / (size_t)width, c = i - j * (size_t)width;
+            const size_t g = (j / (size_t)sub_bk) * (size_t)sub_b + (size_t)sub_k * (size_t)sub_bk + j % (size_t)sub_bk;
+            e = g * (size_t)width + c;
+        }
         const uint32_t u = philox4x32_10_word0((uint32_t)e, (uint32_t)(e >> 32), layer, it, k0, k1);
-        stf(y + e, u >= threshold ? ldf(x + e) * scale : 0.0f);
+        stf(y + i, u >= threshold ? ldf(x + i) * scale : 0.0f);
     }
 }
 // y = x * scale (the backward pass of the kept elements; the dropped ones arrive as zeros)
@@ -729,13 +737,14 @@ __global__ void dropout_state_kernel(uint32_t* state, int mode, uint32_t v0, uin
     if (mode == 0) { state[0] = v0; state[1] = v1; state[2] = v2; state[3] = 0u; }
     else state[2] += 1u;
 }
-cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st)
+cudaError_t launch_dropout_fwd(const void* x, void* y, size_t rows, int width, const uint32_t* state, int layer, int units, bool bf16, cudaStream_t st,
+                               int sub_bk, int sub_b, int sub_k)
 {
     const size_t n = rows * (size_t)width;
     const uint32_t threshold = (uint32_t)units << 16;
     const float scale = 65536.0f / (float)(65536 - units);
-    if (bf16) SB_LAUNCH((dropout_fwd_kernel<__nv_bfloat16>), ew_blocks((long)n), 256, 0, st, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, state, (uint32_t)layer, threshold, scale);
-    else SB_LAUNCH((dropout_fwd_kernel<float>), ew_blocks((long)n), 256, 0, st, (const float*)x, (float*)y, n, state, (uint32_t)layer, threshold, scale);
+    if (bf16) SB_LAUNCH((dropout_fwd_kernel<__nv_bfloat16>), ew_blocks((long)n), 256, 0, st, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, width, state, (uint32_t)layer, threshold, scale, sub_bk, sub_b, sub_k);
+    else SB_LAUNCH((dropout_fwd_kernel<float>), ew_blocks((long)n), 256, 0, st, (const float*)x, (float*)y, n, width, state, (uint32_t)layer, threshold, scale, sub_bk, sub_b, sub_k);
     return cudaGetLastError();
 }
 cudaError_t launch_dropout_bwd(const void* dy, void* dx, size_t n, int units, bool bf16, cudaStream_t st)

@@ -215,6 +215,41 @@ def test_full_size_vgg16_with_dropout_in_the_classifier():
     assert np.isfinite(gm.loss())
 
 
+@pytest.mark.parametrize("name,R,K", [("tensor_core", 2, 2), ("tensor_core", 1, 4), ("ragged", 2, 3)])
+def test_modulo_schedule_with_dropout(name, R, K):
+    """sb_modulo_step: the K sub-iterations are one iteration, and every example meets the mask of its batch row although the
+    sub-batches hold the rows in another order.  Float mode, two iterations, parameters and momentum within 1e-4; the masks
+    of the last sub-iteration bit for bit."""
+    b = sb()
+    base = WORKLOADS[name]()
+    wl = si.Workload(base.name + "_mod", base.layers, base.H, base.W, base.C, 2 * K, R, K)      # b = 2K rows per replica: sub-batches of 2R rows
+    params = si.make_params(wl, bias_std=0.2)
+    x, y = si.make_batch(wl)
+    om = oracle_model(wl, params, False); om.set_dropout(SEED, 77)
+    gm = gpu_model(wl, params, b.SB_FP32, flags=b.SB_FLAG_MODULO_SCHEDULE); gm.dropout_seed(SEED, 77)
+    xs, ys = device_batch(wl, x, y, False)
+    xr, yr = si.split_replicas(x, wl.R), si.split_replicas(y, wl.R)
+    from oracle import splitbrain_oracle as so
+    for step in range(2):
+        lo = float(om.step_modulo(xr, yr, 0.02, 0.9))
+        gm.modulo_step(xs, ys, 0.02, 0.9)
+        assert abs(gm.loss() - lo) / abs(lo) < 1e-4, step
+        for what_w, what_b, ref_list in ((b.SB_T_WEIGHT, b.SB_T_BIAS, om.full_params()), (b.SB_T_MOM_W, b.SB_T_MOM_B, om.full_mom())):
+            got = gm.gather_params(what_w, what_b)
+            for li, (a, ref) in enumerate(zip(got, ref_list)):
+                if ref is not None:
+                    assert maxrel(a["w"].reshape(ref["w"].shape), ref["w"]) < 1e-4, (step, li)
+                    assert maxrel(a["b"], ref["b"]) < 1e-4, (step, li)
+        # the FC-side buffers hold the last sub-iteration in their last B/K rows, rows in sub-iteration order
+        rows = om.modulo_rows(wl.K - 1)
+        for li in drop_layers(wl):
+            act = fc_act(gm, b.SB_T_ACT, li)[-len(rows):]
+            below = fc_act(gm, b.SB_T_ACT, li - 1)[-len(rows):]
+            keep = so.dropout_keep(SEED, 77 + step, li, rows, act.shape[1], wl.layers[li][1])
+            assert np.array_equal(act != 0, keep & (below > 0)), (step, li)
+    assert om.dropout_step == 79
+
+
 def test_dropout_is_refused_where_it_is_not_supported():
     b = sb()
     bad_after_conv = [(si.CONV3X3_RELU, 8), (si.DROPOUT, P25), (si.FC, 4), (si.SOFTMAX_XENT, 4)]
@@ -223,6 +258,3 @@ def test_dropout_is_refused_where_it_is_not_supported():
     bad_p = [(si.CONV3X3_RELU, 8), (si.FC_RELU, 8), (si.DROPOUT, 65536), (si.FC, 4), (si.SOFTMAX_XENT, 4)]
     with pytest.raises(b.SBError, match="drop probability"):
         b.Model(bad_p, 4, 4, 4, 2, 1, 1)
-    wl = WORKLOADS["tensor_core"]()
-    with pytest.raises(b.SBError, match="modulo schedule"):
-        b.Model.from_workload(wl, flags=b.SB_FLAG_MODULO_SCHEDULE)

@@ -247,9 +247,31 @@ def test_bf16_mode_rounds_the_stored_dropout_tensors():
         assert np.array_equal(m.fc_out[li], so.round_bf16(exact)) and not np.array_equal(m.fc_out[li], exact)
 
 
-def test_modulo_schedule_refuses_dropout():
+def test_modulo_schedule_draws_the_same_masks_for_the_same_examples():
+    """The sub-iteration schedule sends every example through the FC stack exactly once per iteration: with the learning
+    rate at zero its FC gradients add up to the synchronous step's, its input gradients are the same, and so are the conv
+    gradients -- provided each example meets the same dropout mask in both schedules."""
     wl = si.Workload("drop_mod", net(), 8, 8, 3, 4, 2, 2)
-    m = make(wl)
     xr, yr = batch(wl)
-    with pytest.raises(AssertionError):
-        m.step_modulo(xr, yr, 0.01, 0.9)
+    a = make(wl, step=9); b_ = make(wl, step=9)
+    la = a.forward(xr, yr); a.backward()
+    lb = b_.step_modulo(xr, yr, 0.0, 0.9)
+    assert lb == pytest.approx(la, rel=1e-13)
+    assert a.dropout_step == b_.dropout_step == 10
+    ga = a.full_grads()
+    for li in range(len(wl.layers)):
+        if ga[li] is None:
+            continue
+        if li < a.first_fc:
+            assert maxrel(b_.grads[li]["w"], ga[li]["w"]) < 1e-12
+        else:
+            tot = sum(np.concatenate([s_["w"] for s_ in gk[li]], 0) for gk in b_.mod_fc_grads)
+            assert maxrel(tot, ga[li]["w"]) < 1e-12
+    # K = 1: one sub-iteration, the same iteration as step()
+    wl1 = wl.with_partition(4, 1)
+    x1, y1 = batch(wl1)
+    c = make(wl1, step=3); d = make(wl1, step=3)
+    assert c.step(x1, y1, 0.05, 0.9) == d.step_modulo(x1, y1, 0.05, 0.9)
+    for p_, q_ in zip(c.full_params(), d.full_params()):
+        if p_ is not None:
+            assert np.array_equal(p_["w"], q_["w"])
