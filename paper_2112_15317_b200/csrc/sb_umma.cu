@@ -271,12 +271,81 @@ __device__ __forceinline__ bool wgrad_sweep_update_epilogue(const UmmaParams& p,
     return ok;
 }
 
+// 16 consecutive output columns of one tile row, as bf16, into the staged tile (64-column slabs of 128 rows x 128 bytes in the
+// 128-byte swizzle of the output tensor map).
+__device__ __forceinline__ void stage_chunk16(const float (&f)[16], uint32_t row_s, uint32_t sw, int c0)
+{
+    uint32_t pk[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+        pk[j] = *(uint32_t*)&t;
+    }
+    const uint32_t slab = row_s + (uint32_t)(c0 >> 6) * 16384u, j0 = (uint32_t)(c0 & 63) >> 3;
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((j0 ^ sw) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + (((j0 + 1u) ^ sw) << 4)), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+}
+
+// Data-gradient epilogue, staged output: the ReLU-mask row of this thread (BN bf16 values of the layer's input at the thread's
+// pixel) is fetched into registers before the accumulator is waited for, so that the loads' latency hides behind the main
+// loop (read per 16-column chunk inside the epilogue it cost 0.5 - 0.8 us per chunk, 3 - 4 us per 128-wide tile).
+// (256-wide tiles keep a window of 128 columns in registers: store_row refills a slot with the values 128 columns further on
+// as soon as it has used it, seven chunks ahead of their use)
+template <int BN> struct MaskRow { static constexpr int SLOTS = (BN < 128 ? BN : 128) / 8; };
+template <int MODE, int BN>
+__device__ __forceinline__ bool prefetch_mask_row(const UmmaParams& p, bool row_ok, size_t row_off, int n0, int n_hi, uint4* refq)
+{
+    if (!(MODE == MODE_DGRAD && p.tma_out && p.epi == UEPI_MASK && p.ref != nullptr)) return false;
+    const uint4* rp = (const uint4*)(p.ref + row_off + n0);
+#pragma unroll
+    for (int j = 0; j < MaskRow<BN>::SLOTS; ++j) refq[j] = (row_ok && n0 + 8 * j < n_hi) ? __ldg(rp + j) : make_uint4(0u, 0u, 0u, 0u);
+    return true;
+}
+
 // Epilogue of one accumulator row: reads BN columns of this warp's TMEM lane quadrant (16 at a time) and
 // writes them as raw split partial sums, or with bias + ReLU / the ReLU mask applied, as float or bf16.
 template <int MODE, int BN>
 __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, bool row_ok, size_t row_off, int n0, int n_hi,
-                                          int split, const float* s_bias, uint8_t* stage = nullptr, int row = 0)
+                                          int split, const float* s_bias, uint8_t* stage = nullptr, int row = 0, const uint4* refq = nullptr)
 {
+    if (MODE == MODE_DGRAD && stage != nullptr && refq != nullptr) {
+        // Staged data-gradient tile whose ReLU-mask row (BN bf16 values of the layer input) the caller fetched into registers
+        // while the main loop ran: nothing in this loop waits for global memory.  Fully unrolled, so that refq[] stays in
+        // registers.
+        const uint32_t row_s = smem_u32(stage) + (uint32_t)row * 128u;
+        const uint32_t sw = (uint32_t)(row & 7);
+        constexpr int SLOTS = MaskRow<BN>::SLOTS;
+        uint4* rq = const_cast<uint4*>(refq);
+        const uint4* rp = (const uint4*)(p.ref + row_off + n0);
+#pragma unroll
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t v[2][16];
+            tmem_ld16(taddr + c0, v[0]);     // warp-collective; two loads per wait
+            tmem_ld16(taddr + c0 + 16, v[1]);
+            tmem_ld_wait();
+            if (n0 + c0 >= n_hi) continue;            // (uniform: whole 64-column slabs)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = c0 + 16 * h;
+                const uint4 r0 = rq[(c / 8) % SLOTS], r1 = rq[(c / 8 + 1) % SLOTS];
+                if (c + 128 < BN) {                       // refill the two slots for the chunk 128 columns on
+                    const bool more = row_ok && n0 + c + 128 < n_hi;
+                    rq[(c / 8) % SLOTS] = more ? __ldg(rp + (c + 128) / 8) : make_uint4(0u, 0u, 0u, 0u);
+                    rq[(c / 8 + 1) % SLOTS] = more ? __ldg(rp + (c + 128) / 8 + 1) : make_uint4(0u, 0u, 0u, 0u);
+                }
+                const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
+                const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
+                float f[16];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    f[j] = (__bfloat162float(rb0[j]) > 0.f) ? __uint_as_float(v[h][j]) : 0.f;
+                    f[8 + j] = (__bfloat162float(rb1[j]) > 0.f) ? __uint_as_float(v[h][8 + j]) : 0.f;
+                }
+                stage_chunk16(f, row_s, sw, c);
+            }
+        }
+        return;
+    }
     if (MODE != MODE_WGRAD && stage != nullptr) {
         // Staged bf16 tile for the TMA store (the planner only selects it for unsplit bf16 outputs whose columns end on
         // 64-column slabs): every decision is taken once, outside the loop -- an epilogue warp runs alone on its
@@ -287,45 +356,41 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
         const uint32_t row_s = smem_u32(stage) + (uint32_t)row * 128u;
         const uint32_t sw = (uint32_t)(row & 7);
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 16) {
-            uint32_t v[16];
-            tmem_ld16(taddr + c0, v);     // warp-collective
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t v[2][16];
+            tmem_ld16(taddr + c0, v[0]);     // warp-collective; two loads per wait
+            tmem_ld16(taddr + c0 + 16, v[1]);
             tmem_ld_wait();
             if (n0 + c0 >= n_hi) continue;            // (uniform: whole 64-column slabs)
-            float f[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]);
-            if (bias_act) {
+            for (int h = 0; h < 2; ++h) {
+                const int c = c0 + 16 * h;
+                float f[16];
 #pragma unroll
-                for (int j4 = 0; j4 < 4; ++j4) {
-                    float b0, b1, b2, b3;
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(bias_s + (uint32_t)(c0 + 4 * j4) * 4u));
-                    f[4 * j4] += b0; f[4 * j4 + 1] += b1; f[4 * j4 + 2] += b2; f[4 * j4 + 3] += b3;
+                for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[h][j]);
+                if (bias_act) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 4; ++j4) {
+                        float b0, b1, b2, b3;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(bias_s + (uint32_t)(c + 4 * j4) * 4u));
+                        f[4 * j4] += b0; f[4 * j4 + 1] += b1; f[4 * j4 + 2] += b2; f[4 * j4 + 3] += b3;
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) f[j] = f[j] > 0.f ? f[j] : 0.f;     // (NaN -> 0, as the reference path)
+                    }
+                } else if (refrow != nullptr) {
+                    const uint4 r0 = *(const uint4*)(refrow + c), r1 = *(const uint4*)(refrow + c + 8);
+                    const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
+                    const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
+                        if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
+                    }
                 }
-                if (relu) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) f[j] = f[j] > 0.f ? f[j] : 0.f;     // (NaN -> 0, as the reference path)
-                }
-            } else if (refrow != nullptr) {
-                const uint4 r0 = *(const uint4*)(refrow + c0), r1 = *(const uint4*)(refrow + c0 + 8);
-                const __nv_bfloat16* rb0 = (const __nv_bfloat16*)&r0;
-                const __nv_bfloat16* rb1 = (const __nv_bfloat16*)&r1;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (!(__bfloat162float(rb0[j]) > 0.f)) f[j] = 0.f;
-                    if (!(__bfloat162float(rb1[j]) > 0.f)) f[8 + j] = 0.f;
-                }
+                stage_chunk16(f, row_s, sw, c);
             }
-            uint32_t pk[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
-                pk[j] = *(uint32_t*)&t;
-            }
-            // 64-column slabs of 128 rows x 128 bytes in the 128-byte swizzle of the tensor map
-            const uint32_t slab = row_s + (uint32_t)(c0 >> 6) * 16384u, j0 = (uint32_t)(c0 & 63) >> 3;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((j0 ^ sw) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + (((j0 + 1u) ^ sw) << 4)), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
         }
         return;
     }
@@ -831,6 +896,8 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             }
             if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
         }
+        uint4 refq[MODE == MODE_DGRAD ? MaskRow<BN>::SLOTS : 1];
+        const bool have_refq = prefetch_mask_row<MODE, BN>(p, row_ok, row_off, n0, n_hi, refq);
         if (lane == 0 && ok) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok && lane == 0) { *abort_flag = 1; atomicMax(p.status, (uint32_t)DEV_TIMEOUT_EPI); }
@@ -858,7 +925,7 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             // (the operand ring is idle once the accumulator is complete: its first bytes stage the output tile)
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, (MODE != MODE_WGRAD && p.tma_out) ? smem : nullptr, row);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, (MODE != MODE_WGRAD && p.tma_out) ? smem : nullptr, row, have_refq ? refq : nullptr);
             if (MODE != MODE_WGRAD && p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
@@ -1157,6 +1224,8 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const bool row_ok = w < p.W && h < p.H && n < p.N;
         const size_t row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
         bool ok = true;
+        uint4 refq[MODE == MODE_DGRAD ? MaskRow<BN>::SLOTS : 1];
+        const bool have_refq = prefetch_mask_row<MODE, BN>(p, row_ok, row_off, n0, n_hi, refq);
         if (lane == 0) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) {
@@ -1166,7 +1235,7 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             // (the rings are idle once the accumulator is complete: their first bytes stage the output tile)
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, p.tma_out ? smem : nullptr, row);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, p.tma_out ? smem : nullptr, row, have_refq ? refq : nullptr);
             if (p.tma_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
@@ -1439,6 +1508,8 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
                 // (the previous tile's epilogue has passed its last barrier: nobody still reads the old bias values)
                 for (int c = t128; c < BN; c += 128) s_bias[c] = (n0 + c < n_hi) ? p.bias[n0 + c] : 0.f;
             }
+            uint4 refq[MODE == MODE_DGRAD ? MaskRow<BN>::SLOTS : 1];
+            const bool have_refq = prefetch_mask_row<MODE, BN>(p, row_ok, row_off, n0, n_hi, refq);
             if (lane == 0) ok = mbar_wait(&acc_full[buf], (uint32_t)((i >> 1) & 1));
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) {
@@ -1449,7 +1520,7 @@ umma_halo_persist_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_
             SB_TLOG(t128 == 0 && i < 4, 8 + 2 * i, clock64());      // accumulator of tile i complete
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, 0, s_bias, stage_out, row);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, 0, s_bias, stage_out, row, have_refq ? refq : nullptr);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_before();
             epi_bar_sync();                       // the tile is staged and every warp has finished reading the accumulator
@@ -1796,6 +1867,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             row_ok = w < p.W && h < p.H && n < p.N;
             row_off = (((size_t)n * p.H + h) * p.W + w) * p.ldc;
         }
+        uint4 refq[MODE == MODE_DGRAD ? MaskRow<BN>::SLOTS : 1];
+        const bool have_refq = prefetch_mask_row<MODE, BN>(p, row_ok, row_off, n0, n_hi, refq);
         if (lane == 0) ok = mbar_wait(acc_full, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) {
@@ -1804,7 +1877,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
             const bool staged_out = MODE != MODE_WGRAD && p.tma_out;
-            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, staged_out ? smem : nullptr, row);
+            store_row<MODE, BN>(p, taddr, row_ok, row_off, n0, n_hi, split, s_bias, staged_out ? smem : nullptr, row, have_refq ? refq : nullptr);
             if (staged_out) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
     }
