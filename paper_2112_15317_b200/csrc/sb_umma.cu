@@ -153,27 +153,33 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;"
 // as 16-byte chunks, chunk c at position c ^ (r & 7) of its 8-chunk group, which spreads a warp's stores over all banks
 // -- and is then swept row by row: half a warp takes one row's 256 contiguous bytes, so every global access of a warp
 // is two whole 256-byte runs.
+// With room for two slabs in the drained ring (two_bufs) consecutive slabs alternate between them, and one barrier per slab
+// is enough: whoever has passed the barrier of slab j has finished sweeping slab j - 1, whose buffer slab j + 1 reuses.
 template <int BN>
 __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32_t taddr, uint8_t* stage, int row, int m0, int m_hi,
-                                                      int n0, int n_hi, size_t tile_off, int slab_mult = 1)
+                                                      int n0, int n_hi, size_t tile_off, int slab_mult = 1, bool two_bufs = false)
 {
     const int t128 = threadIdx.x - 64, q = t128 >> 5, lane = t128 & 31;
     const int hl = lane & 15, sub = lane >> 4;
-    const uint32_t stage_s = smem_u32(stage);
+    const uint32_t stage_base = smem_u32(stage);
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 64) {
         if (n0 + c0 >= n_hi) break;                       // (uniform)
+        const uint32_t stage_s = stage_base + ((two_bufs && (c0 & 64)) ? 32768u : 0u);
 #pragma unroll
-        for (int cc = 0; cc < 64; cc += 16) {
-            uint32_t v[16];
-            tmem_ld16(taddr + c0 + cc, v);
+        for (int cc = 0; cc < 64; cc += 32) {
+            uint32_t v[2][16];
+            tmem_ld16(taddr + c0 + cc, v[0]);             // two loads per wait
+            tmem_ld16(taddr + c0 + cc + 16, v[1]);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t ch = (uint32_t)(cc / 4 + j);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_s + (uint32_t)row * 256u + ((ch ^ (uint32_t)(row & 7)) << 4)),
-                             "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
-            }
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t ch = (uint32_t)((cc + 16 * h) / 4 + j);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_s + (uint32_t)row * 256u + ((ch ^ (uint32_t)(row & 7)) << 4)),
+                                 "r"(v[h][4 * j]), "r"(v[h][4 * j + 1]), "r"(v[h][4 * j + 2]), "r"(v[h][4 * j + 3]) : "memory");
+                }
         }
         epi_bar_sync();
         const int col = n0 + c0 + 4 * hl;
@@ -188,7 +194,7 @@ __device__ __forceinline__ void wgrad_sweep_epilogue(const UmmaParams& p, uint32
                 *(float4*)((float*)p.out + off) = g;
             }
         }
-        epi_bar_sync();                                   // the slab may be overwritten
+        if (!two_bufs) epi_bar_sync();                    // the slab may be overwritten
     }
 }
 
@@ -915,10 +921,12 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     }
                 } else if (BN == 192 && p.hn_order)      // slab j = tap row j of filter column tap_fixed / 3: gradient columns (3 j + column) * Cin ..
                     wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
-                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)(tap_fixed / 3) * p.w_cols, 3);
+                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)(tap_fixed / 3) * p.w_cols, 3,
+                                             STAGES * C::STAGE_BYTES >= 65536);
                 else
                     wgrad_sweep_epilogue<BN>(p, taddr, smem, row, m0, m_hi, n0, n_hi,
-                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0);
+                                             (size_t)split * p.split_stride + (size_t)m0 * p.ldc + (size_t)tap_fixed * p.w_cols + n0, 1,
+                                             STAGES * C::STAGE_BYTES >= 65536);
             }
         } else if (ok) {
             SB_TLOG(threadIdx.x == 64, 4, clock64());      // accumulator complete
