@@ -160,8 +160,8 @@ sb_status sb_model_destroy(sb_model* m);
  *   x      : HOST array of R DEVICE pointers; x[r] = replica r's images [b,H,W,C] in the
  *            activation dtype (float or bfloat16), 16-byte aligned.
  *   labels : HOST array of R DEVICE pointers; labels[r] = int32 [b], values in [0, classes).
- * Row g = r*b + i of every FC-side tensor belongs to replica r (the paper's owner rule
- * "batch example index divided by B/K").  Computes the per-row and mean loss and the gradient
+ * Row g = r*b + i of every FC-side tensor belongs to replica r (the owner rule of the modulo layer:
+ * a batch row's index divided by the rows per worker) [Modulo Layer].  Computes the per-row and mean loss and the gradient
  * of the loss w.r.t. the logits.  The input buffers must stay valid until sb_backward has run.
  */
 sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* labels, void* stream);
@@ -175,13 +175,13 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
 sb_status sb_backward(sb_model* m, void* stream);
 
 /*
- * SGD with momentum on every parameter [Implementation: "SGD in mini-batches"]:
+ * SGD with momentum on every parameter [Implementation]:
  * v <- momentum*v + g ; w <- w - lr*v ; in SB_BF16 mode also refreshes the bf16 weight copies.
  */
 sb_status sb_sgd_step(sb_model* m, float lr, float momentum, void* stream);
 
 /*
- * One iteration in the modulo layer's own schedule [Modulo Layer: "The stateful scheduling for the K iterations"]:
+ * One iteration in the modulo layer's own schedule [Modulo Layer]:
  * the conv-side layers run forward once on all R*b rows; the FC stack then runs K sub-iterations, sub-iteration k
  * on the k-th slice of b/K examples of every replica (inside a sub-batch the row at position p belongs to replica
  * p / (b/K)); every row's loss gradient is (softmax - onehot)/(R*b), which for the FC parameters is the mean over

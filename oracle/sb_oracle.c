@@ -17,13 +17,13 @@
  *  - conv layers are replicated, FC layers are split 1/K by output column, ReLU follows the
  *    partitioned width [Design, Layer Partitioning, Listing 1];
  *  - convolution = 3x3 cross-correlation, stride 1, zero pad 1, one bias per output channel
- *    (the paper only says "kernel and output sizes"; Table 1 counts 9*Cin*Cout weights);
+ *    (the paper specifies a convolutional layer by its kernel and output sizes only; Table 1 counts 9*Cin*Cout weights);
  *  - pooling = 2x2 max, stride 2; ties resolved to the first maximum in scan order
  *    (0,0),(0,1),(1,0),(1,1);  ReLU'(0) = 0;
  *  - loss = log-softmax + negative log-likelihood, mean over the full batch [Listing 1,
  *    LOG_SOFTMAX case];
- *  - SGD with momentum in the Torch form v <- mu*v + g, w <- w - lr*v [Implementation: "SGD in
- *    mini-batches"; the constants come from the benchmark configuration].
+ *  - SGD with momentum in the Torch form v <- mu*v + g, w <- w - lr*v [Implementation; the constants come
+ *    from the benchmark configuration].
  */
 #include <math.h>
 #include <stddef.h>

@@ -85,7 +85,7 @@ sb_status walk(const sb_layer* layers, int32_t n, const sb_config* cfg, std::vec
             }
             flat = true;
             dimF = out;
-            dim = split ? (out + K - 1) / K : out;                       // "1/K size" (the widest shard when K does not divide out)
+            dim = split ? (out + K - 1) / K : out;                       // one K-th of the width (the widest shard when K does not divide out)
             push(SB_NODE_LAYER, i, split ? K : 1, dim, dimF);
         } else if (kind == SB_DROPOUT) {
             // one-to-one functional layer: adapts to the (partitioned) width of the layer below, dim and dimF pass through,
