@@ -407,13 +407,21 @@ __device__ __forceinline__ void store_row(const UmmaParams& p, uint32_t taddr, b
         float* dst = raw_partials ? p.part + (size_t)split * p.split_stride + row_off + n0 : (float*)p.out + row_off + n0;
         const bool vec = raw_partials ? ((p.n_total & 3) == 0 && (n0 & 3) == 0)
                                       : ((p.ldc & 3) == 0 && (n0 & 3) == 0 && ((((size_t)p.split_stride) & 3) == 0) && ((p.w_cols & 3) == 0 || MODE != MODE_WGRAD));
+        // (32-byte stores where the row allows: a thread writes a row of its own, so every store instruction of a warp
+        // touches 32 different lines, and a 16-byte store leaves half of its 32-byte sector to a second instruction)
+        const bool vec8 = vec && ((((uintptr_t)dst) & 31) == 0);
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 16) {
             uint32_t v[16];
             tmem_ld16(taddr + c0, v);     // warp-collective: executed by all lanes regardless of row_ok
             tmem_ld_wait();
             if (!row_ok || n0 + c0 >= n_hi) continue;
-            if (vec && n0 + c0 + 16 <= n_hi) {
+            if (vec8 && n0 + c0 + 16 <= n_hi) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c0 + 8 * j), "r"(v[8 * j]), "r"(v[8 * j + 1]),
+                                 "r"(v[8 * j + 2]), "r"(v[8 * j + 3]), "r"(v[8 * j + 4]), "r"(v[8 * j + 5]), "r"(v[8 * j + 6]), "r"(v[8 * j + 7]) : "memory");
+            } else if (vec && n0 + c0 + 16 <= n_hi) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
                     ((float4*)(dst + c0))[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
