@@ -100,6 +100,7 @@ struct sb_model {
     uint32_t* status = nullptr;
     uint32_t* drop_state = nullptr;   // dropout: {seed lo, seed hi, iteration, 0} (device words, kept between calls)
     int last_dropout = -1;            // index of the network's last dropout layer: its forward kernel is followed by the iteration bump
+    bool st_clean = false;     // the chain stream's last kernel belongs to the current forward / backward pass (it cannot have written weights)
     int pooled_by_conv = -1;   // index of the pool layer whose output the conv kernel just before it has already written (same forward call)
     // Set by the multi-stream backward pass while it enqueues the weight side of one conv layer: the layer's split
     // reduces then apply the update themselves (launch_reduce_sgd) once `ev` (the layer's input-gradient kernel, which
@@ -949,6 +950,28 @@ sb_status sb_model_destroy(sb_model* m)
     return SB_OK;
 }
 
+// One layer's kernels on the chain stream of a pass.  Once a kernel of the same pass precedes it on that stream, a tensor-core
+// forward / data-gradient kernel may fetch its weights before it waits for that predecessor (weights_first()): within a pass
+// nothing on the chain stream writes parameters -- updates run on other streams behind events, or after the pass.
+static sb_status chain_fwd(sb_model* m, int i, cudaStream_t st)
+{
+    weights_first() = m->st_clean ? 1 : 0;
+    const int64_t l0 = m->launches;
+    const sb_status s = forward_layer(m, i, st);
+    weights_first() = 0;
+    if (m->launches > l0) m->st_clean = true;
+    return s;
+}
+static sb_status chain_bwd(sb_model* m, int i, cudaStream_t st, int part)
+{
+    weights_first() = m->st_clean ? 1 : 0;
+    const int64_t l0 = m->launches;
+    const sb_status s = backward_layer(m, i, st, part);
+    weights_first() = 0;
+    if (m->launches > l0) m->st_clean = true;
+    return s;
+}
+
 sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void* const* x, const int32_t* const* labels, void* stream)
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
@@ -958,10 +981,12 @@ sb_status sb_forward_layers(sb_model* m, int32_t first, int32_t last, const void
         if (s != SB_OK) return s;
     }
     m->pooled_by_conv = -1;     // a pool layer run on its own (or first in the range) computes its output itself
+    m->st_clean = false;
     for (int i = first; i <= last; ++i) {
-        sb_status s = forward_layer(m, i, (cudaStream_t)stream);
+        sb_status s = chain_fwd(m, i, (cudaStream_t)stream);
         if (s != SB_OK) return s;
     }
+    m->st_clean = false;
     m->pooled_by_conv = -1;
     return SB_OK;
 }
@@ -970,10 +995,12 @@ sb_status sb_backward_layers(sb_model* m, int32_t last, int32_t first, void* str
 {
     if (!m) return fail(SB_ERR_INVALID_ARG, "null model");
     if (first < 0 || last >= m->n_layers || first > last) return fail(SB_ERR_INVALID_ARG, "bad layer range %d..%d", last, first);
+    m->st_clean = false;
     for (int i = last; i >= first; --i) {
-        sb_status s = backward_layer(m, i, (cudaStream_t)stream);
+        sb_status s = chain_bwd(m, i, (cudaStream_t)stream, SIDE_BOTH);
         if (s != SB_OK) return s;
     }
+    m->st_clean = false;
     return SB_OK;
 }
 
@@ -985,10 +1012,12 @@ sb_status sb_forward(sb_model* m, const void* const* x, const int32_t* const* la
     if (s != SB_OK) return s;
     m->launches = 0;
     m->pooled_by_conv = -1;
+    m->st_clean = false;
     for (int i = 0; i < m->n_layers; ++i) {
-        s = forward_layer(m, i, (cudaStream_t)stream);
+        s = chain_fwd(m, i, (cudaStream_t)stream);
         if (s != SB_OK) return s;
     }
+    m->st_clean = false;
     m->pooled_by_conv = -1;
     m->have_fwd = true;
     return SB_OK;
@@ -1018,6 +1047,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
     const bool two_streams = m->n_wstreams > 0 && !m->profiling && !m->debug_sync;
     const bool fuse = fuse_update && two_streams;
     if (updated) *updated = fuse;
+    m->st_clean = false;
     unsigned used_streams = 0;   // weight streams that received work in this pass (only those are joined)
     bool used_ustream = false;   // likewise the update stream
     for (int i = hi; i >= lo; --i) {
@@ -1046,7 +1076,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
                                             (fc_wgrad_update && l.kind != SB_CONV3X3_RELU && !l.narrow && umma_fc_wgrad_can_update(m, i)));
             sb_status s = SB_OK;
             if (in_reduce) {
-                s = backward_layer(m, i, st, SIDE_D);
+                s = chain_bwd(m, i, st, SIDE_D);
                 if (s != SB_OK) return s;
                 CU_TRY(cudaEventRecord(m->ev_dgrad[i], st));
                 m->fuse.on = true; m->fuse.lr = lr; m->fuse.mu = mu; m->fuse.ev = m->ev_dgrad[i]; m->fuse.waited = false; m->fuse.covered = 0;
@@ -1058,7 +1088,7 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
             } else {
                 s = weight_side(m, i, wst, classic);
                 if (s != SB_OK) return s;
-                s = backward_layer(m, i, st, SIDE_D);
+                s = chain_bwd(m, i, st, SIDE_D);
                 if (s != SB_OK) return s;
             }
             if (fuse) {
@@ -1078,10 +1108,11 @@ static sb_status backward_pass(sb_model* m, cudaStream_t st, bool fuse_update, f
                 }
             }
         } else {
-            sb_status s = backward_layer(m, i, st, SIDE_BOTH);
+            sb_status s = chain_bwd(m, i, st, SIDE_BOTH);
             if (s != SB_OK) return s;
         }
     }
+    m->st_clean = false;
     if (two_streams) {
         for (int k = 0; k < m->n_wstreams; ++k) {
             if (!(used_streams & (1u << k))) continue;
@@ -1136,8 +1167,9 @@ static sb_status modulo_step_direct(sb_model* m, const void* const* x, const int
     m->pooled_by_conv = -1;
     const int ff = m->first_fc, K = m->cfg.K, R = m->cfg.R, b = m->cfg.batch_per_replica, Bk = m->B / K;
     const size_t D = (size_t)m->L[ff].in_f;
+    m->st_clean = false;
     for (int i = 0; i < ff; ++i) {
-        s = forward_layer(m, i, st);
+        s = chain_fwd(m, i, st);
         if (s != SB_OK) return s;
     }
     m->cur_layer = ff;
@@ -1150,8 +1182,10 @@ static sb_status modulo_step_direct(sb_model* m, const void* const* x, const int
         std::swap(m->L, m->mod_L[k]);
         m->B = Bk; m->sub_active = true; m->sub_row0 = k * Bk;
         s = SB_OK;
-        for (int i = ff; i < m->n_layers && s == SB_OK; ++i) s = forward_layer(m, i, st);
-        for (int i = m->n_layers - 1; i >= ff && s == SB_OK; --i) s = backward_layer(m, i, st, SIDE_BOTH);
+        m->st_clean = k == 0;     // (the modulo copy precedes the first sub-iteration; the FC update of the one before, every other)
+        for (int i = ff; i < m->n_layers && s == SB_OK; ++i) s = chain_fwd(m, i, st);
+        for (int i = m->n_layers - 1; i >= ff && s == SB_OK; --i) s = chain_bwd(m, i, st, SIDE_BOTH);
+        m->st_clean = false;
         m->B = m->full_B; m->sub_active = false; m->sub_row0 = 0;
         std::swap(m->L, m->mod_L[k]);
         if (s != SB_OK) return s;

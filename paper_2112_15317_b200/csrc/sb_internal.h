@@ -40,6 +40,9 @@ inline double tune(const char* name, double dflt)
 }
 // (the calling thread can switch the attribute off for the launches it enqueues next: pdl_classic() = 1 ... = 0)
 inline int& pdl_classic() { static thread_local int off = 0; return off; }
+// Set by the calling thread around a launch whose predecessor in the stream is known not to have written the layer's weights
+// (a kernel of the same forward or backward pass): the tensor-core kernel may then fetch weights before it waits for it.
+inline int& weights_first() { static thread_local int on = 0; return on; }
 inline bool pdl_enabled()
 {
     static const bool on = [] { const char* e = getenv("SB_PDL"); return !(e && e[0] == '0'); }();

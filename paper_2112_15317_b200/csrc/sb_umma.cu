@@ -67,6 +67,8 @@ struct UmmaParams {
     // epilogue
     int epi, relu, out_f32;
     int tma_out;          // FWD/DGRAD, bf16 output, no split: the tile is staged in shared memory and written by TMA stores (map C)
+    int w_first;          // FWD/DGRAD: the first ring of WEIGHT loads is issued before the wait for the predecessor kernel (the host sets it
+                          // only when that kernel cannot have written the weights), the activation loads after it
     void* out;            // FWD/DGRAD: [pixels][ldc] bf16 (or float when out_f32); WGRAD: float partial sums
     __nv_bfloat16* pool_out;   // FWD with tma_out, conv layer followed by a 2x2 max-pool: the pool layer's output [N][H/2][W/2][ldc]
     uint8_t* pool_idx;         // ... and its argmax bytes (dh*2+dw), same shape; nullptr = no fused pool
@@ -667,8 +669,10 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     int ld_s = 0;
     uint32_t ld_off = 0;
     const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(&full[0]);
-    auto issue_loads = [&](uint32_t el) {
+    // part 0: both operands; FWD / DGRAD only: 1 = the barrier's byte count and the weight operand, 2 = the activation operand
+    auto issue_loads = [&](uint32_t el, int part = 0) {
         const uint32_t sa = smem0 + ld_off, sb = sa + A_STAGE_BYTES, bar = full0 + 8u * (uint32_t)ld_s;
+        if (part != 2)
         mbar_expect_tx_el(bar, (MODE == MODE_WGRAD && BN == 192 && p.hn_order ? (uint32_t)A_STAGE_BYTES + col_box_bytes : (uint32_t)C::STAGE_BYTES) -
                                    (a_boxes == 2 ? 0u : 8192u), el);
         if (MODE == MODE_WGRAD) {
@@ -706,8 +710,9 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             int dr = 0, ds = 0;
             if (p.ntaps == 9) { const int r3 = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0); dr = r3 - 1; ds = tap - 3 * r3 - 1; }
             if (MODE == MODE_DGRAD) { dr = -dr; ds = -ds; }
-            tma_load_4d_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
-            if (MODE == MODE_FWD) {
+            if (part != 1) tma_load_4d_el(&mapA, sa, bar, kc * 64, pw0 + ds, ph0 + dr, pn0, el);
+            if (part == 2) {
+            } else if (MODE == MODE_FWD) {
                 tma_load_4d_el(&mapB, sb, bar, tap * p.w_cols + kc * 64, n0, 0, 0, el);
             } else {
 #pragma unroll
@@ -735,14 +740,20 @@ umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             SB_TLOG(true, 8, clock64());    // barriers initialised
         }
         __syncwarp();
+        prod_el = elect_one() ? 1u : 0u;
+        if (MODE != MODE_WGRAD && p.w_first) {
+            // the weights are not the predecessor kernel's output: their first ring-full is on its way while that kernel finishes
+            const int a0 = ld_a, b0 = ld_b;
+            for (int it = 0; it < preloaded; ++it) issue_loads(prod_el, 1);
+            ld_a = a0; ld_b = b0; ld_s = 0; ld_off = 0;
+        }
         pdl_wait();
         pdl_trigger();
         SB_TRACE_STAMP(trace_a);
         SB_TLOG(lane == 0, 9, clock64());    // predecessor kernel complete
         // The first ring-full of loads needs nothing but the barriers just initialised: start them now, so that
         // their latency overlaps the TMEM allocation and the rest of the set-up.
-        prod_el = elect_one() ? 1u : 0u;
-        for (int it = 0; it < preloaded; ++it) issue_loads(prod_el);
+        for (int it = 0; it < preloaded; ++it) issue_loads(prod_el, (MODE != MODE_WGRAD && p.w_first) ? 2 : 0);
         SB_TLOG(lane == 0, 10, clock64());   // first ring of loads issued
     }
     if (warp == 1) {
@@ -1106,14 +1117,27 @@ umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncwarp();
+        prod_el = elect_one() ? 1u : 0u;
+        if (p.w_first) {
+            // the weights are not the predecessor kernel's output: the first groups' weight tiles are on their way while that
+            // kernel finishes; the activation halos follow once it has
+            const int kc0 = ld_kc, dsi0 = ld_dsi;
+            for (int g = 0; g < preloaded; ++g) {
+#pragma unroll
+                for (int j = 0; j < 3; ++j) issue_weights(j, prod_el);
+                next_group();
+            }
+            ld_kc = kc0; ld_dsi = dsi0;
+        }
         pdl_wait();
         pdl_trigger();
         SB_TRACE_STAMP(trace_a);
-        prod_el = elect_one() ? 1u : 0u;
         for (int g = 0; g < preloaded; ++g) {
             issue_halo(prod_el);
+            if (!p.w_first) {
 #pragma unroll
-            for (int j = 0; j < 3; ++j) issue_weights(j, prod_el);
+                for (int j = 0; j < 3; ++j) issue_weights(j, prod_el);
+            }
             next_group();
         }
     }
@@ -2219,6 +2243,8 @@ static sb_status launch_op(const UmmaOp& op, cudaStream_t st, int64_t* launches 
     pp.dbg_skip = (int)tune("SB_HALO_SKIP", 0);
 #endif
     if (pp.mode != MODE_WGRAD) {
+        static const bool w_first_on = tune("SB_W_FIRST", 1) != 0;
+        pp.w_first = (w_first_on && weights_first() && !b->pair && !b->persist) ? 1 : 0;
         pp.rcp_tiles_w = fast_rcp((uint32_t)pp.tiles_w);
         pp.rcp_tiles_wh = fast_rcp((uint32_t)(pp.tiles_w * pp.tiles_h));
         pp.rcp_bw = fast_rcp((uint32_t)pp.bw);
